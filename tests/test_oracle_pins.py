@@ -1,0 +1,501 @@
+"""Pins for the CPU oracle: every check here compares the oracle with something other than itself --
+published known-answer vectors, closed forms, library routines on special cases, brute-force
+enumeration on tiny inputs, and distributional tests of the two randomised procedures."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+from scipy.special import logsumexp
+from scipy.stats import chisquare
+
+import oracle
+from helpers import (logit, node_path, np_logits, np_softmax, sigmoid, tiny_problem, tiny_z_path,
+                     z_rows_for_tree)
+from paper_2609_22098_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_values.txt")
+
+
+def golden():
+    out = {}
+    for line in open(GOLDEN):
+        line = line.split("#")[0].strip()
+        if line:
+            k, v = line.split("=")
+            vals = [float(x) for x in v.split()]
+            out[k.strip()] = vals[0] if len(vals) == 1 else vals
+    return out
+
+
+# ----------------------------------------------------------------------------------------------
+# Random numbers
+# ----------------------------------------------------------------------------------------------
+
+PHILOX_KAT = [  # known-answer vectors published with Philox4x32-10 (Random123 test suite)
+    ((0, 0, 0, 0), (0, 0), (0x6627E8D5, 0xE169C58D, 0xBC57AC4C, 0x9B00DBD8)),
+    ((0xFFFFFFFF,) * 4, (0xFFFFFFFF,) * 2, (0x408F276D, 0x41C83B0E, 0xA20BC7C6, 0x6D5451FD)),
+    ((0x243F6A88, 0x85A308D3, 0x13198A2E, 0x03707344), (0xA4093822, 0x299F31D0),
+     (0xD16CFE09, 0x94FDCCEB, 0x5001E420, 0x24126EA1)),
+]
+
+
+@pytest.mark.parametrize("ctr,key,expect", PHILOX_KAT)
+def test_philox_known_answers(ctr, key, expect):
+    assert oracle.philox4x32_10(ctr, key) == expect
+
+
+def test_philox_matches_independent_torch_implementation():
+    # the input generator's Philox is a separate implementation (torch integer ops)
+    for i in range(50):
+        ctr = tuple((0x9E3779B9 * (i + 1) * (k + 3)) & 0xFFFFFFFF for k in range(4))
+        key = ((0x85EBCA6B * (i + 7)) & 0xFFFFFFFF, (0xC2B2AE35 * (i + 11)) & 0xFFFFFFFF)
+        t = [torch.tensor([c], dtype=torch.int64) for c in ctr]
+        got = tuple(int(x) for x in synth.philox4x32_10(*t, key[0], key[1]))
+        assert oracle.philox4x32_10(ctr, key) == got
+
+
+def test_stream_layout_and_uniform_range():
+    seed, req, h = 0x1234567890ABCDEF, 5, 0xDEADBEEFCAFEF00D
+    key = (seed & 0xFFFFFFFF, seed >> 32)
+    for v in (0, 1, 15, 16, 17, 151935):
+        coarse_w = oracle.philox4x32_10((v >> 4, h & 0xFFFFFFFF, h >> 32, req | (1 << 24)), key)
+        fine_w = oracle.philox4x32_10((v >> 2, h & 0xFFFFFFFF, h >> 32, req | (2 << 24)), key)
+        coarse = (coarse_w[(v & 15) >> 2] >> (8 * (v & 3))) & 0xFF
+        x = (coarse << 24) | (fine_w[v & 3] >> 8)
+        assert oracle.u_gumbel(seed, req, h, v) == (x + 0.5) / 2 ** 32
+    w = oracle.philox4x32_10((3, h & 0xFFFFFFFF, h >> 32, req | (3 << 24)), key)
+    assert oracle.u_accept(seed, req, h, 3) == (w[0] + 0.5) / 2 ** 32
+    w = oracle.philox4x32_10((0, h & 0xFFFFFFFF, h >> 32, req | (4 << 24)), key)
+    assert oracle.u_bonus(seed, req, h) == (w[0] + 0.5) / 2 ** 32
+    us = np.array([oracle.u_gumbel(7, 0, 0, v) for v in range(20000)])
+    assert us.min() > 0 and us.max() < 1
+    assert abs(us.mean() - 0.5) < 0.01 and abs(us.var() - 1 / 12) < 0.005
+
+
+def test_path_hash_is_order_free_and_distinct():
+    h1 = oracle.path_hash(oracle.path_hash(0, 5), 9)
+    h2 = oracle.path_hash(oracle.path_hash(0, 9), 5)
+    assert h1 != h2 and h1 == oracle.path_hash(oracle.path_hash(0, 5), 9)
+    # splitmix64 finaliser of (parent ^ (token+1)*golden), written out independently
+    def sm(x):
+        x = (x + 0x9E3779B97F4A7C15) & (2 ** 64 - 1)
+        x = ((x ^ (x >> 30)) * 0xBF58476D1CE4E5B9) & (2 ** 64 - 1)
+        x = ((x ^ (x >> 27)) * 0x94D049BB133111EB) & (2 ** 64 - 1)
+        return x ^ (x >> 31)
+    assert oracle.path_hash(0, 0) == sm(0x9E3779B97F4A7C15)
+    assert oracle.path_hash(12345, 77) == sm(12345 ^ ((78 * 0x9E3779B97F4A7C15) & (2 ** 64 - 1)))
+    assert len({oracle.path_hash(0, t) for t in range(5000)}) == 5000
+
+
+# ----------------------------------------------------------------------------------------------
+# Scoring (Eq. 1)
+# ----------------------------------------------------------------------------------------------
+
+def test_logits_match_library_matvec_and_orientation():
+    V, D, r = 50, 2, 7
+    U, A, W = tiny_problem(3, V, D, r)
+    o = oracle.Oracle(V, D, r, 4, 8)
+    got = o.logits(U[1], A[13], W)
+    np.testing.assert_allclose(got, np_logits(U[1], A[13], W), rtol=0, atol=1e-12)
+    # a transposed or mis-strided W would not survive a one-hot probe
+    a = np.zeros(r, np.float32); a[3] = 2.0
+    np.testing.assert_allclose(o.logits(np.zeros(V, np.float32), a, W), 2.0 * W[3].astype(np.float64), atol=1e-12)
+
+
+@pytest.mark.parametrize("T", [0.0, 0.7, 1.0, 1.3])
+def test_softmax_normalisation_and_logsumexp(T):
+    V, D, r, K = 1000, 2, 8, 4
+    U, A, W = tiny_problem(4, V, D, r, u_std=3.0)
+    o = oracle.Oracle(V, D, r, K, 8)
+    s = o.score_parent(U[0], A[17], W, T, seed=9, req=0, node_hash=0)
+    l = np_logits(U[0], A[17], W)
+    assert abs(np.exp(l - s["lse0"]).sum() - 1.0) < 1e-12
+    assert abs(s["lse0"] - logsumexp(l)) < 1e-12
+    if T > 0:
+        assert abs(np.exp(l / T - s["lseT"]).sum() - 1.0) < 1e-12
+        assert abs(s["lseT"] - logsumexp(l / T)) < 1e-12
+    order = sorted(range(V), key=lambda v: (-l[v], v))[:K]
+    assert list(s["top_tok"]) == order
+    np.testing.assert_allclose(s["top_logit"], l[order], atol=1e-12)
+
+
+def test_zero_head_reduces_to_plain_softmax_of_base_logits():
+    # marginal-tree special case: with A = 0 the conditional is softmax(U_d)
+    V, D, r = 200, 1, 4
+    U, A, W = tiny_problem(5, V, D, r)
+    o = oracle.Oracle(V, D, r, 3, 4)
+    s = o.score_parent(U[0], np.zeros(r, np.float32), W, 0.0, 1, 0, 0)
+    assert abs(s["lse0"] - logsumexp(U[0].astype(np.float64))) < 1e-12
+    assert s["top_tok"][0] == int(np.argmax(U[0]))
+
+
+def test_topk_ties_break_to_lowest_index():
+    V, r = 16, 2
+    U = np.zeros((1, V), np.float32); U[0, [3, 9, 12]] = 1.0
+    o = oracle.Oracle(V, 1, r, 4, 4)
+    s = o.score_parent(U[0], np.zeros(r, np.float32), np.zeros((r, V), np.float32), 0.0, 1, 0, 0)
+    assert list(s["top_tok"]) == [3, 9, 12, 0]
+
+
+def test_sampling_keys_follow_the_gumbel_definition():
+    V, D, r, K, T = 64, 1, 4, 5, 0.7
+    U, A, W = tiny_problem(6, V, D, r)
+    o = oracle.Oracle(V, D, r, K, 8)
+    seed, req, h = 77, 2, oracle.path_hash(0, 5)
+    s = o.score_parent(U[0], A[5], W, T, seed, req, h)
+    l = np_logits(U[0], A[5], W)
+    keys = np.array([l[v] / T - math.log(-math.log(oracle.u_gumbel(seed, req, h, v))) for v in range(V)])
+    order = sorted(range(V), key=lambda v: (-keys[v], v))[:K]
+    assert list(s["draw_tok"]) == order
+    assert len(set(s["draw_tok"])) == K                      # siblings never duplicate
+    np.testing.assert_allclose(s["draw_logit"], l[order], atol=1e-12)
+
+
+@pytest.mark.parametrize("T", [0.7, 1.3])
+def test_draw_order_has_the_law_of_sequential_renormalised_sampling(T):
+    """Eq. 2: the j-th sibling is drawn from q_T with earlier siblings removed and the rest
+    renormalised; so an ordered triple has probability prod_j q(x_j) / (1 - sum_{i<j} q(x_i))."""
+    V, D, r, K = 6, 1, 3, 3
+    U, A, W = tiny_problem(8, V, D, r)
+    o = oracle.Oracle(V, D, r, K, 8)
+    trials = 300000
+    hist = o.draw_order_trials(U[0], A[2], W, T, seed0=1, trials=trials)
+    q = np_softmax(np_logits(U[0], A[2], W), T)
+    obs, exp = [], []
+    for a in range(V):
+        for b in range(V):
+            for c in range(V):
+                if len({a, b, c}) < 3:
+                    assert hist[a, b, c] == 0
+                    continue
+                obs.append(hist[a, b, c])
+                exp.append(trials * q[a] * q[b] / (1 - q[a]) * q[c] / (1 - q[a] - q[b]))
+    assert abs(sum(exp) - trials) < 1e-6 * trials
+    assert chisquare(obs, exp).pvalue > 1e-3
+
+
+# ----------------------------------------------------------------------------------------------
+# Calibration (Eq. 3)
+# ----------------------------------------------------------------------------------------------
+
+def test_platt_closed_form_with_published_constants():
+    g = golden()
+    o = oracle.Oracle(8, 2, 2, 2, 4, calib_mode=0, platt_a=g["platt_a"], platt_b=g["platt_b"])
+    assert abs(o.calib(0, 0.0) - sigmoid(-0.46)) < 1e-15            # q0 = 1/2
+    assert abs(o.calib(0, 0.0) - 0.38698582386066) < 1e-12
+    for q in (0.01, 0.2, 0.5, 0.9, 0.999):
+        assert abs(o.calib(1, logit(q)) - sigmoid(0.67 * logit(q) - 0.46)) < 1e-14
+    # raw q0 over-estimates acceptance in the confident range: the fitted map shrinks it
+    assert o.calib(0, logit(0.9)) < 0.9
+
+
+def test_table_calibration_interpolates_and_is_monotone():
+    wl = synth.WORKLOADS["tiny"]
+    tab = synth.make_calibration_table(wl, 11, "platt").numpy().astype(np.float64)
+    o = oracle.Oracle(8, wl.D, 2, 2, 4, calib_mode=1, calib_table=tab)
+    knots = np.linspace(-10, 10, 16)
+    for d in range(wl.D):
+        assert np.all(np.diff(tab[d]) >= 0) and tab[d].min() > 0 and tab[d].max() <= 1
+        for i, t in enumerate(knots):
+            assert abs(o.calib(d, float(t)) - tab[d, i]) < 1e-12
+        mid = 0.5 * (knots[4] + knots[5])
+        assert abs(o.calib(d, float(mid)) - 0.5 * (tab[d, 4] + tab[d, 5])) < 1e-12
+        assert o.calib(d, -50.0) == tab[d, 0] and o.calib(d, 50.0) == tab[d, 15]
+        xs = np.linspace(-12, 12, 200)
+        ys = [o.calib(d, float(x)) for x in xs]
+        assert np.all(np.diff(ys) >= -1e-15)
+
+
+# ----------------------------------------------------------------------------------------------
+# Expansion (Algorithm 1)
+# ----------------------------------------------------------------------------------------------
+
+def platt(a=0.67, b=-0.46):
+    return lambda d, t: sigmoid(a * max(-30.0, min(30.0, t)) + b)
+
+
+def brute_force_slots(U, A, W, anchor, D, K, T, seed, req, calib):
+    """Every slot of the lazily generated K-ary slot forest, with the key it would be admitted
+    under, its child's survival and token path.  No heap: plain recursion."""
+    V = U.shape[1]
+    out = []
+
+    def rec(tokpath, rankpath, logS, parent_tok, d, h):
+        if d == D:
+            return
+        l = np_logits(U[d], A[parent_tok], W)
+        q = np_softmax(l)
+        top = sorted(range(V), key=lambda v: (-l[v], v))
+        if T == 0:
+            draws = top[:K]
+        else:
+            keys = [l[v] / T - math.log(-math.log(oracle.u_gumbel(seed, req, h, v))) for v in range(V)]
+            draws = sorted(range(V), key=lambda v: (-keys[v], v))[:K]
+        for j in range(min(K, V)):
+            unused = next(t for t in top if t not in draws[:j])
+            key = logS + math.log(calib(d, logit(q[unused])))
+            x = draws[j]
+            ls = logS + math.log(calib(d, logit(q[x])))
+            out.append(dict(key=key, depth=d + 1, ranks=rankpath + (j,), toks=tokpath + (x,), logS=ls))
+            rec(tokpath + (x,), rankpath + (j,), ls, x, d + 1, oracle.path_hash(h, x))
+
+    rec((), (), 0.0, anchor, 0, 0)
+    return out
+
+
+@pytest.mark.parametrize("T", [0.0, 1.0])
+@pytest.mark.parametrize("theta,N", [(0.0, 5), (0.0, 100), (0.05, 100), (0.2, 7), (0.5, 100)])
+def test_best_first_equals_sorted_enumeration_of_all_slots(T, theta, N):
+    V, D, r, K = 8, 3, 4, 3
+    for seed in range(6):
+        U, A, W = tiny_problem(100 + seed, V, D, r, u_std=2.0)
+        o = oracle.Oracle(V, D, r, K, N)
+        tree = o.expand_tree(U, A, W, anchor_tok=1, theta=theta, T=T, seed=seed, req=0)
+        slots = brute_force_slots(U, A, W, 1, D, K, T, seed, 0, platt())
+        slots.sort(key=lambda s: (-s["key"], s["depth"], s["ranks"]))
+        keep = [s for s in slots if theta == 0 or s["key"] >= math.log(theta)][:N]
+        n = tree["n"]
+        assert n == len(keep)
+        got = {node_path(tree, i): i for i in range(n)}
+        assert set(got) == {s["toks"] for s in keep}
+        if theta == 0.0:
+            assert n == min(N, len(slots))                   # theta = 0 is the fixed budget
+        for rank, s in enumerate(keep):
+            i = got[s["toks"]]
+            assert tree["pop_rank"][i] == rank               # heap pops in sorted order
+            assert abs(tree["logkey"][i] - s["key"]) < 1e-10
+            assert abs(tree["logS"][i] - s["logS"]) < 1e-10
+        pops = sorted(range(n), key=lambda i: tree["pop_rank"][i])
+        keys = [tree["logkey"][i] for i in pops]
+        assert all(keys[i] >= keys[i + 1] - 1e-15 for i in range(n - 1))
+        if len(keep) < len(slots) and n < N:                 # stopped by the price, not by the cap
+            assert slots[len(keep)]["key"] < math.log(theta)
+
+
+def test_survival_is_product_of_edge_estimates_and_structure_invariants():
+    V, D, r, K, N = 40, 4, 5, 3, 20
+    U, A, W = tiny_problem(21, V, D, r, u_std=2.5)
+    tab = synth.make_calibration_table(synth.WORKLOADS["tiny"], 5, "fit").numpy().astype(np.float64)
+    o = oracle.Oracle(V, D, r, K, N, calib_mode=1, calib_table=tab)
+    for T in (0.0, 0.8):
+        tree = o.expand_tree(U, A, W, anchor_tok=7, theta=0.02, T=T, seed=3, req=1)
+        n = tree["n"]
+        assert 0 < n <= N
+        knots = np.linspace(-10, 10, 16)
+        for i in range(n):
+            # walk up and multiply independently recomputed edge estimates
+            ls, j = 0.0, i
+            while j >= 0:
+                p = int(tree["parent"][j])
+                ptok = 7 if p < 0 else int(tree["tok"][p])
+                d = int(tree["depth"][j]) - 1
+                q = np_softmax(np_logits(U[d], A[ptok], W))[int(tree["tok"][j])]
+                ls += math.log(np.interp(logit(q), knots, tab[d]))
+                j = p
+            assert abs(ls - tree["logS"][i]) < 1e-10
+            p = int(tree["parent"][i])
+            ptok = 7 if p < 0 else int(tree["tok"][p])
+            l = np_logits(U[tree["depth"][i] - 1], A[ptok], W)
+            assert abs(tree["q0"][i] - np_softmax(l)[tree["tok"][i]]) < 1e-12
+            want = math.log(np_softmax(l, T)[tree["tok"][i]]) if T > 0 else math.log(tree["q0"][i])
+            assert abs(tree["logqT"][i] - want) < 1e-10
+        # canonical order, caps, masks, hashes
+        for i in range(n):
+            p, d = int(tree["parent"][i]), int(tree["depth"][i])
+            assert 1 <= d <= D and p < i
+            assert d == (1 if p < 0 else tree["depth"][p] + 1)
+            assert tree["node_hash"][i + 1] == oracle.path_hash(int(tree["node_hash"][p + 1]), int(tree["tok"][i]))
+            m = int(tree["mask"][i, 0])
+            assert m == ((int(tree["mask"][p, 0]) if p >= 0 else 0) | (1 << i))
+            assert bin(m).count("1") == d                    # a row sees exactly its root path
+            if i:
+                a = (tree["depth"][i - 1], tree["parent"][i - 1], tree["sib_rank"][i - 1])
+                b = (tree["depth"][i], tree["parent"][i], tree["sib_rank"][i])
+                assert a < b
+        for v in range(-1, n):
+            sibs = sorted(int(tree["sib_rank"][i]) for i in range(n) if tree["parent"][i] == v)
+            assert sibs == list(range(len(sibs))) and len(sibs) <= K
+            toks = [int(tree["tok"][i]) for i in range(n) if tree["parent"][i] == v]
+            assert len(set(toks)) == len(toks)
+        assert sorted(tree["pop_rank"][:n]) == list(range(n))
+
+
+def test_linear_tree_reproduces_the_chain_token_for_token():
+    V, D, r = 300, 5, 6
+    U, A, W = tiny_problem(31, V, D, r, u_std=2.0)
+    chain, x = [], 11
+    for d in range(D):                                        # chain decoder: x_k = argmax(U_k + B(x_{k-1}))
+        x = int(np.argmax(np_logits(U[d], A[x], W)))
+        chain.append(x)
+    o = oracle.Oracle(V, D, r, 1, D)
+    t1 = o.expand_tree(U, A, W, 11, theta=0.0, T=0.0, seed=1, req=0)
+    assert t1["n"] == D and list(t1["tok"][:D]) == chain and list(t1["parent"][:D]) == [-1, 0, 1, 2, 3]
+    o2 = oracle.Oracle(V, D, r, 4, 32)                        # theta >= 1: the chain member of the ladder
+    t2 = o2.expand_tree(U, A, W, 11, theta=1.0, T=0.0, seed=1, req=0)
+    assert t2["n"] == D and list(t2["tok"][:D]) == chain
+    t3 = o2.expand_tree(U, A, W, 11, theta=2.5, T=1.0, seed=1, req=0)
+    assert t3["n"] == D and list(t3["depth"][:D]) == [1, 2, 3, 4, 5] and set(t3["sib_rank"][:D]) == {0}
+
+
+def test_calibrator_is_fed_the_untempered_conditional():
+    # tree priorities at T>0 must come from q0; feeding q_T would change logS
+    V, D, r, K = 30, 2, 4, 2
+    U, A, W = tiny_problem(41, V, D, r, u_std=2.0)
+    o = oracle.Oracle(V, D, r, K, 6)
+    tree = o.expand_tree(U, A, W, 3, theta=0.0, T=0.5, seed=5, req=0)
+    i = 0
+    l = np_logits(U[0], A[3], W)
+    q0 = np_softmax(l)[tree["tok"][i]]
+    qT = np_softmax(l, 0.5)[tree["tok"][i]]
+    assert abs(tree["logS"][i] - math.log(sigmoid(0.67 * logit(q0) - 0.46))) < 1e-10
+    assert abs(tree["logS"][i] - math.log(sigmoid(0.67 * logit(qT) - 0.46))) > 1e-3
+
+
+# ----------------------------------------------------------------------------------------------
+# Verification
+# ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("seed", range(8))
+def test_greedy_verification_equals_brute_force_greedy_target_path(seed):
+    V, D, r, K, N = 8, 3, 4, 3, 14
+    U, A, W = tiny_problem(200 + seed, V, D, r, u_std=1.0)
+    Zp = tiny_z_path(300 + seed, U, A, W, D, sigma=0.5, anchor=2)
+    o = oracle.Oracle(V, D, r, K, N)
+    tree = o.expand_tree(U, A, W, 2, theta=0.0, T=0.0, seed=seed, req=0)
+    Z = z_rows_for_tree(tree, Zp, V)
+    res = o.verify_tree(U, A, W, Z, 2, tree, T=0.0, seed=seed, req=0, want_edge_stat=True)
+    # greedy target decoding: follow argmax of the target row while that token is in the tree
+    paths = {node_path(tree, i): i for i in range(tree["n"])}
+    path, toks = (), []
+    from helpers import path_row
+    while True:
+        g = int(np.argmax(Zp[path_row(path, V)]))
+        if path + (g,) in paths:
+            path += (g,)
+            toks.append(g)
+        else:
+            bonus = g
+            break
+    assert res["acc_len"] == len(toks) and list(res["acc_tok"][:len(toks)]) == toks and res["bonus"] == bonus
+    assert [node_path(tree, i) for i in res["acc_node"][:len(toks)]] == [tuple(toks[:k + 1]) for k in range(len(toks))]
+    for i in range(tree["n"]):
+        p = int(tree["parent"][i])
+        g = int(np.argmax(Z[p + 1]))
+        assert res["edge_stat"][i] == (1.0 if tree["tok"][i] == g else 0.0)
+
+
+def test_target_equal_to_drafter_accepts_every_first_sibling():
+    V, D, r, K, N = 8, 3, 4, 3, 14
+    U, A, W = tiny_problem(51, V, D, r)
+    Zp = tiny_z_path(52, U, A, W, D, sigma=0.0, anchor=4)
+    o = oracle.Oracle(V, D, r, K, N)
+    for seed in range(5):
+        tree = o.expand_tree(U, A, W, 4, theta=0.0, T=0.9, seed=seed, req=0)
+        Z = z_rows_for_tree(tree, Zp, V)
+        for cf in (False, True):
+            res = o.verify_tree(U, A, W, Z, 4, tree, 0.9, seed, 0, closed_form=cf, want_edge_stat=True)
+            cur, want = -1, []
+            while True:
+                nxt = [i for i in range(tree["n"]) if tree["parent"][i] == cur and tree["sib_rank"][i] == 0]
+                if not nxt:
+                    break
+                cur = nxt[0]
+                want.append(cur)
+            assert res["acc_len"] == len(want) and list(res["acc_node"][:len(want)]) == want
+            np.testing.assert_allclose(res["edge_stat"][:tree["n"]], 1.0, atol=1e-6)
+
+
+def test_vector_residuals_agree_with_scalar_sequence_form():
+    V, D, r, K, N = 12, 3, 4, 4, 20
+    agree = total = 0
+    for seed in range(300):
+        U, A, W = tiny_problem(400 + seed % 7, V, D, r, u_std=1.2)
+        Zp_rows = None
+        o = oracle.Oracle(V, D, r, K, N)
+        tree = o.expand_tree(U, A, W, 1, theta=0.01, T=1.0, seed=seed, req=0)
+        rng = np.random.RandomState(seed)
+        Z = (rng.randn(tree["n"] + 1, V) * 1.5).astype(np.float32)
+        a = o.verify_tree(U, A, W, Z, 1, tree, 1.0, seed, 0, closed_form=False)
+        b = o.verify_tree(U, A, W, Z, 1, tree, 1.0, seed, 0, closed_form=True)
+        total += 1
+        if (a["flags"] | b["flags"]) & (oracle.FLAG_NEAR_ACCEPT | oracle.FLAG_NEAR_CDF | oracle.FLAG_ZERO_MASS):
+            continue
+        assert a["acc_len"] == b["acc_len"] and a["bonus"] == b["bonus"]
+        assert list(a["acc_tok"]) == list(b["acc_tok"])
+        agree += 1
+    assert agree > 0.95 * total
+
+
+def _lossless_case(V, D, r, K, N, theta, T, trials, seed, mode=0, closed_form=False):
+    U, A, W = tiny_problem(seed, V, D, r, u_std=1.5)
+    Zp = tiny_z_path(seed + 1, U, A, W, D, sigma=1.0, anchor=3)
+    o = oracle.Oracle(V, D, r, K, N)
+    h1, h2, mean_nodes, mean_acc = o.lossless_trials(U, A, W, Zp, 3, theta, T, seed0=10_000, trials=trials,
+                                                     mode=mode, closed_form=closed_form)
+    p_root = np_softmax(Zp[0].astype(np.float64), T)
+    return h1, h2, p_root, Zp, mean_nodes, mean_acc
+
+
+def test_losslessness_chi_square_one_million_trials():
+    """Proposition 1: the first committed token is distributed as the target softmax, and given an
+    accepted first token the next committed token follows the target conditional at that node."""
+    V = 8
+    trials = 1_000_000
+    h1, h2, p_root, Zp, mean_nodes, mean_acc = _lossless_case(V, 3, 4, 4, 12, 0.05, 1.0, trials, seed=60)
+    assert h1.sum() == trials and mean_nodes > 3 and mean_acc > 0.3
+    assert chisquare(h1, p_root * trials).pvalue > 1e-3
+    tv = 0.5 * np.abs(h1 / trials - p_root).sum()
+    assert tv < 2e-3
+    from helpers import path_row
+    checked = 0
+    for x1 in range(V):
+        nrow = int(h2[x1].sum())
+        if nrow < 5000:
+            continue
+        p2 = np_softmax(Zp[path_row((x1,), V)].astype(np.float64), 1.0)
+        assert chisquare(h2[x1], p2 * nrow).pvalue > 1e-4
+        checked += 1
+    assert checked >= 2
+
+
+@pytest.mark.parametrize("K,theta,T", [(1, 0.0, 1.0), (2, 0.1, 0.7), (4, 0.0, 1.3), (4, 0.3, 1.0), (2, 1.5, 1.0)])
+def test_losslessness_across_sibling_counts_prices_and_temperatures(K, theta, T):
+    trials = 200_000
+    for cf in (False, True):
+        h1, h2, p_root, Zp, _, _ = _lossless_case(8, 3, 4, K, 12, theta, T, trials, seed=70 + K, closed_form=cf)
+        assert chisquare(h1, p_root * trials).pvalue > 1e-3
+
+
+def test_biased_control_fails_the_same_test():
+    """Power check: deterministic top-k children with the same rejection walk are biased."""
+    trials = 200_000
+    h1, _, p_root, _, _, _ = _lossless_case(8, 3, 4, 4, 12, 0.05, 1.0, trials, seed=60, mode=1)
+    assert chisquare(h1, p_root * trials).pvalue < 1e-12
+    assert 0.5 * np.abs(h1 / trials - p_root).sum() > 0.02
+
+
+def test_single_sibling_is_textbook_speculative_sampling():
+    """K = 1 at the root: accept x ~ q with probability min(1, p/q), else resample from
+    norm(max(p - q, 0)).  The committed-token law computed in closed form must be p."""
+    V, D, r = 8, 1, 4
+    U, A, W = tiny_problem(80, V, D, r)
+    Zp = tiny_z_path(81, U, A, W, D, sigma=1.0, anchor=0)
+    o = oracle.Oracle(V, D, r, 1, 1)
+    T = 1.0
+    p = np_softmax(Zp[0].astype(np.float64), T)
+    q = np_softmax(np_logits(U[0], A[0], W), T)
+    acc = np.minimum(p, q)                                    # P(draw x and accept it)
+    trials = 200_000
+    h1, h2, *_ = o.lossless_trials(U, A, W, Zp, 0, 0.0, T, 5, trials)
+    accepted_first = h2.sum(axis=1)                           # first token came from an accepted edge
+    assert chisquare(accepted_first, acc / acc.sum() * accepted_first.sum()).pvalue > 1e-3
+    assert abs(accepted_first.sum() / trials - acc.sum()) < 4 * math.sqrt(acc.sum() * (1 - acc.sum()) / trials)
+    assert chisquare(h1, p * trials).pvalue > 1e-3
+
+
+def test_cost_model_matches_the_papers_flop_figure():
+    g = golden()
+    flops = 2 * g["cost_rank"] * g["cost_vocab"]              # one |V| x r mat-vec per scored node
+    assert abs(flops / 1e6 - g["cost_mflop_per_node"]) < 3
