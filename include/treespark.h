@@ -1,0 +1,161 @@
+/*
+ * treespark.h -- C ABI of the B200 (sm_100a) hot path of one TreeSpark decoding round.
+ *
+ * Three calls follow the round as the paper states it (Section 3.2, Algorithm 1, Section 3.3):
+ *   ts_score_parents  parent-conditioned scoring with sibling candidates   (Eq. 1, Eq. 2)
+ *   ts_expand_tree    calibrated best-first expansion with the theta stop  (Algorithm 1, Eq. 3, Section 3.5)
+ *   ts_verify_tree    lossless verification, accepted path + bonus token   (Section 3.2 item 3, Section 3.3)
+ *
+ * Conventions
+ *   - Every function returns a status (TS_OK = 0, negative = error).  No exception crosses the ABI.
+ *   - Pointers marked DEVICE are CUDA device addresses owned by the caller and must be 16-byte
+ *     aligned; pointers marked HOST are host addresses read during the call only.
+ *   - The three hot calls allocate nothing, never synchronise with the host and enqueue all work on
+ *     the caller's stream (a cudaStream_t passed as void*).  Scratch memory is the caller's
+ *     workspace of at least ts_workspace_bytes() bytes; its contents are undefined between calls.
+ *   - Problems found on the device (NaN logits, zero residual mass, a barrier that timed out) are
+ *     reported per request in the caller's status[] array, readable after the stream has drained.
+ *   - Indices: draft depth d of a PARENT is 0-based (the root has depth 0); its children live at
+ *     depth d+1 in 1..D and are scored with base-logit row U[request][d].
+ *   - Random numbers: Philox4x32-10, key = seed, counter = (index, path hash of the node (64 bit),
+ *     request | stream << 24).  Stream 1/2 give the top byte / low 24 bits of the sampling uniform
+ *     of token v (sixteen resp. four tokens per call), stream 3 the accept uniform of sibling j,
+ *     stream 4 the bonus uniform.  hash(root) = 0, hash(child) = splitmix64(hash(parent) XOR
+ *     (token+1) * 0x9E3779B97F4A7C15).  A draw therefore depends on the node's token path only,
+ *     never on the order in which nodes were materialised.
+ */
+#ifndef TREESPARK_H
+#define TREESPARK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TS_OK 0
+#define TS_ERR_INVALID (-1)      /* bad argument (NULL or misaligned pointer, size out of range) */
+#define TS_ERR_UNSUPPORTED (-2)  /* configuration outside what the kernels are built for */
+#define TS_ERR_WORKSPACE (-3)    /* workspace smaller than ts_workspace_bytes() */
+#define TS_ERR_CUDA (-4)         /* a CUDA runtime call failed; see ts_last_error_string() */
+#define TS_ERR_TIMEOUT (-5)      /* device status: a bounded device-side wait ran out */
+#define TS_ERR_OVERFLOW (-6)     /* device status: an internal list overflowed */
+#define TS_ERR_NUMERIC (-7)      /* device status: NaN logits or a residual without mass */
+
+#define TS_DTYPE_F32 0
+#define TS_DTYPE_BF16 1
+
+#define TS_KMAX 16       /* largest sibling cap K */
+#define TS_DMAX 16       /* largest block depth D */
+#define TS_CALIB_KNOTS 16
+
+/* per-request flag bits written by ts_verify_tree */
+#define TS_FLAG_ZERO_MASS 64u  /* a residual target lost all mass; the previous residual was kept */
+
+typedef struct ts_ctx ts_ctx;
+
+typedef struct {
+  int32_t V, D, r, K, Nmax;  /* vocabulary, block depth, Markov rank, sibling cap, node cap (root excluded) */
+  int32_t max_batch;         /* largest B any call will pass */
+  int32_t dt_U, dt_A, dt_W, dt_Z; /* TS_DTYPE_*; this build needs all four equal */
+  int32_t calib_mode;        /* 0 = Platt scalars (Eq. 3), 1 = per-depth table of TS_CALIB_KNOTS knots */
+  float platt_a, platt_b;    /* Eq. 3; the paper's fit is 0.67, -0.46 */
+  float calib_lo, calib_hi;  /* knot range in logit(q0), knots uniform, linear interpolation, clamped */
+  const float* calib_table;  /* HOST [D][16], non-decreasing in (0,1]; copied at create; NULL for mode 0 */
+} ts_config;
+
+/* Create / destroy a context on the current device.  Create copies the calibration table to the
+ * device (the only allocation the library ever makes).  Errors: TS_ERR_INVALID, TS_ERR_UNSUPPORTED
+ * (K > 16, D > 16, Nmax > 256, r > 128, mixed dtypes), TS_ERR_CUDA. */
+int32_t ts_create(const ts_config* cfg, ts_ctx** out);
+int32_t ts_destroy(ts_ctx* ctx);
+
+/* Bytes of workspace the hot calls need for a batch of `batch` requests (<= max_batch). */
+size_t ts_workspace_bytes(const ts_ctx* ctx, int32_t batch);
+
+/* Human-readable description of the last error returned on this thread. */
+const char* ts_last_error_string(void);
+
+/*
+ * Score P parents (Eq. 1; Section 3.2 item 1; Section 5.6 cost per scored node).
+ * For parent i = (request parent_req[i], depth parent_depth[i] in [0,D), token parent_token[i]):
+ *   l = U[req][depth][:] + A[token][:] . W          (never written to memory)
+ *   lse0[i] = log sum exp(l),  lseT[i] = log sum exp(l / T)   (lseT = lse0 when T == 0)
+ *   top_*  [i][K]: the K largest logits, value descending, ties to the lowest token
+ *   draw_* [i][K]: T > 0: the K without-replacement draws from softmax(l/T) in draw order (Eq. 2),
+ *                  realised as the K largest keys l_v/T - log(-log u_v); T == 0: a copy of top_*.
+ * Layout: U DEVICE [B][D][V], A DEVICE [V][r], W DEVICE [r][V], all row-major in the context's
+ * dtype.  parent_* DEVICE [P]; parent_hash = path hash of the parent node.  Outputs DEVICE.
+ * P <= max_batch * Nmax.  Entries beyond the vocabulary size (K > V) hold token -1.
+ */
+int32_t ts_score_parents(ts_ctx* ctx, const void* U, const void* A, const void* W,
+                         int32_t P, const int32_t* parent_req, const int32_t* parent_depth,
+                         const int32_t* parent_token, const uint64_t* parent_hash,
+                         float T, uint64_t seed,
+                         float* lse0, float* lseT,
+                         int32_t* top_tok, float* top_logit,
+                         int32_t* draw_tok, float* draw_logit,
+                         void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Build the draft trees of B requests (Algorithm 1 with the stop rule of Section 3.5).
+ * Slots are admitted in non-increasing order of the candidate survival S(v) * p_hat(best unused
+ * token | v) while fewer than Nmax nodes exist and that survival is >= theta[b]; the child token is
+ * the best unused token (T == 0) or the next without-replacement draw (T > 0); S(child) = S(v) *
+ * p_hat(child | v) with p_hat the calibrated estimate of Eq. 3 fed with the untempered q0.
+ * theta[b] >= 1 selects the chain member of the price ladder (Section 4): one child per node,
+ * exactly D nodes.  theta[b] == 0 is the fixed budget Nmax.
+ *
+ * Outputs (all DEVICE), nodes in canonical order: depth ascending, then parent's index, then
+ * sibling rank.  Arrays are [B][Nmax] unless noted; entries >= n_nodes[b] are undefined.
+ *   n_nodes [B]; tok; parent (-1 = root); depth (1..D); sib_rank (0-based draw order);
+ *   logS = log survival; q0 = q0(token | parent); logqT = log q_T(token | parent) (log q0 at T == 0);
+ *   logkey = log of the slot key the node was admitted under; pop_rank = best-first admission order;
+ *   node_hash [B][Nmax+1] (slot 0 = root); node_lseT [B][Nmax+1] = log-normaliser of q_T(.|node)
+ *   for every node that was scored, NaN otherwise (slot 0 = root);
+ *   mask [B][Nmax][ceil(Nmax/64)]: ancestor bitmask, bit i of row i set, root implicit (the tree
+ *   attention mask of Section 3.2 item 3; position id = depth);
+ *   n_scored [B] = parents scored for the request; status [B].
+ * logkey, pop_rank, node_lseT, n_scored may be NULL.
+ */
+int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, const void* W,
+                       int32_t B, const int32_t* anchor_tok, const float* theta,
+                       float T, uint64_t seed,
+                       int32_t* n_nodes, int32_t* tok, int32_t* parent, int32_t* depth,
+                       int32_t* sib_rank, float* logS, float* q0, float* logqT,
+                       float* logkey, int32_t* pop_rank,
+                       uint64_t* node_hash, float* node_lseT, uint64_t* mask,
+                       int32_t* n_scored, int32_t* status,
+                       void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Verify the trees against target logits (Section 3.2 item 3; Section 3.3).
+ * Z DEVICE [rows][V] in dt_Z: request b owns rows z_row_off[b] .. z_row_off[b] + n_nodes[b];
+ * its first row is the root, row 1+i is node i.  z_row_off DEVICE int64 [B+1].
+ * T == 0: walk from the root to the child whose token equals argmax of the current row (ties to
+ *   the lowest token) until none matches; the bonus token is that argmax.
+ * T > 0: at a visited node the siblings are tested in draw order; sibling j is accepted with
+ *   probability min(1, p_j(x) / q_j(x)), p_1 = softmax(Z[row]/T), q_j = q_T with earlier siblings
+ *   removed and renormalised; after a rejection p_{j+1} = norm(max(p_j - q_j, 0)).  When no sibling
+ *   is accepted the bonus token is drawn from the current residual by inverse CDF in token order.
+ *   The proposal is recomputed from U, A, W; no per-node vocabulary vector is stored.
+ *   logqT and node_lseT (from ts_expand_tree) are required when T > 0.
+ * Outputs DEVICE: acc_len [B] in [0,D]; acc_node, acc_tok [B][D]; bonus_tok [B];
+ *   edge_stat [B][Nmax] or NULL: T == 0 -> 1/0 "token equals the parent's target argmax" for every
+ *   edge, T > 0 -> min(1, p(x)/q_T(x)) for every edge; flags [B]; status [B].
+ */
+int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, const void* W,
+                       const void* Z, const int64_t* z_row_off, int32_t B,
+                       const int32_t* anchor_tok, const int32_t* n_nodes, const int32_t* tok,
+                       const int32_t* parent, const int32_t* depth, const int32_t* sib_rank,
+                       const uint64_t* node_hash, const float* logqT, const float* node_lseT,
+                       float T, uint64_t seed,
+                       int32_t* acc_len, int32_t* acc_node, int32_t* acc_tok, int32_t* bonus_tok,
+                       float* edge_stat, uint32_t* flags, int32_t* status,
+                       void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TREESPARK_H */

@@ -1,0 +1,178 @@
+"""Thin ctypes binding over the TreeSpark C ABI (``include/treespark.h``).
+
+Argument marshalling only: every step of the path runs in the library's kernels.  torch provides
+device memory and the current stream.  The compiled library must exist beside this file; a missing
+library is an error (there is no CPU fallback).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtreespark.so")
+
+TS_OK = 0
+DTYPE_F32, DTYPE_BF16 = 0, 1
+KNOTS = 16
+
+EXPORTS = ("ts_create", "ts_destroy", "ts_workspace_bytes", "ts_last_error_string",
+           "ts_score_parents", "ts_expand_tree", "ts_verify_tree")
+
+
+class TsConfig(C.Structure):
+    _fields_ = [("V", C.c_int32), ("D", C.c_int32), ("r", C.c_int32), ("K", C.c_int32), ("Nmax", C.c_int32),
+                ("max_batch", C.c_int32), ("dt_U", C.c_int32), ("dt_A", C.c_int32), ("dt_W", C.c_int32),
+                ("dt_Z", C.c_int32), ("calib_mode", C.c_int32), ("platt_a", C.c_float), ("platt_b", C.c_float),
+                ("calib_lo", C.c_float), ("calib_hi", C.c_float), ("calib_table", C.POINTER(C.c_float))]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Load the compiled library; raises if it has not been built (run ``python -m paper_2609_22098_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with paper_2609_22098_b200.build.build(); "
+                               "there is no fallback path")
+        L = C.CDLL(LIB_PATH)
+        L.ts_last_error_string.restype = C.c_char_p
+        L.ts_workspace_bytes.restype = C.c_size_t
+        L.ts_workspace_bytes.argtypes = [C.c_void_p, C.c_int32]
+        L.ts_create.argtypes = [C.POINTER(TsConfig), C.POINTER(C.c_void_p)]
+        L.ts_destroy.argtypes = [C.c_void_p]
+        vp, i32, f32, u64, sz = C.c_void_p, C.c_int32, C.c_float, C.c_uint64, C.c_size_t
+        L.ts_score_parents.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, f32, u64] + [vp] * 6 + [vp, sz, vp]
+        L.ts_expand_tree.argtypes = [vp, vp, vp, vp, i32, vp, vp, f32, u64] + [vp] * 15 + [vp, sz, vp]
+        L.ts_verify_tree.argtypes = [vp, vp, vp, vp, vp, vp, i32] + [vp] * 9 + [f32, u64] + [vp] * 7 + [vp, sz, vp]
+        for n in ("ts_create", "ts_destroy", "ts_score_parents", "ts_expand_tree", "ts_verify_tree"):
+            getattr(L, n).restype = C.c_int32
+        _lib = L
+    return _lib
+
+
+class TreeSparkError(RuntimeError):
+    pass
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class TreeSpark:
+    """A library context for one configuration plus its caller-owned workspace."""
+
+    def __init__(self, V, D, r, K, Nmax, max_batch, dtype=torch.bfloat16, calib_mode=0, platt_a=0.67,
+                 platt_b=-0.46, calib_lo=-10.0, calib_hi=10.0, calib_table=None, device="cuda"):
+        self.lib = load_library()
+        self.V, self.D, self.r, self.K, self.Nmax, self.max_batch = V, D, r, K, Nmax, max_batch
+        self.dtype = dtype
+        self.device = torch.device(device)
+        self.words = (Nmax + 63) // 64
+        dt = DTYPE_BF16 if dtype == torch.bfloat16 else DTYPE_F32
+        table_arr = None
+        if calib_mode == 1:
+            flat = [float(x) for x in torch.as_tensor(calib_table, dtype=torch.float32).reshape(-1).tolist()]
+            assert len(flat) == D * KNOTS
+            table_arr = (C.c_float * len(flat))(*flat)
+        cfg = TsConfig(V, D, r, K, Nmax, max_batch, dt, dt, dt, dt, calib_mode, platt_a, platt_b, calib_lo, calib_hi,
+                       C.cast(table_arr, C.POINTER(C.c_float)) if table_arr is not None else None)
+        self._ctx = C.c_void_p()
+        with torch.cuda.device(self.device):
+            self._check(self.lib.ts_create(C.byref(cfg), C.byref(self._ctx)))
+        self.ws_bytes = int(self.lib.ts_workspace_bytes(self._ctx, max_batch))
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=self.device)
+
+    def close(self):
+        if getattr(self, "_ctx", None):
+            self.lib.ts_destroy(self._ctx)
+            self._ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, code: int):
+        if code != TS_OK:
+            raise TreeSparkError(f"status {code}: {self.lib.ts_last_error_string().decode()}")
+
+    # -- output buffers (caller-owned; allocate once, reuse across rounds) -------------------------
+    def alloc_score_outputs(self, P: int) -> Dict[str, torch.Tensor]:
+        d, K = self.device, self.K
+        return dict(lse0=torch.empty(P, dtype=torch.float32, device=d), lseT=torch.empty(P, dtype=torch.float32, device=d),
+                    top_tok=torch.empty(P, K, dtype=torch.int32, device=d), top_logit=torch.empty(P, K, dtype=torch.float32, device=d),
+                    draw_tok=torch.empty(P, K, dtype=torch.int32, device=d), draw_logit=torch.empty(P, K, dtype=torch.float32, device=d))
+
+    def alloc_tree(self, B: int) -> Dict[str, torch.Tensor]:
+        d, N = self.device, self.Nmax
+        i32 = lambda *s: torch.zeros(*s, dtype=torch.int32, device=d)
+        f32 = lambda *s: torch.zeros(*s, dtype=torch.float32, device=d)
+        return dict(n_nodes=i32(B), tok=i32(B, N), parent=i32(B, N), depth=i32(B, N), sib_rank=i32(B, N),
+                    logS=f32(B, N), q0=f32(B, N), logqT=f32(B, N), logkey=f32(B, N), pop_rank=i32(B, N),
+                    node_hash=torch.zeros(B, N + 1, dtype=torch.int64, device=d), node_lseT=f32(B, N + 1),
+                    mask=torch.zeros(B, N, self.words, dtype=torch.int64, device=d), n_scored=i32(B), status=i32(B))
+
+    def alloc_verdict(self, B: int) -> Dict[str, torch.Tensor]:
+        d = self.device
+        i32 = lambda *s: torch.zeros(*s, dtype=torch.int32, device=d)
+        return dict(acc_len=i32(B), acc_node=i32(B, self.D), acc_tok=i32(B, self.D), bonus_tok=i32(B),
+                    edge_stat=torch.zeros(B, self.Nmax, dtype=torch.float32, device=d), flags=i32(B), status=i32(B))
+
+    # -- the three calls -------------------------------------------------------------------------
+    def score_parents(self, U, A, W, parent_req, parent_depth, parent_token, parent_hash, T, seed, out=None):
+        P = int(parent_req.numel())
+        out = out or self.alloc_score_outputs(P)
+        self._check(self.lib.ts_score_parents(self._ctx, _ptr(U), _ptr(A), _ptr(W), P, _ptr(parent_req),
+                                              _ptr(parent_depth), _ptr(parent_token), _ptr(parent_hash),
+                                              float(T), int(seed), _ptr(out["lse0"]), _ptr(out["lseT"]),
+                                              _ptr(out["top_tok"]), _ptr(out["top_logit"]), _ptr(out["draw_tok"]),
+                                              _ptr(out["draw_logit"]), _ptr(self.ws), self.ws_bytes, _stream()))
+        return out
+
+    def expand_tree(self, U, A, W, anchor_tok, theta, T, seed, out=None):
+        B = int(anchor_tok.numel())
+        t = out or self.alloc_tree(B)
+        self._check(self.lib.ts_expand_tree(self._ctx, _ptr(U), _ptr(A), _ptr(W), B, _ptr(anchor_tok), _ptr(theta),
+                                            float(T), int(seed), _ptr(t["n_nodes"]), _ptr(t["tok"]), _ptr(t["parent"]),
+                                            _ptr(t["depth"]), _ptr(t["sib_rank"]), _ptr(t["logS"]), _ptr(t["q0"]),
+                                            _ptr(t["logqT"]), _ptr(t["logkey"]), _ptr(t["pop_rank"]),
+                                            _ptr(t["node_hash"]), _ptr(t["node_lseT"]), _ptr(t["mask"]),
+                                            _ptr(t["n_scored"]), _ptr(t["status"]), _ptr(self.ws), self.ws_bytes,
+                                            _stream()))
+        return t
+
+    def verify_tree(self, U, A, W, Z, z_row_off, anchor_tok, tree, T, seed, out=None, edge_stat=True):
+        B = int(anchor_tok.numel())
+        v = out or self.alloc_verdict(B)
+        self._check(self.lib.ts_verify_tree(self._ctx, _ptr(U), _ptr(A), _ptr(W), _ptr(Z), _ptr(z_row_off), B,
+                                            _ptr(anchor_tok), _ptr(tree["n_nodes"]), _ptr(tree["tok"]),
+                                            _ptr(tree["parent"]), _ptr(tree["depth"]), _ptr(tree["sib_rank"]),
+                                            _ptr(tree["node_hash"]), _ptr(tree["logqT"]), _ptr(tree["node_lseT"]),
+                                            float(T), int(seed), _ptr(v["acc_len"]), _ptr(v["acc_node"]),
+                                            _ptr(v["acc_tok"]), _ptr(v["bonus_tok"]),
+                                            _ptr(v["edge_stat"]) if edge_stat else None, _ptr(v["flags"]),
+                                            _ptr(v["status"]), _ptr(self.ws), self.ws_bytes, _stream()))
+        return v
+
+
+def ts_score_parents(ctx: TreeSpark, *args, **kw):
+    return ctx.score_parents(*args, **kw)
+
+
+def ts_expand_tree(ctx: TreeSpark, *args, **kw):
+    return ctx.expand_tree(*args, **kw)
+
+
+def ts_verify_tree(ctx: TreeSpark, *args, **kw):
+    return ctx.verify_tree(*args, **kw)

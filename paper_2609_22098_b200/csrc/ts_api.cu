@@ -1,0 +1,113 @@
+// Context management, workspace sizing and error strings of the TreeSpark C ABI.
+#include <stdio.h>
+#include <string.h>
+
+#include "ts_internal.h"
+
+namespace ts {
+
+static thread_local char g_err[512] = "no error";
+
+int32_t set_error(int32_t code, const char* msg) {
+  snprintf(g_err, sizeof(g_err), "%s", msg);
+  return code;
+}
+
+int32_t set_cuda_error(const char* where, cudaError_t e) {
+  snprintf(g_err, sizeof(g_err), "%s: CUDA error %d (%s)", where, (int)e, cudaGetErrorString(e));
+  return TS_ERR_CUDA;
+}
+
+// Vocabulary tiling of the scoring kernel: the W tile [r][TV] stays in shared memory next to the
+// per-thread head rows [r][threads] and the noise-bound table; the tile count is a whole number of
+// waves over the SMs.
+static bool choose_tile(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
+  const size_t es = c.dt_W == TS_DTYPE_BF16 ? 2 : 4;
+  const size_t fixed = (size_t)c.r * SCORE_THREADS * 4 + 256 * 4;
+  const size_t budget = (size_t)max_smem > fixed + 1024 ? (size_t)max_smem - fixed - 1024 : 0;
+  int tv_max = (int)(budget / ((size_t)c.r * es) / 64) * 64;
+  if (tv_max < 64) return false;
+  if (tv_max > 4096) tv_max = 4096;
+  const int min_tiles = (c.V + tv_max - 1) / tv_max;
+  const int waves = (min_tiles + num_sms - 1) / num_sms;
+  const int want = waves * num_sms;
+  int tv = ((c.V + want - 1) / want + 63) / 64 * 64;
+  if (tv > tv_max) tv = tv_max;
+  out->TV = tv;
+  out->ntiles = (c.V + tv - 1) / tv;
+  out->smem = (size_t)c.r * tv * es + fixed;
+  return out->ntiles <= 32 * 16;
+}
+
+}  // namespace ts
+
+using namespace ts;
+
+extern "C" const char* ts_last_error_string(void) { return g_err; }
+
+extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
+  if (!cfg || !out) return set_error(TS_ERR_INVALID, "ts_create: null argument");
+  *out = nullptr;
+  if (cfg->V < 1 || cfg->D < 1 || cfg->r < 1 || cfg->K < 1 || cfg->Nmax < 1 || cfg->max_batch < 1)
+    return set_error(TS_ERR_INVALID, "ts_create: sizes must be positive");
+  if (cfg->K > TS_KMAX || cfg->D > TS_DMAX || cfg->Nmax > 256 || cfg->r > 128 || cfg->max_batch > 4096 ||
+      cfg->V > (1 << 24))
+    return set_error(TS_ERR_UNSUPPORTED, "ts_create: K<=16, D<=16, Nmax<=256, r<=128, batch<=4096, V<=2^24 required");
+  if (cfg->dt_U != cfg->dt_A || cfg->dt_U != cfg->dt_W || cfg->dt_U != cfg->dt_Z ||
+      (cfg->dt_U != TS_DTYPE_F32 && cfg->dt_U != TS_DTYPE_BF16))
+    return set_error(TS_ERR_UNSUPPORTED, "ts_create: U, A, W, Z must share one dtype (f32 or bf16)");
+  if (cfg->calib_mode != 0 && cfg->calib_mode != 1) return set_error(TS_ERR_INVALID, "ts_create: calib_mode");
+  if (cfg->calib_mode == 1) {
+    if (!cfg->calib_table || !(cfg->calib_hi > cfg->calib_lo))
+      return set_error(TS_ERR_INVALID, "ts_create: table mode needs calib_table and calib_hi > calib_lo");
+    for (int d = 0; d < cfg->D; ++d)
+      for (int i = 0; i < TS_CALIB_KNOTS; ++i) {
+        const float y = cfg->calib_table[d * TS_CALIB_KNOTS + i];
+        if (!(y > 0.f && y <= 1.f) || (i && y < cfg->calib_table[d * TS_CALIB_KNOTS + i - 1]))
+          return set_error(TS_ERR_INVALID, "ts_create: calibration table must be non-decreasing in (0,1]");
+      }
+  }
+  ts_ctx* ctx = new ts_ctx();
+  ctx->cfg = *cfg;
+  ctx->cfg.calib_table = nullptr;
+  ctx->d_table = nullptr;
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  cudaDeviceProp prop;
+  if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, ctx->device);
+  if (e != cudaSuccess) { delete ctx; return set_cuda_error("ts_create", e); }
+  ctx->num_sms = prop.multiProcessorCount;
+  ctx->max_smem = (int)prop.sharedMemPerBlockOptin;
+  if (!choose_tile(ctx->cfg, ctx->num_sms, ctx->max_smem, &ctx->tile)) {
+    delete ctx;
+    return set_error(TS_ERR_UNSUPPORTED, "ts_create: no vocabulary tiling fits shared memory");
+  }
+  ctx->vt_TV = ((cfg->V + ctx->num_sms - 1) / ctx->num_sms + 63) / 64 * 64;
+  ctx->vt_n = (cfg->V + ctx->vt_TV - 1) / ctx->vt_TV;
+  if (cfg->calib_mode == 1) {
+    const size_t bytes = (size_t)cfg->D * TS_CALIB_KNOTS * sizeof(float);
+    e = cudaMalloc(&ctx->d_table, bytes);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->d_table, cfg->calib_table, bytes, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { cudaFree(ctx->d_table); delete ctx; return set_cuda_error("ts_create", e); }
+  }
+  ctx->calib.mode = cfg->calib_mode;
+  ctx->calib.a = cfg->platt_a; ctx->calib.b = cfg->platt_b;
+  ctx->calib.lo = cfg->calib_lo; ctx->calib.hi = cfg->calib_hi;
+  ctx->calib.table = ctx->d_table;
+  e = score_setup(ctx);
+  if (e == cudaSuccess) e = verify_setup(ctx);
+  if (e != cudaSuccess) { cudaFree(ctx->d_table); delete ctx; return set_cuda_error("ts_create", e); }
+  *out = ctx;
+  return TS_OK;
+}
+
+extern "C" int32_t ts_destroy(ts_ctx* ctx) {
+  if (!ctx) return TS_OK;
+  if (ctx->d_table) cudaFree(ctx->d_table);
+  delete ctx;
+  return TS_OK;
+}
+
+extern "C" size_t ts_workspace_bytes(const ts_ctx* ctx, int32_t batch) {
+  if (!ctx || batch < 1 || batch > ctx->cfg.max_batch) return 0;
+  return make_layout(ctx, batch).total;
+}

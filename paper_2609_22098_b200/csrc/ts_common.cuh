@@ -1,0 +1,292 @@
+// Shared device/host pieces of the TreeSpark CUDA library: context, workspace layout, the
+// counter-based generator, input loads and the per-thread vocabulary scan.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/treespark.h"
+
+namespace ts {
+
+constexpr int KMAX = TS_KMAX;
+constexpr int DMAX = TS_DMAX;
+constexpr int KNOTS = TS_CALIB_KNOTS;
+constexpr int SCORE_THREADS = 128;   // one parent per thread; every thread scans the CTA's whole tile
+constexpr int CHUNK = 16;            // tokens per coarse generator call
+
+enum Stream : uint32_t { STREAM_GUMBEL_COARSE = 1, STREAM_GUMBEL_FINE = 2, STREAM_ACCEPT = 3, STREAM_BONUS = 4 };
+
+// ------------------------------------------------------------------------------------------------
+// Context (host) and the device-visible part of it
+// ------------------------------------------------------------------------------------------------
+struct DevCalib {
+  int mode;
+  double a, b, lo, hi;
+  const float* table;  // device [D][16]
+};
+
+struct TileCfg {
+  int TV;       // tokens per vocabulary tile (multiple of 64)
+  int ntiles;   // tiles covering V
+  size_t smem;  // dynamic shared memory of the scoring kernel
+};
+
+}  // namespace ts
+
+struct ts_ctx {
+  ts_config cfg;
+  float* d_table;
+  int device;
+  int num_sms;
+  int max_smem;
+  ts::TileCfg tile;
+  int vt_TV, vt_n;  // vocabulary ranges of the verification walk, one per CTA
+  ts::DevCalib calib;
+};
+
+namespace ts {
+
+// ------------------------------------------------------------------------------------------------
+// Workspace layout (bytes offsets into the caller's workspace), a function of (config, batch)
+// ------------------------------------------------------------------------------------------------
+struct WsLayout {
+  int B, N, K, Pcap, ntiles, words;
+  // scoring partials, [ntiles][...][Pcap]
+  size_t part_m, part_s0, part_sT, part_topv, part_topi, part_keyv, part_keyi, part_keyl;
+  // merged per-parent results of the level being expanded, [Pcap] / [Pcap][K]
+  size_t res_lse0, res_lseT, res_top_tok, res_top_logit, res_draw_tok, res_draw_logit;
+  // level parent lists (two, alternating) [Pcap]
+  size_t lst_req[2], lst_depth[2], lst_token[2], lst_hash[2], lst_slot[2];
+  size_t lvl_count;      // int[DMAX + 2]
+  // per-request pool, [B][N]
+  size_t pl_alive, pl_depth, pl_parent, pl_sib, pl_tok, pl_lidx, pl_new, pl_logkey, pl_logS, pl_q0, pl_logqT,
+      pl_lseT, pl_hash, pl_path;
+  size_t root_lseT;      // float[B]
+  size_t req_npar, req_base;  // int[B]: parents of the request in the current level list and their base index
+  size_t req_nscored;    // int[B]
+  // candidates of one level, [B][N*K]
+  size_t cd_valid, cd_parent, cd_sib, cd_tok, cd_logkey, cd_logS, cd_q0, cd_logqT, cd_rank;
+  // verification
+  size_t z_max, z_arg, z_lse;            // per Z row, [B*(N+1)]
+  size_t vf_state;                       // VerifyState[B]
+  size_t vf_part;                        // float[B][ntiles]
+  size_t vf_barrier;                     // unsigned[4]
+  size_t total;
+};
+
+__host__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct VerifyState {
+  int cur;        // current node (-1 = root)
+  int j;          // next sibling to test
+  int acc;        // accepted so far
+  int need;       // 0 none, 1 residual pass, 2 in-tile CDF scan, 3 finished
+  int nf;         // tested (frozen) siblings at the current node
+  int scan_tile;  // tile holding the bonus token
+  int row_node;   // node whose rows the pass reads
+  int result;     // token found by the range rescan
+  double C, Zj, Qused, target, before;
+  double passC;   // C of the requested pass
+  double partsC;  // C the stored range sums were computed for (-1 = none)
+  int fx[KMAX];
+  double fC[KMAX];
+  double fp[KMAX], fq[KMAX];
+};
+
+__host__ inline WsLayout make_layout(const ts_ctx* ctx, int B) {
+  WsLayout L{};
+  const ts_config& c = ctx->cfg;
+  L.B = B; L.N = c.Nmax; L.K = c.K; L.Pcap = B * c.Nmax > B ? B * c.Nmax : B; L.ntiles = ctx->tile.ntiles;
+  L.words = (c.Nmax + 63) / 64;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t P = (size_t)L.Pcap, nt = (size_t)L.ntiles, K = (size_t)c.K, N = (size_t)c.Nmax, b = (size_t)B;
+  L.part_m = take(nt * P * 4); L.part_s0 = take(nt * P * 4); L.part_sT = take(nt * P * 4);
+  L.part_topv = take(nt * K * P * 4); L.part_topi = take(nt * K * P * 4);
+  L.part_keyv = take(nt * K * P * 4); L.part_keyi = take(nt * K * P * 4); L.part_keyl = take(nt * K * P * 4);
+  L.res_lse0 = take(P * 4); L.res_lseT = take(P * 4);
+  L.res_top_tok = take(P * K * 4); L.res_top_logit = take(P * K * 4);
+  L.res_draw_tok = take(P * K * 4); L.res_draw_logit = take(P * K * 4);
+  for (int i = 0; i < 2; ++i) {
+    L.lst_req[i] = take(P * 4); L.lst_depth[i] = take(P * 4); L.lst_token[i] = take(P * 4);
+    L.lst_hash[i] = take(P * 8); L.lst_slot[i] = take(P * 4);
+  }
+  L.lvl_count = take((DMAX + 2) * 4);
+  L.pl_alive = take(b * N * 4); L.pl_depth = take(b * N * 4); L.pl_parent = take(b * N * 4);
+  L.pl_sib = take(b * N * 4); L.pl_tok = take(b * N * 4); L.pl_lidx = take(b * N * 4); L.pl_new = take(b * N * 4);
+  L.pl_logkey = take(b * N * 8); L.pl_logS = take(b * N * 8); L.pl_q0 = take(b * N * 4);
+  L.pl_logqT = take(b * N * 4); L.pl_lseT = take(b * N * 4); L.pl_hash = take(b * N * 8); L.pl_path = take(b * N * 8);
+  L.root_lseT = take(b * 4);
+  L.req_npar = take(b * 4); L.req_base = take(b * 4); L.req_nscored = take(b * 4);
+  const size_t NK = N * K;
+  L.cd_valid = take(b * NK * 4); L.cd_parent = take(b * NK * 4); L.cd_sib = take(b * NK * 4);
+  L.cd_tok = take(b * NK * 4); L.cd_logkey = take(b * NK * 8); L.cd_logS = take(b * NK * 8);
+  L.cd_q0 = take(b * NK * 4); L.cd_logqT = take(b * NK * 4); L.cd_rank = take(b * NK * 4);
+  const size_t rows = b * (N + 1);
+  L.z_max = take(rows * 4); L.z_arg = take(rows * 4); L.z_lse = take(rows * 4);
+  L.vf_state = take(b * sizeof(VerifyState));
+  L.vf_part = take(b * (size_t)ctx->vt_n * 4);
+  L.vf_barrier = take(64);
+  L.total = off;
+  return L;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Counter-based random numbers (Philox4x32-10) and the path hash
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                               uint32_t k1) {
+#pragma unroll
+  for (int i = 0; i < 10; ++i) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    c0 = hi1 ^ c1 ^ k0; c1 = lo1; c2 = hi0 ^ c3 ^ k1; c3 = lo0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+__device__ __forceinline__ uint4 stream_words(uint64_t seed, int req, uint64_t hash, uint32_t stream, uint32_t index) {
+  return philox4x32_10(index, (uint32_t)hash, (uint32_t)(hash >> 32), ((uint32_t)req & 0xFFFFFFu) | (stream << 24),
+                       (uint32_t)seed, (uint32_t)(seed >> 32));
+}
+
+__host__ __device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
+  uint64_t z = x + 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+__host__ __device__ __forceinline__ uint64_t path_hash(uint64_t parent_hash, int token) {
+  return splitmix64(parent_hash ^ (((uint64_t)(uint32_t)token + 1ull) * 0x9E3779B97F4A7C15ull));
+}
+
+__device__ __forceinline__ uint32_t word_of(const uint4& w, int i) {
+  return i == 0 ? w.x : (i == 1 ? w.y : (i == 2 ? w.z : w.w));
+}
+
+// uniform in (0,1) from a 32-bit word, in double (scalar uses only)
+__device__ __forceinline__ double u01(uint32_t x) { return ((double)x + 0.5) * (1.0 / 4294967296.0); }
+
+// Gumbel noise -log(-log u) for u = (X + 0.5) / 2^32, accurate in fp32 over the whole range: near
+// u = 1 the complement 1-u is formed exactly from the integer.
+__device__ __forceinline__ float gumbel_from_bits(uint32_t X) {
+  float a;
+  if (X >= 0x80000000u) {
+    const float t = ((float)(0xFFFFFFFFu - X) + 0.5f) * 2.3283064365386963e-10f;
+    a = -log1pf(-t);
+  } else {
+    const float u = ((float)X + 0.5f) * 2.3283064365386963e-10f;
+    a = -logf(u);
+  }
+  return -logf(a);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Input element loads
+// ------------------------------------------------------------------------------------------------
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static constexpr int VEC = 4;  // elements per 16-byte load
+  __device__ static __forceinline__ float to_f(float x) { return x; }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static constexpr int VEC = 8;
+  __device__ static __forceinline__ float to_f(__nv_bfloat16 x) { return __bfloat162float(x); }
+};
+
+// 16 consecutive elements starting at p (p 16-byte aligned when `vec`), as floats
+template <typename T>
+__device__ __forceinline__ void load16(const T* p, bool vec, int valid, float* out);
+
+template <>
+__device__ __forceinline__ void load16<float>(const float* p, bool vec, int valid, float* out) {
+  if (vec && valid >= 16) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(p) + i);
+      out[4 * i] = v.x; out[4 * i + 1] = v.y; out[4 * i + 2] = v.z; out[4 * i + 3] = v.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) out[i] = i < valid ? __ldg(p + i) : 0.f;
+  }
+}
+
+__device__ __forceinline__ void unpack_bf16x8(const uint4& v, float* out) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    out[2 * i] = __uint_as_float(w[i] << 16);
+    out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
+template <>
+__device__ __forceinline__ void load16<__nv_bfloat16>(const __nv_bfloat16* p, bool vec, int valid, float* out) {
+  if (vec && valid >= 16) {
+    const uint4 v0 = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint4 v1 = __ldg(reinterpret_cast<const uint4*>(p) + 1);
+    unpack_bf16x8(v0, out);
+    unpack_bf16x8(v1, out + 8);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) out[i] = i < valid ? __bfloat162float(p[i]) : 0.f;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Calibrated edge estimate (Eq. 3 or the per-depth table), scalar, in double
+// ------------------------------------------------------------------------------------------------
+// log p_hat for a child with logit lx under a parent with log-normaliser lse0 (depth d = parent depth)
+__device__ __forceinline__ double log_phat(const DevCalib& c, int d, double lx, double lse0) {
+  const double lq = lx - lse0;
+  double q = exp(lq);
+  if (q > 1.0 - 1e-12) q = 1.0 - 1e-12;
+  double t = lq - log1p(-q);
+  t = t > 30.0 ? 30.0 : (t < -30.0 ? -30.0 : t);
+  if (c.mode == 0) {
+    const double x = c.a * t + c.b;
+    return x >= 0 ? -log1p(exp(-x)) : x - log1p(exp(x));
+  }
+  const float* y = c.table + d * KNOTS;
+  const double pos = (t - c.lo) / (c.hi - c.lo) * (KNOTS - 1);
+  double v;
+  if (pos <= 0.0) v = y[0];
+  else if (pos >= KNOTS - 1) v = y[KNOTS - 1];
+  else {
+    const int i = (int)floor(pos);
+    const double f = pos - i;
+    v = (double)y[i] + f * ((double)y[i + 1] - (double)y[i]);
+  }
+  return log(v);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Bounded grid barrier for cooperative (co-resident) launches: counter + generation in global memory.
+// Returns false when the wait ran out; the caller must then stop using the barrier and exit.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned nblocks, unsigned& gen) {
+  __syncthreads();
+  bool ok = true;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned target = (gen + 1) * nblocks;
+    atomicAdd(&bar[0], 1u);
+    unsigned spins = 0;
+    while (*((volatile unsigned*)&bar[0]) < target) {
+      if (*((volatile unsigned*)&bar[1]) != 0u) { ok = false; break; }
+      if (++spins > (1u << 22)) { atomicExch(&bar[1], 1u); ok = false; break; }
+      __nanosleep(32);
+    }
+    __threadfence();
+  }
+  gen++;
+  ok = __syncthreads_and((int)ok) != 0;
+  return ok;
+}
+
+}  // namespace ts

@@ -1,0 +1,365 @@
+// Best-first tree expansion with the theta stop (Algorithm 1, Section 3.5), level-synchronous.
+//
+// Why levels give exactly the heap's result: a slot's key never exceeds the key of the slot that
+// created it (p_hat <= 1, p_hat monotone in q0, and a re-pushed sibling slot maximises over a smaller
+// set), so heap pops are non-increasing and the tree is "the first N slots in sorted key order among
+// those with key >= theta" of the lazily generated slot forest.  With ties broken by (depth, sibling
+// rank path) that order puts every slot after the slots it depends on.  Per request a pool of at most
+// N admitted slots is kept; at level d every pool node of depth d whose survival is >= theta is scored
+// in one batched pass, its slots are formed, and the pool is cut back to the best N.  A node outside
+// the pool at its own level can never enter the final tree, so nothing else needs scoring.
+#include <math.h>
+
+#include "ts_internal.h"
+
+namespace ts {
+
+struct ExpandArgs {
+  int B, D, K, N, V;
+  float T;
+  const int* anchor; const float* theta;
+  DevCalib calib;
+  // level lists
+  int* lst_req[2]; int* lst_depth[2]; int* lst_token[2]; uint64_t* lst_hash[2]; int* lst_slot[2];
+  int* lvl_count;
+  // merged scoring results
+  const float *res_lse0, *res_lseT; const int* res_top_tok; const float* res_top_logit;
+  const int* res_draw_tok; const float* res_draw_logit;
+  // pool
+  int *pl_alive, *pl_depth, *pl_parent, *pl_sib, *pl_tok;
+  double *pl_logkey, *pl_logS; float *pl_q0, *pl_logqT, *pl_lseT; uint64_t *pl_hash, *pl_path;
+  float* root_lseT; int *req_npar, *req_base, *req_nscored;
+  // candidates
+  int *cd_valid, *cd_parent, *cd_sib, *cd_tok; double *cd_logkey, *cd_logS; float *cd_q0, *cd_logqT; int* cd_rank;
+  int* status;
+};
+
+__device__ __forceinline__ void request_caps(const ExpandArgs& a, int b, int& K_eff, int& N_eff, double& log_theta) {
+  const float th = a.theta[b];
+  K_eff = a.K < a.V ? a.K : a.V;
+  N_eff = a.N;
+  if (th >= 1.f) {  // chain member of the price ladder
+    K_eff = 1; N_eff = a.D < a.N ? a.D : a.N; log_theta = -INFINITY;
+  } else {
+    log_theta = th > 0.f ? log((double)th) : -INFINITY;
+  }
+}
+
+__global__ void expand_init_kernel(ExpandArgs a) {
+  const int b = blockIdx.x;
+  for (int s = threadIdx.x; s < a.N; s += blockDim.x) a.pl_alive[(size_t)b * a.N + s] = 0;
+  if (threadIdx.x == 0) {
+    const int tok = a.anchor[b];
+    const bool ok = tok >= 0 && tok < a.V && a.theta[b] == a.theta[b];
+    a.status[b] = ok ? TS_OK : TS_ERR_INVALID;
+    a.lst_req[0][b] = b; a.lst_depth[0][b] = 0; a.lst_token[0][b] = ok ? tok : 0; a.lst_hash[0][b] = 0ull;
+    a.lst_slot[0][b] = -1;
+    a.req_npar[b] = 1; a.req_base[b] = b; a.req_nscored[b] = 0;
+    a.root_lseT[b] = nanf("");
+    if (b == 0) {
+      a.lvl_count[0] = a.B;
+      for (int d = 1; d <= DMAX + 1; ++d) a.lvl_count[d] = 0;
+    }
+  }
+}
+
+struct Entry { double key; uint64_t path; int depth; };
+
+__device__ __forceinline__ bool before(double ka, int da, uint64_t pa, double kb, int db, uint64_t pb) {
+  if (ka != kb) return ka > kb;
+  if (da != db) return da < db;
+  return pa < pb;
+}
+
+// One CTA per request; level d = depth of the parents just scored.
+__global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d) {
+  extern __shared__ __align__(16) unsigned char sm_raw[];
+  __shared__ int s_cnt[2];
+  __shared__ int s_base;
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int N = a.N, K = a.K;
+  const int npar = a.req_npar[b], base = a.req_base[b];
+  const int cur = d & 1, nxt = cur ^ 1;
+  int K_eff, N_eff; double log_theta;
+  request_caps(a, b, K_eff, N_eff, log_theta);
+  const size_t pb = (size_t)b * N, cb = (size_t)b * N * K;
+  if (tid == 0) s_base = a.status[b];
+  __syncthreads();
+  if (npar == 0 || s_base != TS_OK) {  // uniform: read once, before any thread can change the status
+    if (tid == 0) a.req_npar[b] = 0;
+    return;
+  }
+  // ---- phase 1: slots of every scored parent -------------------------------------------------
+  for (int i = tid; i < npar; i += blockDim.x) {
+    const int li = base + i;
+    const int slot = a.lst_slot[cur][li];
+    const double logS_v = slot < 0 ? 0.0 : a.pl_logS[pb + slot];
+    const double lse0 = a.res_lse0[li], lseT = a.res_lseT[li];
+    if (slot < 0) a.root_lseT[b] = (float)lseT; else a.pl_lseT[pb + slot] = (float)lseT;
+    if (!(lse0 == lse0) || isinf(lse0)) a.status[b] = TS_ERR_NUMERIC;
+    const int* top_tok = a.res_top_tok + (size_t)li * K; const float* top_logit = a.res_top_logit + (size_t)li * K;
+    const int* draw_tok = a.res_draw_tok + (size_t)li * K; const float* draw_logit = a.res_draw_logit + (size_t)li * K;
+    bool open = true;
+    for (int j = 0; j < K; ++j) {
+      const size_t ci = cb + (size_t)i * K + j;
+      int valid = 0;
+      if (open && j < K_eff) {
+        int bi = j;
+        if (a.T > 0.f) {  // best token of q0 not among the first j draws: the pre-draw bound
+          bi = -1;
+          for (int t = 0; t < K_eff && bi < 0; ++t) {
+            bool used = false;
+            for (int u = 0; u < j; ++u) used |= (draw_tok[u] == top_tok[t]);
+            if (!used) bi = t;
+          }
+        }
+        const int x = draw_tok[j];
+        if (bi >= 0 && top_tok[bi] >= 0 && x >= 0) {
+          const double key = logS_v + log_phat(a.calib, d, (double)top_logit[bi], lse0);
+          if (!(key < log_theta)) {
+            const double lx = draw_logit[j];
+            valid = 1;
+            a.cd_parent[ci] = slot; a.cd_sib[ci] = j; a.cd_tok[ci] = x;
+            a.cd_logkey[ci] = key;
+            a.cd_logS[ci] = logS_v + log_phat(a.calib, d, lx, lse0);
+            a.cd_q0[ci] = (float)exp(lx - lse0);
+            a.cd_logqT[ci] = a.T > 0.f ? (float)(lx / (double)a.T - lseT) : (float)(lx - lse0);
+          }
+        }
+        if (!valid) open = false;  // keys are non-increasing in j: later slots cannot be admitted
+      }
+      a.cd_valid[ci] = valid;
+    }
+  }
+  __syncthreads();
+  // ---- phase 2: who survives the cut to N_eff ------------------------------------------------
+  const int ncand = npar * K;
+  if (tid < 2) s_cnt[tid] = 0;
+  __syncthreads();
+  {
+    int lp = 0, lc = 0;
+    for (int s = tid; s < N; s += blockDim.x) lp += a.pl_alive[pb + s] ? 1 : 0;
+    for (int c = tid; c < ncand; c += blockDim.x) lc += a.cd_valid[cb + c] ? 1 : 0;
+    if (lp) atomicAdd(&s_cnt[0], lp);
+    if (lc) atomicAdd(&s_cnt[1], lc);
+  }
+  __syncthreads();
+  const int n_pool = s_cnt[0], n_valid = s_cnt[1];
+  const int shift = 60 - 4 * d;
+  if (n_pool + n_valid > N_eff) {
+    // rank every entry by counting the entries that come before it in (key desc, depth asc, path asc)
+    Entry* ent = reinterpret_cast<Entry*>(sm_raw);
+    const int M = N + ncand;
+    for (int e = tid; e < M; e += blockDim.x) {
+      Entry x; x.depth = -1; x.key = 0; x.path = 0;
+      if (e < N) {
+        if (a.pl_alive[pb + e]) { x.key = a.pl_logkey[pb + e]; x.depth = a.pl_depth[pb + e]; x.path = a.pl_path[pb + e]; }
+      } else {
+        const size_t ci = cb + (e - N);
+        if (a.cd_valid[ci]) {
+          const int slot = a.cd_parent[ci];
+          x.key = a.cd_logkey[ci]; x.depth = d + 1;
+          x.path = (slot < 0 ? 0ull : a.pl_path[pb + slot]) | ((uint64_t)a.cd_sib[ci] << shift);
+        }
+      }
+      ent[e] = x;
+    }
+    __syncthreads();
+    for (int e = tid; e < M; e += blockDim.x) {
+      const Entry x = ent[e];
+      if (x.depth < 0) continue;
+      int rank = 0;
+      for (int f = 0; f < M; ++f) {
+        const Entry y = ent[f];
+        if (y.depth >= 0 && f != e && before(y.key, y.depth, y.path, x.key, x.depth, x.path)) ++rank;
+      }
+      if (rank >= N_eff) {
+        if (e < N) a.pl_alive[pb + e] = 0; else a.cd_valid[cb + (e - N)] = 0;
+      }
+    }
+    __syncthreads();
+  }
+  // ---- phase 3: place surviving candidates into free pool slots (deterministic order) --------
+  if (tid == 0) {
+    int s = 0, nnext = 0;
+    for (int c = 0; c < ncand; ++c) {
+      const size_t ci = cb + c;
+      if (!a.cd_valid[ci]) continue;
+      while (s < N && a.pl_alive[pb + s]) ++s;
+      if (s >= N) { a.status[b] = TS_ERR_OVERFLOW; break; }
+      const int slot = a.cd_parent[ci];
+      const int x = a.cd_tok[ci];
+      a.pl_alive[pb + s] = 1; a.pl_depth[pb + s] = d + 1; a.pl_parent[pb + s] = slot; a.pl_sib[pb + s] = a.cd_sib[ci];
+      a.pl_tok[pb + s] = x; a.pl_logkey[pb + s] = a.cd_logkey[ci]; a.pl_logS[pb + s] = a.cd_logS[ci];
+      a.pl_q0[pb + s] = a.cd_q0[ci]; a.pl_logqT[pb + s] = a.cd_logqT[ci]; a.pl_lseT[pb + s] = nanf("");
+      a.pl_hash[pb + s] = path_hash(slot < 0 ? 0ull : a.pl_hash[pb + slot], x);
+      a.pl_path[pb + s] = (slot < 0 ? 0ull : a.pl_path[pb + slot]) | ((uint64_t)a.cd_sib[ci] << shift);
+      a.cd_rank[cb + nnext] = s;  // reuse as "slots added at this level"
+      ++nnext;
+    }
+    // next level's parents: new nodes that can still have admissible children
+    int cnt = 0;
+    if (d + 1 < a.D) {
+      for (int i = 0; i < nnext; ++i) {
+        const int sl = a.cd_rank[cb + i];
+        if (!(a.pl_logS[pb + sl] < log_theta)) a.cd_rank[cb + cnt++] = sl;
+      }
+    }
+    int nb = 0;
+    if (cnt > 0) nb = atomicAdd(&a.lvl_count[d + 1], cnt);
+    for (int i = 0; i < cnt; ++i) {
+      const int sl = a.cd_rank[cb + i];
+      const int li = nb + i;
+      a.lst_req[nxt][li] = b; a.lst_depth[nxt][li] = d + 1; a.lst_token[nxt][li] = a.pl_tok[pb + sl];
+      a.lst_hash[nxt][li] = a.pl_hash[pb + sl]; a.lst_slot[nxt][li] = sl;
+    }
+    a.req_nscored[b] += npar;
+    a.req_npar[b] = cnt; a.req_base[b] = nb;
+  }
+}
+
+struct FinalArgs {
+  int B, N, words;
+  const int *pl_alive, *pl_depth, *pl_parent, *pl_sib, *pl_tok;
+  const double *pl_logkey, *pl_logS; const float *pl_q0, *pl_logqT, *pl_lseT; const uint64_t *pl_hash, *pl_path;
+  const float* root_lseT; const int* req_nscored;
+  int *n_nodes, *tok, *parent, *depth, *sib_rank; float *logS, *q0, *logqT, *logkey; int* pop_rank;
+  uint64_t* node_hash; float* node_lseT; uint64_t* mask; int* n_scored;
+};
+
+// Canonical (BFS) renumbering, outputs and ancestor bitmasks; one CTA per request.
+__global__ void __launch_bounds__(256) expand_finalize_kernel(FinalArgs a) {
+  __shared__ int s_canon[256];
+  __shared__ int s_n;
+  const int b = blockIdx.x, tid = threadIdx.x, N = a.N;
+  const size_t pb = (size_t)b * N;
+  if (tid == 0) s_n = 0;
+  __syncthreads();
+  for (int s = tid; s < N; s += blockDim.x) {
+    s_canon[s] = -1;
+    if (!a.pl_alive[pb + s]) continue;
+    const int ds = a.pl_depth[pb + s]; const uint64_t ps = a.pl_path[pb + s]; const double ks = a.pl_logkey[pb + s];
+    int cr = 0, pr = 0;
+    for (int t = 0; t < N; ++t) {
+      if (t == s || !a.pl_alive[pb + t]) continue;
+      const int dt = a.pl_depth[pb + t]; const uint64_t pt = a.pl_path[pb + t];
+      if (dt < ds || (dt == ds && pt < ps)) ++cr;
+      if (before(a.pl_logkey[pb + t], dt, pt, ks, ds, ps)) ++pr;
+    }
+    s_canon[s] = cr;
+    atomicAdd(&s_n, 1);
+    const size_t o = pb + cr;
+    a.tok[o] = a.pl_tok[pb + s]; a.depth[o] = ds; a.sib_rank[o] = a.pl_sib[pb + s];
+    a.logS[o] = (float)a.pl_logS[pb + s]; a.q0[o] = a.pl_q0[pb + s]; a.logqT[o] = a.pl_logqT[pb + s];
+    if (a.logkey) a.logkey[o] = (float)ks;
+    if (a.pop_rank) a.pop_rank[o] = pr;
+    a.node_hash[(size_t)b * (N + 1) + cr + 1] = a.pl_hash[pb + s];
+    if (a.node_lseT) a.node_lseT[(size_t)b * (N + 1) + cr + 1] = a.pl_lseT[pb + s];
+  }
+  __syncthreads();
+  for (int s = tid; s < N; s += blockDim.x) {
+    if (s_canon[s] < 0) continue;
+    const int ps = a.pl_parent[pb + s];
+    a.parent[pb + s_canon[s]] = ps < 0 ? -1 : s_canon[ps];
+  }
+  if (tid == 0) {
+    a.n_nodes[b] = s_n;
+    a.node_hash[(size_t)b * (N + 1)] = 0ull;
+    if (a.node_lseT) a.node_lseT[(size_t)b * (N + 1)] = a.root_lseT[b];
+    if (a.n_scored) a.n_scored[b] = a.req_nscored[b];
+  }
+  __syncthreads();
+  // a node's mask row = its parent's row plus its own bit; parents precede children in canonical order
+  const int n = s_n;
+  if (tid < a.words) {
+    for (int i = 0; i < n; ++i) {
+      const int p = a.parent[pb + i];
+      uint64_t m = p >= 0 ? a.mask[(pb + p) * a.words + tid] : 0ull;
+      if (i / 64 == tid) m |= 1ull << (i % 64);
+      a.mask[(pb + i) * a.words + tid] = m;
+    }
+  }
+}
+
+}  // namespace ts
+
+extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, const void* W, int32_t B,
+                                  const int32_t* anchor_tok, const float* theta, float T, uint64_t seed,
+                                  int32_t* n_nodes, int32_t* tok, int32_t* parent, int32_t* depth, int32_t* sib_rank,
+                                  float* logS, float* q0, float* logqT, float* logkey, int32_t* pop_rank,
+                                  uint64_t* node_hash, float* node_lseT, uint64_t* mask, int32_t* n_scored,
+                                  int32_t* status, void* ws_v, size_t ws_bytes, void* stream) {
+  using namespace ts;
+  if (!ctx) return set_error(TS_ERR_INVALID, "ts_expand_tree: null context");
+  const void* req[] = {U, A, W, anchor_tok, theta, n_nodes, tok, parent, depth, sib_rank, logS, q0, logqT,
+                       node_hash, mask, status, ws_v};
+  for (const void* p : req)
+    if (bad_ptr(p)) return set_error(TS_ERR_INVALID, "ts_expand_tree: null or misaligned pointer");
+  const void* opt[] = {logkey, pop_rank, node_lseT, n_scored};
+  for (const void* p : opt)
+    if (p && ((uintptr_t)p & 15u)) return set_error(TS_ERR_INVALID, "ts_expand_tree: misaligned optional pointer");
+  const ts_config& c = ctx->cfg;
+  if (B < 1 || B > c.max_batch) return set_error(TS_ERR_INVALID, "ts_expand_tree: B out of range");
+  if (!(T >= 0.f)) return set_error(TS_ERR_INVALID, "ts_expand_tree: T must be >= 0");
+  const WsLayout L = make_layout(ctx, B);
+  if (ws_bytes < L.total) return set_error(TS_ERR_WORKSPACE, "ts_expand_tree: workspace too small");
+  char* ws = (char*)ws_v;
+  cudaStream_t st = (cudaStream_t)stream;
+
+  ExpandArgs a{};
+  a.B = B; a.D = c.D; a.K = c.K; a.N = c.Nmax; a.V = c.V; a.T = T; a.anchor = anchor_tok; a.theta = theta;
+  a.calib = ctx->calib;
+  for (int i = 0; i < 2; ++i) {
+    a.lst_req[i] = (int*)(ws + L.lst_req[i]); a.lst_depth[i] = (int*)(ws + L.lst_depth[i]);
+    a.lst_token[i] = (int*)(ws + L.lst_token[i]); a.lst_hash[i] = (uint64_t*)(ws + L.lst_hash[i]);
+    a.lst_slot[i] = (int*)(ws + L.lst_slot[i]);
+  }
+  a.lvl_count = (int*)(ws + L.lvl_count);
+  float* res_lse0 = (float*)(ws + L.res_lse0); float* res_lseT = (float*)(ws + L.res_lseT);
+  int* res_top_tok = (int*)(ws + L.res_top_tok); float* res_top_logit = (float*)(ws + L.res_top_logit);
+  int* res_draw_tok = (int*)(ws + L.res_draw_tok); float* res_draw_logit = (float*)(ws + L.res_draw_logit);
+  a.res_lse0 = res_lse0; a.res_lseT = res_lseT; a.res_top_tok = res_top_tok; a.res_top_logit = res_top_logit;
+  a.res_draw_tok = res_draw_tok; a.res_draw_logit = res_draw_logit;
+  a.pl_alive = (int*)(ws + L.pl_alive); a.pl_depth = (int*)(ws + L.pl_depth); a.pl_parent = (int*)(ws + L.pl_parent);
+  a.pl_sib = (int*)(ws + L.pl_sib); a.pl_tok = (int*)(ws + L.pl_tok);
+  a.pl_logkey = (double*)(ws + L.pl_logkey); a.pl_logS = (double*)(ws + L.pl_logS);
+  a.pl_q0 = (float*)(ws + L.pl_q0); a.pl_logqT = (float*)(ws + L.pl_logqT); a.pl_lseT = (float*)(ws + L.pl_lseT);
+  a.pl_hash = (uint64_t*)(ws + L.pl_hash); a.pl_path = (uint64_t*)(ws + L.pl_path);
+  a.root_lseT = (float*)(ws + L.root_lseT);
+  a.req_npar = (int*)(ws + L.req_npar); a.req_base = (int*)(ws + L.req_base); a.req_nscored = (int*)(ws + L.req_nscored);
+  a.cd_valid = (int*)(ws + L.cd_valid); a.cd_parent = (int*)(ws + L.cd_parent); a.cd_sib = (int*)(ws + L.cd_sib);
+  a.cd_tok = (int*)(ws + L.cd_tok); a.cd_logkey = (double*)(ws + L.cd_logkey); a.cd_logS = (double*)(ws + L.cd_logS);
+  a.cd_q0 = (float*)(ws + L.cd_q0); a.cd_logqT = (float*)(ws + L.cd_logqT); a.cd_rank = (int*)(ws + L.cd_rank);
+  a.status = status;
+
+  expand_init_kernel<<<B, 64, 0, st>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(init)", e);
+  const size_t level_smem = (size_t)(c.Nmax + c.Nmax * c.K) * sizeof(Entry);
+  if (level_smem > 48 * 1024) {
+    e = cudaFuncSetAttribute(expand_level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)level_smem);
+    if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(attr)", e);
+  }
+  for (int d = 0; d < c.D; ++d) {
+    const int cur = d & 1;
+    e = launch_score(ctx, L, ws, U, A, W, 0, a.lvl_count + d, a.lst_req[cur], a.lst_depth[cur], a.lst_token[cur],
+                     a.lst_hash[cur], T, seed, res_lse0, res_lseT, res_top_tok, res_top_logit, res_draw_tok,
+                     res_draw_logit, st);
+    if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(score)", e);
+    expand_level_kernel<<<B, 256, level_smem, st>>>(a, d);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(level)", e);
+  }
+  FinalArgs f{};
+  f.B = B; f.N = c.Nmax; f.words = L.words;
+  f.pl_alive = a.pl_alive; f.pl_depth = a.pl_depth; f.pl_parent = a.pl_parent; f.pl_sib = a.pl_sib; f.pl_tok = a.pl_tok;
+  f.pl_logkey = a.pl_logkey; f.pl_logS = a.pl_logS; f.pl_q0 = a.pl_q0; f.pl_logqT = a.pl_logqT; f.pl_lseT = a.pl_lseT;
+  f.pl_hash = a.pl_hash; f.pl_path = a.pl_path; f.root_lseT = a.root_lseT; f.req_nscored = a.req_nscored;
+  f.n_nodes = n_nodes; f.tok = tok; f.parent = parent; f.depth = depth; f.sib_rank = sib_rank; f.logS = logS; f.q0 = q0;
+  f.logqT = logqT; f.logkey = logkey; f.pop_rank = pop_rank; f.node_hash = node_hash; f.node_lseT = node_lseT;
+  f.mask = mask; f.n_scored = n_scored;
+  expand_finalize_kernel<<<B, 256, 0, st>>>(f);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(finalize)", e);
+  return TS_OK;
+}

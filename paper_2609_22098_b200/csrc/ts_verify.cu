@@ -1,0 +1,558 @@
+// Lossless tree verification (Section 3.2 item 3, Section 3.3).
+//
+// Stage 1 (all rows, fully parallel): max, arg-max and log-sum-exp at temperature T of every target
+//   row, one CTA per row.  With these, the first-sibling accept ratio of every edge is a scalar
+//   expression, so per-edge statistics and greedy walks need no further vocabulary pass.
+// Stage 2, T == 0: pointer chase along arg-max matches.
+// Stage 2, T > 0: one persistent cooperative kernel.  The recursive-rejection walk is run as a
+//   scalar sequence: with R(w) = max(p(w) - C q(w), 0) the unnormalised residual after rejections,
+//   sibling j is accepted with probability min(1, max(p(x)/q(x) - C, 0) / c_j), c_j = Z_j / (1 - Q),
+//   and a rejection moves C to C + c_j and needs Z_{j+1} = sum_w R(w), one reduction over the
+//   vocabulary (tokens already tested keep the residual they had when tested).  Every grid step
+//   runs that reduction for all requests that just rejected, each CTA owning a vocabulary range;
+//   q is recomputed from U, A, W, no per-node vocabulary vector is stored.  The bonus token is the
+//   inverse CDF of the final residual in token order: range sums locate the range, one CTA rescans it.
+#include <cooperative_groups.h>
+#include <math.h>
+
+#include "ts_internal.h"
+
+namespace ts {
+
+constexpr int VT = 256;  // threads of the verification kernels
+
+// ------------------------------------------------------------------------------------------------
+// Stage 1: row statistics
+// ------------------------------------------------------------------------------------------------
+template <typename TIn>
+__global__ void __launch_bounds__(VT) zrow_stats_kernel(const TIn* Z, const int64_t* z_row_off, int B, int V, float T,
+                                                       float* z_max, int* z_arg, float* z_logs) {
+  __shared__ float s_v[VT / 32]; __shared__ int s_i[VT / 32]; __shared__ float s_m;
+  const int64_t rows = z_row_off[B];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int VEC = Elem<TIn>::VEC;
+  const bool vec_ok = (V % VEC) == 0;
+  const float invT = T > 0.f ? 1.f / T : 1.f;
+  for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+    const TIn* z = Z + row * V;
+    float bv = -INFINITY; int bi = 0x7FFFFFFF;
+    if (vec_ok) {
+      for (int c = tid * VEC; c < V; c += VT * VEC) {
+        float x[8];
+        if (sizeof(TIn) == 2) { const uint4 v = __ldg(reinterpret_cast<const uint4*>(z + c)); unpack_bf16x8(v, x); }
+        else { const float4 v = __ldg(reinterpret_cast<const float4*>(z + c)); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) if (x[i] > bv) { bv = x[i]; bi = c + i; }
+      }
+    } else {
+      for (int c = tid; c < V; c += VT) { const float x = Elem<TIn>::to_f(z[c]); if (x > bv) { bv = x; bi = c; } }
+    }
+    for (int off = 16; off > 0; off >>= 1) {
+      const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, off); const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, off);
+      if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    if (lane == 0) { s_v[warp] = bv; s_i[warp] = bi; }
+    __syncthreads();
+    if (tid == 0) {
+      for (int w = 1; w < VT / 32; ++w) if (s_v[w] > bv || (s_v[w] == bv && s_i[w] < bi)) { bv = s_v[w]; bi = s_i[w]; }
+      s_m = bv; z_max[row] = bv; z_arg[row] = bi;
+    }
+    __syncthreads();
+    if (T > 0.f) {
+      const float m = s_m;
+      float s = 0.f;
+      if (vec_ok) {
+        for (int c = tid * VEC; c < V; c += VT * VEC) {
+          float x[8];
+          if (sizeof(TIn) == 2) { const uint4 v = __ldg(reinterpret_cast<const uint4*>(z + c)); unpack_bf16x8(v, x); }
+          else { const float4 v = __ldg(reinterpret_cast<const float4*>(z + c)); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+#pragma unroll
+          for (int i = 0; i < VEC; ++i) s += __expf((x[i] - m) * invT);
+        }
+      } else {
+        for (int c = tid; c < V; c += VT) s += __expf((Elem<TIn>::to_f(z[c]) - m) * invT);
+      }
+      for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+      __syncthreads();
+      if (lane == 0) s_v[warp] = s;
+      __syncthreads();
+      if (tid == 0) { float t = 0.f; for (int w = 0; w < VT / 32; ++w) t += s_v[w]; z_logs[row] = logf(t); }
+    }
+    __syncthreads();
+  }
+}
+
+struct VerifyArgs {
+  const void *U, *A, *W, *Z; const int64_t* z_row_off;
+  int B, V, D, r, K, N; float T; uint64_t seed;
+  const int *anchor, *n_nodes, *tok, *parent, *depth, *sib; const uint64_t* node_hash;
+  const float *logqT, *node_lseT;
+  const float* z_max; const int* z_arg; const float* z_logs;
+  int *acc_len, *acc_node, *acc_tok, *bonus; float* edge_stat; uint32_t* flags; int* status;
+  VerifyState* state; float* part; unsigned* barrier;
+  int vt_TV, vt_n, max_steps;
+};
+
+// ------------------------------------------------------------------------------------------------
+// Stage 2, T == 0
+// ------------------------------------------------------------------------------------------------
+__global__ void verify_greedy_kernel(VerifyArgs a) {
+  const int b = blockIdx.x, N = a.N;
+  const int n = a.n_nodes[b];
+  const int64_t row0 = a.z_row_off[b];
+  const size_t nb = (size_t)b * N;
+  if (a.edge_stat)
+    for (int i = threadIdx.x; i < n; i += blockDim.x)
+      a.edge_stat[nb + i] = (a.tok[nb + i] == a.z_arg[row0 + a.parent[nb + i] + 1]) ? 1.f : 0.f;
+  if (threadIdx.x == 0) {
+    int cur = -1, acc = 0;
+    for (;;) {
+      const int g = a.z_arg[row0 + cur + 1];
+      int hit = -1;
+      for (int i = cur + 1; i < n; ++i)  // children come after their parent in canonical order
+        if (a.parent[nb + i] == cur && a.tok[nb + i] == g) { hit = i; break; }
+      if (hit < 0 || acc >= a.D) { a.bonus[b] = g; break; }
+      a.acc_node[(size_t)b * a.D + acc] = hit; a.acc_tok[(size_t)b * a.D + acc] = g; ++acc; cur = hit;
+    }
+    for (int i = acc; i < a.D; ++i) { a.acc_node[(size_t)b * a.D + i] = -1; a.acc_tok[(size_t)b * a.D + i] = -1; }
+    a.acc_len[b] = acc; a.flags[b] = 0u; a.status[b] = (n >= 0 && n <= N) ? TS_OK : TS_ERR_INVALID;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Stage 2, T > 0
+// ------------------------------------------------------------------------------------------------
+template <typename TIn>
+__device__ __forceinline__ float z_elem(const VerifyArgs& a, int64_t row, int w) {
+  return Elem<TIn>::to_f(reinterpret_cast<const TIn*>(a.Z)[row * a.V + w]);
+}
+
+// probability of token w under softmax(Z[row]/T), double
+template <typename TIn>
+__device__ __forceinline__ double p_of(const VerifyArgs& a, int64_t row, int w) {
+  return exp(((double)z_elem<TIn>(a, row, w) - (double)a.z_max[row]) / (double)a.T - (double)a.z_logs[row]);
+}
+
+// children of node v are contiguous in canonical order; returns the first and the count
+__device__ __forceinline__ void children_of(const VerifyArgs& a, int b, int n, int v, int& first, int& m) {
+  const size_t nb = (size_t)b * a.N;
+  first = -1; m = 0;
+  for (int i = v + 1; i < n; ++i) {
+    if (a.parent[nb + i] == v) { if (first < 0) first = i; ++m; }
+    else if (first >= 0) break;
+  }
+}
+
+// Scalar state machine of one request (lane 0 decides, the warp helps with range sums).
+// need: 0 walking, 1 reduction after a rejection, 4 reduction for the bonus draw, 2 range rescan, 3 finished
+template <typename TIn>
+__device__ void advance(const VerifyArgs& a, int b, int lane) {
+  VerifyState& st = a.state[b];
+  const int N = a.N, n = a.n_nodes[b];
+  const size_t nb = (size_t)b * N;
+  const int64_t row0 = a.z_row_off[b];
+  int need = st.need;
+  if (need == 3) return;
+  // ---- fold in the reduction that just ran -------------------------------------------------
+  double fsum = 0.0;
+  if (need == 1 || need == 4) {
+    for (int t = lane; t < a.vt_n; t += 32) fsum += (double)a.part[(size_t)b * a.vt_n + t];
+    for (int off = 16; off > 0; off >>= 1) fsum += __shfl_xor_sync(0xFFFFFFFFu, fsum, off);
+  }
+  int go_scan = 0;
+  if (lane == 0) {
+    if (need == 1 || need == 4) {
+      double zn = fsum;  // the pass used passC for every token; tested siblings keep their own C_i
+      for (int i = 0; i < st.nf; ++i)
+        zn += fmax(st.fp[i] - st.fC[i] * st.fq[i], 0.0) - fmax(st.fp[i] - st.passC * st.fq[i], 0.0);
+      if (need == 1) {
+        if (zn <= 1e-30 * st.Zj) {  // residual lost its mass: keep the previous one
+          a.flags[b] |= TS_FLAG_ZERO_MASS;
+          st.fC[st.nf - 1] = st.C;
+          st.partsC = -1.0;
+        } else { st.C = st.passC; st.Zj = zn; st.partsC = st.passC; }
+      } else { st.Zj = zn; st.partsC = st.passC; }
+      st.need = 0;
+    }
+    if (st.need == 2) {  // the rescan wrote its token
+      a.bonus[b] = st.result;
+      a.acc_len[b] = st.acc;
+      st.need = 3;
+    }
+    while (st.need == 0) {
+      const int v = st.cur;
+      int first, m;
+      children_of(a, b, n, v, first, m);
+      const int64_t row = row0 + v + 1;
+      const uint64_t hv = a.node_hash[(size_t)b * (N + 1) + v + 1];
+      if (st.j < m && st.acc < a.D) {
+        const int child = first + st.j, x = a.tok[nb + child];
+        const double px = p_of<TIn>(a, row, x), qx = exp((double)a.logqT[nb + child]);
+        const double cj = st.Zj / (1.0 - st.Qused);
+        const double num = fmax(px / qx - st.C, 0.0);
+        const double rho = fmin(1.0, num / cj);
+        const double u = u01(stream_words(a.seed, b, hv, STREAM_ACCEPT, (uint32_t)st.j).x);
+        if (u < rho) {
+          a.acc_node[(size_t)b * a.D + st.acc] = child; a.acc_tok[(size_t)b * a.D + st.acc] = x;
+          st.acc++; st.cur = child; st.j = 0; st.C = 0.0; st.Zj = 1.0; st.Qused = 0.0; st.nf = 0; st.partsC = -1.0;
+        } else {
+          st.fx[st.nf] = x; st.fp[st.nf] = px; st.fq[st.nf] = qx; st.fC[st.nf] = st.C + cj; st.nf++;
+          st.Qused += qx; st.j++;
+          st.passC = st.C + cj; st.row_node = v; st.need = 1;
+        }
+      } else {
+        if (st.partsC != st.C) { st.passC = st.C; st.row_node = v; st.need = 4; }
+        else go_scan = 1;
+        break;
+      }
+    }
+  }
+  go_scan = __shfl_sync(0xFFFFFFFFu, go_scan, 0);
+  __syncwarp();
+  if (go_scan) {
+    // locate the vocabulary range holding the bonus token: cumulative corrected range sums
+    const uint64_t hv = a.node_hash[(size_t)b * (N + 1) + st.cur + 1];
+    const double u = u01(stream_words(a.seed, b, hv, STREAM_BONUS, 0u).x);
+    const double target = u * st.Zj;
+    double carry = 0.0; int found = -1; double before = 0.0; int last_pos = -1;
+    for (int t0 = 0; t0 < a.vt_n && found < 0; t0 += 32) {
+      const int t = t0 + lane;
+      double pt = 0.0;
+      if (t < a.vt_n) {
+        pt = (double)a.part[(size_t)b * a.vt_n + t];
+        for (int i = 0; i < st.nf; ++i)
+          if (st.fx[i] / a.vt_TV == t)
+            pt += fmax(st.fp[i] - st.fC[i] * st.fq[i], 0.0) - fmax(st.fp[i] - st.C * st.fq[i], 0.0);
+        if (pt < 0.0) pt = 0.0;
+      }
+      double inc = pt;
+      for (int off = 1; off < 32; off <<= 1) { const double o = __shfl_up_sync(0xFFFFFFFFu, inc, off); if (lane >= off) inc += o; }
+      const bool cross = (t < a.vt_n) && (carry + inc > target);
+      const unsigned bal = __ballot_sync(0xFFFFFFFFu, cross);
+      const unsigned pos = __ballot_sync(0xFFFFFFFFu, pt > 0.0);
+      if (pos) last_pos = t0 + 31 - __clz(pos);
+      if (bal) {
+        const int src = __ffs(bal) - 1;
+        found = t0 + src;
+        before = carry + __shfl_sync(0xFFFFFFFFu, inc - pt, src);
+      }
+      carry += __shfl_sync(0xFFFFFFFFu, inc, 31);
+    }
+    if (lane == 0) {
+      if (found < 0) { found = last_pos >= 0 ? last_pos : 0; before = -1.0; }  // rounding: take the last range with mass
+      st.scan_tile = found; st.target = target; st.before = before; st.need = 2;
+    }
+  }
+  __syncwarp();
+}
+
+// logits of up to G parents for the VEC tokens at v (global W, coalesced 16-byte loads)
+template <typename TIn, int G>
+__device__ __forceinline__ void logits_group(const VerifyArgs& a, const float* as, int ng, const int* rq_req,
+                                             const int* rq_dep, int v, float (*acc)[8]) {
+  constexpr int VEC = Elem<TIn>::VEC;
+  const TIn* Wg = reinterpret_cast<const TIn*>(a.W);
+  const TIn* Ug = reinterpret_cast<const TIn*>(a.U);
+  for (int g = 0; g < G; ++g) {
+    if (g < ng) {
+      const TIn* u = Ug + ((size_t)rq_req[g] * a.D + rq_dep[g]) * a.V + v;
+      if (sizeof(TIn) == 2) { const uint4 x = __ldg(reinterpret_cast<const uint4*>(u)); unpack_bf16x8(x, acc[g]); }
+      else { const float4 x = __ldg(reinterpret_cast<const float4*>(u)); acc[g][0] = x.x; acc[g][1] = x.y; acc[g][2] = x.z; acc[g][3] = x.w; }
+    }
+  }
+  for (int k = 0; k < a.r; ++k) {
+    float w[8];
+    if (sizeof(TIn) == 2) { const uint4 x = __ldg(reinterpret_cast<const uint4*>(Wg + (size_t)k * a.V + v)); unpack_bf16x8(x, w); }
+    else { const float4 x = __ldg(reinterpret_cast<const float4*>(Wg + (size_t)k * a.V + v)); w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w; }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const float ak = as[g * 128 + k];
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) acc[g][i] = fmaf(ak, w[i], acc[g][i]);
+    }
+  }
+}
+
+template <typename TIn>
+__device__ __forceinline__ float logit_scalar(const VerifyArgs& a, int req, int dep, int ptok, int w) {
+  const TIn* Wg = reinterpret_cast<const TIn*>(a.W);
+  const TIn* Ug = reinterpret_cast<const TIn*>(a.U);
+  const TIn* Ag = reinterpret_cast<const TIn*>(a.A);
+  float acc = Elem<TIn>::to_f(Ug[((size_t)req * a.D + dep) * a.V + w]);
+  for (int k = 0; k < a.r; ++k)
+    acc = fmaf(Elem<TIn>::to_f(Ag[(size_t)ptok * a.r + k]), Elem<TIn>::to_f(Wg[(size_t)k * a.V + w]), acc);
+  return acc;
+}
+
+constexpr int VG = 4;  // requests sharing one sweep over the W columns
+
+template <typename TIn>
+__global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
+  __shared__ float s_a[VG * 128];
+  __shared__ int s_req[VG], s_dep[VG], s_node[VG];
+  __shared__ float s_C[VG], s_zmax[VG], s_zlogs[VG], s_lseT[VG];
+  __shared__ float s_red[VG][VT / 32];
+  __shared__ double s_scan[VT];
+  __shared__ int s_found;
+  __shared__ int s_any;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const unsigned nblocks = gridDim.x;
+  unsigned gen = 0;
+  constexpr int VEC = Elem<TIn>::VEC;
+  const bool vec_ok = (a.V % VEC) == 0;
+  const float invT = 1.f / a.T;
+  const int v_lo = blockIdx.x * a.vt_TV, v_hi = min(a.V, v_lo + a.vt_TV);
+  const TIn* Zg = reinterpret_cast<const TIn*>(a.Z);
+  const TIn* Ag = reinterpret_cast<const TIn*>(a.A);
+
+  // per-edge statistics and state initialisation
+  for (int b = blockIdx.x; b < a.B; b += nblocks) {
+    const int n = a.n_nodes[b];
+    const size_t nb = (size_t)b * a.N;
+    const int64_t row0 = a.z_row_off[b];
+    if (a.edge_stat)
+      for (int i = tid; i < n; i += VT) {
+        const int64_t row = row0 + a.parent[nb + i] + 1;
+        const double lr = ((double)z_elem<TIn>(a, row, a.tok[nb + i]) - (double)a.z_max[row]) / (double)a.T -
+                          (double)a.z_logs[row] - (double)a.logqT[nb + i];
+        a.edge_stat[nb + i] = (float)exp(fmin(lr, 0.0));
+      }
+    if (tid == 0) {
+      VerifyState& st = a.state[b];
+      st.cur = -1; st.j = 0; st.acc = 0; st.need = 0; st.nf = 0; st.scan_tile = -1; st.row_node = -1; st.result = -1;
+      st.C = 0.0; st.Zj = 1.0; st.Qused = 0.0; st.target = 0.0; st.before = 0.0; st.passC = 0.0; st.partsC = -1.0;
+      a.flags[b] = 0u;
+      a.status[b] = (n >= 0 && n <= a.N) ? TS_OK : TS_ERR_INVALID;
+      if (!(n >= 0 && n <= a.N)) { st.need = 3; a.acc_len[b] = 0; a.bonus[b] = -1; }
+      for (int i = 0; i < a.D; ++i) { a.acc_node[(size_t)b * a.D + i] = -1; a.acc_tok[(size_t)b * a.D + i] = -1; }
+    }
+  }
+  __syncthreads();
+
+  for (int step = 0; step < a.max_steps; ++step) {
+    // ---- phase A: scalar walks ---------------------------------------------------------------
+    if (warp == 0)
+      for (int b = blockIdx.x; b < a.B; b += nblocks) advance<TIn>(a, b, lane);
+    if (!grid_barrier(a.barrier, nblocks, gen)) return;
+    // ---- phase B: vocabulary work requested by the walks ----------------------------------------
+    if (tid == 0) s_any = 0;
+    __syncthreads();
+    for (int b0 = 0; b0 < a.B; b0 += VG) {
+      // gather up to VG requests that asked for a reduction
+      if (tid == 0) {
+        int ng = 0;
+        for (int b = b0; b < min(a.B, b0 + VG); ++b) {
+          const VerifyState& st = a.state[b];
+          if (st.need != 3) s_any = 1;
+          if (st.need == 1 || st.need == 4) {
+            const int v = st.row_node;
+            const int64_t row = a.z_row_off[b] + v + 1;
+            s_req[ng] = b; s_node[ng] = v; s_dep[ng] = v < 0 ? 0 : a.depth[(size_t)b * a.N + v];
+            s_C[ng] = (float)st.passC; s_zmax[ng] = a.z_max[row]; s_zlogs[ng] = a.z_logs[row];
+            s_lseT[ng] = a.node_lseT[(size_t)b * (a.N + 1) + v + 1];
+            ++ng;
+          }
+        }
+        s_found = ng;
+      }
+      __syncthreads();
+      const int ng = s_found;
+      if (ng > 0) {
+        for (int i = tid; i < ng * a.r; i += VT) {
+          const int g = i / a.r, k = i % a.r;
+          const int v = s_node[g];
+          const int ptok = v < 0 ? a.anchor[s_req[g]] : a.tok[(size_t)s_req[g] * a.N + v];
+          s_a[g * 128 + k] = Elem<TIn>::to_f(Ag[(size_t)ptok * a.r + k]);
+        }
+        __syncthreads();
+        float sum[VG];
+#pragma unroll
+        for (int g = 0; g < VG; ++g) sum[g] = 0.f;
+        bool need_q = false;
+        for (int g = 0; g < ng; ++g) need_q |= (s_C[g] != 0.f);
+        if (vec_ok) {
+          for (int v = v_lo + tid * VEC; v < v_hi; v += VT * VEC) {
+            float acc[VG][8];
+            if (need_q) logits_group<TIn, VG>(a, s_a, ng, s_req, s_dep, v, acc);
+#pragma unroll
+            for (int g = 0; g < VG; ++g) {
+              if (g < ng) {
+                const int64_t row = a.z_row_off[s_req[g]] + s_node[g] + 1;
+                float z[8];
+                if (sizeof(TIn) == 2) { const uint4 x = __ldg(reinterpret_cast<const uint4*>(Zg + row * a.V + v)); unpack_bf16x8(x, z); }
+                else { const float4 x = __ldg(reinterpret_cast<const float4*>(Zg + row * a.V + v)); z[0] = x.x; z[1] = x.y; z[2] = x.z; z[3] = x.w; }
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) {
+                  const float p = __expf((z[i] - s_zmax[g]) * invT - s_zlogs[g]);
+                  const float q = s_C[g] != 0.f ? __expf(acc[g][i] * invT - s_lseT[g]) : 0.f;
+                  sum[g] += fmaxf(p - s_C[g] * q, 0.f);
+                }
+              }
+            }
+          }
+        } else {
+          for (int v = v_lo + tid; v < v_hi; v += VT) {
+            for (int g = 0; g < ng; ++g) {
+              const int b = s_req[g];
+              const int64_t row = a.z_row_off[b] + s_node[g] + 1;
+              const float p = __expf((z_elem<TIn>(a, row, v) - s_zmax[g]) * invT - s_zlogs[g]);
+              float q = 0.f;
+              if (s_C[g] != 0.f) {
+                const int ptok = s_node[g] < 0 ? a.anchor[b] : a.tok[(size_t)b * a.N + s_node[g]];
+                q = __expf(logit_scalar<TIn>(a, b, s_dep[g], ptok, v) * invT - s_lseT[g]);
+              }
+              sum[g] += fmaxf(p - s_C[g] * q, 0.f);
+            }
+          }
+        }
+#pragma unroll
+        for (int g = 0; g < VG; ++g) {
+          float s = sum[g];
+          for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+          if (lane == 0) s_red[g][warp] = s;
+        }
+        __syncthreads();
+        if (tid < ng) {
+          float t = 0.f;
+          for (int w = 0; w < VT / 32; ++w) t += s_red[tid][w];
+          a.part[(size_t)s_req[tid] * a.vt_n + blockIdx.x] = t;
+        }
+      }
+      __syncthreads();
+    }
+    // range rescans for bonus tokens that fall into this CTA's range
+    for (int b = 0; b < a.B; ++b) {
+      const VerifyState& st = a.state[b];
+      if (st.need != 2 || st.scan_tile != (int)blockIdx.x) continue;
+      const int v = st.cur;
+      const int64_t row = a.z_row_off[b] + v + 1;
+      const int dep = v < 0 ? 0 : a.depth[(size_t)b * a.N + v];
+      const int ptok = v < 0 ? a.anchor[b] : a.tok[(size_t)b * a.N + v];
+      const double C = st.C;
+      const double zmax = a.z_max[row], zlogs = a.z_logs[row];
+      const double lseT = C != 0.0 ? (double)a.node_lseT[(size_t)b * (a.N + 1) + v + 1] : 0.0;
+      const int len = v_hi - v_lo;
+      const int per = (len + VT - 1) / VT;
+      const int w0 = v_lo + tid * per, w1 = min(v_hi, w0 + per);
+      double loc = 0.0;
+      for (int w = w0; w < w1; ++w) {
+        double Cw = C;
+        for (int i = 0; i < st.nf; ++i) if (st.fx[i] == w) Cw = st.fC[i];
+        const double p = exp(((double)z_elem<TIn>(a, row, w) - zmax) / (double)a.T - zlogs);
+        const double q = Cw != 0.0 ? exp((double)logit_scalar<TIn>(a, b, dep, ptok, w) / (double)a.T - lseT) : 0.0;
+        loc += fmax(p - Cw * q, 0.0);
+      }
+      s_scan[tid] = loc;
+      if (tid == 0) s_found = 0x7FFFFFFF;
+      __syncthreads();
+      if (tid == 0) { double c = 0.0; for (int t = 0; t < VT; ++t) { const double x = s_scan[t]; s_scan[t] = c; c += x; } }
+      __syncthreads();
+      const double want = st.before >= 0.0 ? st.target - st.before : 1e300;
+      double cum = s_scan[tid];
+      int lastpos = -1;
+      for (int w = w0; w < w1; ++w) {
+        double Cw = C;
+        for (int i = 0; i < st.nf; ++i) if (st.fx[i] == w) Cw = st.fC[i];
+        const double p = exp(((double)z_elem<TIn>(a, row, w) - zmax) / (double)a.T - zlogs);
+        const double q = Cw != 0.0 ? exp((double)logit_scalar<TIn>(a, b, dep, ptok, w) / (double)a.T - lseT) : 0.0;
+        const double rw = fmax(p - Cw * q, 0.0);
+        cum += rw;
+        if (rw > 0.0) lastpos = w;
+        if (cum > want) { atomicMin(&s_found, w); break; }
+      }
+      __syncthreads();
+      if (s_found == 0x7FFFFFFF) {  // rounding pushed the crossing past this range: last token with mass
+        if (tid == 0) s_found = -1;
+        __syncthreads();
+        if (lastpos >= 0) atomicMax(&s_found, lastpos);
+        __syncthreads();
+        if (tid == 0 && s_found < 0) s_found = v_hi - 1;
+        __syncthreads();
+      }
+      if (tid == 0) a.state[b].result = s_found;
+      __syncthreads();
+    }
+    const int any = s_any;
+    if (!grid_barrier(a.barrier, nblocks, gen)) return;
+    if (!any) return;
+  }
+  // steps ran out
+  for (int b = blockIdx.x; b < a.B; b += nblocks)
+    if (tid == 0 && a.state[b].need != 3) a.status[b] = TS_ERR_TIMEOUT;
+}
+
+// after a barrier timeout the kernel returns early; this marks every unfinished request
+__global__ void verify_check_kernel(VerifyArgs a) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= a.B) return;
+  if (a.barrier[1] != 0u && a.state[b].need != 3) a.status[b] = TS_ERR_TIMEOUT;
+}
+
+cudaError_t verify_setup(ts_ctx* ctx) {
+  (void)ctx;
+  return cudaSuccess;
+}
+
+}  // namespace ts
+
+extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, const void* W, const void* Z,
+                                  const int64_t* z_row_off, int32_t B, const int32_t* anchor_tok,
+                                  const int32_t* n_nodes, const int32_t* tok, const int32_t* parent,
+                                  const int32_t* depth, const int32_t* sib_rank, const uint64_t* node_hash,
+                                  const float* logqT, const float* node_lseT, float T, uint64_t seed,
+                                  int32_t* acc_len, int32_t* acc_node, int32_t* acc_tok, int32_t* bonus_tok,
+                                  float* edge_stat, uint32_t* flags, int32_t* status, void* ws_v, size_t ws_bytes,
+                                  void* stream) {
+  using namespace ts;
+  if (!ctx) return set_error(TS_ERR_INVALID, "ts_verify_tree: null context");
+  const void* req[] = {U, A, W, Z, z_row_off, anchor_tok, n_nodes, tok, parent, depth, sib_rank, node_hash,
+                       acc_len, acc_node, acc_tok, bonus_tok, flags, status, ws_v};
+  for (const void* p : req)
+    if (bad_ptr(p)) return set_error(TS_ERR_INVALID, "ts_verify_tree: null or misaligned pointer");
+  if (edge_stat && ((uintptr_t)edge_stat & 15u)) return set_error(TS_ERR_INVALID, "ts_verify_tree: misaligned edge_stat");
+  const ts_config& c = ctx->cfg;
+  if (B < 1 || B > c.max_batch) return set_error(TS_ERR_INVALID, "ts_verify_tree: B out of range");
+  if (!(T >= 0.f)) return set_error(TS_ERR_INVALID, "ts_verify_tree: T must be >= 0");
+  if (T > 0.f && (bad_ptr(logqT) || bad_ptr(node_lseT)))
+    return set_error(TS_ERR_INVALID, "ts_verify_tree: logqT and node_lseT are required when T > 0");
+  const WsLayout L = make_layout(ctx, B);
+  if (ws_bytes < L.total) return set_error(TS_ERR_WORKSPACE, "ts_verify_tree: workspace too small");
+  char* ws = (char*)ws_v;
+  cudaStream_t st = (cudaStream_t)stream;
+
+  VerifyArgs a{};
+  a.U = U; a.A = A; a.W = W; a.Z = Z; a.z_row_off = z_row_off; a.B = B; a.V = c.V; a.D = c.D; a.r = c.r; a.K = c.K;
+  a.N = c.Nmax; a.T = T; a.seed = seed; a.anchor = anchor_tok; a.n_nodes = n_nodes; a.tok = tok; a.parent = parent;
+  a.depth = depth; a.sib = sib_rank; a.node_hash = node_hash; a.logqT = logqT; a.node_lseT = node_lseT;
+  float* z_max = (float*)(ws + L.z_max); int* z_arg = (int*)(ws + L.z_arg); float* z_logs = (float*)(ws + L.z_lse);
+  a.z_max = z_max; a.z_arg = z_arg; a.z_logs = z_logs;
+  a.acc_len = acc_len; a.acc_node = acc_node; a.acc_tok = acc_tok; a.bonus = bonus_tok; a.edge_stat = edge_stat;
+  a.flags = flags; a.status = status;
+  a.state = (VerifyState*)(ws + L.vf_state); a.part = (float*)(ws + L.vf_part); a.barrier = (unsigned*)(ws + L.vf_barrier);
+  a.vt_TV = ctx->vt_TV; a.vt_n = ctx->vt_n; a.max_steps = 2 * (c.Nmax + c.D) + 8;
+
+  const int max_rows = B * (c.Nmax + 1);
+  int grid_rows = max_rows < 8 * ctx->num_sms ? max_rows : 8 * ctx->num_sms;
+  if (c.dt_Z == TS_DTYPE_BF16)
+    zrow_stats_kernel<__nv_bfloat16><<<grid_rows, VT, 0, st>>>((const __nv_bfloat16*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+  else
+    zrow_stats_kernel<float><<<grid_rows, VT, 0, st>>>((const float*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(rows)", e);
+  if (T == 0.f) {
+    verify_greedy_kernel<<<B, 128, 0, st>>>(a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(greedy)", e);
+    return TS_OK;
+  }
+  e = cudaMemsetAsync(a.barrier, 0, 64, st);
+  if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(memset)", e);
+  void* kargs[] = {(void*)&a};
+  const void* fn = c.dt_Z == TS_DTYPE_BF16 ? (const void*)verify_walk_kernel<__nv_bfloat16> : (const void*)verify_walk_kernel<float>;
+  e = cudaLaunchCooperativeKernel(fn, dim3(a.vt_n), dim3(VT), kargs, 0, st);
+  if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(walk)", e);
+  verify_check_kernel<<<(B + 127) / 128, 128, 0, st>>>(a);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(check)", e);
+  return TS_OK;
+}

@@ -132,8 +132,8 @@ class Workload:
     plant_per_request: bool    # one strength per request (True) or per (request, depth)
     z_sigma: float             # target logits = drafter logits + z_sigma * N(0,1)
     calib_mode: int = 1        # 1 = per-depth 16-knot table, 0 = Platt scalars
-    calib_b_lo: float = 0.9    # per-depth Platt intercept range sampled into the table
-    calib_b_hi: float = 1.3
+    calib_b_lo: float = 0.6    # per-depth Platt intercept range sampled into the table
+    calib_b_hi: float = 1.0
 
     @property
     def torch_dtype(self):
@@ -159,7 +159,7 @@ WORKLOADS = {
     # Wide / deep trees on flat distributions.
     "wide": Workload("wide", B=8, V=128256, D=16, r=128, K=16, Nmax=256, dtype="bf16", theta=0.01,
                      temps=(0.7, 1.3), u_std=2.0, plant_lo=0.0, plant_hi=0.0,
-                     plant_per_request=False, z_sigma=0.8),
+                     plant_per_request=False, z_sigma=0.8, calib_b_lo=3.0, calib_b_hi=3.4),
     # Load sweep: same shape as serve32; the batch and the theta schedule vary.
     "sweep": Workload("sweep", B=16, V=151936, D=8, r=64, K=8, Nmax=64, dtype="bf16", theta=0.1,
                       temps=(1.0,), u_std=4.0, plant_lo=3.0, plant_hi=9.0,
@@ -280,7 +280,8 @@ def make_target_logits(wl: Workload, seed: int, U_full: torch.Tensor, A: torch.T
         dep_l.append(torch.cat([torch.zeros(1, dtype=torch.int64), depth[b, :n].to("cpu", torch.int64)]))
         tok_l.append(torch.cat([anchor[b:b + 1].to("cpu", torch.int64), tok[b, :n].to("cpu", torch.int64)]))
         hash_l.append(node_hash[b, :n + 1].to("cpu", torch.int64))
-    req = torch.cat(req_l).to(dev)
+    req_c = torch.cat(req_l)
+    req = req_c.to(dev)
     dep = torch.cat(dep_l).to(dev)
     tk = torch.cat(tok_l).to(dev)
     hs = torch.cat(hash_l)
@@ -292,7 +293,7 @@ def make_target_logits(wl: Workload, seed: int, U_full: torch.Tensor, A: torch.T
         noise = torch.empty(e - s, wl.V, dtype=torch.float64, device=dev)
         for i in range(s, e):
             h = int(hs[i]) & 0xFFFFFFFFFFFFFFFF
-            tag = (h ^ (int(req[i]) * 0x9E3779B97F4A7C15)) & 0xFFFFFFFFFFFFFFFF
+            tag = (h ^ (int(req_c[i]) * 0x9E3779B97F4A7C15)) & 0xFFFFFFFFFFFFFFFF
             noise[i - s] = normals(seed, STREAM_Z, tag, wl.V, dev)
         Z[s:e] = (base.to(torch.float64) + bias.to(torch.float64) + sigma * noise).to(wl.torch_dtype)
     return Z, off.to(dev)

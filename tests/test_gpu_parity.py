@@ -1,0 +1,210 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle on the same seeded bytes."""
+import dataclasses
+import math
+
+import numpy as np
+import pytest
+import torch
+from scipy.stats import chisquare
+
+import oracle
+from gpu_harness import (ATOL, RTOL, Round, check_round, close, make_gpu, make_oracle, to_cpu)
+from helpers import np_softmax, path_row, tiny_problem, tiny_z_path
+from paper_2609_22098_b200 import synth
+from paper_2609_22098_b200.binding import TreeSpark
+
+pytestmark = pytest.mark.gpu
+
+
+def small(name, **kw):
+    return dataclasses.replace(synth.WORKLOADS[name], **kw)
+
+
+# ---------------------------------------------------------------------------------------------
+# ts_score_parents
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V,r,K", [(1000, 7, 4), (1003, 16, 8), (4096 + 40, 64, 8), (70000, 32, 16), (8, 4, 4), (5, 3, 8)])
+@pytest.mark.parametrize("T", [0.0, 0.7, 1.0])
+def test_score_parents_matches_oracle(dtype, V, r, K, T):
+    wl = small("tiny", V=V, r=r, K=K, D=3, Nmax=16, dtype=dtype, B=3, calib_mode=0)
+    rnd = Round(wl, seed=11 + V)
+    ts = make_gpu(wl, None, max_batch=3)
+    orc = make_oracle(wl, None)
+    P = 11
+    g = torch.Generator().manual_seed(V)
+    req = torch.randint(0, 3, (P,), generator=g, dtype=torch.int32)
+    dep = torch.randint(0, 3, (P,), generator=g, dtype=torch.int32)
+    tok = torch.randint(0, V, (P,), generator=g, dtype=torch.int32)
+    hsh = torch.randint(0, 2 ** 62, (P,), generator=g, dtype=torch.int64)
+    out = to_cpu(ts.score_parents(rnd.U, rnd.A, rnd.W, req.cuda(), dep.cuda(), tok.cuda(), hsh.cuda(), T, seed=99))
+    torch.cuda.synchronize()
+    c = rnd.cpu()
+    Keff = min(K, V)
+    checked = 0
+    for i in range(P):
+        o = orc.score_parent(c["U"][req[i], dep[i]], c["A"][tok[i]], c["W"], T, 99, int(req[i]), int(hsh[i]))
+        assert close(out["lse0"][i], o["lse0"]), (i, float(out["lse0"][i]), o["lse0"])
+        assert close(out["lseT"][i], o["lseT"]), (i, float(out["lseT"][i]), o["lseT"])
+        if o["margins"][0] >= 2e-5:
+            assert out["top_tok"][i, :Keff].tolist() == o["top_tok"][:Keff].tolist()
+            assert all(close(out["top_logit"][i, j], o["top_logit"][j]) for j in range(Keff))
+            checked += 1
+        if o["margins"][1] >= 2e-5:
+            assert out["draw_tok"][i, :Keff].tolist() == o["draw_tok"][:Keff].tolist(), (i, out["draw_tok"][i], o["draw_tok"])
+            assert all(close(out["draw_logit"][i, j], o["draw_logit"][j]) for j in range(Keff))
+        if K > V:
+            assert (out["top_tok"][i, V:] == -1).all() and (out["draw_tok"][i, V:] == -1).all()
+    assert checked >= P - 2
+
+
+# ---------------------------------------------------------------------------------------------
+# full rounds on scaled-down workloads (several tiles, ragged tails, ragged trees)
+# ---------------------------------------------------------------------------------------------
+CASES = [
+    # name, overrides, temperatures, thetas
+    ("tiny", dict(), (0.0, 1.0), (0.05,)),
+    ("tiny", dict(V=3001, Nmax=40, K=3, D=5), (0.0, 0.8), (0.0, 0.02)),
+    ("decode", dict(V=9000 + 24, r=64, B=3), (0.0, 0.7, 1.0), (0.3, 0.1, 0.03)),
+    ("serve32", dict(V=20000, B=9), (1.0,), (0.1, 0.0, 1.0)),
+    ("wide", dict(V=6000 + 8, B=2, Nmax=256, K=16, D=16, r=128), (0.7, 1.3), (0.01,)),
+    ("wide", dict(V=700, B=2, Nmax=70, K=5, D=3, r=9, dtype="f32"), (1.3,), (0.0,)),
+]
+
+
+@pytest.mark.parametrize("name,over,temps,thetas", CASES)
+def test_round_matches_oracle(name, over, temps, thetas):
+    wl = small(name, **over)
+    rnd = Round(wl, seed=1234)
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
+    orc = make_oracle(wl, rnd.table)
+    tot = dict(trees=0, trees_exempt=0, walks=0, walks_exempt=0, nodes=0)
+    for T in temps:
+        for th in thetas:
+            rnd.theta.fill_(th)
+            for rs in range(3):
+                st = check_round(ts, orc, rnd, T, round_seed=1000 + rs)
+                for k in tot:
+                    tot[k] += st[k]
+    assert tot["trees_exempt"] <= 0.1 * tot["trees"] + 1
+    assert tot["walks_exempt"] <= 0.3 * tot["walks"] + 1
+    assert tot["nodes"] > 0
+
+
+def test_tiny_reference_config_100_rounds():
+    """The tiny all-fp32 reference configuration at full size: 100 rounds at T = 0 and T = 1."""
+    wl = synth.WORKLOADS["tiny"]
+    rnd = Round(wl, seed=7)
+    ts = make_gpu(wl, rnd.table, max_batch=1)
+    orc = make_oracle(wl, rnd.table)
+    for T in wl.temps:
+        tot = dict(trees=0, trees_exempt=0, walks=0, walks_exempt=0, nodes=0)
+        for rs in range(100):
+            st = check_round(ts, orc, rnd, T, round_seed=5000 + rs, want_edge=(rs % 10 == 0))
+            for k in tot:
+                tot[k] += st[k]
+        assert tot["trees_exempt"] <= 5 and tot["walks_exempt"] <= 10, tot
+        assert tot["nodes"] >= 100
+
+
+def test_chain_sentinel_and_mixed_prices():
+    wl = small("serve32", V=5000, B=6)
+    rnd = Round(wl, seed=21)
+    rnd.theta.copy_(torch.tensor([1.0, 0.1, 2.0, 0.0, 0.5, 1.0]))
+    ts = make_gpu(wl, rnd.table, max_batch=6)
+    orc = make_oracle(wl, rnd.table)
+    check_round(ts, orc, rnd, 1.0, 77)
+    tree = to_cpu(ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, 0.0, 78))
+    for b in (0, 2, 5):
+        assert int(tree["n_nodes"][b]) == wl.D
+        assert tree["depth"][b, :wl.D].tolist() == list(range(1, wl.D + 1))
+        assert tree["parent"][b, :wl.D].tolist() == list(range(-1, wl.D - 1))
+    assert int(tree["n_nodes"][3]) == wl.Nmax
+
+
+def test_argument_validation_returns_errors_without_launching():
+    from paper_2609_22098_b200.binding import TreeSparkError
+    wl = small("tiny", V=512)
+    rnd = Round(wl, seed=3)
+    ts = make_gpu(wl, rnd.table, max_batch=1)
+    with pytest.raises(TreeSparkError):
+        ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, -1.0, 1)
+    with pytest.raises(TreeSparkError):
+        ts.expand_tree(rnd.U.view(-1)[1:], rnd.A, rnd.W, rnd.anchor, rnd.theta, 1.0, 1)   # misaligned
+    with pytest.raises(TreeSparkError):
+        TreeSpark(512, 4, 16, 32, 16, 1)                                                   # K > 16
+    small_ws = ts.ws_bytes
+    ts.ws_bytes = 1024
+    with pytest.raises(TreeSparkError):
+        ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, 1.0, 1)
+    ts.ws_bytes = small_ws
+    bad = rnd.anchor.clone(); bad[0] = wl.V + 5
+    tree = to_cpu(ts.expand_tree(rnd.U, rnd.A, rnd.W, bad, rnd.theta, 1.0, 1))
+    assert int(tree["status"][0]) == -1 and int(tree["n_nodes"][0]) == 0
+
+
+# ---------------------------------------------------------------------------------------------
+# losslessness on the GPU path itself (Proposition 1), tiny vocabulary, many requests per call
+# ---------------------------------------------------------------------------------------------
+def test_gpu_losslessness_chi_square():
+    V, D, r, K, N, T, theta = 8, 3, 4, 4, 12, 1.0, 0.05
+    U, A, W = tiny_problem(60, V, D, r, u_std=1.5)
+    Zp = tiny_z_path(61, U, A, W, D, sigma=1.0, anchor=3)
+    B = 4096
+    ts = TreeSpark(V, D, r, K, N, B, dtype=torch.float32)
+    Ud = torch.from_numpy(U[:D]).cuda().unsqueeze(0).expand(B, D, V).contiguous()
+    Ad, Wd = torch.from_numpy(A).cuda(), torch.from_numpy(W).cuda()
+    Zpd = torch.from_numpy(Zp).cuda()
+    anchor = torch.full((B,), 3, dtype=torch.int32, device="cuda")
+    th = torch.full((B,), theta, dtype=torch.float32, device="cuda")
+    off_len = torch.tensor([sum(V ** k for k in range(d)) for d in range(D + 1)], device="cuda")
+    h1 = torch.zeros(V, dtype=torch.int64, device="cuda")
+    h2 = torch.zeros(V, V, dtype=torch.int64, device="cuda")
+    calls = 64
+    for c in range(calls):
+        tree = ts.expand_tree(Ud, Ad, Wd, anchor, th, T, seed=900 + c)
+        n = tree["n_nodes"].long()
+        # path index of every node: fold tokens along parent pointers (depth <= 3)
+        tok, par, dep = tree["tok"].long(), tree["parent"].long(), tree["depth"].long()
+        idx = tok.clone()
+        mult = torch.full_like(idx, V)
+        cur = par.clone()
+        for _ in range(D - 1):
+            has = cur >= 0
+            ptok = torch.gather(tok, 1, cur.clamp(min=0))
+            idx = torch.where(has, idx + ptok * mult, idx)
+            mult = torch.where(has, mult * V, mult)
+            cur = torch.where(has, torch.gather(par, 1, cur.clamp(min=0)), cur)
+        prow = off_len[dep.clamp(0, D)] + idx
+        rows = []
+        offs = torch.zeros(B + 1, dtype=torch.int64, device="cuda")
+        offs[1:] = torch.cumsum(n + 1, 0)
+        total = int(offs[-1])
+        Z = torch.empty(total, V, device="cuda")
+        Z[offs[:-1]] = Zpd[0]
+        ar = torch.arange(N, device="cuda").unsqueeze(0).expand(B, N)
+        valid = ar < n.unsqueeze(1)
+        dst = (offs[:-1].unsqueeze(1) + 1 + ar)[valid]
+        Z[dst] = Zpd[prow[valid]]
+        v = ts.verify_tree(Ud, Ad, Wd, Z, offs, anchor, tree, T, seed=900 + c, edge_stat=False)
+        assert int(v["status"].abs().max()) == 0
+        L = v["acc_len"].long()
+        first = torch.where(L >= 1, v["acc_tok"][:, 0].long(), v["bonus_tok"].long())
+        h1 += torch.bincount(first, minlength=V)
+        second = torch.where(L >= 2, v["acc_tok"][:, 1].long(), v["bonus_tok"].long())
+        sel = L >= 1
+        h2 += torch.bincount(first[sel] * V + second[sel], minlength=V * V).reshape(V, V)
+    trials = B * calls
+    h1 = h1.cpu().numpy(); h2 = h2.cpu().numpy()
+    p_root = np_softmax(Zp[0].astype(np.float64), T)
+    assert h1.sum() == trials
+    assert chisquare(h1, p_root * trials).pvalue > 1e-3
+    checked = 0
+    for x1 in range(V):
+        nrow = int(h2[x1].sum())
+        if nrow < 5000:
+            continue
+        p2 = np_softmax(Zp[path_row((x1,), V)].astype(np.float64), T)
+        assert chisquare(h2[x1], p2 * nrow).pvalue > 1e-4
+        checked += 1
+    assert checked >= 2
