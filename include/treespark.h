@@ -155,6 +155,20 @@ int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, const void* W,
                        float* edge_stat, uint32_t* flags, int32_t* status,
                        void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * Instrumentation (no counterpart in the paper): per-kernel device times and launch counts.
+ * ts_profile_enable(capacity > 0) creates `capacity` CUDA event pairs and from then on every kernel
+ * the hot calls launch is bracketed by an event pair on the caller's stream until the pairs run out;
+ * capacity == 0 switches it off and frees the events.  Launches are always counted.
+ * ts_profile_read waits for the recorded events (a host synchronisation: never call it inside a
+ * timed region), adds up the elapsed milliseconds and launch counts per kernel id into ms[0..n) and
+ * launches[0..n) (HOST arrays; ids >= n are dropped) and, when reset != 0, clears both.
+ * ts_kernel_name gives the name of a kernel id, NULL past the last one.
+ */
+int32_t ts_profile_enable(ts_ctx* ctx, int32_t capacity);
+int32_t ts_profile_read(ts_ctx* ctx, int32_t n, double* ms, int64_t* launches, int32_t reset);
+const char* ts_kernel_name(int32_t id);
+
 #ifdef __cplusplus
 }
 #endif

@@ -29,6 +29,7 @@ FLAG_NEAR_ACCEPT = 8
 FLAG_NEAR_CDF = 16
 FLAG_SATURATED = 32
 FLAG_ZERO_MASS = 64
+TOPK_MARGIN = 4e-6
 
 
 def build(force: bool = False) -> str:
@@ -111,14 +112,15 @@ class Oracle:
         lse0, lseT = C.c_double(), C.c_double()
         top_tok = np.empty(K, np.int32); top_logit = np.empty(K, np.float64)
         draw_tok = np.empty(K, np.int32); draw_logit = np.empty(K, np.float64)
-        draw_key = np.empty(K, np.float64); margins = np.empty(2, np.float64)
+        draw_key = np.empty(K, np.float64); margins = np.empty(2 * K, np.float64)
         lib().orc_score_parent(C.byref(self.cfg), _p(U_row, C.c_float), _p(a_row, C.c_float), _p(W, C.c_float),
                                C.c_double(T), C.c_uint64(seed), C.c_int32(req), C.c_uint64(node_hash),
                                C.byref(lse0), C.byref(lseT), _p(top_tok, C.c_int32), _p(top_logit, C.c_double),
                                _p(draw_tok, C.c_int32), _p(draw_logit, C.c_double), _p(draw_key, C.c_double),
                                _p(margins, C.c_double))
         return dict(lse0=lse0.value, lseT=lseT.value, top_tok=top_tok, top_logit=top_logit,
-                    draw_tok=draw_tok, draw_logit=draw_logit, draw_key=draw_key, margins=margins)
+                    draw_tok=draw_tok, draw_logit=draw_logit, draw_key=draw_key,
+                    margins=np.array([margins[:K].min(), margins[K:].min()]), gaps=margins)
 
     # -- expansion -------------------------------------------------------------------------
     def expand_tree(self, U_req, A, W, anchor_tok, theta, T, seed, req):

@@ -144,18 +144,17 @@ static void select_top(const double* val, int V, int K, int32_t* out_idx, double
   free(taken);
 }
 
-static double min_rel_gap(const double* val, const int32_t* idx, int K, double next) {
-  double g = INFINITY;
+/* gap[j] = (value of pick j - value of pick j+1) / max(1, |value of pick j|); pick K is `next` */
+static void rel_gaps(const double* val, const int32_t* idx, int K, double next, double* gap) {
   for (int j = 0; j < K; ++j) {
-    if (idx[j] < 0) break;
+    gap[j] = INFINITY;
+    if (idx[j] < 0) continue;
     double a = val[idx[j]];
     double b = (j + 1 < K) ? (idx[j + 1] >= 0 ? val[idx[j + 1]] : -INFINITY) : next;
-    if (!(b > -INFINITY)) break;
+    if (!(b > -INFINITY)) continue;
     double scale = fabs(a) > 1.0 ? fabs(a) : 1.0;
-    double gap = (a - b) / scale;
-    if (gap < g) g = gap;
+    gap[j] = (a - b) / scale;
   }
-  return g;
 }
 
 void orc_score_parent(const orc_config* cfg, const float* U_row, const float* a_row, const float* W,
@@ -182,7 +181,10 @@ void orc_score_parent(const orc_config* cfg, const float* U_row, const float* a_
   double next = -INFINITY;
   select_top(l, V, K, top_tok, &next);
   for (int j = 0; j < K; ++j) top_logit[j] = l[top_tok[j]];
-  if (margins) { margins[0] = min_rel_gap(l, top_tok, K, next); margins[1] = INFINITY; }
+  if (margins) {
+    for (int j = 0; j < 2 * cfg->K; ++j) margins[j] = INFINITY;
+    rel_gaps(l, top_tok, K, next, margins);
+  }
   if (T > 0.0) {
     /* j-th without-replacement draw = j-th largest of l/T + Gumbel noise (equal in law to Eq. 2) */
     double* key = (double*)malloc(sizeof(double) * (size_t)V);
@@ -192,7 +194,7 @@ void orc_score_parent(const orc_config* cfg, const float* U_row, const float* a_
     }
     select_top(key, V, K, draw_tok, &next);
     for (int j = 0; j < K; ++j) { draw_logit[j] = l[draw_tok[j]]; if (draw_key) draw_key[j] = key[draw_tok[j]]; }
-    if (margins) margins[1] = min_rel_gap(key, draw_tok, K, next);
+    if (margins) rel_gaps(key, draw_tok, K, next, margins + cfg->K);
     free(key);
   } else {
     for (int j = 0; j < K; ++j) { draw_tok[j] = top_tok[j]; draw_logit[j] = top_logit[j]; if (draw_key) draw_key[j] = top_logit[j]; }
@@ -214,6 +216,7 @@ typedef struct {
   double lse0, lseT;
   int32_t top_tok[ORC_KMAX], draw_tok[ORC_KMAX];
   double top_logit[ORC_KMAX], draw_logit[ORC_KMAX];
+  double gap_top[ORC_KMAX], gap_key[ORC_KMAX];
 } node_t;
 
 typedef struct {
@@ -273,12 +276,15 @@ typedef struct {
 
 static void score_node(expand_ctx* c, node_t* nd) {
   const orc_config* cfg = c->cfg;
-  double margins[2];
+  double margins[2 * ORC_KMAX];
   double top_logit[ORC_KMAX], draw_logit[ORC_KMAX];
   orc_score_parent(cfg, c->U_req + (size_t)nd->depth * cfg->V, c->A + (size_t)nd->tok * cfg->r, c->W,
                    c->force_topk ? 0.0 : c->T, c->seed, c->req, nd->hash,
                    &nd->lse0, &nd->lseT, nd->top_tok, top_logit, nd->draw_tok, draw_logit, NULL, margins);
-  for (int j = 0; j < cfg->K; ++j) { nd->top_logit[j] = top_logit[j]; nd->draw_logit[j] = draw_logit[j]; }
+  for (int j = 0; j < cfg->K; ++j) {
+    nd->top_logit[j] = top_logit[j]; nd->draw_logit[j] = draw_logit[j];
+    nd->gap_top[j] = margins[j]; nd->gap_key[j] = margins[cfg->K + j];
+  }
   if (c->force_topk && c->T > 0.0) {
     /* biased control: children are the modes, but the proposal is still q_T */
     double* l = (double*)malloc(sizeof(double) * (size_t)cfg->V);
@@ -290,7 +296,6 @@ static void score_node(expand_ctx* c, node_t* nd) {
     nd->lseT = m / c->T + log(sT);
     free(l);
   }
-  if (margins[0] < 2e-5 || margins[1] < 2e-5) c->flags |= ORC_FLAG_NEAR_TOPK;
   nd->scored = 1;
   c->n_scored++;
 }
@@ -393,10 +398,22 @@ static int32_t expand_impl(const orc_config* cfg, const float* U_req, const floa
       heap_push(nodes, heap, &heap_n, sv);
     }
   }
+  /* a near-tie among a parent's candidates matters only where it decides which token becomes, or
+   * in what order tokens become, one of its materialised children */
+  for (int i = 0; i <= n; ++i) {
+    const node_t* nd = &nodes[i];
+    if (!nd->scored) continue;
+    const double* gap = (T == 0.0 || force_topk) ? nd->gap_top : nd->gap_key;
+    for (int j = 0; j < nd->nchild && j < cfg->K; ++j)
+      if (gap[j] < ORC_TOPK_MARGIN) c.flags |= ORC_FLAG_NEAR_TOPK;
+  }
   if (n == c.N_eff && heap_n > 0) {
     double rest = heap[0].logkey;
     double scale = fabs(rest) > 1.0 ? fabs(rest) : 1.0;
-    if (rest >= c.theta_log && (last_admitted - rest) < 1e-4 * scale) c.flags |= ORC_FLAG_NEAR_CAP;
+    /* bitwise-equal keys come from one parent's unchanged "best unused token" bound (sibling slots
+     * at T>0); the (depth, rank path) order settles those identically in any arithmetic */
+    if (rest >= c.theta_log && last_admitted != rest && (last_admitted - rest) < 1e-4 * scale)
+      c.flags |= ORC_FLAG_NEAR_CAP;
   }
 
   /* canonical order: depth ascending, then the parent's canonical index, then sibling rank */

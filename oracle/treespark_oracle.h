@@ -27,9 +27,10 @@ extern "C" {
 #define ORC_KMAX 16
 #define ORC_DMAX 16
 #define ORC_CALIB_KNOTS 16
+#define ORC_TOPK_MARGIN 4e-6  /* relative gap below which two candidates count as a near-tie */
 
 /* flag bits (per request) */
-#define ORC_FLAG_NEAR_TOPK   1u   /* near-tie among the top-(K+1) logits or sampling keys of a scored parent */
+#define ORC_FLAG_NEAR_TOPK   1u   /* near-tie among candidates that decided a materialised child or its rank */
 #define ORC_FLAG_NEAR_THETA  2u   /* a slot key within 1e-4 (log) of the stop price */
 #define ORC_FLAG_NEAR_CAP    4u   /* last admitted and first excluded key within 1e-4 (log) at the node cap */
 #define ORC_FLAG_NEAR_ACCEPT 8u   /* an accept test with |u - rho| below the accept margin */
@@ -65,8 +66,8 @@ double orc_logit_q0(const double* l, int32_t V, int32_t x, double m, double s0);
 
 /* Score one parent.  top_*: K best logits (value desc, ties lowest token).  draw_*: at T>0 the K
  * without-replacement draws in draw order (largest perturbed keys), at T==0 a copy of top_*.
- * margins (optional, may be NULL): [0] = smallest gap among consecutive top-(K+1) logits relative to
- * max(1,|l|), [1] = same for the sampling keys. */
+ * margins (optional, may be NULL), 2K doubles: [j] = gap between the j-th and (j+1)-th largest logit
+ * relative to max(1,|l|) (the (K+1)-th included), [K+j] = the same for the sampling keys. */
 void orc_score_parent(const orc_config* cfg, const float* U_row, const float* a_row, const float* W,
                       double T, uint64_t seed, int32_t req, uint64_t hash,
                       double* lse0, double* lseT, int32_t* top_tok, double* top_logit,

@@ -20,7 +20,8 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 KNOTS = 16
 
 EXPORTS = ("ts_create", "ts_destroy", "ts_workspace_bytes", "ts_last_error_string",
-           "ts_score_parents", "ts_expand_tree", "ts_verify_tree")
+           "ts_score_parents", "ts_expand_tree", "ts_verify_tree",
+           "ts_profile_enable", "ts_profile_read", "ts_kernel_name")
 
 
 class TsConfig(C.Structure):
@@ -50,7 +51,12 @@ def load_library() -> C.CDLL:
         L.ts_score_parents.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, f32, u64] + [vp] * 6 + [vp, sz, vp]
         L.ts_expand_tree.argtypes = [vp, vp, vp, vp, i32, vp, vp, f32, u64] + [vp] * 15 + [vp, sz, vp]
         L.ts_verify_tree.argtypes = [vp, vp, vp, vp, vp, vp, i32] + [vp] * 9 + [f32, u64] + [vp] * 7 + [vp, sz, vp]
-        for n in ("ts_create", "ts_destroy", "ts_score_parents", "ts_expand_tree", "ts_verify_tree"):
+        L.ts_profile_enable.argtypes = [vp, i32]
+        L.ts_profile_read.argtypes = [vp, i32, vp, vp, i32]
+        L.ts_kernel_name.argtypes = [i32]
+        L.ts_kernel_name.restype = C.c_char_p
+        for n in ("ts_create", "ts_destroy", "ts_score_parents", "ts_expand_tree", "ts_verify_tree",
+                  "ts_profile_enable", "ts_profile_read"):
             getattr(L, n).restype = C.c_int32
         _lib = L
     return _lib
@@ -106,6 +112,20 @@ class TreeSpark:
     def _check(self, code: int):
         if code != TS_OK:
             raise TreeSparkError(f"status {code}: {self.lib.ts_last_error_string().decode()}")
+
+    # -- instrumentation ---------------------------------------------------------------------------
+    def profile_enable(self, capacity: int):
+        self._check(self.lib.ts_profile_enable(self._ctx, int(capacity)))
+
+    def profile_read(self, reset: bool = True):
+        """{kernel name: (milliseconds, launches)} since the last reset; synchronises with the device."""
+        n = 0
+        while self.lib.ts_kernel_name(n) is not None:
+            n += 1
+        ms = (C.c_double * n)()
+        cnt = (C.c_int64 * n)()
+        self._check(self.lib.ts_profile_read(self._ctx, n, ms, cnt, 1 if reset else 0))
+        return {self.lib.ts_kernel_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n)}
 
     # -- output buffers (caller-owned; allocate once, reuse across rounds) -------------------------
     def alloc_score_outputs(self, P: int) -> Dict[str, torch.Tensor]:

@@ -71,14 +71,15 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
   ctx->cfg = *cfg;
   ctx->cfg.calib_table = nullptr;
   ctx->d_table = nullptr;
+  ctx->prof = new Prof();
   cudaError_t e = cudaGetDevice(&ctx->device);
   cudaDeviceProp prop;
   if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, ctx->device);
-  if (e != cudaSuccess) { delete ctx; return set_cuda_error("ts_create", e); }
+  if (e != cudaSuccess) { delete (Prof*)ctx->prof; delete ctx; return set_cuda_error("ts_create", e); }
   ctx->num_sms = prop.multiProcessorCount;
   ctx->max_smem = (int)prop.sharedMemPerBlockOptin;
   if (!choose_tile(ctx->cfg, ctx->num_sms, ctx->max_smem, &ctx->tile)) {
-    delete ctx;
+    delete (Prof*)ctx->prof; delete ctx;
     return set_error(TS_ERR_UNSUPPORTED, "ts_create: no vocabulary tiling fits shared memory");
   }
   ctx->vt_TV = ((cfg->V + ctx->num_sms - 1) / ctx->num_sms + 63) / 64 * 64;
@@ -87,7 +88,7 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
     const size_t bytes = (size_t)cfg->D * TS_CALIB_KNOTS * sizeof(float);
     e = cudaMalloc(&ctx->d_table, bytes);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->d_table, cfg->calib_table, bytes, cudaMemcpyHostToDevice);
-    if (e != cudaSuccess) { cudaFree(ctx->d_table); delete ctx; return set_cuda_error("ts_create", e); }
+    if (e != cudaSuccess) { cudaFree(ctx->d_table); delete (Prof*)ctx->prof; delete ctx; return set_cuda_error("ts_create", e); }
   }
   ctx->calib.mode = cfg->calib_mode;
   ctx->calib.a = cfg->platt_a; ctx->calib.b = cfg->platt_b;
@@ -95,7 +96,7 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
   ctx->calib.table = ctx->d_table;
   e = score_setup(ctx);
   if (e == cudaSuccess) e = verify_setup(ctx);
-  if (e != cudaSuccess) { cudaFree(ctx->d_table); delete ctx; return set_cuda_error("ts_create", e); }
+  if (e != cudaSuccess) { cudaFree(ctx->d_table); delete (Prof*)ctx->prof; delete ctx; return set_cuda_error("ts_create", e); }
   *out = ctx;
   return TS_OK;
 }
@@ -103,6 +104,8 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
 extern "C" int32_t ts_destroy(ts_ctx* ctx) {
   if (!ctx) return TS_OK;
   if (ctx->d_table) cudaFree(ctx->d_table);
+  Prof* p = (Prof*)ctx->prof;
+  if (p) { for (cudaEvent_t e : p->ev) cudaEventDestroy(e); delete p; }
   delete ctx;
   return TS_OK;
 }
@@ -110,4 +113,40 @@ extern "C" int32_t ts_destroy(ts_ctx* ctx) {
 extern "C" size_t ts_workspace_bytes(const ts_ctx* ctx, int32_t batch) {
   if (!ctx || batch < 1 || batch > ctx->cfg.max_batch) return 0;
   return make_layout(ctx, batch).total;
+}
+
+static const char* kKernelNames[K_COUNT] = {"expand_init", "score_tile", "score_merge", "expand_level", "expand_finalize",
+                                            "zrow_stats", "verify_greedy", "verify_walk", "verify_check"};
+
+extern "C" const char* ts_kernel_name(int32_t id) { return (id >= 0 && id < K_COUNT) ? kKernelNames[id] : nullptr; }
+
+extern "C" int32_t ts_profile_enable(ts_ctx* ctx, int32_t capacity) {
+  if (!ctx || capacity < 0) return set_error(TS_ERR_INVALID, "ts_profile_enable: bad argument");
+  Prof* p = (Prof*)ctx->prof;
+  for (cudaEvent_t e : p->ev) cudaEventDestroy(e);
+  p->ev.clear(); p->ids.clear(); p->used = 0; p->on = false;
+  for (int i = 0; i < 2 * capacity; ++i) {
+    cudaEvent_t e;
+    cudaError_t err = cudaEventCreate(&e);
+    if (err != cudaSuccess) return set_cuda_error("ts_profile_enable", err);
+    p->ev.push_back(e);
+  }
+  p->ids.assign((size_t)capacity, 0);
+  p->on = capacity > 0;
+  return TS_OK;
+}
+
+extern "C" int32_t ts_profile_read(ts_ctx* ctx, int32_t n, double* ms, int64_t* launches, int32_t reset) {
+  if (!ctx || n < 0 || (n > 0 && (!ms || !launches))) return set_error(TS_ERR_INVALID, "ts_profile_read: bad argument");
+  Prof* p = (Prof*)ctx->prof;
+  for (int i = 0; i < n; ++i) { ms[i] = 0.0; launches[i] = i < K_COUNT ? p->launches[i] : 0; }
+  for (size_t s = 0; s < p->used; ++s) {
+    cudaError_t err = cudaEventSynchronize(p->ev[2 * s + 1]);
+    float t = 0.f;
+    if (err == cudaSuccess) err = cudaEventElapsedTime(&t, p->ev[2 * s], p->ev[2 * s + 1]);
+    if (err != cudaSuccess) return set_cuda_error("ts_profile_read", err);
+    if (p->ids[s] < n) ms[p->ids[s]] += t;
+  }
+  if (reset) { p->used = 0; for (int i = 0; i < K_COUNT; ++i) p->launches[i] = 0; }
+  return TS_OK;
 }

@@ -44,6 +44,7 @@ struct ts_ctx {
   ts::TileCfg tile;
   int vt_TV, vt_n;  // vocabulary ranges of the verification walk, one per CTA
   ts::DevCalib calib;
+  void* prof;  // ts::Prof*, instrumentation state
 };
 
 namespace ts {

@@ -332,7 +332,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   a.cd_q0 = (float*)(ws + L.cd_q0); a.cd_logqT = (float*)(ws + L.cd_logqT); a.cd_rank = (int*)(ws + L.cd_rank);
   a.status = status;
 
-  expand_init_kernel<<<B, 64, 0, st>>>(a);
+  { ProfScope ps(ctx, K_INIT, st); expand_init_kernel<<<B, 64, 0, st>>>(a); }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(init)", e);
   const size_t level_smem = (size_t)(c.Nmax + c.Nmax * c.K) * sizeof(Entry);
@@ -346,7 +346,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
                      a.lst_hash[cur], T, seed, res_lse0, res_lseT, res_top_tok, res_top_logit, res_draw_tok,
                      res_draw_logit, st);
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(score)", e);
-    expand_level_kernel<<<B, 256, level_smem, st>>>(a, d);
+    { ProfScope ps(ctx, K_LEVEL, st); expand_level_kernel<<<B, 256, level_smem, st>>>(a, d); }
     e = cudaGetLastError();
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(level)", e);
   }
@@ -358,7 +358,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   f.n_nodes = n_nodes; f.tok = tok; f.parent = parent; f.depth = depth; f.sib_rank = sib_rank; f.logS = logS; f.q0 = q0;
   f.logqT = logqT; f.logkey = logkey; f.pop_rank = pop_rank; f.node_hash = node_hash; f.node_lseT = node_lseT;
   f.mask = mask; f.n_scored = n_scored;
-  expand_finalize_kernel<<<B, 256, 0, st>>>(f);
+  { ProfScope ps(ctx, K_FINAL, st); expand_finalize_kernel<<<B, 256, 0, st>>>(f); }
   e = cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(finalize)", e);
   return TS_OK;

@@ -119,6 +119,8 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
   const TIn* Ag = reinterpret_cast<const TIn*>(a.A);
   constexpr int VEC = Elem<TIn>::VEC;
   const bool vec_ok = (V % VEC) == 0;
+  const int P = a.P_dev ? *a.P_dev : a.P;
+  if (P <= 0) return;  // an empty level: nothing to stage
 
   // stage the W tile
   if (vec_ok) {
@@ -143,7 +145,6 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
   }
   __syncthreads();
 
-  const int P = a.P_dev ? *a.P_dev : a.P;
   const float T = a.T, invT = T > 0.f ? 1.f / T : 1.f;
   const int K = a.K;
 
@@ -287,10 +288,13 @@ cudaError_t launch_score(const ts_ctx* ctx, const WsLayout& L, char* ws, const v
   a.part_m = (float*)(ws + L.part_m); a.part_s0 = (float*)(ws + L.part_s0); a.part_sT = (float*)(ws + L.part_sT);
   a.part_topv = (float*)(ws + L.part_topv); a.part_topi = (int*)(ws + L.part_topi);
   a.part_keyv = (float*)(ws + L.part_keyv); a.part_keyi = (int*)(ws + L.part_keyi); a.part_keyl = (float*)(ws + L.part_keyl);
-  if (c.dt_U == TS_DTYPE_BF16)
-    score_tile_kernel<__nv_bfloat16><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
-  else
-    score_tile_kernel<float><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
+  {
+    ProfScope ps(ctx, K_SCORE, st);
+    if (c.dt_U == TS_DTYPE_BF16)
+      score_tile_kernel<__nv_bfloat16><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
+    else
+      score_tile_kernel<float><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   MergeArgs m{};
@@ -302,7 +306,10 @@ cudaError_t launch_score(const ts_ctx* ctx, const WsLayout& L, char* ws, const v
   int blocks = (pmax + 7) / 8;
   if (blocks > 4 * ctx->num_sms) blocks = 4 * ctx->num_sms;
   if (blocks < 1) blocks = 1;
-  merge_kernel<<<blocks, 256, 0, st>>>(m);
+  {
+    ProfScope ps(ctx, K_MERGE, st);
+    merge_kernel<<<blocks, 256, 0, st>>>(m);
+  }
   return cudaGetLastError();
 }
 

@@ -533,14 +533,17 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
 
   const int max_rows = B * (c.Nmax + 1);
   int grid_rows = max_rows < 8 * ctx->num_sms ? max_rows : 8 * ctx->num_sms;
-  if (c.dt_Z == TS_DTYPE_BF16)
-    zrow_stats_kernel<__nv_bfloat16><<<grid_rows, VT, 0, st>>>((const __nv_bfloat16*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
-  else
-    zrow_stats_kernel<float><<<grid_rows, VT, 0, st>>>((const float*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+  {
+    ProfScope ps(ctx, K_ZROWS, st);
+    if (c.dt_Z == TS_DTYPE_BF16)
+      zrow_stats_kernel<__nv_bfloat16><<<grid_rows, VT, 0, st>>>((const __nv_bfloat16*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+    else
+      zrow_stats_kernel<float><<<grid_rows, VT, 0, st>>>((const float*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(rows)", e);
   if (T == 0.f) {
-    verify_greedy_kernel<<<B, 128, 0, st>>>(a);
+    { ProfScope ps(ctx, K_GREEDY, st); verify_greedy_kernel<<<B, 128, 0, st>>>(a); }
     e = cudaGetLastError();
     if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(greedy)", e);
     return TS_OK;
@@ -549,9 +552,9 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(memset)", e);
   void* kargs[] = {(void*)&a};
   const void* fn = c.dt_Z == TS_DTYPE_BF16 ? (const void*)verify_walk_kernel<__nv_bfloat16> : (const void*)verify_walk_kernel<float>;
-  e = cudaLaunchCooperativeKernel(fn, dim3(a.vt_n), dim3(VT), kargs, 0, st);
+  { ProfScope ps(ctx, K_WALK, st); e = cudaLaunchCooperativeKernel(fn, dim3(a.vt_n), dim3(VT), kargs, 0, st); }
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(walk)", e);
-  verify_check_kernel<<<(B + 127) / 128, 128, 0, st>>>(a);
+  { ProfScope ps(ctx, K_CHECK, st); verify_check_kernel<<<(B + 127) / 128, 128, 0, st>>>(a); }
   e = cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(check)", e);
   return TS_OK;
