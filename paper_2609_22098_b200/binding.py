@@ -196,3 +196,54 @@ def ts_expand_tree(ctx: TreeSpark, *args, **kw):
 
 def ts_verify_tree(ctx: TreeSpark, *args, **kw):
     return ctx.verify_tree(*args, **kw)
+
+
+class HostRound:
+    """One whole round for callers whose buffers live in host memory.
+
+    ``run`` copies the step's inputs (base logits, anchors, prices, target logits and their row
+    offsets) from pinned host tensors to device staging buffers, runs ts_expand_tree and
+    ts_verify_tree, copies the tree and the verdict back into pinned host tensors and waits for
+    them.  All staging memory is allocated once in the constructor."""
+
+    TREE_OUT = ("n_nodes", "tok", "parent", "depth", "mask")
+    VERDICT_OUT = ("acc_len", "acc_tok", "bonus_tok")
+
+    @staticmethod
+    def pin_inputs(U, anchor, theta, Z, zoff):
+        return {k: t.detach().to("cpu").contiguous().pin_memory()
+                for k, t in dict(U=U, anchor=anchor, theta=theta, Z=Z, zoff=zoff).items()}
+
+    def __init__(self, ts: TreeSpark, B: int, max_rows: int):
+        self.ts, self.B = ts, B
+        d = ts.device
+        self.U = torch.empty(B, ts.D, ts.V, dtype=ts.dtype, device=d)
+        self.anchor = torch.empty(B, dtype=torch.int32, device=d)
+        self.theta = torch.empty(B, dtype=torch.float32, device=d)
+        self.Z = torch.empty(max_rows, ts.V, dtype=ts.dtype, device=d)
+        self.zoff = torch.empty(B + 1, dtype=torch.int64, device=d)
+        self.tree = ts.alloc_tree(B)
+        self.verdict = ts.alloc_verdict(B)
+        self.host_out = {k: torch.empty_like(self.tree[k], device="cpu").pin_memory() for k in self.TREE_OUT}
+        self.host_out.update({k: torch.empty_like(self.verdict[k], device="cpu").pin_memory() for k in self.VERDICT_OUT})
+        self.h2d_bytes = 0
+        self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.host_out.values())
+
+    def run(self, host, A, W, T, seed, edge_stat=True):
+        ts = self.ts
+        rows = host["Z"].shape[0]
+        self.U.copy_(host["U"], non_blocking=True)
+        self.anchor.copy_(host["anchor"], non_blocking=True)
+        self.theta.copy_(host["theta"], non_blocking=True)
+        ts.expand_tree(self.U, A, W, self.anchor, self.theta, T, seed, out=self.tree)
+        self.Z[:rows].copy_(host["Z"], non_blocking=True)
+        self.zoff.copy_(host["zoff"], non_blocking=True)
+        ts.verify_tree(self.U, A, W, self.Z, self.zoff, self.anchor, self.tree, T, seed, out=self.verdict,
+                       edge_stat=edge_stat)
+        for k in self.TREE_OUT:
+            self.host_out[k].copy_(self.tree[k], non_blocking=True)
+        for k in self.VERDICT_OUT:
+            self.host_out[k].copy_(self.verdict[k], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        self.h2d_bytes = sum(host[k].numel() * host[k].element_size() for k in ("U", "anchor", "theta", "Z", "zoff"))
+        return self.host_out
