@@ -99,6 +99,44 @@ int32_t ts_score_parents(ts_ctx* ctx, const void* U, const void* A, const void* 
                          void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * ts_score_parents_static -- ts_score_parents without a caller workspace.  (The paper has no
+ * counterpart; this exists for deployment reasons only.)
+ *
+ * Who needs it: code that must score parents but is in no position to get device memory for the
+ * library -- for example a plugin inside a serving process whose start-up phase has already handed
+ * every free byte of HBM to the KV-cache pool, or a component whose rules forbid cudaMalloc on the
+ * request path because it can stall the whole device.  Such a caller still owns its inputs and
+ * outputs, but has nowhere to put the scratch that ts_score_parents keeps in `ws`.
+ *
+ * What it does instead: the per-tile records the scoring pass writes and the merge pass reads live in
+ * one array of TS_STATIC_SCRATCH_BYTES (8 MiB) that is part of the library's device image.  Every GPU
+ * that loads the library carries that array until the process ends.  The call makes no cudaMalloc,
+ * cudaFree or other allocating call, and the results are the same as ts_score_parents'.
+ *
+ * Limits and rules:
+ *   - The array bounds P: ntiles * (3 + 5K) * 4 bytes are needed per parent (a few hundred parents
+ *     for a 152k vocabulary with K = 8).  A larger P is refused with TS_ERR_WORKSPACE and a message
+ *     that names the limit; nothing is launched.
+ *   - The context's device must be the current device.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
+ *     remembers it; make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the last call left in it.
+ *     Nothing in it needs clearing (each call overwrites all records it later reads), but two calls
+ *     whose kernels overlap on the GPU (different streams, no ordering between them) race on it:
+ *     keep calls on one stream, or order them with events.
+ * Arguments are those of ts_score_parents minus ws / ws_bytes.
+ */
+#define TS_STATIC_SCRATCH_BYTES (8u << 20)
+int32_t ts_score_parents_static(ts_ctx* ctx, const void* U, const void* A, const void* W,
+                                int32_t P, const int32_t* parent_req, const int32_t* parent_depth,
+                                const int32_t* parent_token, const uint64_t* parent_hash,
+                                float T, uint64_t seed,
+                                float* lse0, float* lseT,
+                                int32_t* top_tok, float* top_logit,
+                                int32_t* draw_tok, float* draw_logit,
+                                void* stream);
+
+/*
  * Build the draft trees of B requests (Algorithm 1 with the stop rule of Section 3.5).
  * Slots are admitted in non-increasing order of the candidate survival S(v) * p_hat(best unused
  * token | v) while fewer than Nmax nodes exist and that survival is >= theta[b]; the child token is

@@ -20,7 +20,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 KNOTS = 16
 
 EXPORTS = ("ts_create", "ts_destroy", "ts_workspace_bytes", "ts_last_error_string",
-           "ts_score_parents", "ts_expand_tree", "ts_verify_tree",
+           "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",
            "ts_profile_enable", "ts_profile_read", "ts_kernel_name")
 
 
@@ -49,13 +49,14 @@ def load_library() -> C.CDLL:
         L.ts_destroy.argtypes = [C.c_void_p]
         vp, i32, f32, u64, sz = C.c_void_p, C.c_int32, C.c_float, C.c_uint64, C.c_size_t
         L.ts_score_parents.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, f32, u64] + [vp] * 6 + [vp, sz, vp]
+        L.ts_score_parents_static.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, f32, u64] + [vp] * 6 + [vp]
         L.ts_expand_tree.argtypes = [vp, vp, vp, vp, i32, vp, vp, f32, u64] + [vp] * 15 + [vp, sz, vp]
         L.ts_verify_tree.argtypes = [vp, vp, vp, vp, vp, vp, i32] + [vp] * 9 + [f32, u64] + [vp] * 7 + [vp, sz, vp]
         L.ts_profile_enable.argtypes = [vp, i32]
         L.ts_profile_read.argtypes = [vp, i32, vp, vp, i32]
         L.ts_kernel_name.argtypes = [i32]
         L.ts_kernel_name.restype = C.c_char_p
-        for n in ("ts_create", "ts_destroy", "ts_score_parents", "ts_expand_tree", "ts_verify_tree",
+        for n in ("ts_create", "ts_destroy", "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",
                   "ts_profile_enable", "ts_profile_read"):
             getattr(L, n).restype = C.c_int32
         _lib = L
@@ -158,6 +159,18 @@ class TreeSpark:
                                               float(T), int(seed), _ptr(out["lse0"]), _ptr(out["lseT"]),
                                               _ptr(out["top_tok"]), _ptr(out["top_logit"]), _ptr(out["draw_tok"]),
                                               _ptr(out["draw_logit"]), _ptr(self.ws), self.ws_bytes, _stream()))
+        return out
+
+    def score_parents_static(self, U, A, W, parent_req, parent_depth, parent_token, parent_hash, T, seed, out):
+        """ts_score_parents for callers without a workspace: scratch is the library's built-in 8 MiB
+        device array, so ``out`` must be given (nothing is allocated here either) and the number of
+        parents is bounded; see the header for the sharing rules."""
+        P = int(parent_req.numel())
+        self._check(self.lib.ts_score_parents_static(self._ctx, _ptr(U), _ptr(A), _ptr(W), P, _ptr(parent_req),
+                                                     _ptr(parent_depth), _ptr(parent_token), _ptr(parent_hash),
+                                                     float(T), int(seed), _ptr(out["lse0"]), _ptr(out["lseT"]),
+                                                     _ptr(out["top_tok"]), _ptr(out["top_logit"]),
+                                                     _ptr(out["draw_tok"]), _ptr(out["draw_logit"]), _stream()))
         return out
 
     def expand_tree(self, U, A, W, anchor_tok, theta, T, seed, out=None):
