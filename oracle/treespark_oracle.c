@@ -54,15 +54,17 @@ static void stream_words(uint64_t seed, int32_t req, uint64_t hash, uint32_t str
   orc_philox4x32_10(ctr, key, out);
 }
 
-/* The sampling uniform of token v is a 32-bit fraction: its top byte comes from a stream that
- * yields sixteen tokens per generator call, its low 24 bits from a stream that yields four. */
+/* The sampling uniform of token v is a 32-bit fraction: its high half comes from generator stream 1,
+ * its low half from stream 2; each call of either stream serves eight consecutive tokens (one 16-bit
+ * half-word per token). */
 double orc_u_gumbel(uint64_t seed, int32_t req, uint64_t hash, int32_t v) {
   uint32_t w[4];
-  stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, (uint32_t)v >> 4, w);
-  uint32_t coarse = (w[((uint32_t)v & 15u) >> 2] >> (8u * ((uint32_t)v & 3u))) & 0xFFu;
-  stream_words(seed, req, hash, STREAM_GUMBEL_FINE, (uint32_t)v >> 2, w);
-  uint32_t fine = w[(uint32_t)v & 3u] >> 8;
-  uint32_t x = (coarse << 24) | fine;
+  const uint32_t vv = (uint32_t)v;
+  stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, vv >> 3, w);
+  uint32_t coarse = (w[(vv & 7u) >> 1] >> (16u * (vv & 1u))) & 0xFFFFu;
+  stream_words(seed, req, hash, STREAM_GUMBEL_FINE, vv >> 3, w);
+  uint32_t fine = (w[(vv & 7u) >> 1] >> (16u * (vv & 1u))) & 0xFFFFu;
+  uint32_t x = (coarse << 16) | fine;
   return ((double)x + 0.5) * (1.0 / 4294967296.0);
 }
 

@@ -1,5 +1,6 @@
 // Context management, workspace sizing and error strings of the TreeSpark C ABI.
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "ts_internal.h"
@@ -23,7 +24,7 @@ int32_t set_cuda_error(const char* where, cudaError_t e) {
 // waves over the SMs.
 static bool choose_tile(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
   const size_t es = c.dt_W == TS_DTYPE_BF16 ? 2 : 4;
-  const size_t fixed = (size_t)c.r * SCORE_THREADS * 4 + 256 * 4;
+  const size_t fixed = (size_t)c.r * SCORE_THREADS * 4 + 512 * 4;  // head rows + both noise-bound tables
   const size_t budget = (size_t)max_smem > fixed + 1024 ? (size_t)max_smem - fixed - 1024 : 0;
   int tv_max = (int)(budget / ((size_t)c.r * es) / 64) * 64;
   if (tv_max < 64) return false;
@@ -78,7 +79,12 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
   if (e != cudaSuccess) { delete (Prof*)ctx->prof; delete ctx; return set_cuda_error("ts_create", e); }
   ctx->num_sms = prop.multiProcessorCount;
   ctx->max_smem = (int)prop.sharedMemPerBlockOptin;
-  if (!choose_tile(ctx->cfg, ctx->num_sms, ctx->max_smem, &ctx->tile)) {
+  // tensor cores for bf16 inputs whose rows allow 16-byte chunks; the fp32 FMA kernel otherwise
+  ctx->use_mma = (cfg->dt_U == TS_DTYPE_BF16 && cfg->r % 8 == 0 && cfg->V % 8 == 0 && prop.major == 10) ? 1 : 0;
+  const char* force = getenv("TS_FORCE_FMA");
+  if (force && force[0] == '1') ctx->use_mma = 0;
+  if (ctx->use_mma && !choose_tile_mma(ctx->cfg, ctx->num_sms, ctx->max_smem, &ctx->tile)) ctx->use_mma = 0;
+  if (!ctx->use_mma && !choose_tile(ctx->cfg, ctx->num_sms, ctx->max_smem, &ctx->tile)) {
     delete (Prof*)ctx->prof; delete ctx;
     return set_error(TS_ERR_UNSUPPORTED, "ts_create: no vocabulary tiling fits shared memory");
   }

@@ -15,6 +15,7 @@ constexpr int DMAX = TS_DMAX;
 constexpr int KNOTS = TS_CALIB_KNOTS;
 constexpr int SCORE_THREADS = 128;   // one parent per thread; every thread scans the CTA's whole tile
 constexpr int CHUNK = 16;            // tokens per coarse generator call
+constexpr int MMA_S = 2;             // column splits per tile in the tensor-core scoring kernel (warps per row quarter)
 
 enum Stream : uint32_t { STREAM_GUMBEL_COARSE = 1, STREAM_GUMBEL_FINE = 2, STREAM_ACCEPT = 3, STREAM_BONUS = 4 };
 
@@ -43,6 +44,7 @@ struct ts_ctx {
   int max_smem;
   ts::TileCfg tile;
   int vt_TV, vt_n;  // vocabulary ranges of the verification walk, one per CTA
+  int use_mma;      // 1: scoring runs on the tensor-core kernel, 0: on the fp32 FMA kernel
   ts::DevCalib calib;
   void* prof;  // ts::Prof*, instrumentation state
 };
@@ -54,8 +56,9 @@ namespace ts {
 // ------------------------------------------------------------------------------------------------
 struct WsLayout {
   int B, N, K, Pcap, ntiles, words;
-  // scoring partials, [ntiles][...][Pcap]
-  size_t part_m, part_s0, part_sT, part_topv, part_topi, part_keyv, part_keyi, part_keyl;
+  // scoring records, [ntiles * S][rec_cap][rec_words]
+  size_t rec; int rec_cap;
+  size_t err;            // int[4]: error word raised by a bounded wait inside the scoring kernel
   // merged per-parent results of the level being expanded, [Pcap] / [Pcap][K]
   size_t res_lse0, res_lseT, res_top_tok, res_top_logit, res_draw_tok, res_draw_logit;
   // level parent lists (two, alternating) [Pcap]
@@ -104,9 +107,13 @@ __host__ inline WsLayout make_layout(const ts_ctx* ctx, int B) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   const size_t P = (size_t)L.Pcap, nt = (size_t)L.ntiles, K = (size_t)c.K, N = (size_t)c.Nmax, b = (size_t)B;
-  L.part_m = take(nt * P * 4); L.part_s0 = take(nt * P * 4); L.part_sT = take(nt * P * 4);
-  L.part_topv = take(nt * K * P * 4); L.part_topi = take(nt * K * P * 4);
-  L.part_keyv = take(nt * K * P * 4); L.part_keyi = take(nt * K * P * 4); L.part_keyl = take(nt * K * P * 4);
+  {
+    int cap = (L.Pcap + 7) / 8 * 8, S = 1;
+    if (ctx->use_mma) { cap = (L.Pcap + 127) / 128 * 128; S = MMA_S; }
+    L.rec_cap = cap;
+    L.rec = take(align_up(nt * S * (size_t)cap * ((4 + 5 * K + 3) & ~(size_t)3) * 4, 256) + (size_t)cap * (2 + 2 * K) * 4);
+    L.err = take(16);
+  }
   L.res_lse0 = take(P * 4); L.res_lseT = take(P * 4);
   L.res_top_tok = take(P * K * 4); L.res_top_logit = take(P * K * 4);
   L.res_draw_tok = take(P * K * 4); L.res_draw_logit = take(P * K * 4);

@@ -31,7 +31,7 @@ struct ExpandArgs {
   float* root_lseT; int *req_npar, *req_base, *req_nscored;
   // candidates
   int *cd_valid, *cd_parent, *cd_sib, *cd_tok; double *cd_logkey, *cd_logS; float *cd_q0, *cd_logqT; int* cd_rank;
-  int* status;
+  int* status; int* err; unsigned* thr; int thr_words;
 };
 
 __device__ __forceinline__ void request_caps(const ExpandArgs& a, int b, int& K_eff, int& N_eff, double& log_theta) {
@@ -48,6 +48,7 @@ __device__ __forceinline__ void request_caps(const ExpandArgs& a, int b, int& K_
 __global__ void expand_init_kernel(ExpandArgs a) {
   const int b = blockIdx.x;
   for (int s = threadIdx.x; s < a.N; s += blockDim.x) a.pl_alive[(size_t)b * a.N + s] = 0;
+  for (int i = b * blockDim.x + threadIdx.x; i < a.thr_words; i += gridDim.x * blockDim.x) a.thr[i] = 0u;
   if (threadIdx.x == 0) {
     const int tok = a.anchor[b];
     const bool ok = tok >= 0 && tok < a.V && a.theta[b] == a.theta[b];
@@ -57,6 +58,7 @@ __global__ void expand_init_kernel(ExpandArgs a) {
     a.req_npar[b] = 1; a.req_base[b] = b; a.req_nscored[b] = 0;
     a.root_lseT[b] = nanf("");
     if (b == 0) {
+      a.err[0] = 0;
       a.lvl_count[0] = a.B;
       for (int d = 1; d <= DMAX + 1; ++d) a.lvl_count[d] = 0;
     }
@@ -83,7 +85,10 @@ __global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d) 
   int K_eff, N_eff; double log_theta;
   request_caps(a, b, K_eff, N_eff, log_theta);
   const size_t pb = (size_t)b * N, cb = (size_t)b * N * K;
-  if (tid == 0) s_base = a.status[b];
+  if (tid == 0) {
+    if (a.err[0] != 0 && a.status[b] == TS_OK) a.status[b] = TS_ERR_TIMEOUT;  // a wait in the scoring kernel ran out
+    s_base = a.status[b];
+  }
   __syncthreads();
   if (npar == 0 || s_base != TS_OK) {  // uniform: read once, before any thread can change the status
     if (tid == 0) a.req_npar[b] = 0;
@@ -330,7 +335,8 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   a.cd_valid = (int*)(ws + L.cd_valid); a.cd_parent = (int*)(ws + L.cd_parent); a.cd_sib = (int*)(ws + L.cd_sib);
   a.cd_tok = (int*)(ws + L.cd_tok); a.cd_logkey = (double*)(ws + L.cd_logkey); a.cd_logS = (double*)(ws + L.cd_logS);
   a.cd_q0 = (float*)(ws + L.cd_q0); a.cd_logqT = (float*)(ws + L.cd_logqT); a.cd_rank = (int*)(ws + L.cd_rank);
-  a.status = status;
+  a.status = status; a.err = (int*)(ws + L.err);
+  a.thr = thr_base(ctx, (float*)(ws + L.rec), L.rec_cap); a.thr_words = (int)(thr_bytes(ctx, L.rec_cap) / 4);
 
   { ProfScope ps(ctx, K_INIT, st); expand_init_kernel<<<B, 64, 0, st>>>(a); }
   cudaError_t e = cudaGetLastError();
@@ -342,7 +348,8 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   }
   for (int d = 0; d < c.D; ++d) {
     const int cur = d & 1;
-    e = launch_score(ctx, L, ws, U, A, W, 0, a.lvl_count + d, a.lst_req[cur], a.lst_depth[cur], a.lst_token[cur],
+    e = launch_score(ctx, (float*)(ws + L.rec), L.rec_cap, (int*)(ws + L.err), U, A, W, 0, a.lvl_count + d,
+                     a.lst_req[cur], a.lst_depth[cur], a.lst_token[cur],
                      a.lst_hash[cur], T, seed, res_lse0, res_lseT, res_top_tok, res_top_logit, res_draw_tok,
                      res_draw_logit, st);
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(score)", e);

@@ -13,11 +13,41 @@ int32_t set_cuda_error(const char* where, cudaError_t e);
 cudaError_t score_setup(ts_ctx* ctx);
 cudaError_t verify_setup(ts_ctx* ctx);
 
+struct ScoreArgs {
+  const void *U, *A, *W;
+  int V, D, r, K;
+  int P; const int* P_dev;
+  const int *p_req, *p_depth, *p_token; const uint64_t* p_hash;
+  float T; uint64_t seed;
+  int TV, ntiles, cap, S;
+  float* rec; int* err;
+  unsigned* thr;    // [2][cap]: launch-wide lower bounds (logit, key) per parent, order-preserving encoding
+  unsigned* slots;  // [2][cap][K]
+};
+
+struct MergeArgs {
+  int P; const int* P_dev; int K, ntiles, cap, S, mma; float T;
+  const float* rec; unsigned* thr; unsigned* slots;
+  float *lse0, *lseT; int* top_tok; float* top_logit; int* draw_tok; float* draw_logit;
+};
+
+// Bytes of record scratch a scoring pass over up to P parents needs, and the slot capacity it implies.
+size_t score_scratch_bytes(const ts_ctx* ctx, int P, int* cap_out);
+// The pruning state (thresholds + slots) sits behind the records; it must be zero before a launch and
+// the merge kernel leaves it zero again.
+unsigned* thr_base(const ts_ctx* ctx, float* rec, int cap);
+size_t thr_bytes(const ts_ctx* ctx, int cap);
+
 // Scoring pass + merge for a parent list whose length is P (host) or *P_dev (device) when P_dev is set.
-cudaError_t launch_score(const ts_ctx* ctx, const WsLayout& L, char* ws, const void* U, const void* A, const void* W,
+// rec: record scratch of score_scratch_bytes(ctx, max parents) bytes with slot capacity cap.
+cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,
                          const uint64_t* p_hash, float T, uint64_t seed, float* lse0, float* lseT, int* top_tok,
                          float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st);
+
+bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out);
+cudaError_t score_mma_setup(ts_ctx* ctx);
+cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st);
 
 enum KernelId { K_INIT, K_SCORE, K_MERGE, K_LEVEL, K_FINAL, K_ZROWS, K_GREEDY, K_WALK, K_CHECK, K_COUNT };
 

@@ -35,24 +35,18 @@ extern "C" int32_t ts_score_parents_static(ts_ctx* ctx, const void* U, const voi
   if (!(T >= 0.f)) return set_error(TS_ERR_INVALID, "ts_score_parents_static: T must be >= 0");
   if (P == 0) return TS_OK;
 
-  // records of P parents over all vocabulary tiles, laid out like the workspace version's
-  WsLayout L{};
-  L.Pcap = (P + 7) / 8 * 8;
-  L.ntiles = ctx->tile.ntiles;
-  L.K = ctx->cfg.K;
-  size_t off = 0;
-  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-  const size_t np = (size_t)L.ntiles * L.Pcap, npk = np * (size_t)L.K;
-  L.part_m = take(np * 4); L.part_s0 = take(np * 4); L.part_sT = take(np * 4);
-  L.part_topv = take(npk * 4); L.part_topi = take(npk * 4);
-  L.part_keyv = take(npk * 4); L.part_keyi = take(npk * 4); L.part_keyl = take(npk * 4);
-  if (off > (size_t)TS_STATIC_SCRATCH_BYTES) {
-    const size_t per_parent = (size_t)L.ntiles * (3 + 5 * (size_t)L.K) * 4;
+  // records of P parents over all vocabulary tiles, plus the scoring kernel's error word
+  int cap = 0;
+  const size_t rec_bytes = align_up(score_scratch_bytes(ctx, P, &cap), 256);
+  const size_t need = rec_bytes + 256;
+  if (need > (size_t)TS_STATIC_SCRATCH_BYTES) {
+    int cap1 = 0;
+    const size_t unit = score_scratch_bytes(ctx, 1, &cap1);  // bytes for the smallest slot block
     char msg[256];
     snprintf(msg, sizeof(msg),
              "ts_score_parents_static: %d parents need %zu bytes of scratch, the built-in array holds %u "
-             "(about %zu parents for this configuration); use ts_score_parents with a workspace instead",
-             P, off, (unsigned)TS_STATIC_SCRATCH_BYTES, (size_t)TS_STATIC_SCRATCH_BYTES / per_parent);
+             "(%zu bytes per block of %d parents for this configuration); use ts_score_parents with a workspace instead",
+             P, need, (unsigned)TS_STATIC_SCRATCH_BYTES, unit, cap1);
     return set_error(TS_ERR_WORKSPACE, msg);
   }
 
@@ -72,10 +66,15 @@ extern "C" int32_t ts_score_parents_static(ts_ctx* ctx, const void* U, const voi
     }
     scratch = g_scratch_addr[dev];
   }
-  // Nothing in the array has to start at zero: the scoring kernel writes every record of
-  // (tile, parent < P) before the merge kernel, next on the same stream, reads exactly those.
-  e = launch_score(ctx, L, (char*)scratch, U, A, W, P, nullptr, parent_req, parent_depth, parent_token, parent_hash,
-                   T, seed, lse0, lseT, top_tok, top_logit, draw_tok, draw_logit, (cudaStream_t)stream);
+  // The records need no clearing: the scoring kernel writes every record of (piece, parent < P) before
+  // the merge kernel, next on the same stream, reads exactly those.  The error word and the pruning
+  // state behind the records must start at zero.
+  int* err = (int*)((char*)scratch + rec_bytes);
+  e = cudaMemsetAsync(err, 0, 16, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(thr_base(ctx, (float*)scratch, cap), 0, thr_bytes(ctx, cap), (cudaStream_t)stream);
+  if (e != cudaSuccess) return set_cuda_error("ts_score_parents_static(memset)", e);
+  e = launch_score(ctx, (float*)scratch, cap, err, U, A, W, P, nullptr, parent_req, parent_depth, parent_token,
+                   parent_hash, T, seed, lse0, lseT, top_tok, top_logit, draw_tok, draw_logit, (cudaStream_t)stream);
   if (e != cudaSuccess) return set_cuda_error("ts_score_parents_static", e);
   return TS_OK;
 }

@@ -1,107 +1,16 @@
 // Parent-conditioned scoring (Eq. 1) fused with logsumexp at temperature 1 and T, top-K logits and
 // Gumbel top-K sibling draws (Eq. 2), one pass over the vocabulary.
 //
-// Decomposition: the vocabulary is split into tiles, one CTA per tile with its W tile resident in
-// shared memory for all parents; every thread owns one parent and scans the tile's tokens in
-// order, so the running max / sums / candidate lists are thread-private.  A second kernel merges
-// the per-tile records of each parent.
+// The vocabulary is split into tiles, one CTA per tile with its W tile resident in shared memory for
+// all parents of the launch.  Two kernels produce the same per-(piece, parent) records:
+//   * score_mma_kernel (ts_score_mma.cu): bf16, the bias [parents x r] . [r x tile] on the tensor
+//     cores (tcgen05, accumulators in tensor memory), the scan as its epilogue;
+//   * score_tile_kernel (here): fp32 FMA, any dtype / rank / vocabulary size.
+// merge_kernel then folds the records of each parent.
 #include "ts_internal.h"
+#include "ts_scan.cuh"
 
 namespace ts {
-
-// Thread-private running state of one parent over the tokens scanned so far.
-struct RowScan {
-  float m, s0, sT;
-  float thrL, thrK;
-  int K;
-  float topv[KMAX]; int topi[KMAX];
-  float keyv[KMAX]; int keyi[KMAX]; float keyl[KMAX];
-
-  __device__ __forceinline__ void init(int K_) {
-    K = K_; m = -INFINITY; s0 = 0.f; sT = 0.f; thrL = -INFINITY; thrK = -INFINITY;
-    for (int i = 0; i < KMAX; ++i) { topv[i] = -INFINITY; topi[i] = -1; keyv[i] = -INFINITY; keyi[i] = -1; keyl[i] = 0.f; }
-  }
-  // tokens arrive in increasing order, so an equal value never displaces an earlier entry
-  __device__ __forceinline__ void insert_top(float v, int tok) {
-    int pos = K - 1;
-    while (pos > 0 && v > topv[pos - 1]) { topv[pos] = topv[pos - 1]; topi[pos] = topi[pos - 1]; --pos; }
-    topv[pos] = v; topi[pos] = tok;
-    thrL = topv[K - 1];
-  }
-  __device__ __forceinline__ void insert_key(float key, int tok, float logit) {
-    int pos = K - 1;
-    while (pos > 0 && key > keyv[pos - 1]) {
-      keyv[pos] = keyv[pos - 1]; keyi[pos] = keyi[pos - 1]; keyl[pos] = keyl[pos - 1]; --pos;
-    }
-    keyv[pos] = key; keyi[pos] = tok; keyl[pos] = logit;
-    thrK = keyv[K - 1];
-  }
-};
-
-struct ScoreArgs {
-  const void *U, *A, *W;
-  int V, D, r, K;
-  int P; const int* P_dev;
-  const int *p_req, *p_depth, *p_token; const uint64_t* p_hash;
-  float T; uint64_t seed;
-  int TV, ntiles, Pcap;
-  float *part_m, *part_s0, *part_sT, *part_topv, *part_keyv, *part_keyl;
-  int *part_topi, *part_keyi;
-};
-
-// One 16-token chunk of one parent: logits l[0..16) for tokens v0.., `valid` of them inside V.
-__device__ __forceinline__ void scan_chunk(RowScan& st, const float* l, int v0, int valid, float T, float invT,
-                                           uint64_t seed, int req, uint64_t hash, const float* ghi) {
-  float cm = -INFINITY;
-#pragma unroll
-  for (int i = 0; i < CHUNK; ++i) if (i < valid) cm = fmaxf(cm, l[i]);
-  if (cm > st.m) {
-    const float d = st.m - cm;  // -inf on the first chunk: both factors become 0
-    st.s0 *= __expf(d);
-    st.sT *= __expf(d * invT);
-    st.m = cm;
-  }
-  float a0 = 0.f, aT = 0.f;
-  const bool two = (T > 0.f) && (T != 1.f);
-#pragma unroll
-  for (int i = 0; i < CHUNK; ++i) {
-    if (i < valid) {
-      const float d = l[i] - st.m;
-      a0 += __expf(d);
-      if (two) aT += __expf(d * invT);
-    }
-  }
-  st.s0 += a0;
-  st.sT += two ? aT : a0;
-  if (cm > st.thrL || st.topi[st.K - 1] < 0) {
-#pragma unroll
-    for (int i = 0; i < CHUNK; ++i)
-      if (i < valid && (l[i] > st.thrL || st.topi[st.K - 1] < 0)) st.insert_top(l[i], v0 + i);
-  }
-  if (T > 0.f) {
-    // top byte of each token's uniform: one generator call for the chunk
-    const uint4 cw = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, (uint32_t)v0 >> 4);
-    uint4 fw = make_uint4(0, 0, 0, 0);
-    int fine_call = -1;
-#pragma unroll
-    for (int i = 0; i < CHUNK; ++i) {
-      if (i < valid) {
-        const uint32_t c8 = (word_of(cw, i >> 2) >> (8 * (i & 3))) & 0xFFu;
-        const float base = l[i] * invT;
-        // ghi[c8] bounds the noise from above given only the top byte; most tokens stop here
-        if (base + ghi[c8] > st.thrK || st.keyi[st.K - 1] < 0) {
-          if (fine_call != (i >> 2)) {
-            fw = stream_words(seed, req, hash, STREAM_GUMBEL_FINE, ((uint32_t)(v0 + i)) >> 2);
-            fine_call = i >> 2;
-          }
-          const uint32_t X = (c8 << 24) | (word_of(fw, i & 3) >> 8);
-          const float key = base + gumbel_from_bits(X);
-          if (key > st.thrK || st.keyi[st.K - 1] < 0) st.insert_key(key, v0 + i, l[i]);
-        }
-      }
-    }
-  }
-}
 
 template <typename TIn>
 __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs a) {
@@ -109,7 +18,7 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
   const int r = a.r, TV = a.TV, V = a.V;
   TIn* Ws = reinterpret_cast<TIn*>(smem_raw);                              // [r][TV]
   float* as = reinterpret_cast<float*>(smem_raw + (size_t)r * TV * sizeof(TIn));  // [r][SCORE_THREADS]
-  float* ghi = as + (size_t)r * SCORE_THREADS;                             // [256]
+  float* ghi = as + (size_t)r * SCORE_THREADS;                             // [512]
   const int tid = threadIdx.x;
   const int tile = blockIdx.x;
   const int t0 = tile * TV;
@@ -137,16 +46,12 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
       Ws[(size_t)k * TV + c] = c < tlen ? Wg[(size_t)k * V + t0 + c] : TIn(0.f);
     }
   }
-  // upper bound of the Gumbel noise given the top byte of the uniform, with a safety margin
-  for (int c = tid; c < 256; c += SCORE_THREADS) {
-    const double u = ((double)(((uint32_t)c << 24) | 0xFFFFFFu) + 0.5) * (1.0 / 4294967296.0);
-    const double g = -log(-log(u));
-    ghi[c] = (float)(g + 1e-4 * fabs(g) + 1e-4);
-  }
+  fill_gumbel_bounds(ghi, tid, SCORE_THREADS);
   __syncthreads();
 
   const float T = a.T, invT = T > 0.f ? 1.f / T : 1.f;
   const int K = a.K;
+  const int rw = rec_words(K);
 
   for (int pg = 0; pg < P; pg += SCORE_THREADS) {
     const int p = pg + tid;
@@ -157,6 +62,8 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
     const TIn* Urow = Ug + ((size_t)req * a.D + dep) * V + t0;
     RowScan st;
     st.init(K);
+    const SharedThr gl{a.slots + (size_t)p * K, tile % K};
+    const SharedThr gk{a.slots + ((size_t)a.cap + p) * K, tile % K};
     for (int c0 = 0; c0 < tlen; c0 += CHUNK) {
       const int valid = min(CHUNK, tlen - c0);
       float l[CHUNK];
@@ -179,96 +86,133 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
 #pragma unroll
         for (int i = 0; i < CHUNK; ++i) l[i] = fmaf(ak, w[i], l[i]);
       }
-      scan_chunk(st, l, t0 + c0, valid, T, invT, a.seed, req, hash, ghi);
+      scan_chunk(st, l, t0 + c0, valid, T, invT, a.seed, req, hash, ghi, gl, gk);
     }
-    // record of (parent, tile)
-    const size_t o = (size_t)tile * a.Pcap + p;
-    a.part_m[o] = st.m; a.part_s0[o] = st.s0; a.part_sT[o] = st.sT;
-    for (int j = 0; j < K; ++j) {
-      const size_t oj = ((size_t)tile * K + j) * a.Pcap + p;
-      a.part_topv[oj] = st.topv[j]; a.part_topi[oj] = st.topi[j];
-      a.part_keyv[oj] = st.keyv[j]; a.part_keyi[oj] = st.keyi[j]; a.part_keyl[oj] = st.keyl[j];
-    }
+    st.store(a.rec + ((size_t)tile * a.cap + p) * rw);  // piece = (tile, 0), slot = p
   }
 }
 
 // ------------------------------------------------------------------------------------------------
-// Merge of the per-tile records: one warp per parent
+// Merge of the per-piece records: one CTA per parent.
+// Every thread folds its share of the pieces into a private (max, sums) pair and private top-K
+// lists; the block then takes K rounds of arg-max over the list heads (value desc, token asc).
 // ------------------------------------------------------------------------------------------------
-struct MergeArgs {
-  int P; const int* P_dev; int K, ntiles, Pcap; float T;
-  const float *part_m, *part_s0, *part_sT, *part_topv, *part_keyv, *part_keyl;
-  const int *part_topi, *part_keyi;
-  float *lse0, *lseT; int* top_tok; float* top_logit; int* draw_tok; float* draw_logit;
+constexpr int MERGE_THREADS = 128;
+
+struct TopList {
+  float v[KMAX]; int i[KMAX]; float l[KMAX]; int n;
+  __device__ __forceinline__ void init() { n = 0; }
+  __device__ __forceinline__ static bool better(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
+  __device__ __forceinline__ void insert(float val, int idx, float lg, int K) {
+    if (n == K && !better(val, idx, v[K - 1], i[K - 1])) return;
+    int pos = n < K ? n : K - 1;
+    while (pos > 0 && better(val, idx, v[pos - 1], i[pos - 1])) { v[pos] = v[pos - 1]; i[pos] = i[pos - 1]; l[pos] = l[pos - 1]; --pos; }
+    v[pos] = val; i[pos] = idx; l[pos] = lg;
+    if (n < K) ++n;
+  }
 };
 
-constexpr int MERGE_MAX_TILES_PER_LANE = 16;
-
-// K rounds of warp-wide arg-max over the heads of the per-tile sorted lists
-__device__ void merge_lists(const float* pv, const int* pi, const float* pl, int p, int K, int ntiles, int Pcap,
-                            int lane, int* out_tok, float* out_val) {
-  unsigned char cur[MERGE_MAX_TILES_PER_LANE];
-  for (int i = 0; i < MERGE_MAX_TILES_PER_LANE; ++i) cur[i] = 0;
+// K rounds of block-wide arg-max over the heads of the threads' sorted lists
+__device__ void block_select(const TopList& mine, int K, int* out_tok, float* out_val, float* s_v, int* s_i, float* s_l) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int head = 0;
   for (int j = 0; j < K; ++j) {
-    float bv = -INFINITY; int bi = 0x7FFFFFFF, bt = -1; float bl = 0.f;
-    for (int s = 0, t = lane; t < ntiles; t += 32, ++s) {
-      if (cur[s] >= K) continue;
-      const size_t o = ((size_t)t * K + cur[s]) * Pcap + p;
-      const int idx = pi[o];
-      if (idx < 0) continue;
-      const float v = pv[o];
-      if (v > bv || (v == bv && idx < bi)) { bv = v; bi = idx; bt = s; bl = pl ? pl[o] : v; }
-    }
-    float wv = bv; int wi = bi;
+    float bv = head < mine.n ? mine.v[head] : -INFINITY;
+    int bi = head < mine.n ? mine.i[head] : 0x7FFFFFFF;
+    float bl = head < mine.n ? mine.l[head] : 0.f;
+    float wv = bv; int wi = bi; float wl = bl;
     for (int off = 16; off > 0; off >>= 1) {
       const float ov = __shfl_xor_sync(0xFFFFFFFFu, wv, off);
       const int oi = __shfl_xor_sync(0xFFFFFFFFu, wi, off);
-      if (ov > wv || (ov == wv && oi < wi)) { wv = ov; wi = oi; }
+      const float ol = __shfl_xor_sync(0xFFFFFFFFu, wl, off);
+      if (TopList::better(ov, oi, wv, wi)) { wv = ov; wi = oi; wl = ol; }
     }
-    const bool mine = (bt >= 0) && (wi == bi) && (wv == bv);
-    if (mine) cur[bt]++;
-    const unsigned who = __ballot_sync(0xFFFFFFFFu, mine);
-    if (who == 0u) { if (lane == 0) { out_tok[j] = -1; out_val[j] = 0.f; } continue; }
-    const int src = __ffs(who) - 1;
-    const float lv = __shfl_sync(0xFFFFFFFFu, bl, src);
-    if (lane == 0) { out_tok[j] = wi; out_val[j] = lv; }
+    if (lane == 0) { s_v[warp] = wv; s_i[warp] = wi; s_l[warp] = wl; }
+    __syncthreads();
+    if (tid == 0) {
+      float gv = s_v[0]; int gi = s_i[0]; float gl = s_l[0];
+      for (int w = 1; w < MERGE_THREADS / 32; ++w)
+        if (TopList::better(s_v[w], s_i[w], gv, gi)) { gv = s_v[w]; gi = s_i[w]; gl = s_l[w]; }
+      s_v[MERGE_THREADS / 32] = gv; s_i[MERGE_THREADS / 32] = gi; s_l[MERGE_THREADS / 32] = gl;
+    }
+    __syncthreads();
+    const int gi = s_i[MERGE_THREADS / 32];
+    if (gi != 0x7FFFFFFF && head < mine.n && mine.i[head] == gi) ++head;  // tokens are unique per list
+    if (tid == 0) { out_tok[j] = gi == 0x7FFFFFFF ? -1 : gi; out_val[j] = gi == 0x7FFFFFFF ? 0.f : s_l[MERGE_THREADS / 32]; }
+    __syncthreads();
   }
 }
 
-__global__ void merge_kernel(MergeArgs a) {
+__global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
+  __shared__ float s_v[MERGE_THREADS / 32 + 1]; __shared__ int s_i[MERGE_THREADS / 32 + 1]; __shared__ float s_l[MERGE_THREADS / 32 + 1];
+  __shared__ float s_m[MERGE_THREADS / 32], s_s0[MERGE_THREADS / 32], s_sT[MERGE_THREADS / 32];
   const int P = a.P_dev ? *a.P_dev : a.P;
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  const int nwarps = (gridDim.x * blockDim.x) >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float invT = a.T > 0.f ? 1.f / a.T : 1.f;
-  for (int p = warp; p < P; p += nwarps) {
-    float m = -INFINITY;
-    for (int t = lane; t < a.ntiles; t += 32) m = fmaxf(m, a.part_m[(size_t)t * a.Pcap + p]);
-    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
-    float s0 = 0.f, sT = 0.f;
-    for (int t = lane; t < a.ntiles; t += 32) {
-      const size_t o = (size_t)t * a.Pcap + p;
-      const float d = a.part_m[o] - m;
-      if (d > -INFINITY) { s0 += a.part_s0[o] * __expf(d); sT += a.part_sT[o] * __expf(d * invT); }
-    }
-    for (int off = 16; off > 0; off >>= 1) {
-      s0 += __shfl_xor_sync(0xFFFFFFFFu, s0, off);
-      sT += __shfl_xor_sync(0xFFFFFFFFu, sT, off);
-    }
-    if (lane == 0) {
-      a.lse0[p] = m + logf(s0);
-      a.lseT[p] = a.T > 0.f ? m * invT + logf(sT) : m + logf(s0);
-    }
-    merge_lists(a.part_topv, a.part_topi, nullptr, p, a.K, a.ntiles, a.Pcap, lane, a.top_tok + (size_t)p * a.K,
-                a.top_logit + (size_t)p * a.K);
-    if (a.T > 0.f) {
-      merge_lists(a.part_keyv, a.part_keyi, a.part_keyl, p, a.K, a.ntiles, a.Pcap, lane,
-                  a.draw_tok + (size_t)p * a.K, a.draw_logit + (size_t)p * a.K);
-    } else {
-      __syncwarp();
-      for (int j = lane; j < a.K; j += 32) {
-        a.draw_tok[(size_t)p * a.K + j] = a.top_tok[(size_t)p * a.K + j];
-        a.draw_logit[(size_t)p * a.K + j] = a.top_logit[(size_t)p * a.K + j];
+  const int K = a.K, rw = rec_words(K);
+  const int R = a.mma ? mma_replicas(P) : 1;
+  const int npieces = a.ntiles * a.S * R;
+  for (int p = blockIdx.x; p < P; p += gridDim.x) {
+    float m = -INFINITY, s0 = 0.f, sT = 0.f;
+    TopList top, key;
+    top.init(); key.init();
+    for (int q = tid; q < npieces; q += MERGE_THREADS) {
+      const int ts_ = q / R, rho = q % R;
+      const int slot = R > 1 ? rho * (128 / R) + p : p;
+      const float* rec = a.rec + ((size_t)ts_ * a.cap + slot) * rw;
+      const float4 h = *reinterpret_cast<const float4*>(rec);
+      if (h.x == -INFINITY) continue;  // a piece that scanned nothing
+      if (h.x > m) { const float d = m - h.x; s0 *= __expf(d); sT *= __expf(d * invT); m = h.x; }
+      const float d = h.x - m;
+      s0 += h.y * __expf(d); sT += h.z * __expf(d * invT);
+      const float* f = rec + 4; const int* ii = reinterpret_cast<const int*>(rec) + 4;
+      for (int j = 0; j < K; ++j) {
+        const int ti = ii[K + j];
+        if (ti < 0) break;
+        top.insert(f[j], ti, f[j], K);
       }
+      if (a.T > 0.f)
+        for (int j = 0; j < K; ++j) {
+          const int ki = ii[3 * K + j];
+          if (ki < 0) break;
+          key.insert(f[2 * K + j], ki, f[4 * K + j], K);
+        }
+    }
+    // fold the (max, sums) pairs
+    for (int off = 16; off > 0; off >>= 1) {
+      const float om = __shfl_xor_sync(0xFFFFFFFFu, m, off);
+      const float o0 = __shfl_xor_sync(0xFFFFFFFFu, s0, off);
+      const float oT = __shfl_xor_sync(0xFFFFFFFFu, sT, off);
+      const float nm = fmaxf(m, om);
+      if (nm > -INFINITY) {
+        s0 = s0 * __expf(m - nm) + o0 * __expf(om - nm);
+        sT = sT * __expf((m - nm) * invT) + oT * __expf((om - nm) * invT);
+      }
+      m = nm;
+    }
+    if (lane == 0) { s_m[warp] = m; s_s0[warp] = s0; s_sT[warp] = sT; }
+    __syncthreads();
+    if (tid == 0) {
+      float gm = -INFINITY;
+      for (int w = 0; w < MERGE_THREADS / 32; ++w) gm = fmaxf(gm, s_m[w]);
+      float g0 = 0.f, gT = 0.f;
+      for (int w = 0; w < MERGE_THREADS / 32; ++w)
+        if (s_m[w] > -INFINITY) { g0 += s_s0[w] * __expf(s_m[w] - gm); gT += s_sT[w] * __expf((s_m[w] - gm) * invT); }
+      a.lse0[p] = gm + logf(g0);
+      a.lseT[p] = a.T > 0.f ? gm * invT + logf(gT) : gm + logf(g0);
+    }
+    __syncthreads();
+    // leave the launch-wide pruning state of this parent clean for the next launch
+    if (tid < 2 * K) a.slots[((size_t)(tid / K) * a.cap + p) * K + tid % K] = 0u;
+    block_select(top, K, a.top_tok + (size_t)p * K, a.top_logit + (size_t)p * K, s_v, s_i, s_l);
+    if (a.T > 0.f) {
+      block_select(key, K, a.draw_tok + (size_t)p * K, a.draw_logit + (size_t)p * K, s_v, s_i, s_l);
+    } else {
+      if (tid < K) {
+        a.draw_tok[(size_t)p * K + tid] = a.top_tok[(size_t)p * K + tid];
+        a.draw_logit[(size_t)p * K + tid] = a.top_logit[(size_t)p * K + tid];
+      }
+      __syncthreads();
     }
   }
 }
@@ -276,7 +220,24 @@ __global__ void merge_kernel(MergeArgs a) {
 // ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
-cudaError_t launch_score(const ts_ctx* ctx, const WsLayout& L, char* ws, const void* U, const void* A, const void* W,
+size_t score_scratch_bytes(const ts_ctx* ctx, int P, int* cap_out) {
+  int cap = (P + 7) / 8 * 8;
+  int S = 1;
+  if (ctx->use_mma) { cap = (P + 127) / 128 * 128; if (cap < 128) cap = 128; S = MMA_S; }
+  if (cap_out) *cap_out = cap;
+  // records, then the pruning state: 2 threshold words and 2K slot words per slot of capacity
+  return align_up((size_t)ctx->tile.ntiles * S * cap * rec_words(ctx->cfg.K) * sizeof(float), 256) +
+         align_up((size_t)cap * (2 + 2 * (size_t)ctx->cfg.K) * sizeof(unsigned), 256);
+}
+
+unsigned* thr_base(const ts_ctx* ctx, float* rec, int cap) {
+  const int S = ctx->use_mma ? MMA_S : 1;
+  return (unsigned*)((char*)rec + align_up((size_t)ctx->tile.ntiles * S * cap * rec_words(ctx->cfg.K) * sizeof(float), 256));
+}
+
+size_t thr_bytes(const ts_ctx* ctx, int cap) { return (size_t)cap * (2 + 2 * (size_t)ctx->cfg.K) * sizeof(unsigned); }
+
+cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,
                          const uint64_t* p_hash, float T, uint64_t seed, float* lse0, float* lseT, int* top_tok,
                          float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st) {
@@ -284,36 +245,38 @@ cudaError_t launch_score(const ts_ctx* ctx, const WsLayout& L, char* ws, const v
   ScoreArgs a{};
   a.U = U; a.A = A; a.W = W; a.V = c.V; a.D = c.D; a.r = c.r; a.K = c.K; a.P = P; a.P_dev = P_dev;
   a.p_req = p_req; a.p_depth = p_depth; a.p_token = p_token; a.p_hash = p_hash; a.T = T; a.seed = seed;
-  a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.Pcap = L.Pcap;
-  a.part_m = (float*)(ws + L.part_m); a.part_s0 = (float*)(ws + L.part_s0); a.part_sT = (float*)(ws + L.part_sT);
-  a.part_topv = (float*)(ws + L.part_topv); a.part_topi = (int*)(ws + L.part_topi);
-  a.part_keyv = (float*)(ws + L.part_keyv); a.part_keyi = (int*)(ws + L.part_keyi); a.part_keyl = (float*)(ws + L.part_keyl);
+  a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.cap = cap; a.S = ctx->use_mma ? MMA_S : 1; a.rec = rec; a.err = err;
+  a.thr = thr_base(ctx, rec, cap); a.slots = a.thr + 2 * (size_t)cap;
+  cudaError_t e;
   {
     ProfScope ps(ctx, K_SCORE, st);
-    if (c.dt_U == TS_DTYPE_BF16)
+    if (ctx->use_mma) {
+      e = launch_score_mma(ctx, a, st);
+      if (e != cudaSuccess) return e;
+    } else if (c.dt_U == TS_DTYPE_BF16) {
       score_tile_kernel<__nv_bfloat16><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
-    else
+    } else {
       score_tile_kernel<float><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
+    }
   }
-  cudaError_t e = cudaGetLastError();
+  e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   MergeArgs m{};
-  m.P = P; m.P_dev = P_dev; m.K = c.K; m.ntiles = a.ntiles; m.Pcap = L.Pcap; m.T = T;
-  m.part_m = a.part_m; m.part_s0 = a.part_s0; m.part_sT = a.part_sT; m.part_topv = a.part_topv;
-  m.part_keyv = a.part_keyv; m.part_keyl = a.part_keyl; m.part_topi = a.part_topi; m.part_keyi = a.part_keyi;
+  m.P = P; m.P_dev = P_dev; m.K = c.K; m.ntiles = a.ntiles; m.cap = cap; m.S = a.S; m.mma = ctx->use_mma ? 1 : 0; m.T = T;
+  m.rec = rec; m.thr = a.thr; m.slots = a.slots;
   m.lse0 = lse0; m.lseT = lseT; m.top_tok = top_tok; m.top_logit = top_logit; m.draw_tok = draw_tok; m.draw_logit = draw_logit;
-  const int pmax = P_dev ? L.Pcap : P;
-  int blocks = (pmax + 7) / 8;
-  if (blocks > 4 * ctx->num_sms) blocks = 4 * ctx->num_sms;
+  int blocks = P_dev ? cap : P;
+  if (blocks > 8 * ctx->num_sms) blocks = 8 * ctx->num_sms;
   if (blocks < 1) blocks = 1;
   {
     ProfScope ps(ctx, K_MERGE, st);
-    merge_kernel<<<blocks, 256, 0, st>>>(m);
+    merge_kernel<<<blocks, MERGE_THREADS, 0, st>>>(m);
   }
   return cudaGetLastError();
 }
 
 cudaError_t score_setup(ts_ctx* ctx) {
+  if (ctx->use_mma) return score_mma_setup(ctx);
   cudaError_t e = cudaFuncSetAttribute(score_tile_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)ctx->tile.smem);
   if (e != cudaSuccess) return e;
@@ -339,9 +302,13 @@ extern "C" int32_t ts_score_parents(ts_ctx* ctx, const void* U, const void* A, c
   if (!(T >= 0.f)) return set_error(TS_ERR_INVALID, "ts_score_parents: T must be >= 0");
   if (ws_bytes < L.total) return set_error(TS_ERR_WORKSPACE, "ts_score_parents: workspace too small");
   if (P == 0) return TS_OK;
-  cudaError_t e = launch_score(ctx, L, (char*)ws, U, A, W, P, nullptr, parent_req, parent_depth, parent_token,
-                               parent_hash, T, seed, lse0, lseT, top_tok, top_logit, draw_tok, draw_logit,
-                               (cudaStream_t)stream);
+  cudaError_t e = cudaMemsetAsync((char*)ws + L.err, 0, 16, (cudaStream_t)stream);
+  if (e == cudaSuccess)
+    e = cudaMemsetAsync(thr_base(ctx, (float*)((char*)ws + L.rec), L.rec_cap), 0, thr_bytes(ctx, L.rec_cap), (cudaStream_t)stream);
+  if (e != cudaSuccess) return set_cuda_error("ts_score_parents(memset)", e);
+  e = launch_score(ctx, (float*)((char*)ws + L.rec), L.rec_cap, (int*)((char*)ws + L.err), U, A, W, P, nullptr,
+                               parent_req, parent_depth, parent_token, parent_hash, T, seed, lse0, lseT, top_tok,
+                               top_logit, draw_tok, draw_logit, (cudaStream_t)stream);
   if (e != cudaSuccess) return set_cuda_error("ts_score_parents", e);
   return TS_OK;
 }

@@ -1,0 +1,287 @@
+// Tensor-core scoring kernel for sm_100a: the low-rank bias [parents x r] . [r x tile] runs on the
+// 5th-generation tensor cores (tcgen05.mma, accumulators in tensor memory), and the vocabulary scan
+// (add base logits, online max / sum-exp, top-K, Gumbel top-K) is its epilogue, one tensor-memory
+// lane = one parent row per thread.
+//
+// CTA = one vocabulary tile, resident for the whole launch.  Shared memory holds
+//   W tile  : B operand, MN-major, 128-byte swizzle: slabs of 64 tokens, slab = [rp rows][128 B]
+//   A tile  : A operand, K-major, 128-byte swizzle: [rp/64 slabs][128 rows][128 B] (gathered rows A[x_p])
+// (rp = r rounded up to 64, padding zero-filled).  Warps 0..7 are epilogue warps: warp w reads the
+// tensor-memory lanes 32*(w%4).. (its quarter of the 128 parent rows) and, of every 128-column block,
+// the 16-token chunks assigned to column split s = w/4.  Warp 8 allocates tensor memory and its lane 0
+// issues the MMAs: per block of 128 tokens rp/16 instructions of M=128, N=128 (64 at a ragged end),
+// K=16 into one of two 128-column accumulator buffers, then a commit that arrives on that buffer's
+// "full" barrier; epilogue warps arrive on its "empty" barrier when they have drained it.
+// Every wait is bounded: when one runs out the kernel raises an error word, skips the remaining work,
+// frees its tensor memory and returns.
+#include "ts_internal.h"
+#include "ts_scan.cuh"
+
+namespace ts {
+
+constexpr int EPI_WARPS = 4 * MMA_S;
+constexpr int MMA_THREADS = (EPI_WARPS + 1) * 32;
+constexpr int BLK_N = 128;
+constexpr uint32_t TMEM_COLS = 256;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait; false = gave up (and said so in *abort / *err)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int* err) {
+  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort) return false;
+    if (i > 64) __nanosleep(64);
+  }
+  *abort = 1;
+  if (err) atomicExch(err, 1);
+  return false;
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// shared-memory matrix descriptor: 128-byte swizzle, descriptor version 1 (sm_100)
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// instruction descriptor: D = f32, A = B = bf16, A K-major, B MN-major, M = 128, N = n
+__device__ __forceinline__ uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) {
+  extern __shared__ unsigned char smem_raw[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int P = a.P_dev ? *a.P_dev : a.P;
+  if (P <= 0) return;  // an empty level: uniform exit before anything is allocated
+
+  const int r = a.r, rp = (r + 63) / 64 * 64, V = a.V, TV = a.TV, K = a.K;
+  const int tile = blockIdx.x, t0 = tile * TV, tlen = min(TV, V - t0);
+  const int nslab = TV / 64;
+  const uint32_t slab_bytes = (uint32_t)rp * 128u;       // one 64-token slab of W
+  const uint32_t a_slab_bytes = 128u * 128u;             // 128 rows x 128 B
+  unsigned char* sm = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  unsigned char* Ws = sm;
+  unsigned char* As = Ws + (size_t)nslab * slab_bytes;
+  float* ghi = reinterpret_cast<float*>(As + (size_t)(rp / 64) * a_slab_bytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ghi + 512);
+  uint64_t* a_full = bars;            // epilogue threads -> MMA: the A tile of this group is in place
+  uint64_t* t_full = bars + 1;        // [2] MMA -> epilogue: accumulator buffer written
+  uint64_t* t_empty = bars + 3;       // [2] epilogue -> MMA: accumulator buffer drained
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 6);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  const __nv_bfloat16* Wg = reinterpret_cast<const __nv_bfloat16*>(a.W);
+  const __nv_bfloat16* Ug = reinterpret_cast<const __nv_bfloat16*>(a.U);
+  const __nv_bfloat16* Ag = reinterpret_cast<const __nv_bfloat16*>(a.A);
+
+  // ---- set-up ------------------------------------------------------------------------------------
+  if (warp == EPI_WARPS) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    mbar_init(a_full, EPI_WARPS * 32);
+    mbar_init(t_full, 1); mbar_init(t_full + 1, 1);
+    mbar_init(t_empty, EPI_WARPS); mbar_init(t_empty + 1, EPI_WARPS);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  {  // W tile: 16-byte chunks (8 tokens of one row), swizzled: chunk j of row k lands at chunk j ^ (k & 7)
+    const int per_slab = rp * 8;
+    for (int idx = tid; idx < nslab * per_slab; idx += MMA_THREADS) {
+      const int slab = idx / per_slab, rem = idx % per_slab, k = rem >> 3, j = rem & 7;
+      const int tok = t0 + slab * 64 + j * 8;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (k < r && tok < V) v = __ldg(reinterpret_cast<const uint4*>(Wg + (size_t)k * V + tok));
+      *reinterpret_cast<uint4*>(Ws + (size_t)slab * slab_bytes + k * 128 + ((j ^ (k & 7)) << 4)) = v;
+    }
+  }
+  fill_gumbel_bounds(ghi, tid, MMA_THREADS);
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+
+  const int R = mma_replicas(P);
+  const int ngroups = R > 1 ? 1 : (P + 127) / 128;
+  const int nblk = (tlen + BLK_N - 1) / BLK_N;
+  const float T = a.T, invT = T > 0.f ? 1.f / T : 1.f;
+  const int rw = rec_words(K);
+
+  if (warp < EPI_WARPS) {
+    // ======================= epilogue warps =======================================================
+    const int q = warp & 3, s = warp >> 2;
+    const int row = q * 32 + lane;
+    const int e = warp * 32 + lane;  // 0..255
+    const int cpr = rp / 8;          // 16-byte chunks per A row
+    bool alive = true;
+    for (int g = 0; g < ngroups && alive; ++g) {
+      // gather this group's parent rows A[x_p] into the swizzled A tile
+      for (int idx = e; idx < 128 * cpr; idx += EPI_WARPS * 32) {
+        const int rr = idx / cpr, ck = idx % cpr;
+        const int p = R > 1 ? rr % (128 / R) : g * 128 + rr;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (p < P && ck * 8 < r) v = __ldg(reinterpret_cast<const uint4*>(Ag + (size_t)a.p_token[p] * r + ck * 8));
+        *reinterpret_cast<uint4*>(As + (size_t)(ck >> 3) * a_slab_bytes + rr * 128 + (((ck & 7) ^ (rr & 7)) << 4)) = v;
+      }
+      fence_async_smem();
+      mbar_arrive(a_full);
+
+      const int p = R > 1 ? row % (128 / R) : g * 128 + row;
+      const int rho = R > 1 ? row / (128 / R) : 0;   // uniform within a warp (128/R is a multiple of 32)
+      const bool active = p < P;
+      int req = 0; uint64_t hash = 0; const __nv_bfloat16* Urow = Ug;
+      if (active) {
+        req = a.p_req[p]; hash = a.p_hash[p];
+        Urow = Ug + ((size_t)req * a.D + a.p_depth[p]) * V;
+      }
+      RowScan st;
+      st.init(K);
+      const int pc = active ? p : 0;
+      const int pid = ((tile * MMA_S + s) * R + rho) % K;   // which of the parent's K slots this piece feeds
+      const SharedThr gl{a.slots + (size_t)pc * K, pid};
+      const SharedThr gk{a.slots + ((size_t)a.cap + pc) * K, pid};
+      for (int nb = 0; nb < nblk; ++nb) {
+        const int it = g * nblk + nb, tb = it & 1, u = it >> 1;
+        int ok = 1;
+        if (lane == 0) ok = mbar_wait(t_full + tb, u & 1, s_abort, a.err) ? 1 : 0;
+        ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+        if (!ok) { alive = false; break; }
+        tc_fence_after();
+        const int nch = min(8, (tlen - nb * BLK_N + 15) / 16);
+        for (int c = 0; c < nch; ++c) {
+          const int cg = nb * 8 + c;
+          if (cg % R != rho || (cg / R) % MMA_S != s) continue;   // warp-uniform
+          float acc[16];
+          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * BLK_N + c * 16), acc);
+          if (active) {
+            const int v0 = t0 + cg * 16;
+            const int valid = min(16, V - v0);   // 8 or 16: V and v0 are multiples of 8
+            float ub[16];
+            unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(Urow + v0)), ub);
+            if (valid > 8) unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(Urow + v0 + 8)), ub + 8);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] + ub[i] : 0.f;
+            scan_chunk(st, acc, v0, valid, T, invT, a.seed, req, hash, ghi, gl, gk);
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(t_empty + tb);
+      }
+      if (alive && active) {
+        const int gslot = R > 1 ? row : g * 128 + row;
+        st.store(a.rec + ((size_t)(tile * MMA_S + s) * a.cap + gslot) * rw);
+      }
+    }
+  } else if (lane == 0) {
+    // ======================= MMA issuer ===========================================================
+    const uint32_t ws_addr = smem_u32(Ws), as_addr = smem_u32(As);
+    bool alive = true;
+    for (int g = 0; g < ngroups && alive; ++g) {
+      if (!mbar_wait(a_full, g & 1, s_abort, a.err)) break;
+      tc_fence_after();
+      for (int nb = 0; nb < nblk; ++nb) {
+        const int it = g * nblk + nb, tb = it & 1, u = it >> 1;
+        if (u >= 1) {
+          if (!mbar_wait(t_empty + tb, (u - 1) & 1, s_abort, a.err)) { alive = false; break; }
+          tc_fence_after();
+        }
+        const int n = (tlen - nb * BLK_N > 64) ? 128 : 64;
+        const uint32_t idesc = instr_desc(n);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
+        for (int ks = 0; ks < rp / 16; ++ks) {
+          const uint64_t adesc = smem_desc(as_addr + (uint32_t)(ks >> 2) * a_slab_bytes + (uint32_t)(ks & 3) * 32u, 16u, 1024u);
+          const uint64_t bdesc = smem_desc(ws_addr + (uint32_t)(2 * nb) * slab_bytes + (uint32_t)ks * 2048u, slab_bytes, 1024u);
+          mma_bf16(d_tmem, adesc, bdesc, idesc, ks > 0 ? 1u : 0u);
+        }
+        mma_commit(t_full + tb);
+      }
+    }
+  }
+  // ---- tear-down -----------------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == EPI_WARPS) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+static size_t mma_smem_bytes(const ts_config& c, int TV) {
+  const size_t rp = (size_t)(c.r + 63) / 64 * 64;
+  return (size_t)(TV / 64) * rp * 128 + (rp / 64) * 128 * 128 + 512 * 4 + 64 + 1024;
+}
+
+// tile size for the tensor-core path: W tile + A tile + table + barriers within the shared-memory limit,
+// a whole number of waves over the SMs
+bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
+  const size_t rp = (size_t)(c.r + 63) / 64 * 64;
+  const size_t fixed = (rp / 64) * 128 * 128 + 512 * 4 + 64 + 1024;
+  if ((size_t)max_smem < fixed + rp * 128) return false;
+  int tv_max = (int)(((size_t)max_smem - fixed) / (rp * 2) / 64) * 64;
+  if (tv_max < 64) return false;
+  if (tv_max > 4096) tv_max = 4096;
+  const int min_tiles = (c.V + tv_max - 1) / tv_max;
+  const int waves = (min_tiles + num_sms - 1) / num_sms;
+  const int want = waves * num_sms;
+  int tv = ((c.V + want - 1) / want + 63) / 64 * 64;
+  if (tv > tv_max) tv = tv_max;
+  out->TV = tv;
+  out->ntiles = (c.V + tv - 1) / tv;
+  out->smem = mma_smem_bytes(c, tv);
+  return out->ntiles <= 4096;
+}
+
+cudaError_t score_mma_setup(ts_ctx* ctx) {
+  return cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
+}
+
+cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st) {
+  score_mma_kernel<<<a.ntiles, MMA_THREADS, ctx->tile.smem, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace ts

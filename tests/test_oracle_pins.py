@@ -59,11 +59,12 @@ def test_philox_matches_independent_torch_implementation():
 def test_stream_layout_and_uniform_range():
     seed, req, h = 0x1234567890ABCDEF, 5, 0xDEADBEEFCAFEF00D
     key = (seed & 0xFFFFFFFF, seed >> 32)
-    for v in (0, 1, 15, 16, 17, 151935):
-        coarse_w = oracle.philox4x32_10((v >> 4, h & 0xFFFFFFFF, h >> 32, req | (1 << 24)), key)
-        fine_w = oracle.philox4x32_10((v >> 2, h & 0xFFFFFFFF, h >> 32, req | (2 << 24)), key)
-        coarse = (coarse_w[(v & 15) >> 2] >> (8 * (v & 3))) & 0xFF
-        x = (coarse << 24) | (fine_w[v & 3] >> 8)
+    for v in (0, 1, 7, 8, 15, 16, 17, 151935):
+        coarse_w = oracle.philox4x32_10((v >> 3, h & 0xFFFFFFFF, h >> 32, req | (1 << 24)), key)
+        fine_w = oracle.philox4x32_10((v >> 3, h & 0xFFFFFFFF, h >> 32, req | (2 << 24)), key)
+        coarse = (coarse_w[(v & 7) >> 1] >> (16 * (v & 1))) & 0xFFFF
+        fine = (fine_w[(v & 7) >> 1] >> (16 * (v & 1))) & 0xFFFF
+        x = (coarse << 16) | fine
         assert oracle.u_gumbel(seed, req, h, v) == (x + 0.5) / 2 ** 32
     w = oracle.philox4x32_10((3, h & 0xFFFFFFFF, h >> 32, req | (3 << 24)), key)
     assert oracle.u_accept(seed, req, h, 3) == (w[0] + 0.5) / 2 ** 32
