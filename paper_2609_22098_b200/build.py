@@ -19,6 +19,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-o", LIB] + srcs
+    extra = os.environ.get("TS_NVCC_FLAGS", "").split()
+    cmd[1:1] = extra
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

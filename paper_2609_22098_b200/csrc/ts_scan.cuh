@@ -11,49 +11,106 @@ namespace ts {
 __host__ __device__ __forceinline__ int rec_words(int K) { return (4 + 5 * K + 3) & ~3; }  // 16-byte multiple
 
 // Candidate lists of one (piece, parent): K best logits and K best sampling keys seen so far, both
-// sorted descending.  They are indexed dynamically, so they live in local memory; everything that
-// touches them sits in the out-of-line functions below, which keeps the hot loop small.
-struct RowLists {
+// sorted descending.  Two holders with the same interface:
+//   RegLists<8>  for K <= 8: fixed-size arrays that only ever see compile-time indices, so they stay in
+//                registers and an insertion is a short predicated shift network;
+//   MemLists     for K <= 16: dynamically indexed (local memory), insertion out of line.
+template <int KR>
+struct RegLists {
+  // The lists always hold KR >= K entries (every index below is a compile-time constant, which is what
+  // keeps them in registers); the pruning threshold is the KR-th entry, a little looser than the K-th
+  // when K < KR, and the record keeps the first K.
+  int K;
+  float topv[KR]; int topi[KR];
+  float keyv[KR]; int keyi[KR]; float keyl[KR];
+  __device__ __forceinline__ void init(int K_) {
+    K = K_;
+#pragma unroll
+    for (int i = 0; i < KR; ++i) { topv[i] = -INFINITY; topi[i] = -1; keyv[i] = -INFINITY; keyi[i] = -1; keyl[i] = 0.f; }
+  }
+  // Callers offer a value only when it beats the last entry.  Tokens arrive in increasing order within
+  // a piece, so an equal value never displaces an earlier one.
+  __device__ __forceinline__ float insert_top(float v, int tok) {
+#pragma unroll
+    for (int j = KR - 1; j >= 0; --j) {
+      const bool up = (j > 0) && (v > topv[j > 0 ? j - 1 : 0]);   // entry j-1 moves down into j
+      const bool here = !up && (j == KR - 1 || v > topv[j]);      // v lands in j
+      if (up) { topv[j] = topv[j > 0 ? j - 1 : 0]; topi[j] = topi[j > 0 ? j - 1 : 0]; }
+      else if (here) { topv[j] = v; topi[j] = tok; }
+    }
+    return topv[KR - 1];
+  }
+  __device__ __forceinline__ float insert_key(float key, int tok, float logit) {
+#pragma unroll
+    for (int j = KR - 1; j >= 0; --j) {
+      const bool up = (j > 0) && (key > keyv[j > 0 ? j - 1 : 0]);
+      const bool here = !up && (j == KR - 1 || key > keyv[j]);
+      if (up) { keyv[j] = keyv[j > 0 ? j - 1 : 0]; keyi[j] = keyi[j > 0 ? j - 1 : 0]; keyl[j] = keyl[j > 0 ? j - 1 : 0]; }
+      else if (here) { keyv[j] = key; keyi[j] = tok; keyl[j] = logit; }
+    }
+    return keyv[KR - 1];
+  }
+  __device__ __forceinline__ void store(float* f, int* ii) const {
+#pragma unroll
+    for (int j = 0; j < KR; ++j)
+      if (j < K) { f[j] = topv[j]; ii[K + j] = topi[j]; f[2 * K + j] = keyv[j]; ii[3 * K + j] = keyi[j]; f[4 * K + j] = keyl[j]; }
+  }
+};
+
+struct MemListsData {
   int K;
   float topv[KMAX]; int topi[KMAX];
   float keyv[KMAX]; int keyi[KMAX]; float keyl[KMAX];
 };
-
-// Thread-private running state of one parent over the tokens scanned so far.
-struct RowScan {
-  float m, s0, sT;
-  float thrL, thrK;      // K-th best of this thread's own lists (-inf until they are full)
-  float gL, gK;          // launch-wide lower bounds of the parent's K-th best logit / key, as last read
-  float bestL, bestK;    // best logit / key this thread has published
-  RowLists L;
-
-  __device__ __forceinline__ void init(int K_) {
-    L.K = K_; m = -INFINITY; s0 = 0.f; sT = 0.f; thrL = -INFINITY; thrK = -INFINITY;
-    gL = -INFINITY; gK = -INFINITY; bestL = -INFINITY; bestK = -INFINITY;
-    for (int i = 0; i < KMAX; ++i) { L.topv[i] = -INFINITY; L.topi[i] = -1; L.keyv[i] = -INFINITY; L.keyi[i] = -1; L.keyl[i] = 0.f; }
-  }
-  // one record, 16-byte aligned
-  __device__ __forceinline__ void store(float* rec) const {
-    float4* r4 = reinterpret_cast<float4*>(rec);
-    r4[0] = make_float4(m, s0, sT, 0.f);
-    float* f = rec + 4;
-    int* ii = reinterpret_cast<int*>(rec) + 4;
-    const int K = L.K;
-    for (int j = 0; j < K; ++j) {
-      f[j] = L.topv[j]; ii[K + j] = L.topi[j]; f[2 * K + j] = L.keyv[j]; ii[3 * K + j] = L.keyi[j]; f[4 * K + j] = L.keyl[j];
-    }
-  }
-};
-
-// Insert into the logit list; returns the list's new K-th value.  Tokens arrive in increasing order
-// within a piece, so an equal value never displaces an earlier entry.
-static __device__ __noinline__ float insert_top(RowLists* L, float v, int tok) {
+static __device__ __noinline__ float mem_insert_top(MemListsData* L, float v, int tok) {
   const int K = L->K;
   int pos = K - 1;
   while (pos > 0 && v > L->topv[pos - 1]) { L->topv[pos] = L->topv[pos - 1]; L->topi[pos] = L->topi[pos - 1]; --pos; }
   L->topv[pos] = v; L->topi[pos] = tok;
   return L->topv[K - 1];
 }
+static __device__ __noinline__ float mem_insert_key(MemListsData* L, float key, int tok, float logit) {
+  const int K = L->K;
+  int pos = K - 1;
+  while (pos > 0 && key > L->keyv[pos - 1]) {
+    L->keyv[pos] = L->keyv[pos - 1]; L->keyi[pos] = L->keyi[pos - 1]; L->keyl[pos] = L->keyl[pos - 1]; --pos;
+  }
+  L->keyv[pos] = key; L->keyi[pos] = tok; L->keyl[pos] = logit;
+  return L->keyv[K - 1];
+}
+struct MemLists {
+  MemListsData d;
+  __device__ __forceinline__ void init(int K_) {
+    d.K = K_;
+    for (int i = 0; i < KMAX; ++i) { d.topv[i] = -INFINITY; d.topi[i] = -1; d.keyv[i] = -INFINITY; d.keyi[i] = -1; d.keyl[i] = 0.f; }
+  }
+  __device__ __forceinline__ float insert_top(float v, int tok) { return mem_insert_top(&d, v, tok); }
+  __device__ __forceinline__ float insert_key(float key, int tok, float logit) { return mem_insert_key(&d, key, tok, logit); }
+  __device__ __forceinline__ void store(float* f, int* ii) const {
+    const int K = d.K;
+    for (int j = 0; j < K; ++j) { f[j] = d.topv[j]; ii[K + j] = d.topi[j]; f[2 * K + j] = d.keyv[j]; ii[3 * K + j] = d.keyi[j]; f[4 * K + j] = d.keyl[j]; }
+  }
+};
+
+// Thread-private running state of one parent over the tokens scanned so far.
+template <class Lists>
+struct RowScan {
+  float m, s0, sT;
+  float thrL, thrK;      // K-th best of this thread's own lists (-inf until they are full)
+  float bestL, bestK;    // best logit / key this thread has published
+  int K;
+  Lists L;
+
+  __device__ __forceinline__ void init(int K_) {
+    K = K_; L.init(K_); m = -INFINITY; s0 = 0.f; sT = 0.f; thrL = -INFINITY; thrK = -INFINITY;
+    bestL = -INFINITY; bestK = -INFINITY;
+  }
+  // one record, 16-byte aligned
+  __device__ __forceinline__ void store(float* rec) const {
+    *reinterpret_cast<float4*>(rec) = make_float4(m, s0, sT, 0.f);
+    L.store(rec + 4, reinterpret_cast<int*>(rec) + 4);
+  }
+};
 
 // Upper bound of the Gumbel noise -log(-log u) given only the leading bits of the 32-bit uniform, with
 // a safety margin so that the bound never prunes a token the exact key would keep.  Table 0 is indexed
@@ -97,32 +154,36 @@ __device__ __forceinline__ unsigned slots_min(const SharedThr& g, int K) {
   return m;
 }
 
-// Exact sampling key of one token (low half of its uniform from the second generator stream) and, if
-// it beats both bounds, insertion into the key list.  Returns (new K-th key of the list, the key if
-// inserted else -inf).  Out of line: it runs for a few tokens per thousand once the bounds are warm.
-static __device__ __noinline__ float2 key_exact(RowLists* L, float base, float logit, uint32_t c16, int v, uint64_t seed,
-                                         int req, uint64_t hash, float thrK, float gK) {
+// Gumbel noise of token v from both halves of its uniform (the low half costs a second generator call;
+// out of line because it runs for a few tokens per thousand once the bounds are warm).
+static __device__ __noinline__ float gumbel_exact(uint32_t c16, int v, uint64_t seed, int req, uint64_t hash) {
   const uint4 fw = stream_words(seed, req, hash, STREAM_GUMBEL_FINE, (uint32_t)v >> 3);
   const uint32_t f16 = (word_of(fw, (v & 7) >> 1) >> (16 * (v & 1))) & 0xFFFFu;
-  const float key = base + gumbel_from_bits((c16 << 16) | f16);
-  if (!(key > thrK && key >= gK)) return make_float2(thrK, -INFINITY);
-  const int K = L->K;
-  int pos = K - 1;
-  while (pos > 0 && key > L->keyv[pos - 1]) {
-    L->keyv[pos] = L->keyv[pos - 1]; L->keyi[pos] = L->keyi[pos - 1]; L->keyl[pos] = L->keyl[pos - 1]; --pos;
-  }
-  L->keyv[pos] = key; L->keyi[pos] = v; L->keyl[pos] = logit;
-  return make_float2(L->keyv[K - 1], key);
+  return gumbel_from_bits((c16 << 16) | f16);
+}
+
+// register-array element by run-time index (a select chain: the array stays in registers)
+__device__ __forceinline__ float pick16(const float* a, int i) {
+  float r = a[0];
+#pragma unroll
+  for (int j = 1; j < 16; ++j) r = (i == j) ? a[j] : r;
+  return r;
+}
+__device__ __forceinline__ uint32_t pick8(const uint4& a, const uint4& b, int i) {
+  uint32_t r = a.x;
+  r = i == 1 ? a.y : r; r = i == 2 ? a.z : r; r = i == 3 ? a.w : r;
+  r = i == 4 ? b.x : r; r = i == 5 ? b.y : r; r = i == 6 ? b.z : r; r = i == 7 ? b.w : r;
+  return r;
 }
 
 // One 16-token chunk of one parent: logits l[0..16) for tokens v0.., `valid` of them inside V.
-__device__ __forceinline__ void scan_chunk(RowScan& st, const float* l, int v0, int valid, float T, float invT,
+// gL / gK: launch-wide lower bounds of the parent's K-th best logit / key as the caller last read them.
+// The common case is branch-free: sums, then one bit per token saying whether it can still be a
+// candidate; the few tokens whose bit is set are handled one at a time by a single copy of the code.
+template <class Lists>
+__device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, int v0, int valid, float T, float invT,
                                            uint64_t seed, int req, uint64_t hash, const float* ghi,
-                                           const SharedThr& gl, const SharedThr& gk) {
-  const int K = st.L.K;
-  // launch-wide bounds: loads issued first, consumed after the sums below
-  const unsigned rdL = slots_min(gl, K);
-  const unsigned rdK = T > 0.f ? slots_min(gk, K) : 0u;
+                                           float gL, float gK, const SharedThr& gl, const SharedThr& gk) {
   float cm = -INFINITY;
 #pragma unroll
   for (int i = 0; i < CHUNK; ++i) if (i < valid) cm = fmaxf(cm, l[i]);
@@ -144,34 +205,43 @@ __device__ __forceinline__ void scan_chunk(RowScan& st, const float* l, int v0, 
   }
   st.s0 += a0;
   st.sT += two ? aT : a0;
-  st.gL = fmaxf(st.gL, dec_f(rdL));
-  st.gK = fmaxf(st.gK, dec_f(rdK));
   // top-K logits: a token below the launch-wide bound cannot be among the parent's K best
-  if (cm > st.thrL && cm >= st.gL) {
+  if (cm > st.thrL && cm >= gL) {
+    uint32_t mk = 0;
 #pragma unroll
-    for (int i = 0; i < CHUNK; ++i)
-      if (i < valid && l[i] > st.thrL && l[i] >= st.gL) st.thrL = insert_top(&st.L, l[i], v0 + i);
+    for (int i = 0; i < CHUNK; ++i) mk |= (uint32_t)(i < valid && l[i] > st.thrL && l[i] >= gL) << i;
+#pragma unroll 1
+    while (mk) {
+      const int i = __ffs(mk) - 1;
+      mk &= mk - 1;
+      const float li = pick16(l, i);
+      if (li > st.thrL) st.thrL = st.L.insert_top(li, v0 + i);
+    }
     if (cm > st.bestL) { st.bestL = cm; publish(gl, cm); }
   }
   if (T > 0.f) {
     // high half of each token's uniform: one generator call per eight tokens
     const uint4 cw0 = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, (uint32_t)v0 >> 3);
     const uint4 cw1 = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, ((uint32_t)v0 >> 3) + 1u);
-    float kmax = -INFINITY;
+    const float thr = fmaxf(st.thrK, gK);
+    uint32_t mk = 0;
 #pragma unroll
     for (int i = 0; i < CHUNK; ++i) {
-      if (i < valid) {
-        const uint32_t word = word_of(i < 8 ? cw0 : cw1, (i & 7) >> 1);
-        const uint32_t c16 = (word >> (16 * (i & 1))) & 0xFFFFu;
-        const float base = l[i] * invT;
-        // the leading bits bound the noise from above; almost every token stops here
-        const float bnd = base + ((c16 >> 8) != 255u ? ghi[c16 >> 8] : ghi[256 + (c16 & 255u)]);
-        if (bnd > st.thrK && bnd >= st.gK) {
-          const float2 r = key_exact(&st.L, base, l[i], c16, v0 + i, seed, req, hash, st.thrK, st.gK);
-          st.thrK = r.x;
-          kmax = fmaxf(kmax, r.y);
-        }
-      }
+      const uint32_t word = word_of(i < 8 ? cw0 : cw1, (i & 7) >> 1);
+      const uint32_t c16 = (word >> (16 * (i & 1))) & 0xFFFFu;
+      // the leading bits bound the noise from above; almost every token stops here
+      const float bnd = l[i] * invT + ((c16 >> 8) != 255u ? ghi[c16 >> 8] : ghi[256 + (c16 & 255u)]);
+      mk |= (uint32_t)(i < valid && bnd >= thr) << i;
+    }
+    float kmax = -INFINITY;
+#pragma unroll 1
+    while (mk) {
+      const int i = __ffs(mk) - 1;
+      mk &= mk - 1;
+      const float li = pick16(l, i);
+      const uint32_t c16 = (pick8(cw0, cw1, i >> 1) >> (16 * (i & 1))) & 0xFFFFu;
+      const float key = li * invT + gumbel_exact(c16, v0 + i, seed, req, hash);
+      if (key > st.thrK && key >= gK) { st.thrK = st.L.insert_key(key, v0 + i, li); kmax = fmaxf(kmax, key); }
     }
     if (kmax > st.bestK) { st.bestK = kmax; publish(gk, kmax); }
   }

@@ -12,7 +12,7 @@
 
 namespace ts {
 
-template <typename TIn>
+template <typename TIn, class Lists>
 __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int r = a.r, TV = a.TV, V = a.V;
@@ -60,8 +60,9 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
     const uint64_t hash = a.p_hash[p];
     for (int k = 0; k < r; ++k) as[k * SCORE_THREADS + tid] = Elem<TIn>::to_f(Ag[(size_t)ptok * r + k]);
     const TIn* Urow = Ug + ((size_t)req * a.D + dep) * V + t0;
-    RowScan st;
+    RowScan<Lists> st;
     st.init(K);
+    float gL = -INFINITY, gK = -INFINITY;
     const SharedThr gl{a.slots + (size_t)p * K, tile % K};
     const SharedThr gk{a.slots + ((size_t)a.cap + p) * K, tile % K};
     for (int c0 = 0; c0 < tlen; c0 += CHUNK) {
@@ -86,7 +87,11 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
 #pragma unroll
         for (int i = 0; i < CHUNK; ++i) l[i] = fmaf(ak, w[i], l[i]);
       }
-      scan_chunk(st, l, t0 + c0, valid, T, invT, a.seed, req, hash, ghi, gl, gk);
+      if ((c0 & (4 * CHUNK - 1)) == 0) {  // refresh the launch-wide bounds every fourth chunk
+        gL = fmaxf(gL, dec_f(slots_min(gl, K)));
+        if (T > 0.f) gK = fmaxf(gK, dec_f(slots_min(gk, K)));
+      }
+      scan_chunk(st, l, t0 + c0, valid, T, invT, a.seed, req, hash, ghi, gL, gK, gl, gk);
     }
     st.store(a.rec + ((size_t)tile * a.cap + p) * rw);  // piece = (tile, 0), slot = p
   }
@@ -254,9 +259,11 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
       e = launch_score_mma(ctx, a, st);
       if (e != cudaSuccess) return e;
     } else if (c.dt_U == TS_DTYPE_BF16) {
-      score_tile_kernel<__nv_bfloat16><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
+      if (c.K <= 8) score_tile_kernel<__nv_bfloat16, RegLists<8>><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
+      else score_tile_kernel<__nv_bfloat16, MemLists><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
     } else {
-      score_tile_kernel<float><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
+      if (c.K <= 8) score_tile_kernel<float, RegLists<8>><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
+      else score_tile_kernel<float, MemLists><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
     }
   }
   e = cudaGetLastError();
@@ -277,10 +284,12 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
 
 cudaError_t score_setup(ts_ctx* ctx) {
   if (ctx->use_mma) return score_mma_setup(ctx);
-  cudaError_t e = cudaFuncSetAttribute(score_tile_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)ctx->tile.smem);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(score_tile_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
+  const int sm = (int)ctx->tile.smem;
+  cudaError_t e = cudaFuncSetAttribute(score_tile_kernel<__nv_bfloat16, RegLists<8>>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_tile_kernel<__nv_bfloat16, MemLists>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_tile_kernel<float, RegLists<8>>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(score_tile_kernel<float, MemLists>, cudaFuncAttributeMaxDynamicSharedMemorySize, sm);
+  return e;
 }
 
 }  // namespace ts

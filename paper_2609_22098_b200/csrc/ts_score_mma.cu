@@ -19,10 +19,20 @@
 
 namespace ts {
 
+#ifdef TS_DEBUG_TIMING
+// developer aid: per-CTA timestamps (globaltimer ns) of the phases of one launch
+__device__ unsigned long long g_dbg[148 * 64];
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define DBG(slot) do { if ((threadIdx.x & 31) == 0 && blockIdx.x < 148) g_dbg[blockIdx.x * 64 + (slot)] = gtime(); } while (0)
+#else
+#define DBG(slot) do { } while (0)
+#endif
+
 constexpr int EPI_WARPS = 4 * MMA_S;
-constexpr int MMA_THREADS = (EPI_WARPS + 1) * 32;
+constexpr int MMA_THREADS = (EPI_WARPS + 2) * 32;   // epilogue warps, the MMA warp, the bounds-refresh warp
 constexpr int BLK_N = 128;
-constexpr uint32_t TMEM_COLS = 256;
+constexpr int NBUF = 4;                 // accumulator buffers of BLK_N columns in tensor memory
+constexpr uint32_t TMEM_COLS = NBUF * BLK_N;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -88,6 +98,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+template <class Lists>
 __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -105,25 +116,29 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
   float* ghi = reinterpret_cast<float*>(As + (size_t)(rp / 64) * a_slab_bytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(ghi + 512);
   uint64_t* a_full = bars;            // epilogue threads -> MMA: the A tile of this group is in place
-  uint64_t* t_full = bars + 1;        // [2] MMA -> epilogue: accumulator buffer written
-  uint64_t* t_empty = bars + 3;       // [2] epilogue -> MMA: accumulator buffer drained
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 6);
+  uint64_t* t_full = bars + 1;             // [NBUF] MMA -> epilogue: accumulator buffer written
+  uint64_t* t_empty = bars + 1 + NBUF;     // [NBUF] epilogue -> MMA: accumulator buffer drained
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 + 2 * NBUF);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  // per-row copies of the launch-wide pruning bounds (logit, key), refreshed once per block of tokens
+  volatile unsigned* s_thr = reinterpret_cast<volatile unsigned*>(s_tmem + 4);   // [group parity][2][128]
+  volatile int* s_done = reinterpret_cast<volatile int*>(s_tmem + 2);             // epilogue warps finished
 
   const __nv_bfloat16* Wg = reinterpret_cast<const __nv_bfloat16*>(a.W);
   const __nv_bfloat16* Ug = reinterpret_cast<const __nv_bfloat16*>(a.U);
   const __nv_bfloat16* Ag = reinterpret_cast<const __nv_bfloat16*>(a.A);
 
   // ---- set-up ------------------------------------------------------------------------------------
+  if (warp == 0) DBG(0);
   if (warp == EPI_WARPS) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   if (tid == 0) {
     mbar_init(a_full, EPI_WARPS * 32);
-    mbar_init(t_full, 1); mbar_init(t_full + 1, 1);
-    mbar_init(t_empty, EPI_WARPS); mbar_init(t_empty + 1, EPI_WARPS);
+    for (int i = 0; i < NBUF; ++i) { mbar_init(t_full + i, 1); mbar_init(t_empty + i, EPI_WARPS); }
     *s_abort = 0;
+    *s_done = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   {  // W tile: 16-byte chunks (8 tokens of one row), swizzled: chunk j of row k lands at chunk j ^ (k & 7)
@@ -136,12 +151,16 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
       *reinterpret_cast<uint4*>(Ws + (size_t)slab * slab_bytes + k * 128 + ((j ^ (k & 7)) << 4)) = v;
     }
   }
+  if (warp == 0) DBG(1);
   fill_gumbel_bounds(ghi, tid, MMA_THREADS);
+  for (int i = tid; i < 512; i += MMA_THREADS) s_thr[i] = 0u;
+  if (warp == 0) DBG(2);
   fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
+  if (warp == 0) DBG(3);
 
   const int R = mma_replicas(P);
   const int ngroups = R > 1 ? 1 : (P + 127) / 128;
@@ -167,6 +186,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
       }
       fence_async_smem();
       mbar_arrive(a_full);
+      if (warp == 0) DBG(4);
 
       const int p = R > 1 ? row % (128 / R) : g * 128 + row;
       const int rho = R > 1 ? row / (128 / R) : 0;   // uniform within a warp (128/R is a multiple of 32)
@@ -176,19 +196,27 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
         req = a.p_req[p]; hash = a.p_hash[p];
         Urow = Ug + ((size_t)req * a.D + a.p_depth[p]) * V;
       }
-      RowScan st;
+      RowScan<Lists> st;
       st.init(K);
+      // where this parent's cached bounds live: rows of group g use the buffer of parity g & 1.  That
+      // buffer last served group g-2; the refresh warp is at group g-1 or g by now (every warp has
+      // passed the A-tile barrier of g-1), so clearing it here cannot be overwritten with stale values.
+      const int prow = (g & 1) * 256 + (R > 1 ? row % (128 / R) : row);
+      if (s == 0) { s_thr[(g & 1) * 256 + row] = 0u; s_thr[(g & 1) * 256 + 128 + row] = 0u; }
+      uint4 nx0 = make_uint4(0, 0, 0, 0), nx1 = nx0;    // prefetched base logits of the next owned chunk
+      bool have_next = false;
       const int pc = active ? p : 0;
       const int pid = ((tile * MMA_S + s) * R + rho) % K;   // which of the parent's K slots this piece feeds
       const SharedThr gl{a.slots + (size_t)pc * K, pid};
       const SharedThr gk{a.slots + ((size_t)a.cap + pc) * K, pid};
       for (int nb = 0; nb < nblk; ++nb) {
-        const int it = g * nblk + nb, tb = it & 1, u = it >> 1;
+        const int it = g * nblk + nb, tb = it % NBUF, u = it / NBUF;
         int ok = 1;
         if (lane == 0) ok = mbar_wait(t_full + tb, u & 1, s_abort, a.err) ? 1 : 0;
         ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
         if (!ok) { alive = false; break; }
         tc_fence_after();
+        if (nb < 10 && g == 0) DBG(8 + warp * 6 + 0 + (nb >= 1 ? 2 : 0) + (nb >= 8 ? 2 : 0));
         const int nch = min(8, (tlen - nb * BLK_N + 15) / 16);
         for (int c = 0; c < nch; ++c) {
           const int cg = nb * 8 + c;
@@ -198,24 +226,62 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
           if (active) {
             const int v0 = t0 + cg * 16;
             const int valid = min(16, V - v0);   // 8 or 16: V and v0 are multiples of 8
+            // this chunk's base logits were requested one chunk ago; request the next owned chunk's now
+            const uint4 u0 = have_next ? nx0 : __ldg(reinterpret_cast<const uint4*>(Urow + v0));
+            const uint4 u1 = have_next ? nx1 : (valid > 8 ? __ldg(reinterpret_cast<const uint4*>(Urow + v0 + 8)) : make_uint4(0, 0, 0, 0));
+            {
+              const int cgn = cg + R * MMA_S;           // the next chunk this warp owns
+              const int vn = t0 + cgn * 16;
+              have_next = (cgn * 16 < tlen);
+              if (have_next) {
+                nx0 = __ldg(reinterpret_cast<const uint4*>(Urow + vn));
+                nx1 = (V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8)) : make_uint4(0, 0, 0, 0);
+              }
+            }
+            const float gLc = dec_f(s_thr[prow]), gKc = dec_f(s_thr[128 + prow]);   // kept fresh by the refresh warp
             float ub[16];
-            unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(Urow + v0)), ub);
-            if (valid > 8) unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(Urow + v0 + 8)), ub + 8);
+            unpack_bf16x8(u0, ub);
+            unpack_bf16x8(u1, ub + 8);
 #pragma unroll
             for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] + ub[i] : 0.f;
-            scan_chunk(st, acc, v0, valid, T, invT, a.seed, req, hash, ghi, gl, gk);
+            scan_chunk(st, acc, v0, valid, T, invT, a.seed, req, hash, ghi, gLc, gKc, gl, gk);
           }
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(t_empty + tb);
+        if (nb < 10 && g == 0) DBG(8 + warp * 6 + 1 + (nb >= 1 ? 2 : 0) + (nb >= 8 ? 2 : 0));
       }
       if (alive && active) {
         const int gslot = R > 1 ? row : g * 128 + row;
         st.store(a.rec + ((size_t)(tile * MMA_S + s) * a.cap + gslot) * rw);
       }
+      if (lane == 0) atomicAdd((int*)s_done, 1);   // one tick per warp per group
     }
-  } else if (lane == 0) {
+    if (!alive && lane == 0) atomicAdd((int*)s_done, 1 << 20);   // gave up: release the refresh warp
+  } else if (warp == EPI_WARPS + 1) {
+    // ======================= bounds-refresh warp ====================================================
+    // keeps the shared-memory copies of every row's launch-wide pruning bounds current, so that the
+    // epilogue threads never wait on those (contended) global words
+    for (int g = 0; g < ngroups; ++g) {
+      const int per = R > 1 ? 128 / R : 128;
+      for (uint32_t spin = 0; spin < WAIT_LIMIT; ++spin) {
+        if (*s_done >= (g + 1) * EPI_WARPS || *s_abort) break;
+        for (int rr = lane; rr < per; rr += 32) {
+          const int p = R > 1 ? rr : g * 128 + rr;
+          if (p >= P) continue;
+          unsigned mL = __ldcg(a.slots + (size_t)p * K), mK = __ldcg(a.slots + ((size_t)a.cap + p) * K);
+          for (int j = 1; j < K; ++j) {
+            mL = min(mL, __ldcg(a.slots + (size_t)p * K + j));
+            mK = min(mK, __ldcg(a.slots + ((size_t)a.cap + p) * K + j));
+          }
+          s_thr[(g & 1) * 256 + rr] = mL; s_thr[(g & 1) * 256 + 128 + rr] = mK;
+        }
+        __nanosleep(200);
+      }
+      __syncwarp();
+    }
+  } else if (warp == EPI_WARPS && lane == 0) {
     // ======================= MMA issuer ===========================================================
     const uint32_t ws_addr = smem_u32(Ws), as_addr = smem_u32(As);
     bool alive = true;
@@ -223,7 +289,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
       if (!mbar_wait(a_full, g & 1, s_abort, a.err)) break;
       tc_fence_after();
       for (int nb = 0; nb < nblk; ++nb) {
-        const int it = g * nblk + nb, tb = it & 1, u = it >> 1;
+        const int it = g * nblk + nb, tb = it % NBUF, u = it / NBUF;
         if (u >= 1) {
           if (!mbar_wait(t_empty + tb, (u - 1) & 1, s_abort, a.err)) { alive = false; break; }
           tc_fence_after();
@@ -241,8 +307,10 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
     }
   }
   // ---- tear-down -----------------------------------------------------------------------------------
+  if (warp == 0) DBG(5);
   tc_fence_before();
   __syncthreads();
+  if (warp == 0) DBG(6);
   if (warp == EPI_WARPS) {
     __syncwarp();
     tc_fence_after();
@@ -252,14 +320,14 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
 
 static size_t mma_smem_bytes(const ts_config& c, int TV) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
-  return (size_t)(TV / 64) * rp * 128 + (rp / 64) * 128 * 128 + 512 * 4 + 64 + 1024;
+  return (size_t)(TV / 64) * rp * 128 + (rp / 64) * 128 * 128 + 512 * 4 + 128 + 512 * 4 + 1024;
 }
 
 // tile size for the tensor-core path: W tile + A tile + table + barriers within the shared-memory limit,
 // a whole number of waves over the SMs
 bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
-  const size_t fixed = (rp / 64) * 128 * 128 + 512 * 4 + 64 + 1024;
+  const size_t fixed = (rp / 64) * 128 * 128 + 512 * 4 + 128 + 512 * 4 + 1024;
   if ((size_t)max_smem < fixed + rp * 128) return false;
   int tv_max = (int)(((size_t)max_smem - fixed) / (rp * 2) / 64) * 64;
   if (tv_max < 64) return false;
@@ -276,11 +344,20 @@ bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out
 }
 
 cudaError_t score_mma_setup(ts_ctx* ctx) {
-  return cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
+  cudaError_t e = cudaFuncSetAttribute(score_mma_kernel<RegLists<8>>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(score_mma_kernel<MemLists>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
 }
 
+#ifdef TS_DEBUG_TIMING
+extern "C" int ts_debug_timing(unsigned long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, g_dbg, sizeof(g_dbg));
+}
+#endif
+
 cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st) {
-  score_mma_kernel<<<a.ntiles, MMA_THREADS, ctx->tile.smem, st>>>(a);
+  if (a.K <= 8) score_mma_kernel<RegLists<8>><<<a.ntiles, MMA_THREADS, ctx->tile.smem, st>>>(a);
+  else score_mma_kernel<MemLists><<<a.ntiles, MMA_THREADS, ctx->tile.smem, st>>>(a);
   return cudaGetLastError();
 }
 
