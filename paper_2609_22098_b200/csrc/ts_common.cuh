@@ -77,6 +77,8 @@ struct WsLayout {
   size_t vf_state;                       // VerifyState[B]
   size_t vf_part;                        // float[B][ntiles]
   size_t vf_barrier;                     // unsigned[4]
+  size_t vf_child;                       // int[2][B][N+1]: first child and child count of every node
+  size_t vf_lists;                       // int[2][B] reduction list, int[2][B] rescan list, int[8] counters
   size_t total;
 };
 
@@ -137,6 +139,8 @@ __host__ inline WsLayout make_layout(const ts_ctx* ctx, int B) {
   L.vf_state = take(b * sizeof(VerifyState));
   L.vf_part = take(b * (size_t)ctx->vt_n * 4);
   L.vf_barrier = take(64);
+  L.vf_child = take(2 * b * (N + 1) * 4);
+  L.vf_lists = take((4 * b + 8) * 4);
   L.total = off;
   return L;
 }
@@ -288,7 +292,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned nblocks, un
     while (*((volatile unsigned*)&bar[0]) < target) {
       if (*((volatile unsigned*)&bar[1]) != 0u) { ok = false; break; }
       if (++spins > (1u << 22)) { atomicExch(&bar[1], 1u); ok = false; break; }
-      __nanosleep(32);
+      if (spins > 256u) __nanosleep(32);
     }
     __threadfence();
   }

@@ -185,41 +185,75 @@ __global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d) 
     __syncthreads();
   }
   // ---- phase 3: place surviving candidates into free pool slots (deterministic order) --------
-  if (tid == 0) {
-    int s = 0, nnext = 0;
-    for (int c = 0; c < ncand; ++c) {
-      const size_t ci = cb + c;
-      if (!a.cd_valid[ci]) continue;
-      while (s < N && a.pl_alive[pb + s]) ++s;
-      if (s >= N) { a.status[b] = TS_ERR_OVERFLOW; break; }
-      const int slot = a.cd_parent[ci];
-      const int x = a.cd_tok[ci];
-      a.pl_alive[pb + s] = 1; a.pl_depth[pb + s] = d + 1; a.pl_parent[pb + s] = slot; a.pl_sib[pb + s] = a.cd_sib[ci];
-      a.pl_tok[pb + s] = x; a.pl_logkey[pb + s] = a.cd_logkey[ci]; a.pl_logS[pb + s] = a.cd_logS[ci];
-      a.pl_q0[pb + s] = a.cd_q0[ci]; a.pl_logqT[pb + s] = a.cd_logqT[ci]; a.pl_lseT[pb + s] = nanf("");
-      a.pl_hash[pb + s] = path_hash(slot < 0 ? 0ull : a.pl_hash[pb + slot], x);
-      a.pl_path[pb + s] = (slot < 0 ? 0ull : a.pl_path[pb + slot]) | ((uint64_t)a.cd_sib[ci] << shift);
-      a.cd_rank[cb + nnext] = s;  // reuse as "slots added at this level"
-      ++nnext;
-    }
-    // next level's parents: new nodes that can still have admissible children
-    int cnt = 0;
-    if (d + 1 < a.D) {
-      for (int i = 0; i < nnext; ++i) {
-        const int sl = a.cd_rank[cb + i];
-        if (!(a.pl_logS[pb + sl] < log_theta)) a.cd_rank[cb + cnt++] = sl;
+  // the t-th surviving candidate (in candidate order) takes the t-th free slot (in slot order)
+  __shared__ int s_free[256], s_new[256], s_warp[8];
+  __shared__ int s_run, s_nb;
+  const int lane = tid & 31, warp = tid >> 5;
+  {
+    const bool fr = tid < N && !a.pl_alive[pb + tid];
+    const unsigned bal = __ballot_sync(0xFFFFFFFFu, fr);
+    if (lane == 0) s_warp[warp] = __popc(bal);
+    __syncthreads();
+    int off = 0;
+    for (int w = 0; w < warp; ++w) off += s_warp[w];
+    if (fr) s_free[off + __popc(bal & ((1u << lane) - 1u))] = tid;
+    if (tid == 0) s_run = 0;
+    __syncthreads();
+  }
+  int nfree = 0;
+  for (int w = 0; w < 8; ++w) nfree += s_warp[w];
+  for (int c0 = 0; c0 < ncand; c0 += blockDim.x) {
+    const int c = c0 + tid;
+    const size_t ci = cb + c;
+    const bool v = c < ncand && a.cd_valid[ci];
+    const unsigned bal = __ballot_sync(0xFFFFFFFFu, v);
+    __syncthreads();  // s_warp is reused
+    if (lane == 0) s_warp[warp] = __popc(bal);
+    __syncthreads();
+    int off = s_run;
+    for (int w = 0; w < warp; ++w) off += s_warp[w];
+    const int t = off + __popc(bal & ((1u << lane) - 1u));
+    if (v) {
+      if (t >= nfree) { a.status[b] = TS_ERR_OVERFLOW; }
+      else {
+        const int sl = s_free[t];
+        const int slot = a.cd_parent[ci];
+        const int x = a.cd_tok[ci];
+        a.pl_alive[pb + sl] = 1; a.pl_depth[pb + sl] = d + 1; a.pl_parent[pb + sl] = slot; a.pl_sib[pb + sl] = a.cd_sib[ci];
+        a.pl_tok[pb + sl] = x; a.pl_logkey[pb + sl] = a.cd_logkey[ci]; a.pl_logS[pb + sl] = a.cd_logS[ci];
+        a.pl_q0[pb + sl] = a.cd_q0[ci]; a.pl_logqT[pb + sl] = a.cd_logqT[ci]; a.pl_lseT[pb + sl] = nanf("");
+        a.pl_hash[pb + sl] = path_hash(slot < 0 ? 0ull : a.pl_hash[pb + slot], x);
+        a.pl_path[pb + sl] = (slot < 0 ? 0ull : a.pl_path[pb + slot]) | ((uint64_t)a.cd_sib[ci] << shift);
+        s_new[t] = sl;
       }
     }
-    int nb = 0;
-    if (cnt > 0) nb = atomicAdd(&a.lvl_count[d + 1], cnt);
-    for (int i = 0; i < cnt; ++i) {
-      const int sl = a.cd_rank[cb + i];
-      const int li = nb + i;
+    __syncthreads();
+    if (tid == 0) { int tot = 0; for (int w = 0; w < 8; ++w) tot += s_warp[w]; s_run += tot; }
+    __syncthreads();
+  }
+  const int nnew = min(s_run, nfree);
+  // ---- phase 4: next level's parents = new nodes that can still have admissible children -----------
+  {
+    const bool par = (d + 1 < a.D) && tid < nnew && !(a.pl_logS[pb + s_new[tid]] < log_theta);
+    const unsigned bal = __ballot_sync(0xFFFFFFFFu, par);
+    __syncthreads();
+    if (lane == 0) s_warp[warp] = __popc(bal);
+    __syncthreads();
+    int off = 0, cnt = 0;
+    for (int w = 0; w < 8; ++w) { if (w < warp) off += s_warp[w]; cnt += s_warp[w]; }
+    if (tid == 0) {
+      s_nb = cnt > 0 ? atomicAdd(&a.lvl_count[d + 1], cnt) : 0;
+      a.req_nscored[b] += npar;
+      a.req_npar[b] = cnt;
+    }
+    __syncthreads();
+    if (tid == 0) a.req_base[b] = s_nb;
+    if (par) {
+      const int sl = s_new[tid];
+      const int li = s_nb + off + __popc(bal & ((1u << lane) - 1u));
       a.lst_req[nxt][li] = b; a.lst_depth[nxt][li] = d + 1; a.lst_token[nxt][li] = a.pl_tok[pb + sl];
       a.lst_hash[nxt][li] = a.pl_hash[pb + sl]; a.lst_slot[nxt][li] = sl;
     }
-    a.req_nscored[b] += npar;
-    a.req_npar[b] = cnt; a.req_base[b] = nb;
   }
 }
 

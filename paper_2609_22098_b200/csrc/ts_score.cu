@@ -102,55 +102,64 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
 // Every thread folds its share of the pieces into a private (max, sums) pair and private top-K
 // lists; the block then takes K rounds of arg-max over the list heads (value desc, token asc).
 // ------------------------------------------------------------------------------------------------
-constexpr int MERGE_THREADS = 128;
+constexpr int MERGE_THREADS = 256;
+constexpr int MERGE_WARPS = MERGE_THREADS / 32;
 
-struct TopList {
-  float v[KMAX]; int i[KMAX]; float l[KMAX]; int n;
-  __device__ __forceinline__ void init() { n = 0; }
-  __device__ __forceinline__ static bool better(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
-  __device__ __forceinline__ void insert(float val, int idx, float lg, int K) {
-    if (n == K && !better(val, idx, v[K - 1], i[K - 1])) return;
-    int pos = n < K ? n : K - 1;
-    while (pos > 0 && better(val, idx, v[pos - 1], i[pos - 1])) { v[pos] = v[pos - 1]; i[pos] = i[pos - 1]; l[pos] = l[pos - 1]; --pos; }
-    v[pos] = val; i[pos] = idx; l[pos] = lg;
-    if (n < K) ++n;
+__device__ __forceinline__ bool better(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
+
+// Sorted list (value desc, token asc) with compile-time indices only, so it lives in registers.
+// The head is always entry 0: taking it shifts the rest up.
+template <int KR>
+struct MList {
+  float v[KR]; int i[KR]; float l[KR];
+  __device__ __forceinline__ void init() {
+#pragma unroll
+    for (int j = 0; j < KR; ++j) { v[j] = -INFINITY; i[j] = 0x7FFFFFFF; l[j] = 0.f; }
+  }
+  __device__ __forceinline__ void insert(float val, int idx, float lg) {
+    if (!better(val, idx, v[KR - 1], i[KR - 1])) return;
+#pragma unroll
+    for (int j = KR - 1; j >= 0; --j) {
+      const bool up = (j > 0) && better(val, idx, v[j > 0 ? j - 1 : 0], i[j > 0 ? j - 1 : 0]);
+      if (up) { v[j] = v[j > 0 ? j - 1 : 0]; i[j] = i[j > 0 ? j - 1 : 0]; l[j] = l[j > 0 ? j - 1 : 0]; }
+      else if (j == KR - 1 || better(val, idx, v[j], i[j])) { v[j] = val; i[j] = idx; l[j] = lg; }
+    }
+  }
+  __device__ __forceinline__ void pop() {
+#pragma unroll
+    for (int j = 0; j + 1 < KR; ++j) { v[j] = v[j + 1]; i[j] = i[j + 1]; l[j] = l[j + 1]; }
+    v[KR - 1] = -INFINITY; i[KR - 1] = 0x7FFFFFFF; l[KR - 1] = 0.f;
   }
 };
 
 // K rounds of block-wide arg-max over the heads of the threads' sorted lists
-__device__ void block_select(const TopList& mine, int K, int* out_tok, float* out_val, float* s_v, int* s_i, float* s_l) {
+template <int KR>
+__device__ void block_select(MList<KR>& mine, int K, int* out_tok, float* out_val, float* s_v, int* s_i, float* s_l) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  int head = 0;
   for (int j = 0; j < K; ++j) {
-    float bv = head < mine.n ? mine.v[head] : -INFINITY;
-    int bi = head < mine.n ? mine.i[head] : 0x7FFFFFFF;
-    float bl = head < mine.n ? mine.l[head] : 0.f;
-    float wv = bv; int wi = bi; float wl = bl;
+    float wv = mine.v[0]; int wi = mine.i[0]; float wl = mine.l[0];
     for (int off = 16; off > 0; off >>= 1) {
       const float ov = __shfl_xor_sync(0xFFFFFFFFu, wv, off);
       const int oi = __shfl_xor_sync(0xFFFFFFFFu, wi, off);
       const float ol = __shfl_xor_sync(0xFFFFFFFFu, wl, off);
-      if (TopList::better(ov, oi, wv, wi)) { wv = ov; wi = oi; wl = ol; }
+      if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; wl = ol; }
     }
     if (lane == 0) { s_v[warp] = wv; s_i[warp] = wi; s_l[warp] = wl; }
     __syncthreads();
-    if (tid == 0) {
-      float gv = s_v[0]; int gi = s_i[0]; float gl = s_l[0];
-      for (int w = 1; w < MERGE_THREADS / 32; ++w)
-        if (TopList::better(s_v[w], s_i[w], gv, gi)) { gv = s_v[w]; gi = s_i[w]; gl = s_l[w]; }
-      s_v[MERGE_THREADS / 32] = gv; s_i[MERGE_THREADS / 32] = gi; s_l[MERGE_THREADS / 32] = gl;
-    }
-    __syncthreads();
-    const int gi = s_i[MERGE_THREADS / 32];
-    if (gi != 0x7FFFFFFF && head < mine.n && mine.i[head] == gi) ++head;  // tokens are unique per list
-    if (tid == 0) { out_tok[j] = gi == 0x7FFFFFFF ? -1 : gi; out_val[j] = gi == 0x7FFFFFFF ? 0.f : s_l[MERGE_THREADS / 32]; }
+    float gv = s_v[0]; int gi = s_i[0]; float gl = s_l[0];
+#pragma unroll
+    for (int w = 1; w < MERGE_WARPS; ++w)
+      if (better(s_v[w], s_i[w], gv, gi)) { gv = s_v[w]; gi = s_i[w]; gl = s_l[w]; }
+    if (gi != 0x7FFFFFFF && mine.i[0] == gi) mine.pop();  // tokens are unique per list
+    if (tid == 0) { out_tok[j] = gi == 0x7FFFFFFF ? -1 : gi; out_val[j] = gi == 0x7FFFFFFF ? 0.f : gl; }
     __syncthreads();
   }
 }
 
+template <int KR>
 __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
-  __shared__ float s_v[MERGE_THREADS / 32 + 1]; __shared__ int s_i[MERGE_THREADS / 32 + 1]; __shared__ float s_l[MERGE_THREADS / 32 + 1];
-  __shared__ float s_m[MERGE_THREADS / 32], s_s0[MERGE_THREADS / 32], s_sT[MERGE_THREADS / 32];
+  __shared__ float s_v[MERGE_WARPS]; __shared__ int s_i[MERGE_WARPS]; __shared__ float s_l[MERGE_WARPS];
+  __shared__ float s_m[MERGE_WARPS], s_s0[MERGE_WARPS], s_sT[MERGE_WARPS];
   const int P = a.P_dev ? *a.P_dev : a.P;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float invT = a.T > 0.f ? 1.f / a.T : 1.f;
@@ -158,30 +167,38 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
   const int R = a.mma ? mma_replicas(P) : 1;
   const int npieces = a.ntiles * a.S * R;
   for (int p = blockIdx.x; p < P; p += gridDim.x) {
+    // final launch-wide lower bounds of this parent's K-th best logit / key: entries below cannot win
+    const SharedThr gl{a.slots + (size_t)p * K, 0}, gk{a.slots + ((size_t)a.cap + p) * K, 0};
+    const float bL = dec_f(slots_min(gl, K)), bK = a.T > 0.f ? dec_f(slots_min(gk, K)) : -INFINITY;
     float m = -INFINITY, s0 = 0.f, sT = 0.f;
-    TopList top, key;
+    MList<KR> top, key;
     top.init(); key.init();
     for (int q = tid; q < npieces; q += MERGE_THREADS) {
       const int ts_ = q / R, rho = q % R;
       const int slot = R > 1 ? rho * (128 / R) + p : p;
       const float* rec = a.rec + ((size_t)ts_ * a.cap + slot) * rw;
-      const float4 h = *reinterpret_cast<const float4*>(rec);
+      const float4 h = __ldcg(reinterpret_cast<const float4*>(rec));
+      const float* f = rec + 4; const int* ii = reinterpret_cast<const int*>(rec) + 4;
+      // all entries of the record are requested at once (independent loads), then filtered
+      float tv[KR], kv[KR], kl[KR]; int ti[KR], ki[KR];
+#pragma unroll
+      for (int j = 0; j < KR; ++j) {
+        const bool in = j < K;
+        ti[j] = in ? __ldcg(ii + K + j) : -1;
+        tv[j] = in ? __ldcg(f + j) : 0.f;
+        ki[j] = (in && a.T > 0.f) ? __ldcg(ii + 3 * K + j) : -1;
+        kv[j] = (in && a.T > 0.f) ? __ldcg(f + 2 * K + j) : 0.f;
+        kl[j] = (in && a.T > 0.f) ? __ldcg(f + 4 * K + j) : 0.f;
+      }
       if (h.x == -INFINITY) continue;  // a piece that scanned nothing
       if (h.x > m) { const float d = m - h.x; s0 *= __expf(d); sT *= __expf(d * invT); m = h.x; }
       const float d = h.x - m;
       s0 += h.y * __expf(d); sT += h.z * __expf(d * invT);
-      const float* f = rec + 4; const int* ii = reinterpret_cast<const int*>(rec) + 4;
-      for (int j = 0; j < K; ++j) {
-        const int ti = ii[K + j];
-        if (ti < 0) break;
-        top.insert(f[j], ti, f[j], K);
+#pragma unroll
+      for (int j = 0; j < KR; ++j) {
+        if (ti[j] >= 0 && tv[j] >= bL) top.insert(tv[j], ti[j], tv[j]);
+        if (ki[j] >= 0 && kv[j] >= bK) key.insert(kv[j], ki[j], kl[j]);
       }
-      if (a.T > 0.f)
-        for (int j = 0; j < K; ++j) {
-          const int ki = ii[3 * K + j];
-          if (ki < 0) break;
-          key.insert(f[2 * K + j], ki, f[4 * K + j], K);
-        }
     }
     // fold the (max, sums) pairs
     for (int off = 16; off > 0; off >>= 1) {
@@ -199,9 +216,9 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
     __syncthreads();
     if (tid == 0) {
       float gm = -INFINITY;
-      for (int w = 0; w < MERGE_THREADS / 32; ++w) gm = fmaxf(gm, s_m[w]);
+      for (int w = 0; w < MERGE_WARPS; ++w) gm = fmaxf(gm, s_m[w]);
       float g0 = 0.f, gT = 0.f;
-      for (int w = 0; w < MERGE_THREADS / 32; ++w)
+      for (int w = 0; w < MERGE_WARPS; ++w)
         if (s_m[w] > -INFINITY) { g0 += s_s0[w] * __expf(s_m[w] - gm); gT += s_sT[w] * __expf((s_m[w] - gm) * invT); }
       a.lse0[p] = gm + logf(g0);
       a.lseT[p] = a.T > 0.f ? gm * invT + logf(gT) : gm + logf(g0);
@@ -209,9 +226,9 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
     __syncthreads();
     // leave the launch-wide pruning state of this parent clean for the next launch
     if (tid < 2 * K) a.slots[((size_t)(tid / K) * a.cap + p) * K + tid % K] = 0u;
-    block_select(top, K, a.top_tok + (size_t)p * K, a.top_logit + (size_t)p * K, s_v, s_i, s_l);
+    block_select<KR>(top, K, a.top_tok + (size_t)p * K, a.top_logit + (size_t)p * K, s_v, s_i, s_l);
     if (a.T > 0.f) {
-      block_select(key, K, a.draw_tok + (size_t)p * K, a.draw_logit + (size_t)p * K, s_v, s_i, s_l);
+      block_select<KR>(key, K, a.draw_tok + (size_t)p * K, a.draw_logit + (size_t)p * K, s_v, s_i, s_l);
     } else {
       if (tid < K) {
         a.draw_tok[(size_t)p * K + tid] = a.top_tok[(size_t)p * K + tid];
@@ -277,7 +294,8 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
   if (blocks < 1) blocks = 1;
   {
     ProfScope ps(ctx, K_MERGE, st);
-    merge_kernel<<<blocks, MERGE_THREADS, 0, st>>>(m);
+    if (c.K <= 8) merge_kernel<8><<<blocks, MERGE_THREADS, 0, st>>>(m);
+    else merge_kernel<16><<<blocks, MERGE_THREADS, 0, st>>>(m);
   }
   return cudaGetLastError();
 }

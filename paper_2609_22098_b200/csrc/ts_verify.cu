@@ -90,6 +90,9 @@ struct VerifyArgs {
   const float* z_max; const int* z_arg; const float* z_logs;
   int *acc_len, *acc_node, *acc_tok, *bonus; float* edge_stat; uint32_t* flags; int* status;
   VerifyState* state; float* part; unsigned* barrier;
+  int* child_first; int* child_cnt;   // [B][N+1], slot 0 = root
+  int* wk_list; int* sc_list;         // [2][B] requests that asked for a reduction / a range rescan, by step parity
+  int* ctr;                           // [0..1] reduction counts, [2..3] rescan counts (by parity), [4] unfinished requests
   int vt_TV, vt_n, max_steps;
 };
 
@@ -133,39 +136,33 @@ __device__ __forceinline__ double p_of(const VerifyArgs& a, int64_t row, int w) 
   return exp(((double)z_elem<TIn>(a, row, w) - (double)a.z_max[row]) / (double)a.T - (double)a.z_logs[row]);
 }
 
-// children of node v are contiguous in canonical order; returns the first and the count
-__device__ __forceinline__ void children_of(const VerifyArgs& a, int b, int n, int v, int& first, int& m) {
-  const size_t nb = (size_t)b * a.N;
-  first = -1; m = 0;
-  for (int i = v + 1; i < n; ++i) {
-    if (a.parent[nb + i] == v) { if (first < 0) first = i; ++m; }
-    else if (first >= 0) break;
-  }
-}
-
-// Scalar state machine of one request (lane 0 decides, the warp helps with range sums).
-// need: 0 walking, 1 reduction after a rejection, 4 reduction for the bonus draw, 2 range rescan, 3 finished
+// Scalar state machine of one request, run by one warp of the request's owner CTA.
+// need: 0 walking, 1 reduction after a rejection, 4 reduction for the bonus draw, 2 range rescan, 3 finished.
+// Lane 0 decides; at every visited node the lanes fetch the accept-test inputs of all its children at
+// once (one memory round trip per node), and the warp folds range sums together.
 template <typename TIn>
-__device__ void advance(const VerifyArgs& a, int b, int lane) {
-  VerifyState& st = a.state[b];
-  const int N = a.N, n = a.n_nodes[b];
+__device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
+  VerifyState* gst = a.state + b;
+  const int N = a.N;
   const size_t nb = (size_t)b * N;
   const int64_t row0 = a.z_row_off[b];
-  int need = st.need;
-  if (need == 3) return;
+  const int need_in = gst->need;
+  if (need_in == 3) return;
   // ---- fold in the reduction that just ran -------------------------------------------------
   double fsum = 0.0;
-  if (need == 1 || need == 4) {
-    for (int t = lane; t < a.vt_n; t += 32) fsum += (double)a.part[(size_t)b * a.vt_n + t];
+  if (need_in == 1 || need_in == 4) {
+    for (int t = lane; t < a.vt_n; t += 32) fsum += (double)__ldcg(a.part + (size_t)b * a.vt_n + t);
     for (int off = 16; off > 0; off >>= 1) fsum += __shfl_xor_sync(0xFFFFFFFFu, fsum, off);
   }
+  VerifyState st;   // working copy (written back once at the end)
+  if (lane == 0) st = *gst;
   int go_scan = 0;
   if (lane == 0) {
-    if (need == 1 || need == 4) {
+    if (need_in == 1 || need_in == 4) {
       double zn = fsum;  // the pass used passC for every token; tested siblings keep their own C_i
       for (int i = 0; i < st.nf; ++i)
         zn += fmax(st.fp[i] - st.fC[i] * st.fq[i], 0.0) - fmax(st.fp[i] - st.passC * st.fq[i], 0.0);
-      if (need == 1) {
+      if (need_in == 1) {
         if (zn <= 1e-30 * st.Zj) {  // residual lost its mass: keep the previous one
           a.flags[b] |= TS_FLAG_ZERO_MASS;
           st.fC[st.nf - 1] = st.C;
@@ -178,53 +175,76 @@ __device__ void advance(const VerifyArgs& a, int b, int lane) {
       a.bonus[b] = st.result;
       a.acc_len[b] = st.acc;
       st.need = 3;
-    }
-    while (st.need == 0) {
-      const int v = st.cur;
-      int first, m;
-      children_of(a, b, n, v, first, m);
-      const int64_t row = row0 + v + 1;
-      const uint64_t hv = a.node_hash[(size_t)b * (N + 1) + v + 1];
-      if (st.j < m && st.acc < a.D) {
-        const int child = first + st.j, x = a.tok[nb + child];
-        const double px = p_of<TIn>(a, row, x), qx = exp((double)a.logqT[nb + child]);
-        const double cj = st.Zj / (1.0 - st.Qused);
-        const double num = fmax(px / qx - st.C, 0.0);
-        const double rho = fmin(1.0, num / cj);
-        const double u = u01(stream_words(a.seed, b, hv, STREAM_ACCEPT, (uint32_t)st.j).x);
-        if (u < rho) {
-          a.acc_node[(size_t)b * a.D + st.acc] = child; a.acc_tok[(size_t)b * a.D + st.acc] = x;
-          st.acc++; st.cur = child; st.j = 0; st.C = 0.0; st.Zj = 1.0; st.Qused = 0.0; st.nf = 0; st.partsC = -1.0;
-        } else {
-          st.fx[st.nf] = x; st.fp[st.nf] = px; st.fq[st.nf] = qx; st.fC[st.nf] = st.C + cj; st.nf++;
-          st.Qused += qx; st.j++;
-          st.passC = st.C + cj; st.row_node = v; st.need = 1;
-        }
-      } else {
-        if (st.partsC != st.C) { st.passC = st.C; st.row_node = v; st.need = 4; }
-        else go_scan = 1;
-        break;
-      }
+      atomicSub(a.ctr + 4, 1);
     }
   }
+  int walking = __shfl_sync(0xFFFFFFFFu, lane == 0 ? (st.need == 0) : 0, 0);
+  while (walking) {
+    // inputs of every child's accept test at the current node, one child per lane
+    const int v = __shfl_sync(0xFFFFFFFFu, st.cur, 0);
+    const int first = a.child_first[(size_t)b * (N + 1) + v + 1], m = a.child_cnt[(size_t)b * (N + 1) + v + 1];
+    const int64_t row = row0 + v + 1;
+    double px = 0.0, qx = 1.0; int x = -1;
+    if (lane < m) {
+      x = a.tok[nb + first + lane];
+      px = exp(((double)z_elem<TIn>(a, row, x) - (double)a.z_max[row]) / (double)a.T - (double)a.z_logs[row]);
+      qx = exp((double)a.logqT[nb + first + lane]);
+    }
+    const uint64_t hv = a.node_hash[(size_t)b * (N + 1) + v + 1];
+    // lane 0 runs the sibling chain at this node until it accepts, needs a reduction, or runs out
+    int again = 0;
+    for (int j = 0; j < 32; ++j) {   // m <= K <= 16
+      const double pxj = __shfl_sync(0xFFFFFFFFu, px, j), qxj = __shfl_sync(0xFFFFFFFFu, qx, j);
+      const int xj = __shfl_sync(0xFFFFFFFFu, x, j);
+      int stop = 0;
+      if (lane == 0) {
+        if (st.j != j) { }   // siblings before st.j were tested in an earlier step
+        else if (st.j < m && st.acc < a.D) {
+          const double cj = st.Zj / (1.0 - st.Qused);
+          const double num = fmax(pxj / qxj - st.C, 0.0);
+          const double rho = fmin(1.0, num / cj);
+          const double u = u01(stream_words(a.seed, b, hv, STREAM_ACCEPT, (uint32_t)st.j).x);
+          if (u < rho) {
+            a.acc_node[(size_t)b * a.D + st.acc] = first + j; a.acc_tok[(size_t)b * a.D + st.acc] = xj;
+            st.acc++; st.cur = first + j; st.j = 0; st.C = 0.0; st.Zj = 1.0; st.Qused = 0.0; st.nf = 0; st.partsC = -1.0;
+            stop = 1; again = 1;          // descend: next node
+          } else {
+            st.fx[st.nf] = xj; st.fp[st.nf] = pxj; st.fq[st.nf] = qxj; st.fC[st.nf] = st.C + cj; st.nf++;
+            st.Qused += qxj; st.j++;
+            st.passC = st.C + cj; st.row_node = v; st.need = 1;
+            stop = 1;                      // wait for the reduction
+          }
+        } else {
+          if (st.partsC != st.C) { st.passC = st.C; st.row_node = v; st.need = 4; }
+          else go_scan = 1;
+          stop = 1;
+        }
+      }
+      stop = __shfl_sync(0xFFFFFFFFu, stop, 0);
+      if (stop) break;
+    }
+    walking = __shfl_sync(0xFFFFFFFFu, again, 0);
+  }
   go_scan = __shfl_sync(0xFFFFFFFFu, go_scan, 0);
-  __syncwarp();
   if (go_scan) {
     // locate the vocabulary range holding the bonus token: cumulative corrected range sums
-    const uint64_t hv = a.node_hash[(size_t)b * (N + 1) + st.cur + 1];
+    const int cur = __shfl_sync(0xFFFFFFFFu, st.cur, 0), nf = __shfl_sync(0xFFFFFFFFu, st.nf, 0);
+    const double C = __shfl_sync(0xFFFFFFFFu, st.C, 0), Zj = __shfl_sync(0xFFFFFFFFu, st.Zj, 0);
+    const uint64_t hv = a.node_hash[(size_t)b * (N + 1) + cur + 1];
     const double u = u01(stream_words(a.seed, b, hv, STREAM_BONUS, 0u).x);
-    const double target = u * st.Zj;
+    const double target = u * Zj;
     double carry = 0.0; int found = -1; double before = 0.0; int last_pos = -1;
     for (int t0 = 0; t0 < a.vt_n && found < 0; t0 += 32) {
       const int t = t0 + lane;
       double pt = 0.0;
-      if (t < a.vt_n) {
-        pt = (double)a.part[(size_t)b * a.vt_n + t];
-        for (int i = 0; i < st.nf; ++i)
-          if (st.fx[i] / a.vt_TV == t)
-            pt += fmax(st.fp[i] - st.fC[i] * st.fq[i], 0.0) - fmax(st.fp[i] - st.C * st.fq[i], 0.0);
-        if (pt < 0.0) pt = 0.0;
+      if (t < a.vt_n) pt = (double)__ldcg(a.part + (size_t)b * a.vt_n + t);
+      for (int i = 0; i < nf; ++i) {   // tested siblings keep the residual they had when tested
+        const int fxi = __shfl_sync(0xFFFFFFFFu, st.fx[i], 0);
+        const double fpi = __shfl_sync(0xFFFFFFFFu, st.fp[i], 0), fqi = __shfl_sync(0xFFFFFFFFu, st.fq[i], 0);
+        const double fCi = __shfl_sync(0xFFFFFFFFu, st.fC[i], 0);
+        if (t < a.vt_n && fxi / a.vt_TV == t) pt += fmax(fpi - fCi * fqi, 0.0) - fmax(fpi - C * fqi, 0.0);
       }
+      if (pt < 0.0) pt = 0.0;
       double inc = pt;
       for (int off = 1; off < 32; off <<= 1) { const double o = __shfl_up_sync(0xFFFFFFFFu, inc, off); if (lane >= off) inc += o; }
       const bool cross = (t < a.vt_n) && (carry + inc > target);
@@ -242,6 +262,12 @@ __device__ void advance(const VerifyArgs& a, int b, int lane) {
       if (found < 0) { found = last_pos >= 0 ? last_pos : 0; before = -1.0; }  // rounding: take the last range with mass
       st.scan_tile = found; st.target = target; st.before = before; st.need = 2;
     }
+  }
+  if (lane == 0) {
+    *gst = st;
+    __threadfence();
+    if (st.need == 1 || st.need == 4) a.wk_list[parity * a.B + atomicAdd(a.ctr + parity, 1)] = b;
+    else if (st.need == 2) a.sc_list[parity * a.B + atomicAdd(a.ctr + 2 + parity, 1)] = b;
   }
   __syncwarp();
 }
@@ -294,7 +320,6 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
   __shared__ float s_red[VG][VT / 32];
   __shared__ double s_scan[VT];
   __shared__ int s_found;
-  __shared__ int s_any;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned nblocks = gridDim.x;
   unsigned gen = 0;
@@ -304,133 +329,139 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
   const int v_lo = blockIdx.x * a.vt_TV, v_hi = min(a.V, v_lo + a.vt_TV);
   const TIn* Zg = reinterpret_cast<const TIn*>(a.Z);
   const TIn* Ag = reinterpret_cast<const TIn*>(a.A);
+  const int N = a.N;
 
-  // per-edge statistics and state initialisation
+  // ---- per-edge statistics, child ranges and state initialisation (owner CTA of each request) ------
+  if (blockIdx.x == 0 && tid < 5) a.ctr[tid] = tid == 4 ? a.B : 0;
   for (int b = blockIdx.x; b < a.B; b += nblocks) {
     const int n = a.n_nodes[b];
-    const size_t nb = (size_t)b * a.N;
+    const bool okn = n >= 0 && n <= N;
+    const size_t nb = (size_t)b * N, cbase = (size_t)b * (N + 1);
     const int64_t row0 = a.z_row_off[b];
-    if (a.edge_stat)
+    for (int i = tid; i <= N; i += VT) { a.child_first[cbase + i] = -1; a.child_cnt[cbase + i] = 0; }
+    __syncthreads();
+    if (okn)
       for (int i = tid; i < n; i += VT) {
-        const int64_t row = row0 + a.parent[nb + i] + 1;
-        const double lr = ((double)z_elem<TIn>(a, row, a.tok[nb + i]) - (double)a.z_max[row]) / (double)a.T -
-                          (double)a.z_logs[row] - (double)a.logqT[nb + i];
-        a.edge_stat[nb + i] = (float)exp(fmin(lr, 0.0));
+        const int par = a.parent[nb + i];
+        if (i == 0 || a.parent[nb + i - 1] != par) a.child_first[cbase + par + 1] = i;   // siblings are contiguous
+        atomicAdd(&a.child_cnt[cbase + par + 1], 1);
+        if (a.edge_stat) {
+          const int64_t row = row0 + par + 1;
+          const double lr = ((double)z_elem<TIn>(a, row, a.tok[nb + i]) - (double)a.z_max[row]) / (double)a.T -
+                            (double)a.z_logs[row] - (double)a.logqT[nb + i];
+          a.edge_stat[nb + i] = (float)exp(fmin(lr, 0.0));
+        }
       }
     if (tid == 0) {
       VerifyState& st = a.state[b];
       st.cur = -1; st.j = 0; st.acc = 0; st.need = 0; st.nf = 0; st.scan_tile = -1; st.row_node = -1; st.result = -1;
       st.C = 0.0; st.Zj = 1.0; st.Qused = 0.0; st.target = 0.0; st.before = 0.0; st.passC = 0.0; st.partsC = -1.0;
       a.flags[b] = 0u;
-      a.status[b] = (n >= 0 && n <= a.N) ? TS_OK : TS_ERR_INVALID;
-      if (!(n >= 0 && n <= a.N)) { st.need = 3; a.acc_len[b] = 0; a.bonus[b] = -1; }
+      a.status[b] = okn ? TS_OK : TS_ERR_INVALID;
+      if (!okn) { st.need = 3; a.acc_len[b] = 0; a.bonus[b] = -1; }
       for (int i = 0; i < a.D; ++i) { a.acc_node[(size_t)b * a.D + i] = -1; a.acc_tok[(size_t)b * a.D + i] = -1; }
     }
+    __syncthreads();
   }
-  __syncthreads();
+  __threadfence();
+  if (!grid_barrier(a.barrier, nblocks, gen)) return;
+  // requests rejected at set-up leave the count of unfinished ones
+  for (int b = blockIdx.x; b < a.B; b += nblocks)
+    if (tid == 0 && a.state[b].need == 3) atomicSub(a.ctr + 4, 1);
 
   for (int step = 0; step < a.max_steps; ++step) {
-    // ---- phase A: scalar walks ---------------------------------------------------------------
-    if (warp == 0)
-      for (int b = blockIdx.x; b < a.B; b += nblocks) advance<TIn>(a, b, lane);
+    const int par = step & 1;
+    // ---- phase A: scalar walks of the requests this CTA owns, one warp each ----------------------
+    for (int b = blockIdx.x + warp * (int)nblocks; b < a.B; b += (VT / 32) * (int)nblocks) advance<TIn>(a, b, lane, par);
     if (!grid_barrier(a.barrier, nblocks, gen)) return;
-    // ---- phase B: vocabulary work requested by the walks ----------------------------------------
-    if (tid == 0) s_any = 0;
-    __syncthreads();
-    for (int b0 = 0; b0 < a.B; b0 += VG) {
-      // gather up to VG requests that asked for a reduction
-      if (tid == 0) {
-        int ng = 0;
-        for (int b = b0; b < min(a.B, b0 + VG); ++b) {
-          const VerifyState& st = a.state[b];
-          if (st.need != 3) s_any = 1;
-          if (st.need == 1 || st.need == 4) {
-            const int v = st.row_node;
-            const int64_t row = a.z_row_off[b] + v + 1;
-            s_req[ng] = b; s_node[ng] = v; s_dep[ng] = v < 0 ? 0 : a.depth[(size_t)b * a.N + v];
-            s_C[ng] = (float)st.passC; s_zmax[ng] = a.z_max[row]; s_zlogs[ng] = a.z_logs[row];
-            s_lseT[ng] = a.node_lseT[(size_t)b * (a.N + 1) + v + 1];
-            ++ng;
-          }
-        }
-        s_found = ng;
+    // ---- phase B: vocabulary work requested by the walks -----------------------------------------
+    const int nwk = __ldcg(a.ctr + par), nsc = __ldcg(a.ctr + 2 + par), left = __ldcg(a.ctr + 4);
+    if (blockIdx.x == 0 && tid < 2) a.ctr[2 * tid + (par ^ 1)] = 0;   // next step's counters
+    for (int w0 = 0; w0 < nwk; w0 += VG) {
+      const int ng = min(VG, nwk - w0);
+      if (tid < ng) {
+        const int b = __ldcg(a.wk_list + par * a.B + w0 + tid);
+        const VerifyState* st = a.state + b;
+        const int v = st->row_node;
+        const int64_t row = a.z_row_off[b] + v + 1;
+        s_req[tid] = b; s_node[tid] = v; s_dep[tid] = v < 0 ? 0 : a.depth[(size_t)b * N + v];
+        s_C[tid] = (float)st->passC; s_zmax[tid] = a.z_max[row]; s_zlogs[tid] = a.z_logs[row];
+        s_lseT[tid] = a.node_lseT[(size_t)b * (N + 1) + v + 1];
       }
       __syncthreads();
-      const int ng = s_found;
-      if (ng > 0) {
-        for (int i = tid; i < ng * a.r; i += VT) {
-          const int g = i / a.r, k = i % a.r;
-          const int v = s_node[g];
-          const int ptok = v < 0 ? a.anchor[s_req[g]] : a.tok[(size_t)s_req[g] * a.N + v];
-          s_a[g * 128 + k] = Elem<TIn>::to_f(Ag[(size_t)ptok * a.r + k]);
-        }
-        __syncthreads();
-        float sum[VG];
+      for (int i = tid; i < ng * a.r; i += VT) {
+        const int g = i / a.r, k = i % a.r;
+        const int v = s_node[g];
+        const int ptok = v < 0 ? a.anchor[s_req[g]] : a.tok[(size_t)s_req[g] * N + v];
+        s_a[g * 128 + k] = Elem<TIn>::to_f(Ag[(size_t)ptok * a.r + k]);
+      }
+      __syncthreads();
+      float sum[VG];
 #pragma unroll
-        for (int g = 0; g < VG; ++g) sum[g] = 0.f;
-        bool need_q = false;
-        for (int g = 0; g < ng; ++g) need_q |= (s_C[g] != 0.f);
-        if (vec_ok) {
-          for (int v = v_lo + tid * VEC; v < v_hi; v += VT * VEC) {
-            float acc[VG][8];
-            if (need_q) logits_group<TIn, VG>(a, s_a, ng, s_req, s_dep, v, acc);
+      for (int g = 0; g < VG; ++g) sum[g] = 0.f;
+      bool need_q = false;
+      for (int g = 0; g < ng; ++g) need_q |= (s_C[g] != 0.f);
+      if (vec_ok) {
+        for (int v = v_lo + tid * VEC; v < v_hi; v += VT * VEC) {
+          float acc[VG][8];
+          if (need_q) logits_group<TIn, VG>(a, s_a, ng, s_req, s_dep, v, acc);
 #pragma unroll
-            for (int g = 0; g < VG; ++g) {
-              if (g < ng) {
-                const int64_t row = a.z_row_off[s_req[g]] + s_node[g] + 1;
-                float z[8];
-                if (sizeof(TIn) == 2) { const uint4 x = __ldg(reinterpret_cast<const uint4*>(Zg + row * a.V + v)); unpack_bf16x8(x, z); }
-                else { const float4 x = __ldg(reinterpret_cast<const float4*>(Zg + row * a.V + v)); z[0] = x.x; z[1] = x.y; z[2] = x.z; z[3] = x.w; }
+          for (int g = 0; g < VG; ++g) {
+            if (g < ng) {
+              const int64_t row = a.z_row_off[s_req[g]] + s_node[g] + 1;
+              float z[8];
+              if (sizeof(TIn) == 2) { const uint4 x = __ldg(reinterpret_cast<const uint4*>(Zg + row * a.V + v)); unpack_bf16x8(x, z); }
+              else { const float4 x = __ldg(reinterpret_cast<const float4*>(Zg + row * a.V + v)); z[0] = x.x; z[1] = x.y; z[2] = x.z; z[3] = x.w; }
 #pragma unroll
-                for (int i = 0; i < VEC; ++i) {
-                  const float p = __expf((z[i] - s_zmax[g]) * invT - s_zlogs[g]);
-                  const float q = s_C[g] != 0.f ? __expf(acc[g][i] * invT - s_lseT[g]) : 0.f;
-                  sum[g] += fmaxf(p - s_C[g] * q, 0.f);
-                }
+              for (int i = 0; i < VEC; ++i) {
+                const float p = __expf((z[i] - s_zmax[g]) * invT - s_zlogs[g]);
+                const float q = s_C[g] != 0.f ? __expf(acc[g][i] * invT - s_lseT[g]) : 0.f;
+                sum[g] += fmaxf(p - s_C[g] * q, 0.f);
               }
             }
           }
-        } else {
-          for (int v = v_lo + tid; v < v_hi; v += VT) {
-            for (int g = 0; g < ng; ++g) {
-              const int b = s_req[g];
-              const int64_t row = a.z_row_off[b] + s_node[g] + 1;
-              const float p = __expf((z_elem<TIn>(a, row, v) - s_zmax[g]) * invT - s_zlogs[g]);
-              float q = 0.f;
-              if (s_C[g] != 0.f) {
-                const int ptok = s_node[g] < 0 ? a.anchor[b] : a.tok[(size_t)b * a.N + s_node[g]];
-                q = __expf(logit_scalar<TIn>(a, b, s_dep[g], ptok, v) * invT - s_lseT[g]);
-              }
-              sum[g] += fmaxf(p - s_C[g] * q, 0.f);
+        }
+      } else {
+        for (int v = v_lo + tid; v < v_hi; v += VT) {
+          for (int g = 0; g < ng; ++g) {
+            const int b = s_req[g];
+            const int64_t row = a.z_row_off[b] + s_node[g] + 1;
+            const float p = __expf((z_elem<TIn>(a, row, v) - s_zmax[g]) * invT - s_zlogs[g]);
+            float q = 0.f;
+            if (s_C[g] != 0.f) {
+              const int ptok = s_node[g] < 0 ? a.anchor[b] : a.tok[(size_t)b * N + s_node[g]];
+              q = __expf(logit_scalar<TIn>(a, b, s_dep[g], ptok, v) * invT - s_lseT[g]);
             }
+            sum[g] += fmaxf(p - s_C[g] * q, 0.f);
           }
         }
+      }
 #pragma unroll
-        for (int g = 0; g < VG; ++g) {
-          float s = sum[g];
-          for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
-          if (lane == 0) s_red[g][warp] = s;
-        }
-        __syncthreads();
-        if (tid < ng) {
-          float t = 0.f;
-          for (int w = 0; w < VT / 32; ++w) t += s_red[tid][w];
-          a.part[(size_t)s_req[tid] * a.vt_n + blockIdx.x] = t;
-        }
+      for (int g = 0; g < VG; ++g) {
+        float sg = sum[g];
+        for (int off = 16; off > 0; off >>= 1) sg += __shfl_xor_sync(0xFFFFFFFFu, sg, off);
+        if (lane == 0) s_red[g][warp] = sg;
+      }
+      __syncthreads();
+      if (tid < ng) {
+        float t = 0.f;
+        for (int w = 0; w < VT / 32; ++w) t += s_red[tid][w];
+        a.part[(size_t)s_req[tid] * a.vt_n + blockIdx.x] = t;
       }
       __syncthreads();
     }
     // range rescans for bonus tokens that fall into this CTA's range
-    for (int b = 0; b < a.B; ++b) {
+    for (int si = 0; si < nsc; ++si) {
+      const int b = __ldcg(a.sc_list + par * a.B + si);
       const VerifyState& st = a.state[b];
-      if (st.need != 2 || st.scan_tile != (int)blockIdx.x) continue;
+      if (st.scan_tile != (int)blockIdx.x) continue;
       const int v = st.cur;
       const int64_t row = a.z_row_off[b] + v + 1;
-      const int dep = v < 0 ? 0 : a.depth[(size_t)b * a.N + v];
-      const int ptok = v < 0 ? a.anchor[b] : a.tok[(size_t)b * a.N + v];
+      const int dep = v < 0 ? 0 : a.depth[(size_t)b * N + v];
+      const int ptok = v < 0 ? a.anchor[b] : a.tok[(size_t)b * N + v];
       const double C = st.C;
       const double zmax = a.z_max[row], zlogs = a.z_logs[row];
-      const double lseT = C != 0.0 ? (double)a.node_lseT[(size_t)b * (a.N + 1) + v + 1] : 0.0;
+      const double lseT = C != 0.0 ? (double)a.node_lseT[(size_t)b * (N + 1) + v + 1] : 0.0;
       const int len = v_hi - v_lo;
       const int per = (len + VT - 1) / VT;
       const int w0 = v_lo + tid * per, w1 = min(v_hi, w0 + per);
@@ -462,6 +493,7 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
       }
       __syncthreads();
       if (s_found == 0x7FFFFFFF) {  // rounding pushed the crossing past this range: last token with mass
+        __syncthreads();
         if (tid == 0) s_found = -1;
         __syncthreads();
         if (lastpos >= 0) atomicMax(&s_found, lastpos);
@@ -472,9 +504,9 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
       if (tid == 0) a.state[b].result = s_found;
       __syncthreads();
     }
-    const int any = s_any;
+    __threadfence();
     if (!grid_barrier(a.barrier, nblocks, gen)) return;
-    if (!any) return;
+    if (left == 0 && nwk == 0 && nsc == 0) return;
   }
   // steps ran out
   for (int b = blockIdx.x; b < a.B; b += nblocks)
@@ -529,6 +561,8 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
   a.acc_len = acc_len; a.acc_node = acc_node; a.acc_tok = acc_tok; a.bonus = bonus_tok; a.edge_stat = edge_stat;
   a.flags = flags; a.status = status;
   a.state = (VerifyState*)(ws + L.vf_state); a.part = (float*)(ws + L.vf_part); a.barrier = (unsigned*)(ws + L.vf_barrier);
+  a.child_first = (int*)(ws + L.vf_child); a.child_cnt = a.child_first + (size_t)B * (c.Nmax + 1);
+  a.wk_list = (int*)(ws + L.vf_lists); a.sc_list = a.wk_list + 2 * (size_t)B; a.ctr = a.sc_list + 2 * (size_t)B;
   a.vt_TV = ctx->vt_TV; a.vt_n = ctx->vt_n; a.max_steps = 2 * (c.Nmax + c.D) + 8;
 
   const int max_rows = B * (c.Nmax + 1);
