@@ -94,46 +94,55 @@ __global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d) 
     if (tid == 0) a.req_npar[b] = 0;
     return;
   }
-  // ---- phase 1: slots of every scored parent -------------------------------------------------
-  for (int i = tid; i < npar; i += blockDim.x) {
+  // ---- phase 1: slots of every scored parent, one thread per (parent, sibling rank) -------------
+  for (int t = tid; t < npar * K; t += blockDim.x) {
+    const int i = t / K, j = t % K;
     const int li = base + i;
     const int slot = a.lst_slot[cur][li];
     const double logS_v = slot < 0 ? 0.0 : a.pl_logS[pb + slot];
     const double lse0 = a.res_lse0[li], lseT = a.res_lseT[li];
-    if (slot < 0) a.root_lseT[b] = (float)lseT; else a.pl_lseT[pb + slot] = (float)lseT;
-    if (!(lse0 == lse0) || isinf(lse0)) a.status[b] = TS_ERR_NUMERIC;
+    if (j == 0) {
+      if (slot < 0) a.root_lseT[b] = (float)lseT; else a.pl_lseT[pb + slot] = (float)lseT;
+      if (!(lse0 == lse0) || isinf(lse0)) a.status[b] = TS_ERR_NUMERIC;
+    }
     const int* top_tok = a.res_top_tok + (size_t)li * K; const float* top_logit = a.res_top_logit + (size_t)li * K;
     const int* draw_tok = a.res_draw_tok + (size_t)li * K; const float* draw_logit = a.res_draw_logit + (size_t)li * K;
+    const size_t ci = cb + (size_t)i * K + j;
+    int valid = 0;
+    if (j < K_eff) {
+      int bi = j;
+      if (a.T > 0.f) {  // best token of q0 not among the first j draws: the pre-draw bound
+        bi = -1;
+        for (int tt = 0; tt < K_eff && bi < 0; ++tt) {
+          bool used = false;
+          for (int u = 0; u < j; ++u) used |= (draw_tok[u] == top_tok[tt]);
+          if (!used) bi = tt;
+        }
+      }
+      const int x = draw_tok[j];
+      if (bi >= 0 && top_tok[bi] >= 0 && x >= 0) {
+        const double key = logS_v + log_phat(a.calib, d, (double)top_logit[bi], lse0);
+        if (!(key < log_theta)) {
+          const double lx = draw_logit[j];
+          valid = 1;
+          a.cd_parent[ci] = slot; a.cd_sib[ci] = j; a.cd_tok[ci] = x;
+          a.cd_logkey[ci] = key;
+          a.cd_logS[ci] = logS_v + log_phat(a.calib, d, lx, lse0);
+          a.cd_q0[ci] = (float)exp(lx - lse0);
+          a.cd_logqT[ci] = a.T > 0.f ? (float)(lx / (double)a.T - lseT) : (float)(lx - lse0);
+        }
+      }
+    }
+    a.cd_valid[ci] = valid;
+  }
+  __syncthreads();
+  // a sibling slot exists only if the one before it was admitted (keys are non-increasing in j)
+  for (int i = tid; i < npar; i += blockDim.x) {
     bool open = true;
     for (int j = 0; j < K; ++j) {
       const size_t ci = cb + (size_t)i * K + j;
-      int valid = 0;
-      if (open && j < K_eff) {
-        int bi = j;
-        if (a.T > 0.f) {  // best token of q0 not among the first j draws: the pre-draw bound
-          bi = -1;
-          for (int t = 0; t < K_eff && bi < 0; ++t) {
-            bool used = false;
-            for (int u = 0; u < j; ++u) used |= (draw_tok[u] == top_tok[t]);
-            if (!used) bi = t;
-          }
-        }
-        const int x = draw_tok[j];
-        if (bi >= 0 && top_tok[bi] >= 0 && x >= 0) {
-          const double key = logS_v + log_phat(a.calib, d, (double)top_logit[bi], lse0);
-          if (!(key < log_theta)) {
-            const double lx = draw_logit[j];
-            valid = 1;
-            a.cd_parent[ci] = slot; a.cd_sib[ci] = j; a.cd_tok[ci] = x;
-            a.cd_logkey[ci] = key;
-            a.cd_logS[ci] = logS_v + log_phat(a.calib, d, lx, lse0);
-            a.cd_q0[ci] = (float)exp(lx - lse0);
-            a.cd_logqT[ci] = a.T > 0.f ? (float)(lx / (double)a.T - lseT) : (float)(lx - lse0);
-          }
-        }
-        if (!valid) open = false;  // keys are non-increasing in j: later slots cannot be admitted
-      }
-      a.cd_valid[ci] = valid;
+      if (!open) a.cd_valid[ci] = 0;
+      else if (!a.cd_valid[ci]) open = false;
     }
   }
   __syncthreads();

@@ -19,6 +19,15 @@
 
 namespace ts {
 
+#ifdef TS_DEBUG_TIMING
+__device__ unsigned long long g_dbgw[4 * 64 * 8];
+__device__ __forceinline__ unsigned long long gtimew() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define DBGW(step, slot) do { if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 70) && (step) < 64) g_dbgw[((blockIdx.x ? 1 : 0) * 64 + (step)) * 8 + (slot)] = gtimew(); } while (0)
+extern "C" int ts_debug_timing_walk(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_dbgw, sizeof(g_dbgw)); }
+#else
+#define DBGW(step, slot) do { } while (0)
+#endif
+
 constexpr int VT = 256;  // threads of the verification kernels
 
 // ------------------------------------------------------------------------------------------------
@@ -94,6 +103,7 @@ struct VerifyArgs {
   int* wk_list; int* sc_list;         // [2][B] requests that asked for a reduction / a range rescan, by step parity
   int* ctr;                           // [0..1] reduction counts, [2..3] rescan counts (by parity), [4] unfinished requests
   int vt_TV, vt_n, max_steps;
+  int w_smem;   // 1: the kernel keeps its range of W in dynamic shared memory
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -275,9 +285,9 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
 // logits of up to G parents for the VEC tokens at v (global W, coalesced 16-byte loads)
 template <typename TIn, int G>
 __device__ __forceinline__ void logits_group(const VerifyArgs& a, const float* as, int ng, const int* rq_req,
-                                             const int* rq_dep, int v, float (*acc)[8]) {
+                                             const int* rq_dep, int v, float (*acc)[8], const TIn* Wsrc, size_t wstride,
+                                             int woff) {
   constexpr int VEC = Elem<TIn>::VEC;
-  const TIn* Wg = reinterpret_cast<const TIn*>(a.W);
   const TIn* Ug = reinterpret_cast<const TIn*>(a.U);
   for (int g = 0; g < G; ++g) {
     if (g < ng) {
@@ -288,8 +298,9 @@ __device__ __forceinline__ void logits_group(const VerifyArgs& a, const float* a
   }
   for (int k = 0; k < a.r; ++k) {
     float w[8];
-    if (sizeof(TIn) == 2) { const uint4 x = __ldg(reinterpret_cast<const uint4*>(Wg + (size_t)k * a.V + v)); unpack_bf16x8(x, w); }
-    else { const float4 x = __ldg(reinterpret_cast<const float4*>(Wg + (size_t)k * a.V + v)); w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w; }
+    // W comes from the CTA's shared-memory copy of its vocabulary range when that fits, else from global
+    if (sizeof(TIn) == 2) { const uint4 x = *reinterpret_cast<const uint4*>(Wsrc + (size_t)k * wstride + woff); unpack_bf16x8(x, w); }
+    else { const float4 x = *reinterpret_cast<const float4*>(Wsrc + (size_t)k * wstride + woff); w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w; }
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       const float ak = as[g * 128 + k];
@@ -312,6 +323,71 @@ __device__ __forceinline__ float logit_scalar(const VerifyArgs& a, int req, int 
 
 constexpr int VG = 4;  // requests sharing one sweep over the W columns
 
+// One work item of a reduction step: NG requests of one group over tokens [c_lo, c_hi) of the CTA's range.
+template <typename TIn>
+struct SweepCtx {
+  const TIn *Z, *U, *Wsrc; size_t wstride; int wshift; int V, D, r; float invT;
+  const float* a; const int *req, *dep; const long long* row; const float *C, *zmax, *zlogs, *lseT;
+};
+
+template <typename TIn, int NG>
+__device__ __forceinline__ void sweep_item(const SweepCtx<TIn>& c, int g0, int c_lo, int c_hi, int lane, float* out) {
+  constexpr int VEC = Elem<TIn>::VEC;
+  float sum[NG];
+  bool need_q = false;
+#pragma unroll
+  for (int g = 0; g < NG; ++g) { sum[g] = 0.f; need_q |= (c.C[g0 + g] != 0.f); }
+  for (int v = c_lo + lane * VEC; v < c_hi; v += 32 * VEC) {
+    float z[NG][8], acc[NG][8];
+#pragma unroll
+    for (int g = 0; g < NG; ++g) {   // every load of the step first: target rows, base rows
+      const TIn* zp = c.Z + c.row[g0 + g] * c.V + v;
+      const TIn* up = c.U + ((size_t)c.req[g0 + g] * c.D + c.dep[g0 + g]) * c.V + v;
+      if (sizeof(TIn) == 2) {
+        unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(zp)), z[g]);
+        if (need_q) unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(up)), acc[g]);
+      } else {
+        const float4 x = __ldg(reinterpret_cast<const float4*>(zp)); z[g][0] = x.x; z[g][1] = x.y; z[g][2] = x.z; z[g][3] = x.w;
+        if (need_q) { const float4 y = __ldg(reinterpret_cast<const float4*>(up)); acc[g][0] = y.x; acc[g][1] = y.y; acc[g][2] = y.z; acc[g][3] = y.w; }
+      }
+    }
+    if (need_q) {
+      const TIn* wp = c.Wsrc + (v + c.wshift);
+#pragma unroll 4
+      for (int k = 0; k < c.r; ++k) {
+        float w[8];
+        if (sizeof(TIn) == 2) unpack_bf16x8(*reinterpret_cast<const uint4*>(wp + (size_t)k * c.wstride), w);
+        else { const float4 x = *reinterpret_cast<const float4*>(wp + (size_t)k * c.wstride); w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w; }
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+          const float ak = c.a[(g0 + g) * 128 + k];
+#pragma unroll
+          for (int i = 0; i < VEC; ++i) acc[g][i] = fmaf(ak, w[i], acc[g][i]);
+        }
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < NG; ++g) {
+      const float Cg = c.C[g0 + g], zm = c.zmax[g0 + g], zl = c.zlogs[g0 + g], lt = c.lseT[g0 + g];
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) {
+        const float p = __expf((z[g][i] - zm) * c.invT - zl);
+        const float q = Cg != 0.f ? __expf(acc[g][i] * c.invT - lt) : 0.f;
+        sum[g] += fmaxf(p - Cg * q, 0.f);
+      }
+    }
+  }
+#pragma unroll
+  for (int g = 0; g < NG; ++g) {
+    float sg = sum[g];
+    for (int off = 16; off > 0; off >>= 1) sg += __shfl_xor_sync(0xFFFFFFFFu, sg, off);
+    if (lane == 0) out[(size_t)g * 16] = sg;
+  }
+}
+
+
+constexpr int SB = 32; // requests whose head rows are staged together
+
 template <typename TIn>
 __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
   __shared__ float s_a[VG * 128];
@@ -319,7 +395,11 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
   __shared__ float s_C[VG], s_zmax[VG], s_zlogs[VG], s_lseT[VG];
   __shared__ float s_red[VG][VT / 32];
   __shared__ double s_scan[VT];
-  __shared__ int s_found;
+  __shared__ int s_found, s_last;
+  __shared__ float sb_a[SB * 128];
+  __shared__ int sb_req[SB], sb_dep[SB], sb_tok[SB];
+  __shared__ long long sb_row[SB];
+  __shared__ float sb_C[SB], sb_zmax[SB], sb_zlogs[SB], sb_lseT[SB], sb_part[SB * 16];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned nblocks = gridDim.x;
   unsigned gen = 0;
@@ -329,7 +409,20 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
   const int v_lo = blockIdx.x * a.vt_TV, v_hi = min(a.V, v_lo + a.vt_TV);
   const TIn* Zg = reinterpret_cast<const TIn*>(a.Z);
   const TIn* Ag = reinterpret_cast<const TIn*>(a.A);
+  const TIn* Wg = reinterpret_cast<const TIn*>(a.W);
   const int N = a.N;
+  extern __shared__ __align__(16) unsigned char w_raw[];
+  TIn* Ws = reinterpret_cast<TIn*>(w_raw);   // [r][vt_TV] when a.w_smem
+  if (a.w_smem && vec_ok) {
+    const int per_row = a.vt_TV / VEC;
+    for (int i = tid; i < a.r * per_row; i += VT) {
+      const int k = i / per_row, c = (i % per_row) * VEC;
+      uint4 x = make_uint4(0, 0, 0, 0);
+      if (v_lo + c < a.V) x = __ldg(reinterpret_cast<const uint4*>(Wg + (size_t)k * a.V + v_lo + c));
+      *reinterpret_cast<uint4*>(Ws + (size_t)k * a.vt_TV + c) = x;
+    }
+  }
+  const bool ws_ok = a.w_smem && vec_ok;
 
   // ---- per-edge statistics, child ranges and state initialisation (owner CTA of each request) ------
   if (blockIdx.x == 0 && tid < 5) a.ctr[tid] = tid == 4 ? a.B : 0;
@@ -371,12 +464,65 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
 
   for (int step = 0; step < a.max_steps; ++step) {
     const int par = step & 1;
+    DBGW(step, 0);
     // ---- phase A: scalar walks of the requests this CTA owns, one warp each ----------------------
     for (int b = blockIdx.x + warp * (int)nblocks; b < a.B; b += (VT / 32) * (int)nblocks) advance<TIn>(a, b, lane, par);
+    DBGW(step, 1);
     if (!grid_barrier(a.barrier, nblocks, gen)) return;
+    DBGW(step, 2);
     // ---- phase B: vocabulary work requested by the walks -----------------------------------------
     const int nwk = __ldcg(a.ctr + par), nsc = __ldcg(a.ctr + 2 + par), left = __ldcg(a.ctr + 4);
     if (blockIdx.x == 0 && tid < 2) a.ctr[2 * tid + (par ^ 1)] = 0;   // next step's counters
+    if (vec_ok) {
+      // Reductions sum_w max(p(w) - C q(w), 0) over this CTA's vocabulary range, for up to SB requests
+      // at a time.  Work item = (group of VG requests, chunk of the range); items are dealt to the warps,
+      // so a single request still uses several warps and many requests run side by side.  Partial sums
+      // are combined in a fixed order.
+      const int len = v_hi - v_lo;
+      const int chunk = max(256, ((len + 15) / 16 + 255) / 256 * 256);   // at most 16 chunks
+      const int nchunk = (len + chunk - 1) / chunk;
+      for (int sb0 = 0; sb0 < nwk; sb0 += SB) {
+        const int nreq = min(SB, nwk - sb0);
+        if (tid < nreq) {
+          const int b = __ldcg(a.wk_list + par * a.B + sb0 + tid);
+          const VerifyState* st = a.state + b;
+          const int v = st->row_node;
+          const int64_t row = a.z_row_off[b] + v + 1;
+          sb_req[tid] = b; sb_row[tid] = row; sb_dep[tid] = v < 0 ? 0 : a.depth[(size_t)b * N + v];
+          sb_tok[tid] = v < 0 ? a.anchor[b] : a.tok[(size_t)b * N + v];
+          sb_C[tid] = (float)st->passC; sb_zmax[tid] = a.z_max[row]; sb_zlogs[tid] = a.z_logs[row];
+          sb_lseT[tid] = a.node_lseT[(size_t)b * (N + 1) + v + 1];
+        }
+        __syncthreads();
+        for (int i = tid; i < nreq * a.r; i += VT) {
+          const int g = i / a.r, k = i % a.r;
+          sb_a[g * 128 + k] = Elem<TIn>::to_f(Ag[(size_t)sb_tok[g] * a.r + k]);
+        }
+        __syncthreads();
+        const int ngrp = (nreq + VG - 1) / VG;
+        for (int item = warp; item < ngrp * nchunk; item += VT / 32) {
+          const int grp = item / nchunk, ch = item % nchunk;
+          const int g0 = grp * VG, ng = min(VG, nreq - g0);
+          const int c_lo = v_lo + ch * chunk, c_hi = min(v_hi, c_lo + chunk);
+          const SweepCtx<TIn> sc{Zg, reinterpret_cast<const TIn*>(a.U), ws_ok ? Ws : Wg, ws_ok ? (size_t)a.vt_TV : (size_t)a.V,
+                                 ws_ok ? -v_lo : 0, a.V, a.D, a.r, invT, sb_a, sb_req, sb_dep, sb_row, sb_C, sb_zmax, sb_zlogs, sb_lseT};
+          float* out = sb_part + (size_t)g0 * 16 + ch;
+          switch (ng) {
+            case 1: sweep_item<TIn, 1>(sc, g0, c_lo, c_hi, lane, out); break;
+            case 2: sweep_item<TIn, 2>(sc, g0, c_lo, c_hi, lane, out); break;
+            case 3: sweep_item<TIn, 3>(sc, g0, c_lo, c_hi, lane, out); break;
+            default: sweep_item<TIn, 4>(sc, g0, c_lo, c_hi, lane, out); break;
+          }
+        }
+        __syncthreads();
+        if (tid < nreq) {
+          float t = 0.f;
+          for (int ch = 0; ch < nchunk; ++ch) t += sb_part[tid * 16 + ch];
+          a.part[(size_t)sb_req[tid] * a.vt_n + blockIdx.x] = t;
+        }
+        __syncthreads();
+      }
+    } else
     for (int w0 = 0; w0 < nwk; w0 += VG) {
       const int ng = min(VG, nwk - w0);
       if (tid < ng) {
@@ -404,7 +550,8 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
       if (vec_ok) {
         for (int v = v_lo + tid * VEC; v < v_hi; v += VT * VEC) {
           float acc[VG][8];
-          if (need_q) logits_group<TIn, VG>(a, s_a, ng, s_req, s_dep, v, acc);
+          if (need_q) logits_group<TIn, VG>(a, s_a, ng, s_req, s_dep, v, acc, ws_ok ? Ws : Wg,
+                                            ws_ok ? (size_t)a.vt_TV : (size_t)a.V, ws_ok ? v - v_lo : v);
 #pragma unroll
           for (int g = 0; g < VG; ++g) {
             if (g < ng) {
@@ -450,7 +597,10 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
       }
       __syncthreads();
     }
-    // range rescans for bonus tokens that fall into this CTA's range
+    DBGW(step, 3);
+    // range rescans for bonus tokens that fall into this CTA's range: the residual of every token of
+    // the range is evaluated once (tokens dealt round-robin to the threads: row i of the range holds
+    // tokens i*VT .. i*VT+VT-1), then prefix sums in token order locate the crossing
     for (int si = 0; si < nsc; ++si) {
       const int b = __ldcg(a.sc_list + par * a.B + si);
       const VerifyState& st = a.state[b];
@@ -462,50 +612,56 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
       const double C = st.C;
       const double zmax = a.z_max[row], zlogs = a.z_logs[row];
       const double lseT = C != 0.0 ? (double)a.node_lseT[(size_t)b * (N + 1) + v + 1] : 0.0;
-      const int len = v_hi - v_lo;
-      const int per = (len + VT - 1) / VT;
-      const int w0 = v_lo + tid * per, w1 = min(v_hi, w0 + per);
-      double loc = 0.0;
-      for (int w = w0; w < w1; ++w) {
-        double Cw = C;
-        for (int i = 0; i < st.nf; ++i) if (st.fx[i] == w) Cw = st.fC[i];
-        const double p = exp(((double)z_elem<TIn>(a, row, w) - zmax) / (double)a.T - zlogs);
-        const double q = Cw != 0.0 ? exp((double)logit_scalar<TIn>(a, b, dep, ptok, w) / (double)a.T - lseT) : 0.0;
-        loc += fmax(p - Cw * q, 0.0);
-      }
-      s_scan[tid] = loc;
-      if (tid == 0) s_found = 0x7FFFFFFF;
-      __syncthreads();
-      if (tid == 0) { double c = 0.0; for (int t = 0; t < VT; ++t) { const double x = s_scan[t]; s_scan[t] = c; c += x; } }
-      __syncthreads();
+      const int nf = st.nf;
       const double want = st.before >= 0.0 ? st.target - st.before : 1e300;
-      double cum = s_scan[tid];
-      int lastpos = -1;
-      for (int w = w0; w < w1; ++w) {
-        double Cw = C;
-        for (int i = 0; i < st.nf; ++i) if (st.fx[i] == w) Cw = st.fC[i];
-        const double p = exp(((double)z_elem<TIn>(a, row, w) - zmax) / (double)a.T - zlogs);
-        const double q = Cw != 0.0 ? exp((double)logit_scalar<TIn>(a, b, dep, ptok, w) / (double)a.T - lseT) : 0.0;
-        const double rw = fmax(p - Cw * q, 0.0);
-        cum += rw;
-        if (rw > 0.0) lastpos = w;
-        if (cum > want) { atomicMin(&s_found, w); break; }
-      }
+      for (int k = tid; k < a.r; k += VT) sb_a[k] = Elem<TIn>::to_f(Ag[(size_t)ptok * a.r + k]);
+      if (tid == 0) { s_found = 0x7FFFFFFF; s_last = -1; }
       __syncthreads();
-      if (s_found == 0x7FFFFFFF) {  // rounding pushed the crossing past this range: last token with mass
+      const int len = v_hi - v_lo;
+      const int nrow = (len + VT - 1) / VT;
+      double carry = 0.0;
+      for (int i = 0; i < nrow; ++i) {
+        const int o = i * VT + tid, w = v_lo + o;
+        double rw = 0.0;
+        if (o < len) {
+          double Cw = C;
+          for (int f = 0; f < nf; ++f) if (st.fx[f] == w) Cw = st.fC[f];
+          const double p = exp(((double)z_elem<TIn>(a, row, w) - zmax) / (double)a.T - zlogs);
+          double q = 0.0;
+          if (Cw != 0.0) {
+            float acc = Elem<TIn>::to_f(reinterpret_cast<const TIn*>(a.U)[((size_t)b * a.D + dep) * a.V + w]);
+            if (ws_ok) { for (int k = 0; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Ws[(size_t)k * a.vt_TV + o]), acc); }
+            else { for (int k = 0; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Wg[(size_t)k * a.V + w]), acc); }
+            q = exp((double)acc / (double)a.T - lseT);
+          }
+          rw = fmax(p - Cw * q, 0.0);
+        }
+        // inclusive prefix over the row in thread (= token) order
+        double inc = rw;
+        for (int off = 1; off < 32; off <<= 1) { const double t = __shfl_up_sync(0xFFFFFFFFu, inc, off); if (lane >= off) inc += t; }
+        if (lane == 31) s_scan[warp] = inc;
         __syncthreads();
-        if (tid == 0) s_found = -1;
+        double wbase = 0.0, rowsum = 0.0;
+        for (int w2 = 0; w2 < VT / 32; ++w2) { if (w2 < warp) wbase += s_scan[w2]; rowsum += s_scan[w2]; }
+        const double cum = carry + wbase + inc;
+        if (o < len && rw > 0.0) atomicMax(&s_last, o);
+        if (o < len && cum > want) atomicMin(&s_found, o);
+        carry += rowsum;
         __syncthreads();
-        if (lastpos >= 0) atomicMax(&s_found, lastpos);
-        __syncthreads();
-        if (tid == 0 && s_found < 0) s_found = v_hi - 1;
-        __syncthreads();
+        if (s_found != 0x7FFFFFFF) break;   // uniform: read after the barrier
       }
-      if (tid == 0) a.state[b].result = s_found;
+      if (tid == 0) {
+        int o = s_found;
+        if (o == 0x7FFFFFFF) o = s_last >= 0 ? s_last : len - 1;   // rounding pushed the crossing past the range
+        a.state[b].result = v_lo + o;
+      }
       __syncthreads();
     }
     __threadfence();
+    DBGW(step, 4);
     if (!grid_barrier(a.barrier, nblocks, gen)) return;
+    DBGW(step, 5);
+    if (threadIdx.x == 0 && blockIdx.x == 0 && step < 64) { DBGW(step, 6); }
     if (left == 0 && nwk == 0 && nsc == 0) return;
   }
   // steps ran out
@@ -521,8 +677,11 @@ __global__ void verify_check_kernel(VerifyArgs a) {
 }
 
 cudaError_t verify_setup(ts_ctx* ctx) {
-  (void)ctx;
-  return cudaSuccess;
+  // the walk kernel may keep its range of W in shared memory: allow the full opt-in size
+  cudaError_t e = cudaFuncSetAttribute(verify_walk_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       ctx->max_smem - 32 * 1024);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(verify_walk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem - 32 * 1024);
 }
 
 }  // namespace ts
@@ -584,9 +743,11 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
   }
   e = cudaMemsetAsync(a.barrier, 0, 64, st);
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(memset)", e);
+  const size_t w_bytes = (size_t)c.r * ctx->vt_TV * (c.dt_W == TS_DTYPE_BF16 ? 2 : 4);
+  a.w_smem = (w_bytes + 32 * 1024 <= (size_t)ctx->max_smem) ? 1 : 0;
   void* kargs[] = {(void*)&a};
   const void* fn = c.dt_Z == TS_DTYPE_BF16 ? (const void*)verify_walk_kernel<__nv_bfloat16> : (const void*)verify_walk_kernel<float>;
-  { ProfScope ps(ctx, K_WALK, st); e = cudaLaunchCooperativeKernel(fn, dim3(a.vt_n), dim3(VT), kargs, 0, st); }
+  { ProfScope ps(ctx, K_WALK, st); e = cudaLaunchCooperativeKernel(fn, dim3(a.vt_n), dim3(VT), kargs, a.w_smem ? w_bytes : 0, st); }
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(walk)", e);
   { ProfScope ps(ctx, K_CHECK, st); verify_check_kernel<<<(B + 127) / 128, 128, 0, st>>>(a); }
   e = cudaGetLastError();
