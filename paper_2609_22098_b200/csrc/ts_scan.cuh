@@ -7,7 +7,8 @@
 
 namespace ts {
 
-// Record layout in 32-bit words: [m, s0, sT, pad, topv[K], topi[K], keyv[K], keyi[K], keyl[K]]
+// Record layout in 32-bit words: [m, s0, sT, counts, topv[K], topi[K], keyv[K], keyi[K], keyl[K]]
+// counts = (#logit entries >= launch-wide bound at store time) | (#key entries >= bound) << 8
 __host__ __device__ __forceinline__ int rec_words(int K) { return (4 + 5 * K + 3) & ~3; }  // 16-byte multiple
 
 // Candidate lists of one (piece, parent): K best logits and K best sampling keys seen so far, both
@@ -50,10 +51,17 @@ struct RegLists {
     }
     return keyv[KR - 1];
   }
-  __device__ __forceinline__ void store(float* f, int* ii) const {
+  // writes the first K entries; returns how many logit / key entries can still matter given the
+  // launch-wide bounds (the lists are sorted, so those are prefixes)
+  __device__ __forceinline__ int store(float* f, int* ii, float gL, float gK) const {
+    int nt = 0, nk = 0;
 #pragma unroll
     for (int j = 0; j < KR; ++j)
-      if (j < K) { f[j] = topv[j]; ii[K + j] = topi[j]; f[2 * K + j] = keyv[j]; ii[3 * K + j] = keyi[j]; f[4 * K + j] = keyl[j]; }
+      if (j < K) {
+        f[j] = topv[j]; ii[K + j] = topi[j]; f[2 * K + j] = keyv[j]; ii[3 * K + j] = keyi[j]; f[4 * K + j] = keyl[j];
+        nt += (topi[j] >= 0 && topv[j] >= gL); nk += (keyi[j] >= 0 && keyv[j] >= gK);
+      }
+    return nt | (nk << 8);
   }
 };
 
@@ -86,9 +94,14 @@ struct MemLists {
   }
   __device__ __forceinline__ float insert_top(float v, int tok) { return mem_insert_top(&d, v, tok); }
   __device__ __forceinline__ float insert_key(float key, int tok, float logit) { return mem_insert_key(&d, key, tok, logit); }
-  __device__ __forceinline__ void store(float* f, int* ii) const {
+  __device__ __forceinline__ int store(float* f, int* ii, float gL, float gK) const {
     const int K = d.K;
-    for (int j = 0; j < K; ++j) { f[j] = d.topv[j]; ii[K + j] = d.topi[j]; f[2 * K + j] = d.keyv[j]; ii[3 * K + j] = d.keyi[j]; f[4 * K + j] = d.keyl[j]; }
+    int nt = 0, nk = 0;
+    for (int j = 0; j < K; ++j) {
+      f[j] = d.topv[j]; ii[K + j] = d.topi[j]; f[2 * K + j] = d.keyv[j]; ii[3 * K + j] = d.keyi[j]; f[4 * K + j] = d.keyl[j];
+      nt += (d.topi[j] >= 0 && d.topv[j] >= gL); nk += (d.keyi[j] >= 0 && d.keyv[j] >= gK);
+    }
+    return nt | (nk << 8);
   }
 };
 
@@ -105,10 +118,10 @@ struct RowScan {
     K = K_; L.init(K_); m = -INFINITY; s0 = 0.f; sT = 0.f; thrL = -INFINITY; thrK = -INFINITY;
     bestL = -INFINITY; bestK = -INFINITY;
   }
-  // one record, 16-byte aligned
-  __device__ __forceinline__ void store(float* rec) const {
-    *reinterpret_cast<float4*>(rec) = make_float4(m, s0, sT, 0.f);
-    L.store(rec + 4, reinterpret_cast<int*>(rec) + 4);
+  // one record, 16-byte aligned; the header's fourth word says how many list entries are worth reading
+  __device__ __forceinline__ void store(float* rec, float gL, float gK) const {
+    const int cnt = L.store(rec + 4, reinterpret_cast<int*>(rec) + 4, gL, gK);
+    *reinterpret_cast<float4*>(rec) = make_float4(m, s0, sT, __int_as_float(cnt));
   }
 };
 

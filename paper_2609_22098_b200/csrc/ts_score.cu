@@ -93,7 +93,9 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
       }
       scan_chunk(st, l, t0 + c0, valid, T, invT, a.seed, req, hash, ghi, gL, gK, gl, gk);
     }
-    st.store(a.rec + ((size_t)tile * a.cap + p) * rw);  // piece = (tile, 0), slot = p
+    gL = fmaxf(gL, dec_f(slots_min(gl, K)));
+    if (T > 0.f) gK = fmaxf(gK, dec_f(slots_min(gk, K)));
+    st.store(a.rec + ((size_t)tile * a.cap + p) * rw, gL, gK);  // piece = (tile, 0), slot = p
   }
 }
 
@@ -156,10 +158,35 @@ __device__ void block_select(MList<KR>& mine, int K, int* out_tok, float* out_va
   }
 }
 
+constexpr int MERGE_CAP = 768;   // candidates per list the fast path can hold
+
+// K rounds of warp-wide arg-max over a candidate array in shared memory (value desc, token asc)
+__device__ void warp_select(float* cv, int* ci, float* cl, int n, int K, int lane, int* out_tok, float* out_val) {
+  for (int j = 0; j < K; ++j) {
+    float bv = -INFINITY; int bi = 0x7FFFFFFF, bp = -1; float bl = 0.f;
+    for (int e = lane; e < n; e += 32) {
+      const int idx = ci[e];
+      if (idx != 0x7FFFFFFF && better(cv[e], idx, bv, bi)) { bv = cv[e]; bi = idx; bp = e; bl = cl[e]; }
+    }
+    float wv = bv; int wi = bi; float wl = bl;
+    for (int off = 16; off > 0; off >>= 1) {
+      const float ov = __shfl_xor_sync(0xFFFFFFFFu, wv, off);
+      const int oi = __shfl_xor_sync(0xFFFFFFFFu, wi, off);
+      const float ol = __shfl_xor_sync(0xFFFFFFFFu, wl, off);
+      if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; wl = ol; }
+    }
+    if (bp >= 0 && bi == wi) ci[bp] = 0x7FFFFFFF;   // taken (tokens are unique per list)
+    __syncwarp();
+    if (lane == 0) { out_tok[j] = wi == 0x7FFFFFFF ? -1 : wi; out_val[j] = wi == 0x7FFFFFFF ? 0.f : wl; }
+  }
+}
+
 template <int KR>
 __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
   __shared__ float s_v[MERGE_WARPS]; __shared__ int s_i[MERGE_WARPS]; __shared__ float s_l[MERGE_WARPS];
   __shared__ float s_m[MERGE_WARPS], s_s0[MERGE_WARPS], s_sT[MERGE_WARPS];
+  __shared__ float c_v[2][MERGE_CAP]; __shared__ int c_i[2][MERGE_CAP]; __shared__ float c_l[2][MERGE_CAP];
+  __shared__ int c_n[2];
   const int P = a.P_dev ? *a.P_dev : a.P;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float invT = a.T > 0.f ? 1.f / a.T : 1.f;
@@ -170,9 +197,9 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
     // final launch-wide lower bounds of this parent's K-th best logit / key: entries below cannot win
     const SharedThr gl{a.slots + (size_t)p * K, 0}, gk{a.slots + ((size_t)a.cap + p) * K, 0};
     const float bL = dec_f(slots_min(gl, K)), bK = a.T > 0.f ? dec_f(slots_min(gk, K)) : -INFINITY;
+    if (tid < 2) c_n[tid] = 0;
+    __syncthreads();
     float m = -INFINITY, s0 = 0.f, sT = 0.f;
-    MList<KR> top, key;
-    top.init(); key.init();
     for (int q = tid; q < npieces; q += MERGE_THREADS) {
       const int ts_ = q / R, rho = q % R;
       const int slot = R > 1 ? rho * (128 / R) + p : p;
@@ -181,14 +208,14 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
       const float* f = rec + 4; const int* ii = reinterpret_cast<const int*>(rec) + 4;
       // all entries of the record are requested at once (independent loads), then filtered
       float tv[KR], kv[KR], kl[KR]; int ti[KR], ki[KR];
+      const int cnt = __float_as_int(h.w), nt = cnt & 255, nk = (cnt >> 8) & 255;   // entries worth reading
 #pragma unroll
       for (int j = 0; j < KR; ++j) {
-        const bool in = j < K;
-        ti[j] = in ? __ldcg(ii + K + j) : -1;
-        tv[j] = in ? __ldcg(f + j) : 0.f;
-        ki[j] = (in && a.T > 0.f) ? __ldcg(ii + 3 * K + j) : -1;
-        kv[j] = (in && a.T > 0.f) ? __ldcg(f + 2 * K + j) : 0.f;
-        kl[j] = (in && a.T > 0.f) ? __ldcg(f + 4 * K + j) : 0.f;
+        ti[j] = j < nt ? __ldcg(ii + K + j) : -1;
+        tv[j] = j < nt ? __ldcg(f + j) : 0.f;
+        ki[j] = (j < nk && a.T > 0.f) ? __ldcg(ii + 3 * K + j) : -1;
+        kv[j] = (j < nk && a.T > 0.f) ? __ldcg(f + 2 * K + j) : 0.f;
+        kl[j] = (j < nk && a.T > 0.f) ? __ldcg(f + 4 * K + j) : 0.f;
       }
       if (h.x == -INFINITY) continue;  // a piece that scanned nothing
       if (h.x > m) { const float d = m - h.x; s0 *= __expf(d); sT *= __expf(d * invT); m = h.x; }
@@ -196,8 +223,14 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
       s0 += h.y * __expf(d); sT += h.z * __expf(d * invT);
 #pragma unroll
       for (int j = 0; j < KR; ++j) {
-        if (ti[j] >= 0 && tv[j] >= bL) top.insert(tv[j], ti[j], tv[j]);
-        if (ki[j] >= 0 && kv[j] >= bK) key.insert(kv[j], ki[j], kl[j]);
+        if (ti[j] >= 0 && tv[j] >= bL) {
+          const int e = atomicAdd(&c_n[0], 1);
+          if (e < MERGE_CAP) { c_v[0][e] = tv[j]; c_i[0][e] = ti[j]; c_l[0][e] = tv[j]; }
+        }
+        if (ki[j] >= 0 && kv[j] >= bK) {
+          const int e = atomicAdd(&c_n[1], 1);
+          if (e < MERGE_CAP) { c_v[1][e] = kv[j]; c_i[1][e] = ki[j]; c_l[1][e] = kl[j]; }
+        }
       }
     }
     // fold the (max, sums) pairs
@@ -223,19 +256,43 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
       a.lse0[p] = gm + logf(g0);
       a.lseT[p] = a.T > 0.f ? gm * invT + logf(gT) : gm + logf(g0);
     }
-    __syncthreads();
     // leave the launch-wide pruning state of this parent clean for the next launch
     if (tid < 2 * K) a.slots[((size_t)(tid / K) * a.cap + p) * K + tid % K] = 0u;
-    block_select<KR>(top, K, a.top_tok + (size_t)p * K, a.top_logit + (size_t)p * K, s_v, s_i, s_l);
-    if (a.T > 0.f) {
-      block_select<KR>(key, K, a.draw_tok + (size_t)p * K, a.draw_logit + (size_t)p * K, s_v, s_i, s_l);
+    const bool fits = c_n[0] <= MERGE_CAP && c_n[1] <= MERGE_CAP;   // uniform: read after the barrier above
+    if (fits) {
+      // the usual case: a few dozen candidates survive the bounds; one warp per list picks the K best
+      if (warp == 0) warp_select(c_v[0], c_i[0], c_l[0], c_n[0], K, lane, a.top_tok + (size_t)p * K, a.top_logit + (size_t)p * K);
+      if (warp == 1 && a.T > 0.f)
+        warp_select(c_v[1], c_i[1], c_l[1], c_n[1], K, lane, a.draw_tok + (size_t)p * K, a.draw_logit + (size_t)p * K);
+      __syncthreads();
     } else {
+      // too many candidates for the shared arrays (bounds not formed, e.g. tiny vocabularies): every
+      // thread rebuilds private sorted lists from its pieces and the block selects over their heads
+      MList<KR> top, key;
+      top.init(); key.init();
+      for (int q = tid; q < npieces; q += MERGE_THREADS) {
+        const int ts_ = q / R, rho = q % R;
+        const int slot = R > 1 ? rho * (128 / R) + p : p;
+        const float* rec = a.rec + ((size_t)ts_ * a.cap + slot) * rw;
+        if (__ldcg(rec) == -INFINITY) continue;
+        const float* f = rec + 4; const int* ii = reinterpret_cast<const int*>(rec) + 4;
+        for (int j = 0; j < K; ++j) {
+          const int t = __ldcg(ii + K + j);
+          if (t >= 0) top.insert(__ldcg(f + j), t, __ldcg(f + j));
+          if (a.T > 0.f) { const int k2 = __ldcg(ii + 3 * K + j); if (k2 >= 0) key.insert(__ldcg(f + 2 * K + j), k2, __ldcg(f + 4 * K + j)); }
+        }
+      }
+      __syncthreads();
+      block_select<KR>(top, K, a.top_tok + (size_t)p * K, a.top_logit + (size_t)p * K, s_v, s_i, s_l);
+      if (a.T > 0.f) block_select<KR>(key, K, a.draw_tok + (size_t)p * K, a.draw_logit + (size_t)p * K, s_v, s_i, s_l);
+    }
+    if (!(a.T > 0.f)) {
       if (tid < K) {
         a.draw_tok[(size_t)p * K + tid] = a.top_tok[(size_t)p * K + tid];
         a.draw_logit[(size_t)p * K + tid] = a.top_logit[(size_t)p * K + tid];
       }
-      __syncthreads();
     }
+    __syncthreads();
   }
 }
 

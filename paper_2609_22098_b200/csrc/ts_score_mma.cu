@@ -254,7 +254,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
       }
       if (alive && active) {
         const int gslot = R > 1 ? row : g * 128 + row;
-        st.store(a.rec + ((size_t)(tile * MMA_S + s) * a.cap + gslot) * rw);
+        st.store(a.rec + ((size_t)(tile * MMA_S + s) * a.cap + gslot) * rw, dec_f(s_thr[prow]), dec_f(s_thr[128 + prow]));
       }
       if (lane == 0) atomicAdd((int*)s_done, 1);   // one tick per warp per group
     }

@@ -29,63 +29,76 @@ extern "C" int ts_debug_timing_walk(unsigned long long* out) { return (int)cudaM
 #endif
 
 constexpr int VT = 256;  // threads of the verification kernels
+constexpr int ZT = 512;  // threads per target row in the row-statistics kernel
 
 // ------------------------------------------------------------------------------------------------
 // Stage 1: row statistics
 // ------------------------------------------------------------------------------------------------
 template <typename TIn>
-__global__ void __launch_bounds__(VT) zrow_stats_kernel(const TIn* Z, const int64_t* z_row_off, int B, int V, float T,
+__global__ void __launch_bounds__(ZT) zrow_stats_kernel(const TIn* Z, const int64_t* z_row_off, int B, int V, float T,
                                                        float* z_max, int* z_arg, float* z_logs) {
-  __shared__ float s_v[VT / 32]; __shared__ int s_i[VT / 32]; __shared__ float s_m;
+  // One CTA per target row, one sweep: every thread keeps a running (max, arg-max, sum of exp((z-max)/T))
+  // over its share of the row, four 16-byte loads in flight, and the block folds the triples.
+  __shared__ float s_v[ZT / 32]; __shared__ int s_i[ZT / 32]; __shared__ float s_s[ZT / 32];
   const int64_t rows = z_row_off[B];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int VEC = Elem<TIn>::VEC;
+  constexpr int UNR = 4;
   const bool vec_ok = (V % VEC) == 0;
   const float invT = T > 0.f ? 1.f / T : 1.f;
   for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
     const TIn* z = Z + row * V;
-    float bv = -INFINITY; int bi = 0x7FFFFFFF;
-    if (vec_ok) {
-      for (int c = tid * VEC; c < V; c += VT * VEC) {
-        float x[8];
-        if (sizeof(TIn) == 2) { const uint4 v = __ldg(reinterpret_cast<const uint4*>(z + c)); unpack_bf16x8(v, x); }
-        else { const float4 v = __ldg(reinterpret_cast<const float4*>(z + c)); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+    float bv = -INFINITY, sum = 0.f; int bi = 0x7FFFFFFF;
+    auto take = [&](const float* x, int c, int n) {
+      float vm = x[0]; int vi = 0;
 #pragma unroll
-        for (int i = 0; i < VEC; ++i) if (x[i] > bv) { bv = x[i]; bi = c + i; }
+      for (int i = 1; i < VEC; ++i) if (i < n && x[i] > vm) { vm = x[i]; vi = i; }
+      if (vm > bv) { sum *= __expf((bv - vm) * invT); bv = vm; bi = c + vi; }   // first maximum wins: indices increase
+      if (T > 0.f) {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) if (i < n) sum += __expf((x[i] - bv) * invT);
+      }
+    };
+    if (vec_ok) {
+      int c = tid * VEC;
+      for (; c + (UNR - 1) * ZT * VEC < V; c += UNR * ZT * VEC) {
+        float x[UNR][8];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+          const TIn* pz = z + c + u * ZT * VEC;
+          if (sizeof(TIn) == 2) unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(pz)), x[u]);
+          else { const float4 v = __ldg(reinterpret_cast<const float4*>(pz)); x[u][0] = v.x; x[u][1] = v.y; x[u][2] = v.z; x[u][3] = v.w; }
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) take(x[u], c + u * ZT * VEC, VEC);
+      }
+      for (; c < V; c += ZT * VEC) {
+        float x[8];
+        if (sizeof(TIn) == 2) unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(z + c)), x);
+        else { const float4 v = __ldg(reinterpret_cast<const float4*>(z + c)); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+        take(x, c, VEC);
       }
     } else {
-      for (int c = tid; c < V; c += VT) { const float x = Elem<TIn>::to_f(z[c]); if (x > bv) { bv = x; bi = c; } }
+      for (int c = tid; c < V; c += ZT) { float x[8]; x[0] = Elem<TIn>::to_f(z[c]); take(x, c, 1); }
     }
+    // fold (max, arg-max, sum): value descending, ties to the lowest token
     for (int off = 16; off > 0; off >>= 1) {
       const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, off); const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, off);
-      if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+      const float os = __shfl_xor_sync(0xFFFFFFFFu, sum, off);
+      const float nm = fmaxf(bv, ov);
+      const float ns = (nm > -INFINITY) ? sum * __expf((bv - nm) * invT) + os * __expf((ov - nm) * invT) : 0.f;
+      if (ov > bv || (ov == bv && oi < bi)) { bi = oi; }
+      bv = nm; sum = ns;
     }
-    if (lane == 0) { s_v[warp] = bv; s_i[warp] = bi; }
+    if (lane == 0) { s_v[warp] = bv; s_i[warp] = bi; s_s[warp] = sum; }
     __syncthreads();
     if (tid == 0) {
-      for (int w = 1; w < VT / 32; ++w) if (s_v[w] > bv || (s_v[w] == bv && s_i[w] < bi)) { bv = s_v[w]; bi = s_i[w]; }
-      s_m = bv; z_max[row] = bv; z_arg[row] = bi;
-    }
-    __syncthreads();
-    if (T > 0.f) {
-      const float m = s_m;
-      float s = 0.f;
-      if (vec_ok) {
-        for (int c = tid * VEC; c < V; c += VT * VEC) {
-          float x[8];
-          if (sizeof(TIn) == 2) { const uint4 v = __ldg(reinterpret_cast<const uint4*>(z + c)); unpack_bf16x8(v, x); }
-          else { const float4 v = __ldg(reinterpret_cast<const float4*>(z + c)); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
-#pragma unroll
-          for (int i = 0; i < VEC; ++i) s += __expf((x[i] - m) * invT);
-        }
-      } else {
-        for (int c = tid; c < V; c += VT) s += __expf((Elem<TIn>::to_f(z[c]) - m) * invT);
-      }
-      for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
-      __syncthreads();
-      if (lane == 0) s_v[warp] = s;
-      __syncthreads();
-      if (tid == 0) { float t = 0.f; for (int w = 0; w < VT / 32; ++w) t += s_v[w]; z_logs[row] = logf(t); }
+      float gv = s_v[0]; int gi = s_i[0];
+      for (int w = 1; w < ZT / 32; ++w) if (s_v[w] > gv || (s_v[w] == gv && s_i[w] < gi)) { gv = s_v[w]; gi = s_i[w]; }
+      float gs = 0.f;
+      for (int w = 0; w < ZT / 32; ++w) if (s_v[w] > -INFINITY) gs += s_s[w] * __expf((s_v[w] - gv) * invT);
+      z_max[row] = gv; z_arg[row] = gi;
+      if (T > 0.f) z_logs[row] = logf(gs);
     }
     __syncthreads();
   }
@@ -729,9 +742,9 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
   {
     ProfScope ps(ctx, K_ZROWS, st);
     if (c.dt_Z == TS_DTYPE_BF16)
-      zrow_stats_kernel<__nv_bfloat16><<<grid_rows, VT, 0, st>>>((const __nv_bfloat16*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+      zrow_stats_kernel<__nv_bfloat16><<<grid_rows, ZT, 0, st>>>((const __nv_bfloat16*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
     else
-      zrow_stats_kernel<float><<<grid_rows, VT, 0, st>>>((const float*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+      zrow_stats_kernel<float><<<grid_rows, ZT, 0, st>>>((const float*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(rows)", e);
