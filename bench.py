@@ -145,7 +145,8 @@ def tree_stats(wl, tree, verdict):
         per_level.append(int((scored & (depth == d)).sum()))
     return dict(nodes=int(n.sum()), parents=parents, u_rows=urows, z_rows=int((n + 1).sum()),
                 levels_used=sum(1 for p in per_level if p > 0), parents_per_level=per_level,
-                acc=int(verdict["acc_len"].sum()), walk_rows=int((verdict["acc_len"].long() + 1).sum()))
+                acc=int(verdict["acc_len"].sum()), walk_rows=int((verdict["acc_len"].long() + 1).sum()),
+                walk_passes=int(((verdict["flags"].long() >> 8) & 0xFFFF).sum()))
 
 
 def snapshot(tree, verdict):
@@ -246,7 +247,10 @@ def run_ours(args, rank, world, device):
     bytes_round_min = mean("u_rows") * row_b + w_b + mean("parents") * wl.r * es + mean("walk_rows") * row_b
     peak, peak_src = measured_peak()
     dom = max(kern, key=lambda k: kern[k]["ms_per_round"]) if kern else None
-    alg = {"score_tile": bytes_score, "zrow_stats": bytes_zrows}
+    # walk: every residual reduction streams one target row and (recomputing the proposal) one base row;
+    # its range of W is staged once per launch
+    bytes_walk = mean("walk_passes") * 2 * row_b + w_b
+    alg = {"score_tile": bytes_score, "zrow_stats": bytes_zrows, "verify_walk": bytes_walk}
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
     if dom and os.path.exists(tpath):
@@ -286,6 +290,7 @@ def run_ours(args, rank, world, device):
         "parents_scored_per_s": world * mean("parents") / sec, "nodes_per_s": world * mean("nodes") / sec,
         "detail": {"mean_nodes_per_tree": mean("nodes") / B, "mean_parents_per_round": mean("parents"),
                    "mean_accepted_len": mean("acc") / B, "mean_z_rows": mean("z_rows"),
+                   "mean_walk_reductions": mean("walk_passes"),
                    "parents_per_level": used[0]["parents_per_level"], "outputs_reproduced": same},
         "clocks": clocks, "gpu_launches": launches, "kernels": kern, "roofline": roofline, "round_hbm": round_hbm,
         "e2e": e2e,

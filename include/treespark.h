@@ -50,8 +50,10 @@ extern "C" {
 #define TS_DMAX 16       /* largest block depth D */
 #define TS_CALIB_KNOTS 16
 
-/* per-request flag bits written by ts_verify_tree */
+/* per-request flag word written by ts_verify_tree: bits 0..7 flags, bits 8..23 the number of
+ * vocabulary-wide residual reductions the walk of that request needed (T > 0; a statistic) */
 #define TS_FLAG_ZERO_MASS 64u  /* a residual target lost all mass; the previous residual was kept */
+#define TS_FLAGS_MASK 0xFFu
 
 typedef struct ts_ctx ts_ctx;
 

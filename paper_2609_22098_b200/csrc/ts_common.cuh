@@ -93,6 +93,8 @@ struct VerifyState {
   int scan_tile;  // tile holding the bonus token
   int row_node;   // node whose rows the pass reads
   int result;     // token found by the range rescan
+  int npass;      // vocabulary reductions this request has asked for
+  int pad_;
   double C, Zj, Qused, target, before;
   double passC;   // C of the requested pass
   double partsC;  // C the stored range sums were computed for (-1 = none)

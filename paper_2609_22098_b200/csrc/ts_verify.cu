@@ -197,6 +197,7 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
     if (st.need == 2) {  // the rescan wrote its token
       a.bonus[b] = st.result;
       a.acc_len[b] = st.acc;
+      a.flags[b] |= (uint32_t)min(st.npass, 0xFFFF) << 8;   // bits 8..23: reductions this walk needed
       st.need = 3;
       atomicSub(a.ctr + 4, 1);
     }
@@ -290,6 +291,7 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
     *gst = st;
     __threadfence();
     if (st.need == 1 || st.need == 4) a.wk_list[parity * a.B + atomicAdd(a.ctr + parity, 1)] = b;
+    if (st.need == 1 || st.need == 4) gst->npass = st.npass + 1;
     else if (st.need == 2) a.sc_list[parity * a.B + atomicAdd(a.ctr + 2 + parity, 1)] = b;
   }
   __syncwarp();
@@ -462,6 +464,7 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
       VerifyState& st = a.state[b];
       st.cur = -1; st.j = 0; st.acc = 0; st.need = 0; st.nf = 0; st.scan_tile = -1; st.row_node = -1; st.result = -1;
       st.C = 0.0; st.Zj = 1.0; st.Qused = 0.0; st.target = 0.0; st.before = 0.0; st.passC = 0.0; st.partsC = -1.0;
+      st.npass = 0; st.pad_ = 0;
       a.flags[b] = 0u;
       a.status[b] = okn ? TS_OK : TS_ERR_INVALID;
       if (!okn) { st.need = 3; a.acc_len[b] = 0; a.bonus[b] = -1; }

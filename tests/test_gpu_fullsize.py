@@ -1,0 +1,54 @@
+"""Parity at the benchmark configurations' full sizes, in the launch configuration bench.py times:
+the whole batch runs on the GPU, the oracle recomputes a sample of the requests one by one on the
+same bytes (a full batch would take the oracle minutes)."""
+import dataclasses
+
+import pytest
+import torch
+
+from gpu_harness import Round, check_round, make_gpu, make_oracle
+from paper_2609_22098_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def run(wl, T, theta, reqs, seed, round_seed=77, B=None):
+    rnd = Round(wl, seed=seed, B=B, theta=theta)
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
+    orc = make_oracle(wl, rnd.table)
+    st = check_round(ts, orc, rnd, T, round_seed=round_seed, reqs=reqs)
+    assert st["trees"] == len(reqs)
+    return st
+
+
+def test_serve32_full_size_sampled_requests():
+    wl = synth.WORKLOADS["serve32"]
+    st = run(wl, 1.0, wl.theta, reqs=list(range(0, 32, 2)), seed=2609)
+    assert st["nodes"] > 0 and st["trees_exempt"] <= 2
+
+
+@pytest.mark.parametrize("T,theta", [(0.0, 0.1), (0.7, 0.03), (1.0, 0.3)])
+def test_decode_full_size(T, theta):
+    wl = synth.WORKLOADS["decode"]
+    st = run(wl, T, theta, reqs=[0], seed=31 + int(10 * T))
+    assert st["trees"] == 1
+
+
+def test_wide_full_size_one_request():
+    wl = synth.WORKLOADS["wide"]
+    st = run(wl, 0.7, wl.theta, reqs=[3], seed=5)
+    assert st["nodes"] >= 16
+
+
+def test_sweep_largest_batch_is_the_chain():
+    wl = synth.WORKLOADS["sweep"]
+    theta = synth.sweep_theta(128, seed=9)
+    assert theta >= 1.0 and synth.sweep_theta(1, seed=9) < synth.sweep_theta(16, seed=9) < 1.0
+    st = run(wl, 1.0, theta, reqs=[0, 64, 127], seed=9, B=128)
+    assert st["nodes"] == 3 * wl.D          # theta >= 1: every request is a chain of D nodes
+
+
+def test_sweep_mid_batch():
+    wl = synth.WORKLOADS["sweep"]
+    st = run(wl, 1.0, synth.sweep_theta(16, seed=9), reqs=[1, 9], seed=10, B=16)
+    assert st["trees"] == 2
