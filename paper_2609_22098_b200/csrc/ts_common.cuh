@@ -188,15 +188,17 @@ __device__ __forceinline__ double u01(uint32_t x) { return ((double)x + 0.5) * (
 // Gumbel noise -log(-log u) for u = (X + 0.5) / 2^32, accurate in fp32 over the whole range: near
 // u = 1 the complement 1-u is formed exactly from the integer.
 __device__ __forceinline__ float gumbel_from_bits(uint32_t X) {
+  // absolute error of the fast logarithm is ~1e-7 * |log2 x|: a few 1e-6 on the key at most, far
+  // inside the near-tie margin the parity tests use; log1pf keeps the u -> 1 end exact
   float a;
   if (X >= 0x80000000u) {
     const float t = ((float)(0xFFFFFFFFu - X) + 0.5f) * 2.3283064365386963e-10f;
     a = -log1pf(-t);
   } else {
     const float u = ((float)X + 0.5f) * 2.3283064365386963e-10f;
-    a = -logf(u);
+    a = -__logf(u);
   }
-  return -logf(a);
+  return -__logf(a);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -167,12 +167,10 @@ __device__ __forceinline__ unsigned slots_min(const SharedThr& g, int K) {
   return m;
 }
 
-// Gumbel noise of token v from both halves of its uniform (the low half costs a second generator call;
-// out of line because it runs for a few tokens per thousand once the bounds are warm).
-static __device__ __noinline__ float gumbel_exact(uint32_t c16, int v, uint64_t seed, int req, uint64_t hash) {
-  const uint4 fw = stream_words(seed, req, hash, STREAM_GUMBEL_FINE, (uint32_t)v >> 3);
-  const uint32_t f16 = (word_of(fw, (v & 7) >> 1) >> (16 * (v & 1))) & 0xFFFFu;
-  return gumbel_from_bits((c16 << 16) | f16);
+// low halves of the uniforms of the eight tokens around v: second generator stream, out of line because
+// it runs for a few tokens per thousand once the bounds are warm
+static __device__ __noinline__ uint4 fine_words(int v, uint64_t seed, int req, uint64_t hash) {
+  return stream_words(seed, req, hash, STREAM_GUMBEL_FINE, (uint32_t)v >> 3);
 }
 
 // register-array element by run-time index (a select chain: the array stays in registers)
@@ -247,13 +245,17 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
       mk |= (uint32_t)(i < valid && bnd >= thr) << i;
     }
     float kmax = -INFINITY;
+    uint4 fw = make_uint4(0, 0, 0, 0);
+    int fine_call = -1;
 #pragma unroll 1
     while (mk) {
       const int i = __ffs(mk) - 1;
       mk &= mk - 1;
       const float li = pick16(l, i);
       const uint32_t c16 = (pick8(cw0, cw1, i >> 1) >> (16 * (i & 1))) & 0xFFFFu;
-      const float key = li * invT + gumbel_exact(c16, v0 + i, seed, req, hash);
+      if (fine_call != (i >> 3)) { fw = fine_words(v0 + i, seed, req, hash); fine_call = i >> 3; }
+      const uint32_t fword = ((i & 7) >> 1) == 0 ? fw.x : (((i & 7) >> 1) == 1 ? fw.y : (((i & 7) >> 1) == 2 ? fw.z : fw.w));
+      const float key = li * invT + gumbel_from_bits((c16 << 16) | ((fword >> (16 * (i & 1))) & 0xFFFFu));
       if (key > st.thrK && key >= gK) { st.thrK = st.L.insert_key(key, v0 + i, li); kmax = fmaxf(kmax, key); }
     }
     if (kmax > st.bestK) { st.bestK = kmax; publish(gk, kmax); }

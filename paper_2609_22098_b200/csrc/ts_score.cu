@@ -347,7 +347,7 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
   m.rec = rec; m.thr = a.thr; m.slots = a.slots;
   m.lse0 = lse0; m.lseT = lseT; m.top_tok = top_tok; m.top_logit = top_logit; m.draw_tok = draw_tok; m.draw_logit = draw_logit;
   int blocks = P_dev ? cap : P;
-  if (blocks > 8 * ctx->num_sms) blocks = 8 * ctx->num_sms;
+  if (blocks > 2 * ctx->num_sms) blocks = 2 * ctx->num_sms;   // parents beyond that are looped over
   if (blocks < 1) blocks = 1;
   {
     ProfScope ps(ctx, K_MERGE, st);

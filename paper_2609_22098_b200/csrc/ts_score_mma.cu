@@ -57,7 +57,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort) return false;
-    if (i > 64) __nanosleep(64);
+    if (i > 8) __nanosleep(100);
   }
   *abort = 1;
   if (err) atomicExch(err, 1);
@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
           }
           s_thr[(g & 1) * 256 + rr] = mL; s_thr[(g & 1) * 256 + 128 + rr] = mK;
         }
-        __nanosleep(200);
+        __nanosleep(1000);
       }
       __syncwarp();
     }
