@@ -13,6 +13,10 @@ namespace ts {
 constexpr int KMAX = TS_KMAX;
 constexpr int DMAX = TS_DMAX;
 constexpr int KNOTS = TS_CALIB_KNOTS;
+// Words between two pruning-bound slots: one 128-byte line each.  Every piece of a launch publishes into
+// these words with atomicMax in the launch's first microseconds; packed together they queue up on a
+// handful of L2 lines (measured: a third of the scoring launch at stride 1).
+constexpr int SLOT_STRIDE = 32;
 constexpr int SCORE_THREADS = 128;   // one parent per thread; every thread scans the CTA's whole tile
 constexpr int CHUNK = 16;            // tokens per coarse generator call
 constexpr int MMA_S = 2;             // column splits per tile in the tensor-core scoring kernel (warps per row quarter)
@@ -47,6 +51,11 @@ struct ts_ctx {
   int use_mma;      // 1: scoring runs on the tensor-core kernel, 0: on the fp32 FMA kernel
   ts::DevCalib calib;
   void* prof;  // ts::Prof*, instrumentation state
+  // tensor-map descriptor of the W matrix last scored with (bulk-tensor loads of the W tile); -1: the
+  // driver's encoder is not available, the kernel stages W with plain loads
+  alignas(64) unsigned char tmapW[128];
+  const void* tmapW_ptr;
+  int tma_state;   // 0 not tried yet, 1 encoder found, -1 unavailable
 };
 
 namespace ts {
@@ -115,7 +124,7 @@ __host__ inline WsLayout make_layout(const ts_ctx* ctx, int B) {
     int cap = (L.Pcap + 7) / 8 * 8, S = 1;
     if (ctx->use_mma) { cap = (L.Pcap + 127) / 128 * 128; S = MMA_S; }
     L.rec_cap = cap;
-    L.rec = take(align_up(nt * S * (size_t)cap * ((4 + 5 * K + 3) & ~(size_t)3) * 4, 256) + (size_t)cap * (2 + 2 * K) * 4);
+    L.rec = take(align_up(nt * S * (size_t)cap * ((4 + 5 * K + 3) & ~(size_t)3) * 4, 256) + (size_t)cap * (2 + 2 * K * SLOT_STRIDE) * 4);
     L.err = take(16);
   }
   L.res_lse0 = take(P * 4); L.res_lseT = take(P * 4);

@@ -31,7 +31,7 @@ struct ExpandArgs {
   float* root_lseT; int *req_npar, *req_base, *req_nscored;
   // candidates
   int *cd_valid, *cd_parent, *cd_sib, *cd_tok; double *cd_logkey, *cd_logS; float *cd_q0, *cd_logqT; int* cd_rank;
-  int* status; int* err; unsigned* thr; int thr_words;
+  int* status; int* err; unsigned* thr; int thr_head, thr_words;
 };
 
 __device__ __forceinline__ void request_caps(const ExpandArgs& a, int b, int& K_eff, int& N_eff, double& log_theta) {
@@ -47,8 +47,12 @@ __device__ __forceinline__ void request_caps(const ExpandArgs& a, int b, int& K_
 
 __global__ void expand_init_kernel(ExpandArgs a) {
   const int b = blockIdx.x;
+  // pruning state of the scoring launches: the threshold words, then one word per slot (the slots sit
+  // SLOT_STRIDE words apart; only the first word of each is ever used)
+  for (int i = b * blockDim.x + threadIdx.x; i < a.thr_words; i += gridDim.x * blockDim.x)
+    a.thr[i < a.thr_head ? i : a.thr_head + (size_t)(i - a.thr_head) * SLOT_STRIDE] = 0u;
+  if (b >= a.B) return;
   for (int s = threadIdx.x; s < a.N; s += blockDim.x) a.pl_alive[(size_t)b * a.N + s] = 0;
-  for (int i = b * blockDim.x + threadIdx.x; i < a.thr_words; i += gridDim.x * blockDim.x) a.thr[i] = 0u;
   if (threadIdx.x == 0) {
     const int tok = a.anchor[b];
     const bool ok = tok >= 0 && tok < a.V && a.theta[b] == a.theta[b];
@@ -379,9 +383,10 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   a.cd_tok = (int*)(ws + L.cd_tok); a.cd_logkey = (double*)(ws + L.cd_logkey); a.cd_logS = (double*)(ws + L.cd_logS);
   a.cd_q0 = (float*)(ws + L.cd_q0); a.cd_logqT = (float*)(ws + L.cd_logqT); a.cd_rank = (int*)(ws + L.cd_rank);
   a.status = status; a.err = (int*)(ws + L.err);
-  a.thr = thr_base(ctx, (float*)(ws + L.rec), L.rec_cap); a.thr_words = (int)(thr_bytes(ctx, L.rec_cap) / 4);
+  a.thr = thr_base(ctx, (float*)(ws + L.rec), L.rec_cap);
+  a.thr_head = 2 * L.rec_cap; a.thr_words = a.thr_head + 2 * L.rec_cap * c.K;   // words to clear, not their span
 
-  { ProfScope ps(ctx, K_INIT, st); expand_init_kernel<<<B, 64, 0, st>>>(a); }
+  { ProfScope ps(ctx, K_INIT, st); expand_init_kernel<<<B > 296 ? B : 296, 256, 0, st>>>(a); }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(init)", e);
   const size_t level_smem = (size_t)(c.Nmax + c.Nmax * c.K) * sizeof(Entry);

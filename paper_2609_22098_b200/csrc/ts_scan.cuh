@@ -159,11 +159,11 @@ struct SharedThr {
   int mine;         // this piece's slot
 };
 
-__device__ __forceinline__ void publish(const SharedThr& g, float x) { atomicMax(g.slot + g.mine, enc_f(x)); }
+__device__ __forceinline__ void publish(const SharedThr& g, float x) { atomicMax(g.slot + g.mine * SLOT_STRIDE, enc_f(x)); }
 
 __device__ __forceinline__ unsigned slots_min(const SharedThr& g, int K) {
   unsigned m = __ldcg(g.slot);
-  for (int j = 1; j < K; ++j) m = min(m, __ldcg(g.slot + j));
+  for (int j = 1; j < K; ++j) m = min(m, __ldcg(g.slot + j * SLOT_STRIDE));
   return m;
 }
 
@@ -194,7 +194,8 @@ __device__ __forceinline__ uint32_t pick8(const uint4& a, const uint4& b, int i)
 template <class Lists>
 __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, int v0, int valid, float T, float invT,
                                            uint64_t seed, int req, uint64_t hash, const float* ghi,
-                                           float gL, float gK, const SharedThr& gl, const SharedThr& gk) {
+                                           float gL, float gK, const SharedThr& gl, const SharedThr& gk,
+                                           const volatile unsigned* liveL = nullptr, const volatile unsigned* liveK = nullptr) {
   float cm = -INFINITY;
 #pragma unroll
   for (int i = 0; i < CHUNK; ++i) if (i < valid) cm = fmaxf(cm, l[i]);
@@ -226,9 +227,13 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
       const int i = __ffs(mk) - 1;
       mk &= mk - 1;
       const float li = pick16(l, i);
-      if (li > st.thrL) st.thrL = st.L.insert_top(li, v0 + i);
+      if (liveL) gL = fmaxf(gL, dec_f(*liveL));
+      if (li > st.thrL && li >= gL) {
+        st.thrL = st.L.insert_top(li, v0 + i);
+        // publish at once: early in a launch every piece is waiting for the first bounds
+        if (li > st.bestL) { st.bestL = li; publish(gl, li); }
+      }
     }
-    if (cm > st.bestL) { st.bestL = cm; publish(gl, cm); }
   }
   if (T > 0.f) {
     // high half of each token's uniform: one generator call per eight tokens
@@ -244,7 +249,6 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
       const float bnd = l[i] * invT + ((c16 >> 8) != 255u ? ghi[c16 >> 8] : ghi[256 + (c16 & 255u)]);
       mk |= (uint32_t)(i < valid && bnd >= thr) << i;
     }
-    float kmax = -INFINITY;
     uint4 fw = make_uint4(0, 0, 0, 0);
     int fine_call = -1;
 #pragma unroll 1
@@ -253,12 +257,20 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
       mk &= mk - 1;
       const float li = pick16(l, i);
       const uint32_t c16 = (pick8(cw0, cw1, i >> 1) >> (16 * (i & 1))) & 0xFFFFu;
+      if (liveK) {
+        // the bounds may have risen since the mask was built (they do, steeply, while a launch warms up)
+        gK = fmaxf(gK, dec_f(*liveK));
+        const float bnd = li * invT + ((c16 >> 8) != 255u ? ghi[c16 >> 8] : ghi[256 + (c16 & 255u)]);
+        if (bnd < fmaxf(st.thrK, gK)) continue;
+      }
       if (fine_call != (i >> 3)) { fw = fine_words(v0 + i, seed, req, hash); fine_call = i >> 3; }
       const uint32_t fword = ((i & 7) >> 1) == 0 ? fw.x : (((i & 7) >> 1) == 1 ? fw.y : (((i & 7) >> 1) == 2 ? fw.z : fw.w));
       const float key = li * invT + gumbel_from_bits((c16 << 16) | ((fword >> (16 * (i & 1))) & 0xFFFFu));
-      if (key > st.thrK && key >= gK) { st.thrK = st.L.insert_key(key, v0 + i, li); kmax = fmaxf(kmax, key); }
+      if (key > st.thrK && key >= gK) {
+        st.thrK = st.L.insert_key(key, v0 + i, li);
+        if (key > st.bestK) { st.bestK = key; publish(gk, key); }
+      }
     }
-    if (kmax > st.bestK) { st.bestK = kmax; publish(gk, kmax); }
   }
 }
 

@@ -63,8 +63,8 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
     RowScan<Lists> st;
     st.init(K);
     float gL = -INFINITY, gK = -INFINITY;
-    const SharedThr gl{a.slots + (size_t)p * K, tile % K};
-    const SharedThr gk{a.slots + ((size_t)a.cap + p) * K, tile % K};
+    const SharedThr gl{a.slots + (size_t)p * K * SLOT_STRIDE, tile % K};
+    const SharedThr gk{a.slots + ((size_t)a.cap + p) * K * SLOT_STRIDE, tile % K};
     for (int c0 = 0; c0 < tlen; c0 += CHUNK) {
       const int valid = min(CHUNK, tlen - c0);
       float l[CHUNK];
@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
   const int npieces = a.ntiles * a.S * R;
   for (int p = blockIdx.x; p < P; p += gridDim.x) {
     // final launch-wide lower bounds of this parent's K-th best logit / key: entries below cannot win
-    const SharedThr gl{a.slots + (size_t)p * K, 0}, gk{a.slots + ((size_t)a.cap + p) * K, 0};
+    const SharedThr gl{a.slots + (size_t)p * K * SLOT_STRIDE, 0}, gk{a.slots + ((size_t)a.cap + p) * K * SLOT_STRIDE, 0};
     const float bL = dec_f(slots_min(gl, K)), bK = a.T > 0.f ? dec_f(slots_min(gk, K)) : -INFINITY;
     if (tid < 2) c_n[tid] = 0;
     __syncthreads();
@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
       a.lseT[p] = a.T > 0.f ? gm * invT + logf(gT) : gm + logf(g0);
     }
     // leave the launch-wide pruning state of this parent clean for the next launch
-    if (tid < 2 * K) a.slots[((size_t)(tid / K) * a.cap + p) * K + tid % K] = 0u;
+    if (tid < 2 * K) a.slots[(((size_t)(tid / K) * a.cap + p) * K + tid % K) * SLOT_STRIDE] = 0u;
     const bool fits = c_n[0] <= MERGE_CAP && c_n[1] <= MERGE_CAP;   // uniform: read after the barrier above
     if (fits) {
       // the usual case: a few dozen candidates survive the bounds; one warp per list picks the K best
@@ -306,7 +306,7 @@ size_t score_scratch_bytes(const ts_ctx* ctx, int P, int* cap_out) {
   if (cap_out) *cap_out = cap;
   // records, then the pruning state: 2 threshold words and 2K slot words per slot of capacity
   return align_up((size_t)ctx->tile.ntiles * S * cap * rec_words(ctx->cfg.K) * sizeof(float), 256) +
-         align_up((size_t)cap * (2 + 2 * (size_t)ctx->cfg.K) * sizeof(unsigned), 256);
+         align_up((size_t)cap * (2 + 2 * (size_t)ctx->cfg.K * SLOT_STRIDE) * sizeof(unsigned), 256);
 }
 
 unsigned* thr_base(const ts_ctx* ctx, float* rec, int cap) {
@@ -314,7 +314,7 @@ unsigned* thr_base(const ts_ctx* ctx, float* rec, int cap) {
   return (unsigned*)((char*)rec + align_up((size_t)ctx->tile.ntiles * S * cap * rec_words(ctx->cfg.K) * sizeof(float), 256));
 }
 
-size_t thr_bytes(const ts_ctx* ctx, int cap) { return (size_t)cap * (2 + 2 * (size_t)ctx->cfg.K) * sizeof(unsigned); }
+size_t thr_bytes(const ts_ctx* ctx, int cap) { return (size_t)cap * (2 + 2 * (size_t)ctx->cfg.K * SLOT_STRIDE) * sizeof(unsigned); }
 
 cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,

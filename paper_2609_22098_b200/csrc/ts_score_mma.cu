@@ -14,6 +14,7 @@
 // "full" barrier; epilogue warps arrive on its "empty" barrier when they have drained it.
 // Every wait is bounded: when one runs out the kernel raises an error word, skips the remaining work,
 // frees its tensor memory and returns.
+#include <cuda.h>   // CUtensorMap and its enums; the encoder itself is looked up at run time
 #include "ts_internal.h"
 #include "ts_scan.cuh"
 
@@ -34,6 +35,7 @@ constexpr int BLK_N = 128;
 constexpr int NBUF = 4;                 // accumulator buffers of BLK_N columns in tensor memory
 constexpr uint32_t TMEM_COLS = NBUF * BLK_N;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr int MAX_BLK = 32;             // blocks of BLK_N tokens in the largest tile (4096 tokens)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -67,6 +69,16 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// one box of the W tensor map (64 tokens x rp rows, 128-byte swizzle) into shared memory; completion
+// is counted in bytes on `bar`.  c0 (the token coordinate) must be a multiple of 8.
+__device__ __forceinline__ void tma_load_box(void* dst, const CUtensorMap* tm, int c0, int c1, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
+}
+
 // shared-memory matrix descriptor: 128-byte swizzle, descriptor version 1 (sm_100)
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
@@ -99,7 +111,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 }
 
 template <class Lists>
-__global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) {
+__global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma) {
   extern __shared__ unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = a.P_dev ? *a.P_dev : a.P;
@@ -108,6 +120,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
   const int r = a.r, rp = (r + 63) / 64 * 64, V = a.V, TV = a.TV, K = a.K;
   const int tile = blockIdx.x, t0 = tile * TV, tlen = min(TV, V - t0);
   const int nslab = TV / 64;
+  const int nblk_w = (tlen + BLK_N - 1) / BLK_N;
   const uint32_t slab_bytes = (uint32_t)rp * 128u;       // one 64-token slab of W
   const uint32_t a_slab_bytes = 128u * 128u;             // 128 rows x 128 B
   unsigned char* sm = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -123,6 +136,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
   // per-row copies of the launch-wide pruning bounds (logit, key), refreshed once per block of tokens
   volatile unsigned* s_thr = reinterpret_cast<volatile unsigned*>(s_tmem + 4);   // [group parity][2][128]
   volatile int* s_done = reinterpret_cast<volatile int*>(s_tmem + 2);             // epilogue warps finished
+  uint64_t* w_full = reinterpret_cast<uint64_t*>(const_cast<unsigned*>(s_thr) + 512);   // [MAX_BLK] W slabs of block nb landed
 
   const __nv_bfloat16* Wg = reinterpret_cast<const __nv_bfloat16*>(a.W);
   const __nv_bfloat16* Ug = reinterpret_cast<const __nv_bfloat16*>(a.U);
@@ -139,9 +153,20 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
     for (int i = 0; i < NBUF; ++i) { mbar_init(t_full + i, 1); mbar_init(t_empty + i, EPI_WARPS); }
     *s_abort = 0;
     *s_done = 0;
+    if (use_tma) for (int i = 0; i < nblk_w; ++i) mbar_init(w_full + i, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (use_tma) {
+      // W tile by bulk-tensor loads, one barrier per block of 128 tokens so that the first MMAs start
+      // while the rest of the tile is still in flight; tokens past V and rows past r arrive as zeros
+      for (int nb = 0; nb < nblk_w; ++nb) {
+        const int ns = (tlen - nb * BLK_N > 64) ? 2 : 1;
+        mbar_expect_tx(w_full + nb, (uint32_t)ns * slab_bytes);
+        for (int h = 0; h < ns; ++h)
+          tma_load_box(Ws + (size_t)(2 * nb + h) * slab_bytes, &tmW, t0 + (2 * nb + h) * 64, 0, w_full + nb);
+      }
+    }
   }
-  {  // W tile: 16-byte chunks (8 tokens of one row), swizzled: chunk j of row k lands at chunk j ^ (k & 7)
+  if (!use_tma) {  // W tile: 16-byte chunks (8 tokens of one row), swizzled: chunk j of row k lands at chunk j ^ (k & 7)
     const int per_slab = rp * 8;
     for (int idx = tid; idx < nslab * per_slab; idx += MMA_THREADS) {
       const int slab = idx / per_slab, rem = idx % per_slab, k = rem >> 3, j = rem & 7;
@@ -207,8 +232,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
       bool have_next = false;
       const int pc = active ? p : 0;
       const int pid = ((tile * MMA_S + s) * R + rho) % K;   // which of the parent's K slots this piece feeds
-      const SharedThr gl{a.slots + (size_t)pc * K, pid};
-      const SharedThr gk{a.slots + ((size_t)a.cap + pc) * K, pid};
+      const SharedThr gl{a.slots + (size_t)pc * K * SLOT_STRIDE, pid};
+      const SharedThr gk{a.slots + ((size_t)a.cap + pc) * K * SLOT_STRIDE, pid};
       for (int nb = 0; nb < nblk; ++nb) {
         const int it = g * nblk + nb, tb = it % NBUF, u = it / NBUF;
         int ok = 1;
@@ -244,7 +269,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
             unpack_bf16x8(u1, ub + 8);
 #pragma unroll
             for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] + ub[i] : 0.f;
-            scan_chunk(st, acc, v0, valid, T, invT, a.seed, req, hash, ghi, gLc, gKc, gl, gk);
+            scan_chunk(st, acc, v0, valid, T, invT, a.seed, req, hash, ghi, gLc, gKc, gl, gk, s_thr + prow, s_thr + 128 + prow);
           }
         }
         tc_fence_before();
@@ -270,10 +295,12 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
         for (int rr = lane; rr < per; rr += 32) {
           const int p = R > 1 ? rr : g * 128 + rr;
           if (p >= P) continue;
-          unsigned mL = __ldcg(a.slots + (size_t)p * K), mK = __ldcg(a.slots + ((size_t)a.cap + p) * K);
+          const unsigned* sl = a.slots + (size_t)p * K * SLOT_STRIDE;
+          const unsigned* sk = a.slots + ((size_t)a.cap + p) * K * SLOT_STRIDE;
+          unsigned mL = __ldcg(sl), mK = __ldcg(sk);
           for (int j = 1; j < K; ++j) {
-            mL = min(mL, __ldcg(a.slots + (size_t)p * K + j));
-            mK = min(mK, __ldcg(a.slots + ((size_t)a.cap + p) * K + j));
+            mL = min(mL, __ldcg(sl + j * SLOT_STRIDE));
+            mK = min(mK, __ldcg(sk + j * SLOT_STRIDE));
           }
           s_thr[(g & 1) * 256 + rr] = mL; s_thr[(g & 1) * 256 + 128 + rr] = mK;
         }
@@ -294,6 +321,9 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
           if (!mbar_wait(t_empty + tb, (u - 1) & 1, s_abort, a.err)) { alive = false; break; }
           tc_fence_after();
         }
+        if (use_tma && g == 0) {
+          if (!mbar_wait(w_full + nb, 0, s_abort, a.err)) { alive = false; break; }
+        }
         const int n = (tlen - nb * BLK_N > 64) ? 128 : 64;
         const uint32_t idesc = instr_desc(n);
         const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
@@ -308,6 +338,13 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
   }
   // ---- tear-down -----------------------------------------------------------------------------------
   if (warp == 0) DBG(5);
+  if (use_tma && tid == 0 && *s_abort) {
+    // gave up somewhere: do not leave while a bulk load may still be writing this CTA's shared memory
+    for (int nb = 0; nb < nblk_w; ++nb) {
+      bool done = false;
+      for (uint32_t i = 0; i < WAIT_LIMIT && !done; ++i) { done = mbar_try_wait(w_full + nb, 0); if (!done) __nanosleep(100); }
+    }
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) DBG(6);
@@ -320,14 +357,14 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(ScoreArgs a) 
 
 static size_t mma_smem_bytes(const ts_config& c, int TV) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
-  return (size_t)(TV / 64) * rp * 128 + (rp / 64) * 128 * 128 + 512 * 4 + 128 + 512 * 4 + 1024;
+  return (size_t)(TV / 64) * rp * 128 + (rp / 64) * 128 * 128 + 512 * 4 + 128 + 512 * 4 + MAX_BLK * 8 + 1024;
 }
 
 // tile size for the tensor-core path: W tile + A tile + table + barriers within the shared-memory limit,
 // a whole number of waves over the SMs
 bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
-  const size_t fixed = (rp / 64) * 128 * 128 + 512 * 4 + 128 + 512 * 4 + 1024;
+  const size_t fixed = (rp / 64) * 128 * 128 + 512 * 4 + 128 + 512 * 4 + MAX_BLK * 8 + 1024;
   if ((size_t)max_smem < fixed + rp * 128) return false;
   int tv_max = (int)(((size_t)max_smem - fixed) / (rp * 2) / 64) * 64;
   if (tv_max < 64) return false;
@@ -355,9 +392,52 @@ extern "C" int ts_debug_timing(unsigned long long* out) {
 }
 #endif
 
+// Tensor map of W = [r][V] bf16 for boxes of 64 tokens x rp rows with the 128-byte swizzle the MMA's
+// B descriptor expects.  The encoder lives in the driver library; it is looked up through the runtime
+// so that this library has no link-time dependency on the driver.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
+static bool w_tensor_map(ts_ctx* ctx, const void* W) {
+  if (ctx->tma_state < 0) return false;
+  const int rp = (ctx->cfg.r + 63) / 64 * 64;
+  if (rp > 256 || ((uintptr_t)W & 15u) != 0) return false;   // box rows are limited to 256
+  if (ctx->tma_state == 1 && ctx->tmapW_ptr == W) return true;
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+        q != cudaDriverEntryPointSuccess) {
+      (void)cudaGetLastError();
+      ctx->tma_state = -1;
+      return false;
+    }
+    g_encode = (EncodeTiledFn)fn;
+  }
+  const cuuint64_t gdim[2] = {(cuuint64_t)ctx->cfg.V, (cuuint64_t)ctx->cfg.r};
+  const cuuint64_t gstride[1] = {(cuuint64_t)ctx->cfg.V * 2};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)rp};
+  const cuuint32_t estr[2] = {1u, 1u};
+  CUtensorMap tm;
+  const CUresult rc = g_encode(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(W), gdim, gstride, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (rc != CUDA_SUCCESS) { ctx->tma_state = -1; return false; }
+  memcpy(ctx->tmapW, &tm, sizeof(tm));
+  ctx->tmapW_ptr = W;
+  ctx->tma_state = 1;
+  return true;
+}
+
 cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st) {
-  if (a.K <= 8) score_mma_kernel<RegLists<8>><<<a.ntiles, MMA_THREADS, ctx->tile.smem, st>>>(a);
-  else score_mma_kernel<MemLists><<<a.ntiles, MMA_THREADS, ctx->tile.smem, st>>>(a);
+  ts_ctx* c = const_cast<ts_ctx*>(ctx);
+  const int use_tma = w_tensor_map(c, a.W) ? 1 : 0;
+  CUtensorMap tm;
+  memcpy(&tm, c->tmapW, sizeof(tm));
+  if (a.K <= 8) score_mma_kernel<RegLists<8>><<<a.ntiles, MMA_THREADS, ctx->tile.smem, st>>>(a, tm, use_tma);
+  else score_mma_kernel<MemLists><<<a.ntiles, MMA_THREADS, ctx->tile.smem, st>>>(a, tm, use_tma);
   return cudaGetLastError();
 }
 
