@@ -5,6 +5,9 @@
 
 #include "ts_common.cuh"
 
+#ifndef TS_SCAN_MARK
+#define TS_SCAN_MARK(n) do { } while (0)
+#endif
 namespace ts {
 
 // Record layout in 32-bit words: [m, s0, sT, counts, topv[K], topi[K], keyv[K], keyi[K], keyl[K]]
@@ -196,6 +199,7 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
                                            uint64_t seed, int req, uint64_t hash, const float* ghi,
                                            float gL, float gK, const SharedThr& gl, const SharedThr& gk,
                                            const volatile unsigned* liveL = nullptr, const volatile unsigned* liveK = nullptr) {
+  if (valid) TS_SCAN_MARK(0);
   float cm = -INFINITY;
 #pragma unroll
   for (int i = 0; i < CHUNK; ++i) if (i < valid) cm = fmaxf(cm, l[i]);
@@ -217,6 +221,7 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
   }
   st.s0 += a0;
   st.sT += two ? aT : a0;
+  if (valid) TS_SCAN_MARK(1);
   // top-K logits: a token below the launch-wide bound cannot be among the parent's K best
   if (cm > st.thrL && cm >= gL) {
     uint32_t mk = 0;
@@ -235,22 +240,36 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
       }
     }
   }
+  if (valid) TS_SCAN_MARK(2);
   if (T > 0.f) {
     // high half of each token's uniform: one generator call per eight tokens
     const uint4 cw0 = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, (uint32_t)v0 >> 3);
     const uint4 cw1 = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, ((uint32_t)v0 >> 3) + 1u);
     const float thr = fmaxf(st.thrK, gK);
     uint32_t mk = 0;
+    // Four tokens at a time: their best logit plus the noise bound of their largest leading bits bounds
+    // all four keys.  Only when that passes (a few groups per thousand) are the four looked at singly.
 #pragma unroll
-    for (int i = 0; i < CHUNK; ++i) {
-      const uint32_t word = word_of(i < 8 ? cw0 : cw1, (i & 7) >> 1);
-      const uint32_t c16 = (word >> (16 * (i & 1))) & 0xFFFFu;
-      // the leading bits bound the noise from above; almost every token stops here
-      const float bnd = l[i] * invT + ((c16 >> 8) != 255u ? ghi[c16 >> 8] : ghi[256 + (c16 & 255u)]);
-      mk |= (uint32_t)(i < valid && bnd >= thr) << i;
+    for (int sg = 0; sg < 4; ++sg) {
+      const uint4& cw = sg < 2 ? cw0 : cw1;
+      const uint32_t wa = (sg & 1) ? cw.z : cw.x, wb = (sg & 1) ? cw.w : cw.y;
+      const uint32_t m2 = __vmaxu2(wa, wb);
+      const uint32_t c16m = max(m2 & 0xFFFFu, m2 >> 16);
+      const float lm = fmaxf(fmaxf(l[4 * sg], l[4 * sg + 1]), fmaxf(l[4 * sg + 2], l[4 * sg + 3]));
+      const float gb = lm * invT + ((c16m >> 8) != 255u ? ghi[c16m >> 8] : ghi[256 + (c16m & 255u)]);
+      if (4 * sg < valid && gb >= thr) {
+#pragma unroll
+        for (int i = 4 * sg; i < 4 * sg + 4; ++i) {
+          const uint32_t word = word_of(i < 8 ? cw0 : cw1, (i & 7) >> 1);
+          const uint32_t c16 = (word >> (16 * (i & 1))) & 0xFFFFu;
+          const float bnd = l[i] * invT + ((c16 >> 8) != 255u ? ghi[c16 >> 8] : ghi[256 + (c16 & 255u)]);
+          mk |= (uint32_t)(i < valid && bnd >= thr) << i;
+        }
+      }
     }
     uint4 fw = make_uint4(0, 0, 0, 0);
     int fine_call = -1;
+    if (valid) TS_SCAN_MARK(3);
 #pragma unroll 1
     while (mk) {
       const int i = __ffs(mk) - 1;
@@ -272,6 +291,7 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
       }
     }
   }
+  if (valid) TS_SCAN_MARK(4);
 }
 
 // Replication of parents over the 128 rows of a tensor-core tile when a level has few parents:

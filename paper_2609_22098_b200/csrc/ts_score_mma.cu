@@ -16,18 +16,21 @@
 // frees its tensor memory and returns.
 #include <cuda.h>   // CUtensorMap and its enums; the encoder itself is looked up at run time
 #include "ts_internal.h"
-#include "ts_scan.cuh"
-
 namespace ts {
-
 #ifdef TS_DEBUG_TIMING
 // developer aid: per-CTA timestamps (globaltimer ns) of the phases of one launch
 __device__ unsigned long long g_dbg[148 * 64];
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #define DBG(slot) do { if ((threadIdx.x & 31) == 0 && blockIdx.x < 148) g_dbg[blockIdx.x * 64 + (slot)] = gtime(); } while (0)
+#define TS_SCAN_MARK(n) do { if (threadIdx.x == 0 && blockIdx.x < 148 && g_dbg[blockIdx.x * 64 + 56 + (n)] == 0ull) g_dbg[blockIdx.x * 64 + 56 + (n)] = gtime(); } while (0)
 #else
 #define DBG(slot) do { } while (0)
 #endif
+
+}  // namespace ts
+#include "ts_scan.cuh"
+
+namespace ts {
 
 constexpr int EPI_WARPS = 4 * MMA_S;
 constexpr int MMA_THREADS = (EPI_WARPS + 2) * 32;   // epilogue warps, the MMA warp, the bounds-refresh warp
@@ -234,25 +237,37 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       const int pid = ((tile * MMA_S + s) * R + rho) % K;   // which of the parent's K slots this piece feeds
       const SharedThr gl{a.slots + (size_t)pc * K * SLOT_STRIDE, pid};
       const SharedThr gk{a.slots + ((size_t)a.cap + pc) * K * SLOT_STRIDE, pid};
-      for (int nb = 0; nb < nblk; ++nb) {
-        const int it = g * nblk + nb, tb = it % NBUF, u = it / NBUF;
-        int ok = 1;
-        if (lane == 0) ok = mbar_wait(t_full + tb, u & 1, s_abort, a.err) ? 1 : 0;
-        ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-        if (!ok) { alive = false; break; }
-        tc_fence_after();
-        if (nb < 10 && g == 0) DBG(8 + warp * 6 + 0 + (nb >= 1 ? 2 : 0) + (nb >= 8 ? 2 : 0));
-        const int nch = min(8, (tlen - nb * BLK_N + 15) / 16);
+      // Pass nb = -1 is a dry run of the scan on an empty chunk while the first MMAs are still on their
+      // way: it changes nothing in `st`, but it brings the scan's instructions into the instruction cache
+      // and requests the base logits of the first chunk this warp owns.
+      for (int nb = -1; nb < nblk; ++nb) {
+        const bool dry = nb < 0;
+        const int it = g * nblk + (dry ? 0 : nb), tb = it % NBUF, u = it / NBUF;
+        if (!dry) {
+          int ok = 1;
+          if (lane == 0) ok = mbar_wait(t_full + tb, u & 1, s_abort, a.err) ? 1 : 0;
+          ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+          if (!ok) { alive = false; break; }
+          tc_fence_after();
+          if (nb < 10 && g == 0) DBG(8 + warp * 6 + 0 + (nb >= 1 ? 2 : 0) + (nb >= 8 ? 2 : 0));
+        }
+        const int nch = dry ? 1 : min(8, (tlen - nb * BLK_N + 15) / 16);
         for (int c = 0; c < nch; ++c) {
-          const int cg = nb * 8 + c;
-          if (cg % R != rho || (cg / R) % MMA_S != s) continue;   // warp-uniform
+          // owned chunks: cg = rho + R * (s + MMA_S * j); the dry pass sits one step before the first
+          const int cg = dry ? rho + R * s - R * MMA_S : nb * 8 + c;
+          if (!dry && (cg % R != rho || (cg / R) % MMA_S != s)) continue;   // warp-uniform
           float acc[16];
-          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * BLK_N + c * 16), acc);
+          if (!dry) {
+            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * BLK_N + c * 16), acc);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+          }
           if (active) {
-            const int v0 = t0 + cg * 16;
-            const int valid = min(16, V - v0);   // 8 or 16: V and v0 are multiples of 8
+            const int v0 = dry ? t0 : t0 + cg * 16;
+            const int valid = dry ? 0 : min(16, V - v0);   // 8 or 16: V and v0 are multiples of 8
             // this chunk's base logits were requested one chunk ago; request the next owned chunk's now
-            const uint4 u0 = have_next ? nx0 : __ldg(reinterpret_cast<const uint4*>(Urow + v0));
+            const uint4 u0 = have_next ? nx0 : (dry ? make_uint4(0, 0, 0, 0) : __ldg(reinterpret_cast<const uint4*>(Urow + v0)));
             const uint4 u1 = have_next ? nx1 : (valid > 8 ? __ldg(reinterpret_cast<const uint4*>(Urow + v0 + 8)) : make_uint4(0, 0, 0, 0));
             {
               const int cgn = cg + R * MMA_S;           // the next chunk this warp owns
@@ -263,15 +278,16 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
                 nx1 = (V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8)) : make_uint4(0, 0, 0, 0);
               }
             }
-            const float gLc = dec_f(s_thr[prow]), gKc = dec_f(s_thr[128 + prow]);   // kept fresh by the refresh warp
             float ub[16];
             unpack_bf16x8(u0, ub);
             unpack_bf16x8(u1, ub + 8);
 #pragma unroll
             for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] + ub[i] : 0.f;
+            const float gLc = dec_f(s_thr[prow]), gKc = dec_f(s_thr[128 + prow]);   // kept fresh by the refresh warp
             scan_chunk(st, acc, v0, valid, T, invT, a.seed, req, hash, ghi, gLc, gKc, gl, gk, s_thr + prow, s_thr + 128 + prow);
           }
         }
+        if (dry) continue;
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(t_empty + tb);
@@ -297,11 +313,16 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
           if (p >= P) continue;
           const unsigned* sl = a.slots + (size_t)p * K * SLOT_STRIDE;
           const unsigned* sk = a.slots + ((size_t)a.cap + p) * K * SLOT_STRIDE;
-          unsigned mL = __ldcg(sl), mK = __ldcg(sk);
-          for (int j = 1; j < K; ++j) {
-            mL = min(mL, __ldcg(sl + j * SLOT_STRIDE));
-            mK = min(mK, __ldcg(sk + j * SLOT_STRIDE));
+          // all 2K loads in flight together: one L2 round trip per row, not one per slot
+          unsigned vL[KMAX], vK[KMAX];
+#pragma unroll
+          for (int j = 0; j < KMAX; ++j) {
+            vL[j] = j < K ? __ldcg(sl + j * SLOT_STRIDE) : 0xFFFFFFFFu;
+            vK[j] = j < K ? __ldcg(sk + j * SLOT_STRIDE) : 0xFFFFFFFFu;
           }
+          unsigned mL = vL[0], mK = vK[0];
+#pragma unroll
+          for (int j = 1; j < KMAX; ++j) { mL = min(mL, vL[j]); mK = min(mK, vK[j]); }
           s_thr[(g & 1) * 256 + rr] = mL; s_thr[(g & 1) * 256 + 128 + rr] = mK;
         }
         __nanosleep(1000);
@@ -388,7 +409,10 @@ cudaError_t score_mma_setup(ts_ctx* ctx) {
 
 #ifdef TS_DEBUG_TIMING
 extern "C" int ts_debug_timing(unsigned long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, g_dbg, sizeof(g_dbg));
+  const int rc = (int)cudaMemcpyFromSymbol(out, g_dbg, sizeof(g_dbg));
+  static unsigned long long zeros[148 * 64];
+  cudaMemcpyToSymbol(g_dbg, zeros, sizeof(zeros));
+  return rc;
 }
 #endif
 
