@@ -48,6 +48,8 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
 bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out);
 cudaError_t score_mma_setup(ts_ctx* ctx);
 cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st);
+// encodes (or finds cached in the context) the tensor map of W for 64-token boxes; false: not available
+bool w_tensor_map(ts_ctx* ctx, const void* W);
 
 enum KernelId { K_INIT, K_SCORE, K_MERGE, K_LEVEL, K_FINAL, K_ZROWS, K_GREEDY, K_WALK, K_CHECK, K_COUNT };
 

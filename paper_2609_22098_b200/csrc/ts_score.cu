@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
 // Every thread folds its share of the pieces into a private (max, sums) pair and private top-K
 // lists; the block then takes K rounds of arg-max over the list heads (value desc, token asc).
 // ------------------------------------------------------------------------------------------------
-constexpr int MERGE_THREADS = 256;
+constexpr int MERGE_THREADS = 512;
 constexpr int MERGE_WARPS = MERGE_THREADS / 32;
 
 __device__ __forceinline__ bool better(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
@@ -160,25 +160,17 @@ __device__ void block_select(MList<KR>& mine, int K, int* out_tok, float* out_va
 
 constexpr int MERGE_CAP = 768;   // candidates per list the fast path can hold
 
-// K rounds of warp-wide arg-max over a candidate array in shared memory (value desc, token asc)
-__device__ void warp_select(float* cv, int* ci, float* cl, int n, int K, int lane, int* out_tok, float* out_val) {
-  for (int j = 0; j < K; ++j) {
-    float bv = -INFINITY; int bi = 0x7FFFFFFF, bp = -1; float bl = 0.f;
-    for (int e = lane; e < n; e += 32) {
-      const int idx = ci[e];
-      if (idx != 0x7FFFFFFF && better(cv[e], idx, bv, bi)) { bv = cv[e]; bi = idx; bp = e; bl = cl[e]; }
-    }
-    float wv = bv; int wi = bi; float wl = bl;
-    for (int off = 16; off > 0; off >>= 1) {
-      const float ov = __shfl_xor_sync(0xFFFFFFFFu, wv, off);
-      const int oi = __shfl_xor_sync(0xFFFFFFFFu, wi, off);
-      const float ol = __shfl_xor_sync(0xFFFFFFFFu, wl, off);
-      if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; wl = ol; }
-    }
-    if (bp >= 0 && bi == wi) ci[bp] = 0x7FFFFFFF;   // taken (tokens are unique per list)
-    __syncwarp();
-    if (lane == 0) { out_tok[j] = wi == 0x7FFFFFFF ? -1 : wi; out_val[j] = wi == 0x7FFFFFFF ? 0.f : wl; }
+// The K best of a candidate array in shared memory (value desc, token asc), by counting: a candidate's
+// place is the number of candidates that beat it (tokens are unique per list, so places are too).  With
+// tight bounds a few dozen candidates arrive here, and the whole selection is one short pass.
+__device__ void rank_select(const float* cv, const int* ci, const float* cl, int n, int K, int t, int nt, int* out_tok, float* out_val) {
+  for (int e = t; e < n; e += nt) {
+    const float v = cv[e]; const int idx = ci[e];
+    int rank = 0;
+    for (int f = 0; f < n; ++f) rank += better(cv[f], ci[f], v, idx) ? 1 : 0;
+    if (rank < K) { out_tok[rank] = idx; out_val[rank] = cl[e]; }
   }
+  for (int j = n + t; j < K; j += nt) { out_tok[j] = -1; out_val[j] = 0.f; }
 }
 
 template <int KR>
@@ -200,11 +192,19 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
     if (tid < 2) c_n[tid] = 0;
     __syncthreads();
     float m = -INFINITY, s0 = 0.f, sT = 0.f;
-    for (int q = tid; q < npieces; q += MERGE_THREADS) {
+    auto rec_of = [&](int q) {
       const int ts_ = q / R, rho = q % R;
       const int slot = R > 1 ? rho * (128 / R) + p : p;
-      const float* rec = a.rec + ((size_t)ts_ * a.cap + slot) * rw;
-      const float4 h = __ldcg(reinterpret_cast<const float4*>(rec));
+      return a.rec + ((size_t)ts_ * a.cap + slot) * rw;
+    };
+    // the header of the next record is requested before this one's entries, so that a thread with
+    // several records pays one memory round trip per record, not two
+    float4 hn = make_float4(-INFINITY, 0.f, 0.f, 0.f);
+    if (tid < npieces) hn = __ldcg(reinterpret_cast<const float4*>(rec_of(tid)));
+    for (int q = tid; q < npieces; q += MERGE_THREADS) {
+      const float* rec = rec_of(q);
+      const float4 h = hn;
+      if (q + MERGE_THREADS < npieces) hn = __ldcg(reinterpret_cast<const float4*>(rec_of(q + MERGE_THREADS)));
       const float* f = rec + 4; const int* ii = reinterpret_cast<const int*>(rec) + 4;
       // all entries of the record are requested at once (independent loads), then filtered
       float tv[KR], kv[KR], kl[KR]; int ti[KR], ki[KR];
@@ -262,10 +262,11 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
 #endif
     const bool fits = c_n[0] <= MERGE_CAP && c_n[1] <= MERGE_CAP;   // uniform: read after the barrier above
     if (fits) {
-      // the usual case: a few dozen candidates survive the bounds; one warp per list picks the K best
-      if (warp == 0) warp_select(c_v[0], c_i[0], c_l[0], c_n[0], K, lane, a.top_tok + (size_t)p * K, a.top_logit + (size_t)p * K);
-      if (warp == 1 && a.T > 0.f)
-        warp_select(c_v[1], c_i[1], c_l[1], c_n[1], K, lane, a.draw_tok + (size_t)p * K, a.draw_logit + (size_t)p * K);
+      // the usual case: a few dozen candidates survive the bounds; half of the block ranks each list
+      const int half = tid / (MERGE_THREADS / 2), t = tid % (MERGE_THREADS / 2);
+      if (half == 0) rank_select(c_v[0], c_i[0], c_l[0], c_n[0], K, t, MERGE_THREADS / 2, a.top_tok + (size_t)p * K, a.top_logit + (size_t)p * K);
+      else if (a.T > 0.f)
+        rank_select(c_v[1], c_i[1], c_l[1], c_n[1], K, t, MERGE_THREADS / 2, a.draw_tok + (size_t)p * K, a.draw_logit + (size_t)p * K);
       __syncthreads();
     } else {
       // too many candidates for the shared arrays (bounds not formed, e.g. tiny vocabularies): every

@@ -14,7 +14,7 @@
 // "full" barrier; epilogue warps arrive on its "empty" barrier when they have drained it.
 // Every wait is bounded: when one runs out the kernel raises an error word, skips the remaining work,
 // frees its tensor memory and returns.
-#include <cuda.h>   // CUtensorMap and its enums; the encoder itself is looked up at run time
+#include "ts_tc.cuh"
 #include "ts_internal.h"
 namespace ts {
 #ifdef TS_DEBUG_TIMING
@@ -37,81 +37,7 @@ constexpr int MMA_THREADS = (EPI_WARPS + 2) * 32;   // epilogue warps, the MMA w
 constexpr int BLK_N = 128;
 constexpr int NBUF = 4;                 // accumulator buffers of BLK_N columns in tensor memory
 constexpr uint32_t TMEM_COLS = NBUF * BLK_N;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int MAX_BLK = 32;             // blocks of BLK_N tokens in the largest tile (4096 tokens)
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// bounded wait; false = gave up (and said so in *abort / *err)
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int* err) {
-  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*abort) return false;
-    if (i > 8) __nanosleep(100);
-  }
-  *abort = 1;
-  if (err) atomicExch(err, 1);
-  return false;
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-// one box of the W tensor map (64 tokens x rp rows, 128-byte swizzle) into shared memory; completion
-// is counted in bytes on `bar`.  c0 (the token coordinate) must be a multiple of 8.
-__device__ __forceinline__ void tma_load_box(void* dst, const CUtensorMap* tm, int c0, int c1, uint64_t* bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-               ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
-}
-
-// shared-memory matrix descriptor: 128-byte swizzle, descriptor version 1 (sm_100)
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
-         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
-}
-// instruction descriptor: D = f32, A = B = bf16, A K-major, B MN-major, M = 128, N = n
-__device__ __forceinline__ uint32_t instr_desc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
-}
-__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
-  uint32_t r[16];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr) : "memory");
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
 
 template <class Lists>
 __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma) {
@@ -190,7 +116,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   const uint32_t tmem_base = *s_tmem;
   if (warp == 0) DBG(3);
 
-  const int R = mma_replicas(P);
+  const int R = mma_replicas(P), rsh = R == 4 ? 2 : (R == 2 ? 1 : 0);
   const int ngroups = R > 1 ? 1 : (P + 127) / 128;
   const int nblk = (tlen + BLK_N - 1) / BLK_N;
   const float T = a.T, invT = T > 0.f ? 1.f / T : 1.f;
@@ -255,7 +181,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
         for (int c = 0; c < nch; ++c) {
           // owned chunks: cg = rho + R * (s + MMA_S * j); the dry pass sits one step before the first
           const int cg = dry ? rho + R * s - R * MMA_S : nb * 8 + c;
-          if (!dry && (cg % R != rho || (cg / R) % MMA_S != s)) continue;   // warp-uniform
+          if (!dry && ((cg & (R - 1)) != rho || ((cg >> rsh) % MMA_S) != s)) continue;   // warp-uniform; R is 1, 2 or 4
           float acc[16];
           if (!dry) {
             tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * BLK_N + c * 16), acc);
@@ -424,7 +350,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 static EncodeTiledFn g_encode = nullptr;
 
-static bool w_tensor_map(ts_ctx* ctx, const void* W) {
+bool w_tensor_map(ts_ctx* ctx, const void* W) {
   if (ctx->tma_state < 0) return false;
   const int rp = (ctx->cfg.r + 63) / 64 * 64;
   if (rp > 256 || ((uintptr_t)W & 15u) != 0) return false;   // box rows are limited to 256

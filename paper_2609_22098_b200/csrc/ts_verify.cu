@@ -16,6 +16,8 @@
 #include <math.h>
 
 #include "ts_internal.h"
+#include "ts_scan.cuh"
+#include "ts_tc.cuh"
 
 namespace ts {
 
@@ -27,8 +29,14 @@ extern "C" int ts_debug_timing_walk(unsigned long long* out) { return (int)cudaM
 #else
 #define DBGW(step, slot) do { } while (0)
 #endif
+#ifdef TS_DEBUG_TIMING
+__device__ unsigned long long g_dbgp[64];
+#define DBGP(slot) do { if (blockIdx.x == 0 && (slot) < 64) g_dbgp[slot] = gtimew(); } while (0)
+extern "C" int ts_debug_timing_pass(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_dbgp, sizeof(g_dbgp)); }
+#else
+#define DBGP(slot) do { } while (0)
+#endif
 
-constexpr int VT = 256;  // threads of the verification kernels
 constexpr int ZT = 512;  // threads per target row in the row-statistics kernel
 
 // ------------------------------------------------------------------------------------------------
@@ -402,19 +410,204 @@ __device__ __forceinline__ void sweep_item(const SweepCtx<TIn>& c, int g0, int c
 
 
 constexpr int SB = 32; // requests whose head rows are staged together
+constexpr int WT = 288;       // threads of the walk kernel: eight worker warps and the warp that issues the MMAs
+constexpr int WALK_EPI = 8;   // worker warps that read the accumulators of a tensor-core reduction
+constexpr int WALK_NBUF = 4;  // accumulator buffers of 128 columns in tensor memory
+constexpr int WALK_MAX_BLK = 32;
+
+// Tensor-core state of one walk CTA: shared-memory operands, barriers, tensor-memory base and the running
+// count of 128-token blocks issued so far (it selects the accumulator buffer and the barrier parity).
+struct WalkTc {
+  unsigned char* Ws; unsigned char* As; uint64_t* t_full; uint64_t* t_empty; volatile int* s_abort;
+  uint32_t tmem_base, slab_bytes; int rp; uint32_t it;
+};
+
+// One reduction step on the tensor cores: sum over this CTA's tokens [t0, t0 + tlen) of
+// max(p(w) - C q(w), 0) for up to 128 requests at once.  The low-rank part of the draft logits,
+// [requests x r] . [r x tokens], is one MMA tile per 128 tokens (requests on the rows, replicated when
+// there are few); worker warp w reads the rows of quarter w % 4 and the 16-token chunks of column split
+// w / 4, adds the base logits, and accumulates the residual with the target row.  Partial sums are
+// combined in a fixed order.  Returns false when a bounded wait ran out.
+__device__ __forceinline__ float fast_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 
 template <typename TIn>
-__global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
+__device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int tlen, float invT,
+                         const int* sb_req, const int* sb_dep, const int* sb_tok, const long long* sb_row,
+                         const float* sb_C, const float* sb_zmax, const float* sb_zlogs, const float* sb_lseT, float* s_part) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int r = a.r, rp = tc.rp, V = a.V;
+  const int R = mma_replicas(nreq), per = 128 / R, rsh = R == 4 ? 2 : (R == 2 ? 1 : 0), psh = 7 - rsh;
+  const int cpr = rp / 8;                      // 16-byte chunks per A row
+  const uint32_t a_slab_bytes = 128u * 128u;
+  const __nv_bfloat16* Ag = reinterpret_cast<const __nv_bfloat16*>(a.A);
+  if (tid == 0) DBGP(0);
+  {
+    // ask L2 for this CTA's share of every request's target row and base-logit row now; the worker warps
+    // come for them a few microseconds later, after the MMAs
+    const int lines = (tlen * 2 + 127) / 128;
+    const __nv_bfloat16* Zg = reinterpret_cast<const __nv_bfloat16*>(a.Z);
+    const __nv_bfloat16* Ug = reinterpret_cast<const __nv_bfloat16*>(a.U);
+    for (int i = tid; i < nreq * lines * 2; i += WT) {
+      const int g = i / (lines * 2), rem = i % (lines * 2), which = rem / lines, ln = rem % lines;
+      const __nv_bfloat16* base = which == 0 ? Zg + (size_t)sb_row[g] * V : Ug + ((size_t)sb_req[g] * a.D + sb_dep[g]) * V;
+      if (which == 0 || sb_C[g] != 0.f) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + t0 + ln * 64));
+    }
+  }
+  // head rows A[x] of the requests' current nodes, K-major with the 128-byte swizzle
+  for (int idx = tid; idx < 128 * cpr; idx += WT) {
+    const int rr = idx / cpr, ck = idx % cpr;
+    const int g = rr % per;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (g < nreq && ck * 8 < r) v = __ldg(reinterpret_cast<const uint4*>(Ag + (size_t)sb_tok[g] * r + ck * 8));
+    *reinterpret_cast<uint4*>(tc.As + (size_t)(ck >> 3) * a_slab_bytes + rr * 128 + (((ck & 7) ^ (rr & 7)) << 4)) = v;
+  }
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const int nblk = (tlen + 127) / 128;
+  if (tid == 0) DBGP(1);
+  if (warp < WALK_EPI) {
+    const int q = warp & 3, s = warp >> 2;
+    const int row = q * 32 + lane;
+    const int g = row & (per - 1), rho = row >> psh;   // rho is uniform within a warp
+    const bool active = g < nreq;
+    const __nv_bfloat16* Zrow = reinterpret_cast<const __nv_bfloat16*>(a.Z);
+    const __nv_bfloat16* Urow = reinterpret_cast<const __nv_bfloat16*>(a.U);
+    float C = 0.f, zs = 0.f, zoff = 0.f, qoff = 0.f;
+    if (active) {
+      Zrow += (size_t)sb_row[g] * V;
+      Urow += ((size_t)sb_req[g] * a.D + sb_dep[g]) * V;
+      C = sb_C[g];
+      zs = invT * 1.4426950408889634f;                         // exponentials as powers of two
+      zoff = (-sb_zmax[g] * invT - sb_zlogs[g]) * 1.4426950408889634f;
+      qoff = C != 0.f ? -sb_lseT[g] * 1.4426950408889634f : -1e30f;   // lseT may be NaN where it is not needed
+    }
+    float sum = 0.f;
+    bool alive = true;
+    const bool need_q = C != 0.f;
+    // the rows of the next owned chunk are requested while this one is worked on
+    uint4 nz0 = make_uint4(0, 0, 0, 0), nz1 = nz0, nu0 = nz0, nu1 = nz0;
+    {
+      const int cg0 = rho + R * s;           // owned chunks: cg = rho + R * (s + 2 j)
+      const int vn = t0 + cg0 * 16;
+      if (active && cg0 * 16 < tlen) {
+        nz0 = __ldg(reinterpret_cast<const uint4*>(Zrow + vn));
+        if (V - vn > 8) nz1 = __ldg(reinterpret_cast<const uint4*>(Zrow + vn + 8));
+        if (need_q) {
+          nu0 = __ldg(reinterpret_cast<const uint4*>(Urow + vn));
+          if (V - vn > 8) nu1 = __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8));
+        }
+      }
+    }
+    for (int nb = 0; nb < nblk && alive; ++nb) {
+      const uint32_t it = tc.it + (uint32_t)nb, tb = it % WALK_NBUF, u = it / WALK_NBUF;
+      int ok = 1;
+      if (lane == 0) ok = mbar_wait(tc.t_full + tb, u & 1, tc.s_abort, nullptr) ? 1 : 0;
+      ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+      if (!ok) { alive = false; break; }
+      tc_fence_after();
+      if (tid == 0) DBGP(4 + 2 * nb);
+      const int nch = min(8, (tlen - nb * 128 + 15) / 16);
+      for (int c = 0; c < nch; ++c) {
+        const int cg = nb * 8 + c;
+        if ((cg & (R - 1)) != rho || ((cg >> rsh) & 1) != s) continue;   // warp-uniform; R is 1, 2 or 4
+        float acc[16];
+        if (tid == 0 && nb == 4) DBGP(40);
+        tmem_ld16(tc.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * 128 + c * 16), acc);
+        if (tid == 0 && nb == 4) DBGP(41);
+        if (active) {
+          const int v0 = t0 + cg * 16;
+          const int valid = min(16, V - v0);   // 8 or 16: V and v0 are multiples of 8
+          const uint4 z0 = nz0, z1 = nz1, u0 = nu0, u1 = nu1;
+          {
+            const int cgn = cg + R * 2;
+            const int vn = t0 + cgn * 16;
+            if (cgn * 16 < tlen) {
+              nz0 = __ldg(reinterpret_cast<const uint4*>(Zrow + vn));
+              nz1 = (V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Zrow + vn + 8)) : make_uint4(0, 0, 0, 0);
+              if (need_q) {
+                nu0 = __ldg(reinterpret_cast<const uint4*>(Urow + vn));
+                nu1 = (V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8)) : make_uint4(0, 0, 0, 0);
+              }
+            }
+          }
+          if (tid == 0 && nb == 4) DBGP(42);
+          float zz[16];
+          unpack_bf16x8(z0, zz);
+          unpack_bf16x8(z1, zz + 8);
+          if (tid == 0 && nb == 4) DBGP(43);
+          // one path for every lane: a request with C == 0 has qoff = -huge, so its q term vanishes
+          float ub[16];
+          unpack_bf16x8(u0, ub);
+          unpack_bf16x8(u1, ub + 8);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float p = fast_ex2(fmaf(zz[i], zs, zoff));
+            const float qq = fast_ex2(fmaf(acc[i] + ub[i], zs, qoff));
+            if (i < valid) sum += fmaxf(fmaf(-C, qq, p), 0.f);
+          }
+          if (tid == 0 && nb == 4) DBGP(44);
+        }
+      }
+      if (tid == 0 && nb == 4) DBGP(45);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tc.t_empty + tb);
+      if (tid == 0) DBGP(5 + 2 * nb);
+    }
+    s_part[row * 2 + s] = active ? sum : 0.f;
+  } else if (warp == WALK_EPI && lane == 0) {
+    const uint32_t ws_addr = smem_u32(tc.Ws), as_addr = smem_u32(tc.As);
+    for (int nb = 0; nb < nblk; ++nb) {
+      const uint32_t it = tc.it + (uint32_t)nb, tb = it % WALK_NBUF, u = it / WALK_NBUF;
+      if (u >= 1) {
+        if (!mbar_wait(tc.t_empty + tb, (u - 1) & 1, tc.s_abort, nullptr)) break;
+        tc_fence_after();
+      }
+      const int n = (tlen - nb * 128 > 64) ? 128 : 64;
+      const uint32_t idesc = instr_desc(n);
+      const uint32_t d_tmem = tc.tmem_base + tb * 128u;
+      for (int ks = 0; ks < rp / 16; ++ks) {
+        const uint64_t adesc = smem_desc(as_addr + (uint32_t)(ks >> 2) * a_slab_bytes + (uint32_t)(ks & 3) * 32u, 16u, 1024u);
+        const uint64_t bdesc = smem_desc(ws_addr + (uint32_t)(2 * nb) * tc.slab_bytes + (uint32_t)ks * 2048u, tc.slab_bytes, 1024u);
+        mma_bf16(d_tmem, adesc, bdesc, idesc, ks > 0 ? 1u : 0u);
+      }
+      mma_commit(tc.t_full + tb);
+      DBGP(30 + nb);
+    }
+  }
+  tc.it += (uint32_t)nblk;
+  if (tid == 0) DBGP(2);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (*tc.s_abort) return false;
+  if (tid < nreq) {
+    float t = 0.f;
+    for (int rho = 0; rho < R; ++rho) { t += s_part[(rho * per + tid) * 2]; t += s_part[(rho * per + tid) * 2 + 1]; }
+    a.part[(size_t)sb_req[tid] * a.vt_n + blockIdx.x] = t;
+  }
+  __syncthreads();
+  if (tid == 0) DBGP(3);
+  return true;
+}
+
+
+// The walk proper.  Returns false when a bounded wait ran out (every thread of the CTA returns the same).
+template <typename TIn, bool MMA>
+__device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsigned char* w_raw) {
+  constexpr int SBX = MMA ? 128 : SB;   // requests per reduction pass
   __shared__ float s_a[VG * 128];
   __shared__ int s_req[VG], s_dep[VG], s_node[VG];
   __shared__ float s_C[VG], s_zmax[VG], s_zlogs[VG], s_lseT[VG];
-  __shared__ float s_red[VG][VT / 32];
-  __shared__ double s_scan[VT];
+  __shared__ float s_red[VG][WT / 32];
+  __shared__ double s_scan[WT];
   __shared__ int s_found, s_last;
-  __shared__ float sb_a[SB * 128];
-  __shared__ int sb_req[SB], sb_dep[SB], sb_tok[SB];
-  __shared__ long long sb_row[SB];
-  __shared__ float sb_C[SB], sb_zmax[SB], sb_zlogs[SB], sb_lseT[SB], sb_part[SB * 16];
+  __shared__ float sb_a[MMA ? 256 : SB * 128];
+  __shared__ int sb_req[SBX], sb_dep[SBX], sb_tok[SBX];
+  __shared__ long long sb_row[SBX];
+  __shared__ float sb_C[SBX], sb_zmax[SBX], sb_zlogs[SBX], sb_lseT[SBX], sb_part[MMA ? 256 : SB * 16];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned nblocks = gridDim.x;
   unsigned gen = 0;
@@ -426,18 +619,17 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
   const TIn* Ag = reinterpret_cast<const TIn*>(a.A);
   const TIn* Wg = reinterpret_cast<const TIn*>(a.W);
   const int N = a.N;
-  extern __shared__ __align__(16) unsigned char w_raw[];
   TIn* Ws = reinterpret_cast<TIn*>(w_raw);   // [r][vt_TV] when a.w_smem
-  if (a.w_smem && vec_ok) {
+  if (!MMA && a.w_smem && vec_ok) {
     const int per_row = a.vt_TV / VEC;
-    for (int i = tid; i < a.r * per_row; i += VT) {
+    for (int i = tid; i < a.r * per_row; i += WT) {
       const int k = i / per_row, c = (i % per_row) * VEC;
       uint4 x = make_uint4(0, 0, 0, 0);
       if (v_lo + c < a.V) x = __ldg(reinterpret_cast<const uint4*>(Wg + (size_t)k * a.V + v_lo + c));
       *reinterpret_cast<uint4*>(Ws + (size_t)k * a.vt_TV + c) = x;
     }
   }
-  const bool ws_ok = a.w_smem && vec_ok;
+  const bool ws_ok = !MMA && a.w_smem && vec_ok;
 
   // ---- per-edge statistics, child ranges and state initialisation (owner CTA of each request) ------
   if (blockIdx.x == 0 && tid < 5) a.ctr[tid] = tid == 4 ? a.B : 0;
@@ -446,10 +638,10 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
     const bool okn = n >= 0 && n <= N;
     const size_t nb = (size_t)b * N, cbase = (size_t)b * (N + 1);
     const int64_t row0 = a.z_row_off[b];
-    for (int i = tid; i <= N; i += VT) { a.child_first[cbase + i] = -1; a.child_cnt[cbase + i] = 0; }
+    for (int i = tid; i <= N; i += WT) { a.child_first[cbase + i] = -1; a.child_cnt[cbase + i] = 0; }
     __syncthreads();
     if (okn)
-      for (int i = tid; i < n; i += VT) {
+      for (int i = tid; i < n; i += WT) {
         const int par = a.parent[nb + i];
         if (i == 0 || a.parent[nb + i - 1] != par) a.child_first[cbase + par + 1] = i;   // siblings are contiguous
         atomicAdd(&a.child_cnt[cbase + par + 1], 1);
@@ -473,7 +665,7 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
     __syncthreads();
   }
   __threadfence();
-  if (!grid_barrier(a.barrier, nblocks, gen)) return;
+  if (!grid_barrier(a.barrier, nblocks, gen)) return false;
   // requests rejected at set-up leave the count of unfinished ones
   for (int b = blockIdx.x; b < a.B; b += nblocks)
     if (tid == 0 && a.state[b].need == 3) atomicSub(a.ctr + 4, 1);
@@ -482,14 +674,34 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
     const int par = step & 1;
     DBGW(step, 0);
     // ---- phase A: scalar walks of the requests this CTA owns, one warp each ----------------------
-    for (int b = blockIdx.x + warp * (int)nblocks; b < a.B; b += (VT / 32) * (int)nblocks) advance<TIn>(a, b, lane, par);
+    for (int b = blockIdx.x + warp * (int)nblocks; b < a.B; b += (WT / 32) * (int)nblocks) advance<TIn>(a, b, lane, par);
     DBGW(step, 1);
-    if (!grid_barrier(a.barrier, nblocks, gen)) return;
+    if (!grid_barrier(a.barrier, nblocks, gen)) return false;
     DBGW(step, 2);
     // ---- phase B: vocabulary work requested by the walks -----------------------------------------
     const int nwk = __ldcg(a.ctr + par), nsc = __ldcg(a.ctr + 2 + par), left = __ldcg(a.ctr + 4);
     if (blockIdx.x == 0 && tid < 2) a.ctr[2 * tid + (par ^ 1)] = 0;   // next step's counters
-    if (vec_ok) {
+    if (MMA) {
+      for (int sb0 = 0; sb0 < nwk; sb0 += SBX) {
+        const int nreq = min(SBX, nwk - sb0);
+        if (tid < nreq) {
+          const int b = __ldcg(a.wk_list + par * a.B + sb0 + tid);
+          const VerifyState* st = a.state + b;
+          const int v = st->row_node;
+          const int64_t row = a.z_row_off[b] + v + 1;
+          sb_req[tid] = b; sb_row[tid] = row; sb_dep[tid] = v < 0 ? 0 : a.depth[(size_t)b * N + v];
+          sb_tok[tid] = v < 0 ? a.anchor[b] : a.tok[(size_t)b * N + v];
+          sb_C[tid] = (float)st->passC; sb_zmax[tid] = a.z_max[row]; sb_zlogs[tid] = a.z_logs[row];
+          sb_lseT[tid] = a.node_lseT[(size_t)b * (N + 1) + v + 1];
+        }
+        __syncthreads();
+        if (!mma_pass<TIn>(a, tc, nreq, v_lo, v_hi - v_lo, invT, sb_req, sb_dep, sb_tok, sb_row, sb_C, sb_zmax, sb_zlogs,
+                           sb_lseT, sb_part)) {
+          if (tid == 0) atomicExch(a.barrier + 1, 1u);   // the word the follow-up kernel checks
+          return false;
+        }
+      }
+    } else if (vec_ok) {
       // Reductions sum_w max(p(w) - C q(w), 0) over this CTA's vocabulary range, for up to SB requests
       // at a time.  Work item = (group of VG requests, chunk of the range); items are dealt to the warps,
       // so a single request still uses several warps and many requests run side by side.  Partial sums
@@ -510,13 +722,13 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
           sb_lseT[tid] = a.node_lseT[(size_t)b * (N + 1) + v + 1];
         }
         __syncthreads();
-        for (int i = tid; i < nreq * a.r; i += VT) {
+        for (int i = tid; i < nreq * a.r; i += WT) {
           const int g = i / a.r, k = i % a.r;
           sb_a[g * 128 + k] = Elem<TIn>::to_f(Ag[(size_t)sb_tok[g] * a.r + k]);
         }
         __syncthreads();
         const int ngrp = (nreq + VG - 1) / VG;
-        for (int item = warp; item < ngrp * nchunk; item += VT / 32) {
+        for (int item = warp; item < ngrp * nchunk; item += WT / 32) {
           const int grp = item / nchunk, ch = item % nchunk;
           const int g0 = grp * VG, ng = min(VG, nreq - g0);
           const int c_lo = v_lo + ch * chunk, c_hi = min(v_hi, c_lo + chunk);
@@ -551,7 +763,7 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
         s_lseT[tid] = a.node_lseT[(size_t)b * (N + 1) + v + 1];
       }
       __syncthreads();
-      for (int i = tid; i < ng * a.r; i += VT) {
+      for (int i = tid; i < ng * a.r; i += WT) {
         const int g = i / a.r, k = i % a.r;
         const int v = s_node[g];
         const int ptok = v < 0 ? a.anchor[s_req[g]] : a.tok[(size_t)s_req[g] * N + v];
@@ -564,7 +776,7 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
       bool need_q = false;
       for (int g = 0; g < ng; ++g) need_q |= (s_C[g] != 0.f);
       if (vec_ok) {
-        for (int v = v_lo + tid * VEC; v < v_hi; v += VT * VEC) {
+        for (int v = v_lo + tid * VEC; v < v_hi; v += WT * VEC) {
           float acc[VG][8];
           if (need_q) logits_group<TIn, VG>(a, s_a, ng, s_req, s_dep, v, acc, ws_ok ? Ws : Wg,
                                             ws_ok ? (size_t)a.vt_TV : (size_t)a.V, ws_ok ? v - v_lo : v);
@@ -585,7 +797,7 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
           }
         }
       } else {
-        for (int v = v_lo + tid; v < v_hi; v += VT) {
+        for (int v = v_lo + tid; v < v_hi; v += WT) {
           for (int g = 0; g < ng; ++g) {
             const int b = s_req[g];
             const int64_t row = a.z_row_off[b] + s_node[g] + 1;
@@ -608,7 +820,7 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
       __syncthreads();
       if (tid < ng) {
         float t = 0.f;
-        for (int w = 0; w < VT / 32; ++w) t += s_red[tid][w];
+        for (int w = 0; w < WT / 32; ++w) t += s_red[tid][w];
         a.part[(size_t)s_req[tid] * a.vt_n + blockIdx.x] = t;
       }
       __syncthreads();
@@ -616,7 +828,7 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
     DBGW(step, 3);
     // range rescans for bonus tokens that fall into this CTA's range: the residual of every token of
     // the range is evaluated once (tokens dealt round-robin to the threads: row i of the range holds
-    // tokens i*VT .. i*VT+VT-1), then prefix sums in token order locate the crossing
+    // tokens i*WT .. i*WT+WT-1), then prefix sums in token order locate the crossing
     for (int si = 0; si < nsc; ++si) {
       const int b = __ldcg(a.sc_list + par * a.B + si);
       const VerifyState& st = a.state[b];
@@ -630,14 +842,14 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
       const double lseT = C != 0.0 ? (double)a.node_lseT[(size_t)b * (N + 1) + v + 1] : 0.0;
       const int nf = st.nf;
       const double want = st.before >= 0.0 ? st.target - st.before : 1e300;
-      for (int k = tid; k < a.r; k += VT) sb_a[k] = Elem<TIn>::to_f(Ag[(size_t)ptok * a.r + k]);
+      for (int k = tid; k < a.r; k += WT) sb_a[k] = Elem<TIn>::to_f(Ag[(size_t)ptok * a.r + k]);
       if (tid == 0) { s_found = 0x7FFFFFFF; s_last = -1; }
       __syncthreads();
       const int len = v_hi - v_lo;
-      const int nrow = (len + VT - 1) / VT;
+      const int nrow = (len + WT - 1) / WT;
       double carry = 0.0;
       for (int i = 0; i < nrow; ++i) {
-        const int o = i * VT + tid, w = v_lo + o;
+        const int o = i * WT + tid, w = v_lo + o;
         double rw = 0.0;
         if (o < len) {
           double Cw = C;
@@ -646,7 +858,14 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
           double q = 0.0;
           if (Cw != 0.0) {
             float acc = Elem<TIn>::to_f(reinterpret_cast<const TIn*>(a.U)[((size_t)b * a.D + dep) * a.V + w]);
-            if (ws_ok) { for (int k = 0; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Ws[(size_t)k * a.vt_TV + o]), acc); }
+            if (MMA) {
+              // the range's W columns sit in the tensor-core operand layout: 64-token slabs of [rp][128 B],
+              // 16-byte chunk j of row k at chunk j ^ (k & 7)
+              const unsigned char* wsl = tc.Ws + (size_t)(o >> 6) * tc.slab_bytes + (o & 7) * 2;
+              const int j = (o & 63) >> 3;
+              for (int k = 0; k < a.r; ++k)
+                acc = fmaf(sb_a[k], __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(wsl + k * 128 + ((j ^ (k & 7)) << 4))), acc);
+            } else if (ws_ok) { for (int k = 0; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Ws[(size_t)k * a.vt_TV + o]), acc); }
             else { for (int k = 0; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Wg[(size_t)k * a.V + w]), acc); }
             q = exp((double)acc / (double)a.T - lseT);
           }
@@ -658,7 +877,7 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
         if (lane == 31) s_scan[warp] = inc;
         __syncthreads();
         double wbase = 0.0, rowsum = 0.0;
-        for (int w2 = 0; w2 < VT / 32; ++w2) { if (w2 < warp) wbase += s_scan[w2]; rowsum += s_scan[w2]; }
+        for (int w2 = 0; w2 < WT / 32; ++w2) { if (w2 < warp) wbase += s_scan[w2]; rowsum += s_scan[w2]; }
         const double cum = carry + wbase + inc;
         if (o < len && rw > 0.0) atomicMax(&s_last, o);
         if (o < len && cum > want) atomicMin(&s_found, o);
@@ -675,15 +894,99 @@ __global__ void __launch_bounds__(VT) verify_walk_kernel(VerifyArgs a) {
     }
     __threadfence();
     DBGW(step, 4);
-    if (!grid_barrier(a.barrier, nblocks, gen)) return;
+    if (!grid_barrier(a.barrier, nblocks, gen)) return false;
     DBGW(step, 5);
     if (threadIdx.x == 0 && blockIdx.x == 0 && step < 64) { DBGW(step, 6); }
-    if (left == 0 && nwk == 0 && nsc == 0) return;
+    if (left == 0 && nwk == 0 && nsc == 0) return true;
   }
   // steps ran out
   for (int b = blockIdx.x; b < a.B; b += nblocks)
     if (tid == 0 && a.state[b].need != 3) a.status[b] = TS_ERR_TIMEOUT;
+  return true;
 }
+
+// Kernel wrapper.  MMA = true (bf16 inputs on sm_100): the CTA's range of W is loaded once in the tensor-core
+// operand layout (bulk-tensor loads when a tensor map is available, plain loads otherwise), tensor memory is
+// allocated for the accumulators, and both are released on every way out.
+template <typename TIn, bool MMA>
+__global__ void __launch_bounds__(WT, 1) verify_walk_kernel(const VerifyArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma) {
+  extern __shared__ __align__(16) unsigned char w_raw[];
+  WalkTc tc{};
+  if (!MMA) { walk_body<TIn, false>(a, tc, w_raw); return; }
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int r = a.r, rp = (r + 63) / 64 * 64;
+  const int t0 = blockIdx.x * a.vt_TV, tlen = min(a.vt_TV, a.V - t0);
+  const int nslab = a.vt_TV / 64, nblk = (tlen + 127) / 128;
+  unsigned char* sm = w_raw + ((1024u - (smem_u32(w_raw) & 1023u)) & 1023u);
+  tc.rp = rp; tc.slab_bytes = (uint32_t)rp * 128u; tc.it = 0;
+  tc.Ws = sm;
+  tc.As = tc.Ws + (size_t)nslab * tc.slab_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tc.As + (size_t)(rp / 64) * 128 * 128);
+  tc.t_full = bars; tc.t_empty = bars + WALK_NBUF;
+  uint64_t* w_full = bars + 2 * WALK_NBUF;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(w_full + WALK_MAX_BLK);
+  tc.s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  constexpr uint32_t TMEM_COLS = WALK_NBUF * 128;
+  if (warp == WALK_EPI) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    for (int i = 0; i < WALK_NBUF; ++i) { mbar_init(tc.t_full + i, 1); mbar_init(tc.t_empty + i, WALK_EPI); }
+    *tc.s_abort = 0;
+    if (use_tma) for (int i = 0; i < nblk; ++i) mbar_init(w_full + i, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (use_tma) {
+      for (int nb = 0; nb < nblk; ++nb) {
+        const int ns = (tlen - nb * 128 > 64) ? 2 : 1;
+        mbar_expect_tx(w_full + nb, (uint32_t)ns * tc.slab_bytes);
+        for (int h = 0; h < ns; ++h) tma_load_box(tc.Ws + (size_t)(2 * nb + h) * tc.slab_bytes, &tmW, t0 + (2 * nb + h) * 64, 0, w_full + nb);
+      }
+    }
+  }
+  if (!use_tma) {
+    const __nv_bfloat16* Wg = reinterpret_cast<const __nv_bfloat16*>(a.W);
+    const int per_slab = rp * 8;
+    for (int idx = tid; idx < nslab * per_slab; idx += WT) {
+      const int slab = idx / per_slab, rem = idx % per_slab, k = rem >> 3, j = rem & 7;
+      const int tok = t0 + slab * 64 + j * 8;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (k < r && tok < a.V) v = __ldg(reinterpret_cast<const uint4*>(Wg + (size_t)k * a.V + tok));
+      *reinterpret_cast<uint4*>(tc.Ws + (size_t)slab * tc.slab_bytes + k * 128 + ((j ^ (k & 7)) << 4)) = v;
+    }
+  }
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  tc.tmem_base = *s_tmem;
+  bool ok = true;
+  if (use_tma) {
+    // the whole range must have landed before anything reads it (the rescans read it with plain loads)
+    if (tid == 0)
+      for (int nb = 0; nb < nblk; ++nb) if (!mbar_wait(w_full + nb, 0, tc.s_abort, nullptr)) break;
+    __syncthreads();
+    ok = *tc.s_abort == 0;
+    if (!ok && tid == 0) atomicExch(a.barrier + 1, 1u);
+  }
+  if (ok) walk_body<TIn, true>(a, tc, w_raw);
+  if (use_tma && !ok && tid == 0) {
+    // gave up on a load: do not leave while it may still be writing this CTA's shared memory
+    for (int nb = 0; nb < nblk; ++nb) {
+      bool done = false;
+      for (uint32_t i = 0; i < WAIT_LIMIT && !done; ++i) { done = mbar_try_wait(w_full + nb, 0); if (!done) __nanosleep(100); }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == WALK_EPI) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tc.tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+
 
 // after a barrier timeout the kernel returns early; this marks every unfinished request
 __global__ void verify_check_kernel(VerifyArgs a) {
@@ -694,10 +997,12 @@ __global__ void verify_check_kernel(VerifyArgs a) {
 
 cudaError_t verify_setup(ts_ctx* ctx) {
   // the walk kernel may keep its range of W in shared memory: allow the full opt-in size
-  cudaError_t e = cudaFuncSetAttribute(verify_walk_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(verify_walk_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        ctx->max_smem - 32 * 1024);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(verify_walk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem - 32 * 1024);
+  e = cudaFuncSetAttribute(verify_walk_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem - 32 * 1024);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(verify_walk_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem - 32 * 1024);
 }
 
 }  // namespace ts
@@ -759,11 +1064,24 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
   }
   e = cudaMemsetAsync(a.barrier, 0, 64, st);
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(memset)", e);
-  const size_t w_bytes = (size_t)c.r * ctx->vt_TV * (c.dt_W == TS_DTYPE_BF16 ? 2 : 4);
+  size_t w_bytes = (size_t)c.r * ctx->vt_TV * (c.dt_W == TS_DTYPE_BF16 ? 2 : 4);
   a.w_smem = (w_bytes + 32 * 1024 <= (size_t)ctx->max_smem) ? 1 : 0;
-  void* kargs[] = {(void*)&a};
-  const void* fn = c.dt_Z == TS_DTYPE_BF16 ? (const void*)verify_walk_kernel<__nv_bfloat16> : (const void*)verify_walk_kernel<float>;
-  { ProfScope ps(ctx, K_WALK, st); e = cudaLaunchCooperativeKernel(fn, dim3(a.vt_n), dim3(VT), kargs, a.w_smem ? w_bytes : 0, st); }
+  // tensor-core reductions: bf16 everywhere, the range of W in operand layout plus the A tile within shared memory
+  const size_t rp = (size_t)(c.r + 63) / 64 * 64;
+  const size_t mma_bytes = (size_t)(ctx->vt_TV / 64) * rp * 128 + (rp / 64) * 128 * 128 + (2 * WALK_NBUF + WALK_MAX_BLK) * 8 + 64 + 1024;
+  const bool mma = ctx->use_mma && c.dt_Z == TS_DTYPE_BF16 && c.dt_U == TS_DTYPE_BF16 && c.dt_W == TS_DTYPE_BF16 &&
+                   c.dt_A == TS_DTYPE_BF16 && ctx->vt_TV % 64 == 0 && ctx->vt_TV / 128 < WALK_MAX_BLK &&
+                   mma_bytes + 32 * 1024 <= (size_t)ctx->max_smem;
+  int use_tma = 0;
+  CUtensorMap tm;
+  memset(&tm, 0, sizeof(tm));
+  if (mma && w_tensor_map(ctx, W)) { memcpy(&tm, ctx->tmapW, sizeof(tm)); use_tma = 1; }
+  void* kargs[] = {(void*)&a, (void*)&tm, (void*)&use_tma};
+  const void* fn = mma ? (const void*)verify_walk_kernel<__nv_bfloat16, true>
+                       : (c.dt_Z == TS_DTYPE_BF16 ? (const void*)verify_walk_kernel<__nv_bfloat16, false>
+                                                  : (const void*)verify_walk_kernel<float, false>);
+  if (mma) w_bytes = mma_bytes;
+  { ProfScope ps(ctx, K_WALK, st); e = cudaLaunchCooperativeKernel(fn, dim3(a.vt_n), dim3(WT), kargs, (mma || a.w_smem) ? w_bytes : 0, st); }
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(walk)", e);
   { ProfScope ps(ctx, K_CHECK, st); verify_check_kernel<<<(B + 127) / 128, 128, 0, st>>>(a); }
   e = cudaGetLastError();
