@@ -412,7 +412,8 @@ __device__ __forceinline__ void sweep_item(const SweepCtx<TIn>& c, int g0, int c
 constexpr int SB = 32; // requests whose head rows are staged together
 constexpr int WT = 288;       // threads of the walk kernel: eight worker warps and the warp that issues the MMAs
 constexpr int WALK_EPI = 8;   // worker warps that read the accumulators of a tensor-core reduction
-constexpr int WALK_NBUF = 4;  // accumulator buffers of 128 columns in tensor memory
+constexpr int WALK_BLK = 256;  // tokens per MMA block (one accumulator buffer)
+constexpr int WALK_NBUF = 2;  // accumulator buffers in tensor memory
 constexpr int WALK_MAX_BLK = 32;
 
 // Tensor-core state of one walk CTA: shared-memory operands, barriers, tensor-memory base and the running
@@ -465,7 +466,7 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const int nblk = (tlen + 127) / 128;
+  const int nblk = (tlen + WALK_BLK - 1) / WALK_BLK;
   if (tid == 0) DBGP(1);
   if (warp < WALK_EPI) {
     const int q = warp & 3, s = warp >> 2;
@@ -483,23 +484,37 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
       zoff = (-sb_zmax[g] * invT - sb_zlogs[g]) * 1.4426950408889634f;
       qoff = C != 0.f ? -sb_lseT[g] * 1.4426950408889634f : -1e30f;   // lseT may be NaN where it is not needed
     }
-    float sum = 0.f;
+    float sum = 0.f, sum2 = 0.f;
     bool alive = true;
     const bool need_q = C != 0.f;
-    // the rows of the next owned chunk are requested while this one is worked on
-    uint4 nz0 = make_uint4(0, 0, 0, 0), nz1 = nz0, nu0 = nz0, nu1 = nz0;
-    {
-      const int cg0 = rho + R * s;           // owned chunks: cg = rho + R * (s + 2 j)
-      const int vn = t0 + cg0 * 16;
-      if (active && cg0 * 16 < tlen) {
-        nz0 = __ldg(reinterpret_cast<const uint4*>(Zrow + vn));
-        if (V - vn > 8) nz1 = __ldg(reinterpret_cast<const uint4*>(Zrow + vn + 8));
-        if (need_q) {
-          nu0 = __ldg(reinterpret_cast<const uint4*>(Urow + vn));
-          if (V - vn > 8) nu1 = __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8));
-        }
+    // Owned chunks of a block: c = c0 + 2R j (2R divides the 16 chunks of a block).  They are taken two
+    // at a time so that the two chunks' loads and exponentials overlap; the target and base-logit rows
+    // of the next pair are requested while this pair is worked on.
+    const int c0 = rho + R * s, cstep = 2 * R;
+    uint4 nz[2][2], nu[2][2];
+    auto request = [&](int cg, int h) {
+      const int vn = t0 + cg * 16;
+      const uint4 zero = make_uint4(0, 0, 0, 0);
+      const bool in = active && cg * 16 < tlen;
+      nz[h][0] = in ? __ldg(reinterpret_cast<const uint4*>(Zrow + vn)) : zero;
+      nz[h][1] = (in && V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Zrow + vn + 8)) : zero;
+      nu[h][0] = (in && need_q) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn)) : zero;
+      nu[h][1] = (in && need_q && V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8)) : zero;
+    };
+    auto residual = [&](const uint32_t* racc, const uint4& z0, const uint4& z1, const uint4& u0, const uint4& u1, int valid, float& acc_sum) {
+      float zz[16], ub[16];
+      unpack_bf16x8(z0, zz); unpack_bf16x8(z1, zz + 8);
+      unpack_bf16x8(u0, ub); unpack_bf16x8(u1, ub + 8);
+      // one path for every lane: a request with C == 0 has qoff = -huge, so its q term vanishes
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const float p = fast_ex2(fmaf(zz[i], zs, zoff));
+        const float qq = fast_ex2(fmaf(__uint_as_float(racc[i]) + ub[i], zs, qoff));
+        if (i < valid) acc_sum += fmaxf(fmaf(-C, qq, p), 0.f);
       }
-    }
+    };
+    request(c0, 0);
+    request(c0 + cstep, 1);
     for (int nb = 0; nb < nblk && alive; ++nb) {
       const uint32_t it = tc.it + (uint32_t)nb, tb = it % WALK_NBUF, u = it / WALK_NBUF;
       int ok = 1;
@@ -508,54 +523,37 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
       if (!ok) { alive = false; break; }
       tc_fence_after();
       if (tid == 0) DBGP(4 + 2 * nb);
-      const int nch = min(8, (tlen - nb * 128 + 15) / 16);
-      for (int c = 0; c < nch; ++c) {
-        const int cg = nb * 8 + c;
-        if ((cg & (R - 1)) != rho || ((cg >> rsh) & 1) != s) continue;   // warp-uniform; R is 1, 2 or 4
-        float acc[16];
-        if (tid == 0 && nb == 4) DBGP(40);
-        tmem_ld16(tc.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * 128 + c * 16), acc);
-        if (tid == 0 && nb == 4) DBGP(41);
+      const int nch = min(WALK_BLK / 16, (tlen - nb * WALK_BLK + 15) / 16);
+      for (int ca = c0; ca < nch; ca += 2 * cstep) {
+        const int cb = ca + cstep;
+        const bool hb = cb < nch;   // warp-uniform
+        const int cga = nb * (WALK_BLK / 16) + ca, cgb = cga + cstep;
+        uint32_t ra[16], rb[16];
+        const uint32_t tbase = tc.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * WALK_BLK);
+        tmem_ld16_issue(tbase + (uint32_t)(ca * 16), ra);
+        if (hb) tmem_ld16_issue(tbase + (uint32_t)(cb * 16), rb);
+        tmem_ld_wait();
+        const uint4 za0 = nz[0][0], za1 = nz[0][1], ua0 = nu[0][0], ua1 = nu[0][1];
+        const uint4 zb0 = nz[1][0], zb1 = nz[1][1], ub0 = nu[1][0], ub1 = nu[1][1];
+        // next pair: the rest of this block, else the first pair of the next block
+        {
+          int na = cga + 2 * cstep;
+          if (ca + 2 * cstep >= WALK_BLK / 16) na = (nb + 1) * (WALK_BLK / 16) + c0;
+          request(na, 0);
+          request(na + cstep, 1);
+        }
         if (active) {
-          const int v0 = t0 + cg * 16;
-          const int valid = min(16, V - v0);   // 8 or 16: V and v0 are multiples of 8
-          const uint4 z0 = nz0, z1 = nz1, u0 = nu0, u1 = nu1;
-          {
-            const int cgn = cg + R * 2;
-            const int vn = t0 + cgn * 16;
-            if (cgn * 16 < tlen) {
-              nz0 = __ldg(reinterpret_cast<const uint4*>(Zrow + vn));
-              nz1 = (V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Zrow + vn + 8)) : make_uint4(0, 0, 0, 0);
-              if (need_q) {
-                nu0 = __ldg(reinterpret_cast<const uint4*>(Urow + vn));
-                nu1 = (V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8)) : make_uint4(0, 0, 0, 0);
-              }
-            }
-          }
-          if (tid == 0 && nb == 4) DBGP(42);
-          float zz[16];
-          unpack_bf16x8(z0, zz);
-          unpack_bf16x8(z1, zz + 8);
-          if (tid == 0 && nb == 4) DBGP(43);
-          // one path for every lane: a request with C == 0 has qoff = -huge, so its q term vanishes
-          float ub[16];
-          unpack_bf16x8(u0, ub);
-          unpack_bf16x8(u1, ub + 8);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float p = fast_ex2(fmaf(zz[i], zs, zoff));
-            const float qq = fast_ex2(fmaf(acc[i] + ub[i], zs, qoff));
-            if (i < valid) sum += fmaxf(fmaf(-C, qq, p), 0.f);
-          }
-          if (tid == 0 && nb == 4) DBGP(44);
+          const int va = t0 + cga * 16, vb = t0 + cgb * 16;
+          residual(ra, za0, za1, ua0, ua1, min(16, V - va), sum);
+          if (hb) residual(rb, zb0, zb1, ub0, ub1, min(16, V - vb), sum2);
         }
       }
-      if (tid == 0 && nb == 4) DBGP(45);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tc.t_empty + tb);
       if (tid == 0) DBGP(5 + 2 * nb);
     }
+    sum += sum2;
     s_part[row * 2 + s] = active ? sum : 0.f;
   } else if (warp == WALK_EPI && lane == 0) {
     const uint32_t ws_addr = smem_u32(tc.Ws), as_addr = smem_u32(tc.As);
@@ -565,12 +563,12 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
         if (!mbar_wait(tc.t_empty + tb, (u - 1) & 1, tc.s_abort, nullptr)) break;
         tc_fence_after();
       }
-      const int n = (tlen - nb * 128 > 64) ? 128 : 64;
+      const int n = min(WALK_BLK, (tlen - nb * WALK_BLK + 63) / 64 * 64);   // whole 64-token slabs
       const uint32_t idesc = instr_desc(n);
-      const uint32_t d_tmem = tc.tmem_base + tb * 128u;
+      const uint32_t d_tmem = tc.tmem_base + tb * (uint32_t)WALK_BLK;
       for (int ks = 0; ks < rp / 16; ++ks) {
         const uint64_t adesc = smem_desc(as_addr + (uint32_t)(ks >> 2) * a_slab_bytes + (uint32_t)(ks & 3) * 32u, 16u, 1024u);
-        const uint64_t bdesc = smem_desc(ws_addr + (uint32_t)(2 * nb) * tc.slab_bytes + (uint32_t)ks * 2048u, tc.slab_bytes, 1024u);
+        const uint64_t bdesc = smem_desc(ws_addr + (uint32_t)(WALK_BLK / 64 * nb) * tc.slab_bytes + (uint32_t)ks * 2048u, tc.slab_bytes, 1024u);
         mma_bf16(d_tmem, adesc, bdesc, idesc, ks > 0 ? 1u : 0u);
       }
       mma_commit(tc.t_full + tb);
@@ -926,7 +924,7 @@ __global__ void __launch_bounds__(WT, 1) verify_walk_kernel(const VerifyArgs a, 
   uint64_t* w_full = bars + 2 * WALK_NBUF;
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(w_full + WALK_MAX_BLK);
   tc.s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
-  constexpr uint32_t TMEM_COLS = WALK_NBUF * 128;
+  constexpr uint32_t TMEM_COLS = WALK_NBUF * WALK_BLK;
   if (warp == WALK_EPI) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
