@@ -88,6 +88,7 @@ struct WsLayout {
   size_t vf_barrier;                     // unsigned[4]
   size_t vf_child;                       // int[2][B][N+1]: first child and child count of every node
   size_t vf_lists;                       // int[2][B] reduction list, int[2][B] rescan list, int[8] counters
+  size_t vf_edge;                        // double[3][B][N]: per edge p(x), q(x) and the accept uniform
   size_t total;
 };
 
@@ -152,6 +153,7 @@ __host__ inline WsLayout make_layout(const ts_ctx* ctx, int B) {
   L.vf_barrier = take(64);
   L.vf_child = take(2 * b * (N + 1) * 4);
   L.vf_lists = take((4 * b + 8) * 4);
+  L.vf_edge = take(3 * b * N * 8);
   L.total = off;
   return L;
 }

@@ -119,6 +119,7 @@ struct VerifyArgs {
   const float *logqT, *node_lseT;
   const float* z_max; const int* z_arg; const float* z_logs;
   int *acc_len, *acc_node, *acc_tok, *bonus; float* edge_stat; uint32_t* flags; int* status;
+  double *edge_px, *edge_qx, *edge_u;   // per edge: target and draft probability of its token, its accept uniform
   VerifyState* state; float* part; unsigned* barrier;
   int* child_first; int* child_cnt;   // [B][N+1], slot 0 = root
   int* wk_list; int* sc_list;         // [2][B] requests that asked for a reduction / a range rescan, by step parity
@@ -176,13 +177,17 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
   VerifyState* gst = a.state + b;
   const int N = a.N;
   const size_t nb = (size_t)b * N;
-  const int64_t row0 = a.z_row_off[b];
   const int need_in = gst->need;
   if (need_in == 3) return;
   // ---- fold in the reduction that just ran -------------------------------------------------
   double fsum = 0.0;
   if (need_in == 1 || need_in == 4) {
-    for (int t = lane; t < a.vt_n; t += 32) fsum += (double)__ldcg(a.part + (size_t)b * a.vt_n + t);
+    float pv[8];   // the first 256 range sums in one memory round trip
+#pragma unroll
+    for (int k = 0; k < 8; ++k) pv[k] = (k * 32 + lane < a.vt_n) ? __ldcg(a.part + (size_t)b * a.vt_n + k * 32 + lane) : 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) if (k * 32 + lane < a.vt_n) fsum += (double)pv[k];
+    for (int t = 256 + lane; t < a.vt_n; t += 32) fsum += (double)__ldcg(a.part + (size_t)b * a.vt_n + t);
     for (int off = 16; off > 0; off >>= 1) fsum += __shfl_xor_sync(0xFFFFFFFFu, fsum, off);
   }
   VerifyState st;   // working copy (written back once at the end)
@@ -215,19 +220,18 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
     // inputs of every child's accept test at the current node, one child per lane
     const int v = __shfl_sync(0xFFFFFFFFu, st.cur, 0);
     const int first = a.child_first[(size_t)b * (N + 1) + v + 1], m = a.child_cnt[(size_t)b * (N + 1) + v + 1];
-    const int64_t row = row0 + v + 1;
     double px = 0.0, qx = 1.0; int x = -1;
-    if (lane < m) {
+    double ux = 0.0;
+    if (lane < m) {   // computed for every edge when the walk was set up
       x = a.tok[nb + first + lane];
-      px = exp(((double)z_elem<TIn>(a, row, x) - (double)a.z_max[row]) / (double)a.T - (double)a.z_logs[row]);
-      qx = exp((double)a.logqT[nb + first + lane]);
+      px = a.edge_px[nb + first + lane]; qx = a.edge_qx[nb + first + lane]; ux = a.edge_u[nb + first + lane];
     }
-    const uint64_t hv = a.node_hash[(size_t)b * (N + 1) + v + 1];
     // lane 0 runs the sibling chain at this node until it accepts, needs a reduction, or runs out
     int again = 0;
     for (int j = 0; j < 32; ++j) {   // m <= K <= 16
       const double pxj = __shfl_sync(0xFFFFFFFFu, px, j), qxj = __shfl_sync(0xFFFFFFFFu, qx, j);
       const int xj = __shfl_sync(0xFFFFFFFFu, x, j);
+      const double uj = __shfl_sync(0xFFFFFFFFu, ux, j);
       int stop = 0;
       if (lane == 0) {
         if (st.j != j) { }   // siblings before st.j were tested in an earlier step
@@ -235,8 +239,7 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
           const double cj = st.Zj / (1.0 - st.Qused);
           const double num = fmax(pxj / qxj - st.C, 0.0);
           const double rho = fmin(1.0, num / cj);
-          const double u = u01(stream_words(a.seed, b, hv, STREAM_ACCEPT, (uint32_t)st.j).x);
-          if (u < rho) {
+          if (uj < rho) {
             a.acc_node[(size_t)b * a.D + st.acc] = first + j; a.acc_tok[(size_t)b * a.D + st.acc] = xj;
             st.acc++; st.cur = first + j; st.j = 0; st.C = 0.0; st.Zj = 1.0; st.Qused = 0.0; st.nf = 0; st.partsC = -1.0;
             stop = 1; again = 1;          // descend: next node
@@ -266,10 +269,19 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
     const double u = u01(stream_words(a.seed, b, hv, STREAM_BONUS, 0u).x);
     const double target = u * Zj;
     double carry = 0.0; int found = -1; double before = 0.0; int last_pos = -1;
+    // the first 256 range sums are requested together (one memory round trip for the usual grid sizes)
+    float pre[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) pre[k] = (k * 32 + lane < a.vt_n) ? __ldcg(a.part + (size_t)b * a.vt_n + k * 32 + lane) : 0.f;
     for (int t0 = 0; t0 < a.vt_n && found < 0; t0 += 32) {
       const int t = t0 + lane;
       double pt = 0.0;
-      if (t < a.vt_n) pt = (double)__ldcg(a.part + (size_t)b * a.vt_n + t);
+      if (t0 < 256) {
+        float pv = pre[0];
+#pragma unroll
+        for (int k = 1; k < 8; ++k) pv = (t0 >> 5) == k ? pre[k] : pv;
+        pt = (double)pv;
+      } else if (t < a.vt_n) pt = (double)__ldcg(a.part + (size_t)b * a.vt_n + t);
       for (int i = 0; i < nf; ++i) {   // tested siblings keep the residual they had when tested
         const int fxi = __shfl_sync(0xFFFFFFFFu, st.fx[i], 0);
         const double fpi = __shfl_sync(0xFFFFFFFFu, st.fp[i], 0), fqi = __shfl_sync(0xFFFFFFFFu, st.fq[i], 0);
@@ -643,6 +655,16 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
         const int par = a.parent[nb + i];
         if (i == 0 || a.parent[nb + i - 1] != par) a.child_first[cbase + par + 1] = i;   // siblings are contiguous
         atomicAdd(&a.child_cnt[cbase + par + 1], 1);
+        {
+          // what the accept test of this edge needs, off the walk's critical path: p(x), q(x) and the uniform
+          // of sibling j at its parent (j = place among the contiguous siblings)
+          const int64_t row = row0 + par + 1;
+          int j = 0;
+          while (i - j - 1 >= 0 && a.parent[nb + i - j - 1] == par) ++j;
+          a.edge_px[nb + i] = exp(((double)z_elem<TIn>(a, row, a.tok[nb + i]) - (double)a.z_max[row]) / (double)a.T - (double)a.z_logs[row]);
+          a.edge_qx[nb + i] = exp((double)a.logqT[nb + i]);
+          a.edge_u[nb + i] = u01(stream_words(a.seed, b, a.node_hash[(size_t)b * (N + 1) + par + 1], STREAM_ACCEPT, (uint32_t)j).x);
+        }
         if (a.edge_stat) {
           const int64_t row = row0 + par + 1;
           const double lr = ((double)z_elem<TIn>(a, row, a.tok[nb + i]) - (double)a.z_max[row]) / (double)a.T -
@@ -1040,6 +1062,7 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
   a.flags = flags; a.status = status;
   a.state = (VerifyState*)(ws + L.vf_state); a.part = (float*)(ws + L.vf_part); a.barrier = (unsigned*)(ws + L.vf_barrier);
   a.child_first = (int*)(ws + L.vf_child); a.child_cnt = a.child_first + (size_t)B * (c.Nmax + 1);
+  a.edge_px = (double*)(ws + L.vf_edge); a.edge_qx = a.edge_px + (size_t)B * c.Nmax; a.edge_u = a.edge_qx + (size_t)B * c.Nmax;
   a.wk_list = (int*)(ws + L.vf_lists); a.sc_list = a.wk_list + 2 * (size_t)B; a.ctr = a.sc_list + 2 * (size_t)B;
   a.vt_TV = ctx->vt_TV; a.vt_n = ctx->vt_n; a.max_steps = 2 * (c.Nmax + c.D) + 8;
 
