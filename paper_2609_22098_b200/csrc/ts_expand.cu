@@ -142,11 +142,16 @@ __global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d) 
   __syncthreads();
   // a sibling slot exists only if the one before it was admitted (keys are non-increasing in j)
   for (int i = tid; i < npar; i += blockDim.x) {
+    int vals[KMAX];   // all flags of the parent first: independent loads, one round trip
+#pragma unroll
+    for (int j = 0; j < KMAX; ++j) vals[j] = j < K ? a.cd_valid[cb + (size_t)i * K + j] : 0;
     bool open = true;
-    for (int j = 0; j < K; ++j) {
-      const size_t ci = cb + (size_t)i * K + j;
-      if (!open) a.cd_valid[ci] = 0;
-      else if (!a.cd_valid[ci]) open = false;
+#pragma unroll
+    for (int j = 0; j < KMAX; ++j) {
+      if (j < K) {
+        if (!open && vals[j]) a.cd_valid[cb + (size_t)i * K + j] = 0;
+        else if (!vals[j]) open = false;
+      }
     }
   }
   __syncthreads();
@@ -281,22 +286,30 @@ struct FinalArgs {
 
 // Canonical (BFS) renumbering, outputs and ancestor bitmasks; one CTA per request.
 __global__ void __launch_bounds__(256) expand_finalize_kernel(FinalArgs a) {
-  __shared__ int s_canon[256];
+  // the pool of one request is small: it is ranked, renumbered and masked out of shared memory
+  __shared__ int s_canon[256], s_alive[256], s_depth[256], s_par[256], s_cpar[256];
+  __shared__ uint64_t s_path[256];
+  __shared__ double s_key[256];
+  __shared__ uint64_t s_mask[256 * 4];
   __shared__ int s_n;
   const int b = blockIdx.x, tid = threadIdx.x, N = a.N;
   const size_t pb = (size_t)b * N;
   if (tid == 0) s_n = 0;
+  for (int s = tid; s < N; s += blockDim.x) {
+    s_alive[s] = a.pl_alive[pb + s]; s_depth[s] = a.pl_depth[pb + s]; s_path[s] = a.pl_path[pb + s];
+    s_key[s] = a.pl_logkey[pb + s]; s_par[s] = a.pl_parent[pb + s];
+  }
   __syncthreads();
   for (int s = tid; s < N; s += blockDim.x) {
     s_canon[s] = -1;
-    if (!a.pl_alive[pb + s]) continue;
-    const int ds = a.pl_depth[pb + s]; const uint64_t ps = a.pl_path[pb + s]; const double ks = a.pl_logkey[pb + s];
+    if (!s_alive[s]) continue;
+    const int ds = s_depth[s]; const uint64_t ps = s_path[s]; const double ks = s_key[s];
     int cr = 0, pr = 0;
     for (int t = 0; t < N; ++t) {
-      if (t == s || !a.pl_alive[pb + t]) continue;
-      const int dt = a.pl_depth[pb + t]; const uint64_t pt = a.pl_path[pb + t];
+      if (t == s || !s_alive[t]) continue;
+      const int dt = s_depth[t]; const uint64_t pt = s_path[t];
       if (dt < ds || (dt == ds && pt < ps)) ++cr;
-      if (before(a.pl_logkey[pb + t], dt, pt, ks, ds, ps)) ++pr;
+      if (before(s_key[t], dt, pt, ks, ds, ps)) ++pr;
     }
     s_canon[s] = cr;
     atomicAdd(&s_n, 1);
@@ -311,8 +324,10 @@ __global__ void __launch_bounds__(256) expand_finalize_kernel(FinalArgs a) {
   __syncthreads();
   for (int s = tid; s < N; s += blockDim.x) {
     if (s_canon[s] < 0) continue;
-    const int ps = a.pl_parent[pb + s];
-    a.parent[pb + s_canon[s]] = ps < 0 ? -1 : s_canon[ps];
+    const int ps = s_par[s];
+    const int cp = ps < 0 ? -1 : s_canon[ps];
+    s_cpar[s_canon[s]] = cp;
+    a.parent[pb + s_canon[s]] = cp;
   }
   if (tid == 0) {
     a.n_nodes[b] = s_n;
@@ -325,12 +340,14 @@ __global__ void __launch_bounds__(256) expand_finalize_kernel(FinalArgs a) {
   const int n = s_n;
   if (tid < a.words) {
     for (int i = 0; i < n; ++i) {
-      const int p = a.parent[pb + i];
-      uint64_t m = p >= 0 ? a.mask[(pb + p) * a.words + tid] : 0ull;
+      const int p = s_cpar[i];
+      uint64_t m = p >= 0 ? s_mask[p * a.words + tid] : 0ull;
       if (i / 64 == tid) m |= 1ull << (i % 64);
-      a.mask[(pb + i) * a.words + tid] = m;
+      s_mask[i * a.words + tid] = m;
     }
   }
+  __syncthreads();
+  for (int i = tid; i < n * a.words; i += blockDim.x) a.mask[pb * a.words + i] = s_mask[i];
 }
 
 }  // namespace ts
