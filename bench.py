@@ -35,7 +35,7 @@ FALLBACK_HBM_GBS = 6650.0
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="serve32", choices=list(synth.WORKLOADS))
@@ -81,9 +81,15 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.monotonic(), line.strip()))
 
-    def stop(self):
+    def wait_first(self, limit=2.0):
+        """nvidia-smi takes a moment to start: wait (bounded) for its first line."""
+        t0 = time.monotonic()
+        while self.proc and not self.lines and time.monotonic() - t0 < limit:
+            time.sleep(0.01)
+
+    def stop(self, t_lo=None, t_hi=None):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
         self.proc.terminate()
@@ -93,7 +99,10 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        inside = [ln for (t, ln) in self.lines if t_lo is not None and t_lo <= t <= t_hi]
+        # samples inside the timed region when it is long enough to hold some, else every sample since the
+        # warm-up began (the GPU runs the same rounds from there to the end of the timed region)
+        for ln in (inside if inside else [ln for (_, ln) in self.lines]):
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 7:
                 continue
@@ -105,7 +114,7 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "samples_in_timed_region": len(inside), "reasons": sorted(reasons)}
 
 
 class InputSet:
@@ -201,19 +210,21 @@ def run_ours(args, rank, world, device):
         torch.cuda.synchronize()
 
     # ---- timed region -----------------------------------------------------------------------
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    sampler.wait_first()
     for i in range(args.warmup):
         one_round(i)
     ts.profile_read(reset=True)
-    sampler = ClockSampler(torch.cuda.current_device())
-    sampler.start()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_lo = time.monotonic()
     e0.record()
     for i in range(args.steps):
         one_round(args.warmup + i)
     e1.record()
     barrier()
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_lo, time.monotonic())
     total_ms = e0.elapsed_time(e1)
     launches = sum(c for _, c in ts.profile_read(reset=True).values())
     last = (args.warmup + args.steps - 1) % len(sets)
@@ -251,11 +262,16 @@ def run_ours(args, rank, world, device):
     # its range of W is staged once per launch
     bytes_walk = mean("walk_passes") * 2 * row_b + w_b
     alg = {"score_tile": bytes_score, "zrow_stats": bytes_zrows, "verify_walk": bytes_walk}
-    traffic = None
+    # DRAM bytes of the dominant kernel from a committed ncu capture of one round of this workload
+    # (per launch: the round's bytes over the round's launches), null where none was captured
+    traffic, traffic_src = None, None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
     if dom and os.path.exists(tpath):
         try:
-            traffic = json.load(open(tpath)).get(args.workload, {}).get(dom)
+            ent = json.load(open(tpath)).get(args.workload, {}).get(dom)
+            if ent:
+                traffic = ent["dram_bytes_per_round"] / ent["launches_per_round"]
+                traffic_src = ent.get("source")
         except Exception:
             traffic = None
     roofline = None
@@ -265,7 +281,9 @@ def run_ours(args, rank, world, device):
         achieved = (a_bytes / (kern[dom]["ms_per_round"] * 1e-3) / 1e9) if a_bytes else None
         roofline = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": (achieved / peak) if achieved else None, "peak_source": f"of {peak_src}",
-                    "traffic": traffic, "alg_bytes_per_round": a_bytes, "ms_per_launch": per_launch_ms,
+                    "traffic": traffic, "traffic_source": traffic_src,
+                    "alg_bytes_per_launch": (a_bytes / max(kern[dom]["launches_per_round"], 1e-9)) if a_bytes else None,
+                    "alg_bytes_per_round": a_bytes, "ms_per_launch": per_launch_ms,
                     "launches_per_round": kern[dom]["launches_per_round"], "share_of_kernel_time": kern[dom]["share"]}
     sec = ms_per_step * 1e-3
     round_hbm = {"alg_bytes_all_rows": bytes_round_all, "alg_bytes_walk_rows_only": bytes_round_min,

@@ -37,6 +37,9 @@ extern "C" int ts_debug_timing_pass(unsigned long long* out) { return (int)cudaM
 #define DBGP(slot) do { } while (0)
 #endif
 
+// 2^x by the hardware approximation (the library exp2f costs several times more in the hot loops here)
+__device__ __forceinline__ float fast_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+
 constexpr int ZT = 512;  // threads per target row in the row-statistics kernel
 
 // ------------------------------------------------------------------------------------------------
@@ -57,14 +60,24 @@ __global__ void __launch_bounds__(ZT) zrow_stats_kernel(const TIn* Z, const int6
   for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
     const TIn* z = Z + row * V;
     float bv = -INFINITY, sum = 0.f; int bi = 0x7FFFFFFF;
+    // per vector: the maximum by a compare tree (its position is looked for only when it beats the running
+    // maximum, which is rare), then one fused multiply-add and one ex2 per element
+    const float sc = invT * 1.4426950408889634f;
+    float boff = 0.f;   // -bv * sc while bv is finite
     auto take = [&](const float* x, int c, int n) {
-      float vm = x[0]; int vi = 0;
+      float vm = x[0];
 #pragma unroll
-      for (int i = 1; i < VEC; ++i) if (i < n && x[i] > vm) { vm = x[i]; vi = i; }
-      if (vm > bv) { sum *= __expf((bv - vm) * invT); bv = vm; bi = c + vi; }   // first maximum wins: indices increase
+      for (int i = 1; i < VEC; ++i) if (i < n) vm = fmaxf(vm, x[i]);
+      if (vm > bv) {   // first maximum wins: indices increase
+        int vi = 0;
+#pragma unroll
+        for (int i = VEC - 1; i >= 0; --i) if (i < n && x[i] == vm) vi = i;
+        sum *= fast_ex2((bv - vm) * sc);
+        bv = vm; bi = c + vi; boff = -vm * sc;
+      }
       if (T > 0.f) {
 #pragma unroll
-        for (int i = 0; i < VEC; ++i) if (i < n) sum += __expf((x[i] - bv) * invT);
+        for (int i = 0; i < VEC; ++i) if (i < n) sum += fast_ex2(fmaf(x[i], sc, boff));
       }
     };
     if (vec_ok) {
@@ -441,8 +454,6 @@ struct WalkTc {
 // there are few); worker warp w reads the rows of quarter w % 4 and the 16-token chunks of column split
 // w / 4, adds the base logits, and accumulates the residual with the target row.  Partial sums are
 // combined in a fixed order.  Returns false when a bounded wait ran out.
-__device__ __forceinline__ float fast_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
-
 template <typename TIn>
 __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int tlen, float invT,
                          const int* sb_req, const int* sb_dep, const int* sb_tok, const long long* sb_row,
