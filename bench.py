@@ -26,7 +26,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2609_22098_b200 import synth  # noqa: E402
+from paper_2609_22098_b200 import shard, synth  # noqa: E402
 
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
@@ -176,7 +176,7 @@ def run_ours(args, rank, world, device):
     T = wl.temps[-1] if args.T is None else args.T
     theta = wl.theta if args.theta is None else args.theta
     es = 2 if wl.dtype == "bf16" else 4
-    seed = args.seed + 1000 * rank
+    seed = shard.shard_seed(args.seed, rank)
     table = synth.make_calibration_table(wl, args.seed + 4, "fit")
     A, W = synth.make_head(wl, args.seed + 1, device)
     ts = TreeSpark(wl.V, wl.D, wl.r, wl.K, wl.Nmax, B, dtype=wl.torch_dtype, calib_mode=wl.calib_mode,
@@ -229,10 +229,7 @@ def run_ours(args, rank, world, device):
     launches = sum(c for _, c in ts.profile_read(reset=True).values())
     last = (args.warmup + args.steps - 1) % len(sets)
     same = all(bool(torch.equal(a, b)) for a, b in zip(ref_out[last], snapshot(tree, verdict)))
-    if world > 1:
-        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        total_ms = float(t[0])
+    total_ms = shard.max_over_ranks(total_ms, device)   # the slowest rank's device time
     ms_per_step = total_ms / args.steps
 
     # ---- per-kernel device times (separate, instrumented loop; not the headline number) ----------
@@ -335,10 +332,7 @@ def run_e2e(args, ts, wl, sets, A, W, T, B, world, device, barrier):
     e1.record()
     barrier()
     ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device=device, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t[0])
+    ms = shard.max_over_ranks(ms, device)
     return {"value": world * steps * 1e3 / ms, "unit": "rounds/s", "steps": steps,
             "h2d_bytes_per_step": hr.h2d_bytes, "d2h_bytes_per_step": hr.d2h_bytes,
             "acc_len_sum_last": int(res["acc_len"].sum())}
