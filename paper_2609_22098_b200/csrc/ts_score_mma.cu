@@ -4,16 +4,20 @@
 // lane = one parent row per thread.
 //
 // CTA = one vocabulary tile, resident for the whole launch.  Shared memory holds
-//   W tile  : B operand, MN-major, 128-byte swizzle: slabs of 64 tokens, slab = [rp rows][128 B]
+//   W tile  : B operand, MN-major, 128-byte swizzle: slabs of 64 tokens, slab = [rp rows][128 B];
+//             loaded by bulk-tensor copies (one mbarrier per 128-token block), or by plain loads when
+//             no tensor map could be encoded
 //   A tile  : A operand, K-major, 128-byte swizzle: [rp/64 slabs][128 rows][128 B] (gathered rows A[x_p])
 // (rp = r rounded up to 64, padding zero-filled).  Warps 0..7 are epilogue warps: warp w reads the
-// tensor-memory lanes 32*(w%4).. (its quarter of the 128 parent rows) and, of every 128-column block,
-// the 16-token chunks assigned to column split s = w/4.  Warp 8 allocates tensor memory and its lane 0
-// issues the MMAs: per block of 128 tokens rp/16 instructions of M=128, N=128 (64 at a ragged end),
-// K=16 into one of two 128-column accumulator buffers, then a commit that arrives on that buffer's
-// "full" barrier; epilogue warps arrive on its "empty" barrier when they have drained it.
+// tensor-memory lanes 32*(w%4).. (its quarter of the 128 parent rows).  When a level has few parents the
+// rows are replicated R = 2 or 4 times over the quarters; of the tile's 16-token chunks, chunk cg belongs
+// to replica cg % R and column split (cg / R) % 2 (= w / 4).  Warp 8 allocates tensor memory and its
+// lane 0 issues the MMAs: per block of 128 tokens rp/16 instructions of M=128, N=128 (64 at a ragged
+// end), K=16 into one of four 128-column accumulator buffers, then a commit that arrives on that
+// buffer's "full" barrier; epilogue warps arrive on its "empty" barrier when they have drained it.
+// Warp 9 keeps shared-memory copies of the launch-wide pruning bounds of every row current.
 // Every wait is bounded: when one runs out the kernel raises an error word, skips the remaining work,
-// frees its tensor memory and returns.
+// waits (again bounded) for bulk loads still in flight, frees its tensor memory and returns.
 #include "ts_tc.cuh"
 #include "ts_internal.h"
 namespace ts {
