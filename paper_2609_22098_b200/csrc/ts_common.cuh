@@ -13,6 +13,14 @@ namespace ts {
 constexpr int KMAX = TS_KMAX;
 constexpr int DMAX = TS_DMAX;
 constexpr int KNOTS = TS_CALIB_KNOTS;
+// Programmatic dependent launch (the kernels of one expansion are chained with it).  pdl_wait(): everything
+// the kernels before this one in the stream wrote is visible afterwards; a kernel launched without the
+// attribute passes straight through.  pdl_launch_dependents(): the next kernel in the stream may start its
+// own preamble now.  Every chained kernel waits before it lets its dependents go and before it exits, so
+// a kernel that has passed its wait knows that ALL earlier kernels of the chain have completed.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Words between two pruning-bound slots: one 128-byte line each.  Every piece of a launch publishes into
 // these words with atomicMax in the launch's first microseconds; packed together they queue up on a
 // handful of L2 lines (measured: a third of the scoring launch at stride 1).

@@ -46,6 +46,7 @@ __device__ __forceinline__ void request_caps(const ExpandArgs& a, int b, int& K_
 }
 
 __global__ void expand_init_kernel(ExpandArgs a) {
+  pdl_launch_dependents();   // the first scoring launch may run its preamble beside this kernel
   const int b = blockIdx.x;
   // pruning state of the scoring launches: the threshold words, then one word per slot (the slots sit
   // SLOT_STRIDE words apart; only the first word of each is ever used)
@@ -84,6 +85,8 @@ __global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d) 
   __shared__ int s_base;
   const int b = blockIdx.x, tid = threadIdx.x;
   const int N = a.N, K = a.K;
+  pdl_wait();               // merged scoring results of this level
+  pdl_launch_dependents();
   const int npar = a.req_npar[b], base = a.req_base[b];
   const int cur = d & 1, nxt = cur ^ 1;
   int K_eff, N_eff; double log_theta;
@@ -294,6 +297,7 @@ __global__ void __launch_bounds__(256) expand_finalize_kernel(FinalArgs a) {
   __shared__ int s_n;
   const int b = blockIdx.x, tid = threadIdx.x, N = a.N;
   const size_t pb = (size_t)b * N;
+  pdl_wait();
   if (tid == 0) s_n = 0;
   for (int s = tid; s < N; s += blockDim.x) {
     s_alive[s] = a.pl_alive[pb + s]; s_depth[s] = a.pl_depth[pb + s]; s_path[s] = a.pl_path[pb + s];
@@ -416,10 +420,10 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
     e = launch_score(ctx, (float*)(ws + L.rec), L.rec_cap, (int*)(ws + L.err), U, A, W, 0, a.lvl_count + d,
                      a.lst_req[cur], a.lst_depth[cur], a.lst_token[cur],
                      a.lst_hash[cur], T, seed, res_lse0, res_lseT, res_top_tok, res_top_logit, res_draw_tok,
-                     res_draw_logit, st);
+                     res_draw_logit, st, /*pdl=*/true, d > 0 ? a.lvl_count + d - 1 : nullptr);
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(score)", e);
-    { ProfScope ps(ctx, K_LEVEL, st); expand_level_kernel<<<B, 256, level_smem, st>>>(a, d); }
-    e = cudaGetLastError();
+    { ProfScope ps(ctx, K_LEVEL, st); e = launch_kernel(expand_level_kernel, B, 256, level_smem, st, true, a, d); }
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(level)", e);
   }
   FinalArgs f{};
@@ -430,8 +434,8 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   f.n_nodes = n_nodes; f.tok = tok; f.parent = parent; f.depth = depth; f.sib_rank = sib_rank; f.logS = logS; f.q0 = q0;
   f.logqT = logqT; f.logkey = logkey; f.pop_rank = pop_rank; f.node_hash = node_hash; f.node_lseT = node_lseT;
   f.mask = mask; f.n_scored = n_scored;
-  { ProfScope ps(ctx, K_FINAL, st); expand_finalize_kernel<<<B, 256, 0, st>>>(f); }
-  e = cudaGetLastError();
+  { ProfScope ps(ctx, K_FINAL, st); e = launch_kernel(expand_finalize_kernel, B, 256, 0, st, true, f); }
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(finalize)", e);
   return TS_OK;
 }

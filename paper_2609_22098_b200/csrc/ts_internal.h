@@ -17,6 +17,8 @@ struct ScoreArgs {
   const void *U, *A, *W;
   int V, D, r, K;
   int P; const int* P_dev;
+  const int* P_prev_dev;   // parent count of the previous level (nullptr: none); 0 there means 0 here
+  int pdl;                 // host side: launch with programmatic stream serialization
   const int *p_req, *p_depth, *p_token; const uint64_t* p_hash;
   float T; uint64_t seed;
   int TV, ntiles, cap, S;
@@ -27,6 +29,7 @@ struct ScoreArgs {
 
 struct MergeArgs {
   int P; const int* P_dev; int K, ntiles, cap, S, mma; float T;
+  int pdl;   // host side: launch with programmatic stream serialization
   const float* rec; unsigned* thr; unsigned* slots;
   float *lse0, *lseT; int* top_tok; float* top_logit; int* draw_tok; float* draw_logit;
 };
@@ -43,7 +46,23 @@ size_t thr_bytes(const ts_ctx* ctx, int cap);
 cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,
                          const uint64_t* p_hash, float T, uint64_t seed, float* lse0, float* lseT, int* top_tok,
-                         float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st);
+                         float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st,
+                         bool pdl = false, const int* P_prev_dev = nullptr);
+
+// Kernel launch, optionally with programmatic stream serialization: the kernel may then start while the
+// kernel before it in the stream is still running, and must execute pdl_wait() before it touches anything
+// that kernel (or, transitively, an earlier one) wrote.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                                 Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out);
 cudaError_t score_mma_setup(ts_ctx* ctx);

@@ -28,6 +28,8 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
   const TIn* Ag = reinterpret_cast<const TIn*>(a.A);
   constexpr int VEC = Elem<TIn>::VEC;
   const bool vec_ok = (V % VEC) == 0;
+  pdl_wait();
+  pdl_launch_dependents();
   const int P = a.P_dev ? *a.P_dev : a.P;
   if (P <= 0) return;  // an empty level: nothing to stage
 
@@ -179,6 +181,8 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
   __shared__ float s_m[MERGE_WARPS], s_s0[MERGE_WARPS], s_sT[MERGE_WARPS];
   __shared__ float c_v[2][MERGE_CAP]; __shared__ int c_i[2][MERGE_CAP]; __shared__ float c_l[2][MERGE_CAP];
   __shared__ int c_n[2];
+  pdl_wait();               // the scoring launch's records and the level's parent count
+  pdl_launch_dependents();
   const int P = a.P_dev ? *a.P_dev : a.P;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float invT = a.T > 0.f ? 1.f / a.T : 1.f;
@@ -322,9 +326,10 @@ size_t thr_bytes(const ts_ctx* ctx, int cap) { return (size_t)cap * (2 + 2 * (si
 cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,
                          const uint64_t* p_hash, float T, uint64_t seed, float* lse0, float* lseT, int* top_tok,
-                         float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st) {
+                         float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st, bool pdl, const int* P_prev_dev) {
   const ts_config& c = ctx->cfg;
   ScoreArgs a{};
+  a.pdl = pdl ? 1 : 0; a.P_prev_dev = P_prev_dev;
   a.U = U; a.A = A; a.W = W; a.V = c.V; a.D = c.D; a.r = c.r; a.K = c.K; a.P = P; a.P_dev = P_dev;
   a.p_req = p_req; a.p_depth = p_depth; a.p_token = p_token; a.p_hash = p_hash; a.T = T; a.seed = seed;
   a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.cap = cap; a.S = ctx->use_mma ? MMA_S : 1; a.rec = rec; a.err = err;
@@ -336,16 +341,18 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
       e = launch_score_mma(ctx, a, st);
       if (e != cudaSuccess) return e;
     } else if (c.dt_U == TS_DTYPE_BF16) {
-      if (c.K <= 8) score_tile_kernel<__nv_bfloat16, RegLists<8>><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
-      else score_tile_kernel<__nv_bfloat16, MemLists><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
+      if (c.K <= 8) e = launch_kernel(score_tile_kernel<__nv_bfloat16, RegLists<8>>, a.ntiles, SCORE_THREADS, ctx->tile.smem, st, pdl, a);
+      else e = launch_kernel(score_tile_kernel<__nv_bfloat16, MemLists>, a.ntiles, SCORE_THREADS, ctx->tile.smem, st, pdl, a);
     } else {
-      if (c.K <= 8) score_tile_kernel<float, RegLists<8>><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
-      else score_tile_kernel<float, MemLists><<<a.ntiles, SCORE_THREADS, ctx->tile.smem, st>>>(a);
+      if (c.K <= 8) e = launch_kernel(score_tile_kernel<float, RegLists<8>>, a.ntiles, SCORE_THREADS, ctx->tile.smem, st, pdl, a);
+      else e = launch_kernel(score_tile_kernel<float, MemLists>, a.ntiles, SCORE_THREADS, ctx->tile.smem, st, pdl, a);
     }
   }
+  if (e != cudaSuccess) return e;
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   MergeArgs m{};
+  m.pdl = a.pdl;
   m.P = P; m.P_dev = P_dev; m.K = c.K; m.ntiles = a.ntiles; m.cap = cap; m.S = a.S; m.mma = ctx->use_mma ? 1 : 0; m.T = T;
   m.rec = rec; m.thr = a.thr; m.slots = a.slots;
   m.lse0 = lse0; m.lseT = lseT; m.top_tok = top_tok; m.top_logit = top_logit; m.draw_tok = draw_tok; m.draw_logit = draw_logit;
@@ -354,9 +361,10 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
   if (blocks < 1) blocks = 1;
   {
     ProfScope ps(ctx, K_MERGE, st);
-    if (c.K <= 8) merge_kernel<8><<<blocks, MERGE_THREADS, 0, st>>>(m);
-    else merge_kernel<16><<<blocks, MERGE_THREADS, 0, st>>>(m);
+    if (c.K <= 8) e = launch_kernel(merge_kernel<8>, blocks, MERGE_THREADS, 0, st, pdl, m);
+    else e = launch_kernel(merge_kernel<16>, blocks, MERGE_THREADS, 0, st, pdl, m);
   }
+  if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }
 

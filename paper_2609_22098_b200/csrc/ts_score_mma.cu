@@ -47,8 +47,10 @@ template <class Lists>
 __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma) {
   extern __shared__ unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int P = a.P_dev ? *a.P_dev : a.P;
-  if (P <= 0) return;  // an empty level: uniform exit before anything is allocated
+  // The preamble below (shared-memory carve-up, tensor-memory allocation, barriers, bulk loads of W, noise
+  // table) reads nothing an earlier kernel of the stream wrote, so in a chained launch it runs while the
+  // previous kernel is still finishing.  When the level before this one was empty, this one is too.
+  if (a.P_prev_dev && *a.P_prev_dev <= 0) { pdl_wait(); return; }
 
   const int r = a.r, rp = (r + 63) / 64 * 64, V = a.V, TV = a.TV, K = a.K;
   const int tile = blockIdx.x, t0 = tile * TV, tlen = min(TV, V - t0);
@@ -119,9 +121,12 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
   if (warp == 0) DBG(3);
+  pdl_wait();                // parent lists and the level's parent count come from the previous kernel
+  pdl_launch_dependents();
+  const int P = a.P_dev ? *a.P_dev : a.P;   // may be 0: an empty level only tears down
 
   const int R = mma_replicas(P), rsh = R == 4 ? 2 : (R == 2 ? 1 : 0);
-  const int ngroups = R > 1 ? 1 : (P + 127) / 128;
+  const int ngroups = P <= 0 ? 0 : (R > 1 ? 1 : (P + 127) / 128);
   const int nblk = (tlen + BLK_N - 1) / BLK_N;
   const float T = a.T, invT = T > 0.f ? 1.f / T : 1.f;
   const int rw = rec_words(K);
@@ -289,8 +294,9 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   }
   // ---- tear-down -----------------------------------------------------------------------------------
   if (warp == 0) DBG(5);
-  if (use_tma && tid == 0 && *s_abort) {
-    // gave up somewhere: do not leave while a bulk load may still be writing this CTA's shared memory
+  if (use_tma && tid == 0 && (*s_abort || P <= 0)) {
+    // gave up somewhere, or nothing to score: do not leave while a bulk load may still be writing this
+    // CTA's shared memory
     for (int nb = 0; nb < nblk_w; ++nb) {
       bool done = false;
       for (uint32_t i = 0; i < WAIT_LIMIT && !done; ++i) { done = mbar_try_wait(w_full + nb, 0); if (!done) __nanosleep(100); }
@@ -390,9 +396,10 @@ cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t
   const int use_tma = w_tensor_map(c, a.W) ? 1 : 0;
   CUtensorMap tm;
   memcpy(&tm, c->tmapW, sizeof(tm));
-  if (a.K <= 8) score_mma_kernel<RegLists<8>><<<a.ntiles, MMA_THREADS, ctx->tile.smem, st>>>(a, tm, use_tma);
-  else score_mma_kernel<MemLists><<<a.ntiles, MMA_THREADS, ctx->tile.smem, st>>>(a, tm, use_tma);
-  return cudaGetLastError();
+  cudaError_t e;
+  if (a.K <= 8) e = launch_kernel(score_mma_kernel<RegLists<8>>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma);
+  else e = launch_kernel(score_mma_kernel<MemLists>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace ts
