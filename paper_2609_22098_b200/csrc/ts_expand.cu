@@ -46,6 +46,7 @@ __device__ __forceinline__ void request_caps(const ExpandArgs& a, int b, int& K_
 }
 
 __global__ void expand_init_kernel(ExpandArgs a) {
+  pdl_wait();                // whatever ran before in the stream may still be reading what this kernel resets
   pdl_launch_dependents();   // the first scoring launch may run its preamble beside this kernel
   const int b = blockIdx.x;
   // pruning state of the scoring launches: the threshold words, then one word per slot (the slots sit
@@ -407,8 +408,9 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   a.thr = thr_base(ctx, (float*)(ws + L.rec), L.rec_cap);
   a.thr_head = 2 * L.rec_cap; a.thr_words = a.thr_head + 2 * L.rec_cap * c.K;   // words to clear, not their span
 
-  { ProfScope ps(ctx, K_INIT, st); expand_init_kernel<<<B > 296 ? B : 296, 256, 0, st>>>(a); }
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e0;
+  { ProfScope ps(ctx, K_INIT, st); e0 = launch_kernel(expand_init_kernel, B > 296 ? B : 296, 256, 0, st, true, a); }
+  cudaError_t e = e0 != cudaSuccess ? e0 : cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(init)", e);
   const size_t level_smem = (size_t)(c.Nmax + c.Nmax * c.K) * sizeof(Entry);
   if (level_smem > 48 * 1024) {

@@ -51,6 +51,7 @@ __global__ void __launch_bounds__(ZT) zrow_stats_kernel(const TIn* Z, const int6
   // One CTA per target row, one sweep: every thread keeps a running (max, arg-max, sum of exp((z-max)/T))
   // over its share of the row, four 16-byte loads in flight, and the block folds the triples.
   __shared__ float s_v[ZT / 32]; __shared__ int s_i[ZT / 32]; __shared__ float s_s[ZT / 32];
+  pdl_wait();   // the target logits (and the tree) may come from the kernel just before this one
   const int64_t rows = z_row_off[B];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int VEC = Elem<TIn>::VEC;
@@ -1079,14 +1080,15 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
 
   const int max_rows = B * (c.Nmax + 1);
   int grid_rows = max_rows < 8 * ctx->num_sms ? max_rows : 8 * ctx->num_sms;
+  cudaError_t ez;
   {
     ProfScope ps(ctx, K_ZROWS, st);
     if (c.dt_Z == TS_DTYPE_BF16)
-      zrow_stats_kernel<__nv_bfloat16><<<grid_rows, ZT, 0, st>>>((const __nv_bfloat16*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+      ez = launch_kernel(zrow_stats_kernel<__nv_bfloat16>, grid_rows, ZT, 0, st, true, (const __nv_bfloat16*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
     else
-      zrow_stats_kernel<float><<<grid_rows, ZT, 0, st>>>((const float*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+      ez = launch_kernel(zrow_stats_kernel<float>, grid_rows, ZT, 0, st, true, (const float*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
   }
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = ez != cudaSuccess ? ez : cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(rows)", e);
   if (T == 0.f) {
     { ProfScope ps(ctx, K_GREEDY, st); verify_greedy_kernel<<<B, 128, 0, st>>>(a); }
