@@ -64,6 +64,7 @@ struct ts_ctx {
   alignas(64) unsigned char tmapW[128];
   const void* tmapW_ptr;
   int tma_state;   // 0 not tried yet, 1 encoder found, -1 unavailable
+  int walk_pdl;    // -1: the driver refused a cooperative launch with programmatic serialization
 };
 
 namespace ts {

@@ -47,11 +47,15 @@ constexpr int ZT = 512;  // threads per target row in the row-statistics kernel
 // ------------------------------------------------------------------------------------------------
 template <typename TIn>
 __global__ void __launch_bounds__(ZT) zrow_stats_kernel(const TIn* Z, const int64_t* z_row_off, int B, int V, float T,
-                                                       float* z_max, int* z_arg, float* z_logs) {
+                                                       float* z_max, int* z_arg, float* z_logs, unsigned* walk_barrier) {
   // One CTA per target row, one sweep: every thread keeps a running (max, arg-max, sum of exp((z-max)/T))
   // over its share of the row, four 16-byte loads in flight, and the block folds the triples.
   __shared__ float s_v[ZT / 32]; __shared__ int s_i[ZT / 32]; __shared__ float s_s[ZT / 32];
   pdl_wait();   // the target logits (and the tree) may come from the kernel just before this one
+  pdl_launch_dependents();
+  // the walk's barrier words start at zero (done here rather than by a memset, which would sit between
+  // this kernel and the walk in the stream and keep the walk from starting its preamble early)
+  if (walk_barrier && blockIdx.x == 0 && threadIdx.x < 16) walk_barrier[threadIdx.x] = 0u;
   const int64_t rows = z_row_off[B];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int VEC = Elem<TIn>::VEC;
@@ -944,7 +948,7 @@ template <typename TIn, bool MMA>
 __global__ void __launch_bounds__(WT, 1) verify_walk_kernel(const VerifyArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma) {
   extern __shared__ __align__(16) unsigned char w_raw[];
   WalkTc tc{};
-  if (!MMA) { walk_body<TIn, false>(a, tc, w_raw); return; }
+  if (!MMA) { pdl_wait(); walk_body<TIn, false>(a, tc, w_raw); return; }
   const int tid = threadIdx.x, warp = tid >> 5;
   const int r = a.r, rp = (r + 63) / 64 * 64;
   const int t0 = blockIdx.x * a.vt_TV, tlen = min(a.vt_TV, a.V - t0);
@@ -992,6 +996,7 @@ __global__ void __launch_bounds__(WT, 1) verify_walk_kernel(const VerifyArgs a, 
   __syncthreads();
   tc_fence_after();
   tc.tmem_base = *s_tmem;
+  pdl_wait();   // row statistics and the tree come from earlier kernels; W (loaded above) does not
   bool ok = true;
   if (use_tma) {
     // the whole range must have landed before anything reads it (the rescans read it with plain loads)
@@ -1084,9 +1089,9 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
   {
     ProfScope ps(ctx, K_ZROWS, st);
     if (c.dt_Z == TS_DTYPE_BF16)
-      ez = launch_kernel(zrow_stats_kernel<__nv_bfloat16>, grid_rows, ZT, 0, st, true, (const __nv_bfloat16*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+      ez = launch_kernel(zrow_stats_kernel<__nv_bfloat16>, grid_rows, ZT, 0, st, true, (const __nv_bfloat16*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs, T > 0.f ? a.barrier : (unsigned*)nullptr);
     else
-      ez = launch_kernel(zrow_stats_kernel<float>, grid_rows, ZT, 0, st, true, (const float*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs);
+      ez = launch_kernel(zrow_stats_kernel<float>, grid_rows, ZT, 0, st, true, (const float*)Z, z_row_off, B, c.V, T, z_max, z_arg, z_logs, T > 0.f ? a.barrier : (unsigned*)nullptr);
   }
   cudaError_t e = ez != cudaSuccess ? ez : cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(rows)", e);
@@ -1096,8 +1101,6 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
     if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(greedy)", e);
     return TS_OK;
   }
-  e = cudaMemsetAsync(a.barrier, 0, 64, st);
-  if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(memset)", e);
   size_t w_bytes = (size_t)c.r * ctx->vt_TV * (c.dt_W == TS_DTYPE_BF16 ? 2 : 4);
   a.w_smem = (w_bytes + 32 * 1024 <= (size_t)ctx->max_smem) ? 1 : 0;
   // tensor-core reductions: bf16 everywhere, the range of W in operand layout plus the A tile within shared memory
@@ -1115,7 +1118,24 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
                        : (c.dt_Z == TS_DTYPE_BF16 ? (const void*)verify_walk_kernel<__nv_bfloat16, false>
                                                   : (const void*)verify_walk_kernel<float, false>);
   if (mma) w_bytes = mma_bytes;
-  { ProfScope ps(ctx, K_WALK, st); e = cudaLaunchCooperativeKernel(fn, dim3(a.vt_n), dim3(WT), kargs, (mma || a.w_smem) ? w_bytes : 0, st); }
+  {
+    ProfScope ps(ctx, K_WALK, st);
+    // cooperative (the grid barriers need every CTA resident) and, where the driver takes both attributes,
+    // chained to the row statistics so that the W load and the tensor-memory allocation run beside them
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.vt_n); cfg.blockDim = dim3(WT); cfg.dynamicSmemBytes = (mma || a.w_smem) ? w_bytes : 0; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative; attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = ctx->walk_pdl >= 0 ? 2 : 1;
+    e = cudaLaunchKernelExC(&cfg, fn, kargs);
+    if (e != cudaSuccess && cfg.numAttrs == 2) {   // not accepted together: remember, and launch cooperative only
+      (void)cudaGetLastError();
+      ctx->walk_pdl = -1;
+      cfg.numAttrs = 1;
+      e = cudaLaunchKernelExC(&cfg, fn, kargs);
+    }
+  }
   if (e != cudaSuccess) return set_cuda_error("ts_verify_tree(walk)", e);
   { ProfScope ps(ctx, K_CHECK, st); verify_check_kernel<<<(B + 127) / 128, 128, 0, st>>>(a); }
   e = cudaGetLastError();
