@@ -222,24 +222,9 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
   st.s0 += a0;
   st.sT += two ? aT : a0;
   if (valid) TS_SCAN_MARK(1);
-  // top-K logits: a token below the launch-wide bound cannot be among the parent's K best
-  if (cm > st.thrL && cm >= gL) {
-    uint32_t mk = 0;
-#pragma unroll
-    for (int i = 0; i < CHUNK; ++i) mk |= (uint32_t)(i < valid && l[i] > st.thrL && l[i] >= gL) << i;
-#pragma unroll 1
-    while (mk) {
-      const int i = __ffs(mk) - 1;
-      mk &= mk - 1;
-      const float li = pick16(l, i);
-      if (liveL) gL = fmaxf(gL, dec_f(*liveL));
-      if (li > st.thrL && li >= gL) {
-        st.thrL = st.L.insert_top(li, v0 + i);
-        // publish at once: early in a launch every piece is waiting for the first bounds
-        if (li > st.bestL) { st.bestL = li; publish(gl, li); }
-      }
-    }
-  }
+  // the chunk's best logit is a candidate for the top-K list (it is inserted further down): publishing it
+  // right away costs nothing and gives the other pieces of the launch their first logit bounds early
+  if (cm > st.bestL && cm > st.thrL && cm >= gL) { st.bestL = cm; publish(gl, cm); }
   if (valid) TS_SCAN_MARK(2);
   if (T > 0.f) {
     // high half of each token's uniform: one generator call per eight tokens
@@ -288,6 +273,27 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
       if (key > st.thrK && key >= gK) {
         st.thrK = st.L.insert_key(key, v0 + i, li);
         if (key > st.bestK) { st.bestK = key; publish(gk, key); }
+      }
+    }
+  }
+  // top-K logits, after the keys: in the first chunks of a launch the key section is the longer one and
+  // the one whose published values the other pieces wait for.  A token below the launch-wide bound cannot
+  // be among the parent's K best.
+  if (liveL) gL = fmaxf(gL, dec_f(*liveL));
+  if (cm > st.thrL && cm >= gL) {
+    uint32_t mk = 0;
+#pragma unroll
+    for (int i = 0; i < CHUNK; ++i) mk |= (uint32_t)(i < valid && l[i] > st.thrL && l[i] >= gL) << i;
+#pragma unroll 1
+    while (mk) {
+      const int i = __ffs(mk) - 1;
+      mk &= mk - 1;
+      const float li = pick16(l, i);
+      if (liveL) gL = fmaxf(gL, dec_f(*liveL));
+      if (li > st.thrL && li >= gL) {
+        st.thrL = st.L.insert_top(li, v0 + i);
+        // publish at once: early in a launch every piece is waiting for the first bounds
+        if (li > st.bestL) { st.bestL = li; publish(gl, li); }
       }
     }
   }

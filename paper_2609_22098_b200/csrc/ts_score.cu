@@ -261,9 +261,8 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
       a.lseT[p] = a.T > 0.f ? gm * invT + logf(gT) : gm + logf(g0);
     }
     // leave the launch-wide pruning state of this parent clean for the next launch
-#ifndef TS_DEBUG_KEEP_BOUNDS
     if (tid < 2 * K) a.slots[(((size_t)(tid / K) * a.cap + p) * K + tid % K) * SLOT_STRIDE] = 0u;
-#endif
+    if (tid < 2) a.thr[(size_t)tid * a.cap + p] = 0u;   // and its condensed copy
     const bool fits = c_n[0] <= MERGE_CAP && c_n[1] <= MERGE_CAP;   // uniform: read after the barrier above
     if (fits) {
       // the usual case: a few dozen candidates survive the bounds; half of the block ranks each list
@@ -398,10 +397,8 @@ extern "C" int32_t ts_score_parents(ts_ctx* ctx, const void* U, const void* A, c
   if (ws_bytes < L.total) return set_error(TS_ERR_WORKSPACE, "ts_score_parents: workspace too small");
   if (P == 0) return TS_OK;
   cudaError_t e = cudaMemsetAsync((char*)ws + L.err, 0, 16, (cudaStream_t)stream);
-#ifndef TS_DEBUG_KEEP_BOUNDS
   if (e == cudaSuccess)
     e = cudaMemsetAsync(thr_base(ctx, (float*)((char*)ws + L.rec), L.rec_cap), 0, thr_bytes(ctx, L.rec_cap), (cudaStream_t)stream);
-#endif
   if (e != cudaSuccess) return set_cuda_error("ts_score_parents(memset)", e);
   e = launch_score(ctx, (float*)((char*)ws + L.rec), L.rec_cap, (int*)((char*)ws + L.err), U, A, W, P, nullptr,
                                parent_req, parent_depth, parent_token, parent_hash, T, seed, lse0, lseT, top_tok,

@@ -243,24 +243,40 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       const int per = R > 1 ? 128 / R : 128;
       for (uint32_t spin = 0; spin < WAIT_LIMIT; ++spin) {
         if (*s_done >= (g + 1) * EPI_WARPS || *s_abort) break;
-        for (int rr = lane; rr < per; rr += 32) {
-          const int p = R > 1 ? rr : g * 128 + rr;
-          if (p >= P) continue;
-          const unsigned* sl = a.slots + (size_t)p * K * SLOT_STRIDE;
-          const unsigned* sk = a.slots + ((size_t)a.cap + p) * K * SLOT_STRIDE;
-          // all 2K loads in flight together: one L2 round trip per row, not one per slot
-          unsigned vL[KMAX], vK[KMAX];
+        // (1) This CTA condenses the slots of the parents it is responsible for (parent p belongs to tile
+        // p mod ntiles) into two words per parent; (2) every CTA reads the condensed words of its rows.
+        // Only one CTA per parent reads the slot lines, which every piece of the launch is hitting with
+        // atomics.  The loads of both steps are issued together: one memory round trip per pass.
+        const int p_lo = R > 1 ? 0 : g * 128, p_hi = min(P, p_lo + per);
+        const int nt = a.ntiles;
+        const int p_own = p_lo + ((tile - p_lo % nt + nt) % nt);   // first parent of this group this CTA owns
+        const int which = lane >> 4, j = lane & 15;                  // lanes 0..15: logit slots, 16..31: key slots
+        unsigned v = 0xFFFFFFFFu;
+        if (p_own < p_hi && j < K) v = __ldcg(a.slots + (((size_t)which * a.cap + p_own) * K + j) * SLOT_STRIDE);
+        unsigned rL[4], rK[4];
 #pragma unroll
-          for (int j = 0; j < KMAX; ++j) {
-            vL[j] = j < K ? __ldcg(sl + j * SLOT_STRIDE) : 0xFFFFFFFFu;
-            vK[j] = j < K ? __ldcg(sk + j * SLOT_STRIDE) : 0xFFFFFFFFu;
-          }
-          unsigned mL = vL[0], mK = vK[0];
-#pragma unroll
-          for (int j = 1; j < KMAX; ++j) { mL = min(mL, vL[j]); mK = min(mK, vK[j]); }
-          s_thr[(g & 1) * 256 + rr] = mL; s_thr[(g & 1) * 256 + 128 + rr] = mK;
+        for (int k = 0; k < 4; ++k) {
+          const int rr = lane + 32 * k, p = R > 1 ? rr : g * 128 + rr;
+          const bool in = rr < per && p < P;
+          rL[k] = in ? __ldcg(a.thr + p) : 0u;
+          rK[k] = in ? __ldcg(a.thr + (size_t)a.cap + p) : 0u;
         }
-        __nanosleep(1000);
+#pragma unroll
+        for (int off = 8; off > 0; off >>= 1) v = min(v, __shfl_xor_sync(0xFFFFFFFFu, v, off));
+        if (p_own < p_hi && j == 0) __stcg(a.thr + (size_t)which * a.cap + p_own, v);
+        for (int p = p_own + nt; p < p_hi; p += nt) {   // more parents than tiles: the rest, one at a time
+          unsigned w = 0xFFFFFFFFu;
+          if (j < K) w = __ldcg(a.slots + (((size_t)which * a.cap + p) * K + j) * SLOT_STRIDE);
+#pragma unroll
+          for (int off = 8; off > 0; off >>= 1) w = min(w, __shfl_xor_sync(0xFFFFFFFFu, w, off));
+          if (j == 0) __stcg(a.thr + (size_t)which * a.cap + p, w);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int rr = lane + 32 * k, p = R > 1 ? rr : g * 128 + rr;
+          if (rr < per && p < P) { s_thr[(g & 1) * 256 + rr] = rL[k]; s_thr[(g & 1) * 256 + 128 + rr] = rK[k]; }
+        }
+        if (spin >= 24u) __nanosleep(500);   // poll flat out while the launch warms up, then back off
       }
       __syncwarp();
     }
