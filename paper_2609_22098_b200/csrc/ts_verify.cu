@@ -187,16 +187,19 @@ __device__ __forceinline__ double p_of(const VerifyArgs& a, int64_t row, int w) 
 }
 
 // Scalar state machine of one request, run by one warp of the request's owner CTA.
-// need: 0 walking, 1 reduction after a rejection, 4 reduction for the bonus draw, 2 range rescan, 3 finished.
+// need: 0 walking, 1 reduction after a rejection, 4 reduction for the bonus draw, 5 walk over (bonus token
+// still to be drawn), 2 range rescan, 3 finished.  The bonus draws of all requests are left to the end of
+// the kernel (closing == true): locating the range and rescanning it would otherwise hold up, at every
+// step, the requests that are still walking.
 // Lane 0 decides; at every visited node the lanes fetch the accept-test inputs of all its children at
 // once (one memory round trip per node), and the warp folds range sums together.
 template <typename TIn>
-__device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
+__device__ void advance(const VerifyArgs& a, int b, int lane, int parity, bool closing) {
   VerifyState* gst = a.state + b;
   const int N = a.N;
   const size_t nb = (size_t)b * N;
   const int need_in = gst->need;
-  if (need_in == 3) return;
+  if (need_in == 3 || (need_in == 5 && !closing)) return;
   // ---- fold in the reduction that just ran -------------------------------------------------
   double fsum = 0.0;
   if (need_in == 1 || need_in == 4) {
@@ -230,8 +233,8 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
       a.acc_len[b] = st.acc;
       a.flags[b] |= (uint32_t)min(st.npass, 0xFFFF) << 8;   // bits 8..23: reductions this walk needed
       st.need = 3;
-      atomicSub(a.ctr + 4, 1);
     }
+    if (st.need == 5) go_scan = 1;   // closing: draw the bonus token now
   }
   int walking = __shfl_sync(0xFFFFFFFFu, lane == 0 ? (st.need == 0) : 0, 0);
   while (walking) {
@@ -279,7 +282,9 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity) {
     walking = __shfl_sync(0xFFFFFFFFu, again, 0);
   }
   go_scan = __shfl_sync(0xFFFFFFFFu, go_scan, 0);
-  if (go_scan) {
+  if (go_scan && !closing) {
+    if (lane == 0) { st.need = 5; atomicSub(a.ctr + 4, 1); }   // one walker fewer
+  } else if (go_scan) {
     // locate the vocabulary range holding the bonus token: cumulative corrected range sums
     const int cur = __shfl_sync(0xFFFFFFFFu, st.cur, 0), nf = __shfl_sync(0xFFFFFFFFu, st.nf, 0);
     const double C = __shfl_sync(0xFFFFFFFFu, st.C, 0), Zj = __shfl_sync(0xFFFFFFFFu, st.Zj, 0);
@@ -706,11 +711,15 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
   for (int b = blockIdx.x; b < a.B; b += nblocks)
     if (tid == 0 && a.state[b].need == 3) atomicSub(a.ctr + 4, 1);
 
+  // stage 0: walk steps until every request's walk is over; stage 1: one step that locates and rescans the
+  // range of every bonus token; stage 2: the owners commit the results
+  int stage = 0;
   for (int step = 0; step < a.max_steps; ++step) {
     const int par = step & 1;
     DBGW(step, 0);
     // ---- phase A: scalar walks of the requests this CTA owns, one warp each ----------------------
-    for (int b = blockIdx.x + warp * (int)nblocks; b < a.B; b += (WT / 32) * (int)nblocks) advance<TIn>(a, b, lane, par);
+    for (int b = blockIdx.x + warp * (int)nblocks; b < a.B; b += (WT / 32) * (int)nblocks) advance<TIn>(a, b, lane, par, stage > 0);
+    if (stage == 2) return true;
     DBGW(step, 1);
     if (!grid_barrier(a.barrier, nblocks, gen)) return false;
     DBGW(step, 2);
@@ -933,7 +942,8 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
     if (!grid_barrier(a.barrier, nblocks, gen)) return false;
     DBGW(step, 5);
     if (threadIdx.x == 0 && blockIdx.x == 0 && step < 64) { DBGW(step, 6); }
-    if (left == 0 && nwk == 0 && nsc == 0) return true;
+    if (stage == 1) stage = 2;
+    else if (left == 0 && nwk == 0) stage = 1;   // uniform over the grid: both were read after the step's first barrier
   }
   // steps ran out
   for (int b = blockIdx.x; b < a.B; b += nblocks)
@@ -1081,7 +1091,7 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
   a.child_first = (int*)(ws + L.vf_child); a.child_cnt = a.child_first + (size_t)B * (c.Nmax + 1);
   a.edge_px = (double*)(ws + L.vf_edge); a.edge_qx = a.edge_px + (size_t)B * c.Nmax; a.edge_u = a.edge_qx + (size_t)B * c.Nmax;
   a.wk_list = (int*)(ws + L.vf_lists); a.sc_list = a.wk_list + 2 * (size_t)B; a.ctr = a.sc_list + 2 * (size_t)B;
-  a.vt_TV = ctx->vt_TV; a.vt_n = ctx->vt_n; a.max_steps = 2 * (c.Nmax + c.D) + 8;
+  a.vt_TV = ctx->vt_TV; a.vt_n = ctx->vt_n; a.max_steps = 2 * (c.Nmax + c.D) + 10;
 
   const int max_rows = B * (c.Nmax + 1);
   int grid_rows = max_rows < 8 * ctx->num_sms ? max_rows : 8 * ctx->num_sms;
