@@ -292,6 +292,16 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity, bool c
     const double u = u01(stream_words(a.seed, b, hv, STREAM_BONUS, 0u).x);
     const double target = u * Zj;
     double carry = 0.0; int found = -1; double before = 0.0; int last_pos = -1;
+    // correction of tested sibling i (lane i): its range, and the difference between the residual it kept
+    // and the one the last reduction gave it (the state in global memory is current: this runs in a later
+    // step than the one that wrote it)
+    int f_tile = -1; double f_delta = 0.0;
+    if (lane < nf) {
+      const int fxi = gst->fx[lane];
+      const double fpi = gst->fp[lane], fqi = gst->fq[lane], fCi = gst->fC[lane];
+      f_tile = fxi / a.vt_TV;
+      f_delta = fmax(fpi - fCi * fqi, 0.0) - fmax(fpi - C * fqi, 0.0);
+    }
     // the first 256 range sums are requested together (one memory round trip for the usual grid sizes)
     float pre[8];
 #pragma unroll
@@ -306,10 +316,9 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity, bool c
         pt = (double)pv;
       } else if (t < a.vt_n) pt = (double)__ldcg(a.part + (size_t)b * a.vt_n + t);
       for (int i = 0; i < nf; ++i) {   // tested siblings keep the residual they had when tested
-        const int fxi = __shfl_sync(0xFFFFFFFFu, st.fx[i], 0);
-        const double fpi = __shfl_sync(0xFFFFFFFFu, st.fp[i], 0), fqi = __shfl_sync(0xFFFFFFFFu, st.fq[i], 0);
-        const double fCi = __shfl_sync(0xFFFFFFFFu, st.fC[i], 0);
-        if (t < a.vt_n && fxi / a.vt_TV == t) pt += fmax(fpi - fCi * fqi, 0.0) - fmax(fpi - C * fqi, 0.0);
+        const int ti = __shfl_sync(0xFFFFFFFFu, f_tile, i);
+        const double di = __shfl_sync(0xFFFFFFFFu, f_delta, i);
+        if (t == ti) pt += di;
       }
       if (pt < 0.0) pt = 0.0;
       double inc = pt;
@@ -874,10 +883,14 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
     // range rescans for bonus tokens that fall into this CTA's range: the residual of every token of
     // the range is evaluated once (tokens dealt round-robin to the threads: row i of the range holds
     // tokens i*WT .. i*WT+WT-1), then prefix sums in token order locate the crossing
-    for (int si = 0; si < nsc; ++si) {
+    // Rescans are dealt round-robin to the CTAs (several bonus tokens often fall into one range, and a
+    // rescan needs nothing of the CTA that owns the range except its columns of W, which any CTA can read
+    // from global memory).
+    for (int si = blockIdx.x; si < nsc; si += (int)nblocks) {
       const int b = __ldcg(a.sc_list + par * a.B + si);
       const VerifyState& st = a.state[b];
-      if (st.scan_tile != (int)blockIdx.x) continue;
+      const int s_lo = st.scan_tile * a.vt_TV, s_hi = min(a.V, s_lo + a.vt_TV);
+      const bool own = st.scan_tile == (int)blockIdx.x;   // this CTA's own range: W is in shared memory
       const int v = st.cur;
       const int64_t row = a.z_row_off[b] + v + 1;
       const int dep = v < 0 ? 0 : a.depth[(size_t)b * N + v];
@@ -890,11 +903,11 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
       for (int k = tid; k < a.r; k += WT) sb_a[k] = Elem<TIn>::to_f(Ag[(size_t)ptok * a.r + k]);
       if (tid == 0) { s_found = 0x7FFFFFFF; s_last = -1; }
       __syncthreads();
-      const int len = v_hi - v_lo;
+      const int len = s_hi - s_lo;
       const int nrow = (len + WT - 1) / WT;
       double carry = 0.0;
       for (int i = 0; i < nrow; ++i) {
-        const int o = i * WT + tid, w = v_lo + o;
+        const int o = i * WT + tid, w = s_lo + o;
         double rw = 0.0;
         if (o < len) {
           double Cw = C;
@@ -903,14 +916,14 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
           double q = 0.0;
           if (Cw != 0.0) {
             float acc = Elem<TIn>::to_f(reinterpret_cast<const TIn*>(a.U)[((size_t)b * a.D + dep) * a.V + w]);
-            if (MMA) {
+            if (MMA && own) {
               // the range's W columns sit in the tensor-core operand layout: 64-token slabs of [rp][128 B],
               // 16-byte chunk j of row k at chunk j ^ (k & 7)
               const unsigned char* wsl = tc.Ws + (size_t)(o >> 6) * tc.slab_bytes + (o & 7) * 2;
               const int j = (o & 63) >> 3;
               for (int k = 0; k < a.r; ++k)
                 acc = fmaf(sb_a[k], __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(wsl + k * 128 + ((j ^ (k & 7)) << 4))), acc);
-            } else if (ws_ok) { for (int k = 0; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Ws[(size_t)k * a.vt_TV + o]), acc); }
+            } else if (ws_ok && own) { for (int k = 0; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Ws[(size_t)k * a.vt_TV + o]), acc); }
             else { for (int k = 0; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Wg[(size_t)k * a.V + w]), acc); }
             q = exp((double)acc / (double)a.T - lseT);
           }
@@ -933,7 +946,7 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
       if (tid == 0) {
         int o = s_found;
         if (o == 0x7FFFFFFF) o = s_last >= 0 ? s_last : len - 1;   // rounding pushed the crossing past the range
-        a.state[b].result = v_lo + o;
+        a.state[b].result = s_lo + o;
       }
       __syncthreads();
     }
