@@ -113,6 +113,7 @@ struct VerifyState {
   int row_node;   // node whose rows the pass reads
   int result;     // token found by the range rescan
   int npass;      // vocabulary reductions this request has asked for
+  int cfirst, ccnt;  // first child and child count of the current node (saves the walk a dependent load)
   int pad_;
   double C, Zj, Qused, target, before;
   double passC;   // C of the requested pass

@@ -199,7 +199,15 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity, bool c
   const int N = a.N;
   const size_t nb = (size_t)b * N;
   const int need_in = gst->need;
+  const int cur0 = gst->cur, cf0 = gst->cfirst, cc0 = gst->ccnt;
   if (need_in == 3 || (need_in == 5 && !closing)) return;
+  // accept-test inputs of the current node's children, requested together with everything else this step
+  // needs (the range sums, the state): one memory round trip instead of a chain of three
+  int x0 = -1; double px0 = 0.0, qx0 = 1.0, ux0 = 0.0;
+  if ((need_in == 0 || need_in == 1 || need_in == 4) && lane < cc0) {
+    x0 = a.tok[nb + cf0 + lane];
+    px0 = a.edge_px[nb + cf0 + lane]; qx0 = a.edge_qx[nb + cf0 + lane]; ux0 = a.edge_u[nb + cf0 + lane];
+  }
   // ---- fold in the reduction that just ran -------------------------------------------------
   double fsum = 0.0;
   if (need_in == 1 || need_in == 4) {
@@ -237,19 +245,26 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity, bool c
     if (st.need == 5) go_scan = 1;   // closing: draw the bonus token now
   }
   int walking = __shfl_sync(0xFFFFFFFFu, lane == 0 ? (st.need == 0) : 0, 0);
+  bool at_start = true;   // still at the node the step began at: its children were fetched above
   while (walking) {
     // inputs of every child's accept test at the current node, one child per lane
     const int v = __shfl_sync(0xFFFFFFFFu, st.cur, 0);
-    const int first = a.child_first[(size_t)b * (N + 1) + v + 1], m = a.child_cnt[(size_t)b * (N + 1) + v + 1];
-    double px = 0.0, qx = 1.0; int x = -1;
-    double ux = 0.0;
-    if (lane < m) {   // computed for every edge when the walk was set up
-      x = a.tok[nb + first + lane];
-      px = a.edge_px[nb + first + lane]; qx = a.edge_qx[nb + first + lane]; ux = a.edge_u[nb + first + lane];
+    int first = cf0, m = cc0;
+    double px = px0, qx = qx0; int x = x0;
+    double ux = ux0;
+    if (!at_start || v != cur0) {
+      first = a.child_first[(size_t)b * (N + 1) + v + 1]; m = a.child_cnt[(size_t)b * (N + 1) + v + 1];
+      px = 0.0; qx = 1.0; x = -1; ux = 0.0;
+      if (lane < m) {   // computed for every edge when the walk was set up
+        x = a.tok[nb + first + lane];
+        px = a.edge_px[nb + first + lane]; qx = a.edge_qx[nb + first + lane]; ux = a.edge_u[nb + first + lane];
+      }
+      if (lane == 0) { st.cfirst = first; st.ccnt = m; }
     }
+    at_start = false;
     // lane 0 runs the sibling chain at this node until it accepts, needs a reduction, or runs out
     int again = 0;
-    for (int j = 0; j < 32; ++j) {   // m <= K <= 16
+    for (int j = __shfl_sync(0xFFFFFFFFu, st.j, 0); j < 32; ++j) {   // m <= K <= 16; earlier siblings were tested in earlier steps
       const double pxj = __shfl_sync(0xFFFFFFFFu, px, j), qxj = __shfl_sync(0xFFFFFFFFu, qx, j);
       const int xj = __shfl_sync(0xFFFFFFFFu, x, j);
       const double uj = __shfl_sync(0xFFFFFFFFu, ux, j);
@@ -340,8 +355,7 @@ __device__ void advance(const VerifyArgs& a, int b, int lane, int parity, bool c
     }
   }
   if (lane == 0) {
-    *gst = st;
-    __threadfence();
+    *gst = st;   // made visible to the other CTAs by the fence of the grid barrier that follows
     if (st.need == 1 || st.need == 4) a.wk_list[parity * a.B + atomicAdd(a.ctr + parity, 1)] = b;
     if (st.need == 1 || st.need == 4) gst->npass = st.npass + 1;
     else if (st.need == 2) a.sc_list[parity * a.B + atomicAdd(a.ctr + 2 + parity, 1)] = b;
@@ -702,11 +716,13 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
           a.edge_stat[nb + i] = (float)exp(fmin(lr, 0.0));
         }
       }
+    __syncthreads();   // the root's child range is read below
     if (tid == 0) {
       VerifyState& st = a.state[b];
       st.cur = -1; st.j = 0; st.acc = 0; st.need = 0; st.nf = 0; st.scan_tile = -1; st.row_node = -1; st.result = -1;
       st.C = 0.0; st.Zj = 1.0; st.Qused = 0.0; st.target = 0.0; st.before = 0.0; st.passC = 0.0; st.partsC = -1.0;
       st.npass = 0; st.pad_ = 0;
+      st.cfirst = a.child_first[cbase]; st.ccnt = a.child_cnt[cbase];   // children of the root
       a.flags[b] = 0u;
       a.status[b] = okn ? TS_OK : TS_ERR_INVALID;
       if (!okn) { st.need = 3; a.acc_len[b] = 0; a.bonus[b] = -1; }
