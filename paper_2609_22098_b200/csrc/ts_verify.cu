@@ -940,7 +940,19 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
               for (int k = 0; k < a.r; ++k)
                 acc = fmaf(sb_a[k], __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(wsl + k * 128 + ((j ^ (k & 7)) << 4))), acc);
             } else if (ws_ok && own) { for (int k = 0; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Ws[(size_t)k * a.vt_TV + o]), acc); }
-            else { for (int k = 0; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Wg[(size_t)k * a.V + w]), acc); }
+            else {
+              // another CTA's range: the column of W comes from global memory, eight rows requested at a time
+              // (same order of the multiply-adds as above, so the same bits)
+              int k = 0;
+              for (; k + 8 <= a.r; k += 8) {
+                TIn wv[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) wv[u] = Wg[(size_t)(k + u) * a.V + w];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) acc = fmaf(sb_a[k + u], Elem<TIn>::to_f(wv[u]), acc);
+              }
+              for (; k < a.r; ++k) acc = fmaf(sb_a[k], Elem<TIn>::to_f(Wg[(size_t)k * a.V + w]), acc);
+            }
             q = exp((double)acc / (double)a.T - lseT);
           }
           rw = fmax(p - Cw * q, 0.0);
