@@ -356,7 +356,7 @@ bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out
 cudaError_t score_mma_setup(ts_ctx* ctx) {
   cudaError_t e = cudaFuncSetAttribute(score_mma_kernel<RegLists<8>>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(score_mma_kernel<MemLists>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
+  return cudaFuncSetAttribute(score_mma_kernel<RegLists<16>>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
 }
 
 #ifdef TS_DEBUG_TIMING
@@ -414,7 +414,7 @@ cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t
   memcpy(&tm, c->tmapW, sizeof(tm));
   cudaError_t e;
   if (a.K <= 8) e = launch_kernel(score_mma_kernel<RegLists<8>>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma);
-  else e = launch_kernel(score_mma_kernel<MemLists>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma);
+  else e = launch_kernel(score_mma_kernel<RegLists<16>>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
