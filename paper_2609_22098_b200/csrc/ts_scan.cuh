@@ -200,14 +200,24 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
                                            float gL, float gK, const SharedThr& gl, const SharedThr& gk,
                                            const volatile unsigned* liveL = nullptr, const volatile unsigned* liveK = nullptr) {
   if (valid) TS_SCAN_MARK(0);
+  // High half of each token's uniform, one generator call per eight tokens.  Issued first and in the same
+  // straight-line block as the sums below: the generator's long dependent chains and the exponentials'
+  // latencies then overlap instead of following each other.
+  uint4 cw0 = make_uint4(0, 0, 0, 0), cw1 = cw0;
+  if (T > 0.f) {
+    cw0 = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, (uint32_t)v0 >> 3);
+    cw1 = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, ((uint32_t)v0 >> 3) + 1u);
+  }
   float cm = -INFINITY;
 #pragma unroll
   for (int i = 0; i < CHUNK; ++i) if (i < valid) cm = fmaxf(cm, l[i]);
-  if (cm > st.m) {
-    const float d = st.m - cm;  // -inf on the first chunk: both factors become 0
+  {
+    // rescale to the new running maximum without a branch (no change: factor 1; first chunk: factor 0)
+    const float nm = fmaxf(st.m, cm);
+    const float d = (st.m == nm) ? 0.f : st.m - nm;
     st.s0 *= __expf(d);
     st.sT *= __expf(d * invT);
-    st.m = cm;
+    st.m = nm;
   }
   float a0 = 0.f, aT = 0.f;
   const bool two = (T > 0.f) && (T != 1.f);
@@ -227,9 +237,6 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
   if (cm > st.bestL && cm > st.thrL && cm >= gL) { st.bestL = cm; publish(gl, cm); }
   if (valid) TS_SCAN_MARK(2);
   if (T > 0.f) {
-    // high half of each token's uniform: one generator call per eight tokens
-    const uint4 cw0 = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, (uint32_t)v0 >> 3);
-    const uint4 cw1 = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, ((uint32_t)v0 >> 3) + 1u);
     const float thr = fmaxf(st.thrK, gK);
     uint32_t mk = 0;
     // Four tokens at a time: their best logit plus the noise bound of their largest leading bits bounds
