@@ -107,6 +107,44 @@ def test_tiny_reference_config_100_rounds():
         assert tot["nodes"] >= 100
 
 
+def test_back_to_back_rounds_reproduce_bitwise():
+    """Rounds queued back to back on one stream, no host synchronisation in between, alternating between two
+    input sets: the kernels of a round start while the previous kernel is still finishing (chained launches),
+    so every result is compared bit for bit with the one the same inputs gave when run alone."""
+    wl = small("serve32", V=20000 + 8, B=6)
+    sets = [Round(wl, seed=300), Round(wl, seed=301)]
+    ts = make_gpu(wl, sets[0].table, max_batch=6)
+    alone = []
+    for rnd in sets:
+        tree = ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, 1.0, 42)
+        Z, off = rnd.target_logits(tree)
+        verdict = ts.verify_tree(rnd.U, rnd.A, rnd.W, Z, off, rnd.anchor, tree, 1.0, 42)
+        torch.cuda.synchronize()
+        alone.append((Z, off, {k: v.clone() for k, v in to_cpu(tree).items()}, {k: v.clone() for k, v in to_cpu(verdict).items()}))
+    queued = []
+    for i in range(12):
+        rnd = sets[i % 2]
+        Z, off, _, _ = alone[i % 2]
+        tree = ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, 1.0, 42)
+        verdict = ts.verify_tree(rnd.U, rnd.A, rnd.W, Z, off, rnd.anchor, tree, 1.0, 42)
+        queued.append((tree, verdict))   # every call has its own output buffers
+    torch.cuda.synchronize()
+    for i, (tree, verdict) in enumerate(queued):
+        _, _, t0, v0 = alone[i % 2]
+        n = t0["n_nodes"]
+        assert torch.equal(tree["n_nodes"].cpu(), n)
+        for b in range(len(n)):
+            nb = int(n[b])
+            for key in ("tok", "parent", "depth", "sib_rank", "logS", "q0", "logqT"):
+                assert torch.equal(tree[key].cpu()[b, :nb], t0[key][b, :nb]), (i, b, key)
+            assert torch.equal(tree["mask"].cpu()[b, :nb], t0["mask"][b, :nb]), (i, b)
+        for key in ("acc_len", "bonus_tok", "status"):
+            assert torch.equal(verdict[key].cpu(), v0[key]), (i, key)
+        for b in range(len(n)):
+            L = int(v0["acc_len"][b])
+            assert torch.equal(verdict["acc_tok"].cpu()[b, :L], v0["acc_tok"][b, :L]), (i, b)
+
+
 def test_chain_sentinel_and_mixed_prices():
     wl = small("serve32", V=5000, B=6)
     rnd = Round(wl, seed=21)
