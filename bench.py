@@ -315,6 +315,19 @@ def run_ours(args, rank, world, device):
     return out
 
 
+def short_side_run(args, device, workload, steps=200):
+    """Rounds/s of another configuration, timed the same way in a short run (context beside the headline
+    workload: the single-request decode shape)."""
+    import copy
+    a2 = copy.copy(args)
+    a2.workload, a2.steps, a2.warmup, a2.batch, a2.T, a2.theta = workload, steps, 5, None, None, None
+    a2.no_e2e, a2.no_cpu = True, True
+    r = run_ours(a2, 0, 1, device)
+    return {"workload": r["config"]["workload"], "value": r["value"], "unit": r["unit"], "ms_per_step": r["ms_per_step"],
+            "steps": steps, "parents_scored_per_s": r["parents_scored_per_s"], "nodes_per_s": r["nodes_per_s"],
+            "detail": r["detail"]}
+
+
 def run_e2e(args, ts, wl, sets, A, W, T, B, world, device, barrier):
     """Same metric through the host-buffer API: every step copies that step's inputs (base logits,
     anchors, prices, target logits) from pinned host memory and reads the round's results back."""
@@ -444,6 +457,12 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         torch.distributed.init_process_group("nccl", device_id=device)
     out = run_ours(args, rank, world, device)
+    if world == 1 and args.workload == "serve32" and not args.no_cpu and not args.no_e2e:
+        # the default run also reports the single-request decode shape, briefly
+        try:
+            out["also"] = {"decode": short_side_run(args, device, "decode")}
+        except Exception as e:  # the headline line must not depend on the side run
+            out["also"] = {"decode": {"error": repr(e)}}
     if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:
