@@ -10,7 +10,7 @@ import oracle
 from paper_2609_22098_b200 import synth
 from paper_2609_22098_b200.binding import TreeSpark
 
-# Tolerances (see DESIGN.md "Tolerances"): probabilities and log-survivals are accumulated in fp32 on
+# Tolerances: probabilities and log-survivals are accumulated in fp32 on
 # the GPU and compared at 1e-5 relative plus an absolute floor of two fp32 ulps of a logit of
 # magnitude <= 32 (the inputs of every scalar are such logits).
 RTOL = 1e-5
