@@ -81,8 +81,12 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
   ctx->max_smem = (int)prop.sharedMemPerBlockOptin;
   // tensor cores for bf16 inputs whose rows allow 16-byte chunks; the fp32 FMA kernel otherwise
   ctx->use_mma = (cfg->dt_U == TS_DTYPE_BF16 && cfg->r % 8 == 0 && cfg->V % 8 == 0 && prop.major == 10) ? 1 : 0;
+  // developer switches: TS_FORCE_FMA=1 keeps bf16 inputs on the fp32-FMA kernels, TS_NO_TMA=1 makes the
+  // tensor-core kernels stage W with plain loads (the path taken when no tensor map can be encoded)
   const char* force = getenv("TS_FORCE_FMA");
   if (force && force[0] == '1') ctx->use_mma = 0;
+  const char* no_tma = getenv("TS_NO_TMA");
+  if (no_tma && no_tma[0] == '1') ctx->tma_state = -1;
   if (ctx->use_mma && !choose_tile_mma(ctx->cfg, ctx->num_sms, ctx->max_smem, &ctx->tile)) ctx->use_mma = 0;
   if (!ctx->use_mma && !choose_tile(ctx->cfg, ctx->num_sms, ctx->max_smem, &ctx->tile)) {
     delete (Prof*)ctx->prof; delete ctx;

@@ -145,6 +145,21 @@ def test_back_to_back_rounds_reproduce_bitwise():
             assert torch.equal(verdict["acc_tok"].cpu()[b, :L], v0["acc_tok"][b, :L]), (i, b)
 
 
+@pytest.mark.parametrize("env", ["TS_FORCE_FMA", "TS_NO_TMA"])
+def test_alternative_kernel_paths_match_oracle(env, monkeypatch):
+    """bf16 inputs on the fp32-FMA kernels, and the tensor-core kernels with W staged by plain loads (the
+    path taken when no tensor map can be encoded): both are chosen when the context is created."""
+    monkeypatch.setenv(env, "1")
+    wl = small("serve32", V=20000, B=5)
+    rnd = Round(wl, seed=77)
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
+    monkeypatch.delenv(env)
+    orc = make_oracle(wl, rnd.table)
+    for T in (0.0, 1.0):
+        st = check_round(ts, orc, rnd, T, round_seed=900)
+        assert st["nodes"] > 0
+
+
 def test_chain_sentinel_and_mixed_prices():
     wl = small("serve32", V=5000, B=6)
     rnd = Round(wl, seed=21)
