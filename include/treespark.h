@@ -116,9 +116,11 @@ int32_t ts_score_parents(ts_ctx* ctx, const void* U, const void* A, const void* 
  * cudaFree or other allocating call, and the results are the same as ts_score_parents'.
  *
  * Limits and rules:
- *   - The array bounds P: ntiles * (3 + 5K) * 4 bytes are needed per parent (a few hundred parents
- *     for a 152k vocabulary with K = 8).  A larger P is refused with TS_ERR_WORKSPACE and a message
- *     that names the limit; nothing is launched.
+ *   - The array bounds P: every parent slot needs one record of (4 + 5K) words (rounded up to 16 bytes)
+ *     per vocabulary tile and column split, plus its pruning-bound words, and slots come in blocks of
+ *     128 on the tensor-core path: 128 parents for a 152k vocabulary with K = 8 in bf16, a few hundred
+ *     on the fp32 path.  A larger P is refused with TS_ERR_WORKSPACE and a message that names the
+ *     limit; nothing is launched.
  *   - The context's device must be the current device.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
  *     remembers it; make that first call before starting any stream capture.
