@@ -104,6 +104,11 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
   ctx->calib.a = cfg->platt_a; ctx->calib.b = cfg->platt_b;
   ctx->calib.lo = cfg->calib_lo; ctx->calib.hi = cfg->calib_hi;
   ctx->calib.table = ctx->d_table;
+  // developer switch: TS_NO_FEW=1 sends every level to the tile kernels
+  {
+    const char* no_few = getenv("TS_NO_FEW");
+    ctx->few_ok = (few_supported(ctx) && !(no_few && no_few[0] == '1')) ? 1 : 0;
+  }
   e = score_setup(ctx);
   if (e == cudaSuccess) e = verify_setup(ctx);
   if (e != cudaSuccess) { cudaFree(ctx->d_table); delete (Prof*)ctx->prof; delete ctx; return set_cuda_error("ts_create", e); }
@@ -126,7 +131,7 @@ extern "C" size_t ts_workspace_bytes(const ts_ctx* ctx, int32_t batch) {
 }
 
 static const char* kKernelNames[K_COUNT] = {"expand_init", "score_tile", "score_merge", "expand_level", "expand_finalize",
-                                            "zrow_stats", "verify_greedy", "verify_walk", "verify_check"};
+                                            "zrow_stats", "verify_greedy", "verify_walk", "verify_check", "score_few"};
 
 extern "C" const char* ts_kernel_name(int32_t id) { return (id >= 0 && id < K_COUNT) ? kKernelNames[id] : nullptr; }
 

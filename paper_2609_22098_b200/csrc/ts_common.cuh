@@ -25,6 +25,7 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 // these words with atomicMax in the launch's first microseconds; packed together they queue up on a
 // handful of L2 lines (measured: a third of the scoring launch at stride 1).
 constexpr int SLOT_STRIDE = 32;
+constexpr int FEW_MAX = 8;           // levels with at most this many parents go to the few-parents scoring kernel
 constexpr int SCORE_THREADS = 128;   // one parent per thread; every thread scans the CTA's whole tile
 constexpr int CHUNK = 16;            // tokens per coarse generator call
 constexpr int MMA_S = 2;             // column splits per tile in the tensor-core scoring kernel (warps per row quarter)
@@ -57,6 +58,7 @@ struct ts_ctx {
   ts::TileCfg tile;
   int vt_TV, vt_n;  // vocabulary ranges of the verification walk, one per CTA
   int use_mma;      // 1: scoring runs on the tensor-core kernel, 0: on the fp32 FMA kernel
+  int few_ok;       // 1: levels with <= FEW_MAX parents run on the few-parents kernel instead
   ts::DevCalib calib;
   void* prof;  // ts::Prof*, instrumentation state
   // tensor-map descriptor of the W matrix last scored with (bulk-tensor loads of the W tile); -1: the
@@ -123,6 +125,17 @@ struct VerifyState {
   double fp[KMAX], fq[KMAX];
 };
 
+// Bytes of the scoring records for `cap` parent slots: one record per (tile, column split, slot) of the
+// tile kernels, and room for the few-parents kernel's records (one per 256-token tile and parent, at most
+// FEW_MAX parents), whichever is larger.
+__host__ inline size_t record_bytes(const ts_ctx* ctx, int cap) {
+  const size_t rw = (4 + 5 * (size_t)ctx->cfg.K + 3) & ~(size_t)3;
+  const size_t S = ctx->use_mma ? MMA_S : 1;
+  const size_t tile = (size_t)ctx->tile.ntiles * S * (size_t)cap;
+  const size_t few = (size_t)((ctx->cfg.V + 255) / 256) * FEW_MAX;
+  return align_up((tile > few ? tile : few) * rw * sizeof(float), 256);
+}
+
 __host__ inline WsLayout make_layout(const ts_ctx* ctx, int B) {
   WsLayout L{};
   const ts_config& c = ctx->cfg;
@@ -130,12 +143,12 @@ __host__ inline WsLayout make_layout(const ts_ctx* ctx, int B) {
   L.words = (c.Nmax + 63) / 64;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-  const size_t P = (size_t)L.Pcap, nt = (size_t)L.ntiles, K = (size_t)c.K, N = (size_t)c.Nmax, b = (size_t)B;
+  const size_t P = (size_t)L.Pcap, K = (size_t)c.K, N = (size_t)c.Nmax, b = (size_t)B;
   {
-    int cap = (L.Pcap + 7) / 8 * 8, S = 1;
-    if (ctx->use_mma) { cap = (L.Pcap + 127) / 128 * 128; S = MMA_S; }
+    int cap = (L.Pcap + 7) / 8 * 8;
+    if (ctx->use_mma) cap = (L.Pcap + 127) / 128 * 128;
     L.rec_cap = cap;
-    L.rec = take(align_up(nt * S * (size_t)cap * ((4 + 5 * K + 3) & ~(size_t)3) * 4, 256) + (size_t)cap * (2 + 2 * K * SLOT_STRIDE) * 4);
+    L.rec = take(record_bytes(ctx, cap) + (size_t)cap * (2 + 2 * K * SLOT_STRIDE) * 4);
     L.err = take(16);
   }
   L.res_lse0 = take(P * 4); L.res_lseT = take(P * 4);

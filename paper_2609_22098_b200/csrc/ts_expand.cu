@@ -417,12 +417,14 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
     e = cudaFuncSetAttribute(expand_level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)level_smem);
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(attr)", e);
   }
+  long long level_bound = B;   // parents a level can have at most: B at the root, K times more per level, B * Nmax overall
   for (int d = 0; d < c.D; ++d) {
     const int cur = d & 1;
     e = launch_score(ctx, (float*)(ws + L.rec), L.rec_cap, (int*)(ws + L.err), U, A, W, 0, a.lvl_count + d,
                      a.lst_req[cur], a.lst_depth[cur], a.lst_token[cur],
                      a.lst_hash[cur], T, seed, res_lse0, res_lseT, res_top_tok, res_top_logit, res_draw_tok,
-                     res_draw_logit, st, /*pdl=*/true, d > 0 ? a.lvl_count + d - 1 : nullptr);
+                     res_draw_logit, st, /*pdl=*/true, d > 0 ? a.lvl_count + d - 1 : nullptr, (int)level_bound);
+    level_bound = level_bound * c.K < (long long)B * c.Nmax ? level_bound * c.K : (long long)B * c.Nmax;
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(score)", e);
     { ProfScope ps(ctx, K_LEVEL, st); e = launch_kernel(expand_level_kernel, B, 256, level_smem, st, true, a, d); }
     if (e == cudaSuccess) e = cudaGetLastError();

@@ -19,6 +19,7 @@ struct ScoreArgs {
   int P; const int* P_dev;
   const int* P_prev_dev;   // parent count of the previous level (nullptr: none); 0 there means 0 here
   int pdl;                 // host side: launch with programmatic stream serialization
+  int few;                 // host side: this launch runs on the few-parents kernel
   const int *p_req, *p_depth, *p_token; const uint64_t* p_hash;
   float T; uint64_t seed;
   int TV, ntiles, cap, S;
@@ -30,6 +31,7 @@ struct ScoreArgs {
 struct MergeArgs {
   int P; const int* P_dev; int K, ntiles, cap, S, mma; float T;
   int pdl;   // host side: launch with programmatic stream serialization
+  int few_ntiles;   // > 0: the level was scored by the few-parents kernel over this many tiles
   const float* rec; unsigned* thr; unsigned* slots;
   float *lse0, *lseT; int* top_tok; float* top_logit; int* draw_tok; float* draw_logit;
 };
@@ -41,13 +43,15 @@ size_t score_scratch_bytes(const ts_ctx* ctx, int P, int* cap_out);
 unsigned* thr_base(const ts_ctx* ctx, float* rec, int cap);
 size_t thr_bytes(const ts_ctx* ctx, int cap);
 
-// Scoring pass + merge for a parent list whose length is P (host) or *P_dev (device) when P_dev is set.
+// Scoring pass + merge for a parent list whose length is P (host) or *P_dev (device) when P_dev is set;
+// p_bound: an upper bound of *P_dev the host knows (-1: none).  A list that cannot exceed FEW_MAX parents
+// goes to the few-parents kernel where the context has one.
 // rec: record scratch of score_scratch_bytes(ctx, max parents) bytes with slot capacity cap.
 cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,
                          const uint64_t* p_hash, float T, uint64_t seed, float* lse0, float* lseT, int* top_tok,
                          float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st,
-                         bool pdl = false, const int* P_prev_dev = nullptr);
+                         bool pdl = false, const int* P_prev_dev = nullptr, int p_bound = -1);
 
 // Kernel launch, optionally with programmatic stream serialization: the kernel may then start while the
 // kernel before it in the stream is still running, and must execute pdl_wait() before it touches anything
@@ -67,10 +71,14 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
 bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out);
 cudaError_t score_mma_setup(ts_ctx* ctx);
 cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st);
+// the few-parents kernel (ts_score_few.cu)
+int few_tiles(const ts_config& c);
+bool few_supported(const ts_ctx* ctx);
+cudaError_t launch_score_few(const ts_ctx* ctx, const ScoreArgs& a, int p_bound, cudaStream_t st);
 // encodes (or finds cached in the context) the tensor map of W for 64-token boxes; false: not available
 bool w_tensor_map(ts_ctx* ctx, const void* W);
 
-enum KernelId { K_INIT, K_SCORE, K_MERGE, K_LEVEL, K_FINAL, K_ZROWS, K_GREEDY, K_WALK, K_CHECK, K_COUNT };
+enum KernelId { K_INIT, K_SCORE, K_MERGE, K_LEVEL, K_FINAL, K_ZROWS, K_GREEDY, K_WALK, K_CHECK, K_SCORE_FEW, K_COUNT };
 
 struct Prof {
   bool on = false;

@@ -187,8 +187,9 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float invT = a.T > 0.f ? 1.f / a.T : 1.f;
   const int K = a.K, rw = rec_words(K);
-  const int R = a.mma ? mma_replicas(P) : 1;
-  const int npieces = a.ntiles * a.S * R;
+  const bool few = a.few_ntiles > 0;   // the level was scored by the few-parents kernel
+  const int R = few ? 1 : (a.mma ? mma_replicas(P) : 1);
+  const int npieces = few ? a.few_ntiles : a.ntiles * a.S * R;
   for (int p = blockIdx.x; p < P; p += gridDim.x) {
     // final launch-wide lower bounds of this parent's K-th best logit / key: entries below cannot win
     const SharedThr gl{a.slots + (size_t)p * K * SLOT_STRIDE, 0}, gk{a.slots + ((size_t)a.cap + p) * K * SLOT_STRIDE, 0};
@@ -197,22 +198,34 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
     __syncthreads();
     float m = -INFINITY, s0 = 0.f, sT = 0.f;
     auto rec_of = [&](int q) {
+      if (few) return a.rec + ((size_t)q * FEW_MAX + p) * rw;
       const int ts_ = q / R, rho = q % R;
       const int slot = R > 1 ? rho * (128 / R) + p : p;
       return a.rec + ((size_t)ts_ * a.cap + slot) * rw;
     };
     // the header of the next record is requested before this one's entries, so that a thread with
     // several records pays one memory round trip per record, not two
+    // ... together with the record's best key: a record whose best logit (its maximum, in the header) and
+    // best key are below the final bounds has nothing to offer, and its entries are not read at all
     float4 hn = make_float4(-INFINITY, 0.f, 0.f, 0.f);
-    if (tid < npieces) hn = __ldcg(reinterpret_cast<const float4*>(rec_of(tid)));
+    float kn = -INFINITY;
+    if (tid < npieces) {
+      hn = __ldcg(reinterpret_cast<const float4*>(rec_of(tid)));
+      if (a.T > 0.f) kn = __ldcg(rec_of(tid) + 4 + 2 * K);
+    }
     for (int q = tid; q < npieces; q += MERGE_THREADS) {
       const float* rec = rec_of(q);
       const float4 h = hn;
-      if (q + MERGE_THREADS < npieces) hn = __ldcg(reinterpret_cast<const float4*>(rec_of(q + MERGE_THREADS)));
+      const float kbest = kn;
+      if (q + MERGE_THREADS < npieces) {
+        hn = __ldcg(reinterpret_cast<const float4*>(rec_of(q + MERGE_THREADS)));
+        if (a.T > 0.f) kn = __ldcg(rec_of(q + MERGE_THREADS) + 4 + 2 * K);
+      }
       const float* f = rec + 4; const int* ii = reinterpret_cast<const int*>(rec) + 4;
       // all entries of the record are requested at once (independent loads), then filtered
       float tv[KR], kv[KR], kl[KR]; int ti[KR], ki[KR];
-      const int cnt = __float_as_int(h.w), nt = cnt & 255, nk = (cnt >> 8) & 255;   // entries worth reading
+      const int cnt = __float_as_int(h.w);
+      const int nt = h.x >= bL ? (cnt & 255) : 0, nk = kbest >= bK ? ((cnt >> 8) & 255) : 0;   // entries worth reading
 #pragma unroll
       for (int j = 0; j < KR; ++j) {
         ti[j] = j < nt ? __ldcg(ii + K + j) : -1;
@@ -277,9 +290,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
       MList<KR> top, key;
       top.init(); key.init();
       for (int q = tid; q < npieces; q += MERGE_THREADS) {
-        const int ts_ = q / R, rho = q % R;
-        const int slot = R > 1 ? rho * (128 / R) + p : p;
-        const float* rec = a.rec + ((size_t)ts_ * a.cap + slot) * rw;
+        const float* rec = rec_of(q);
         if (__ldcg(rec) == -INFINITY) continue;
         const float* f = rec + 4; const int* ii = reinterpret_cast<const int*>(rec) + 4;
         for (int j = 0; j < K; ++j) {
@@ -307,17 +318,14 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
 // ------------------------------------------------------------------------------------------------
 size_t score_scratch_bytes(const ts_ctx* ctx, int P, int* cap_out) {
   int cap = (P + 7) / 8 * 8;
-  int S = 1;
-  if (ctx->use_mma) { cap = (P + 127) / 128 * 128; if (cap < 128) cap = 128; S = MMA_S; }
+  if (ctx->use_mma) { cap = (P + 127) / 128 * 128; if (cap < 128) cap = 128; }
   if (cap_out) *cap_out = cap;
   // records, then the pruning state: 2 threshold words and 2K slot words per slot of capacity
-  return align_up((size_t)ctx->tile.ntiles * S * cap * rec_words(ctx->cfg.K) * sizeof(float), 256) +
-         align_up((size_t)cap * (2 + 2 * (size_t)ctx->cfg.K * SLOT_STRIDE) * sizeof(unsigned), 256);
+  return record_bytes(ctx, cap) + align_up((size_t)cap * (2 + 2 * (size_t)ctx->cfg.K * SLOT_STRIDE) * sizeof(unsigned), 256);
 }
 
 unsigned* thr_base(const ts_ctx* ctx, float* rec, int cap) {
-  const int S = ctx->use_mma ? MMA_S : 1;
-  return (unsigned*)((char*)rec + align_up((size_t)ctx->tile.ntiles * S * cap * rec_words(ctx->cfg.K) * sizeof(float), 256));
+  return (unsigned*)((char*)rec + record_bytes(ctx, cap));
 }
 
 size_t thr_bytes(const ts_ctx* ctx, int cap) { return (size_t)cap * (2 + 2 * (size_t)ctx->cfg.K * SLOT_STRIDE) * sizeof(unsigned); }
@@ -325,7 +333,8 @@ size_t thr_bytes(const ts_ctx* ctx, int cap) { return (size_t)cap * (2 + 2 * (si
 cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,
                          const uint64_t* p_hash, float T, uint64_t seed, float* lse0, float* lseT, int* top_tok,
-                         float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st, bool pdl, const int* P_prev_dev) {
+                         float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st, bool pdl, const int* P_prev_dev,
+                         int p_bound) {
   const ts_config& c = ctx->cfg;
   ScoreArgs a{};
   a.pdl = pdl ? 1 : 0; a.P_prev_dev = P_prev_dev;
@@ -333,12 +342,17 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
   a.p_req = p_req; a.p_depth = p_depth; a.p_token = p_token; a.p_hash = p_hash; a.T = T; a.seed = seed;
   a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.cap = cap; a.S = ctx->use_mma ? MMA_S : 1; a.rec = rec; a.err = err;
   a.thr = thr_base(ctx, rec, cap); a.slots = a.thr + 2 * (size_t)cap;
-  cudaError_t e;
-  {
+  cudaError_t e = cudaSuccess;
+  // Which kernel scores the level: the few-parents kernel when the host knows that the list cannot hold
+  // more than FEW_MAX parents (its own P, or a bound of the device-side count), the tile kernel otherwise.
+  const int bound = P_dev ? p_bound : P;
+  const bool run_few = ctx->use_mma && ctx->few_ok && bound >= 0 && bound <= FEW_MAX;
+  const bool run_tile = !run_few;
+  a.few = run_few ? 1 : 0;
+  if (run_tile) {
     ProfScope ps(ctx, K_SCORE, st);
     if (ctx->use_mma) {
       e = launch_score_mma(ctx, a, st);
-      if (e != cudaSuccess) return e;
     } else if (c.dt_U == TS_DTYPE_BF16) {
       if (c.K <= 8) e = launch_kernel(score_tile_kernel<__nv_bfloat16, RegLists<8>>, a.ntiles, SCORE_THREADS, ctx->tile.smem, st, pdl, a);
       else e = launch_kernel(score_tile_kernel<__nv_bfloat16, MemLists>, a.ntiles, SCORE_THREADS, ctx->tile.smem, st, pdl, a);
@@ -346,12 +360,18 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
       if (c.K <= 8) e = launch_kernel(score_tile_kernel<float, RegLists<8>>, a.ntiles, SCORE_THREADS, ctx->tile.smem, st, pdl, a);
       else e = launch_kernel(score_tile_kernel<float, MemLists>, a.ntiles, SCORE_THREADS, ctx->tile.smem, st, pdl, a);
     }
+    if (e != cudaSuccess) return e;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
   }
-  if (e != cudaSuccess) return e;
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  if (run_few) {
+    ProfScope ps(ctx, K_SCORE_FEW, st);
+    e = launch_score_few(ctx, a, bound, st);
+    if (e != cudaSuccess) return e;
+  }
   MergeArgs m{};
   m.pdl = a.pdl;
+  m.few_ntiles = run_few ? few_tiles(c) : 0;
   m.P = P; m.P_dev = P_dev; m.K = c.K; m.ntiles = a.ntiles; m.cap = cap; m.S = a.S; m.mma = ctx->use_mma ? 1 : 0; m.T = T;
   m.rec = rec; m.thr = a.thr; m.slots = a.slots;
   m.lse0 = lse0; m.lseT = lseT; m.top_tok = top_tok; m.top_logit = top_logit; m.draw_tok = draw_tok; m.draw_logit = draw_logit;
