@@ -122,7 +122,7 @@ def test_back_to_back_rounds_reproduce_bitwise():
         torch.cuda.synchronize()
         alone.append((Z, off, {k: v.clone() for k, v in to_cpu(tree).items()}, {k: v.clone() for k, v in to_cpu(verdict).items()}))
     queued = []
-    for i in range(12):
+    for i in range(300):
         rnd = sets[i % 2]
         Z, off, _, _ = alone[i % 2]
         tree = ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, 1.0, 42)
