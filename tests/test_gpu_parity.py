@@ -26,12 +26,12 @@ def small(name, **kw):
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("V,r,K", [(1000, 7, 4), (1003, 16, 8), (4096 + 40, 64, 8), (70000, 32, 16), (8, 4, 4), (5, 3, 8)])
 @pytest.mark.parametrize("T", [0.0, 0.7, 1.0])
-def test_score_parents_matches_oracle(dtype, V, r, K, T):
+@pytest.mark.parametrize("P", [11, 3])   # 3: the few-parents kernel where the context has one
+def test_score_parents_matches_oracle(dtype, V, r, K, T, P):
     wl = small("tiny", V=V, r=r, K=K, D=3, Nmax=16, dtype=dtype, B=3, calib_mode=0)
     rnd = Round(wl, seed=11 + V)
     ts = make_gpu(wl, None, max_batch=3)
     orc = make_oracle(wl, None)
-    P = 11
     g = torch.Generator().manual_seed(V)
     req = torch.randint(0, 3, (P,), generator=g, dtype=torch.int32)
     dep = torch.randint(0, 3, (P,), generator=g, dtype=torch.int32)
