@@ -83,6 +83,15 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  const bool early_w = !a.P_prev_dev || *a.P_prev_dev >= 16;
+  auto issue_w = [&]() {   // one thread
+    for (int nb = 0; nb < nblk_w; ++nb) {
+      const int ns = (tlen - nb * BLK_N > 64) ? 2 : 1;
+      mbar_expect_tx(w_full + nb, (uint32_t)ns * slab_bytes);
+      for (int h = 0; h < ns; ++h)
+        tma_load_box(Ws + (size_t)(2 * nb + h) * slab_bytes, &tmW, t0 + (2 * nb + h) * 64, 0, w_full + nb);
+    }
+  };
   if (tid == 0) {
     mbar_init(a_full, EPI_WARPS * 32);
     for (int i = 0; i < NBUF; ++i) { mbar_init(t_full + i, 1); mbar_init(t_empty + i, EPI_WARPS); }
@@ -90,16 +99,12 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
     *s_done = 0;
     if (use_tma) for (int i = 0; i < nblk_w; ++i) mbar_init(w_full + i, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    if (use_tma) {
-      // W tile by bulk-tensor loads, one barrier per block of 128 tokens so that the first MMAs start
-      // while the rest of the tile is still in flight; tokens past V and rows past r arrive as zeros
-      for (int nb = 0; nb < nblk_w; ++nb) {
-        const int ns = (tlen - nb * BLK_N > 64) ? 2 : 1;
-        mbar_expect_tx(w_full + nb, (uint32_t)ns * slab_bytes);
-        for (int h = 0; h < ns; ++h)
-          tma_load_box(Ws + (size_t)(2 * nb + h) * slab_bytes, &tmW, t0 + (2 * nb + h) * 64, 0, w_full + nb);
-      }
-    }
+    // W tile by bulk-tensor loads, one barrier per block of 128 tokens so that the first MMAs start while
+    // the rest of the tile is still in flight; tokens past V and rows past r arrive as zeros.  Issued here,
+    // before the kernel may look at its own parent count, when the level before was large enough for this
+    // one to be populated almost surely; after the count is known otherwise (a level that turns out empty then
+    // fetches nothing).
+    if (use_tma && early_w) issue_w();
   }
   if (!use_tma) {  // W tile: 16-byte chunks (8 tokens of one row), swizzled: chunk j of row k lands at chunk j ^ (k & 7)
     const int per_slab = rp * 8;
@@ -124,6 +129,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   pdl_wait();                // parent lists and the level's parent count come from the previous kernel
   pdl_launch_dependents();
   const int P = a.P_dev ? *a.P_dev : a.P;   // may be 0: an empty level only tears down
+  if (use_tma && !early_w && P > 0 && tid == 0) issue_w();
 
   const int R = mma_replicas(P), rsh = R == 4 ? 2 : (R == 2 ? 1 : 0);
   const int ngroups = P <= 0 ? 0 : (R > 1 ? 1 : (P + 127) / 128);
@@ -310,7 +316,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   }
   // ---- tear-down -----------------------------------------------------------------------------------
   if (warp == 0) DBG(5);
-  if (use_tma && tid == 0 && (*s_abort || P <= 0)) {
+  if (use_tma && tid == 0 && ((*s_abort && (early_w || P > 0)) || (P <= 0 && early_w))) {
     // gave up somewhere, or nothing to score: do not leave while a bulk load may still be writing this
     // CTA's shared memory
     for (int nb = 0; nb < nblk_w; ++nb) {
