@@ -217,7 +217,13 @@ class HostRound:
     ``run`` copies the step's inputs (base logits, anchors, prices, target logits and their row
     offsets) from pinned host tensors to device staging buffers, runs ts_expand_tree and
     ts_verify_tree, copies the tree and the verdict back into pinned host tensors and waits for
-    them.  All staging memory is allocated once in the constructor."""
+    them.  All staging memory is allocated once in the constructor.
+
+    ``submit`` / ``collect`` are the same round split in two for callers that keep the copy engine busy:
+    ``submit`` queues the host-to-device copies of a step on a copy stream and the round behind them on the
+    caller's stream, into one of two staging slots; ``collect`` waits for the oldest submitted step and
+    returns its host outputs.  With two steps in flight the copies of one step run beside the kernels of
+    the step before."""
 
     TREE_OUT = ("n_nodes", "tok", "parent", "depth", "mask")
     VERDICT_OUT = ("acc_len", "acc_tok", "bonus_tok")
@@ -241,6 +247,63 @@ class HostRound:
         self.host_out.update({k: torch.empty_like(self.verdict[k], device="cpu").pin_memory() for k in self.VERDICT_OUT})
         self.h2d_bytes = 0
         self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.host_out.values())
+        self._max_rows = max_rows
+        self._slots = None      # second staging slot, copy stream and events: built on the first submit
+        self._pending = []
+
+    def _make_slots(self):
+        ts, B, d = self.ts, self.B, self.ts.device
+        slots = [dict(U=self.U, anchor=self.anchor, theta=self.theta, Z=self.Z, zoff=self.zoff, tree=self.tree,
+                      verdict=self.verdict, out=self.host_out)]
+        slots.append(dict(U=torch.empty_like(self.U), anchor=torch.empty_like(self.anchor), theta=torch.empty_like(self.theta),
+                          Z=torch.empty_like(self.Z), zoff=torch.empty_like(self.zoff), tree=ts.alloc_tree(B),
+                          verdict=ts.alloc_verdict(B),
+                          out={k: torch.empty_like(v).pin_memory() for k, v in self.host_out.items()}))
+        for sl in slots:
+            sl["copied"] = torch.cuda.Event()
+            sl["done"] = torch.cuda.Event()
+            sl["free"] = torch.cuda.Event()
+            sl["free"].record()
+        self._copy_stream = torch.cuda.Stream(device=d)
+        self._slots, self._next = slots, 0
+
+    def submit(self, host, A, W, T, seed, edge_stat=True):
+        """Queue one round; at most two may be in flight (collect the older one first)."""
+        if self._slots is None:
+            self._make_slots()
+        if len(self._pending) >= 2:
+            raise RuntimeError("HostRound.submit: two rounds already in flight; call collect() first")
+        ts = self.ts
+        sl = self._slots[self._next]
+        self._next ^= 1
+        rows = host["Z"].shape[0]
+        main = torch.cuda.current_stream()
+        with torch.cuda.stream(self._copy_stream):
+            self._copy_stream.wait_event(sl["free"])      # the round that used this slot last has finished
+            sl["U"].copy_(host["U"], non_blocking=True)
+            sl["anchor"].copy_(host["anchor"], non_blocking=True)
+            sl["theta"].copy_(host["theta"], non_blocking=True)
+            sl["Z"][:rows].copy_(host["Z"], non_blocking=True)
+            sl["zoff"].copy_(host["zoff"], non_blocking=True)
+            sl["copied"].record()
+        main.wait_event(sl["copied"])
+        ts.expand_tree(sl["U"], A, W, sl["anchor"], sl["theta"], T, seed, out=sl["tree"])
+        ts.verify_tree(sl["U"], A, W, sl["Z"], sl["zoff"], sl["anchor"], sl["tree"], T, seed, out=sl["verdict"],
+                       edge_stat=edge_stat)
+        for k in self.TREE_OUT:
+            sl["out"][k].copy_(sl["tree"][k], non_blocking=True)
+        for k in self.VERDICT_OUT:
+            sl["out"][k].copy_(sl["verdict"][k], non_blocking=True)
+        sl["done"].record()
+        sl["free"].record()
+        self._pending.append(sl)
+        self.h2d_bytes = sum(host[k].numel() * host[k].element_size() for k in ("U", "anchor", "theta", "Z", "zoff"))
+
+    def collect(self):
+        """Host outputs of the oldest submitted round (waits for it)."""
+        sl = self._pending.pop(0)
+        sl["done"].synchronize()
+        return sl["out"]
 
     def run(self, host, A, W, T, seed, edge_stat=True):
         ts = self.ts

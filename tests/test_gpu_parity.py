@@ -160,6 +160,38 @@ def test_alternative_kernel_paths_match_oracle(env, monkeypatch):
         assert st["nodes"] > 0
 
 
+def test_host_round_two_in_flight_equals_one_at_a_time():
+    """The host-buffer round: submit / collect with two rounds in flight returns what run() returns."""
+    from paper_2609_22098_b200.binding import HostRound
+    wl = small("serve32", V=20000 + 16, B=5)
+    rnds = [Round(wl, seed=500 + i) for i in range(3)]
+    ts = make_gpu(wl, rnds[0].table, max_batch=5)
+    A, W = rnds[0].A, rnds[0].W   # one head for all three input sets
+    host = []
+    for rnd in rnds:
+        tree = ts.expand_tree(rnd.U, A, W, rnd.anchor, rnd.theta, 1.0, 9)   # the tree the round below will build
+        Z, off = rnd.target_logits(tree)                                      # one target row per node of that tree
+        host.append(HostRound.pin_inputs(rnd.U, rnd.anchor, rnd.theta, Z, off))
+    hr = HostRound(ts, 5, max(int(h["Z"].shape[0]) for h in host))
+    ref = []
+    for h in host:
+        out = hr.run(h, A, W, 1.0, 9)
+        ref.append({k: v.clone() for k, v in out.items()})
+    got = []
+    for i in range(9):
+        hr.submit(host[i % 3], A, W, 1.0, 9)
+        if i > 0:
+            got.append({k: v.clone() for k, v in hr.collect().items()})
+    got.append({k: v.clone() for k, v in hr.collect().items()})
+    for i, g in enumerate(got):
+        r = ref[i % 3]
+        n = r["n_nodes"]
+        assert torch.equal(g["n_nodes"], n) and torch.equal(g["acc_len"], r["acc_len"]) and torch.equal(g["bonus_tok"], r["bonus_tok"])
+        for b in range(5):
+            assert torch.equal(g["tok"][b, :int(n[b])], r["tok"][b, :int(n[b])])
+            assert torch.equal(g["acc_tok"][b, :int(r["acc_len"][b])], r["acc_tok"][b, :int(r["acc_len"][b])])
+
+
 def test_chain_sentinel_and_mixed_prices():
     wl = small("serve32", V=5000, B=6)
     rnd = Round(wl, seed=21)
