@@ -192,6 +192,26 @@ def test_host_round_two_in_flight_equals_one_at_a_time():
             assert torch.equal(g["acc_tok"][b, :int(r["acc_len"][b])], r["acc_tok"][b, :int(r["acc_len"][b])])
 
 
+@pytest.mark.parametrize("which", ["marginal_tree", "raw_priority"])
+def test_ablation_settings_match_oracle(which):
+    """Two of the paper's ablation axes need no code of their own: the marginal tree (scores from the base
+    logits only) is a zero head matrix A, and the uncalibrated sum-of-log-q priority is the Platt map with
+    a = 1, b = 0 (p-hat = q_0).  Both must match the oracle like any other setting."""
+    wl = small("serve32", V=12000 + 8, B=4, calib_mode=0)
+    rnd = Round(wl, seed=910)
+    a, b = (0.67, -0.46)
+    if which == "marginal_tree":
+        rnd.A.zero_()
+    else:
+        a, b = 1.0, 0.0
+    ts = TreeSpark(wl.V, wl.D, wl.r, wl.K, wl.Nmax, rnd.B, dtype=wl.torch_dtype, calib_mode=0, platt_a=a, platt_b=b)
+    orc = oracle.Oracle(wl.V, wl.D, wl.r, wl.K, wl.Nmax, calib_mode=0, platt_a=a, platt_b=b)
+    rnd.theta.fill_(0.02)
+    for T in (0.0, 1.0):
+        st = check_round(ts, orc, rnd, T, round_seed=31)
+        assert st["trees"] == rnd.B
+
+
 def test_chain_sentinel_and_mixed_prices():
     wl = small("serve32", V=5000, B=6)
     rnd = Round(wl, seed=21)
