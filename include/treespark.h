@@ -198,6 +198,34 @@ int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, const void* W,
                        void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Cut the trees of a batch back to one node budget (Section 4, "per-request budget allocation").
+ * The scheduler chooses the tree sizes N_b that maximise the expected number of accepted tokens under
+ * a total of `budget` verified nodes; with concave per-request gain curves greedy water-filling does
+ * it: the budget is handed out one node at a time to the request whose next candidate -- in its own
+ * best-first admission order, pop_rank -- was admitted under the largest key (logkey; equal keys go
+ * to the lowest request, then to the earlier admission).  The gain credited to a candidate is its
+ * admission key, never a value drawn for it, so the resulting shapes stay within Proposition 1.
+ * With budget = the number of candidates whose key is >= theta this is the theta stop rule.
+ *
+ * Input: the outputs of ts_expand_tree for the same B (DEVICE, same shapes), logkey and pop_rank
+ * required.  The call keeps, per request, the keep[b] nodes admitted first, renumbers them in
+ * canonical order (their relative order does not change), rewrites parent and mask to the new
+ * numbering and moves every per-node array in place, node_hash and node_lseT (slot 0 = root) included;
+ * n_nodes[b] becomes keep[b].  Array arguments other than n_nodes, logkey and pop_rank may be NULL and
+ * are then skipped.  log_price DEVICE float[1] or NULL: logkey of the last node handed out, -inf when
+ * none was.  budget >= the number of nodes leaves every tree as it is.  Trees of requests on the chain
+ * member of the price ladder take part like any other.
+ * One CTA selects the price, so the cost grows with B * Nmax (32,768 candidates at most in the
+ * workloads this library is sized for).  Errors as for the other calls; nothing is launched on error.
+ */
+int32_t ts_allocate_budget(ts_ctx* ctx, int32_t B, int32_t budget,
+                           int32_t* n_nodes, int32_t* tok, int32_t* parent, int32_t* depth,
+                           int32_t* sib_rank, float* logS, float* q0, float* logqT,
+                           float* logkey, int32_t* pop_rank,
+                           uint64_t* node_hash, float* node_lseT, uint64_t* mask,
+                           float* log_price, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Instrumentation (no counterpart in the paper): per-kernel device times and launch counts.
  * ts_profile_enable(capacity > 0) creates `capacity` CUDA event pairs and from then on every kernel
  * the hot calls launch is bracketed by an event pair on the caller's stream until the pairs run out;

@@ -21,7 +21,7 @@ KNOTS = 16
 
 EXPORTS = ("ts_create", "ts_destroy", "ts_workspace_bytes", "ts_last_error_string",
            "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",
-           "ts_profile_enable", "ts_profile_read", "ts_kernel_name")
+           "ts_allocate_budget", "ts_profile_enable", "ts_profile_read", "ts_kernel_name")
 
 
 class TsConfig(C.Structure):
@@ -52,12 +52,13 @@ def load_library() -> C.CDLL:
         L.ts_score_parents_static.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, f32, u64] + [vp] * 6 + [vp]
         L.ts_expand_tree.argtypes = [vp, vp, vp, vp, i32, vp, vp, f32, u64] + [vp] * 15 + [vp, sz, vp]
         L.ts_verify_tree.argtypes = [vp, vp, vp, vp, vp, vp, i32] + [vp] * 9 + [f32, u64] + [vp] * 7 + [vp, sz, vp]
+        L.ts_allocate_budget.argtypes = [vp, i32, i32] + [vp] * 14 + [vp, sz, vp]
         L.ts_profile_enable.argtypes = [vp, i32]
         L.ts_profile_read.argtypes = [vp, i32, vp, vp, i32]
         L.ts_kernel_name.argtypes = [i32]
         L.ts_kernel_name.restype = C.c_char_p
         for n in ("ts_create", "ts_destroy", "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",
-                  "ts_profile_enable", "ts_profile_read"):
+                  "ts_allocate_budget", "ts_profile_enable", "ts_profile_read"):
             getattr(L, n).restype = C.c_int32
         _lib = L
     return _lib
@@ -184,6 +185,18 @@ class TreeSpark:
                                             _ptr(t["n_scored"]), _ptr(t["status"]), _ptr(self.ws), self.ws_bytes,
                                             _stream()))
         return t
+
+    def allocate_budget(self, tree, budget, log_price=None):
+        """Cut the trees of ``tree`` (the dict ts_expand_tree filled) back, in place, to ``budget`` nodes
+        for the whole batch; ``log_price`` is an optional float32 device tensor of one element."""
+        B = int(tree["n_nodes"].numel())
+        self._check(self.lib.ts_allocate_budget(self._ctx, B, int(budget), _ptr(tree["n_nodes"]), _ptr(tree["tok"]),
+                                                _ptr(tree["parent"]), _ptr(tree["depth"]), _ptr(tree["sib_rank"]),
+                                                _ptr(tree["logS"]), _ptr(tree["q0"]), _ptr(tree["logqT"]),
+                                                _ptr(tree["logkey"]), _ptr(tree["pop_rank"]), _ptr(tree["node_hash"]),
+                                                _ptr(tree["node_lseT"]), _ptr(tree["mask"]), _ptr(log_price),
+                                                _ptr(self.ws), self.ws_bytes, _stream()))
+        return tree
 
     def verify_tree(self, U, A, W, Z, z_row_off, anchor_tok, tree, T, seed, out=None, edge_stat=True):
         B = int(anchor_tok.numel())
