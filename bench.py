@@ -328,6 +328,51 @@ def short_side_run(args, device, workload, steps=200):
             "detail": r["detail"]}
 
 
+def allocate_side_run(args, device, steps=200):
+    """Device time of ts_allocate_budget (batch-wide node budget, Section 4) on the headline batch: trees
+    grown under a low price, then cut to half their nodes.  Every timed call starts from the same trees
+    (restored outside the timed events).  The oracle's allocation is timed beside it on the host."""
+    from oracle import allocate as orc_alloc
+    from paper_2609_22098_b200.binding import TreeSpark
+    wl = synth.WORKLOADS["serve32"]
+    B, T = wl.B, wl.temps[-1]
+    table = synth.make_calibration_table(wl, args.seed + 4, "fit")
+    A, W = synth.make_head(wl, args.seed + 1, device)
+    ts = TreeSpark(wl.V, wl.D, wl.r, wl.K, wl.Nmax, B, dtype=wl.torch_dtype, calib_mode=wl.calib_mode,
+                   calib_table=table, device=device)
+    s = InputSet(wl, args.seed + 900, B, 0.02, A, W, device)
+    grown = ts.expand_tree(s.U, A, W, s.anchor, s.theta, T, s.round_seed)
+    torch.cuda.synchronize()
+    total = int(grown["n_nodes"].sum())
+    budget = total // 2
+    tree = {k: v.clone() for k, v in grown.items()}
+    price = torch.zeros(4, dtype=torch.float32, device=device)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for i in range(5 + steps):
+        for k in tree:
+            tree[k].copy_(grown[k])
+        if i >= 5:
+            ev[i - 5][0].record()
+        ts.allocate_budget(tree, budget, price)
+        if i >= 5:
+            ev[i - 5][1].record()
+    torch.cuda.synchronize()
+    us = sorted(a.elapsed_time(b) * 1e3 for a, b in ev)
+    kept = int(tree["n_nodes"].sum())
+    g = {k: v.cpu() for k, v in grown.items()}
+    t0 = time.perf_counter()
+    keep, _ = orc_alloc.water_fill(g["n_nodes"].numpy(), g["logkey"].numpy(), g["pop_rank"].numpy(), budget)
+    t_cpu = time.perf_counter() - t0
+    words = (wl.Nmax + 63) // 64
+    node_bytes = 9 * 4 + 8 + 4 + 8 * words          # per-node arrays read and written by the cut
+    alg = total * 4 + total * 4 + (total + kept) * node_bytes
+    return {"workload": f"serve32 trees grown at theta=0.02 ({total} nodes in {B} trees), budget {budget}",
+            "us_per_call_median": us[len(us) // 2], "us_per_call_mean": sum(us) / len(us), "calls": steps,
+            "kernels_per_call": 2, "nodes_kept": kept, "matches_oracle_sizes": tree["n_nodes"].cpu().tolist() == list(keep),
+            "alg_bytes_per_call": alg, "bound": "launch latency (two small kernels; the bytes are noise)",
+            "oracle_water_fill_ms": t_cpu * 1e3}
+
+
 def run_e2e(args, ts, wl, sets, A, W, T, B, world, device, barrier):
     """Same metric through the host-buffer API: every step copies that step's inputs (base logits,
     anchors, prices, target logits) from pinned host memory and reads the round's results back."""
@@ -482,6 +527,10 @@ def main():
             out["also"] = {"decode": short_side_run(args, device, "decode")}
         except Exception as e:  # the headline line must not depend on the side run
             out["also"] = {"decode": {"error": repr(e)}}
+        try:
+            out["also"]["allocate_budget"] = allocate_side_run(args, device)
+        except Exception as e:
+            out["also"]["allocate_budget"] = {"error": repr(e)}
     if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:

@@ -7,8 +7,8 @@
 // the allocation is one selection: find the key of the budget-th candidate (a most-significant-digit
 // radix select over the order-preserving integer image of the fp32 keys, four passes of eight bits),
 // count per request the candidates above it, and hand the candidates equal to it out in request order
-// until the budget is gone.  One CTA does this; the keys (at most a few hundred KB) stay in L2 between
-// the passes.  A second kernel, one CTA per request and one thread per node, compacts the per-node
+// until the budget is gone.  One CTA does this; the keys' images stay in shared memory between the passes
+// when they fit (11k candidates), else the keys are re-read from L2 (a few hundred KB at most).  A second kernel, one CTA per request and one thread per node, compacts the per-node
 // arrays in place: all reads, a barrier, all writes.
 #include "ts_internal.h"
 
@@ -67,50 +67,66 @@ __device__ void block_excl_scan(int* s, int n, int* tmp, int* total) {
   __syncthreads();
 }
 
-__global__ void __launch_bounds__(SEL_THREADS) allocate_select_kernel(const AllocArgs a) {
-  extern __shared__ int s_dyn[];   // gt[B], tie[B]
+__global__ void __launch_bounds__(SEL_THREADS) allocate_select_kernel(const AllocArgs a, const int cached) {
+  extern __shared__ int s_dyn[];   // n[B], counts[B], then (cached) the key images [B * N]
   __shared__ int s_hist[256];
   __shared__ int s_tmp[33];
   __shared__ int s_total;
   __shared__ unsigned s_prefix;
   __shared__ int s_remaining;
-  int* s_gt = s_dyn; int* s_tie = s_dyn + a.B;
+  int* s_n = s_dyn; int* s_cnt = s_dyn + a.B;
+  unsigned* s_img = reinterpret_cast<unsigned*>(s_dyn + 2 * a.B);
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   pdl_wait();                 // the trees come from the kernels before this one
   pdl_launch_dependents();
   const int B = a.B, N = a.N, M = B * N;
 
-  // how many candidates there are at all
-  for (int b = t; b < B; b += SEL_THREADS) { s_gt[b] = min(max(a.n_nodes[b], 0), N); s_tie[b] = 0; }
+  for (int b = t; b < B; b += SEL_THREADS) { s_n[b] = min(max(a.n_nodes[b], 0), N); s_cnt[b] = 0; }
   __syncthreads();
+  // image of candidate e, 0 (below every key) where the tree has no node e
+  auto image = [&](int e) -> unsigned {
+    if (cached) return s_img[e];
+    const int b = e / N;
+    return e - b * N < s_n[b] ? key_image(a.logkey[e]) : 0u;
+  };
   {
-    int sum = 0;
-    for (int b = t; b < B; b += SEL_THREADS) sum += s_gt[b];
+    int sum = 0;   // how many candidates there are at all
+    for (int b = t; b < B; b += SEL_THREADS) sum += s_n[b];
+    if (cached)
+      for (int e = t; e < M; e += SEL_THREADS) {
+        const int b = e / N;
+        s_img[e] = e - b * N < s_n[b] ? key_image(a.logkey[e]) : 0u;
+      }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, off);
     if (lane == 0) s_tmp[warp] = sum;
     __syncthreads();
-    if (t == 0) { int tot = 0; for (int w = 0; w < SEL_THREADS / 32; ++w) tot += s_tmp[w]; s_total = tot; }
+    if (warp == 0) {
+      int tot = s_tmp[lane];
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xFFFFFFFFu, tot, off);
+      if (lane == 0) s_total = tot;
+    }
     __syncthreads();
   }
   const int total = s_total;
   const int want = min(max(a.budget, 0), total);
   if (want == 0 || want == total) {   // nothing to hand out, or enough for everybody: no selection
-    for (int b = t; b < B; b += SEL_THREADS) a.keep[b] = want ? s_gt[b] : 0;
+    for (int b = t; b < B; b += SEL_THREADS) a.keep[b] = want ? s_n[b] : 0;
     if (a.log_price) {
       // the smallest key of the batch is the price when every candidate is taken
-      float mn = INFINITY;
+      unsigned mn = 0xFFFFFFFFu;
       if (want)
-        for (int e = t; e < M; e += SEL_THREADS) { const int b = e / N, i = e - b * N; if (i < s_gt[b]) mn = fminf(mn, a.logkey[e] + 0.f); }
+        for (int e = t; e < M; e += SEL_THREADS) { const unsigned img = image(e); if (img) mn = min(mn, img); }
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
+      for (int off = 16; off > 0; off >>= 1) mn = min(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, off));
       __syncthreads();
-      if (lane == 0) s_tmp[warp] = __float_as_int(mn);
+      if (lane == 0) s_tmp[warp] = (int)mn;
       __syncthreads();
       if (t == 0) {
-        float m = INFINITY;
-        for (int w = 0; w < SEL_THREADS / 32; ++w) m = fminf(m, __int_as_float(s_tmp[w]));
-        *a.log_price = want ? m : -INFINITY;
+        unsigned m = 0xFFFFFFFFu;
+        for (int w = 0; w < SEL_THREADS / 32; ++w) m = min(m, (unsigned)s_tmp[w]);
+        *a.log_price = want ? key_of_image(m) : -INFINITY;
       }
     }
     return;
@@ -124,10 +140,8 @@ __global__ void __launch_bounds__(SEL_THREADS) allocate_select_kernel(const Allo
     __syncthreads();
     const unsigned prefix = s_prefix;
     for (int e = t; e < M; e += SEL_THREADS) {
-      const int b = e / N, i = e - b * N;
-      if (i >= s_gt[b]) continue;
-      const unsigned img = key_image(a.logkey[e]);
-      if ((img & fixed) == prefix) atomicAdd(&s_hist[(img >> shift) & 255u], 1);
+      const unsigned img = image(e);
+      if (img && (img & fixed) == prefix) atomicAdd(&s_hist[(img >> shift) & 255u], 1);
     }
     __syncthreads();
     if (warp == 0) {
@@ -156,39 +170,28 @@ __global__ void __launch_bounds__(SEL_THREADS) allocate_select_kernel(const Allo
   const unsigned thr = s_prefix;
   const int ties_taken = s_remaining;   // 1 .. number of candidates equal to the price
 
-  // ---- per request: candidates above the price, candidates at the price --------------------------------------
-  for (int b = t; b < B; b += SEL_THREADS) s_tie[b] = 0;
-  __syncthreads();
-  // s_gt still holds n_nodes
+  // ---- per request: candidates above the price (low half), candidates at the price (high half) -----------------
   for (int e = t; e < M; e += SEL_THREADS) {
-    const int b = e / N, i = e - b * N;
-    if (i >= s_gt[b]) continue;
-    const unsigned img = key_image(a.logkey[e]);
-    if (img == thr) atomicAdd(&s_tie[b], 1);
-    else if (img < thr) atomicAdd(&s_tie[b], 1 << 16);   // high half: candidates below the price
+    const unsigned img = image(e);
+    if (img > thr) atomicAdd(&s_cnt[e / N], 1);
+    else if (img == thr) atomicAdd(&s_cnt[e / N], 1 << 16);
   }
   __syncthreads();
-  // gt[b] = n - ties - below; then the ties are handed out in request order
-  for (int b = t; b < B; b += SEL_THREADS) {
-    const int w = s_tie[b];
-    s_gt[b] = s_gt[b] - (w & 0xFFFF) - (w >> 16);
-    s_tie[b] = w & 0xFFFF;
-  }
-  __syncthreads();
-  // keep the tie counts, scan a copy: the dynamic array has room for two ints per request only, so the
-  // scan runs in place and the count is recovered from the neighbour difference
-  int my_tie[4];   // requests b = t, t + 1024, ... (max_batch <= 4096)
-#pragma unroll
-  for (int k = 0; k < 4; ++k) { const int b = t + k * SEL_THREADS; my_tie[k] = b < B ? s_tie[b] : 0; }
-  __syncthreads();
-  block_excl_scan(s_tie, B, s_tmp, &s_total);
+  // the candidates at the price are handed out in request order: exclusive prefix sums of their counts
+  int my_gt[4], my_tie[4];   // requests b = t, t + 1024, ... (max_batch <= 4096)
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const int b = t + k * SEL_THREADS;
-    if (b < B) {
-      const int left = ties_taken - s_tie[b];
-      a.keep[b] = s_gt[b] + min(max(left, 0), my_tie[k]);
-    }
+    const int w = b < B ? s_cnt[b] : 0;
+    my_gt[k] = w & 0xFFFF; my_tie[k] = w >> 16;
+    if (b < B) s_n[b] = my_tie[k];
+  }
+  __syncthreads();
+  block_excl_scan(s_n, B, s_tmp, &s_total);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int b = t + k * SEL_THREADS;
+    if (b < B) a.keep[b] = my_gt[k] + min(max(ties_taken - s_n[b], 0), my_tie[k]);
   }
   if (t == 0 && a.log_price) *a.log_price = key_of_image(thr);
 }
@@ -307,7 +310,10 @@ extern "C" int32_t ts_allocate_budget(ts_ctx* ctx, int32_t B, int32_t budget, in
   cudaError_t e;
   {
     ProfScope ps(ctx, K_ALLOC_SELECT, st);
-    e = launch_kernel(allocate_select_kernel, dim3(1), dim3(SEL_THREADS), (size_t)2 * B * sizeof(int), st, true, a);
+    // the key images stay in shared memory between the passes when they fit the default 48 KB
+    const size_t small = (size_t)2 * B * sizeof(int), all = small + (size_t)B * c.Nmax * sizeof(unsigned);
+    const int cached = all <= 48 * 1024 - 2048 ? 1 : 0;
+    e = launch_kernel(allocate_select_kernel, dim3(1), dim3(SEL_THREADS), cached ? all : small, st, true, a, cached);
   }
   if (e == cudaSuccess) {
     ProfScope ps(ctx, K_ALLOC_CUT, st);

@@ -61,6 +61,7 @@ def budgets_for(total):
     ("wide", dict(V=9000, B=8), 0.7),          # Nmax = 256: four mask words, every thread of the cut has a node
     ("decode", dict(V=8000), 1.0),             # one request
     ("sweep", dict(V=6000, B=128), 1.0),       # 128 requests, mixed prices, chain members among them
+    ("serve32", dict(V=4000, B=256), 1.0),     # more candidates than the selection keeps in shared memory
 ])
 def test_allocation_and_cut_match_oracle(name, kw, T):
     wl = small(name, **kw)
