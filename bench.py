@@ -373,6 +373,57 @@ def allocate_side_run(args, device, steps=200):
             "oracle_water_fill_ms": t_cpu * 1e3}
 
 
+def calibrate_side_run(args, device, steps=200):
+    """Device time of the calibration-statistics calls (Section 3.4) on the headline batch: one
+    ts_calib_accumulate per verified round, and one ts_calib_refit over the accumulated cells."""
+    from oracle import calibrate as orc_cal
+    from paper_2609_22098_b200.binding import TreeSpark
+    wl = synth.WORKLOADS["serve32"]
+    B, T = wl.B, wl.temps[-1]
+    table = synth.make_calibration_table(wl, args.seed + 4, "fit")
+    A, W = synth.make_head(wl, args.seed + 1, device)
+    ts = TreeSpark(wl.V, wl.D, wl.r, wl.K, wl.Nmax, B, dtype=wl.torch_dtype, calib_mode=wl.calib_mode,
+                   calib_table=table, device=device)
+    s = InputSet(wl, args.seed + 950, B, wl.theta, A, W, device)
+    tree = ts.expand_tree(s.U, A, W, s.anchor, s.theta, T, s.round_seed)
+    torch.cuda.synchronize()
+    s.make_targets(wl, args.seed, tree)
+    verdict = ts.verify_tree(s.U, A, W, s.Z, s.zoff, s.anchor, tree, T, s.round_seed)
+    stats = ts.calib_new_stats()
+    out_table = torch.empty(wl.D, 16, dtype=torch.float32, device=device)
+    out_platt = torch.empty(4, dtype=torch.float64, device=device)
+
+    def timed(fn):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(5 + steps):
+            if i >= 5:
+                ev[i - 5][0].record()
+            fn()
+            if i >= 5:
+                ev[i - 5][1].record()
+        torch.cuda.synchronize()
+        us = sorted(a.elapsed_time(b) * 1e3 for a, b in ev)
+        return us[len(us) // 2]
+
+    acc_us = timed(lambda: ts.calib_accumulate(tree, verdict, stats))
+    fit_us = timed(lambda: ts.calib_refit(stats, 1, 4, None, out_table, out_platt))
+    edges = int(tree["n_nodes"].sum())
+    g = {k: v.cpu() for k, v in tree.items()}
+    v = {k: t.cpu() for k, t in verdict.items()}
+    ref = orc_cal.new_stats(wl.D)
+    t0 = time.perf_counter()
+    for b in range(B):
+        orc_cal.accumulate(ref, wl.D, -10.0, 10.0, int(g["n_nodes"][b]), g["parent"][b].numpy(), g["depth"][b].numpy(),
+                           g["q0"][b].numpy(), v["edge_stat"][b].numpy(), int(v["acc_len"][b]), v["acc_node"][b].numpy())
+    t_cpu = time.perf_counter() - t0
+    calls = 2 * (5 + steps)   # the same round was added this many times
+    same = bool((stats.cpu().numpy()[..., :2] == ref[..., :2] * (calls // 2)).all())
+    return {"workload": f"serve32 round ({edges} edges in {B} trees)", "accumulate_us_median": acc_us,
+            "refit_us_median": fit_us, "platt": out_platt.cpu().tolist(),
+            "counts_and_label_sums_equal_oracle": same, "oracle_accumulate_ms": t_cpu * 1e3,
+            "bound": "launch latency (one small kernel each)"}
+
+
 def run_e2e(args, ts, wl, sets, A, W, T, B, world, device, barrier):
     """Same metric through the host-buffer API: every step copies that step's inputs (base logits,
     anchors, prices, target logits) from pinned host memory and reads the round's results back."""
@@ -531,6 +582,10 @@ def main():
             out["also"]["allocate_budget"] = allocate_side_run(args, device)
         except Exception as e:
             out["also"]["allocate_budget"] = {"error": repr(e)}
+        try:
+            out["also"]["calibration"] = calibrate_side_run(args, device)
+        except Exception as e:
+            out["also"]["calibration"] = {"error": repr(e)}
     if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:

@@ -226,6 +226,45 @@ int32_t ts_allocate_budget(ts_ctx* ctx, int32_t B, int32_t budget,
                            float* log_price, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Calibration statistics from verified trees and the refit of the edge-acceptance map (Section 3.4).
+ * Verification labels every materialised edge; the map p_hat (Eq. 3, or the per-depth table) is fitted on
+ * the edges whose ancestors were all accepted, the population a path-survival product conditions on.
+ *
+ * stats: DEVICE uint64 [2][D][TS_CALIB_KNOTS][3], zeroed by the caller before the first call and added
+ * to by every call (integer sums: rounds can be accumulated in any order, on any number of streams that
+ * do not overlap).  Population 0 = every edge, 1 = edges whose ancestors were all accepted (the parent
+ * is the root or lies on the committed path).  Row = depth of the edge's parent (the row of the
+ * per-depth table that priced it); cell = the knot nearest to logit(q0) (knots uniform on
+ * [calib_lo, calib_hi], the logit clamped to [-30, 30]).  Words of a cell: number of edges; sum of
+ * labels in units of 2^-24; sum of (logit + 32) in units of 2^-24.  The label of an edge is edge_stat
+ * of ts_verify_tree: 1/0 at T == 0, the first-stage acceptance probability at T > 0.
+ *
+ * ts_calib_accumulate: adds the edges of B verified trees.  n_nodes, parent, depth, q0 as written by
+ * ts_expand_tree (or cut by ts_allocate_budget); acc_len, acc_node, edge_stat as written by
+ * ts_verify_tree for those trees.  All DEVICE.
+ *
+ * ts_calib_refit: from the cells of `population`,
+ *   platt DEVICE double[4] (or NULL) = a, b of the maximum-likelihood logistic map over the cells (each
+ *     cell = its count of edges at its mean logit with its mean label; depths pooled; Newton's method
+ *     from (1, 0), at most 50 steps, stop when both move by < 1e-12), the steps taken, the edges used;
+ *   table DEVICE float[D][TS_CALIB_KNOTS] (or NULL) = per knot (label sum + 1) / (count + 2) of its cell
+ *     (the rule-of-succession estimate: a cell whose edges were all rejected stays away from 0) where
+ *     the cell has >= min_count edges, made non-decreasing per depth by weighted pool-adjacent-violators,
+ *     knots without data interpolated linearly between neighbours with data and held constant outside,
+ *     clamped to [1e-6, 1]; a depth without data takes its row from fallback (DEVICE float[D][16]), or,
+ *     when fallback is NULL, from the context's own map sampled at the knots.
+ * ts_calib_load_table: copies a DEVICE table [D][16] (non-decreasing rows in (0, 1], as ts_calib_refit
+ *   writes them; not checked) into a context created in table mode, in stream order: calls issued after it
+ *   on the same stream price edges with the new table.  TS_ERR_INVALID in Platt mode.
+ */
+int32_t ts_calib_accumulate(ts_ctx* ctx, int32_t B, const int32_t* n_nodes, const int32_t* parent,
+                            const int32_t* depth, const float* q0, const int32_t* acc_len,
+                            const int32_t* acc_node, const float* edge_stat, uint64_t* stats, void* stream);
+int32_t ts_calib_refit(ts_ctx* ctx, const uint64_t* stats, int32_t population, int32_t min_count,
+                       const float* fallback, float* table, double* platt, void* stream);
+int32_t ts_calib_load_table(ts_ctx* ctx, const float* table, void* stream);
+
+/*
  * Instrumentation (no counterpart in the paper): per-kernel device times and launch counts.
  * ts_profile_enable(capacity > 0) creates `capacity` CUDA event pairs and from then on every kernel
  * the hot calls launch is bracketed by an event pair on the caller's stream until the pairs run out;

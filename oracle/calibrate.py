@@ -21,9 +21,11 @@ Readings taken where the paper leaves the arithmetic open:
     each cell standing for `count` edges at its mean logit with its mean label (exact when the edges of
     a cell share one logit), pooled over depths; Newton's method from (a, b) = (1, 0), at most 50 steps,
     stopped when both components move by less than 1e-12.
-  * Table refit: knot value = mean label of its cell where the cell holds at least `min_count` edges;
-    the values of a depth row are made non-decreasing by weighted pool-adjacent-violators (weights =
-    counts); knots without data are filled by linear interpolation between their neighbours with data
+  * Table refit: knot value = (label sum + 1) / (count + 2) of its cell -- the rule-of-succession
+    estimate, the smoothing Platt's method applies to its targets; it keeps a cell whose edges were all
+    rejected away from 0, where log p_hat would be unbounded -- where the cell holds at least
+    `min_count` edges; the values of a depth row are made non-decreasing by weighted
+    pool-adjacent-violators (weights = counts); knots without data are filled by linear interpolation between their neighbours with data
     and held constant outside them; a depth row without any data keeps the row given as `fallback`;
     everything is clamped to [1e-6, 1] (the table format wants values in (0, 1]).
 """
@@ -142,7 +144,7 @@ def refit_table(stats, pop, min_count, fallback):
         have = [j for j in range(KNOTS) if int(stats[pop][d][j][0]) >= max(int(min_count), 1)]
         if not have:
             continue
-        vals = [int(stats[pop][d][j][1]) / UNIT / int(stats[pop][d][j][0]) for j in have]
+        vals = [(int(stats[pop][d][j][1]) / UNIT + 1.0) / (int(stats[pop][d][j][0]) + 2.0) for j in have]
         wts = [int(stats[pop][d][j][0]) for j in have]
         iso = pav(vals, wts)
         row = np.empty(KNOTS)

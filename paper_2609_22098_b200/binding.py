@@ -21,7 +21,8 @@ KNOTS = 16
 
 EXPORTS = ("ts_create", "ts_destroy", "ts_workspace_bytes", "ts_last_error_string",
            "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",
-           "ts_allocate_budget", "ts_profile_enable", "ts_profile_read", "ts_kernel_name")
+           "ts_allocate_budget", "ts_calib_accumulate", "ts_calib_refit", "ts_calib_load_table",
+           "ts_profile_enable", "ts_profile_read", "ts_kernel_name")
 
 
 class TsConfig(C.Structure):
@@ -53,12 +54,16 @@ def load_library() -> C.CDLL:
         L.ts_expand_tree.argtypes = [vp, vp, vp, vp, i32, vp, vp, f32, u64] + [vp] * 15 + [vp, sz, vp]
         L.ts_verify_tree.argtypes = [vp, vp, vp, vp, vp, vp, i32] + [vp] * 9 + [f32, u64] + [vp] * 7 + [vp, sz, vp]
         L.ts_allocate_budget.argtypes = [vp, i32, i32] + [vp] * 14 + [vp, sz, vp]
+        L.ts_calib_accumulate.argtypes = [vp, i32] + [vp] * 8 + [vp]
+        L.ts_calib_refit.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+        L.ts_calib_load_table.argtypes = [vp, vp, vp]
         L.ts_profile_enable.argtypes = [vp, i32]
         L.ts_profile_read.argtypes = [vp, i32, vp, vp, i32]
         L.ts_kernel_name.argtypes = [i32]
         L.ts_kernel_name.restype = C.c_char_p
         for n in ("ts_create", "ts_destroy", "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",
-                  "ts_allocate_budget", "ts_profile_enable", "ts_profile_read"):
+                  "ts_allocate_budget", "ts_calib_accumulate", "ts_calib_refit", "ts_calib_load_table",
+           "ts_profile_enable", "ts_profile_read"):
             getattr(L, n).restype = C.c_int32
         _lib = L
     return _lib
@@ -197,6 +202,30 @@ class TreeSpark:
                                                 _ptr(tree["node_lseT"]), _ptr(tree["mask"]), _ptr(log_price),
                                                 _ptr(self.ws), self.ws_bytes, _stream()))
         return tree
+
+    # -- calibration statistics (Section 3.4) -------------------------------------------------------
+    def calib_new_stats(self) -> torch.Tensor:
+        """Zeroed statistics array [2][D][16][3] (int64 holding the library's unsigned 64-bit sums)."""
+        return torch.zeros(2, self.D, KNOTS, 3, dtype=torch.int64, device=self.device)
+
+    def calib_accumulate(self, tree, verdict, stats):
+        B = int(tree["n_nodes"].numel())
+        self._check(self.lib.ts_calib_accumulate(self._ctx, B, _ptr(tree["n_nodes"]), _ptr(tree["parent"]),
+                                                 _ptr(tree["depth"]), _ptr(tree["q0"]), _ptr(verdict["acc_len"]),
+                                                 _ptr(verdict["acc_node"]), _ptr(verdict["edge_stat"]), _ptr(stats),
+                                                 _stream()))
+        return stats
+
+    def calib_refit(self, stats, population=1, min_count=1, fallback=None, table=None, platt=None):
+        """(table float32 [D][16], platt float64 [4] = a, b, Newton steps, edges used), both on the device."""
+        table = torch.empty(self.D, KNOTS, dtype=torch.float32, device=self.device) if table is None else table
+        platt = torch.empty(4, dtype=torch.float64, device=self.device) if platt is None else platt
+        self._check(self.lib.ts_calib_refit(self._ctx, _ptr(stats), int(population), int(min_count), _ptr(fallback),
+                                            _ptr(table), _ptr(platt), _stream()))
+        return table, platt
+
+    def calib_load_table(self, table):
+        self._check(self.lib.ts_calib_load_table(self._ctx, _ptr(table), _stream()))
 
     def verify_tree(self, U, A, W, Z, z_row_off, anchor_tok, tree, T, seed, out=None, edge_stat=True):
         B = int(anchor_tok.numel())

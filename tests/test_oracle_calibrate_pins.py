@@ -137,7 +137,7 @@ def test_monotone_table_matches_a_library_isotonic_regression():
         assert np.array_equal(table[2], fallback[2])
         for d in range(2):
             have = [j for j in range(cal.KNOTS) if stats[1, d, j, 0] >= min_count]
-            vals = [stats[1, d, j, 1] / cal.UNIT / stats[1, d, j, 0] for j in have]
+            vals = [(stats[1, d, j, 1] / cal.UNIT + 1) / (stats[1, d, j, 0] + 2) for j in have]   # rule of succession
             wts = [stats[1, d, j, 0] for j in have]
             lib = IsotonicRegression(increasing=True, out_of_bounds="clip").fit(have, vals, sample_weight=wts)
             want = np.clip(lib.predict(np.arange(cal.KNOTS)), 1e-6, 1.0)   # linear between data knots, constant outside
@@ -145,10 +145,11 @@ def test_monotone_table_matches_a_library_isotonic_regression():
             assert (np.diff(table[d]) >= -1e-15).all() and (table[d] > 0).all() and (table[d] <= 1).all()
 
 
-def test_monotone_cells_are_left_as_measured():
+def test_monotone_cells_keep_their_smoothed_frequencies():
     stats = cal.new_stats(1)
-    rates = np.linspace(0.05, 0.95, cal.KNOTS)
+    rates = np.linspace(0.0, 1.0, cal.KNOTS)                  # the ends: all rejected, all accepted
     for j in range(cal.KNOTS):
         stats[0, 0, j] = (1000, int(round(rates[j] * 1000)) << 24, 0)
     table = cal.refit_table(stats, 0, 1, np.zeros((1, cal.KNOTS)) + 0.5)
-    assert np.allclose(table[0], np.round(rates * 1000) / 1000, atol=1e-12)
+    assert np.allclose(table[0], (np.round(rates * 1000) + 1) / 1002, atol=1e-12)
+    assert table[0, 0] == pytest.approx(1 / 1002) and table[0, -1] == pytest.approx(1001 / 1002)
