@@ -246,7 +246,8 @@ int32_t ts_allocate_budget(ts_ctx* ctx, int32_t B, int32_t budget,
  * ts_calib_refit: from the cells of `population`,
  *   platt DEVICE double[4] (or NULL) = a, b of the maximum-likelihood logistic map over the cells (each
  *     cell = its count of edges at its mean logit with its mean label; depths pooled; Newton's method
- *     from (1, 0), at most 50 steps, stop when both move by < 1e-12), the steps taken, the edges used;
+ *     from (0, 0), 1e-12 on the Hessian's diagonal, the step halved until the likelihood does not get
+ *     worse, at most 100 steps, stop when both move by < 1e-12), the steps taken, the edges used;
  *   table DEVICE float[D][TS_CALIB_KNOTS] (or NULL) = per knot (label sum + 1) / (count + 2) of its cell
  *     (the rule-of-succession estimate: a cell whose edges were all rejected stays away from 0) where
  *     the cell has >= min_count edges, made non-decreasing per depth by weighted pool-adjacent-violators,

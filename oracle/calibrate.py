@@ -19,8 +19,11 @@ Readings taken where the paper leaves the arithmetic open:
     first-stage acceptance probability min(1, p(x)/q_T(x)) at T > 0.
   * Two-scalar refit (Eq. 3): maximum likelihood of the logistic model over the cells of one population,
     each cell standing for `count` edges at its mean logit with its mean label (exact when the edges of
-    a cell share one logit), pooled over depths; Newton's method from (a, b) = (1, 0), at most 50 steps,
-    stopped when both components move by less than 1e-12.
+    a cell share one logit), pooled over depths; Newton's method from (a, b) = (0, 0) with 1e-12 added
+    to the Hessian's diagonal and the step halved (at most 30 times) until the likelihood does not get
+    worse -- the safeguards of the usual implementation of Platt scaling; a plain Newton step from a
+    start where most cells are saturated overshoots --, at most 100 steps, stopped when both components
+    move by less than 1e-12 or no step helps.
   * Table refit: knot value = (label sum + 1) / (count + 2) of its cell -- the rule-of-succession
     estimate, the smoothing Platt's method applies to its targets; it keeps a cell whose edges were all
     rejected away from 0, where log p_hat would be unbounded -- where the cell holds at least
@@ -85,10 +88,21 @@ def new_stats(D):
     return np.zeros((2, D, KNOTS, 3), dtype=np.int64)
 
 
-def fit_platt(cells, max_iter=50, tol=1e-12):
+def neg_log_likelihood(cells, a, b):
+    f = 0.0
+    for n, x, y in cells:
+        if n <= 0:
+            continue
+        z = a * x + b
+        f += n * (max(z, 0.0) + math.log1p(math.exp(-abs(z))) - y * z)
+    return f
+
+
+def fit_platt(cells, max_iter=100, tol=1e-12):
     """Maximum-likelihood (a, b) of y ~ sigmoid(a x + b) over weighted cells [(count, mean x, mean y)].
     Returns (a, b, iterations)."""
-    a, b = 1.0, 0.0
+    a, b = 0.0, 0.0
+    f = neg_log_likelihood(cells, a, b)
     it = 0
     for it in range(1, max_iter + 1):
         ga = gb = haa = hab = hbb = 0.0
@@ -100,13 +114,25 @@ def fit_platt(cells, max_iter=50, tol=1e-12):
             w = n * p * (1.0 - p)
             ga += r * x; gb += r
             haa += w * x * x; hab += w * x; hbb += w
+        haa += 1e-12; hbb += 1e-12
         det = haa * hbb - hab * hab
         if not (det > 1e-300):
             break
         da = (hbb * ga - hab * gb) / det
         db = (haa * gb - hab * ga) / det
-        a += da; b += db
-        if abs(da) < tol and abs(db) < tol:
+        step, ok = 1.0, False
+        for _ in range(30):                                   # halve the step until the likelihood does not get worse
+            na, nb = a + step * da, b + step * db
+            nf = neg_log_likelihood(cells, na, nb)
+            if nf <= f:
+                ok = True
+                break
+            step *= 0.5
+        if not ok:
+            break
+        moved = max(abs(na - a), abs(nb - b))
+        a, b, f = na, nb, nf
+        if moved < tol:
             break
     return a, b, it
 

@@ -6,8 +6,8 @@
 // a histogram in shared memory, and the CTA's non-empty cells go to the caller's array with one atomic
 // each.  Integer sums: the array does not depend on the order in which CTAs, rounds or streams add.
 //
-// Refit: one CTA, one thread per cell (depth row, knot).  The two scalars of Eq. 3 by Newton's method on
-// the cell-weighted logistic likelihood (five block-wide sums per step, every thread takes the same
+// Refit: one CTA, one thread per cell (depth row, knot).  The two scalars of Eq. 3 by Newton's method with
+// step halving on the cell-weighted logistic likelihood (block-wide sums, every thread takes the same
 // step), the table by pool-adjacent-violators over the sixteen cells of a depth row (one thread per row).
 #include "ts_internal.h"
 
@@ -109,9 +109,19 @@ __global__ void __launch_bounds__(CAL_THREADS) calib_refit_kernel(const CalFitAr
 
   // ---- the two scalars of Eq. 3 -------------------------------------------------------------------
   if (a.platt) {
-    double pa = 1.0, pb = 0.0;
+    // negative log-likelihood of the cells under (qa, qb); the same value in every thread
+    auto nll = [&](double qa, double qb) -> double {
+      double f = 0.0;
+      if (has) {
+        const double z = qa * x + qb;
+        f = n * (fmax(z, 0.0) + log1p(exp(-fabs(z))) - y * z);
+      }
+      return block_sum(f, s_part);
+    };
+    double pa = 0.0, pb = 0.0;
+    double f = nll(pa, pb);
     int it = 0;
-    for (it = 1; it <= 50; ++it) {
+    for (it = 1; it <= 100; ++it) {
       double r = 0.0, w = 0.0;
       if (has) {
         const double p = 1.0 / (1.0 + exp(-(pa * x + pb)));
@@ -119,14 +129,26 @@ __global__ void __launch_bounds__(CAL_THREADS) calib_refit_kernel(const CalFitAr
         w = n * p * (1.0 - p);
       }
       const double ga = block_sum(r * x, s_part), gb = block_sum(r, s_part);
-      const double haa = block_sum(w * x * x, s_part), hab = block_sum(w * x, s_part), hbb = block_sum(w, s_part);
+      const double haa = block_sum(w * x * x, s_part) + 1e-12, hab = block_sum(w * x, s_part);
+      const double hbb = block_sum(w, s_part) + 1e-12;
       const double det = haa * hbb - hab * hab;
       if (!(det > 1e-300)) break;
       const double da = (hbb * ga - hab * gb) / det, db = (haa * gb - hab * ga) / det;
-      pa += da; pb += db;
-      if (fabs(da) < 1e-12 && fabs(db) < 1e-12) break;
+      // halve the step until the likelihood does not get worse (every thread takes the same decisions)
+      double step = 1.0, na = pa, nb = pb, nf = f;
+      bool ok = false;
+      for (int h = 0; h < 30; ++h) {
+        na = pa + step * da; nb = pb + step * db;
+        nf = nll(na, nb);
+        if (nf <= f) { ok = true; break; }
+        step *= 0.5;
+      }
+      if (!ok) break;
+      const double moved = fmax(fabs(na - pa), fabs(nb - pb));
+      pa = na; pb = nb; f = nf;
+      if (moved < 1e-12) break;
     }
-    if (it > 50) it = 50;
+    if (it > 100) it = 100;
     const double used = block_sum(n, s_part);
     if (t == 0) { a.platt[0] = pa; a.platt[1] = pb; a.platt[2] = (double)it; a.platt[3] = used; }
   }

@@ -97,8 +97,25 @@ def test_two_scalar_fit_matches_a_library_logistic_regression():
     a, b, it = cal.fit_platt(cells)
     lib = LogisticRegression(C=np.inf, tol=1e-12, max_iter=10000).fit(np.array(X), np.array(y), sample_weight=np.array(w))
     assert abs(a - lib.coef_[0, 0]) < 1e-5 and abs(b - lib.intercept_[0]) < 1e-5
-    assert it < 50
+    assert it < 30
     assert abs(a - a0) < 0.05 and abs(b - b0) < 0.08          # and it recovers the generating map
+
+
+def test_two_scalar_fit_survives_cells_far_out_in_the_tails():
+    # logits spread over the whole knot range with most of the mass in the tails: an unguarded Newton step
+    # from a saturated start leaves for infinity; the guarded iteration lands on the library's optimum
+    rng = np.random.default_rng(9)
+    xs = np.linspace(-10, 10, 16)
+    cells, X, y, w = [], [], [], []
+    for x in xs:
+        n = int(3000 * (0.1 + abs(x) / 10))
+        s = int(rng.binomial(n, 1 / (1 + math.exp(-(1.4 * x + 0.8)))))
+        cells.append((float(n), float(x), s / n))
+        X += [[x], [x]]; y += [1, 0]; w += [s, n - s]
+    a, b, it = cal.fit_platt(cells)
+    lib = LogisticRegression(C=np.inf, tol=1e-12, max_iter=10000).fit(np.array(X), np.array(y), sample_weight=np.array(w))
+    assert abs(a - lib.coef_[0, 0]) < 1e-4 and abs(b - lib.intercept_[0]) < 1e-4
+    assert abs(a - 1.4) < 0.1 and it < 40
 
 
 def test_two_scalar_fit_closed_form_with_two_logits():
