@@ -405,6 +405,8 @@ def calibrate_side_run(args, device, steps=200):
         us = sorted(a.elapsed_time(b) * 1e3 for a, b in ev)
         return us[len(us) // 2]
 
+    att = ts.emit_attention_inputs(s.anchor, tree)
+    att_us = timed(lambda: ts.emit_attention_inputs(s.anchor, tree, out=att))
     acc_us = timed(lambda: ts.calib_accumulate(tree, verdict, stats))
     fit_us = timed(lambda: ts.calib_refit(stats, 1, 4, None, out_table, out_platt))
     edges = int(tree["n_nodes"].sum())
@@ -421,6 +423,8 @@ def calibrate_side_run(args, device, steps=200):
     return {"workload": f"serve32 round ({edges} edges in {B} trees)", "accumulate_us_median": acc_us,
             "refit_us_median": fit_us, "platt": out_platt.cpu().tolist(),
             "counts_and_label_sums_equal_oracle": same, "oracle_accumulate_ms": t_cpu * 1e3,
+            "attention_inputs_us_median": att_us,
+            "attention_inputs_bytes": int(sum(t.numel() * t.element_size() for t in att.values())),
             "bound": "launch latency (one small kernel each)"}
 
 

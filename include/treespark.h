@@ -226,6 +226,23 @@ int32_t ts_allocate_budget(ts_ctx* ctx, int32_t B, int32_t budget,
                            float* log_price, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Inputs of the target forward over the flattened trees (Section 3.2 item 3: row i attends to its root
+ * path only; a node's position is its depth below the anchor), in a dense layout an attention kernel
+ * can take as is.  Per request Nmax + 1 rows: row 0 = the anchor (root), row 1 + i = node i.
+ *   flat_tok [B][Nmax+1]: anchor token, then node tokens; -1 in unused rows.
+ *   pos_ids  [B][Nmax+1]: base_pos[b] + depth (base_pos DEVICE [B] or NULL = 0); 0 in unused rows.
+ *   dense_mask [B][Nmax+1][Nmax+1] float: 0 where the row may attend the column, -inf elsewhere.  An
+ *     unused row attends to itself only (a softmax over it stays defined); no used row attends to an
+ *     unused column.
+ * n_nodes, tok, depth, mask as written by ts_expand_tree.  Any of the three outputs may be NULL.
+ * All DEVICE.  No counterpart of this layout is fixed by the paper.
+ */
+int32_t ts_emit_attention_inputs(ts_ctx* ctx, int32_t B, const int32_t* anchor_tok, const int32_t* base_pos,
+                                 const int32_t* n_nodes, const int32_t* tok, const int32_t* depth,
+                                 const uint64_t* mask, int32_t* flat_tok, int32_t* pos_ids,
+                                 float* dense_mask, void* stream);
+
+/*
  * Calibration statistics from verified trees and the refit of the edge-acceptance map (Section 3.4).
  * Verification labels every materialised edge; the map p_hat (Eq. 3, or the per-depth table) is fitted on
  * the edges whose ancestors were all accepted, the population a path-survival product conditions on.

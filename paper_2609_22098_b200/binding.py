@@ -22,7 +22,7 @@ KNOTS = 16
 EXPORTS = ("ts_create", "ts_destroy", "ts_workspace_bytes", "ts_last_error_string",
            "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",
            "ts_allocate_budget", "ts_calib_accumulate", "ts_calib_refit", "ts_calib_load_table",
-           "ts_profile_enable", "ts_profile_read", "ts_kernel_name")
+           "ts_emit_attention_inputs", "ts_profile_enable", "ts_profile_read", "ts_kernel_name")
 
 
 class TsConfig(C.Structure):
@@ -57,13 +57,14 @@ def load_library() -> C.CDLL:
         L.ts_calib_accumulate.argtypes = [vp, i32] + [vp] * 8 + [vp]
         L.ts_calib_refit.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
         L.ts_calib_load_table.argtypes = [vp, vp, vp]
+        L.ts_emit_attention_inputs.argtypes = [vp, i32] + [vp] * 9 + [vp]
         L.ts_profile_enable.argtypes = [vp, i32]
         L.ts_profile_read.argtypes = [vp, i32, vp, vp, i32]
         L.ts_kernel_name.argtypes = [i32]
         L.ts_kernel_name.restype = C.c_char_p
         for n in ("ts_create", "ts_destroy", "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",
                   "ts_allocate_budget", "ts_calib_accumulate", "ts_calib_refit", "ts_calib_load_table",
-           "ts_profile_enable", "ts_profile_read"):
+           "ts_emit_attention_inputs", "ts_profile_enable", "ts_profile_read"):
             getattr(L, n).restype = C.c_int32
         _lib = L
     return _lib
@@ -202,6 +203,18 @@ class TreeSpark:
                                                 _ptr(tree["node_lseT"]), _ptr(tree["mask"]), _ptr(log_price),
                                                 _ptr(self.ws), self.ws_bytes, _stream()))
         return tree
+
+    def emit_attention_inputs(self, anchor_tok, tree, base_pos=None, out=None):
+        """Token ids, position ids and the dense additive mask of the flattened trees (Section 3.2 item 3)."""
+        B, R, d = int(anchor_tok.numel()), self.Nmax + 1, self.device
+        out = out or dict(flat_tok=torch.empty(B, R, dtype=torch.int32, device=d),
+                          pos_ids=torch.empty(B, R, dtype=torch.int32, device=d),
+                          dense_mask=torch.empty(B, R, R, dtype=torch.float32, device=d))
+        self._check(self.lib.ts_emit_attention_inputs(self._ctx, B, _ptr(anchor_tok), _ptr(base_pos), _ptr(tree["n_nodes"]),
+                                                      _ptr(tree["tok"]), _ptr(tree["depth"]), _ptr(tree["mask"]),
+                                                      _ptr(out.get("flat_tok")), _ptr(out.get("pos_ids")),
+                                                      _ptr(out.get("dense_mask")), _stream()))
+        return out
 
     # -- calibration statistics (Section 3.4) -------------------------------------------------------
     def calib_new_stats(self) -> torch.Tensor:

@@ -78,7 +78,7 @@ cudaError_t launch_score_few(const ts_ctx* ctx, const ScoreArgs& a, int p_bound,
 // encodes (or finds cached in the context) the tensor map of W for 64-token boxes; false: not available
 bool w_tensor_map(ts_ctx* ctx, const void* W);
 
-enum KernelId { K_INIT, K_SCORE, K_MERGE, K_LEVEL, K_FINAL, K_ZROWS, K_GREEDY, K_WALK, K_CHECK, K_SCORE_FEW, K_ALLOC_SELECT, K_ALLOC_CUT, K_CALIB_ACC, K_CALIB_FIT, K_COUNT };
+enum KernelId { K_INIT, K_SCORE, K_MERGE, K_LEVEL, K_FINAL, K_ZROWS, K_GREEDY, K_WALK, K_CHECK, K_SCORE_FEW, K_ALLOC_SELECT, K_ALLOC_CUT, K_CALIB_ACC, K_CALIB_FIT, K_ATTN_INPUTS, K_COUNT };
 
 struct Prof {
   bool on = false;
