@@ -69,7 +69,7 @@ typedef struct {
 
 /* Create / destroy a context on the current device.  Create copies the calibration table to the
  * device (the only allocation the library ever makes).  Errors: TS_ERR_INVALID, TS_ERR_UNSUPPORTED
- * (K > 16, D > 16, Nmax > 256, r > 128, mixed dtypes), TS_ERR_CUDA. */
+ * (K > 16, D > 16, Nmax > 256, r > 256, mixed dtypes), TS_ERR_CUDA. */
 int32_t ts_create(const ts_config* cfg, ts_ctx** out);
 int32_t ts_destroy(ts_ctx* ctx);
 

@@ -51,9 +51,9 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
   *out = nullptr;
   if (cfg->V < 1 || cfg->D < 1 || cfg->r < 1 || cfg->K < 1 || cfg->Nmax < 1 || cfg->max_batch < 1)
     return set_error(TS_ERR_INVALID, "ts_create: sizes must be positive");
-  if (cfg->K > TS_KMAX || cfg->D > TS_DMAX || cfg->Nmax > 256 || cfg->r > 128 || cfg->max_batch > 4096 ||
+  if (cfg->K > TS_KMAX || cfg->D > TS_DMAX || cfg->Nmax > 256 || cfg->r > RMAX || cfg->max_batch > 4096 ||
       cfg->V > (1 << 24))
-    return set_error(TS_ERR_UNSUPPORTED, "ts_create: K<=16, D<=16, Nmax<=256, r<=128, batch<=4096, V<=2^24 required");
+    return set_error(TS_ERR_UNSUPPORTED, "ts_create: K<=16, D<=16, Nmax<=256, r<=256, batch<=4096, V<=2^24 required");
   if (cfg->dt_U != cfg->dt_A || cfg->dt_U != cfg->dt_W || cfg->dt_U != cfg->dt_Z ||
       (cfg->dt_U != TS_DTYPE_F32 && cfg->dt_U != TS_DTYPE_BF16))
     return set_error(TS_ERR_UNSUPPORTED, "ts_create: U, A, W, Z must share one dtype (f32 or bf16)");

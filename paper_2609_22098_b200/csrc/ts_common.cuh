@@ -13,6 +13,7 @@ namespace ts {
 constexpr int KMAX = TS_KMAX;
 constexpr int DMAX = TS_DMAX;
 constexpr int KNOTS = TS_CALIB_KNOTS;
+constexpr int RMAX = 256;   // largest Markov rank r (the paper's head has r = 256)
 // Programmatic dependent launch (the kernels of one expansion are chained with it).  pdl_wait(): everything
 // the kernels before this one in the stream wrote is visible afterwards; a kernel launched without the
 // attribute passes straight through.  pdl_launch_dependents(): the next kernel in the stream may start its

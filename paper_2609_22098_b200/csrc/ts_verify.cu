@@ -384,7 +384,7 @@ __device__ __forceinline__ void logits_group(const VerifyArgs& a, const float* a
     else { const float4 x = *reinterpret_cast<const float4*>(Wsrc + (size_t)k * wstride + woff); w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w; }
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      const float ak = as[g * 128 + k];
+      const float ak = as[g * RMAX + k];
 #pragma unroll
       for (int i = 0; i < VEC; ++i) acc[g][i] = fmaf(ak, w[i], acc[g][i]);
     }
@@ -441,7 +441,7 @@ __device__ __forceinline__ void sweep_item(const SweepCtx<TIn>& c, int g0, int c
         else { const float4 x = *reinterpret_cast<const float4*>(wp + (size_t)k * c.wstride); w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w; }
 #pragma unroll
         for (int g = 0; g < NG; ++g) {
-          const float ak = c.a[(g0 + g) * 128 + k];
+          const float ak = c.a[(g0 + g) * RMAX + k];
 #pragma unroll
           for (int i = 0; i < VEC; ++i) acc[g][i] = fmaf(ak, w[i], acc[g][i]);
         }
@@ -652,13 +652,13 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
 template <typename TIn, bool MMA>
 __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsigned char* w_raw) {
   constexpr int SBX = MMA ? 128 : SB;   // requests per reduction pass
-  __shared__ float s_a[VG * 128];
+  __shared__ float s_a[VG * RMAX];
   __shared__ int s_req[VG], s_dep[VG], s_node[VG];
   __shared__ float s_C[VG], s_zmax[VG], s_zlogs[VG], s_lseT[VG];
   __shared__ float s_red[VG][WT / 32];
   __shared__ double s_scan[WT];
   __shared__ int s_found, s_last;
-  __shared__ float sb_a[MMA ? 256 : SB * 128];
+  __shared__ float sb_a[MMA ? 256 : SB * RMAX];
   __shared__ int sb_req[SBX], sb_dep[SBX], sb_tok[SBX];
   __shared__ long long sb_row[SBX];
   __shared__ float sb_C[SBX], sb_zmax[SBX], sb_zlogs[SBX], sb_lseT[SBX], sb_part[MMA ? 256 : SB * 16];
@@ -794,7 +794,7 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
         __syncthreads();
         for (int i = tid; i < nreq * a.r; i += WT) {
           const int g = i / a.r, k = i % a.r;
-          sb_a[g * 128 + k] = Elem<TIn>::to_f(Ag[(size_t)sb_tok[g] * a.r + k]);
+          sb_a[g * RMAX + k] = Elem<TIn>::to_f(Ag[(size_t)sb_tok[g] * a.r + k]);
         }
         __syncthreads();
         const int ngrp = (nreq + VG - 1) / VG;
@@ -837,7 +837,7 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
         const int g = i / a.r, k = i % a.r;
         const int v = s_node[g];
         const int ptok = v < 0 ? a.anchor[s_req[g]] : a.tok[(size_t)s_req[g] * N + v];
-        s_a[g * 128 + k] = Elem<TIn>::to_f(Ag[(size_t)ptok * a.r + k]);
+        s_a[g * RMAX + k] = Elem<TIn>::to_f(Ag[(size_t)ptok * a.r + k]);
       }
       __syncthreads();
       float sum[VG];
@@ -1086,11 +1086,11 @@ __global__ void verify_check_kernel(VerifyArgs a) {
 cudaError_t verify_setup(ts_ctx* ctx) {
   // the walk kernel may keep its range of W in shared memory: allow the full opt-in size
   cudaError_t e = cudaFuncSetAttribute(verify_walk_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       ctx->max_smem - 32 * 1024);
+                                       ctx->max_smem - 40 * 1024);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(verify_walk_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem - 32 * 1024);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(verify_walk_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem - 32 * 1024);
+  return cudaFuncSetAttribute(verify_walk_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem - 40 * 1024);
 }
 
 }  // namespace ts
@@ -1153,7 +1153,7 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
     return TS_OK;
   }
   size_t w_bytes = (size_t)c.r * ctx->vt_TV * (c.dt_W == TS_DTYPE_BF16 ? 2 : 4);
-  a.w_smem = (w_bytes + 32 * 1024 <= (size_t)ctx->max_smem) ? 1 : 0;
+  a.w_smem = (w_bytes + 40 * 1024 <= (size_t)ctx->max_smem) ? 1 : 0;
   // tensor-core reductions: bf16 everywhere, the range of W in operand layout plus the A tile within shared memory
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
   const size_t mma_bytes = (size_t)(ctx->vt_TV / 64) * rp * 128 + (rp / 64) * 128 * 128 + (2 * WALK_NBUF + WALK_MAX_BLK) * 8 + 64 + 1024;

@@ -164,6 +164,11 @@ WORKLOADS = {
     "sweep": Workload("sweep", B=16, V=151936, D=8, r=64, K=8, Nmax=64, dtype="bf16", theta=0.1,
                       temps=(1.0,), u_std=4.0, plant_lo=3.0, plant_hi=9.0,
                       plant_per_request=True, z_sigma=0.8),
+    # The paper's own head and tree shape (Section 5.1: rank 256, block of 7, at most 56 nodes, 8 siblings)
+    # on the serving batch; inputs as in serve32.
+    "paper": Workload("paper", B=32, V=151936, D=7, r=256, K=8, Nmax=56, dtype="bf16", theta=0.1,
+                      temps=(1.0,), u_std=4.0, plant_lo=3.0, plant_hi=9.0,
+                      plant_per_request=True, z_sigma=0.8),
 }
 
 SWEEP_BATCHES = (1, 4, 16, 64, 128)

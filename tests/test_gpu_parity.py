@@ -24,7 +24,8 @@ def small(name, **kw):
 # ts_score_parents
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("V,r,K", [(1000, 7, 4), (1003, 16, 8), (4096 + 40, 64, 8), (70000, 32, 16), (8, 4, 4), (5, 3, 8)])
+@pytest.mark.parametrize("V,r,K", [(1000, 7, 4), (1003, 16, 8), (4096 + 40, 64, 8), (70000, 32, 16), (8, 4, 4), (5, 3, 8),
+                                   (9000 + 16, 256, 8), (3000, 200, 4)])   # the paper's rank, and one that pads to it
 @pytest.mark.parametrize("T", [0.0, 0.7, 1.0])
 @pytest.mark.parametrize("P", [11, 3])   # 3: the few-parents kernel where the context has one
 def test_score_parents_matches_oracle(dtype, V, r, K, T, P):
@@ -210,6 +211,19 @@ def test_ablation_settings_match_oracle(which):
     for T in (0.0, 1.0):
         st = check_round(ts, orc, rnd, T, round_seed=31)
         assert st["trees"] == rnd.B
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_round_at_the_papers_own_shape_matches_oracle(dtype):
+    # rank 256, block of 7, 56 nodes, 8 siblings (Section 5.1), on a vocabulary the oracle finishes quickly
+    wl = small("serve32", V=20000 + 8, r=256, D=7, Nmax=56, K=8, B=6, dtype=dtype)
+    rnd = Round(wl, seed=97)
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
+    orc = make_oracle(wl, rnd.table)
+    rnd.theta.fill_(0.03)
+    for T in (0.0, 1.0):
+        st = check_round(ts, orc, rnd, T, round_seed=41)
+        assert st["trees"] == rnd.B and st["nodes"] > 4 * rnd.B
 
 
 def test_chain_sentinel_and_mixed_prices():
