@@ -44,7 +44,8 @@ def build(force: bool = False) -> str:
 class _Config(C.Structure):
     _fields_ = [("V", C.c_int32), ("D", C.c_int32), ("r", C.c_int32), ("K", C.c_int32), ("Nmax", C.c_int32),
                 ("calib_mode", C.c_int32), ("platt_a", C.c_double), ("platt_b", C.c_double),
-                ("calib_lo", C.c_double), ("calib_hi", C.c_double), ("calib_table", C.POINTER(C.c_double))]
+                ("calib_lo", C.c_double), ("calib_hi", C.c_double), ("calib_table", C.POINTER(C.c_double)),
+                ("calib_input", C.c_int32)]
 
 
 _lib = None
@@ -84,7 +85,7 @@ class Oracle:
     """One configuration of the method (vocabulary, depth, rank, caps, calibration)."""
 
     def __init__(self, V, D, r, K, Nmax, calib_mode=0, platt_a=0.67, platt_b=-0.46,
-                 calib_lo=-10.0, calib_hi=10.0, calib_table=None):
+                 calib_lo=-10.0, calib_hi=10.0, calib_table=None, calib_input=0):
         assert K <= KMAX and D <= DMAX
         self.V, self.D, self.r, self.K, self.Nmax = V, D, r, K, Nmax
         self.words = (Nmax + 63) // 64
@@ -92,7 +93,7 @@ class Oracle:
         if calib_mode == 1:
             self._table = np.ascontiguousarray(np.asarray(calib_table, dtype=np.float64).reshape(D, KNOTS))
         self.cfg = _Config(V, D, r, K, Nmax, calib_mode, platt_a, platt_b, calib_lo, calib_hi,
-                           _p(self._table, C.c_double) if self._table is not None else None)
+                           _p(self._table, C.c_double) if self._table is not None else None, calib_input)
 
     # -- scalars ---------------------------------------------------------------------------
     def calib(self, d: int, t: float) -> float:

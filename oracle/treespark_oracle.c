@@ -307,11 +307,15 @@ static void score_node(expand_ctx* c, node_t* nd) {
  * sum is taken directly from the parent's recomputed logit vector. */
 static double edge_logit_q0(expand_ctx* c, const node_t* nd, int x, double lx) {
   const orc_config* cfg = c->cfg;
-  double lq = lx - nd->lse0;
+  /* ablation: the calibrator sees the tempered conditional q_T instead of q0 */
+  const int tempered = cfg->calib_input == 1 && c->T > 0.0;
+  const double scale = tempered ? 1.0 / c->T : 1.0;
+  double lq = tempered ? lx / c->T - nd->lseT : lx - nd->lse0;
   double qv = exp(lq);
   if (qv <= 0.5) return lq - log1p(-qv);
   double* l = (double*)malloc(sizeof(double) * (size_t)cfg->V);
   orc_logits(cfg, c->U_req + (size_t)nd->depth * cfg->V, c->A + (size_t)nd->tok * cfg->r, c->W, l);
+  if (tempered) for (int v = 0; v < cfg->V; ++v) l[v] *= scale;
   double m = l[0];
   for (int v = 1; v < cfg->V; ++v) if (l[v] > m) m = l[v];
   double s0 = 0.0;

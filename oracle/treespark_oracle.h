@@ -44,6 +44,8 @@ typedef struct {
   double platt_a, platt_b;
   double calib_lo, calib_hi;     /* knot range in logit(q0) */
   const double* calib_table;     /* [D][16] when calib_mode == 1 */
+  int32_t calib_input;           /* 0 = the calibrator is fed the untempered q0 (the method); 1 = it is fed
+                                    q_T when T > 0 (the ablation of Section 5.5) */
 } orc_config;
 
 /* Philox4x32-10 (Salmon et al., SC'11). */

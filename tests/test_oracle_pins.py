@@ -354,6 +354,37 @@ def test_calibrator_is_fed_the_untempered_conditional():
     assert abs(tree["logS"][i] - math.log(sigmoid(0.67 * logit(qT) - 0.46))) > 1e-3
 
 
+def test_ablation_switch_feeds_the_tempered_conditional_and_grows_larger_trees():
+    # Section 5.5: with q_T in place of q0 the survival of every node is the product of the estimates at
+    # q_T along its path (recomputed here with numpy), sharper proposals (T < 1) price edges higher and the
+    # same theta admits more nodes; at T = 0 the switch changes nothing
+    V, D, r, K, N = 30, 3, 4, 3, 20
+    sizes = [0, 0]
+    for seed in range(6):
+        U, A, W = tiny_problem(140 + seed, V, D, r, u_std=2.0)
+        trees = []
+        for inp in (0, 1):
+            o = oracle.Oracle(V, D, r, K, N, calib_input=inp)
+            t = o.expand_tree(U, A, W, 3, theta=0.08, T=0.5, seed=seed, req=0)
+            trees.append(t)
+            sizes[inp] += t["n"]
+            for i in range(t["n"]):
+                ls, j = 0.0, i
+                while j >= 0:
+                    p = int(t["parent"][j])
+                    ptok = 3 if p < 0 else int(t["tok"][p])
+                    l = np_logits(U[int(t["depth"][j]) - 1], A[ptok], W)
+                    q = np_softmax(l, 0.5 if inp else 1.0)[int(t["tok"][j])]
+                    ls += math.log(sigmoid(0.67 * logit(q) - 0.46))
+                    j = p
+                assert abs(ls - t["logS"][i]) < 1e-9
+        o0, o1 = oracle.Oracle(V, D, r, K, N), oracle.Oracle(V, D, r, K, N, calib_input=1)
+        g0 = o0.expand_tree(U, A, W, 3, theta=0.08, T=0.0, seed=seed, req=0)
+        g1 = o1.expand_tree(U, A, W, 3, theta=0.08, T=0.0, seed=seed, req=0)
+        assert g0["n"] == g1["n"] and np.array_equal(g0["tok"], g1["tok"]) and np.array_equal(g0["logS"], g1["logS"])
+    assert sizes[1] > sizes[0]
+
+
 # ----------------------------------------------------------------------------------------------
 # Verification
 # ----------------------------------------------------------------------------------------------
