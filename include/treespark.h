@@ -73,6 +73,14 @@ typedef struct {
 int32_t ts_create(const ts_config* cfg, ts_ctx** out);
 int32_t ts_destroy(ts_ctx* ctx);
 
+/* Ablation switches for study (Section 5.5); 0, the default, is the method.  Takes effect for calls
+ * issued afterwards.  TS_ABLATE_CALIB_QT: at T > 0 the calibrator of ts_expand_tree is fed the tempered
+ * conditional q_T instead of the untempered q0 (the paper finds that this inflates the trees and loses
+ * the advantage of the price rule).  The marginal-tree ablation needs no switch (pass zero head rows A),
+ * nor does the raw priority (Platt mode with a = 1, b = 0). */
+#define TS_ABLATE_CALIB_QT 1u
+int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags);
+
 /* Bytes of workspace the hot calls need for a batch of `batch` requests (<= max_batch). */
 size_t ts_workspace_bytes(const ts_ctx* ctx, int32_t batch);
 

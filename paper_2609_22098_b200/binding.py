@@ -19,7 +19,9 @@ TS_OK = 0
 DTYPE_F32, DTYPE_BF16 = 0, 1
 KNOTS = 16
 
-EXPORTS = ("ts_create", "ts_destroy", "ts_workspace_bytes", "ts_last_error_string",
+ABLATE_CALIB_QT = 1
+
+EXPORTS = ("ts_create", "ts_destroy", "ts_set_ablation", "ts_workspace_bytes", "ts_last_error_string",
            "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",
            "ts_allocate_budget", "ts_calib_accumulate", "ts_calib_refit", "ts_calib_load_table",
            "ts_emit_attention_inputs", "ts_profile_enable", "ts_profile_read", "ts_kernel_name")
@@ -48,6 +50,8 @@ def load_library() -> C.CDLL:
         L.ts_workspace_bytes.argtypes = [C.c_void_p, C.c_int32]
         L.ts_create.argtypes = [C.POINTER(TsConfig), C.POINTER(C.c_void_p)]
         L.ts_destroy.argtypes = [C.c_void_p]
+        L.ts_set_ablation.argtypes = [C.c_void_p, C.c_uint32]
+        L.ts_set_ablation.restype = C.c_int32
         vp, i32, f32, u64, sz = C.c_void_p, C.c_int32, C.c_float, C.c_uint64, C.c_size_t
         L.ts_score_parents.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, f32, u64] + [vp] * 6 + [vp, sz, vp]
         L.ts_score_parents_static.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, f32, u64] + [vp] * 6 + [vp]
@@ -120,6 +124,9 @@ class TreeSpark:
     def _check(self, code: int):
         if code != TS_OK:
             raise TreeSparkError(f"status {code}: {self.lib.ts_last_error_string().decode()}")
+
+    def set_ablation(self, flags: int):
+        self._check(self.lib.ts_set_ablation(self._ctx, int(flags)))
 
     # -- instrumentation ---------------------------------------------------------------------------
     def profile_enable(self, capacity: int):

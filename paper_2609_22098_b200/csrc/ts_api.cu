@@ -73,6 +73,7 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
   ctx->cfg.calib_table = nullptr;
   ctx->d_table = nullptr;
   ctx->prof = new Prof();
+  ctx->ablation = 0;
   cudaError_t e = cudaGetDevice(&ctx->device);
   cudaDeviceProp prop;
   if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, ctx->device);
@@ -122,6 +123,13 @@ extern "C" int32_t ts_destroy(ts_ctx* ctx) {
   Prof* p = (Prof*)ctx->prof;
   if (p) { for (cudaEvent_t e : p->ev) cudaEventDestroy(e); delete p; }
   delete ctx;
+  return TS_OK;
+}
+
+extern "C" int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags) {
+  if (!ctx) return set_error(TS_ERR_INVALID, "ts_set_ablation: null context");
+  if (flags & ~(uint32_t)TS_ABLATE_CALIB_QT) return set_error(TS_ERR_INVALID, "ts_set_ablation: unknown switch");
+  ctx->ablation = flags;
   return TS_OK;
 }
 

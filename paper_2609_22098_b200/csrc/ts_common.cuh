@@ -68,6 +68,7 @@ struct ts_ctx {
   const void* tmapW_ptr;
   int tma_state;   // 0 not tried yet, 1 encoder found, -1 unavailable
   int walk_pdl;    // -1: the driver refused a cooperative launch with programmatic serialization
+  unsigned ablation;   // TS_ABLATE_* switches (0 = the method)
 };
 
 namespace ts {

@@ -32,6 +32,7 @@ struct ExpandArgs {
   // candidates
   int *cd_valid, *cd_parent, *cd_sib, *cd_tok; double *cd_logkey, *cd_logS; float *cd_q0, *cd_logqT; int* cd_rank;
   int* status; int* err; unsigned* thr; int thr_head, thr_words;
+  int calib_qT;   // ablation: the calibrator is fed the tempered conditional when T > 0
 };
 
 __device__ __forceinline__ void request_caps(const ExpandArgs& a, int b, int& K_eff, int& N_eff, double& log_theta) {
@@ -129,13 +130,16 @@ __global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d) 
       }
       const int x = draw_tok[j];
       if (bi >= 0 && top_tok[bi] >= 0 && x >= 0) {
-        const double key = logS_v + log_phat(a.calib, d, (double)top_logit[bi], lse0);
+        // the calibrator's input: the untempered conditional, or (ablation) the tempered one
+        const bool tempered = a.calib_qT && a.T > 0.f;
+        const double lsc = tempered ? 1.0 / (double)a.T : 1.0, lsn = tempered ? lseT : lse0;
+        const double key = logS_v + log_phat(a.calib, d, (double)top_logit[bi] * lsc, lsn);
         if (!(key < log_theta)) {
           const double lx = draw_logit[j];
           valid = 1;
           a.cd_parent[ci] = slot; a.cd_sib[ci] = j; a.cd_tok[ci] = x;
           a.cd_logkey[ci] = key;
-          a.cd_logS[ci] = logS_v + log_phat(a.calib, d, lx, lse0);
+          a.cd_logS[ci] = logS_v + log_phat(a.calib, d, lx * lsc, lsn);
           a.cd_q0[ci] = (float)exp(lx - lse0);
           a.cd_logqT[ci] = a.T > 0.f ? (float)(lx / (double)a.T - lseT) : (float)(lx - lse0);
         }
@@ -383,6 +387,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   ExpandArgs a{};
   a.B = B; a.D = c.D; a.K = c.K; a.N = c.Nmax; a.V = c.V; a.T = T; a.anchor = anchor_tok; a.theta = theta;
   a.calib = ctx->calib;
+  a.calib_qT = (ctx->ablation & TS_ABLATE_CALIB_QT) ? 1 : 0;
   for (int i = 0; i < 2; ++i) {
     a.lst_req[i] = (int*)(ws + L.lst_req[i]); a.lst_depth[i] = (int*)(ws + L.lst_depth[i]);
     a.lst_token[i] = (int*)(ws + L.lst_token[i]); a.lst_hash[i] = (uint64_t*)(ws + L.lst_hash[i]);

@@ -213,6 +213,31 @@ def test_ablation_settings_match_oracle(which):
         assert st["trees"] == rnd.B
 
 
+@pytest.mark.parametrize("calib_mode", [0, 1])
+def test_tempered_calibrator_switch_matches_oracle(calib_mode):
+    """The ablation that feeds the calibrator q_T instead of q0 (Section 5.5), against the oracle's switch;
+    the trees must also differ from the method's at T != 1 (the switch does something) and not at T = 0."""
+    wl = small("serve32", V=12000 + 8, B=6, calib_mode=calib_mode)
+    rnd = Round(wl, seed=920)
+    table = rnd.table if calib_mode == 1 else None
+    ts = make_gpu(wl, table, max_batch=rnd.B)
+    plain = {T: to_cpu(ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, 37)) for T in (0.0, 0.6)}
+    ts.set_ablation(1)
+    orc = oracle.Oracle(wl.V, wl.D, wl.r, wl.K, wl.Nmax, calib_mode=calib_mode, calib_input=1,
+                        calib_table=None if table is None else table.numpy().astype(np.float64))
+    for T in (0.0, 0.6, 1.0):
+        st = check_round(ts, orc, rnd, T, round_seed=37)
+        assert st["trees"] == rnd.B
+    fed = {T: to_cpu(ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, 37)) for T in (0.0, 0.6)}
+    assert torch.equal(fed[0.0]["logS"], plain[0.0]["logS"]) and torch.equal(fed[0.0]["n_nodes"], plain[0.0]["n_nodes"])
+    assert int(fed[0.6]["n_nodes"].sum()) > int(plain[0.6]["n_nodes"].sum())   # sharper proposal, larger trees
+    ts.set_ablation(0)
+    back = to_cpu(ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, 0.6, 37))
+    assert torch.equal(back["n_nodes"], plain[0.6]["n_nodes"])
+    with pytest.raises(Exception):
+        ts.set_ablation(2)
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_round_at_the_papers_own_shape_matches_oracle(dtype):
     # rank 256, block of 7, 56 nodes, 8 siblings (Section 5.1), on a vocabulary the oracle finishes quickly
