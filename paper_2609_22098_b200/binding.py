@@ -288,7 +288,7 @@ class HostRound:
     the step before."""
 
     TREE_OUT = ("n_nodes", "tok", "parent", "depth", "mask")
-    VERDICT_OUT = ("acc_len", "acc_tok", "bonus_tok")
+    RESULT_KEYS = ("acc_len", "acc_tok", "bonus_tok")
 
     @staticmethod
     def pin_inputs(U, anchor, theta, Z, zoff):
@@ -306,7 +306,7 @@ class HostRound:
         self.tree = ts.alloc_tree(B)
         self.verdict = ts.alloc_verdict(B)
         self.host_out = {k: torch.empty_like(self.tree[k], device="cpu").pin_memory() for k in self.TREE_OUT}
-        self.host_out.update({k: torch.empty_like(self.verdict[k], device="cpu").pin_memory() for k in self.VERDICT_OUT})
+        self.host_out.update({k: torch.empty_like(self.verdict[k], device="cpu").pin_memory() for k in self.RESULT_KEYS})
         self.h2d_bytes = 0
         self.d2h_bytes = sum(t.numel() * t.element_size() for t in self.host_out.values())
         self._max_rows = max_rows
@@ -354,7 +354,7 @@ class HostRound:
                        edge_stat=edge_stat)
         for k in self.TREE_OUT:
             sl["out"][k].copy_(sl["tree"][k], non_blocking=True)
-        for k in self.VERDICT_OUT:
+        for k in self.RESULT_KEYS:
             sl["out"][k].copy_(sl["verdict"][k], non_blocking=True)
         sl["done"].record()
         sl["free"].record()
@@ -380,7 +380,7 @@ class HostRound:
                        edge_stat=edge_stat)
         for k in self.TREE_OUT:
             self.host_out[k].copy_(self.tree[k], non_blocking=True)
-        for k in self.VERDICT_OUT:
+        for k in self.RESULT_KEYS:
             self.host_out[k].copy_(self.verdict[k], non_blocking=True)
         torch.cuda.current_stream().synchronize()
         self.h2d_bytes = sum(host[k].numel() * host[k].element_size() for k in ("U", "anchor", "theta", "Z", "zoff"))
