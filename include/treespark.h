@@ -18,8 +18,9 @@
  *   - Indices: draft depth d of a PARENT is 0-based (the root has depth 0); its children live at
  *     depth d+1 in 1..D and are scored with base-logit row U[request][d].
  *   - Random numbers: Philox4x32-10, key = seed, counter = (index, path hash of the node (64 bit),
- *     request | stream << 24).  Stream 1/2 give the top byte / low 24 bits of the sampling uniform
- *     of token v (sixteen resp. four tokens per call), stream 3 the accept uniform of sibling j,
+ *     request | stream << 24).  Stream 1/2 give the high / low 16 bits of the sampling uniform of
+ *     token v (index = v / 8: one call serves eight consecutive tokens, one half-word each),
+ *     stream 3 the accept uniform of sibling j,
  *     stream 4 the bonus uniform.  hash(root) = 0, hash(child) = splitmix64(hash(parent) XOR
  *     (token+1) * 0x9E3779B97F4A7C15).  A draw therefore depends on the node's token path only,
  *     never on the order in which nodes were materialised.
