@@ -299,6 +299,9 @@ __device__ __forceinline__ double log_phat(const DevCalib& c, int d, double lx, 
   double q = exp(lq);
   if (q > 1.0 - 1e-12) q = 1.0 - 1e-12;
   double t = lq - log1p(-q);
+  // non-finite logits (reported per request as TS_ERR_NUMERIC) must not reach the table lookup below: a NaN
+  // position passes both range tests and its integer part is not a usable index
+  if (!(t == t)) return t;
   t = t > 30.0 ? 30.0 : (t < -30.0 ? -30.0 : t);
   if (c.mode == 0) {
     const double x = c.a * t + c.b;
@@ -310,7 +313,8 @@ __device__ __forceinline__ double log_phat(const DevCalib& c, int d, double lx, 
   if (pos <= 0.0) v = y[0];
   else if (pos >= KNOTS - 1) v = y[KNOTS - 1];
   else {
-    const int i = (int)floor(pos);
+    int i = (int)floor(pos);
+    i = i < 0 ? 0 : (i > KNOTS - 2 ? KNOTS - 2 : i);
     const double f = pos - i;
     v = (double)y[i] + f * ((double)y[i + 1] - (double)y[i]);
   }

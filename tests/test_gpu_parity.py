@@ -287,6 +287,30 @@ def test_argument_validation_returns_errors_without_launching():
     assert int(tree["status"][0]) == -1 and int(tree["n_nodes"][0]) == 0
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_non_finite_base_logits_are_reported_for_their_request_only(dtype):
+    """A NaN row or an infinite logit cannot be scored: the request's status says so, the call returns, and
+    the other requests of the batch get exactly the trees they get without the bad neighbour."""
+    wl = small("serve32", V=12000 + 8, B=5, dtype=dtype)
+    rnd = Round(wl, seed=930)
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
+    clean = to_cpu(ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, 1.0, 5))
+    U = rnd.U.clone()
+    U[1, 0, :] = float("nan")                                 # a whole row
+    U[3, 0, 777] = float("inf")                               # one token
+    bad = to_cpu(ts.expand_tree(U, rnd.A, rnd.W, rnd.anchor, rnd.theta, 1.0, 5))
+    torch.cuda.synchronize()
+    assert bad["status"].tolist() == [0, -7, 0, -7, 0]
+    for b in (0, 2, 4):
+        n = int(clean["n_nodes"][b])
+        assert int(bad["n_nodes"][b]) == n
+        for name in ("tok", "parent", "depth", "sib_rank", "logS", "pop_rank"):
+            assert torch.equal(bad[name][b, :n], clean[name][b, :n]), (b, name)
+    again = to_cpu(ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, 1.0, 5))   # the context is unharmed
+    assert torch.equal(again["n_nodes"], clean["n_nodes"]) and torch.equal(again["tok"], clean["tok"])
+    assert (again["status"] == 0).all()
+
+
 # ---------------------------------------------------------------------------------------------
 # losslessness on the GPU path itself (Proposition 1), tiny vocabulary, many requests per call
 # ---------------------------------------------------------------------------------------------
