@@ -195,6 +195,9 @@ int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, const void* W,
  * Outputs DEVICE: acc_len [B] in [0,D]; acc_node, acc_tok [B][D]; bonus_tok [B];
  *   edge_stat [B][Nmax] or NULL: T == 0 -> 1/0 "token equals the parent's target argmax" for every
  *   edge, T > 0 -> min(1, p(x)/q_T(x)) for every edge; flags [B]; status [B].
+ * A request one of whose target rows holds a NaN or no finite mass (T > 0: also an infinite logit), or
+ * whose tree carries a NaN proposal probability, is not walked: status TS_ERR_NUMERIC, acc_len 0,
+ * bonus_tok -1, edge_stat 0; the other requests of the call are unaffected.
  */
 int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, const void* W,
                        const void* Z, const int64_t* z_row_off, int32_t B,

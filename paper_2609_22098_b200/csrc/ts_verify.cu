@@ -40,6 +40,9 @@ extern "C" int ts_debug_timing_pass(unsigned long long* out) { return (int)cudaM
 // 2^x by the hardware approximation (the library exp2f costs several times more in the hot loops here)
 __device__ __forceinline__ float fast_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 
+// maximum that returns NaN when either operand is NaN (fmaxf drops NaNs)
+__device__ __forceinline__ float max_nan(float a, float b) { float y; asm("max.NaN.f32 %0, %1, %2;" : "=f"(y) : "f"(a), "f"(b)); return y; }
+
 constexpr int ZT = 512;  // threads per target row in the row-statistics kernel
 
 // ------------------------------------------------------------------------------------------------
@@ -69,10 +72,12 @@ __global__ void __launch_bounds__(ZT) zrow_stats_kernel(const TIn* Z, const int6
     // maximum, which is rare), then one fused multiply-add and one ex2 per element
     const float sc = invT * 1.4426950408889634f;
     float boff = 0.f;   // -bv * sc while bv is finite
+    bool has_nan = false;
     auto take = [&](const float* x, int c, int n) {
       float vm = x[0];
 #pragma unroll
-      for (int i = 1; i < VEC; ++i) if (i < n) vm = fmaxf(vm, x[i]);
+      for (int i = 1; i < VEC; ++i) if (i < n) vm = max_nan(vm, x[i]);
+      has_nan |= vm != vm;   // one test per vector: a NaN anywhere in it survives the maximum
       if (vm > bv) {   // first maximum wins: indices increase
         int vi = 0;
 #pragma unroll
@@ -117,13 +122,13 @@ __global__ void __launch_bounds__(ZT) zrow_stats_kernel(const TIn* Z, const int6
       bv = nm; sum = ns;
     }
     if (lane == 0) { s_v[warp] = bv; s_i[warp] = bi; s_s[warp] = sum; }
-    __syncthreads();
+    const int row_nan = __syncthreads_or(has_nan ? 1 : 0);
     if (tid == 0) {
       float gv = s_v[0]; int gi = s_i[0];
       for (int w = 1; w < ZT / 32; ++w) if (s_v[w] > gv || (s_v[w] == gv && s_i[w] < gi)) { gv = s_v[w]; gi = s_i[w]; }
       float gs = 0.f;
       for (int w = 0; w < ZT / 32; ++w) if (s_v[w] > -INFINITY) gs += s_s[w] * __expf((s_v[w] - gv) * invT);
-      z_max[row] = gv; z_arg[row] = gi;
+      z_max[row] = row_nan ? nanf("") : gv; z_arg[row] = gi;   // a NaN maximum marks a row that holds a NaN
       if (T > 0.f) z_logs[row] = logf(gs);
     }
     __syncthreads();
@@ -151,24 +156,35 @@ struct VerifyArgs {
 // ------------------------------------------------------------------------------------------------
 __global__ void verify_greedy_kernel(VerifyArgs a) {
   const int b = blockIdx.x, N = a.N;
-  const int n = a.n_nodes[b];
+  const int n_in = a.n_nodes[b];
+  const bool okn = n_in >= 0 && n_in <= N;
+  const int n = okn ? n_in : 0;
   const int64_t row0 = a.z_row_off[b];
   const size_t nb = (size_t)b * N;
+  // a target row that holds a NaN (its maximum is NaN) or nothing finite has no arg-max
+  int bad = 0;
+  for (int i = threadIdx.x; i <= n; i += blockDim.x) {
+    const float zm = a.z_max[row0 + i];
+    bad |= (zm != zm || zm == -INFINITY) ? 1 : 0;
+  }
+  bad = __syncthreads_or(okn ? bad : 0);
   if (a.edge_stat)
     for (int i = threadIdx.x; i < n; i += blockDim.x)
-      a.edge_stat[nb + i] = (a.tok[nb + i] == a.z_arg[row0 + a.parent[nb + i] + 1]) ? 1.f : 0.f;
+      a.edge_stat[nb + i] = (!bad && a.tok[nb + i] == a.z_arg[row0 + a.parent[nb + i] + 1]) ? 1.f : 0.f;
   if (threadIdx.x == 0) {
     int cur = -1, acc = 0;
-    for (;;) {
-      const int g = a.z_arg[row0 + cur + 1];
-      int hit = -1;
-      for (int i = cur + 1; i < n; ++i)  // children come after their parent in canonical order
-        if (a.parent[nb + i] == cur && a.tok[nb + i] == g) { hit = i; break; }
-      if (hit < 0 || acc >= a.D) { a.bonus[b] = g; break; }
-      a.acc_node[(size_t)b * a.D + acc] = hit; a.acc_tok[(size_t)b * a.D + acc] = g; ++acc; cur = hit;
-    }
+    if (!okn || bad) a.bonus[b] = -1;
+    else
+      for (;;) {
+        const int g = a.z_arg[row0 + cur + 1];
+        int hit = -1;
+        for (int i = cur + 1; i < n; ++i)  // children come after their parent in canonical order
+          if (a.parent[nb + i] == cur && a.tok[nb + i] == g) { hit = i; break; }
+        if (hit < 0 || acc >= a.D) { a.bonus[b] = g; break; }
+        a.acc_node[(size_t)b * a.D + acc] = hit; a.acc_tok[(size_t)b * a.D + acc] = g; ++acc; cur = hit;
+      }
     for (int i = acc; i < a.D; ++i) { a.acc_node[(size_t)b * a.D + i] = -1; a.acc_tok[(size_t)b * a.D + i] = -1; }
-    a.acc_len[b] = acc; a.flags[b] = 0u; a.status[b] = (n >= 0 && n <= N) ? TS_OK : TS_ERR_INVALID;
+    a.acc_len[b] = acc; a.flags[b] = 0u; a.status[b] = !okn ? TS_ERR_INVALID : (bad ? TS_ERR_NUMERIC : TS_OK);
   }
 }
 
@@ -693,8 +709,20 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
     const size_t nb = (size_t)b * N, cbase = (size_t)b * (N + 1);
     const int64_t row0 = a.z_row_off[b];
     for (int i = tid; i <= N; i += WT) { a.child_first[cbase + i] = -1; a.child_cnt[cbase + i] = 0; }
-    __syncthreads();
-    if (okn)
+    // non-finite inputs: a target row with a NaN (its maximum is NaN), without finite mass, or a node whose
+    // proposal log-probability is NaN (its expansion was reported TS_ERR_NUMERIC) -- the request is not walked
+    int bad = 0;
+    if (okn) {
+      for (int i = tid; i <= n; i += WT) {
+        const float zm = a.z_max[row0 + i], zl = a.z_logs[row0 + i];
+        bad |= (zm != zm || isinf(zm) || zl != zl || isinf(zl)) ? 1 : 0;
+      }
+      for (int i = tid; i < n; i += WT) { const float lq = a.logqT[nb + i]; bad |= (lq != lq) ? 1 : 0; }
+    }
+    bad = __syncthreads_or(bad);
+    if (bad && a.edge_stat)
+      for (int i = tid; i < n; i += WT) a.edge_stat[nb + i] = 0.f;
+    if (okn && !bad)
       for (int i = tid; i < n; i += WT) {
         const int par = a.parent[nb + i];
         if (i == 0 || a.parent[nb + i - 1] != par) a.child_first[cbase + par + 1] = i;   // siblings are contiguous
@@ -724,8 +752,8 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
       st.npass = 0; st.pad_ = 0;
       st.cfirst = a.child_first[cbase]; st.ccnt = a.child_cnt[cbase];   // children of the root
       a.flags[b] = 0u;
-      a.status[b] = okn ? TS_OK : TS_ERR_INVALID;
-      if (!okn) { st.need = 3; a.acc_len[b] = 0; a.bonus[b] = -1; }
+      a.status[b] = !okn ? TS_ERR_INVALID : (bad ? TS_ERR_NUMERIC : TS_OK);
+      if (!okn || bad) { st.need = 3; a.acc_len[b] = 0; a.bonus[b] = -1; }
       for (int i = 0; i < a.D; ++i) { a.acc_node[(size_t)b * a.D + i] = -1; a.acc_tok[(size_t)b * a.D + i] = -1; }
     }
     __syncthreads();

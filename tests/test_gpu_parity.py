@@ -311,6 +311,38 @@ def test_non_finite_base_logits_are_reported_for_their_request_only(dtype):
     assert (again["status"] == 0).all()
 
 
+@pytest.mark.parametrize("T", [0.0, 1.0])
+def test_non_finite_target_logits_are_reported_for_their_request_only(T):
+    """A NaN anywhere in a target row of a request: that request is not walked (status, no accepted
+    tokens, no bonus token), the others get exactly the verdict they get without it."""
+    wl = small("serve32", V=12000 + 8, B=5)
+    rnd = Round(wl, seed=940)
+    rnd.theta.fill_(0.03)
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
+    tree = ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, 6)
+    Z, off = rnd.target_logits(tree)
+    clean = to_cpu(ts.verify_tree(rnd.U, rnd.A, rnd.W, Z, off, rnd.anchor, tree, T, 6))
+    assert (clean["status"] == 0).all()
+    offc = off.cpu()
+    Zb = Z.clone()
+    Zb[int(offc[1]), 4321] = float("nan")                     # the root row of request 1
+    Zb[int(offc[4]) - 1, 17] = float("nan")                   # the last row of request 3
+    bad = to_cpu(ts.verify_tree(rnd.U, rnd.A, rnd.W, Zb, off, rnd.anchor, tree, T, 6))
+    torch.cuda.synchronize()
+    assert bad["status"].tolist() == [0, -7, 0, -7, 0]
+    for b in (1, 3):
+        assert int(bad["acc_len"][b]) == 0 and int(bad["bonus_tok"][b]) == -1
+        assert (bad["edge_stat"][b, :int(tree["n_nodes"][b])] == 0).all()
+    for b in (0, 2, 4):
+        for name in ("acc_len", "acc_node", "acc_tok", "bonus_tok", "flags"):
+            assert torch.equal(bad[name][b], clean[name][b]), (b, name)
+        n = int(tree["n_nodes"][b])
+        assert torch.equal(bad["edge_stat"][b, :n], clean["edge_stat"][b, :n])
+    again = to_cpu(ts.verify_tree(rnd.U, rnd.A, rnd.W, Z, off, rnd.anchor, tree, T, 6))   # the context is unharmed
+    for name in ("status", "acc_len", "acc_tok", "bonus_tok"):
+        assert torch.equal(again[name], clean[name]), name
+
+
 # ---------------------------------------------------------------------------------------------
 # losslessness on the GPU path itself (Proposition 1), tiny vocabulary, many requests per call
 # ---------------------------------------------------------------------------------------------
