@@ -343,6 +343,27 @@ def test_non_finite_target_logits_are_reported_for_their_request_only(T):
         assert torch.equal(again[name], clean[name]), name
 
 
+@pytest.mark.parametrize("T", [0.0, 1.0])
+def test_impossible_node_count_is_refused_for_its_request_only(T):
+    wl = small("serve32", V=12000 + 8, B=4)
+    rnd = Round(wl, seed=950)
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
+    tree = ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, 8)
+    Z, off = rnd.target_logits(tree)
+    clean = to_cpu(ts.verify_tree(rnd.U, rnd.A, rnd.W, Z, off, rnd.anchor, tree, T, 8))
+    broken = dict(tree)
+    broken["n_nodes"] = tree["n_nodes"].clone()
+    broken["n_nodes"][2] = wl.Nmax + 7
+    broken["n_nodes"][0] = -3
+    got = to_cpu(ts.verify_tree(rnd.U, rnd.A, rnd.W, Z, off, rnd.anchor, broken, T, 8))
+    torch.cuda.synchronize()
+    assert got["status"].tolist() == [-1, 0, -1, 0]
+    assert got["acc_len"][[0, 2]].tolist() == [0, 0] and got["bonus_tok"][[0, 2]].tolist() == [-1, -1]
+    for b in (1, 3):
+        for name in ("acc_len", "acc_tok", "bonus_tok"):
+            assert torch.equal(got[name][b], clean[name][b]), (b, name)
+
+
 # ---------------------------------------------------------------------------------------------
 # losslessness on the GPU path itself (Proposition 1), tiny vocabulary, many requests per call
 # ---------------------------------------------------------------------------------------------
