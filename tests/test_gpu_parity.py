@@ -92,6 +92,20 @@ def test_round_matches_oracle(name, over, temps, thetas):
     assert tot["nodes"] > 0
 
 
+@pytest.mark.parametrize("T", [0.0, 1.0])
+def test_empty_trees_only_draw_the_bonus_token(T):
+    """A price no edge can meet (but below the chain sentinel): every tree is empty, verification commits
+    nothing and emits the bonus token from the root row alone."""
+    wl = small("serve32", V=9000 + 8, B=7)
+    rnd = Round(wl, seed=77)
+    rnd.theta.fill_(0.99999)
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
+    orc = make_oracle(wl, rnd.table)
+    for rs in range(3):
+        st = check_round(ts, orc, rnd, T, round_seed=300 + rs)
+        assert st["trees"] == rnd.B and st["nodes"] == 0 and st["acc"] == 0
+
+
 def test_tiny_reference_config_100_rounds():
     """The tiny all-fp32 reference configuration at full size: 100 rounds at T = 0 and T = 1."""
     wl = synth.WORKLOADS["tiny"]
