@@ -175,6 +175,55 @@ def test_alternative_kernel_paths_match_oracle(env, monkeypatch):
         assert st["nodes"] > 0
 
 
+@pytest.mark.parametrize("T", [0.0, 1.0])
+def test_round_replayed_from_a_cuda_graph_equals_direct_calls(T):
+    """The hot calls allocate nothing and never synchronise: a whole round (every launch of expand and
+    verify, cooperative walk included) is captured in a CUDA graph and its replays give the direct results,
+    also after the inputs behind the captured pointers have changed."""
+    wl = small("serve32", V=20000, B=6)
+    rnd = Round(wl, seed=66)
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
+    tree, verdict = ts.alloc_tree(rnd.B), ts.alloc_verdict(rnd.B)
+    U = rnd.U.clone()
+    ts.expand_tree(U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, 21, out=tree)   # also encodes the tensor map before capture
+    Z, off = rnd.target_logits(tree)
+    ts.verify_tree(U, rnd.A, rnd.W, Z, off, rnd.anchor, tree, T, 21, out=verdict)
+    torch.cuda.synchronize()
+    want = (to_cpu(tree), to_cpu(verdict))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        ts.expand_tree(U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, 21, out=tree)
+        ts.verify_tree(U, rnd.A, rnd.W, Z, off, rnd.anchor, tree, T, 21, out=verdict)
+    torch.cuda.current_stream().wait_stream(side)
+
+    def same(a, b):
+        n = a["n_nodes"]
+        ok = torch.equal(a["n_nodes"], b["n_nodes"])
+        for bb in range(rnd.B):
+            for k in ("tok", "parent", "depth", "logS", "pop_rank"):
+                ok = ok and torch.equal(a[k][bb, :int(n[bb])], b[k][bb, :int(n[bb])])
+        return ok
+
+    for _ in range(3):
+        for t in list(tree.values()) + list(verdict.values()):
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        got = (to_cpu(tree), to_cpu(verdict))
+        assert same(want[0], got[0])
+        for k in ("acc_len", "acc_tok", "bonus_tok", "status"):
+            assert torch.equal(want[1][k], got[1][k]), k
+    # other base logits behind the same pointer: the replay follows them (trees change), as a direct call does
+    U.copy_(Round(wl, seed=67).U)
+    g.replay()
+    torch.cuda.synchronize()
+    replayed = to_cpu(tree)
+    direct = to_cpu(ts.expand_tree(U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, 21))
+    assert same(direct, replayed) and not torch.equal(replayed["tok"], want[0]["tok"])
+
+
 def test_host_round_two_in_flight_equals_one_at_a_time():
     """The host-buffer round: submit / collect with two rounds in flight returns what run() returns."""
     from paper_2609_22098_b200.binding import HostRound
