@@ -190,11 +190,19 @@ __device__ __forceinline__ uint32_t pick8(const uint4& a, const uint4& b, int i)
   return r;
 }
 
+// 2^x by the hardware approximation
+__device__ __forceinline__ float ex2_approx(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+// index into the two noise-bound tables for the leading 16 bits of a uniform: by top byte, or, inside the top
+// bucket, by the second byte
+__device__ __forceinline__ uint32_t noise_bound_index(uint32_t c16) { return (c16 >> 8) != 255u ? (c16 >> 8) : 256u + (c16 & 255u); }
+
 // One 16-token chunk of one parent: logits l[0..16) for tokens v0.., `valid` of them inside V.
 // gL / gK: launch-wide lower bounds of the parent's K-th best logit / key as the caller last read them.
 // The common case is branch-free: sums, then one bit per token saying whether it can still be a
 // candidate; the few tokens whose bit is set are handled one at a time by a single copy of the code.
-template <class Lists>
+// Padded == true: the caller guarantees that l[i] is -infinity for every i >= valid (the tensor-core kernel
+// does); the per-token range tests then fall away: -infinity loses every comparison and adds exp(-inf) = 0.
+template <class Lists, bool Padded = false>
 __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, int v0, int valid, float T, float invT,
                                            uint64_t seed, int req, uint64_t hash, const float* ghi,
                                            float gL, float gK, const SharedThr& gl, const SharedThr& gk,
@@ -209,8 +217,17 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
     cw1 = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, ((uint32_t)v0 >> 3) + 1u);
   }
   float cm = -INFINITY;
+  float gmax[4];   // best logit of each group of four tokens (the key gate below uses them again)
+  if constexpr (Padded) {
 #pragma unroll
-  for (int i = 0; i < CHUNK; ++i) if (i < valid) cm = fmaxf(cm, l[i]);
+    for (int sg = 0; sg < 4; ++sg) {
+      gmax[sg] = fmaxf(fmaxf(l[4 * sg], l[4 * sg + 1]), fmaxf(l[4 * sg + 2], l[4 * sg + 3]));
+      cm = fmaxf(cm, gmax[sg]);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < CHUNK; ++i) if (i < valid) cm = fmaxf(cm, l[i]);
+  }
   {
     // rescale to the new running maximum without a branch (no change: factor 1; first chunk: factor 0)
     const float nm = fmaxf(st.m, cm);
@@ -221,12 +238,25 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
   }
   float a0 = 0.f, aT = 0.f;
   const bool two = (T > 0.f) && (T != 1.f);
+  if constexpr (Padded) {
+    // exp(l - m) as ex2(l * log2(e) - m * log2(e)): one fused multiply-add and one ex2 per token.  While
+    // nothing finite has been seen (m = -inf) the offset is 0: every l is -inf then and contributes 0.
+    constexpr float LOG2E = 1.4426950408889634f;
+    const float mref = st.m == -INFINITY ? 0.f : st.m;
+    const float off0 = -mref * LOG2E, scT = LOG2E * invT, offT = off0 * invT;
 #pragma unroll
-  for (int i = 0; i < CHUNK; ++i) {
-    if (i < valid) {
-      const float d = l[i] - st.m;
-      a0 += __expf(d);
-      if (two) aT += __expf(d * invT);
+    for (int i = 0; i < CHUNK; ++i) {
+      a0 += ex2_approx(fmaf(l[i], LOG2E, off0));
+      if (two) aT += ex2_approx(fmaf(l[i], scT, offT));
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < CHUNK; ++i) {
+      if (i < valid) {
+        const float d = l[i] - st.m;
+        a0 += __expf(d);
+        if (two) aT += __expf(d * invT);
+      }
     }
   }
   st.s0 += a0;
@@ -247,15 +277,28 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
       const uint32_t wa = (sg & 1) ? cw.z : cw.x, wb = (sg & 1) ? cw.w : cw.y;
       const uint32_t m2 = __vmaxu2(wa, wb);
       const uint32_t c16m = max(m2 & 0xFFFFu, m2 >> 16);
-      const float lm = fmaxf(fmaxf(l[4 * sg], l[4 * sg + 1]), fmaxf(l[4 * sg + 2], l[4 * sg + 3]));
-      const float gb = lm * invT + ((c16m >> 8) != 255u ? ghi[c16m >> 8] : ghi[256 + (c16m & 255u)]);
-      if (4 * sg < valid && gb >= thr) {
+      if constexpr (Padded) {
+        const float gb = gmax[sg] * invT + ghi[noise_bound_index(c16m)];
+        if (gb >= thr && gmax[sg] > -INFINITY) {   // (while no bound exists thr is -inf, and so is a padded group's gb)
 #pragma unroll
-        for (int i = 4 * sg; i < 4 * sg + 4; ++i) {
-          const uint32_t word = word_of(i < 8 ? cw0 : cw1, (i & 7) >> 1);
-          const uint32_t c16 = (word >> (16 * (i & 1))) & 0xFFFFu;
-          const float bnd = l[i] * invT + ((c16 >> 8) != 255u ? ghi[c16 >> 8] : ghi[256 + (c16 & 255u)]);
-          mk |= (uint32_t)(i < valid && bnd >= thr) << i;
+          for (int i = 4 * sg; i < 4 * sg + 4; ++i) {
+            const uint32_t word = word_of(i < 8 ? cw0 : cw1, (i & 7) >> 1);
+            const uint32_t c16 = (word >> (16 * (i & 1))) & 0xFFFFu;
+            const float bnd = l[i] * invT + ghi[noise_bound_index(c16)];
+            mk |= (uint32_t)(bnd >= thr && l[i] > -INFINITY) << i;
+          }
+        }
+      } else {
+        const float lm = fmaxf(fmaxf(l[4 * sg], l[4 * sg + 1]), fmaxf(l[4 * sg + 2], l[4 * sg + 3]));
+        const float gb = lm * invT + ((c16m >> 8) != 255u ? ghi[c16m >> 8] : ghi[256 + (c16m & 255u)]);
+        if (4 * sg < valid && gb >= thr) {
+#pragma unroll
+          for (int i = 4 * sg; i < 4 * sg + 4; ++i) {
+            const uint32_t word = word_of(i < 8 ? cw0 : cw1, (i & 7) >> 1);
+            const uint32_t c16 = (word >> (16 * (i & 1))) & 0xFFFFu;
+            const float bnd = l[i] * invT + ((c16 >> 8) != 255u ? ghi[c16 >> 8] : ghi[256 + (c16 & 255u)]);
+            mk |= (uint32_t)(i < valid && bnd >= thr) << i;
+          }
         }
       }
     }
@@ -290,7 +333,7 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
   if (cm > st.thrL && cm >= gL) {
     uint32_t mk = 0;
 #pragma unroll
-    for (int i = 0; i < CHUNK; ++i) mk |= (uint32_t)(i < valid && l[i] > st.thrL && l[i] >= gL) << i;
+    for (int i = 0; i < CHUNK; ++i) mk |= (uint32_t)((Padded || i < valid) && l[i] > st.thrL && l[i] >= gL) << i;
 #pragma unroll 1
     while (mk) {
       const int i = __ffs(mk) - 1;

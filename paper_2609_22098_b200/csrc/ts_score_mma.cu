@@ -223,9 +223,9 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
             unpack_bf16x8(u0, ub);
             unpack_bf16x8(u1, ub + 8);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] + ub[i] : 0.f;
+            for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] + ub[i] : -INFINITY;   // the scan's padding value
             const float gLc = dec_f(s_thr[prow]), gKc = dec_f(s_thr[128 + prow]);   // kept fresh by the refresh warp
-            scan_chunk(st, acc, v0, valid, T, invT, a.seed, req, hash, ghi, gLc, gKc, gl, gk, s_thr + prow, s_thr + 128 + prow);
+            scan_chunk<Lists, true>(st, acc, v0, valid, T, invT, a.seed, req, hash, ghi, gLc, gKc, gl, gk, s_thr + prow, s_thr + 128 + prow);
           }
         }
         if (dry) continue;
