@@ -269,8 +269,18 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
   if (T > 0.f) {
     const float thr = fmaxf(st.thrK, gK);
     uint32_t mk = 0;
+    // The whole chunk first (padded chunks): its best logit plus the noise bound of the largest leading bits
+    // among its sixteen tokens bounds every key in it.
+    bool chunk_may = true;
+    if constexpr (Padded) {
+      const uint32_t m8 = __vmaxu2(__vmaxu2(__vmaxu2(cw0.x, cw0.y), __vmaxu2(cw0.z, cw0.w)),
+                                   __vmaxu2(__vmaxu2(cw1.x, cw1.y), __vmaxu2(cw1.z, cw1.w)));
+      const uint32_t c16all = max(m8 & 0xFFFFu, m8 >> 16);
+      chunk_may = cm * invT + ghi[noise_bound_index(c16all)] >= thr && cm > -INFINITY;
+    }
     // Four tokens at a time: their best logit plus the noise bound of their largest leading bits bounds
     // all four keys.  Only when that passes (a few groups per thousand) are the four looked at singly.
+    if (chunk_may)
 #pragma unroll
     for (int sg = 0; sg < 4; ++sg) {
       const uint4& cw = sg < 2 ? cw0 : cw1;
