@@ -131,10 +131,14 @@ def test_uniform_price_reproduces_the_theta_rule_on_the_gpu(T):
     cut = to_cpu(tree)
     assert float(price_dev[0]) >= math.log(theta) - 1e-6
     assert cut["n_nodes"].tolist() == stopped["n_nodes"].tolist()
+    # the two expansions score different parent sets per launch, so their sums are taken in different orders:
+    # structure is compared exactly, the floating-point fields under the parity tolerance
     for b in range(rnd.B):
         n = int(cut["n_nodes"][b])
-        for name in NODE_FIELDS + ("mask",):
+        for name in ("tok", "parent", "depth", "sib_rank", "pop_rank", "mask"):
             assert torch.equal(cut[name][b, :n], stopped[name][b, :n]), (b, name)
+        for name in ("logS", "q0", "logqT", "logkey"):
+            assert torch.allclose(cut[name][b, :n], stopped[name][b, :n], rtol=1e-5, atol=4e-6), (b, name)
         assert torch.equal(cut["node_hash"][b, :n + 1], stopped["node_hash"][b, :n + 1])
 
 

@@ -367,8 +367,10 @@ def test_non_finite_base_logits_are_reported_for_their_request_only(dtype):
     for b in (0, 2, 4):
         n = int(clean["n_nodes"][b])
         assert int(bad["n_nodes"][b]) == n
-        for name in ("tok", "parent", "depth", "sib_rank", "logS", "pop_rank"):
+        for name in ("tok", "parent", "depth", "sib_rank", "pop_rank"):
             assert torch.equal(bad[name][b, :n], clean[name][b, :n]), (b, name)
+        # (the two calls score different parent sets per launch: sums in another order, last-place differences)
+        assert torch.allclose(bad["logS"][b, :n], clean["logS"][b, :n], rtol=1e-5, atol=4e-6)
     again = to_cpu(ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, 1.0, 5))   # the context is unharmed
     assert torch.equal(again["n_nodes"], clean["n_nodes"]) and torch.equal(again["tok"], clean["tok"])
     assert (again["status"] == 0).all()
