@@ -223,7 +223,11 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
             unpack_bf16x8(u0, ub);
             unpack_bf16x8(u1, ub + 8);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] + ub[i] : -INFINITY;   // the scan's padding value
+            for (int i = 0; i < 16; ++i) acc[i] += ub[i];
+            if (valid < 16) {   // warp-uniform and rare (the vocabulary's last chunk, the dry pass): the scan's padding value
+#pragma unroll
+              for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] : -INFINITY;
+            }
             const float gLc = dec_f(s_thr[prow]), gKc = dec_f(s_thr[128 + prow]);   // kept fresh by the refresh warp
             scan_chunk<Lists, true>(st, acc, v0, valid, T, invT, a.seed, req, hash, ghi, gLc, gKc, gl, gk, s_thr + prow, s_thr + 128 + prow);
           }
