@@ -568,12 +568,14 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
       const int vn = t0 + cg * 16;
       const uint4 zero = make_uint4(0, 0, 0, 0);
       const bool in = active && cg * 16 < tlen;
-      nz[h][0] = in ? __ldg(reinterpret_cast<const uint4*>(Zrow + vn)) : zero;
-      nz[h][1] = (in && V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Zrow + vn + 8)) : zero;
+      // target logits outside the vocabulary are -inf (eight bf16 -inf): p = 0 there and the residual term vanishes
+      const uint4 ninf = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+      nz[h][0] = in ? __ldg(reinterpret_cast<const uint4*>(Zrow + vn)) : ninf;
+      nz[h][1] = (in && V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Zrow + vn + 8)) : ninf;
       nu[h][0] = (in && need_q) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn)) : zero;
       nu[h][1] = (in && need_q && V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8)) : zero;
     };
-    auto residual = [&](const uint32_t* racc, const uint4& z0, const uint4& z1, const uint4& u0, const uint4& u1, int valid, float& acc_sum) {
+    auto residual = [&](const uint32_t* racc, const uint4& z0, const uint4& z1, const uint4& u0, const uint4& u1, float& acc_sum) {
       float zz[16], ub[16];
       unpack_bf16x8(z0, zz); unpack_bf16x8(z1, zz + 8);
       unpack_bf16x8(u0, ub); unpack_bf16x8(u1, ub + 8);
@@ -582,7 +584,7 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
       for (int i = 0; i < 16; ++i) {
         const float p = fast_ex2(fmaf(zz[i], zs, zoff));
         const float qq = fast_ex2(fmaf(__uint_as_float(racc[i]) + ub[i], zs, qoff));
-        if (i < valid) acc_sum += fmaxf(fmaf(-C, qq, p), 0.f);
+        acc_sum += fmaxf(fmaf(-C, qq, p), 0.f);   // tokens past the vocabulary: p = 0, C >= 0, term 0
       }
     };
     request(c0, 0);
@@ -599,7 +601,7 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
       for (int ca = c0; ca < nch; ca += 2 * cstep) {
         const int cb = ca + cstep;
         const bool hb = cb < nch;   // warp-uniform
-        const int cga = nb * (WALK_BLK / 16) + ca, cgb = cga + cstep;
+        const int cga = nb * (WALK_BLK / 16) + ca;
         uint32_t ra[16], rb[16];
         const uint32_t tbase = tc.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * WALK_BLK);
         tmem_ld16_issue(tbase + (uint32_t)(ca * 16), ra);
@@ -615,9 +617,8 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
           request(na + cstep, 1);
         }
         if (active) {
-          const int va = t0 + cga * 16, vb = t0 + cgb * 16;
-          residual(ra, za0, za1, ua0, ua1, min(16, V - va), sum);
-          if (hb) residual(rb, zb0, zb1, ub0, ub1, min(16, V - vb), sum2);
+          residual(ra, za0, za1, ua0, ua1, sum);
+          if (hb) residual(rb, zb0, zb1, ub0, ub1, sum2);
         }
       }
       tc_fence_before();
