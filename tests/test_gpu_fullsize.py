@@ -52,3 +52,11 @@ def test_sweep_mid_batch():
     wl = synth.WORKLOADS["sweep"]
     st = run(wl, 1.0, synth.sweep_theta(16, seed=9), reqs=[1, 9], seed=10, B=16)
     assert st["trees"] == 2
+
+
+@pytest.mark.parametrize("T", [0.0, 1.0])
+def test_paper_shape_full_size_sampled_requests(T):
+    # the paper's own head and tree shape (rank 256, block of 7, 56 nodes) on the full vocabulary and batch
+    wl = synth.WORKLOADS["paper"]
+    st = run(wl, T, wl.theta, reqs=[0, 13, 31], seed=2610)
+    assert st["trees"] == 3 and st["nodes"] > 0
