@@ -82,6 +82,28 @@ int32_t ts_destroy(ts_ctx* ctx);
 #define TS_ABLATE_CALIB_QT 1u
 int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags);
 
+/* Switches for the library's own tests (the paper has no counterpart; 0, the default, is the product).
+ * They select kernel paths that the configuration or the device would otherwise select, and shorten
+ * or break the bounded device-side waits so that their give-up path can be exercised without hanging
+ * anything.  Call it right after ts_create, before ts_workspace_bytes and before any other call on the
+ * context: the workspace size depends on the path.  Errors: TS_ERR_INVALID (unknown switch),
+ * TS_ERR_UNSUPPORTED (the forced path has no tiling for this configuration), TS_ERR_CUDA.
+ *   TS_TEST_FORCE_FMA     bf16 inputs run on the fp32 fused-multiply-add kernels (no tensor cores)
+ *   TS_TEST_NO_TMA        the tensor-core kernels stage W with plain loads (no tensor map)
+ *   TS_TEST_NO_FEW        levels with few parents run on the tile kernel too
+ *   TS_TEST_NO_SEED       the tensor-core scoring kernel starts without seeded pruning bounds
+ *   TS_TEST_SHORT_WAITS   bounded waits give up after 4096 polls instead of 2^22
+ *   TS_TEST_LOST_ARRIVAL  the walk's grid barriers and the scoring kernel's operand barrier expect one
+ *                         arrival more than will come: the waits run out, the kernels return, and the
+ *                         requests are reported with TS_ERR_TIMEOUT in status[] */
+#define TS_TEST_FORCE_FMA 1u
+#define TS_TEST_NO_TMA 2u
+#define TS_TEST_NO_FEW 4u
+#define TS_TEST_NO_SEED 8u
+#define TS_TEST_SHORT_WAITS 16u
+#define TS_TEST_LOST_ARRIVAL 32u
+int32_t ts_set_test_mode(ts_ctx* ctx, uint32_t flags);
+
 /* Bytes of workspace the hot calls need for a batch of `batch` requests (<= max_batch). */
 size_t ts_workspace_bytes(const ts_ctx* ctx, int32_t batch);
 

@@ -20,8 +20,9 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 KNOTS = 16
 
 ABLATE_CALIB_QT = 1
+TEST_FORCE_FMA, TEST_NO_TMA, TEST_NO_FEW, TEST_NO_SEED, TEST_SHORT_WAITS, TEST_LOST_ARRIVAL = 1, 2, 4, 8, 16, 32
 
-EXPORTS = ("ts_create", "ts_destroy", "ts_set_ablation", "ts_workspace_bytes", "ts_last_error_string",
+EXPORTS = ("ts_create", "ts_destroy", "ts_set_ablation", "ts_set_test_mode", "ts_workspace_bytes", "ts_last_error_string",
            "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",
            "ts_allocate_budget", "ts_calib_accumulate", "ts_calib_refit", "ts_calib_load_table",
            "ts_emit_attention_inputs", "ts_profile_enable", "ts_profile_read", "ts_kernel_name")
@@ -52,6 +53,8 @@ def load_library() -> C.CDLL:
         L.ts_destroy.argtypes = [C.c_void_p]
         L.ts_set_ablation.argtypes = [C.c_void_p, C.c_uint32]
         L.ts_set_ablation.restype = C.c_int32
+        L.ts_set_test_mode.argtypes = [C.c_void_p, C.c_uint32]
+        L.ts_set_test_mode.restype = C.c_int32
         vp, i32, f32, u64, sz = C.c_void_p, C.c_int32, C.c_float, C.c_uint64, C.c_size_t
         L.ts_score_parents.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, f32, u64] + [vp] * 6 + [vp, sz, vp]
         L.ts_score_parents_static.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, f32, u64] + [vp] * 6 + [vp]
@@ -90,7 +93,7 @@ class TreeSpark:
     """A library context for one configuration plus its caller-owned workspace."""
 
     def __init__(self, V, D, r, K, Nmax, max_batch, dtype=torch.bfloat16, calib_mode=0, platt_a=0.67,
-                 platt_b=-0.46, calib_lo=-10.0, calib_hi=10.0, calib_table=None, device="cuda"):
+                 platt_b=-0.46, calib_lo=-10.0, calib_hi=10.0, calib_table=None, device="cuda", test_mode=0):
         self.lib = load_library()
         self.V, self.D, self.r, self.K, self.Nmax, self.max_batch = V, D, r, K, Nmax, max_batch
         self.dtype = dtype
@@ -107,6 +110,8 @@ class TreeSpark:
         self._ctx = C.c_void_p()
         with torch.cuda.device(self.device):
             self._check(self.lib.ts_create(C.byref(cfg), C.byref(self._ctx)))
+            if test_mode:   # the library's own tests: other kernel paths, shortened waits
+                self._check(self.lib.ts_set_test_mode(self._ctx, int(test_mode)))
         self.ws_bytes = int(self.lib.ts_workspace_bytes(self._ctx, max_batch))
         self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=self.device)
 
@@ -124,6 +129,11 @@ class TreeSpark:
     def _check(self, code: int):
         if code != TS_OK:
             raise TreeSparkError(f"status {code}: {self.lib.ts_last_error_string().decode()}")
+
+    def set_test_mode(self, flags: int):
+        """Switch test modes after construction; only the modes that leave the workspace size alone
+        (wait limits, lost arrival, seeding) may be changed this way."""
+        self._check(self.lib.ts_set_test_mode(self._ctx, int(flags)))
 
     def set_ablation(self, flags: int):
         self._check(self.lib.ts_set_ablation(self._ctx, int(flags)))

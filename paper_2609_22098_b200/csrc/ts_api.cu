@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include "ts_internal.h"
+#include "ts_tc.cuh"
 
 namespace ts {
 
@@ -38,6 +39,22 @@ static bool choose_tile(const ts_config& c, int num_sms, int max_smem, TileCfg* 
   out->ntiles = (c.V + tv - 1) / tv;
   out->smem = (size_t)c.r * tv * es + fixed;
   return out->ntiles <= 32 * 16;
+}
+
+// Which kernels serve this configuration (and with which wait limits), from the configuration, the
+// device and the test switches.  False: no vocabulary tiling fits shared memory.
+static bool select_paths(ts_ctx* ctx) {
+  const ts_config& c = ctx->cfg;
+  const unsigned tm = ctx->test_mode;
+  // tensor cores for bf16 inputs whose rows allow 16-byte chunks; the fp32 FMA kernel otherwise
+  ctx->use_mma = (c.dt_U == TS_DTYPE_BF16 && c.r % 8 == 0 && c.V % 8 == 0 && ctx->cc_major == 10 && !(tm & TS_TEST_FORCE_FMA)) ? 1 : 0;
+  ctx->tma_state = (tm & TS_TEST_NO_TMA) ? -1 : 0;
+  ctx->tmapW_ptr = nullptr;
+  if (ctx->use_mma && !choose_tile_mma(c, ctx->num_sms, ctx->max_smem, &ctx->tile)) ctx->use_mma = 0;
+  if (!ctx->use_mma && !choose_tile(c, ctx->num_sms, ctx->max_smem, &ctx->tile)) return false;
+  ctx->few_ok = (few_supported(ctx) && !(tm & TS_TEST_NO_FEW)) ? 1 : 0;
+  ctx->wait_limit = (tm & TS_TEST_SHORT_WAITS) ? 4096u : WAIT_LIMIT;
+  return true;
 }
 
 }  // namespace ts
@@ -80,16 +97,9 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
   if (e != cudaSuccess) { delete (Prof*)ctx->prof; delete ctx; return set_cuda_error("ts_create", e); }
   ctx->num_sms = prop.multiProcessorCount;
   ctx->max_smem = (int)prop.sharedMemPerBlockOptin;
-  // tensor cores for bf16 inputs whose rows allow 16-byte chunks; the fp32 FMA kernel otherwise
-  ctx->use_mma = (cfg->dt_U == TS_DTYPE_BF16 && cfg->r % 8 == 0 && cfg->V % 8 == 0 && prop.major == 10) ? 1 : 0;
-  // developer switches: TS_FORCE_FMA=1 keeps bf16 inputs on the fp32-FMA kernels, TS_NO_TMA=1 makes the
-  // tensor-core kernels stage W with plain loads (the path taken when no tensor map can be encoded)
-  const char* force = getenv("TS_FORCE_FMA");
-  if (force && force[0] == '1') ctx->use_mma = 0;
-  const char* no_tma = getenv("TS_NO_TMA");
-  if (no_tma && no_tma[0] == '1') ctx->tma_state = -1;
-  if (ctx->use_mma && !choose_tile_mma(ctx->cfg, ctx->num_sms, ctx->max_smem, &ctx->tile)) ctx->use_mma = 0;
-  if (!ctx->use_mma && !choose_tile(ctx->cfg, ctx->num_sms, ctx->max_smem, &ctx->tile)) {
+  ctx->cc_major = prop.major;
+  ctx->test_mode = 0;
+  if (!select_paths(ctx)) {
     delete (Prof*)ctx->prof; delete ctx;
     return set_error(TS_ERR_UNSUPPORTED, "ts_create: no vocabulary tiling fits shared memory");
   }
@@ -105,13 +115,9 @@ extern "C" int32_t ts_create(const ts_config* cfg, ts_ctx** out) {
   ctx->calib.a = cfg->platt_a; ctx->calib.b = cfg->platt_b;
   ctx->calib.lo = cfg->calib_lo; ctx->calib.hi = cfg->calib_hi;
   ctx->calib.table = ctx->d_table;
-  // developer switch: TS_NO_FEW=1 sends every level to the tile kernels
-  {
-    const char* no_few = getenv("TS_NO_FEW");
-    ctx->few_ok = (few_supported(ctx) && !(no_few && no_few[0] == '1')) ? 1 : 0;
-  }
   e = score_setup(ctx);
   if (e == cudaSuccess) e = verify_setup(ctx);
+  if (e == cudaSuccess) e = expand_setup(ctx);
   if (e != cudaSuccess) { cudaFree(ctx->d_table); delete (Prof*)ctx->prof; delete ctx; return set_cuda_error("ts_create", e); }
   *out = ctx;
   return TS_OK;
@@ -130,6 +136,22 @@ extern "C" int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags) {
   if (!ctx) return set_error(TS_ERR_INVALID, "ts_set_ablation: null context");
   if (flags & ~(uint32_t)TS_ABLATE_CALIB_QT) return set_error(TS_ERR_INVALID, "ts_set_ablation: unknown switch");
   ctx->ablation = flags;
+  return TS_OK;
+}
+
+extern "C" int32_t ts_set_test_mode(ts_ctx* ctx, uint32_t flags) {
+  if (!ctx) return set_error(TS_ERR_INVALID, "ts_set_test_mode: null context");
+  const uint32_t known = TS_TEST_FORCE_FMA | TS_TEST_NO_TMA | TS_TEST_NO_FEW | TS_TEST_NO_SEED | TS_TEST_SHORT_WAITS | TS_TEST_LOST_ARRIVAL;
+  if (flags & ~known) return set_error(TS_ERR_INVALID, "ts_set_test_mode: unknown switch");
+  const unsigned before = ctx->test_mode;
+  ctx->test_mode = flags;
+  if (!select_paths(ctx)) {
+    ctx->test_mode = before;
+    select_paths(ctx);
+    return set_error(TS_ERR_UNSUPPORTED, "ts_set_test_mode: no vocabulary tiling fits shared memory on that path");
+  }
+  const cudaError_t e = score_setup(ctx);
+  if (e != cudaSuccess) return set_cuda_error("ts_set_test_mode", e);
   return TS_OK;
 }
 

@@ -29,7 +29,7 @@ constexpr int SLOT_STRIDE = 32;
 constexpr int FEW_MAX = 8;           // levels with at most this many parents go to the few-parents scoring kernel
 constexpr int SCORE_THREADS = 128;   // one parent per thread; every thread scans the CTA's whole tile
 constexpr int CHUNK = 16;            // tokens per coarse generator call
-constexpr int MMA_S = 2;             // column splits per tile in the tensor-core scoring kernel (warps per row quarter)
+constexpr int MMA_S = 4;             // column splits per tile in the tensor-core scoring kernel (scanning warps per row quarter)
 
 enum Stream : uint32_t { STREAM_GUMBEL_COARSE = 1, STREAM_GUMBEL_FINE = 2, STREAM_ACCEPT = 3, STREAM_BONUS = 4 };
 
@@ -55,6 +55,7 @@ struct ts_ctx {
   float* d_table;
   int device;
   int num_sms;
+  int cc_major;
   int max_smem;
   ts::TileCfg tile;
   int vt_TV, vt_n;  // vocabulary ranges of the verification walk, one per CTA
@@ -69,6 +70,8 @@ struct ts_ctx {
   int tma_state;   // 0 not tried yet, 1 encoder found, -1 unavailable
   int walk_pdl;    // -1: the driver refused a cooperative launch with programmatic serialization
   unsigned ablation;   // TS_ABLATE_* switches (0 = the method)
+  unsigned test_mode;  // TS_TEST_* switches (0 = the product's kernel selection and wait limits)
+  uint32_t wait_limit; // polls before a bounded device-side wait gives up
 };
 
 namespace ts {
@@ -127,13 +130,12 @@ struct VerifyState {
   double fp[KMAX], fq[KMAX];
 };
 
-// Bytes of the scoring records for `cap` parent slots: one record per (tile, column split, slot) of the
-// tile kernels, and room for the few-parents kernel's records (one per 256-token tile and parent, at most
-// FEW_MAX parents), whichever is larger.
+// Bytes of the scoring records for `cap` parent slots: one record per (tile, slot) of the tile kernels,
+// and room for the few-parents kernel's records (one per 256-token tile and parent, at most FEW_MAX
+// parents), whichever is larger.
 __host__ inline size_t record_bytes(const ts_ctx* ctx, int cap) {
   const size_t rw = (4 + 5 * (size_t)ctx->cfg.K + 3) & ~(size_t)3;
-  const size_t S = ctx->use_mma ? MMA_S : 1;
-  const size_t tile = (size_t)ctx->tile.ntiles * S * (size_t)cap;
+  const size_t tile = (size_t)ctx->tile.ntiles * (size_t)cap;
   const size_t few = (size_t)((ctx->cfg.V + 255) / 256) * FEW_MAX;
   return align_up((tile > few ? tile : few) * rw * sizeof(float), 256);
 }
@@ -325,7 +327,7 @@ __device__ __forceinline__ double log_phat(const DevCalib& c, int d, double lx, 
 // Bounded grid barrier for cooperative (co-resident) launches: counter + generation in global memory.
 // Returns false when the wait ran out; the caller must then stop using the barrier and exit.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned nblocks, unsigned& gen) {
+__device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned nblocks, unsigned& gen, unsigned limit = 1u << 22) {
   __syncthreads();
   bool ok = true;
   if (threadIdx.x == 0) {
@@ -335,7 +337,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned nblocks, un
     unsigned spins = 0;
     while (*((volatile unsigned*)&bar[0]) < target) {
       if (*((volatile unsigned*)&bar[1]) != 0u) { ok = false; break; }
-      if (++spins > (1u << 22)) { atomicExch(&bar[1], 1u); ok = false; break; }
+      if (++spins > limit) { atomicExch(&bar[1], 1u); ok = false; break; }
       if (spins > 256u) __nanosleep(32);
     }
     __threadfence();

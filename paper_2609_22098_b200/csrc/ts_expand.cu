@@ -359,6 +359,13 @@ __global__ void __launch_bounds__(256) expand_finalize_kernel(FinalArgs a) {
   for (int i = tid; i < n * a.words; i += blockDim.x) a.mask[pb * a.words + i] = s_mask[i];
 }
 
+// the level kernel ranks a request's pool and candidates out of dynamic shared memory: opt in once per context
+cudaError_t expand_setup(ts_ctx* ctx) {
+  const size_t level_smem = (size_t)(ctx->cfg.Nmax + ctx->cfg.Nmax * ctx->cfg.K) * sizeof(Entry);
+  if (level_smem <= 48 * 1024) return cudaSuccess;
+  return cudaFuncSetAttribute(expand_level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)level_smem);
+}
+
 }  // namespace ts
 
 extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, const void* W, int32_t B,
@@ -417,11 +424,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   { ProfScope ps(ctx, K_INIT, st); e0 = launch_kernel(expand_init_kernel, B > 296 ? B : 296, 256, 0, st, true, a); }
   cudaError_t e = e0 != cudaSuccess ? e0 : cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(init)", e);
-  const size_t level_smem = (size_t)(c.Nmax + c.Nmax * c.K) * sizeof(Entry);
-  if (level_smem > 48 * 1024) {
-    e = cudaFuncSetAttribute(expand_level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)level_smem);
-    if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(attr)", e);
-  }
+  const size_t level_smem = (size_t)(c.Nmax + c.Nmax * c.K) * sizeof(Entry);   // opted into at ts_create when above 48 KB
   long long level_bound = B;   // parents a level can have at most: B at the root, K times more per level, B * Nmax overall
   for (int d = 0; d < c.D; ++d) {
     const int cur = d & 1;

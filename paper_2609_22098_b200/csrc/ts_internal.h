@@ -12,6 +12,7 @@ int32_t set_cuda_error(const char* where, cudaError_t e);
 
 cudaError_t score_setup(ts_ctx* ctx);
 cudaError_t verify_setup(ts_ctx* ctx);
+cudaError_t expand_setup(ts_ctx* ctx);
 
 struct ScoreArgs {
   const void *U, *A, *W;
@@ -26,6 +27,9 @@ struct ScoreArgs {
   float* rec; int* err;
   unsigned* thr;    // [2][cap]: launch-wide lower bounds (logit, key) per parent, order-preserving encoding
   unsigned* slots;  // [2][cap][K]
+  uint32_t wait_limit;   // polls before a bounded device-side wait gives up
+  int lost_arrival;      // test switch: the A-tile barrier expects one arrival more than will come
+  int seed_bounds;       // 1: pieces publish an exactly evaluated token before they scan (tensor-core kernel)
 };
 
 struct MergeArgs {

@@ -5,9 +5,6 @@
 
 #include "ts_common.cuh"
 
-#ifndef TS_SCAN_MARK
-#define TS_SCAN_MARK(n) do { } while (0)
-#endif
 namespace ts {
 
 // Record layout in 32-bit words: [m, s0, sT, counts, topv[K], topi[K], keyv[K], keyi[K], keyl[K]]
@@ -207,7 +204,6 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
                                            uint64_t seed, int req, uint64_t hash, const float* ghi,
                                            float gL, float gK, const SharedThr& gl, const SharedThr& gk,
                                            const volatile unsigned* liveL = nullptr, const volatile unsigned* liveK = nullptr) {
-  if (valid) TS_SCAN_MARK(0);
   // High half of each token's uniform, one generator call per eight tokens.  Issued first and in the same
   // straight-line block as the sums below: the generator's long dependent chains and the exponentials'
   // latencies then overlap instead of following each other.
@@ -261,11 +257,9 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
   }
   st.s0 += a0;
   st.sT += two ? aT : a0;
-  if (valid) TS_SCAN_MARK(1);
   // the chunk's best logit is a candidate for the top-K list (it is inserted further down): publishing it
   // right away costs nothing and gives the other pieces of the launch their first logit bounds early
   if (cm > st.bestL && cm > st.thrL && cm >= gL) { st.bestL = cm; publish(gl, cm); }
-  if (valid) TS_SCAN_MARK(2);
   if (T > 0.f) {
     const float thr = fmaxf(st.thrK, gK);
     uint32_t mk = 0;
@@ -314,7 +308,6 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
     }
     uint4 fw = make_uint4(0, 0, 0, 0);
     int fine_call = -1;
-    if (valid) TS_SCAN_MARK(3);
 #pragma unroll 1
     while (mk) {
       const int i = __ffs(mk) - 1;
@@ -357,7 +350,6 @@ __device__ __forceinline__ void scan_chunk(RowScan<Lists>& st, const float* l, i
       }
     }
   }
-  if (valid) TS_SCAN_MARK(4);
 }
 
 // Replication of parents over the 128 rows of a tensor-core tile when a level has few parents:

@@ -340,7 +340,9 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
   a.pdl = pdl ? 1 : 0; a.P_prev_dev = P_prev_dev;
   a.U = U; a.A = A; a.W = W; a.V = c.V; a.D = c.D; a.r = c.r; a.K = c.K; a.P = P; a.P_dev = P_dev;
   a.p_req = p_req; a.p_depth = p_depth; a.p_token = p_token; a.p_hash = p_hash; a.T = T; a.seed = seed;
-  a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.cap = cap; a.S = ctx->use_mma ? MMA_S : 1; a.rec = rec; a.err = err;
+  a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.cap = cap; a.S = 1; a.rec = rec; a.err = err;
+  a.wait_limit = ctx->wait_limit; a.seed_bounds = (ctx->test_mode & TS_TEST_NO_SEED) ? 0 : 1;
+  a.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
   a.thr = thr_base(ctx, rec, cap); a.slots = a.thr + 2 * (size_t)cap;
   cudaError_t e = cudaSuccess;
   // Which kernel scores the level: the few-parents kernel when the host knows that the list cannot hold

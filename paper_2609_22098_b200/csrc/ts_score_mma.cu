@@ -1,49 +1,142 @@
 // Tensor-core scoring kernel for sm_100a: the low-rank bias [parents x r] . [r x tile] runs on the
 // 5th-generation tensor cores (tcgen05.mma, accumulators in tensor memory), and the vocabulary scan
-// (add base logits, online max / sum-exp, top-K, Gumbel top-K) is its epilogue, one tensor-memory
-// lane = one parent row per thread.
+// (add base logits, online max / sum-exp, candidates for the top-K and Gumbel top-K lists) is its
+// epilogue, one tensor-memory lane = one parent row per thread.
 //
 // CTA = one vocabulary tile, resident for the whole launch.  Shared memory holds
 //   W tile  : B operand, MN-major, 128-byte swizzle: slabs of 64 tokens, slab = [rp rows][128 B];
 //             loaded by bulk-tensor copies (one mbarrier per 128-token block), or by plain loads when
 //             no tensor map could be encoded
 //   A tile  : A operand, K-major, 128-byte swizzle: [rp/64 slabs][128 rows][128 B] (gathered rows A[x_p])
-// (rp = r rounded up to 64, padding zero-filled).  Warps 0..7 are epilogue warps: warp w reads the
-// tensor-memory lanes 32*(w%4).. (its quarter of the 128 parent rows).  When a level has few parents the
-// rows are replicated R = 2 or 4 times over the quarters; of the tile's 16-token chunks, chunk cg belongs
-// to replica cg % R and column split (cg / R) % 2 (= w / 4).  Warp 8 allocates tensor memory and its
-// lane 0 issues the MMAs: per block of 128 tokens rp/16 instructions of M=128, N=128 (64 at a ragged
-// end), K=16 into one of four 128-column accumulator buffers, then a commit that arrives on that
-// buffer's "full" barrier; epilogue warps arrive on its "empty" barrier when they have drained it.
-// Warp 9 keeps shared-memory copies of the launch-wide pruning bounds of every row current.
+//   lists   : per parent row the K best logits and K best sampling keys this CTA has seen
+//   queues  : candidates on their way from the scanning warps to the selector warps
+// (rp = r rounded up to 64, padding zero-filled).
+//
+// Warps 0..15 scan: warp w reads the tensor-memory lanes 32*(w%4).. (its quarter of the 128 parent
+// rows) and, of the tile's 16-token chunks, those of column split w/4.  When a level has few parents
+// the rows are replicated R = 2 or 4 times over the quarters and the copies split the chunks too:
+// chunk cg belongs to replica cg % R and split (cg / R) % 4.  A scanning thread keeps only the running
+// (max, sums) of its row; a token that can still be among the row's K best (its logit, or the upper
+// bound of its sampling key given the leading 16 bits of its uniform, reaches the row's current bound)
+// is appended to a queue with a few instructions, so that the 32 rows of a warp never wait for the
+// rare, long evaluation of one of them.  Warps 18 and 19 (rows 0..63 / 64..127) drain the queues, one
+// candidate per lane: exact key (second generator call, two logarithms), insertion into the row's
+// sorted lists, publication of new bests.  Warp 16 allocates tensor memory and its lane 0 issues the
+// MMAs: per block of 128 tokens rp/16 instructions of M=128, N=128 (64 at a ragged end), K=16 into one
+// of four 128-column accumulator buffers, then a commit that arrives on that buffer's "full" barrier;
+// scanning warps arrive on its "empty" barrier when they have drained it.  Warp 17 keeps shared-memory
+// copies of the launch-wide pruning bounds of every row current.
+//
+// Launch-wide bounds.  Per parent K slots in global memory; slot j holds the best value published by
+// the pieces (tile, split, replica) whose number is j modulo K.  Pieces hold disjoint tokens, so the
+// slots hold values of K different tokens and their minimum is a lower bound of the parent's K-th best
+// value: a token strictly below it cannot be among the K best.  So that bounds exist before the scan
+// begins, every scanning thread first evaluates exactly the best-logit token of its first chunk and
+// publishes its logit and key (the seed), then waits a few microseconds (bounded) for the bounds of
+// its row to arrive.
+//
 // Every wait is bounded: when one runs out the kernel raises an error word, skips the remaining work,
 // waits (again bounded) for bulk loads still in flight, frees its tensor memory and returns.
 #include "ts_tc.cuh"
 #include "ts_internal.h"
-namespace ts {
-#ifdef TS_DEBUG_TIMING
-// developer aid: per-CTA timestamps (globaltimer ns) of the phases of one launch
-__device__ unsigned long long g_dbg[148 * 64];
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define DBG(slot) do { if ((threadIdx.x & 31) == 0 && blockIdx.x < 148) g_dbg[blockIdx.x * 64 + (slot)] = gtime(); } while (0)
-#define TS_SCAN_MARK(n) do { if (threadIdx.x == 0 && blockIdx.x < 148 && g_dbg[blockIdx.x * 64 + 56 + (n)] == 0ull) g_dbg[blockIdx.x * 64 + 56 + (n)] = gtime(); } while (0)
-#else
-#define DBG(slot) do { } while (0)
-#endif
-
-}  // namespace ts
 #include "ts_scan.cuh"
 
 namespace ts {
 
-constexpr int EPI_WARPS = 4 * MMA_S;
-constexpr int MMA_THREADS = (EPI_WARPS + 2) * 32;   // epilogue warps, the MMA warp, the bounds-refresh warp
+constexpr int EPI_S = MMA_S;                // column splits = scanning warps per row quarter
+constexpr int EPI_WARPS = 4 * EPI_S;
+constexpr int W_MMA = EPI_WARPS;            // warp roles
+constexpr int W_REFRESH = EPI_WARPS + 1;
+constexpr int W_SEL = EPI_WARPS + 2;
+constexpr int NSEL = 2;                     // selector warps (rows 0..63, 64..127)
+constexpr int MMA_THREADS = (EPI_WARPS + 2 + NSEL) * 32;
 constexpr int BLK_N = 128;
 constexpr int NBUF = 4;                 // accumulator buffers of BLK_N columns in tensor memory
 constexpr uint32_t TMEM_COLS = NBUF * BLK_N;
 constexpr int MAX_BLK = 32;             // blocks of BLK_N tokens in the largest tile (4096 tokens)
+constexpr int QCAP = 256;               // entries per candidate queue (power of two)
+constexpr uint32_t KIND_TOP = 1u, KIND_KEY = 2u;
 
-template <class Lists>
+// Shared-memory state of the selection side of one CTA.
+struct SelShared {
+  float* lists;             // [128][5K]: topv, topi, keyv, keyi, keyl of every row, sorted (value desc, token asc)
+  volatile float* lthr;     // [2][128]: K-th best logit / key of the row's lists (-inf until they are full)
+  volatile float* best;     // [2][EPI_S][128]: best logit / key published so far by the piece (row, split)
+  uint4* q;                 // [NSEL][QCAP] entries: token, logit, row | split << 8 | kind << 12 | c16 << 16, tag
+  volatile unsigned* q_head;   // [NSEL] entries consumed
+  unsigned* q_tail;            // [NSEL] entries claimed
+};
+
+// insertion into one sorted list of K entries (value desc, token asc); returns the new K-th value
+__device__ __forceinline__ float list_insert(float* v, int* t, float* aux, int K, float val, int tok, float lg) {
+  int pos = K - 1;
+  if (!(val > v[pos] || (val == v[pos] && (unsigned)tok < (unsigned)t[pos]))) return v[pos];
+  while (pos > 0 && (val > v[pos - 1] || (val == v[pos - 1] && (unsigned)tok < (unsigned)t[pos - 1]))) {
+    v[pos] = v[pos - 1]; t[pos] = t[pos - 1];
+    if (aux) aux[pos] = aux[pos - 1];
+    --pos;
+  }
+  v[pos] = val; t[pos] = tok;
+  if (aux) aux[pos] = lg;
+  return v[K - 1];
+}
+
+// The seed of one piece: its first chunk's best-logit token, evaluated exactly, gives every parent a
+// lower bound of its K-th best logit and key before the scan proper begins.
+static __device__ __noinline__ void publish_seed(const float* l, int v0, float invT, bool keys, uint64_t seed, int req,
+                                                 uint64_t hash, unsigned* slotL, unsigned* slotK) {
+  float bl = l[0]; int bi = 0;
+#pragma unroll
+  for (int i = 1; i < 16; ++i) if (l[i] > bl) { bl = l[i]; bi = i; }
+  if (!(bl > -INFINITY)) return;
+  atomicMax(slotL, enc_f(bl));
+  if (keys) {
+    const int v = v0 + bi;
+    const uint4 cw = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, (uint32_t)v >> 3);
+    const uint4 fw = stream_words(seed, req, hash, STREAM_GUMBEL_FINE, (uint32_t)v >> 3);
+    const uint32_t c16 = (word_of(cw, (v & 7) >> 1) >> (16 * (v & 1))) & 0xFFFFu;
+    const uint32_t f16 = (word_of(fw, (v & 7) >> 1) >> (16 * (v & 1))) & 0xFFFFu;
+    atomicMax(slotK, enc_f(bl * invT + gumbel_from_bits((c16 << 16) | f16)));
+  }
+}
+
+// One candidate, handled by one selector lane: exact key, insertion, publication.
+__device__ __forceinline__ void select_candidate(const ScoreArgs& a, const SelShared& sh, const uint4 e, const float* ghi,
+                                                 float invT, int K, int tile, int R, int g, const volatile unsigned* s_thr,
+                                                 int pbase, bool do_insert) {
+  const int tok = (int)e.x;
+  const float lg = __uint_as_float(e.y);
+  const int row = (int)(e.z & 0xFFu), s = (int)((e.z >> 8) & 0xFu);
+  const uint32_t kind = (e.z >> 12) & 0xFu, c16 = e.z >> 16;
+  const int per = 128 / R;
+  const int p = R > 1 ? row % per : g * 128 + row, rho = R > 1 ? row / per : 0;
+  const int prow = pbase + (R > 1 ? row % per : row);
+  const int pid = ((tile * EPI_S + s) * R + rho) % K;
+  float* L = sh.lists + (size_t)row * 5 * K;
+  if (kind & KIND_TOP) {
+    const float gL = dec_f(s_thr[prow]);
+    if (lg >= gL && lg >= sh.lthr[row] && do_insert) {
+      sh.lthr[row] = list_insert(L, reinterpret_cast<int*>(L) + K, nullptr, K, lg, tok, 0.f);
+      volatile float* b = sh.best + (0 * EPI_S + s) * 128 + row;
+      if (lg > *b) { *b = lg; atomicMax(a.slots + ((size_t)p * K + pid) * SLOT_STRIDE, enc_f(lg)); }
+    }
+  }
+  if (kind & KIND_KEY) {
+    const float thr = fmaxf(dec_f(s_thr[128 + prow]), sh.lthr[128 + row]);
+    const float bnd = lg * invT + ghi[noise_bound_index(c16)];
+    if (bnd >= thr && do_insert) {   // the bounds have often risen since the candidate was queued
+      const uint4 fw = stream_words(a.seed, a.p_req[p], a.p_hash[p], STREAM_GUMBEL_FINE, (uint32_t)tok >> 3);
+      const uint32_t f16 = (word_of(fw, (tok & 7) >> 1) >> (16 * (tok & 1))) & 0xFFFFu;
+      const float key = lg * invT + gumbel_from_bits((c16 << 16) | f16);
+      if (key >= thr) {
+        sh.lthr[128 + row] = list_insert(L + 2 * K, reinterpret_cast<int*>(L) + 3 * K, L + 4 * K, K, key, tok, lg);
+        volatile float* b = sh.best + (1 * EPI_S + s) * 128 + row;
+        if (key > *b) { *b = key; atomicMax(a.slots + (((size_t)a.cap + p) * K + pid) * SLOT_STRIDE, enc_f(key)); }
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma) {
   extern __shared__ unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -62,24 +155,31 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   unsigned char* Ws = sm;
   unsigned char* As = Ws + (size_t)nslab * slab_bytes;
   float* ghi = reinterpret_cast<float*>(As + (size_t)(rp / 64) * a_slab_bytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ghi + 512);
-  uint64_t* a_full = bars;            // epilogue threads -> MMA: the A tile of this group is in place
-  uint64_t* t_full = bars + 1;             // [NBUF] MMA -> epilogue: accumulator buffer written
-  uint64_t* t_empty = bars + 1 + NBUF;     // [NBUF] epilogue -> MMA: accumulator buffer drained
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 + 2 * NBUF);
+  SelShared sh;
+  sh.q = reinterpret_cast<uint4*>(ghi + 512);                                   // 16-byte aligned
+  sh.lists = reinterpret_cast<float*>(sh.q + NSEL * QCAP);
+  sh.lthr = sh.lists + (size_t)128 * 5 * K;
+  sh.best = sh.lthr + 2 * 128;
+  float* s_part = const_cast<float*>(sh.best) + 2 * EPI_S * 128;                // [EPI_S][128][4]: m, s0, sT of every (split, row)
+  volatile unsigned* s_thr = reinterpret_cast<volatile unsigned*>(s_part + EPI_S * 128 * 4);   // [group parity][2][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(const_cast<unsigned*>(s_thr) + 512);
+  uint64_t* a_full = bars;            // scanning threads -> MMA: the A tile of this group is in place
+  uint64_t* t_full = bars + 1;             // [NBUF] MMA -> scan: accumulator buffer written
+  uint64_t* t_empty = bars + 1 + NBUF;     // [NBUF] scan -> MMA: accumulator buffer drained
+  uint64_t* w_full = bars + 1 + 2 * NBUF;  // [MAX_BLK] W slabs of block nb landed
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(w_full + MAX_BLK);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
-  // per-row copies of the launch-wide pruning bounds (logit, key), refreshed once per block of tokens
-  volatile unsigned* s_thr = reinterpret_cast<volatile unsigned*>(s_tmem + 4);   // [group parity][2][128]
-  volatile int* s_done = reinterpret_cast<volatile int*>(s_tmem + 2);             // epilogue warps finished
-  uint64_t* w_full = reinterpret_cast<uint64_t*>(const_cast<unsigned*>(s_thr) + 512);   // [MAX_BLK] W slabs of block nb landed
+  volatile int* s_done = reinterpret_cast<volatile int*>(s_tmem + 2);             // scanning warps finished (cumulative)
+  sh.q_head = reinterpret_cast<volatile unsigned*>(s_tmem + 4);
+  sh.q_tail = s_tmem + 4 + NSEL;
 
   const __nv_bfloat16* Wg = reinterpret_cast<const __nv_bfloat16*>(a.W);
   const __nv_bfloat16* Ug = reinterpret_cast<const __nv_bfloat16*>(a.U);
   const __nv_bfloat16* Ag = reinterpret_cast<const __nv_bfloat16*>(a.A);
+  const uint32_t wait_limit = a.wait_limit;
 
   // ---- set-up ------------------------------------------------------------------------------------
-  if (warp == 0) DBG(0);
-  if (warp == EPI_WARPS) {
+  if (warp == W_MMA) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -93,10 +193,11 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
     }
   };
   if (tid == 0) {
-    mbar_init(a_full, EPI_WARPS * 32);
+    mbar_init(a_full, EPI_WARPS * 32 + (a.lost_arrival ? 1 : 0));
     for (int i = 0; i < NBUF; ++i) { mbar_init(t_full + i, 1); mbar_init(t_empty + i, EPI_WARPS); }
     *s_abort = 0;
     *s_done = 0;
+    for (int i = 0; i < NSEL; ++i) { sh.q_head[i] = 0u; sh.q_tail[i] = 0u; }
     if (use_tma) for (int i = 0; i < nblk_w; ++i) mbar_init(w_full + i, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // W tile by bulk-tensor loads, one barrier per block of 128 tokens so that the first MMAs start while
@@ -116,146 +217,237 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       *reinterpret_cast<uint4*>(Ws + (size_t)slab * slab_bytes + k * 128 + ((j ^ (k & 7)) << 4)) = v;
     }
   }
-  if (warp == 0) DBG(1);
   fill_gumbel_bounds(ghi, tid, MMA_THREADS);
   for (int i = tid; i < 512; i += MMA_THREADS) s_thr[i] = 0u;
-  if (warp == 0) DBG(2);
+  for (int i = tid; i < NSEL * QCAP; i += MMA_THREADS) sh.q[i] = make_uint4(0u, 0u, 0u, 0u);   // tag 0 = never written
   fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  if (warp == 0) DBG(3);
   pdl_wait();                // parent lists and the level's parent count come from the previous kernel
   pdl_launch_dependents();
   const int P = a.P_dev ? *a.P_dev : a.P;   // may be 0: an empty level only tears down
   if (use_tma && !early_w && P > 0 && tid == 0) issue_w();
 
   const int R = mma_replicas(P), rsh = R == 4 ? 2 : (R == 2 ? 1 : 0);
+  const int per = 128 / R;
   const int ngroups = P <= 0 ? 0 : (R > 1 ? 1 : (P + 127) / 128);
   const int nblk = (tlen + BLK_N - 1) / BLK_N;
   const float T = a.T, invT = T > 0.f ? 1.f / T : 1.f;
+  const bool keys = T > 0.f;
   const int rw = rec_words(K);
+  // launch-wide bounds can form only when every one of the K slots has a piece that feeds it
+  const bool seeded = (long long)a.ntiles * EPI_S * R >= 2 * K && a.seed_bounds != 0;
 
-  if (warp < EPI_WARPS) {
-    // ======================= epilogue warps =======================================================
-    const int q = warp & 3, s = warp >> 2;
-    const int row = q * 32 + lane;
-    const int e = warp * 32 + lane;  // 0..255
-    const int cpr = rp / 8;          // 16-byte chunks per A row
-    bool alive = true;
-    for (int g = 0; g < ngroups && alive; ++g) {
+  for (int g = 0; g < ngroups; ++g) {
+    const int pbase = (g & 1) * 256;   // rows of group g use the bound buffer of parity g & 1
+    // ---- per-group reset of the selection state (every thread) ---------------------------------------
+    for (int i = tid; i < 128 * 5 * K; i += MMA_THREADS) {
+      const int f = (i / K) % 5;   // fields: topv, topi, keyv, keyi, keyl
+      sh.lists[i] = (f == 0 || f == 2) ? -INFINITY : ((f == 1 || f == 3) ? __int_as_float(-1) : 0.f);
+    }
+    for (int i = tid; i < 2 * 128; i += MMA_THREADS) { sh.lthr[i] = -INFINITY; s_thr[pbase + i] = 0u; }
+    for (int i = tid; i < 2 * EPI_S * 128; i += MMA_THREADS) sh.best[i] = -INFINITY;
+    __syncthreads();
+
+    if (warp < EPI_WARPS) {
+      // ======================= scanning warps =======================================================
+      const int q = warp & 3, s = warp >> 2;
+      const int row = q * 32 + lane;
+      const int e = warp * 32 + lane;
+      const int cpr = rp / 8;          // 16-byte chunks per A row
       // gather this group's parent rows A[x_p] into the swizzled A tile
       for (int idx = e; idx < 128 * cpr; idx += EPI_WARPS * 32) {
         const int rr = idx / cpr, ck = idx % cpr;
-        const int p = R > 1 ? rr % (128 / R) : g * 128 + rr;
+        const int p = R > 1 ? rr % per : g * 128 + rr;
         uint4 v = make_uint4(0, 0, 0, 0);
         if (p < P && ck * 8 < r) v = __ldg(reinterpret_cast<const uint4*>(Ag + (size_t)a.p_token[p] * r + ck * 8));
         *reinterpret_cast<uint4*>(As + (size_t)(ck >> 3) * a_slab_bytes + rr * 128 + (((ck & 7) ^ (rr & 7)) << 4)) = v;
       }
       fence_async_smem();
       mbar_arrive(a_full);
-      if (warp == 0) DBG(4);
 
-      const int p = R > 1 ? row % (128 / R) : g * 128 + row;
-      const int rho = R > 1 ? row / (128 / R) : 0;   // uniform within a warp (128/R is a multiple of 32)
+      const int p = R > 1 ? row % per : g * 128 + row;
+      const int rho = R > 1 ? row / per : 0;   // uniform within a warp (128/R is a multiple of 32)
       const bool active = p < P;
       int req = 0; uint64_t hash = 0; const __nv_bfloat16* Urow = Ug;
       if (active) {
         req = a.p_req[p]; hash = a.p_hash[p];
         Urow = Ug + ((size_t)req * a.D + a.p_depth[p]) * V;
       }
-      RowScan<Lists> st;
-      st.init(K);
-      // where this parent's cached bounds live: rows of group g use the buffer of parity g & 1.  That
-      // buffer last served group g-2; the refresh warp is at group g-1 or g by now (every warp has
-      // passed the A-tile barrier of g-1), so clearing it here cannot be overwritten with stale values.
-      const int prow = (g & 1) * 256 + (R > 1 ? row % (128 / R) : row);
-      if (s == 0) { s_thr[(g & 1) * 256 + row] = 0u; s_thr[(g & 1) * 256 + 128 + row] = 0u; }
+      const int prow = pbase + (R > 1 ? row % per : row);
+      const int sel = row >> 6;
+      const uint32_t ztag = (uint32_t)row | ((uint32_t)s << 8);
+      float m = -INFINITY, s0 = 0.f, sT = 0.f;
       uint4 nx0 = make_uint4(0, 0, 0, 0), nx1 = nx0;    // prefetched base logits of the next owned chunk
       bool have_next = false;
-      const int pc = active ? p : 0;
-      const int pid = ((tile * MMA_S + s) * R + rho) % K;   // which of the parent's K slots this piece feeds
-      const SharedThr gl{a.slots + (size_t)pc * K * SLOT_STRIDE, pid};
-      const SharedThr gk{a.slots + ((size_t)a.cap + pc) * K * SLOT_STRIDE, pid};
-      // Pass nb = -1 is a dry run of the scan on an empty chunk while the first MMAs are still on their
-      // way: it changes nothing in `st`, but it brings the scan's instructions into the instruction cache
-      // and requests the base logits of the first chunk this warp owns.
-      for (int nb = -1; nb < nblk; ++nb) {
-        const bool dry = nb < 0;
-        const int it = g * nblk + (dry ? 0 : nb), tb = it % NBUF, u = it / NBUF;
-        if (!dry) {
+      bool first = true;
+      bool alive = true;
+      for (int nb = 0; nb < nblk && alive; ++nb) {
+        const int it = g * nblk + nb, tb = it % NBUF, u = it / NBUF;
+        {
           int ok = 1;
-          if (lane == 0) ok = mbar_wait(t_full + tb, u & 1, s_abort, a.err) ? 1 : 0;
+          if (lane == 0) ok = mbar_wait(t_full + tb, u & 1, s_abort, a.err, wait_limit) ? 1 : 0;
           ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
           if (!ok) { alive = false; break; }
           tc_fence_after();
-          if (nb < 10 && g == 0) DBG(8 + warp * 6 + 0 + (nb >= 1 ? 2 : 0) + (nb >= 8 ? 2 : 0));
         }
-        const int nch = dry ? 1 : min(8, (tlen - nb * BLK_N + 15) / 16);
+        const int nch = min(8, (tlen - nb * BLK_N + 15) / 16);
         for (int c = 0; c < nch; ++c) {
-          // owned chunks: cg = rho + R * (s + MMA_S * j); the dry pass sits one step before the first
-          const int cg = dry ? rho + R * s - R * MMA_S : nb * 8 + c;
-          if (!dry && ((cg & (R - 1)) != rho || ((cg >> rsh) % MMA_S) != s)) continue;   // warp-uniform; R is 1, 2 or 4
+          const int cg = nb * 8 + c;
+          if ((cg & (R - 1)) != rho || ((cg >> rsh) % EPI_S) != s) continue;   // warp-uniform; R is 1, 2 or 4
           float acc[16];
-          if (!dry) {
-            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * BLK_N + c * 16), acc);
-          } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] = 0.f;
-          }
-          if (active) {
-            const int v0 = dry ? t0 : t0 + cg * 16;
-            const int valid = dry ? 0 : min(16, V - v0);   // 8 or 16: V and v0 are multiples of 8
-            // this chunk's base logits were requested one chunk ago; request the next owned chunk's now
-            const uint4 u0 = have_next ? nx0 : (dry ? make_uint4(0, 0, 0, 0) : __ldg(reinterpret_cast<const uint4*>(Urow + v0)));
-            const uint4 u1 = have_next ? nx1 : (valid > 8 ? __ldg(reinterpret_cast<const uint4*>(Urow + v0 + 8)) : make_uint4(0, 0, 0, 0));
-            {
-              const int cgn = cg + R * MMA_S;           // the next chunk this warp owns
-              const int vn = t0 + cgn * 16;
-              have_next = (cgn * 16 < tlen);
-              if (have_next) {
-                nx0 = __ldg(reinterpret_cast<const uint4*>(Urow + vn));
-                nx1 = (V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8)) : make_uint4(0, 0, 0, 0);
-              }
+          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * BLK_N + c * 16), acc);
+          if (!active) continue;
+          const int v0 = t0 + cg * 16;
+          const int valid = min(16, V - v0);   // 8 or 16: V and v0 are multiples of 8
+          // this chunk's base logits were requested one chunk ago; request the next owned chunk's now
+          const uint4 u0 = have_next ? nx0 : __ldg(reinterpret_cast<const uint4*>(Urow + v0));
+          const uint4 u1 = have_next ? nx1 : (valid > 8 ? __ldg(reinterpret_cast<const uint4*>(Urow + v0 + 8)) : make_uint4(0, 0, 0, 0));
+          {
+            const int cgn = cg + R * EPI_S;           // the next chunk this warp owns
+            const int vn = t0 + cgn * 16;
+            have_next = (cgn * 16 < tlen);
+            if (have_next) {
+              nx0 = __ldg(reinterpret_cast<const uint4*>(Urow + vn));
+              nx1 = (V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8)) : make_uint4(0, 0, 0, 0);
             }
+          }
+          {
             float ub[16];
             unpack_bf16x8(u0, ub);
             unpack_bf16x8(u1, ub + 8);
 #pragma unroll
             for (int i = 0; i < 16; ++i) acc[i] += ub[i];
-            if (valid < 16) {   // warp-uniform and rare (the vocabulary's last chunk, the dry pass): the scan's padding value
+          }
+          if (valid < 16) {   // warp-uniform and rare (the vocabulary's last chunk): padding that loses every comparison
 #pragma unroll
-              for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] : -INFINITY;
+            for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] : -INFINITY;
+          }
+          if (first) {
+            first = false;
+            if (seeded) {
+              const int pid = ((tile * EPI_S + s) * R + rho) % K;
+              publish_seed(acc, v0, invT, keys, a.seed, req, hash, a.slots + ((size_t)p * K + pid) * SLOT_STRIDE,
+                           a.slots + (((size_t)a.cap + p) * K + pid) * SLOT_STRIDE);
+              // the bounds of this row arrive a few microseconds later (the refresh warp copies them here)
+              const volatile unsigned* wthr = s_thr + (keys ? 128 : 0) + prow;
+              for (int spin = 0; spin < 96 && *wthr == 0u && !*s_abort; ++spin) __nanosleep(64);
             }
-            const float gLc = dec_f(s_thr[prow]), gKc = dec_f(s_thr[128 + prow]);   // kept fresh by the refresh warp
-            scan_chunk<Lists, true>(st, acc, v0, valid, T, invT, a.seed, req, hash, ghi, gLc, gKc, gl, gk, s_thr + prow, s_thr + 128 + prow);
+          }
+          // ---- the scan of one chunk -------------------------------------------------------------
+          // high halves of the sixteen uniforms: two generator calls, issued first so that their long
+          // dependent chains overlap the exponentials below
+          uint4 cw0 = make_uint4(0, 0, 0, 0), cw1 = cw0;
+          if (keys) {
+            cw0 = stream_words(a.seed, req, hash, STREAM_GUMBEL_COARSE, (uint32_t)v0 >> 3);
+            cw1 = stream_words(a.seed, req, hash, STREAM_GUMBEL_COARSE, ((uint32_t)v0 >> 3) + 1u);
+          }
+          float gmax[4];
+          float cm = -INFINITY;
+#pragma unroll
+          for (int sg = 0; sg < 4; ++sg) {
+            gmax[sg] = fmaxf(fmaxf(acc[4 * sg], acc[4 * sg + 1]), fmaxf(acc[4 * sg + 2], acc[4 * sg + 3]));
+            cm = fmaxf(cm, gmax[sg]);
+          }
+          {
+            // rescale to the new running maximum without a branch (no change: factor 1; first chunk: factor 0)
+            const float nm = fmaxf(m, cm);
+            const float d = (m == nm) ? 0.f : m - nm;
+            s0 *= __expf(d);
+            sT *= __expf(d * invT);
+            m = nm;
+          }
+          {
+            // exp(l - m) as ex2(l * log2(e) - m * log2(e)): one fused multiply-add and one ex2 per token.  While
+            // nothing finite has been seen (m = -inf) the offset is 0: every l is -inf then and contributes 0.
+            constexpr float LOG2E = 1.4426950408889634f;
+            const bool two = keys && (T != 1.f);
+            const float mref = m == -INFINITY ? 0.f : m;
+            const float off0 = -mref * LOG2E, scT = LOG2E * invT, offT = off0 * invT;
+            float a0 = 0.f, a1 = 0.f, aT = 0.f;
+#pragma unroll
+            for (int i = 0; i < 16; i += 2) {
+              a0 += ex2_approx(fmaf(acc[i], LOG2E, off0));
+              a1 += ex2_approx(fmaf(acc[i + 1], LOG2E, off0));
+              if (two) aT += ex2_approx(fmaf(acc[i], scT, offT)) + ex2_approx(fmaf(acc[i + 1], scT, offT));
+            }
+            a0 += a1;
+            s0 += a0;
+            sT += two ? aT : a0;
+          }
+          // ---- candidates ---------------------------------------------------------------------------
+          uint32_t mkK = 0, mkL = 0;
+          const float thrL = fmaxf(dec_f(s_thr[prow]), sh.lthr[row]);
+          if (cm >= thrL) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) mkL |= (uint32_t)(acc[i] >= thrL && acc[i] > -INFINITY) << i;
+          }
+          if (keys) {
+            const float thr = fmaxf(dec_f(s_thr[128 + prow]), sh.lthr[128 + row]);
+            // the whole chunk first: its best logit plus the noise bound of the largest leading bits among its
+            // sixteen tokens bounds every key in it; then four tokens at a time, then singly
+            const uint32_t m8 = __vmaxu2(__vmaxu2(__vmaxu2(cw0.x, cw0.y), __vmaxu2(cw0.z, cw0.w)),
+                                         __vmaxu2(__vmaxu2(cw1.x, cw1.y), __vmaxu2(cw1.z, cw1.w)));
+            const uint32_t c16all = max(m8 & 0xFFFFu, m8 >> 16);
+            if (cm * invT + ghi[noise_bound_index(c16all)] >= thr && cm > -INFINITY) {
+#pragma unroll
+              for (int sg = 0; sg < 4; ++sg) {
+                const uint4& cw = sg < 2 ? cw0 : cw1;
+                const uint32_t wa = (sg & 1) ? cw.z : cw.x, wb = (sg & 1) ? cw.w : cw.y;
+                const uint32_t m2 = __vmaxu2(wa, wb);
+                const uint32_t c16m = max(m2 & 0xFFFFu, m2 >> 16);
+                if (gmax[sg] * invT + ghi[noise_bound_index(c16m)] >= thr && gmax[sg] > -INFINITY) {
+#pragma unroll
+                  for (int i = 4 * sg; i < 4 * sg + 4; ++i) {
+                    const uint32_t word = word_of(i < 8 ? cw0 : cw1, (i & 7) >> 1);
+                    const uint32_t c16 = (word >> (16 * (i & 1))) & 0xFFFFu;
+                    mkK |= (uint32_t)(acc[i] * invT + ghi[noise_bound_index(c16)] >= thr && acc[i] > -INFINITY) << i;
+                  }
+                }
+              }
+            }
+          }
+          uint32_t mk = mkK | mkL;
+#pragma unroll 1
+          while (mk) {   // rare: hand the token to the selector warp of this row
+            const int i = __ffs(mk) - 1;
+            mk &= mk - 1;
+            const uint32_t kind = ((mkL >> i) & 1u) * KIND_TOP | ((mkK >> i) & 1u) * KIND_KEY;
+            const uint32_t c16 = (pick8(cw0, cw1, i >> 1) >> (16 * (i & 1))) & 0xFFFFu;
+            const unsigned idx = atomicAdd(sh.q_tail + sel, 1u);
+            uint32_t spin = 0;
+            while ((int)(idx - sh.q_head[sel]) >= QCAP) {   // queue full: the selector is behind
+              if (*s_abort) break;
+              if (++spin > wait_limit) { *s_abort = 1; if (a.err) atomicExch(a.err, 1); break; }
+              __nanosleep(64);
+            }
+            uint4* slot = sh.q + sel * QCAP + (idx & (QCAP - 1));
+            slot->x = (uint32_t)(v0 + i); slot->y = __float_as_uint(pick16(acc, i));
+            slot->z = ztag | (kind << 12) | (c16 << 16);
+            __threadfence_block();
+            *reinterpret_cast<volatile uint32_t*>(&slot->w) = idx + 1u;   // tag: the entry is complete
           }
         }
-        if (dry) continue;
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(t_empty + tb);
-        if (nb < 10 && g == 0) DBG(8 + warp * 6 + 1 + (nb >= 1 ? 2 : 0) + (nb >= 8 ? 2 : 0));
       }
-      if (alive && active) {
-        const int gslot = R > 1 ? row : g * 128 + row;
-        st.store(a.rec + ((size_t)(tile * MMA_S + s) * a.cap + gslot) * rw, dec_f(s_thr[prow]), dec_f(s_thr[128 + prow]));
-      }
-      if (lane == 0) atomicAdd((int*)s_done, 1);   // one tick per warp per group
-    }
-    if (!alive && lane == 0) atomicAdd((int*)s_done, 1 << 20);   // gave up: release the refresh warp
-  } else if (warp == EPI_WARPS + 1) {
-    // ======================= bounds-refresh warp ====================================================
-    // keeps the shared-memory copies of every row's launch-wide pruning bounds current, so that the
-    // epilogue threads never wait on those (contended) global words
-    for (int g = 0; g < ngroups; ++g) {
-      const int per = R > 1 ? 128 / R : 128;
-      for (uint32_t spin = 0; spin < WAIT_LIMIT; ++spin) {
+      // this piece's sums; the row's record is put together when the group is over
+      *reinterpret_cast<float4*>(s_part + ((size_t)s * 128 + row) * 4) = make_float4(m, s0, sT, 0.f);
+      __threadfence_block();
+      __syncwarp();
+      if (lane == 0) atomicAdd((int*)s_done, alive ? 1 : (1 << 20));   // one tick per warp per group (a large one releases the others after a failed wait)
+    } else if (warp == W_REFRESH) {
+      // ======================= bounds-refresh warp ====================================================
+      // keeps the shared-memory copies of every row's launch-wide pruning bounds current, so that the
+      // other warps never wait on those (contended) global words
+      for (uint32_t spin = 0; spin < wait_limit; ++spin) {
         if (*s_done >= (g + 1) * EPI_WARPS || *s_abort) break;
         // (1) This CTA condenses the slots of the parents it is responsible for (parent p belongs to tile
         // p mod ntiles) into two words per parent; (2) every CTA reads the condensed words of its rows.
-        // Only one CTA per parent reads the slot lines, which every piece of the launch is hitting with
+        // Only one CTA per parent reads the slot lines, which the whole launch is hitting with
         // atomics.  The loads of both steps are issued together: one memory round trip per pass.
         const int p_lo = R > 1 ? 0 : g * 128, p_hi = min(P, p_lo + per);
         const int nt = a.ntiles;
@@ -284,42 +476,115 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int rr = lane + 32 * k, p = R > 1 ? rr : g * 128 + rr;
-          if (rr < per && p < P) { s_thr[(g & 1) * 256 + rr] = rL[k]; s_thr[(g & 1) * 256 + 128 + rr] = rK[k]; }
+          if (rr < per && p < P) { s_thr[pbase + rr] = rL[k]; s_thr[pbase + 128 + rr] = rK[k]; }
         }
-        if (spin >= 24u) __nanosleep(500);   // poll flat out while the launch warms up, then back off
+        if (spin >= 48u) __nanosleep(500);   // poll flat out while the launch warms up, then back off
       }
       __syncwarp();
-    }
-  } else if (warp == EPI_WARPS && lane == 0) {
-    // ======================= MMA issuer ===========================================================
-    const uint32_t ws_addr = smem_u32(Ws), as_addr = smem_u32(As);
-    bool alive = true;
-    for (int g = 0; g < ngroups && alive; ++g) {
-      if (!mbar_wait(a_full, g & 1, s_abort, a.err)) break;
-      tc_fence_after();
-      for (int nb = 0; nb < nblk; ++nb) {
-        const int it = g * nblk + nb, tb = it % NBUF, u = it / NBUF;
-        if (u >= 1) {
-          if (!mbar_wait(t_empty + tb, (u - 1) & 1, s_abort, a.err)) { alive = false; break; }
-          tc_fence_after();
+    } else if (warp >= W_SEL) {
+      // ======================= selector warps ==========================================================
+      const int sel = warp - W_SEL;
+      unsigned head = sh.q_head[sel];
+      const int done_target = (g + 1) * EPI_WARPS;
+      for (uint32_t spin = 0; spin < wait_limit; ++spin) {
+        if (*s_abort) break;
+        const bool finished = *s_done >= done_target;   // read before the tail: pushes precede the tick
+        const unsigned tail = *reinterpret_cast<volatile unsigned*>(sh.q_tail + sel);
+        const int avail = (int)(tail - head);
+        if (avail <= 0) {
+          if (finished) break;
+          __nanosleep(100);
+          continue;
         }
-        if (use_tma && g == 0) {
-          if (!mbar_wait(w_full + nb, 0, s_abort, a.err)) { alive = false; break; }
+        spin = 0;
+        const int n = min(avail, 32);
+        uint4 e = make_uint4(0u, 0u, 0u, 0u);
+        bool have = false;
+        if (lane < n) {
+          uint4* slot = sh.q + sel * QCAP + ((head + lane) & (QCAP - 1));
+          uint32_t w = 0;
+          for (uint32_t t = 0; t < wait_limit; ++t) {   // the producer writes right after claiming: a few cycles
+            w = *reinterpret_cast<volatile uint32_t*>(&slot->w);
+            if (w == head + lane + 1u || *s_abort) break;
+          }
+          have = (w == head + lane + 1u);
+          __threadfence_block();
+          if (have) { e.x = slot->x; e.y = slot->y; e.z = slot->z; }
         }
-        const int n = (tlen - nb * BLK_N > 64) ? 128 : 64;
-        const uint32_t idesc = instr_desc(n);
-        const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
-        for (int ks = 0; ks < rp / 16; ++ks) {
-          const uint64_t adesc = smem_desc(as_addr + (uint32_t)(ks >> 2) * a_slab_bytes + (uint32_t)(ks & 3) * 32u, 16u, 1024u);
-          const uint64_t bdesc = smem_desc(ws_addr + (uint32_t)(2 * nb) * slab_bytes + (uint32_t)ks * 2048u, slab_bytes, 1024u);
-          mma_bf16(d_tmem, adesc, bdesc, idesc, ks > 0 ? 1u : 0u);
+        __threadfence_block();
+        __syncwarp();
+        head += (unsigned)n;
+        if (lane == 0) sh.q_head[sel] = head;   // the slots may be reused
+        // candidates of one row are inserted one after the other (lanes of a row take turns)
+        const unsigned peers = __match_any_sync(0xFFFFFFFFu, have ? (int)(e.z & 0xFFu) : -1 - lane);
+        const int turn = __popc(peers & ((1u << lane) - 1u));
+        const int turns = __reduce_max_sync(0xFFFFFFFFu, have ? turn + 1 : 0);
+        for (int t = 0; t < turns; ++t) {
+          if (have && turn == t) select_candidate(a, sh, e, ghi, invT, K, tile, R, g, s_thr, pbase, true);
+          __syncwarp();
         }
-        mma_commit(t_full + tb);
+      }
+    } else if (warp == W_MMA && lane == 0) {
+      // ======================= MMA issuer ===========================================================
+      const uint32_t ws_addr = smem_u32(Ws), as_addr = smem_u32(As);
+      if (mbar_wait(a_full, g & 1, s_abort, a.err, wait_limit)) {
+        tc_fence_after();
+        for (int nb = 0; nb < nblk; ++nb) {
+          const int it = g * nblk + nb, tb = it % NBUF, u = it / NBUF;
+          if (u >= 1) {
+            if (!mbar_wait(t_empty + tb, (u - 1) & 1, s_abort, a.err, wait_limit)) break;
+            tc_fence_after();
+          }
+          if (use_tma && g == 0) {
+            if (!mbar_wait(w_full + nb, 0, s_abort, a.err, wait_limit)) break;
+          }
+          const int n = (tlen - nb * BLK_N > 64) ? 128 : 64;
+          const uint32_t idesc = instr_desc(n);
+          const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
+          for (int ks = 0; ks < rp / 16; ++ks) {
+            const uint64_t adesc = smem_desc(as_addr + (uint32_t)(ks >> 2) * a_slab_bytes + (uint32_t)(ks & 3) * 32u, 16u, 1024u);
+            const uint64_t bdesc = smem_desc(ws_addr + (uint32_t)(2 * nb) * slab_bytes + (uint32_t)ks * 2048u, slab_bytes, 1024u);
+            mma_bf16(d_tmem, adesc, bdesc, idesc, ks > 0 ? 1u : 0u);
+          }
+          mma_commit(t_full + tb);
+        }
       }
     }
+    // ---- the group is over: one record per row -----------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (*s_abort) break;
+    if (tid < 128) {
+      const int row = tid;
+      const int p = R > 1 ? row % per : g * 128 + row;
+      if (p < P) {
+        // the splits' (max, sums) in split order: the same bits on every run
+        float m = -INFINITY, s0 = 0.f, sT = 0.f;
+#pragma unroll
+        for (int s = 0; s < EPI_S; ++s) {
+          const float4 h = *reinterpret_cast<const float4*>(s_part + ((size_t)s * 128 + row) * 4);
+          if (h.x == -INFINITY) continue;
+          if (h.x > m) { const float d = m - h.x; s0 *= __expf(d); sT *= __expf(d * invT); m = h.x; }
+          const float d = h.x - m;
+          s0 += h.y * __expf(d); sT += h.z * __expf(d * invT);
+        }
+        const int prow = pbase + (R > 1 ? row % per : row);
+        const float gL = dec_f(s_thr[prow]), gK = dec_f(s_thr[128 + prow]);
+        const float* L = sh.lists + (size_t)row * 5 * K;
+        const int* Li = reinterpret_cast<const int*>(L);
+        const int gslot = R > 1 ? row : g * 128 + row;
+        float* rec = a.rec + ((size_t)tile * a.cap + gslot) * rw;
+        int* reci = reinterpret_cast<int*>(rec) + 4;   // the lists go out as the bits they are (two of the five hold tokens)
+        int nt = 0, nk = 0;
+        for (int j = 0; j < 5 * K; ++j) reci[j] = Li[j];
+        for (int j = 0; j < K; ++j) { nt += (Li[K + j] >= 0 && L[j] >= gL); nk += (Li[3 * K + j] >= 0 && L[2 * K + j] >= gK); }
+        *reinterpret_cast<float4*>(rec) = make_float4(m, s0, sT, __int_as_float(nt | (nk << 8)));
+      }
+    }
+    __syncthreads();
   }
   // ---- tear-down -----------------------------------------------------------------------------------
-  if (warp == 0) DBG(5);
   if (use_tma && tid == 0 && ((*s_abort && (early_w || P > 0)) || (P <= 0 && early_w))) {
     // gave up somewhere, or nothing to score: do not leave while a bulk load may still be writing this
     // CTA's shared memory
@@ -330,24 +595,26 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) DBG(6);
-  if (warp == EPI_WARPS) {
+  if (warp == W_MMA) {
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
-static size_t mma_smem_bytes(const ts_config& c, int TV) {
+// shared memory beside the W tile: A tile, noise tables, queues, lists, bounds, partial sums, barriers
+static size_t mma_fixed_smem(const ts_config& c) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
-  return (size_t)(TV / 64) * rp * 128 + (rp / 64) * 128 * 128 + 512 * 4 + 128 + 512 * 4 + MAX_BLK * 8 + 1024;
+  const size_t K = (size_t)c.K;
+  return (rp / 64) * 128 * 128 + 512 * 4 + (size_t)NSEL * QCAP * 16 + 128 * 5 * K * 4 + 2 * 128 * 4 + 2 * EPI_S * 128 * 4 +
+         EPI_S * 128 * 16 + 512 * 4 + (1 + 2 * NBUF + MAX_BLK) * 8 + 64 + 1024;
 }
 
-// tile size for the tensor-core path: W tile + A tile + table + barriers within the shared-memory limit,
+// tile size for the tensor-core path: W tile + the rest within the shared-memory limit,
 // a whole number of waves over the SMs
 bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
-  const size_t fixed = (rp / 64) * 128 * 128 + 512 * 4 + 128 + 512 * 4 + MAX_BLK * 8 + 1024;
+  const size_t fixed = mma_fixed_smem(c);
   if ((size_t)max_smem < fixed + rp * 128) return false;
   int tv_max = (int)(((size_t)max_smem - fixed) / (rp * 2) / 64) * 64;
   if (tv_max < 64) return false;
@@ -359,24 +626,13 @@ bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out
   if (tv > tv_max) tv = tv_max;
   out->TV = tv;
   out->ntiles = (c.V + tv - 1) / tv;
-  out->smem = mma_smem_bytes(c, tv);
+  out->smem = (size_t)(tv / 64) * rp * 128 + fixed;
   return out->ntiles <= 4096;
 }
 
 cudaError_t score_mma_setup(ts_ctx* ctx) {
-  cudaError_t e = cudaFuncSetAttribute(score_mma_kernel<RegLists<8>>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(score_mma_kernel<RegLists<16>>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
+  return cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
 }
-
-#ifdef TS_DEBUG_TIMING
-extern "C" int ts_debug_timing(unsigned long long* out) {
-  const int rc = (int)cudaMemcpyFromSymbol(out, g_dbg, sizeof(g_dbg));
-  static unsigned long long zeros[148 * 64];
-  cudaMemcpyToSymbol(g_dbg, zeros, sizeof(zeros));
-  return rc;
-}
-#endif
 
 // Tensor map of W = [r][V] bf16 for boxes of 64 tokens x rp rows with the 128-byte swizzle the MMA's
 // B descriptor expects.  The encoder lives in the driver library; it is looked up through the runtime
@@ -422,9 +678,7 @@ cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t
   const int use_tma = w_tensor_map(c, a.W) ? 1 : 0;
   CUtensorMap tm;
   memcpy(&tm, c->tmapW, sizeof(tm));
-  cudaError_t e;
-  if (a.K <= 8) e = launch_kernel(score_mma_kernel<RegLists<8>>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma);
-  else e = launch_kernel(score_mma_kernel<RegLists<16>>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma);
+  const cudaError_t e = launch_kernel(score_mma_kernel, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 

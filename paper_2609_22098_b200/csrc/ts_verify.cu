@@ -21,22 +21,6 @@
 
 namespace ts {
 
-#ifdef TS_DEBUG_TIMING
-__device__ unsigned long long g_dbgw[4 * 64 * 8];
-__device__ __forceinline__ unsigned long long gtimew() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define DBGW(step, slot) do { if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 70) && (step) < 64) g_dbgw[((blockIdx.x ? 1 : 0) * 64 + (step)) * 8 + (slot)] = gtimew(); } while (0)
-extern "C" int ts_debug_timing_walk(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_dbgw, sizeof(g_dbgw)); }
-#else
-#define DBGW(step, slot) do { } while (0)
-#endif
-#ifdef TS_DEBUG_TIMING
-__device__ unsigned long long g_dbgp[64];
-#define DBGP(slot) do { if (blockIdx.x == 0 && (slot) < 64) g_dbgp[slot] = gtimew(); } while (0)
-extern "C" int ts_debug_timing_pass(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_dbgp, sizeof(g_dbgp)); }
-#else
-#define DBGP(slot) do { } while (0)
-#endif
-
 // 2^x by the hardware approximation (the library exp2f costs several times more in the hot loops here)
 __device__ __forceinline__ float fast_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 
@@ -148,6 +132,8 @@ struct VerifyArgs {
   int* wk_list; int* sc_list;         // [2][B] requests that asked for a reduction / a range rescan, by step parity
   int* ctr;                           // [0..1] reduction counts, [2..3] rescan counts (by parity), [4] unfinished requests
   int vt_TV, vt_n, max_steps;
+  uint32_t wait_limit;   // polls before a bounded wait (grid barrier, mbarrier) gives up
+  int lost_arrival;      // test switch: grid barriers expect one arrival more than will come
   int w_smem;   // 1: the kernel keeps its range of W in dynamic shared memory
 };
 
@@ -440,12 +426,17 @@ __device__ __forceinline__ void sweep_item(const SweepCtx<TIn>& c, int g0, int c
     for (int g = 0; g < NG; ++g) {   // every load of the step first: target rows, base rows
       const TIn* zp = c.Z + c.row[g0 + g] * c.V + v;
       const TIn* up = c.U + ((size_t)c.req[g0 + g] * c.D + c.dep[g0 + g]) * c.V + v;
+      const bool ldq = need_q && c.C[g0 + g] != 0.f;   // a member with C = 0 needs no proposal: its base row is not touched
       if (sizeof(TIn) == 2) {
         unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(zp)), z[g]);
-        if (need_q) unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(up)), acc[g]);
+        if (ldq) unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(up)), acc[g]);
       } else {
         const float4 x = __ldg(reinterpret_cast<const float4*>(zp)); z[g][0] = x.x; z[g][1] = x.y; z[g][2] = x.z; z[g][3] = x.w;
-        if (need_q) { const float4 y = __ldg(reinterpret_cast<const float4*>(up)); acc[g][0] = y.x; acc[g][1] = y.y; acc[g][2] = y.z; acc[g][3] = y.w; }
+        if (ldq) { const float4 y = __ldg(reinterpret_cast<const float4*>(up)); acc[g][0] = y.x; acc[g][1] = y.y; acc[g][2] = y.z; acc[g][3] = y.w; }
+      }
+      if (need_q && !ldq) {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) acc[g][i] = 0.f;
       }
     }
     if (need_q) {
@@ -513,7 +504,6 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
   const int cpr = rp / 8;                      // 16-byte chunks per A row
   const uint32_t a_slab_bytes = 128u * 128u;
   const __nv_bfloat16* Ag = reinterpret_cast<const __nv_bfloat16*>(a.A);
-  if (tid == 0) DBGP(0);
   {
     // ask L2 for this CTA's share of every request's target row and base-logit row now; the worker warps
     // come for them a few microseconds later, after the MMAs
@@ -539,7 +529,6 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
   __syncthreads();
   tc_fence_after();
   const int nblk = (tlen + WALK_BLK - 1) / WALK_BLK;
-  if (tid == 0) DBGP(1);
   if (warp < WALK_EPI) {
     const int q = warp & 3, s = warp >> 2;
     const int row = q * 32 + lane;
@@ -592,11 +581,10 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
     for (int nb = 0; nb < nblk && alive; ++nb) {
       const uint32_t it = tc.it + (uint32_t)nb, tb = it % WALK_NBUF, u = it / WALK_NBUF;
       int ok = 1;
-      if (lane == 0) ok = mbar_wait(tc.t_full + tb, u & 1, tc.s_abort, nullptr) ? 1 : 0;
+      if (lane == 0) ok = mbar_wait(tc.t_full + tb, u & 1, tc.s_abort, nullptr, a.wait_limit) ? 1 : 0;
       ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
       if (!ok) { alive = false; break; }
       tc_fence_after();
-      if (tid == 0) DBGP(4 + 2 * nb);
       const int nch = min(WALK_BLK / 16, (tlen - nb * WALK_BLK + 15) / 16);
       for (int ca = c0; ca < nch; ca += 2 * cstep) {
         const int cb = ca + cstep;
@@ -624,7 +612,6 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tc.t_empty + tb);
-      if (tid == 0) DBGP(5 + 2 * nb);
     }
     sum += sum2;
     s_part[row * 2 + s] = active ? sum : 0.f;
@@ -633,7 +620,7 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
     for (int nb = 0; nb < nblk; ++nb) {
       const uint32_t it = tc.it + (uint32_t)nb, tb = it % WALK_NBUF, u = it / WALK_NBUF;
       if (u >= 1) {
-        if (!mbar_wait(tc.t_empty + tb, (u - 1) & 1, tc.s_abort, nullptr)) break;
+        if (!mbar_wait(tc.t_empty + tb, (u - 1) & 1, tc.s_abort, nullptr, a.wait_limit)) break;
         tc_fence_after();
       }
       const int n = min(WALK_BLK, (tlen - nb * WALK_BLK + 63) / 64 * 64);   // whole 64-token slabs
@@ -645,11 +632,9 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
         mma_bf16(d_tmem, adesc, bdesc, idesc, ks > 0 ? 1u : 0u);
       }
       mma_commit(tc.t_full + tb);
-      DBGP(30 + nb);
     }
   }
   tc.it += (uint32_t)nblk;
-  if (tid == 0) DBGP(2);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -660,7 +645,6 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
     a.part[(size_t)sb_req[tid] * a.vt_n + blockIdx.x] = t;
   }
   __syncthreads();
-  if (tid == 0) DBGP(3);
   return true;
 }
 
@@ -681,6 +665,7 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
   __shared__ float sb_C[SBX], sb_zmax[SBX], sb_zlogs[SBX], sb_lseT[SBX], sb_part[MMA ? 256 : SB * 16];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned nblocks = gridDim.x;
+  const unsigned nexpect = nblocks + (a.lost_arrival ? 1u : 0u);   // arrivals a grid barrier waits for
   unsigned gen = 0;
   constexpr int VEC = Elem<TIn>::VEC;
   const bool vec_ok = (a.V % VEC) == 0;
@@ -760,7 +745,7 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
     __syncthreads();
   }
   __threadfence();
-  if (!grid_barrier(a.barrier, nblocks, gen)) return false;
+  if (!grid_barrier(a.barrier, nexpect, gen, a.wait_limit)) return false;
   // requests rejected at set-up leave the count of unfinished ones
   for (int b = blockIdx.x; b < a.B; b += nblocks)
     if (tid == 0 && a.state[b].need == 3) atomicSub(a.ctr + 4, 1);
@@ -770,13 +755,10 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
   int stage = 0;
   for (int step = 0; step < a.max_steps; ++step) {
     const int par = step & 1;
-    DBGW(step, 0);
     // ---- phase A: scalar walks of the requests this CTA owns, one warp each ----------------------
     for (int b = blockIdx.x + warp * (int)nblocks; b < a.B; b += (WT / 32) * (int)nblocks) advance<TIn>(a, b, lane, par, stage > 0);
     if (stage == 2) return true;
-    DBGW(step, 1);
-    if (!grid_barrier(a.barrier, nblocks, gen)) return false;
-    DBGW(step, 2);
+    if (!grid_barrier(a.barrier, nexpect, gen, a.wait_limit)) return false;
     // ---- phase B: vocabulary work requested by the walks -----------------------------------------
     const int nwk = __ldcg(a.ctr + par), nsc = __ldcg(a.ctr + 2 + par), left = __ldcg(a.ctr + 4);
     if (blockIdx.x == 0 && tid < 2) a.ctr[2 * tid + (par ^ 1)] = 0;   // next step's counters
@@ -788,7 +770,7 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
           const VerifyState* st = a.state + b;
           const int v = st->row_node;
           const int64_t row = a.z_row_off[b] + v + 1;
-          sb_req[tid] = b; sb_row[tid] = row; sb_dep[tid] = v < 0 ? 0 : a.depth[(size_t)b * N + v];
+          sb_req[tid] = b; sb_row[tid] = row; sb_dep[tid] = v < 0 ? 0 : min(a.depth[(size_t)b * N + v], a.D - 1);   // a leaf at depth D asks only for its target row (C = 0): keep the base-row index inside U
           sb_tok[tid] = v < 0 ? a.anchor[b] : a.tok[(size_t)b * N + v];
           sb_C[tid] = (float)st->passC; sb_zmax[tid] = a.z_max[row]; sb_zlogs[tid] = a.z_logs[row];
           sb_lseT[tid] = a.node_lseT[(size_t)b * (N + 1) + v + 1];
@@ -815,7 +797,7 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
           const VerifyState* st = a.state + b;
           const int v = st->row_node;
           const int64_t row = a.z_row_off[b] + v + 1;
-          sb_req[tid] = b; sb_row[tid] = row; sb_dep[tid] = v < 0 ? 0 : a.depth[(size_t)b * N + v];
+          sb_req[tid] = b; sb_row[tid] = row; sb_dep[tid] = v < 0 ? 0 : min(a.depth[(size_t)b * N + v], a.D - 1);   // a leaf at depth D asks only for its target row (C = 0): keep the base-row index inside U
           sb_tok[tid] = v < 0 ? a.anchor[b] : a.tok[(size_t)b * N + v];
           sb_C[tid] = (float)st->passC; sb_zmax[tid] = a.z_max[row]; sb_zlogs[tid] = a.z_logs[row];
           sb_lseT[tid] = a.node_lseT[(size_t)b * (N + 1) + v + 1];
@@ -857,7 +839,7 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
         const VerifyState* st = a.state + b;
         const int v = st->row_node;
         const int64_t row = a.z_row_off[b] + v + 1;
-        s_req[tid] = b; s_node[tid] = v; s_dep[tid] = v < 0 ? 0 : a.depth[(size_t)b * N + v];
+        s_req[tid] = b; s_node[tid] = v; s_dep[tid] = v < 0 ? 0 : min(a.depth[(size_t)b * N + v], a.D - 1);
         s_C[tid] = (float)st->passC; s_zmax[tid] = a.z_max[row]; s_zlogs[tid] = a.z_logs[row];
         s_lseT[tid] = a.node_lseT[(size_t)b * (N + 1) + v + 1];
       }
@@ -924,7 +906,6 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
       }
       __syncthreads();
     }
-    DBGW(step, 3);
     // range rescans for bonus tokens that fall into this CTA's range: the residual of every token of
     // the range is evaluated once (tokens dealt round-robin to the threads: row i of the range holds
     // tokens i*WT .. i*WT+WT-1), then prefix sums in token order locate the crossing
@@ -1008,10 +989,7 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
       __syncthreads();
     }
     __threadfence();
-    DBGW(step, 4);
-    if (!grid_barrier(a.barrier, nblocks, gen)) return false;
-    DBGW(step, 5);
-    if (threadIdx.x == 0 && blockIdx.x == 0 && step < 64) { DBGW(step, 6); }
+    if (!grid_barrier(a.barrier, nexpect, gen, a.wait_limit)) return false;
     if (stage == 1) stage = 2;
     else if (left == 0 && nwk == 0) stage = 1;   // uniform over the grid: both were read after the step's first barrier
   }
@@ -1081,7 +1059,7 @@ __global__ void __launch_bounds__(WT, 1) verify_walk_kernel(const VerifyArgs a, 
   if (use_tma) {
     // the whole range must have landed before anything reads it (the rescans read it with plain loads)
     if (tid == 0)
-      for (int nb = 0; nb < nblk; ++nb) if (!mbar_wait(w_full + nb, 0, tc.s_abort, nullptr)) break;
+      for (int nb = 0; nb < nblk; ++nb) if (!mbar_wait(w_full + nb, 0, tc.s_abort, nullptr, a.wait_limit)) break;
     __syncthreads();
     ok = *tc.s_abort == 0;
     if (!ok && tid == 0) atomicExch(a.barrier + 1, 1u);
@@ -1162,6 +1140,7 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
   a.edge_px = (double*)(ws + L.vf_edge); a.edge_qx = a.edge_px + (size_t)B * c.Nmax; a.edge_u = a.edge_qx + (size_t)B * c.Nmax;
   a.wk_list = (int*)(ws + L.vf_lists); a.sc_list = a.wk_list + 2 * (size_t)B; a.ctr = a.sc_list + 2 * (size_t)B;
   a.vt_TV = ctx->vt_TV; a.vt_n = ctx->vt_n; a.max_steps = 2 * (c.Nmax + c.D) + 10;
+  a.wait_limit = ctx->wait_limit; a.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
 
   const int max_rows = B * (c.Nmax + 1);
   int grid_rows = max_rows < 8 * ctx->num_sms ? max_rows : 8 * ctx->num_sms;

@@ -25,9 +25,9 @@ def make_oracle(wl, table):
                          calib_table=None if table is None else table.numpy().astype(np.float64))
 
 
-def make_gpu(wl, table, max_batch):
+def make_gpu(wl, table, max_batch, test_mode=0):
     return TreeSpark(wl.V, wl.D, wl.r, wl.K, wl.Nmax, max_batch, dtype=wl.torch_dtype, calib_mode=wl.calib_mode,
-                     calib_table=table)
+                     calib_table=table, test_mode=test_mode)
 
 
 def close(a, b, rtol=RTOL, atol=ATOL):

@@ -160,15 +160,15 @@ def test_back_to_back_rounds_reproduce_bitwise():
             assert torch.equal(verdict["acc_tok"].cpu()[b, :L], v0["acc_tok"][b, :L]), (i, b)
 
 
-@pytest.mark.parametrize("env", ["TS_FORCE_FMA", "TS_NO_TMA"])
-def test_alternative_kernel_paths_match_oracle(env, monkeypatch):
-    """bf16 inputs on the fp32-FMA kernels, and the tensor-core kernels with W staged by plain loads (the
-    path taken when no tensor map can be encoded): both are chosen when the context is created."""
-    monkeypatch.setenv(env, "1")
+@pytest.mark.parametrize("mode", ["TEST_FORCE_FMA", "TEST_NO_TMA", "TEST_NO_FEW", "TEST_NO_SEED"])
+def test_alternative_kernel_paths_match_oracle(mode):
+    """bf16 inputs on the fp32-FMA kernels; the tensor-core kernels with W staged by plain loads (the path
+    taken when no tensor map can be encoded); every level on the tile kernel; the tile kernel without seeded
+    bounds (the path of vocabularies with fewer pieces than bound slots): chosen by the library's test switches."""
+    from paper_2609_22098_b200 import binding
     wl = small("serve32", V=20000, B=5)
     rnd = Round(wl, seed=77)
-    ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
-    monkeypatch.delenv(env)
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B, test_mode=getattr(binding, mode))
     orc = make_oracle(wl, rnd.table)
     for T in (0.0, 1.0):
         st = check_round(ts, orc, rnd, T, round_seed=900)
