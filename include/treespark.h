@@ -91,7 +91,7 @@ int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags);
  *   TS_TEST_FORCE_FMA     bf16 inputs run on the fp32 fused-multiply-add kernels (no tensor cores)
  *   TS_TEST_NO_TMA        the tensor-core kernels stage W with plain loads (no tensor map)
  *   TS_TEST_NO_FEW        levels with few parents run on the tile kernel too
- *   TS_TEST_NO_SEED       the tensor-core scoring kernel starts without seeded pruning bounds
+ *   TS_TEST_NO_SEED       the tensor-core scoring kernel runs without seed bounds (no seed kernel ahead of it)
  *   TS_TEST_SHORT_WAITS   bounded waits give up after 4096 polls instead of 2^22
  *   TS_TEST_LOST_ARRIVAL  the walk's grid barriers and the scoring kernel's operand barrier expect one
  *                         arrival more than will come: the waits run out, the kernels return, and the

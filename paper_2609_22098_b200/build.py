@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtreespark.so")
-SOURCES = ["ts_api.cu", "ts_score.cu", "ts_score_mma.cu", "ts_score_few.cu", "ts_expand.cu", "ts_verify.cu", "ts_allocate.cu", "ts_calib.cu", "ts_attn_inputs.cu",
+SOURCES = ["ts_api.cu", "ts_score.cu", "ts_score_mma.cu", "ts_seed.cu", "ts_score_few.cu", "ts_expand.cu", "ts_verify.cu", "ts_allocate.cu", "ts_calib.cu", "ts_attn_inputs.cu",
            "ts_noalloc.cu"]
 
 

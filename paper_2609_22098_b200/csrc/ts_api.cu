@@ -162,7 +162,7 @@ extern "C" size_t ts_workspace_bytes(const ts_ctx* ctx, int32_t batch) {
 
 static const char* kKernelNames[K_COUNT] = {"expand_init", "score_tile", "score_merge", "expand_level", "expand_finalize",
                                             "zrow_stats", "verify_greedy", "verify_walk", "verify_check", "score_few", "allocate_select", "allocate_cut",
-                                            "calib_accumulate", "calib_refit", "attention_inputs"};
+                                            "calib_accumulate", "calib_refit", "attention_inputs", "score_seed"};
 
 extern "C" const char* ts_kernel_name(int32_t id) { return (id >= 0 && id < K_COUNT) ? kKernelNames[id] : nullptr; }
 

@@ -26,6 +26,10 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 // these words with atomicMax in the launch's first microseconds; packed together they queue up on a
 // handful of L2 lines (measured: a third of the scoring launch at stride 1).
 constexpr int SLOT_STRIDE = 32;
+// Seed kernel: a parent's base-logit row is swept by up to SEED_PARTS_MAX CTAs when there are few parents;
+// the parts of at most SEED_SPLIT_PARENTS parents meet in a scratch of NSEED_MAX candidates per part.
+constexpr int SEED_PARTS_MAX = 16, SEED_SPLIT_PARENTS = 256, NSEED_MAX = 32;
+constexpr size_t SEED_CAND_WORDS = (size_t)SEED_SPLIT_PARENTS * SEED_PARTS_MAX * NSEED_MAX * 2;
 constexpr int FEW_MAX = 8;           // levels with at most this many parents go to the few-parents scoring kernel
 constexpr int SCORE_THREADS = 128;   // one parent per thread; every thread scans the CTA's whole tile
 constexpr int CHUNK = 16;            // tokens per coarse generator call
@@ -89,6 +93,7 @@ struct WsLayout {
   // level parent lists (two, alternating) [Pcap]
   size_t lst_req[2], lst_depth[2], lst_token[2], lst_hash[2], lst_slot[2];
   size_t lvl_count;      // int[DMAX + 2]
+  size_t utop;           // uint2[B][D][ntiles]: best base logit (value, token) of every vocabulary tile of every row
   // per-request pool, [B][N]
   size_t pl_alive, pl_depth, pl_parent, pl_sib, pl_tok, pl_lidx, pl_new, pl_logkey, pl_logS, pl_q0, pl_logqT,
       pl_lseT, pl_hash, pl_path;
@@ -152,7 +157,7 @@ __host__ inline WsLayout make_layout(const ts_ctx* ctx, int B) {
     int cap = (L.Pcap + 7) / 8 * 8;
     if (ctx->use_mma) cap = (L.Pcap + 127) / 128 * 128;
     L.rec_cap = cap;
-    L.rec = take(record_bytes(ctx, cap) + (size_t)cap * (2 + 2 * K * SLOT_STRIDE) * 4);
+    L.rec = take(record_bytes(ctx, cap) + ((size_t)cap * (4 + 2 * K * SLOT_STRIDE) + SEED_SPLIT_PARENTS + SEED_CAND_WORDS) * 4);
     L.err = take(16);
   }
   L.res_lse0 = take(P * 4); L.res_lseT = take(P * 4);
@@ -163,6 +168,7 @@ __host__ inline WsLayout make_layout(const ts_ctx* ctx, int B) {
     L.lst_hash[i] = take(P * 8); L.lst_slot[i] = take(P * 4);
   }
   L.lvl_count = take((DMAX + 2) * 4);
+  L.utop = take(b * (size_t)c.D * (size_t)ctx->tile.ntiles * 8);
   L.pl_alive = take(b * N * 4); L.pl_depth = take(b * N * 4); L.pl_parent = take(b * N * 4);
   L.pl_sib = take(b * N * 4); L.pl_tok = take(b * N * 4); L.pl_lidx = take(b * N * 4); L.pl_new = take(b * N * 4);
   L.pl_logkey = take(b * N * 8); L.pl_logS = take(b * N * 8); L.pl_q0 = take(b * N * 4);

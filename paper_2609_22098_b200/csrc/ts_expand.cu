@@ -11,6 +11,7 @@
 #include <math.h>
 
 #include "ts_internal.h"
+#include "ts_scan.cuh"
 
 namespace ts {
 
@@ -32,6 +33,9 @@ struct ExpandArgs {
   // candidates
   int *cd_valid, *cd_parent, *cd_sib, *cd_tok; double *cd_logkey, *cd_logS; float *cd_q0, *cd_logqT; int* cd_rank;
   int* status; int* err; unsigned* thr; int thr_head, thr_words;
+  unsigned* seed_cnt;   // the seed kernel's arrival counters
+  // seed bounds of the next level's parents (made by the level kernel from the scoring kernel's scouting)
+  const void *U, *A, *W; int r, ntiles, cap; uint64_t seed; const uint2* utop; unsigned* thr0;
   int calib_qT;   // ablation: the calibrator is fed the tempered conditional when T > 0
 };
 
@@ -54,6 +58,7 @@ __global__ void expand_init_kernel(ExpandArgs a) {
   // SLOT_STRIDE words apart; only the first word of each is ever used)
   for (int i = b * blockDim.x + threadIdx.x; i < a.thr_words; i += gridDim.x * blockDim.x)
     a.thr[i < a.thr_head ? i : a.thr_head + (size_t)(i - a.thr_head) * SLOT_STRIDE] = 0u;
+  if (b == 0) for (int i = threadIdx.x; i < SEED_SPLIT_PARENTS; i += blockDim.x) a.seed_cnt[i] = 0u;
   if (b >= a.B) return;
   for (int s = threadIdx.x; s < a.N; s += blockDim.x) a.pl_alive[(size_t)b * a.N + s] = 0;
   if (threadIdx.x == 0) {
@@ -81,7 +86,7 @@ __device__ __forceinline__ bool before(double ka, int da, uint64_t pa, double kb
 }
 
 // One CTA per request; level d = depth of the parents just scored.
-__global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d) {
+__global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d, int seed_next) {
   extern __shared__ __align__(16) unsigned char sm_raw[];
   __shared__ int s_cnt[2];
   __shared__ int s_base;
@@ -274,11 +279,104 @@ __global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d) 
     }
     __syncthreads();
     if (tid == 0) a.req_base[b] = s_nb;
+    int my_li = -1;
     if (par) {
       const int sl = s_new[tid];
       const int li = s_nb + off + __popc(bal & ((1u << lane) - 1u));
       a.lst_req[nxt][li] = b; a.lst_depth[nxt][li] = d + 1; a.lst_token[nxt][li] = a.pl_tok[pb + sl];
       a.lst_hash[nxt][li] = a.pl_hash[pb + sl]; a.lst_slot[nxt][li] = sl;
+      my_li = li;
+    }
+    // ---- phase 5: seed bounds of those parents (bf16 tensor-core path; see ts_seed.cu for what they are) ----
+    // The scoring launch of this level left the best base logit of every vocabulary tile of row U[b][d+1]:
+    // the warps pick 2K good tokens from those, the tokens' columns of W are staged once for the request,
+    // every (parent, token) pair is evaluated exactly by one thread, and one thread per parent takes the
+    // K-th best logit and key, less the rounding margin.
+    if (seed_next && cnt > 0) {
+      __shared__ int s_stok[NSEED_MAX], s_pli[256], s_ptok[256];
+      __shared__ float s_sval[NSEED_MAX];
+      __shared__ uint64_t s_phash[256];
+      const int r = a.r, V = a.V;
+      const int npick = max(1, min(2 * K, NSEED_MAX) / 8), NSn = 8 * npick;
+      const float invT = a.T > 0.f ? 1.f / a.T : 1.f;
+      __syncthreads();   // the Entry array in dynamic shared memory is free now
+      float* Wc = reinterpret_cast<float*>(sm_raw);            // [NSn][r]
+      float* res = Wc + (size_t)NSn * r;                        // [cnt][NSn][2]: logit, key
+      if (par) {
+        const int i = off + __popc(bal & ((1u << lane) - 1u));
+        s_pli[i] = my_li; s_ptok[i] = a.pl_tok[pb + s_new[tid]]; s_phash[i] = a.pl_hash[pb + s_new[tid]];
+      }
+      {
+        const uint2* ut = a.utop + ((size_t)b * a.D + (d + 1)) * a.ntiles;
+        float bv = -INFINITY; int bi = 0x7FFFFFFF;
+        for (int t = lane * 8 + warp; t < a.ntiles; t += blockDim.x) {   // consecutive tiles go to different warps
+          const uint2 e = __ldcg(ut + t);
+          const float v = __uint_as_float(e.x);
+          if (v > bv || (v == bv && (int)e.y < bi)) { bv = v; bi = (int)e.y; }
+        }
+        for (int i = 0; i < npick; ++i) {   // every warp hands over its npick best
+          float wv = bv; int wi = bi;
+#pragma unroll
+          for (int o2 = 16; o2 > 0; o2 >>= 1) {
+            const float ov = __shfl_xor_sync(0xFFFFFFFFu, wv, o2);
+            const int oi = __shfl_xor_sync(0xFFFFFFFFu, wi, o2);
+            if (ov > wv || (ov == wv && oi < wi)) { wv = ov; wi = oi; }
+          }
+          if (wi == bi && bv > -INFINITY) { bv = -INFINITY; bi = 0x7FFFFFFF; }
+          if (lane == 0) { s_stok[warp * npick + i] = (wv > -INFINITY && wi >= 0 && wi < V) ? wi : -1; }
+        }
+      }
+      __syncthreads();
+      const __nv_bfloat16* Wg = reinterpret_cast<const __nv_bfloat16*>(a.W);
+      const __nv_bfloat16* Ag = reinterpret_cast<const __nv_bfloat16*>(a.A);
+      const __nv_bfloat16* Urow = reinterpret_cast<const __nv_bfloat16*>(a.U) + ((size_t)b * a.D + (d + 1)) * V;
+      for (int e = tid; e < NSn * r; e += blockDim.x) {
+        const int j = e / r, k = e % r;
+        Wc[e] = s_stok[j] >= 0 ? __bfloat162float(Wg[(size_t)k * V + s_stok[j]]) : 0.f;
+      }
+      if (tid < NSn) s_sval[tid] = s_stok[tid] >= 0 ? __bfloat162float(Urow[s_stok[tid]]) : -INFINITY;
+      __syncthreads();
+      for (int e = tid; e < cnt * NSn; e += blockDim.x) {
+        const int i = e / NSn, j = e % NSn;
+        float lg = -INFINITY, key = -INFINITY;
+        const int tok = s_stok[j];
+        if (tok >= 0) {
+          const uint4* arow = reinterpret_cast<const uint4*>(Ag + (size_t)s_ptok[i] * r);   // r is a multiple of 8 on this path
+          float dot = 0.f;
+          for (int k8 = 0; k8 < r / 8; ++k8) {
+            float av[8];
+            unpack_bf16x8(__ldg(arow + k8), av);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) dot = fmaf(av[u], Wc[(size_t)j * r + k8 * 8 + u], dot);
+          }
+          lg = s_sval[j] + dot;
+          key = lg;
+          if (a.T > 0.f) {
+            const uint4 cw = stream_words(a.seed, b, s_phash[i], STREAM_GUMBEL_COARSE, (uint32_t)tok >> 3);
+            const uint4 fw = stream_words(a.seed, b, s_phash[i], STREAM_GUMBEL_FINE, (uint32_t)tok >> 3);
+            const uint32_t c16 = (word_of(cw, (tok & 7) >> 1) >> (16 * (tok & 1))) & 0xFFFFu;
+            const uint32_t f16 = (word_of(fw, (tok & 7) >> 1) >> (16 * (tok & 1))) & 0xFFFFu;
+            key = lg * invT + gumbel_from_bits((c16 << 16) | f16);
+          }
+        }
+        res[2 * e] = lg; res[2 * e + 1] = key;
+      }
+      __syncthreads();
+      for (int e = tid; e < 2 * cnt; e += blockDim.x) a.thr0[(size_t)(e & 1) * a.cap + s_pli[e >> 1]] = 0u;   // no bound unless K finite values turn up
+      __syncthreads();
+      for (int e = tid; e < 2 * cnt * NSn; e += blockDim.x) {
+        // one thread per value: the one with exactly K - 1 values before it (ties broken by place) is the K-th best
+        const int j = e % NSn, which = (e / NSn) & 1, i = e / (2 * NSn);
+        if (which == 1 && !(a.T > 0.f)) continue;
+        const float* val = res + (size_t)i * NSn * 2 + which;
+        const float mine = val[2 * j];
+        int before = 0;
+        for (int t = 0; t < NSn; ++t) before += (val[2 * t] > mine || (val[2 * t] == mine && t < j)) ? 1 : 0;
+        if (before == K - 1 && mine == mine && fabsf(mine) < INFINITY) {
+          const float margin = (2e-4f + 4e-5f * fabsf(mine)) * (which == 0 ? 1.f : fmaxf(invT, 1.f)) + (which == 0 ? 0.f : 2e-4f);
+          a.thr0[(size_t)which * a.cap + s_pli[i]] = enc_f(mine - margin);
+        }
+      }
     }
   }
 }
@@ -360,8 +458,17 @@ __global__ void __launch_bounds__(256) expand_finalize_kernel(FinalArgs a) {
 }
 
 // the level kernel ranks a request's pool and candidates out of dynamic shared memory: opt in once per context
+// dynamic shared memory of the level kernel: the ranking entries of a request's pool and candidates, later
+// reused for the seed bounds' staged W columns [2K][r] and per-pair results [Nmax][2K][2]
+size_t level_smem_bytes(const ts_config& c) {
+  const size_t entries = (size_t)(c.Nmax + c.Nmax * c.K) * sizeof(Entry);
+  const size_t ns = (size_t)(2 * c.K > NSEED_MAX ? NSEED_MAX : (2 * c.K < 8 ? 8 : 2 * c.K));
+  const size_t seeds = ns * (size_t)c.r * 4 + (size_t)c.Nmax * ns * 2 * 4;
+  return entries > seeds ? entries : seeds;
+}
+
 cudaError_t expand_setup(ts_ctx* ctx) {
-  const size_t level_smem = (size_t)(ctx->cfg.Nmax + ctx->cfg.Nmax * ctx->cfg.K) * sizeof(Entry);
+  const size_t level_smem = level_smem_bytes(ctx->cfg);
   if (level_smem <= 48 * 1024) return cudaSuccess;
   return cudaFuncSetAttribute(expand_level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)level_smem);
 }
@@ -419,22 +526,37 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   a.status = status; a.err = (int*)(ws + L.err);
   a.thr = thr_base(ctx, (float*)(ws + L.rec), L.rec_cap);
   a.thr_head = 2 * L.rec_cap; a.thr_words = a.thr_head + 2 * L.rec_cap * c.K;   // words to clear, not their span
+  a.thr0 = a.thr + 2 * (size_t)L.rec_cap + 2 * (size_t)L.rec_cap * c.K * SLOT_STRIDE;
+  a.seed_cnt = a.thr0 + 2 * (size_t)L.rec_cap;
+  a.U = U; a.A = A; a.W = W; a.r = c.r; a.ntiles = ctx->tile.ntiles; a.cap = L.rec_cap; a.seed = seed;
+  a.utop = (const uint2*)(ws + L.utop);
 
   cudaError_t e0;
   { ProfScope ps(ctx, K_INIT, st); e0 = launch_kernel(expand_init_kernel, B > 296 ? B : 296, 256, 0, st, true, a); }
   cudaError_t e = e0 != cudaSuccess ? e0 : cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(init)", e);
-  const size_t level_smem = (size_t)(c.Nmax + c.Nmax * c.K) * sizeof(Entry);   // opted into at ts_create when above 48 KB
+  const size_t level_smem = level_smem_bytes(c);   // opted into at ts_create when above 48 KB
   long long level_bound = B;   // parents a level can have at most: B at the root, K times more per level, B * Nmax overall
+  // Seed bounds of a level on the tensor-core kernel: made by the level kernel before it when that level's scoring
+  // launch scouted the rows (it does whenever it runs on the tensor-core kernel itself); by a seed launch otherwise
+  // (the root level, and the first tensor-core level after levels on the few-parents kernel).
+  const bool seeds_on = ctx->use_mma && !(ctx->test_mode & TS_TEST_NO_SEED);
+  bool scouted_prev = false;
   for (int d = 0; d < c.D; ++d) {
     const int cur = d & 1;
+    const bool on_mma = ctx->use_mma && !(ctx->few_ok && level_bound <= FEW_MAX);
+    ScoreExtras ex;
+    ex.thr0_ready = scouted_prev;
+    const bool scout = seeds_on && on_mma && d + 1 < c.D;
+    if (scout) { ex.utop = (uint2*)(ws + L.utop); ex.scout_live = a.req_npar; ex.scout_B = B; ex.scout_depth = d + 1; }
     e = launch_score(ctx, (float*)(ws + L.rec), L.rec_cap, (int*)(ws + L.err), U, A, W, 0, a.lvl_count + d,
                      a.lst_req[cur], a.lst_depth[cur], a.lst_token[cur],
                      a.lst_hash[cur], T, seed, res_lse0, res_lseT, res_top_tok, res_top_logit, res_draw_tok,
-                     res_draw_logit, st, /*pdl=*/true, d > 0 ? a.lvl_count + d - 1 : nullptr, (int)level_bound);
+                     res_draw_logit, st, /*pdl=*/true, d > 0 ? a.lvl_count + d - 1 : nullptr, (int)level_bound, &ex);
     level_bound = level_bound * c.K < (long long)B * c.Nmax ? level_bound * c.K : (long long)B * c.Nmax;
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(score)", e);
-    { ProfScope ps(ctx, K_LEVEL, st); e = launch_kernel(expand_level_kernel, B, 256, level_smem, st, true, a, d); }
+    { ProfScope ps(ctx, K_LEVEL, st); e = launch_kernel(expand_level_kernel, B, 256, level_smem, st, true, a, d, scout ? 1 : 0); }
+    scouted_prev = scout;
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(level)", e);
   }

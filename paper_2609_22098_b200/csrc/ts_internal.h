@@ -13,6 +13,7 @@ int32_t set_cuda_error(const char* where, cudaError_t e);
 cudaError_t score_setup(ts_ctx* ctx);
 cudaError_t verify_setup(ts_ctx* ctx);
 cudaError_t expand_setup(ts_ctx* ctx);
+size_t level_smem_bytes(const ts_config& c);
 
 struct ScoreArgs {
   const void *U, *A, *W;
@@ -27,16 +28,23 @@ struct ScoreArgs {
   float* rec; int* err;
   unsigned* thr;    // [2][cap]: launch-wide lower bounds (logit, key) per parent, order-preserving encoding
   unsigned* slots;  // [2][cap][K]
+  // Scouting for the next level (expansion only; utop == nullptr: none): while its first MMAs are on their
+  // way, the tensor-core kernel finds the best base logit of its vocabulary tile in row U[b][scout_depth] of
+  // every request b < scout_B that has parents in this launch (scout_live[b] > 0), and leaves (value, token)
+  // at utop[(b * D + scout_depth) * ntiles + tile]: the next level's seed bounds are made from those.
+  const int* scout_live; int scout_B, scout_depth; uint2* utop;
+  unsigned* seed_cnt;    // [SEED_SPLIT_PARENTS] arrival counters of the seed kernel (zero between launches)
+  unsigned* seed_cand;   // [SEED_SPLIT_PARENTS][SEED_PARTS_MAX][NSEED_MAX][2] candidates (value, token) of the parts
+  unsigned* thr0;   // [2][cap]: seed bounds (logit, key) per parent, written ahead of the launch; nullptr: none
   uint32_t wait_limit;   // polls before a bounded device-side wait gives up
   int lost_arrival;      // test switch: the A-tile barrier expects one arrival more than will come
-  int seed_bounds;       // 1: pieces publish an exactly evaluated token before they scan (tensor-core kernel)
 };
 
 struct MergeArgs {
   int P; const int* P_dev; int K, ntiles, cap, S, mma; float T;
   int pdl;   // host side: launch with programmatic stream serialization
   int few_ntiles;   // > 0: the level was scored by the few-parents kernel over this many tiles
-  const float* rec; unsigned* thr; unsigned* slots;
+  const float* rec; unsigned* thr; unsigned* slots; const unsigned* thr0;
   float *lse0, *lseT; int* top_tok; float* top_logit; int* draw_tok; float* draw_logit;
 };
 
@@ -51,11 +59,17 @@ size_t thr_bytes(const ts_ctx* ctx, int cap);
 // p_bound: an upper bound of *P_dev the host knows (-1: none).  A list that cannot exceed FEW_MAX parents
 // goes to the few-parents kernel where the context has one.
 // rec: record scratch of score_scratch_bytes(ctx, max parents) bytes with slot capacity cap.
+// What the expansion adds to a scoring pass: seed bounds that the level kernel already wrote (no seed launch),
+// and scouting of the next level's rows (see ScoreArgs).
+struct ScoreExtras {
+  bool thr0_ready = false;
+  const int* scout_live = nullptr; int scout_B = 0, scout_depth = -1; uint2* utop = nullptr;
+};
 cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,
                          const uint64_t* p_hash, float T, uint64_t seed, float* lse0, float* lseT, int* top_tok,
                          float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st,
-                         bool pdl = false, const int* P_prev_dev = nullptr, int p_bound = -1);
+                         bool pdl = false, const int* P_prev_dev = nullptr, int p_bound = -1, const ScoreExtras* extras = nullptr);
 
 // Kernel launch, optionally with programmatic stream serialization: the kernel may then start while the
 // kernel before it in the stream is still running, and must execute pdl_wait() before it touches anything
@@ -75,6 +89,8 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
 bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out);
 cudaError_t score_mma_setup(ts_ctx* ctx);
 cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st);
+// seed bounds of every parent of the list (ts_seed.cu); runs ahead of the tensor-core scoring kernel
+cudaError_t launch_seed(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st);
 // the few-parents kernel (ts_score_few.cu)
 int few_tiles(const ts_config& c);
 bool few_supported(const ts_ctx* ctx);
@@ -82,7 +98,7 @@ cudaError_t launch_score_few(const ts_ctx* ctx, const ScoreArgs& a, int p_bound,
 // encodes (or finds cached in the context) the tensor map of W for 64-token boxes; false: not available
 bool w_tensor_map(ts_ctx* ctx, const void* W);
 
-enum KernelId { K_INIT, K_SCORE, K_MERGE, K_LEVEL, K_FINAL, K_ZROWS, K_GREEDY, K_WALK, K_CHECK, K_SCORE_FEW, K_ALLOC_SELECT, K_ALLOC_CUT, K_CALIB_ACC, K_CALIB_FIT, K_ATTN_INPUTS, K_COUNT };
+enum KernelId { K_INIT, K_SCORE, K_MERGE, K_LEVEL, K_FINAL, K_ZROWS, K_GREEDY, K_WALK, K_CHECK, K_SCORE_FEW, K_ALLOC_SELECT, K_ALLOC_CUT, K_CALIB_ACC, K_CALIB_FIT, K_ATTN_INPUTS, K_SEED, K_COUNT };
 
 struct Prof {
   bool on = false;

@@ -193,7 +193,11 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
   for (int p = blockIdx.x; p < P; p += gridDim.x) {
     // final launch-wide lower bounds of this parent's K-th best logit / key: entries below cannot win
     const SharedThr gl{a.slots + (size_t)p * K * SLOT_STRIDE, 0}, gk{a.slots + ((size_t)a.cap + p) * K * SLOT_STRIDE, 0};
-    const float bL = dec_f(slots_min(gl, K)), bK = a.T > 0.f ? dec_f(slots_min(gk, K)) : -INFINITY;
+    float bL = dec_f(slots_min(gl, K)), bK = a.T > 0.f ? dec_f(slots_min(gk, K)) : -INFINITY;
+    if (a.thr0) {   // never below the parent's seed bounds
+      bL = fmaxf(bL, dec_f(__ldcg(a.thr0 + p)));
+      if (a.T > 0.f) bK = fmaxf(bK, dec_f(__ldcg(a.thr0 + (size_t)a.cap + p)));
+    }
     if (tid < 2) c_n[tid] = 0;
     __syncthreads();
     float m = -INFINITY, s0 = 0.f, sT = 0.f;
@@ -321,29 +325,33 @@ size_t score_scratch_bytes(const ts_ctx* ctx, int P, int* cap_out) {
   if (ctx->use_mma) { cap = (P + 127) / 128 * 128; if (cap < 128) cap = 128; }
   if (cap_out) *cap_out = cap;
   // records, then the pruning state: 2 threshold words and 2K slot words per slot of capacity
-  return record_bytes(ctx, cap) + align_up((size_t)cap * (2 + 2 * (size_t)ctx->cfg.K * SLOT_STRIDE) * sizeof(unsigned), 256);
+  return record_bytes(ctx, cap) + align_up(((size_t)cap * (4 + 2 * (size_t)ctx->cfg.K * SLOT_STRIDE) + SEED_SPLIT_PARENTS + SEED_CAND_WORDS) * sizeof(unsigned), 256);
 }
 
 unsigned* thr_base(const ts_ctx* ctx, float* rec, int cap) {
   return (unsigned*)((char*)rec + record_bytes(ctx, cap));
 }
 
-size_t thr_bytes(const ts_ctx* ctx, int cap) { return (size_t)cap * (2 + 2 * (size_t)ctx->cfg.K * SLOT_STRIDE) * sizeof(unsigned); }
+// thresholds [2][cap], slots [2][cap][K] (one 128-byte line each), seed bounds [2][cap], the seed kernel's arrival
+// counters [SEED_SPLIT_PARENTS]: the part of the pruning state that must be zero before a launch (the seed
+// kernel's candidate scratch follows it and needs no clearing)
+size_t thr_bytes(const ts_ctx* ctx, int cap) { return ((size_t)cap * (4 + 2 * (size_t)ctx->cfg.K * SLOT_STRIDE) + SEED_SPLIT_PARENTS) * sizeof(unsigned); }
 
 cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,
                          const uint64_t* p_hash, float T, uint64_t seed, float* lse0, float* lseT, int* top_tok,
                          float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st, bool pdl, const int* P_prev_dev,
-                         int p_bound) {
+                         int p_bound, const ScoreExtras* extras) {
   const ts_config& c = ctx->cfg;
   ScoreArgs a{};
   a.pdl = pdl ? 1 : 0; a.P_prev_dev = P_prev_dev;
   a.U = U; a.A = A; a.W = W; a.V = c.V; a.D = c.D; a.r = c.r; a.K = c.K; a.P = P; a.P_dev = P_dev;
   a.p_req = p_req; a.p_depth = p_depth; a.p_token = p_token; a.p_hash = p_hash; a.T = T; a.seed = seed;
   a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.cap = cap; a.S = 1; a.rec = rec; a.err = err;
-  a.wait_limit = ctx->wait_limit; a.seed_bounds = (ctx->test_mode & TS_TEST_NO_SEED) ? 0 : 1;
+  a.wait_limit = ctx->wait_limit;
   a.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
   a.thr = thr_base(ctx, rec, cap); a.slots = a.thr + 2 * (size_t)cap;
+  a.thr0 = nullptr;
   cudaError_t e = cudaSuccess;
   // Which kernel scores the level: the few-parents kernel when the host knows that the list cannot hold
   // more than FEW_MAX parents (its own P, or a bound of the device-side count), the tile kernel otherwise.
@@ -351,6 +359,20 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
   const bool run_few = ctx->use_mma && ctx->few_ok && bound >= 0 && bound <= FEW_MAX;
   const bool run_tile = !run_few;
   a.few = run_few ? 1 : 0;
+  if (run_tile && ctx->use_mma && !(ctx->test_mode & TS_TEST_NO_SEED)) {
+    // seed bounds first: exact values of the tokens with the largest base logits of every parent's row
+    a.thr0 = a.slots + 2 * (size_t)cap * c.K * SLOT_STRIDE;
+    a.seed_cnt = a.thr0 + 2 * (size_t)cap;
+    a.seed_cand = a.seed_cnt + SEED_SPLIT_PARENTS;
+    if (!(extras && extras->thr0_ready)) {   // (an expansion's level kernel writes them for the level after it)
+      ProfScope ps(ctx, K_SEED, st);
+      e = launch_seed(ctx, a, st);
+      if (e != cudaSuccess) return e;
+    }
+    if (extras && extras->utop) {
+      a.utop = extras->utop; a.scout_live = extras->scout_live; a.scout_B = extras->scout_B; a.scout_depth = extras->scout_depth;
+    }
+  }
   if (run_tile) {
     ProfScope ps(ctx, K_SCORE, st);
     if (ctx->use_mma) {
@@ -375,7 +397,7 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
   m.pdl = a.pdl;
   m.few_ntiles = run_few ? few_tiles(c) : 0;
   m.P = P; m.P_dev = P_dev; m.K = c.K; m.ntiles = a.ntiles; m.cap = cap; m.S = a.S; m.mma = ctx->use_mma ? 1 : 0; m.T = T;
-  m.rec = rec; m.thr = a.thr; m.slots = a.slots;
+  m.rec = rec; m.thr = a.thr; m.slots = a.slots; m.thr0 = a.thr0;
   m.lse0 = lse0; m.lseT = lseT; m.top_tok = top_tok; m.top_logit = top_logit; m.draw_tok = draw_tok; m.draw_logit = draw_logit;
   int blocks = P_dev ? cap : P;
   if (blocks > 2 * ctx->num_sms) blocks = 2 * ctx->num_sms;   // parents beyond that are looped over

@@ -13,17 +13,17 @@
 // (rp = r rounded up to 64, padding zero-filled).
 //
 // Warps 0..15 scan: warp w reads the tensor-memory lanes 32*(w%4).. (its quarter of the 128 parent
-// rows) and, of the tile's 16-token chunks, those of column split w/4.  When a level has few parents
-// the rows are replicated R = 2 or 4 times over the quarters and the copies split the chunks too:
-// chunk cg belongs to replica cg % R and split (cg / R) % 4.  A scanning thread keeps only the running
+// rows) and, of the tile's 64-token blocks, those of split w/4 (block nb belongs to split nb % 4).  When
+// a level has few parents the rows are replicated R = 2 or 4 times over the quarters and the copies
+// split a block's four 16-token chunks: chunk c belongs to replica c % R.  A scanning thread keeps only the running
 // (max, sums) of its row; a token that can still be among the row's K best (its logit, or the upper
 // bound of its sampling key given the leading 16 bits of its uniform, reaches the row's current bound)
 // is appended to a queue with a few instructions, so that the 32 rows of a warp never wait for the
 // rare, long evaluation of one of them.  Warps 18 and 19 (rows 0..63 / 64..127) drain the queues, one
 // candidate per lane: exact key (second generator call, two logarithms), insertion into the row's
 // sorted lists, publication of new bests.  Warp 16 allocates tensor memory and its lane 0 issues the
-// MMAs: per block of 128 tokens rp/16 instructions of M=128, N=128 (64 at a ragged end), K=16 into one
-// of four 128-column accumulator buffers, then a commit that arrives on that buffer's "full" barrier;
+// MMAs: per block of 64 tokens rp/16 instructions of M=128, N=64, K=16 into one of eight 64-column
+// accumulator buffers (two per split), then a commit that arrives on that buffer's "full" barrier;
 // scanning warps arrive on its "empty" barrier when they have drained it.  Warp 17 keeps shared-memory
 // copies of the launch-wide pruning bounds of every row current.
 //
@@ -31,9 +31,9 @@
 // the pieces (tile, split, replica) whose number is j modulo K.  Pieces hold disjoint tokens, so the
 // slots hold values of K different tokens and their minimum is a lower bound of the parent's K-th best
 // value: a token strictly below it cannot be among the K best.  So that bounds exist before the scan
-// begins, every scanning thread first evaluates exactly the best-logit token of its first chunk and
-// publishes its logit and key (the seed), then waits a few microseconds (bounded) for the bounds of
-// its row to arrive.
+// begins, a kernel ahead of this one (seed_parents_kernel) evaluates for every parent the tokens with the
+// largest base logits exactly and leaves the K-th best logit and key among them, less a rounding margin,
+// as the parent's seed bounds; the bounds used here are never below those.
 //
 // Every wait is bounded: when one runs out the kernel raises an error word, skips the remaining work,
 // waits (again bounded) for bulk loads still in flight, frees its tensor memory and returns.
@@ -50,10 +50,11 @@ constexpr int W_REFRESH = EPI_WARPS + 1;
 constexpr int W_SEL = EPI_WARPS + 2;
 constexpr int NSEL = 2;                     // selector warps (rows 0..63, 64..127)
 constexpr int MMA_THREADS = (EPI_WARPS + 2 + NSEL) * 32;
-constexpr int BLK_N = 128;
-constexpr int NBUF = 4;                 // accumulator buffers of BLK_N columns in tensor memory
+constexpr int BLK_N = 64;               // tokens per block: one MMA tile, one accumulator buffer, one slab of W
+constexpr int WBLK = 128;               // tokens per bulk-load barrier of W (two slabs)
+constexpr int NBUF = 8;                 // accumulator buffers of BLK_N columns in tensor memory: two per split
 constexpr uint32_t TMEM_COLS = NBUF * BLK_N;
-constexpr int MAX_BLK = 32;             // blocks of BLK_N tokens in the largest tile (4096 tokens)
+constexpr int MAX_BLK = 32;             // W load barriers (WBLK tokens each) of the largest tile (4096 tokens)
 constexpr int QCAP = 256;               // entries per candidate queue (power of two)
 constexpr uint32_t KIND_TOP = 1u, KIND_KEY = 2u;
 
@@ -79,25 +80,6 @@ __device__ __forceinline__ float list_insert(float* v, int* t, float* aux, int K
   v[pos] = val; t[pos] = tok;
   if (aux) aux[pos] = lg;
   return v[K - 1];
-}
-
-// The seed of one piece: its first chunk's best-logit token, evaluated exactly, gives every parent a
-// lower bound of its K-th best logit and key before the scan proper begins.
-static __device__ __noinline__ void publish_seed(const float* l, int v0, float invT, bool keys, uint64_t seed, int req,
-                                                 uint64_t hash, unsigned* slotL, unsigned* slotK) {
-  float bl = l[0]; int bi = 0;
-#pragma unroll
-  for (int i = 1; i < 16; ++i) if (l[i] > bl) { bl = l[i]; bi = i; }
-  if (!(bl > -INFINITY)) return;
-  atomicMax(slotL, enc_f(bl));
-  if (keys) {
-    const int v = v0 + bi;
-    const uint4 cw = stream_words(seed, req, hash, STREAM_GUMBEL_COARSE, (uint32_t)v >> 3);
-    const uint4 fw = stream_words(seed, req, hash, STREAM_GUMBEL_FINE, (uint32_t)v >> 3);
-    const uint32_t c16 = (word_of(cw, (v & 7) >> 1) >> (16 * (v & 1))) & 0xFFFFu;
-    const uint32_t f16 = (word_of(fw, (v & 7) >> 1) >> (16 * (v & 1))) & 0xFFFFu;
-    atomicMax(slotK, enc_f(bl * invT + gumbel_from_bits((c16 << 16) | f16)));
-  }
 }
 
 // One candidate, handled by one selector lane: exact key, insertion, publication.
@@ -148,7 +130,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   const int r = a.r, rp = (r + 63) / 64 * 64, V = a.V, TV = a.TV, K = a.K;
   const int tile = blockIdx.x, t0 = tile * TV, tlen = min(TV, V - t0);
   const int nslab = TV / 64;
-  const int nblk_w = (tlen + BLK_N - 1) / BLK_N;
+  const int nblk_w = (tlen + WBLK - 1) / WBLK;
   const uint32_t slab_bytes = (uint32_t)rp * 128u;       // one 64-token slab of W
   const uint32_t a_slab_bytes = 128u * 128u;             // 128 rows x 128 B
   unsigned char* sm = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -186,7 +168,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   const bool early_w = !a.P_prev_dev || *a.P_prev_dev >= 16;
   auto issue_w = [&]() {   // one thread
     for (int nb = 0; nb < nblk_w; ++nb) {
-      const int ns = (tlen - nb * BLK_N > 64) ? 2 : 1;
+      const int ns = (tlen - nb * WBLK > 64) ? 2 : 1;
       mbar_expect_tx(w_full + nb, (uint32_t)ns * slab_bytes);
       for (int h = 0; h < ns; ++h)
         tma_load_box(Ws + (size_t)(2 * nb + h) * slab_bytes, &tmW, t0 + (2 * nb + h) * 64, 0, w_full + nb);
@@ -194,7 +176,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   };
   if (tid == 0) {
     mbar_init(a_full, EPI_WARPS * 32 + (a.lost_arrival ? 1 : 0));
-    for (int i = 0; i < NBUF; ++i) { mbar_init(t_full + i, 1); mbar_init(t_empty + i, EPI_WARPS); }
+    for (int i = 0; i < NBUF; ++i) { mbar_init(t_full + i, 1); mbar_init(t_empty + i, 4); }   // a buffer is drained by the four quarter warps of one split
     *s_abort = 0;
     *s_done = 0;
     for (int i = 0; i < NSEL; ++i) { sh.q_head[i] = 0u; sh.q_tail[i] = 0u; }
@@ -219,6 +201,15 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   }
   fill_gumbel_bounds(ghi, tid, MMA_THREADS);
   for (int i = tid; i < 512; i += MMA_THREADS) s_thr[i] = 0u;
+  auto reset_selection = [&]() {   // empty lists, no local thresholds, nothing published
+    for (int i = tid; i < 128 * 5 * K; i += MMA_THREADS) {
+      const int f = (i / K) % 5;   // fields: topv, topi, keyv, keyi, keyl
+      sh.lists[i] = (f == 0 || f == 2) ? -INFINITY : ((f == 1 || f == 3) ? __int_as_float(-1) : 0.f);
+    }
+    for (int i = tid; i < 2 * 128; i += MMA_THREADS) sh.lthr[i] = -INFINITY;
+    for (int i = tid; i < 2 * EPI_S * 128; i += MMA_THREADS) sh.best[i] = -INFINITY;
+  };
+  reset_selection();   // the first group's, here in the preamble; later groups' when they begin
   for (int i = tid; i < NSEL * QCAP; i += MMA_THREADS) sh.q[i] = make_uint4(0u, 0u, 0u, 0u);   // tag 0 = never written
   fence_async_smem();
   tc_fence_before();
@@ -230,25 +221,24 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   const int P = a.P_dev ? *a.P_dev : a.P;   // may be 0: an empty level only tears down
   if (use_tma && !early_w && P > 0 && tid == 0) issue_w();
 
-  const int R = mma_replicas(P), rsh = R == 4 ? 2 : (R == 2 ? 1 : 0);
+  const int R = mma_replicas(P);
   const int per = 128 / R;
   const int ngroups = P <= 0 ? 0 : (R > 1 ? 1 : (P + 127) / 128);
   const int nblk = (tlen + BLK_N - 1) / BLK_N;
   const float T = a.T, invT = T > 0.f ? 1.f / T : 1.f;
   const bool keys = T > 0.f;
   const int rw = rec_words(K);
-  // launch-wide bounds can form only when every one of the K slots has a piece that feeds it
-  const bool seeded = (long long)a.ntiles * EPI_S * R >= 2 * K && a.seed_bounds != 0;
 
   for (int g = 0; g < ngroups; ++g) {
     const int pbase = (g & 1) * 256;   // rows of group g use the bound buffer of parity g & 1
     // ---- per-group reset of the selection state (every thread) ---------------------------------------
-    for (int i = tid; i < 128 * 5 * K; i += MMA_THREADS) {
-      const int f = (i / K) % 5;   // fields: topv, topi, keyv, keyi, keyl
-      sh.lists[i] = (f == 0 || f == 2) ? -INFINITY : ((f == 1 || f == 3) ? __int_as_float(-1) : 0.f);
+    if (g > 0) reset_selection();
+    for (int i = tid; i < 2 * 128; i += MMA_THREADS) {
+      // the row's bounds start at its parent's seed bounds (exact values of K tokens, found before the launch)
+      const int which = i >> 7, rr = i & 127;
+      const int p = R > 1 ? rr % per : g * 128 + rr;
+      s_thr[pbase + i] = (a.thr0 && p < P && (R == 1 || rr < per)) ? __ldcg(a.thr0 + (size_t)which * a.cap + p) : 0u;
     }
-    for (int i = tid; i < 2 * 128; i += MMA_THREADS) { sh.lthr[i] = -INFINITY; s_thr[pbase + i] = 0u; }
-    for (int i = tid; i < 2 * EPI_S * 128; i += MMA_THREADS) sh.best[i] = -INFINITY;
     __syncthreads();
 
     if (warp < EPI_WARPS) {
@@ -267,6 +257,38 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       }
       fence_async_smem();
       mbar_arrive(a_full);
+      if (a.utop && g == 0) {
+        // scouting (see ScoreArgs): fills the wait for the first accumulators, and brings the rows the next
+        // level will score into L2
+        const int nvec = tlen / 8;
+        for (int b = warp; b < a.scout_B; b += EPI_WARPS) {
+          if (a.scout_live[b] <= 0) continue;   // warp-uniform
+          const uint4* src = reinterpret_cast<const uint4*>(Ug + ((size_t)b * a.D + a.scout_depth) * V + t0);
+          float bv = -INFINITY; int bi = 0x7FFFFFFF;
+          for (int c0 = 0; c0 < nvec; c0 += 5 * 32) {
+            uint4 x[5];
+#pragma unroll
+            for (int u = 0; u < 5; ++u) {
+              const int c = c0 + u * 32 + lane;
+              x[u] = c < nvec ? __ldg(src + c) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // -inf
+            }
+#pragma unroll
+            for (int u = 0; u < 5; ++u) {
+              float f[8];
+              unpack_bf16x8(x[u], f);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) if (f[i] > bv) { bv = f[i]; bi = t0 + (c0 + u * 32 + lane) * 8 + i; }
+            }
+          }
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, off);
+            const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, off);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+          }
+          if (lane == 0) a.utop[((size_t)b * a.D + a.scout_depth) * a.ntiles + tile] = make_uint2(__float_as_uint(bv), (unsigned)bi);
+        }
+      }
 
       const int p = R > 1 ? row % per : g * 128 + row;
       const int rho = R > 1 ? row / per : 0;   // uniform within a warp (128/R is a multiple of 32)
@@ -282,10 +304,21 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       float m = -INFINITY, s0 = 0.f, sT = 0.f;
       uint4 nx0 = make_uint4(0, 0, 0, 0), nx1 = nx0;    // prefetched base logits of the next owned chunk
       bool have_next = false;
-      bool first = true;
       bool alive = true;
-      for (int nb = 0; nb < nblk && alive; ++nb) {
-        const int it = g * nblk + nb, tb = it % NBUF, u = it / NBUF;
+      // Blocks of 64 tokens are dealt to the splits round-robin (block nb belongs to split nb % 4), and a split
+      // alternates between two accumulator buffers of its own, so its four quarter warps and the MMA issuer form a
+      // pipeline of their own: a slow warp holds up three others, not fifteen, and the next block's accumulators
+      // are written while this one is scanned.  A row's 128 bytes of base logits per block are one cache line;
+      // the line of the split's next block is requested from L2 when a block begins.
+      const int nuse = nblk > s ? (nblk - s + EPI_S - 1) / EPI_S : 0;   // blocks of this split per group
+      auto prefetch_block = [&](int nb) {
+        if (active && nb < nblk) asm volatile("prefetch.global.L2 [%0];" ::"l"(Urow + t0 + nb * BLK_N));
+      };
+      prefetch_block(s);
+      for (int nb = s; nb < nblk && alive; nb += EPI_S) {
+        const int j = nb / EPI_S, h = j & 1;
+        const int tb = s + EPI_S * h, u = g * ((nuse + 1 - h) >> 1) + (j >> 1);   // buffer, and how often it was used before
+        prefetch_block(nb + EPI_S);
         {
           int ok = 1;
           if (lane == 0) ok = mbar_wait(t_full + tb, u & 1, s_abort, a.err, wait_limit) ? 1 : 0;
@@ -293,10 +326,10 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
           if (!ok) { alive = false; break; }
           tc_fence_after();
         }
-        const int nch = min(8, (tlen - nb * BLK_N + 15) / 16);
+        const int nch = min(BLK_N / 16, (tlen - nb * BLK_N + 15) / 16);
         for (int c = 0; c < nch; ++c) {
-          const int cg = nb * 8 + c;
-          if ((cg & (R - 1)) != rho || ((cg >> rsh) % EPI_S) != s) continue;   // warp-uniform; R is 1, 2 or 4
+          const int cg = nb * (BLK_N / 16) + c;
+          if ((c & (R - 1)) != rho) continue;   // warp-uniform; R is 1, 2 or 4: the replicas split a block's chunks
           float acc[16];
           tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * BLK_N + c * 16), acc);
           if (!active) continue;
@@ -306,7 +339,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
           const uint4 u0 = have_next ? nx0 : __ldg(reinterpret_cast<const uint4*>(Urow + v0));
           const uint4 u1 = have_next ? nx1 : (valid > 8 ? __ldg(reinterpret_cast<const uint4*>(Urow + v0 + 8)) : make_uint4(0, 0, 0, 0));
           {
-            const int cgn = cg + R * EPI_S;           // the next chunk this warp owns
+            const int cgn = (c + R < BLK_N / 16) ? cg + R : (nb + EPI_S) * (BLK_N / 16) + rho;   // the next chunk this warp owns
             const int vn = t0 + cgn * 16;
             have_next = (cgn * 16 < tlen);
             if (have_next) {
@@ -325,17 +358,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
 #pragma unroll
             for (int i = 0; i < 16; ++i) acc[i] = (i < valid) ? acc[i] : -INFINITY;
           }
-          if (first) {
-            first = false;
-            if (seeded) {
-              const int pid = ((tile * EPI_S + s) * R + rho) % K;
-              publish_seed(acc, v0, invT, keys, a.seed, req, hash, a.slots + ((size_t)p * K + pid) * SLOT_STRIDE,
-                           a.slots + (((size_t)a.cap + p) * K + pid) * SLOT_STRIDE);
-              // the bounds of this row arrive a few microseconds later (the refresh warp copies them here)
-              const volatile unsigned* wthr = s_thr + (keys ? 128 : 0) + prow;
-              for (int spin = 0; spin < 96 && *wthr == 0u && !*s_abort; ++spin) __nanosleep(64);
-            }
-          }
+          // the row's bounds as the refresh warp last left them (read here: the loads' latency hides under the scan)
+          const float thrL = dec_f(s_thr[prow]), thrK = dec_f(s_thr[128 + prow]);
           // ---- the scan of one chunk -------------------------------------------------------------
           // high halves of the sixteen uniforms: two generator calls, issued first so that their long
           // dependent chains overlap the exponentials below
@@ -379,13 +403,12 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
           }
           // ---- candidates ---------------------------------------------------------------------------
           uint32_t mkK = 0, mkL = 0;
-          const float thrL = fmaxf(dec_f(s_thr[prow]), sh.lthr[row]);
           if (cm >= thrL) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) mkL |= (uint32_t)(acc[i] >= thrL && acc[i] > -INFINITY) << i;
           }
           if (keys) {
-            const float thr = fmaxf(dec_f(s_thr[128 + prow]), sh.lthr[128 + row]);
+            const float thr = thrK;
             // the whole chunk first: its best logit plus the noise bound of the largest leading bits among its
             // sixteen tokens bounds every key in it; then four tokens at a time, then singly
             const uint32_t m8 = __vmaxu2(__vmaxu2(__vmaxu2(cw0.x, cw0.y), __vmaxu2(cw0.z, cw0.w)),
@@ -462,6 +485,10 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
           const bool in = rr < per && p < P;
           rL[k] = in ? __ldcg(a.thr + p) : 0u;
           rK[k] = in ? __ldcg(a.thr + (size_t)a.cap + p) : 0u;
+          if (in && a.thr0) {   // never below the seed bounds
+            rL[k] = max(rL[k], __ldcg(a.thr0 + p));
+            rK[k] = max(rK[k], __ldcg(a.thr0 + (size_t)a.cap + p));
+          }
         }
 #pragma unroll
         for (int off = 8; off > 0; off >>= 1) v = min(v, __shfl_xor_sync(0xFFFFFFFFu, v, off));
@@ -529,24 +556,40 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       const uint32_t ws_addr = smem_u32(Ws), as_addr = smem_u32(As);
       if (mbar_wait(a_full, g & 1, s_abort, a.err, wait_limit)) {
         tc_fence_after();
-        for (int nb = 0; nb < nblk; ++nb) {
-          const int it = g * nblk + nb, tb = it % NBUF, u = it / NBUF;
-          if (u >= 1) {
-            if (!mbar_wait(t_empty + tb, (u - 1) & 1, s_abort, a.err, wait_limit)) break;
+        // each split's pipeline advances on its own: whichever buffer is drained (and whose W block has landed) is refilled
+        int nxt[EPI_S];
+#pragma unroll
+        for (int i = 0; i < EPI_S; ++i) nxt[i] = i;
+        int remaining = nblk;
+        uint32_t spin = 0;
+        while (remaining > 0) {
+          bool progressed = false;
+#pragma unroll
+          for (int sp = 0; sp < EPI_S; ++sp) {
+            const int nb = nxt[sp];
+            if (nb >= nblk) continue;
+            const int nuse = (nblk - sp + EPI_S - 1) / EPI_S;
+            const int j = nb / EPI_S, h = j & 1, tb = sp + EPI_S * h;
+            const int u = g * ((nuse + 1 - h) >> 1) + (j >> 1);
+            if (u >= 1 && !mbar_try_wait(t_empty + tb, (u - 1) & 1)) continue;
+            if (use_tma && g == 0 && !mbar_try_wait(w_full + nb * BLK_N / WBLK, 0)) continue;
             tc_fence_after();
+            const uint32_t idesc = instr_desc(BLK_N);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
+            for (int ks = 0; ks < rp / 16; ++ks) {
+              const uint64_t adesc = smem_desc(as_addr + (uint32_t)(ks >> 2) * a_slab_bytes + (uint32_t)(ks & 3) * 32u, 16u, 1024u);
+              const uint64_t bdesc = smem_desc(ws_addr + (uint32_t)nb * slab_bytes + (uint32_t)ks * 2048u, slab_bytes, 1024u);
+              mma_bf16(d_tmem, adesc, bdesc, idesc, ks > 0 ? 1u : 0u);
+            }
+            mma_commit(t_full + tb);
+            nxt[sp] = nb + EPI_S;
+            --remaining;
+            progressed = true;
           }
-          if (use_tma && g == 0) {
-            if (!mbar_wait(w_full + nb, 0, s_abort, a.err, wait_limit)) break;
-          }
-          const int n = (tlen - nb * BLK_N > 64) ? 128 : 64;
-          const uint32_t idesc = instr_desc(n);
-          const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
-          for (int ks = 0; ks < rp / 16; ++ks) {
-            const uint64_t adesc = smem_desc(as_addr + (uint32_t)(ks >> 2) * a_slab_bytes + (uint32_t)(ks & 3) * 32u, 16u, 1024u);
-            const uint64_t bdesc = smem_desc(ws_addr + (uint32_t)(2 * nb) * slab_bytes + (uint32_t)ks * 2048u, slab_bytes, 1024u);
-            mma_bf16(d_tmem, adesc, bdesc, idesc, ks > 0 ? 1u : 0u);
-          }
-          mma_commit(t_full + tb);
+          if (progressed) { spin = 0; continue; }
+          if (*s_abort) break;
+          if (++spin > wait_limit) { *s_abort = 1; if (a.err) atomicExch(a.err, 1); break; }
+          if (spin > 8) __nanosleep(32);
         }
       }
     }
