@@ -141,7 +141,7 @@ extern "C" int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags) {
 
 extern "C" int32_t ts_set_test_mode(ts_ctx* ctx, uint32_t flags) {
   if (!ctx) return set_error(TS_ERR_INVALID, "ts_set_test_mode: null context");
-  const uint32_t known = TS_TEST_FORCE_FMA | TS_TEST_NO_TMA | TS_TEST_NO_FEW | TS_TEST_NO_SEED | TS_TEST_SHORT_WAITS | TS_TEST_LOST_ARRIVAL;
+  const uint32_t known = TS_TEST_FORCE_FMA | TS_TEST_NO_TMA | TS_TEST_NO_FEW | TS_TEST_NO_SEED | TS_TEST_SHORT_WAITS | TS_TEST_LOST_ARRIVAL | TS_TEST_NO_PERSIST;
   if (flags & ~known) return set_error(TS_ERR_INVALID, "ts_set_test_mode: unknown switch");
   const unsigned before = ctx->test_mode;
   ctx->test_mode = flags;
@@ -162,7 +162,7 @@ extern "C" size_t ts_workspace_bytes(const ts_ctx* ctx, int32_t batch) {
 
 static const char* kKernelNames[K_COUNT] = {"expand_init", "score_tile", "score_merge", "expand_level", "expand_finalize",
                                             "zrow_stats", "verify_greedy", "verify_walk", "verify_check", "score_few", "allocate_select", "allocate_cut",
-                                            "calib_accumulate", "calib_refit", "attention_inputs", "score_seed"};
+                                            "calib_accumulate", "calib_refit", "attention_inputs", "score_seed", "expand_persistent"};
 
 extern "C" const char* ts_kernel_name(int32_t id) { return (id >= 0 && id < K_COUNT) ? kKernelNames[id] : nullptr; }
 

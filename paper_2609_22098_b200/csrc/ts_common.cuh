@@ -73,6 +73,7 @@ struct ts_ctx {
   const void* tmapW_ptr;
   int tma_state;   // 0 not tried yet, 1 encoder found, -1 unavailable
   int walk_pdl;    // -1: the driver refused a cooperative launch with programmatic serialization
+  int persist_pdl; // the same for the persistent expansion kernel
   unsigned ablation;   // TS_ABLATE_* switches (0 = the method)
   unsigned test_mode;  // TS_TEST_* switches (0 = the product's kernel selection and wait limits)
   uint32_t wait_limit; // polls before a bounded device-side wait gives up
@@ -93,6 +94,7 @@ struct WsLayout {
   // level parent lists (two, alternating) [Pcap]
   size_t lst_req[2], lst_depth[2], lst_token[2], lst_hash[2], lst_slot[2];
   size_t lvl_count;      // int[DMAX + 2]
+  size_t ex_barrier;     // unsigned[4]: grid barrier of the persistent expansion kernel
   size_t utop;           // uint2[B][D][ntiles]: best base logit (value, token) of every vocabulary tile of every row
   // per-request pool, [B][N]
   size_t pl_alive, pl_depth, pl_parent, pl_sib, pl_tok, pl_lidx, pl_new, pl_logkey, pl_logS, pl_q0, pl_logqT,
@@ -168,6 +170,7 @@ __host__ inline WsLayout make_layout(const ts_ctx* ctx, int B) {
     L.lst_hash[i] = take(P * 8); L.lst_slot[i] = take(P * 4);
   }
   L.lvl_count = take((DMAX + 2) * 4);
+  L.ex_barrier = take(64);
   L.utop = take(b * (size_t)c.D * (size_t)ctx->tile.ntiles * 8);
   L.pl_alive = take(b * N * 4); L.pl_depth = take(b * N * 4); L.pl_parent = take(b * N * 4);
   L.pl_sib = take(b * N * 4); L.pl_tok = take(b * N * 4); L.pl_lidx = take(b * N * 4); L.pl_new = take(b * N * 4);

@@ -12,43 +12,9 @@
 
 #include "ts_internal.h"
 #include "ts_scan.cuh"
+#include "ts_level.cuh"
 
 namespace ts {
-
-struct ExpandArgs {
-  int B, D, K, N, V;
-  float T;
-  const int* anchor; const float* theta;
-  DevCalib calib;
-  // level lists
-  int* lst_req[2]; int* lst_depth[2]; int* lst_token[2]; uint64_t* lst_hash[2]; int* lst_slot[2];
-  int* lvl_count;
-  // merged scoring results
-  const float *res_lse0, *res_lseT; const int* res_top_tok; const float* res_top_logit;
-  const int* res_draw_tok; const float* res_draw_logit;
-  // pool
-  int *pl_alive, *pl_depth, *pl_parent, *pl_sib, *pl_tok;
-  double *pl_logkey, *pl_logS; float *pl_q0, *pl_logqT, *pl_lseT; uint64_t *pl_hash, *pl_path;
-  float* root_lseT; int *req_npar, *req_base, *req_nscored;
-  // candidates
-  int *cd_valid, *cd_parent, *cd_sib, *cd_tok; double *cd_logkey, *cd_logS; float *cd_q0, *cd_logqT; int* cd_rank;
-  int* status; int* err; unsigned* thr; int thr_head, thr_words;
-  unsigned* seed_cnt;   // the seed kernel's arrival counters
-  // seed bounds of the next level's parents (made by the level kernel from the scoring kernel's scouting)
-  const void *U, *A, *W; int r, ntiles, cap; uint64_t seed; const uint2* utop; unsigned* thr0;
-  int calib_qT;   // ablation: the calibrator is fed the tempered conditional when T > 0
-};
-
-__device__ __forceinline__ void request_caps(const ExpandArgs& a, int b, int& K_eff, int& N_eff, double& log_theta) {
-  const float th = a.theta[b];
-  K_eff = a.K < a.V ? a.K : a.V;
-  N_eff = a.N;
-  if (th >= 1.f) {  // chain member of the price ladder
-    K_eff = 1; N_eff = a.D < a.N ? a.D : a.N; log_theta = -INFINITY;
-  } else {
-    log_theta = th > 0.f ? log((double)th) : -INFINITY;
-  }
-}
 
 __global__ void expand_init_kernel(ExpandArgs a) {
   pdl_wait();                // whatever ran before in the stream may still be reading what this kernel resets
@@ -59,6 +25,7 @@ __global__ void expand_init_kernel(ExpandArgs a) {
   for (int i = b * blockDim.x + threadIdx.x; i < a.thr_words; i += gridDim.x * blockDim.x)
     a.thr[i < a.thr_head ? i : a.thr_head + (size_t)(i - a.thr_head) * SLOT_STRIDE] = 0u;
   if (b == 0) for (int i = threadIdx.x; i < SEED_SPLIT_PARENTS; i += blockDim.x) a.seed_cnt[i] = 0u;
+  if (b == 0 && threadIdx.x < 4) a.ex_barrier[threadIdx.x] = 0u;
   if (b >= a.B) return;
   for (int s = threadIdx.x; s < a.N; s += blockDim.x) a.pl_alive[(size_t)b * a.N + s] = 0;
   if (threadIdx.x == 0) {
@@ -77,308 +44,13 @@ __global__ void expand_init_kernel(ExpandArgs a) {
   }
 }
 
-struct Entry { double key; uint64_t path; int depth; };
-
-__device__ __forceinline__ bool before(double ka, int da, uint64_t pa, double kb, int db, uint64_t pb) {
-  if (ka != kb) return ka > kb;
-  if (da != db) return da < db;
-  return pa < pb;
-}
-
-// One CTA per request; level d = depth of the parents just scored.
-__global__ void __launch_bounds__(256) expand_level_kernel(ExpandArgs a, int d, int seed_next) {
+// One CTA per request; level d = depth of the parents just scored (body in ts_level.cuh).
+__global__ void __launch_bounds__(LEVEL_THREADS) expand_level_kernel(ExpandArgs a, int d, int seed_next) {
   extern __shared__ __align__(16) unsigned char sm_raw[];
-  __shared__ int s_cnt[2];
-  __shared__ int s_base;
-  const int b = blockIdx.x, tid = threadIdx.x;
-  const int N = a.N, K = a.K;
+  __shared__ LevelSmem sm;
   pdl_wait();               // merged scoring results of this level
   pdl_launch_dependents();
-  const int npar = a.req_npar[b], base = a.req_base[b];
-  const int cur = d & 1, nxt = cur ^ 1;
-  int K_eff, N_eff; double log_theta;
-  request_caps(a, b, K_eff, N_eff, log_theta);
-  const size_t pb = (size_t)b * N, cb = (size_t)b * N * K;
-  if (tid == 0) {
-    if (a.err[0] != 0 && a.status[b] == TS_OK) a.status[b] = TS_ERR_TIMEOUT;  // a wait in the scoring kernel ran out
-    s_base = a.status[b];
-  }
-  __syncthreads();
-  if (npar == 0 || s_base != TS_OK) {  // uniform: read once, before any thread can change the status
-    if (tid == 0) a.req_npar[b] = 0;
-    return;
-  }
-  // ---- phase 1: slots of every scored parent, one thread per (parent, sibling rank) -------------
-  for (int t = tid; t < npar * K; t += blockDim.x) {
-    const int i = t / K, j = t % K;
-    const int li = base + i;
-    const int slot = a.lst_slot[cur][li];
-    const double logS_v = slot < 0 ? 0.0 : a.pl_logS[pb + slot];
-    const double lse0 = a.res_lse0[li], lseT = a.res_lseT[li];
-    if (j == 0) {
-      if (slot < 0) a.root_lseT[b] = (float)lseT; else a.pl_lseT[pb + slot] = (float)lseT;
-      if (!(lse0 == lse0) || isinf(lse0)) a.status[b] = TS_ERR_NUMERIC;
-    }
-    const int* top_tok = a.res_top_tok + (size_t)li * K; const float* top_logit = a.res_top_logit + (size_t)li * K;
-    const int* draw_tok = a.res_draw_tok + (size_t)li * K; const float* draw_logit = a.res_draw_logit + (size_t)li * K;
-    const size_t ci = cb + (size_t)i * K + j;
-    int valid = 0;
-    if (j < K_eff) {
-      int bi = j;
-      if (a.T > 0.f) {  // best token of q0 not among the first j draws: the pre-draw bound
-        bi = -1;
-        for (int tt = 0; tt < K_eff && bi < 0; ++tt) {
-          bool used = false;
-          for (int u = 0; u < j; ++u) used |= (draw_tok[u] == top_tok[tt]);
-          if (!used) bi = tt;
-        }
-      }
-      const int x = draw_tok[j];
-      if (bi >= 0 && top_tok[bi] >= 0 && x >= 0) {
-        // the calibrator's input: the untempered conditional, or (ablation) the tempered one
-        const bool tempered = a.calib_qT && a.T > 0.f;
-        const double lsc = tempered ? 1.0 / (double)a.T : 1.0, lsn = tempered ? lseT : lse0;
-        const double key = logS_v + log_phat(a.calib, d, (double)top_logit[bi] * lsc, lsn);
-        if (!(key < log_theta)) {
-          const double lx = draw_logit[j];
-          valid = 1;
-          a.cd_parent[ci] = slot; a.cd_sib[ci] = j; a.cd_tok[ci] = x;
-          a.cd_logkey[ci] = key;
-          a.cd_logS[ci] = logS_v + log_phat(a.calib, d, lx * lsc, lsn);
-          a.cd_q0[ci] = (float)exp(lx - lse0);
-          a.cd_logqT[ci] = a.T > 0.f ? (float)(lx / (double)a.T - lseT) : (float)(lx - lse0);
-        }
-      }
-    }
-    a.cd_valid[ci] = valid;
-  }
-  __syncthreads();
-  // a sibling slot exists only if the one before it was admitted (keys are non-increasing in j)
-  for (int i = tid; i < npar; i += blockDim.x) {
-    int vals[KMAX];   // all flags of the parent first: independent loads, one round trip
-#pragma unroll
-    for (int j = 0; j < KMAX; ++j) vals[j] = j < K ? a.cd_valid[cb + (size_t)i * K + j] : 0;
-    bool open = true;
-#pragma unroll
-    for (int j = 0; j < KMAX; ++j) {
-      if (j < K) {
-        if (!open && vals[j]) a.cd_valid[cb + (size_t)i * K + j] = 0;
-        else if (!vals[j]) open = false;
-      }
-    }
-  }
-  __syncthreads();
-  // ---- phase 2: who survives the cut to N_eff ------------------------------------------------
-  const int ncand = npar * K;
-  if (tid < 2) s_cnt[tid] = 0;
-  __syncthreads();
-  {
-    int lp = 0, lc = 0;
-    for (int s = tid; s < N; s += blockDim.x) lp += a.pl_alive[pb + s] ? 1 : 0;
-    for (int c = tid; c < ncand; c += blockDim.x) lc += a.cd_valid[cb + c] ? 1 : 0;
-    if (lp) atomicAdd(&s_cnt[0], lp);
-    if (lc) atomicAdd(&s_cnt[1], lc);
-  }
-  __syncthreads();
-  const int n_pool = s_cnt[0], n_valid = s_cnt[1];
-  const int shift = 60 - 4 * d;
-  if (n_pool + n_valid > N_eff) {
-    // rank every entry by counting the entries that come before it in (key desc, depth asc, path asc)
-    Entry* ent = reinterpret_cast<Entry*>(sm_raw);
-    const int M = N + ncand;
-    for (int e = tid; e < M; e += blockDim.x) {
-      Entry x; x.depth = -1; x.key = 0; x.path = 0;
-      if (e < N) {
-        if (a.pl_alive[pb + e]) { x.key = a.pl_logkey[pb + e]; x.depth = a.pl_depth[pb + e]; x.path = a.pl_path[pb + e]; }
-      } else {
-        const size_t ci = cb + (e - N);
-        if (a.cd_valid[ci]) {
-          const int slot = a.cd_parent[ci];
-          x.key = a.cd_logkey[ci]; x.depth = d + 1;
-          x.path = (slot < 0 ? 0ull : a.pl_path[pb + slot]) | ((uint64_t)a.cd_sib[ci] << shift);
-        }
-      }
-      ent[e] = x;
-    }
-    __syncthreads();
-    for (int e = tid; e < M; e += blockDim.x) {
-      const Entry x = ent[e];
-      if (x.depth < 0) continue;
-      int rank = 0;
-      for (int f = 0; f < M; ++f) {
-        const Entry y = ent[f];
-        if (y.depth >= 0 && f != e && before(y.key, y.depth, y.path, x.key, x.depth, x.path)) ++rank;
-      }
-      if (rank >= N_eff) {
-        if (e < N) a.pl_alive[pb + e] = 0; else a.cd_valid[cb + (e - N)] = 0;
-      }
-    }
-    __syncthreads();
-  }
-  // ---- phase 3: place surviving candidates into free pool slots (deterministic order) --------
-  // the t-th surviving candidate (in candidate order) takes the t-th free slot (in slot order)
-  __shared__ int s_free[256], s_new[256], s_warp[8];
-  __shared__ int s_run, s_nb;
-  const int lane = tid & 31, warp = tid >> 5;
-  {
-    const bool fr = tid < N && !a.pl_alive[pb + tid];
-    const unsigned bal = __ballot_sync(0xFFFFFFFFu, fr);
-    if (lane == 0) s_warp[warp] = __popc(bal);
-    __syncthreads();
-    int off = 0;
-    for (int w = 0; w < warp; ++w) off += s_warp[w];
-    if (fr) s_free[off + __popc(bal & ((1u << lane) - 1u))] = tid;
-    if (tid == 0) s_run = 0;
-    __syncthreads();
-  }
-  int nfree = 0;
-  for (int w = 0; w < 8; ++w) nfree += s_warp[w];
-  for (int c0 = 0; c0 < ncand; c0 += blockDim.x) {
-    const int c = c0 + tid;
-    const size_t ci = cb + c;
-    const bool v = c < ncand && a.cd_valid[ci];
-    const unsigned bal = __ballot_sync(0xFFFFFFFFu, v);
-    __syncthreads();  // s_warp is reused
-    if (lane == 0) s_warp[warp] = __popc(bal);
-    __syncthreads();
-    int off = s_run;
-    for (int w = 0; w < warp; ++w) off += s_warp[w];
-    const int t = off + __popc(bal & ((1u << lane) - 1u));
-    if (v) {
-      if (t >= nfree) { a.status[b] = TS_ERR_OVERFLOW; }
-      else {
-        const int sl = s_free[t];
-        const int slot = a.cd_parent[ci];
-        const int x = a.cd_tok[ci];
-        a.pl_alive[pb + sl] = 1; a.pl_depth[pb + sl] = d + 1; a.pl_parent[pb + sl] = slot; a.pl_sib[pb + sl] = a.cd_sib[ci];
-        a.pl_tok[pb + sl] = x; a.pl_logkey[pb + sl] = a.cd_logkey[ci]; a.pl_logS[pb + sl] = a.cd_logS[ci];
-        a.pl_q0[pb + sl] = a.cd_q0[ci]; a.pl_logqT[pb + sl] = a.cd_logqT[ci]; a.pl_lseT[pb + sl] = nanf("");
-        a.pl_hash[pb + sl] = path_hash(slot < 0 ? 0ull : a.pl_hash[pb + slot], x);
-        a.pl_path[pb + sl] = (slot < 0 ? 0ull : a.pl_path[pb + slot]) | ((uint64_t)a.cd_sib[ci] << shift);
-        s_new[t] = sl;
-      }
-    }
-    __syncthreads();
-    if (tid == 0) { int tot = 0; for (int w = 0; w < 8; ++w) tot += s_warp[w]; s_run += tot; }
-    __syncthreads();
-  }
-  const int nnew = min(s_run, nfree);
-  // ---- phase 4: next level's parents = new nodes that can still have admissible children -----------
-  {
-    const bool par = (d + 1 < a.D) && tid < nnew && !(a.pl_logS[pb + s_new[tid]] < log_theta);
-    const unsigned bal = __ballot_sync(0xFFFFFFFFu, par);
-    __syncthreads();
-    if (lane == 0) s_warp[warp] = __popc(bal);
-    __syncthreads();
-    int off = 0, cnt = 0;
-    for (int w = 0; w < 8; ++w) { if (w < warp) off += s_warp[w]; cnt += s_warp[w]; }
-    if (tid == 0) {
-      s_nb = cnt > 0 ? atomicAdd(&a.lvl_count[d + 1], cnt) : 0;
-      a.req_nscored[b] += npar;
-      a.req_npar[b] = cnt;
-    }
-    __syncthreads();
-    if (tid == 0) a.req_base[b] = s_nb;
-    int my_li = -1;
-    if (par) {
-      const int sl = s_new[tid];
-      const int li = s_nb + off + __popc(bal & ((1u << lane) - 1u));
-      a.lst_req[nxt][li] = b; a.lst_depth[nxt][li] = d + 1; a.lst_token[nxt][li] = a.pl_tok[pb + sl];
-      a.lst_hash[nxt][li] = a.pl_hash[pb + sl]; a.lst_slot[nxt][li] = sl;
-      my_li = li;
-    }
-    // ---- phase 5: seed bounds of those parents (bf16 tensor-core path; see ts_seed.cu for what they are) ----
-    // The scoring launch of this level left the best base logit of every vocabulary tile of row U[b][d+1]:
-    // the warps pick 2K good tokens from those, the tokens' columns of W are staged once for the request,
-    // every (parent, token) pair is evaluated exactly by one thread, and one thread per parent takes the
-    // K-th best logit and key, less the rounding margin.
-    if (seed_next && cnt > 0) {
-      __shared__ int s_stok[NSEED_MAX], s_pli[256], s_ptok[256];
-      __shared__ float s_sval[NSEED_MAX];
-      __shared__ uint64_t s_phash[256];
-      const int r = a.r, V = a.V;
-      const int npick = max(1, min(2 * K, NSEED_MAX) / 8), NSn = 8 * npick;
-      const float invT = a.T > 0.f ? 1.f / a.T : 1.f;
-      __syncthreads();   // the Entry array in dynamic shared memory is free now
-      float* Wc = reinterpret_cast<float*>(sm_raw);            // [NSn][r]
-      float* res = Wc + (size_t)NSn * r;                        // [cnt][NSn][2]: logit, key
-      if (par) {
-        const int i = off + __popc(bal & ((1u << lane) - 1u));
-        s_pli[i] = my_li; s_ptok[i] = a.pl_tok[pb + s_new[tid]]; s_phash[i] = a.pl_hash[pb + s_new[tid]];
-      }
-      {
-        const uint2* ut = a.utop + ((size_t)b * a.D + (d + 1)) * a.ntiles;
-        float bv = -INFINITY; int bi = 0x7FFFFFFF;
-        for (int t = lane * 8 + warp; t < a.ntiles; t += blockDim.x) {   // consecutive tiles go to different warps
-          const uint2 e = __ldcg(ut + t);
-          const float v = __uint_as_float(e.x);
-          if (v > bv || (v == bv && (int)e.y < bi)) { bv = v; bi = (int)e.y; }
-        }
-        for (int i = 0; i < npick; ++i) {   // every warp hands over its npick best
-          float wv = bv; int wi = bi;
-#pragma unroll
-          for (int o2 = 16; o2 > 0; o2 >>= 1) {
-            const float ov = __shfl_xor_sync(0xFFFFFFFFu, wv, o2);
-            const int oi = __shfl_xor_sync(0xFFFFFFFFu, wi, o2);
-            if (ov > wv || (ov == wv && oi < wi)) { wv = ov; wi = oi; }
-          }
-          if (wi == bi && bv > -INFINITY) { bv = -INFINITY; bi = 0x7FFFFFFF; }
-          if (lane == 0) { s_stok[warp * npick + i] = (wv > -INFINITY && wi >= 0 && wi < V) ? wi : -1; }
-        }
-      }
-      __syncthreads();
-      const __nv_bfloat16* Wg = reinterpret_cast<const __nv_bfloat16*>(a.W);
-      const __nv_bfloat16* Ag = reinterpret_cast<const __nv_bfloat16*>(a.A);
-      const __nv_bfloat16* Urow = reinterpret_cast<const __nv_bfloat16*>(a.U) + ((size_t)b * a.D + (d + 1)) * V;
-      for (int e = tid; e < NSn * r; e += blockDim.x) {
-        const int j = e / r, k = e % r;
-        Wc[e] = s_stok[j] >= 0 ? __bfloat162float(Wg[(size_t)k * V + s_stok[j]]) : 0.f;
-      }
-      if (tid < NSn) s_sval[tid] = s_stok[tid] >= 0 ? __bfloat162float(Urow[s_stok[tid]]) : -INFINITY;
-      __syncthreads();
-      for (int e = tid; e < cnt * NSn; e += blockDim.x) {
-        const int i = e / NSn, j = e % NSn;
-        float lg = -INFINITY, key = -INFINITY;
-        const int tok = s_stok[j];
-        if (tok >= 0) {
-          const uint4* arow = reinterpret_cast<const uint4*>(Ag + (size_t)s_ptok[i] * r);   // r is a multiple of 8 on this path
-          float dot = 0.f;
-          for (int k8 = 0; k8 < r / 8; ++k8) {
-            float av[8];
-            unpack_bf16x8(__ldg(arow + k8), av);
-#pragma unroll
-            for (int u = 0; u < 8; ++u) dot = fmaf(av[u], Wc[(size_t)j * r + k8 * 8 + u], dot);
-          }
-          lg = s_sval[j] + dot;
-          key = lg;
-          if (a.T > 0.f) {
-            const uint4 cw = stream_words(a.seed, b, s_phash[i], STREAM_GUMBEL_COARSE, (uint32_t)tok >> 3);
-            const uint4 fw = stream_words(a.seed, b, s_phash[i], STREAM_GUMBEL_FINE, (uint32_t)tok >> 3);
-            const uint32_t c16 = (word_of(cw, (tok & 7) >> 1) >> (16 * (tok & 1))) & 0xFFFFu;
-            const uint32_t f16 = (word_of(fw, (tok & 7) >> 1) >> (16 * (tok & 1))) & 0xFFFFu;
-            key = lg * invT + gumbel_from_bits((c16 << 16) | f16);
-          }
-        }
-        res[2 * e] = lg; res[2 * e + 1] = key;
-      }
-      __syncthreads();
-      for (int e = tid; e < 2 * cnt; e += blockDim.x) a.thr0[(size_t)(e & 1) * a.cap + s_pli[e >> 1]] = 0u;   // no bound unless K finite values turn up
-      __syncthreads();
-      for (int e = tid; e < 2 * cnt * NSn; e += blockDim.x) {
-        // one thread per value: the one with exactly K - 1 values before it (ties broken by place) is the K-th best
-        const int j = e % NSn, which = (e / NSn) & 1, i = e / (2 * NSn);
-        if (which == 1 && !(a.T > 0.f)) continue;
-        const float* val = res + (size_t)i * NSn * 2 + which;
-        const float mine = val[2 * j];
-        int before = 0;
-        for (int t = 0; t < NSn; ++t) before += (val[2 * t] > mine || (val[2 * t] == mine && t < j)) ? 1 : 0;
-        if (before == K - 1 && mine == mine && fabsf(mine) < INFINITY) {
-          const float margin = (2e-4f + 4e-5f * fabsf(mine)) * (which == 0 ? 1.f : fmaxf(invT, 1.f)) + (which == 0 ? 0.f : 2e-4f);
-          a.thr0[(size_t)which * a.cap + s_pli[i]] = enc_f(mine - margin);
-        }
-      }
-    }
-  }
+  level_step(a, d, seed_next, (int)blockIdx.x, sm, sm_raw, (int)threadIdx.x, [] { __syncthreads(); });
 }
 
 struct FinalArgs {
@@ -388,6 +60,7 @@ struct FinalArgs {
   const float* root_lseT; const int* req_nscored;
   int *n_nodes, *tok, *parent, *depth, *sib_rank; float *logS, *q0, *logqT, *logkey; int* pop_rank;
   uint64_t* node_hash; float* node_lseT; uint64_t* mask; int* n_scored;
+  const int* err; int* status;   // a bounded wait that ran out during the expansion is reported for every request still marked fine
 };
 
 // Canonical (BFS) renumbering, outputs and ancestor bitmasks; one CTA per request.
@@ -437,6 +110,7 @@ __global__ void __launch_bounds__(256) expand_finalize_kernel(FinalArgs a) {
     a.parent[pb + s_canon[s]] = cp;
   }
   if (tid == 0) {
+    if (*reinterpret_cast<const volatile int*>(a.err) != 0 && a.status[b] == TS_OK) a.status[b] = TS_ERR_TIMEOUT;
     a.n_nodes[b] = s_n;
     a.node_hash[(size_t)b * (N + 1)] = 0ull;
     if (a.node_lseT) a.node_lseT[(size_t)b * (N + 1)] = a.root_lseT[b];
@@ -530,19 +204,42 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   a.seed_cnt = a.thr0 + 2 * (size_t)L.rec_cap;
   a.U = U; a.A = A; a.W = W; a.r = c.r; a.ntiles = ctx->tile.ntiles; a.cap = L.rec_cap; a.seed = seed;
   a.utop = (const uint2*)(ws + L.utop);
+  a.ex_barrier = (unsigned*)(ws + L.ex_barrier);
 
   cudaError_t e0;
   { ProfScope ps(ctx, K_INIT, st); e0 = launch_kernel(expand_init_kernel, B > 296 ? B : 296, 256, 0, st, true, a); }
   cudaError_t e = e0 != cudaSuccess ? e0 : cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(init)", e);
   const size_t level_smem = level_smem_bytes(c);   // opted into at ts_create when above 48 KB
+  const bool seeds_on = ctx->use_mma && !(ctx->test_mode & TS_TEST_NO_SEED);
+  const bool persistent = seeds_on && !(ctx->test_mode & TS_TEST_NO_PERSIST) && persistent_supported(ctx, B);
+  if (persistent) {
+    // One cooperative launch runs every level: scan, merge, level step, separated by grid barriers.  Ahead of it the
+    // seed bounds of the root level (deeper levels get theirs from the level step before them).
+    ScoreArgs sa = make_score_args(ctx, (float*)(ws + L.rec), L.rec_cap, (int*)(ws + L.err), U, A, W, T, seed);
+    sa.pdl = 1; sa.P = 0; sa.P_dev = a.lvl_count;
+    sa.p_req = a.lst_req[0]; sa.p_depth = a.lst_depth[0]; sa.p_token = a.lst_token[0]; sa.p_hash = a.lst_hash[0];
+    set_seed_pointers(ctx, sa);
+    { ProfScope ps(ctx, K_SEED, st); e = launch_seed(ctx, sa, st); }
+    if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(seed)", e);
+    sa.utop = (uint2*)(ws + L.utop); sa.scout_live = a.req_npar; sa.scout_B = B; sa.scout_depth = 1;
+    PersistArgs pa{};
+    pa.on = 1; pa.nlevels = c.D; pa.ex = a; pa.barrier = a.ex_barrier;
+    pa.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
+    MergeArgs& m = pa.mg;
+    m.pdl = 0; m.few_ntiles = 0; m.P = 0; m.P_dev = nullptr; m.K = c.K; m.ntiles = sa.ntiles; m.cap = L.rec_cap; m.S = 1; m.mma = 1; m.T = T;
+    m.rec = sa.rec; m.thr = sa.thr; m.slots = sa.slots; m.thr0 = sa.thr0;
+    m.lse0 = res_lse0; m.lseT = res_lseT; m.top_tok = res_top_tok; m.top_logit = res_top_logit; m.draw_tok = res_draw_tok;
+    m.draw_logit = res_draw_logit;
+    { ProfScope ps(ctx, K_PERSIST, st); e = launch_expand_persistent(ctx, sa, pa, st); }
+    if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(persistent)", e);
+  }
   long long level_bound = B;   // parents a level can have at most: B at the root, K times more per level, B * Nmax overall
   // Seed bounds of a level on the tensor-core kernel: made by the level kernel before it when that level's scoring
   // launch scouted the rows (it does whenever it runs on the tensor-core kernel itself); by a seed launch otherwise
   // (the root level, and the first tensor-core level after levels on the few-parents kernel).
-  const bool seeds_on = ctx->use_mma && !(ctx->test_mode & TS_TEST_NO_SEED);
   bool scouted_prev = false;
-  for (int d = 0; d < c.D; ++d) {
+  for (int d = 0; d < c.D && !persistent; ++d) {
     const int cur = d & 1;
     const bool on_mma = ctx->use_mma && !(ctx->few_ok && level_bound <= FEW_MAX);
     ScoreExtras ex;
@@ -555,7 +252,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
                      res_draw_logit, st, /*pdl=*/true, d > 0 ? a.lvl_count + d - 1 : nullptr, (int)level_bound, &ex);
     level_bound = level_bound * c.K < (long long)B * c.Nmax ? level_bound * c.K : (long long)B * c.Nmax;
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(score)", e);
-    { ProfScope ps(ctx, K_LEVEL, st); e = launch_kernel(expand_level_kernel, B, 256, level_smem, st, true, a, d, scout ? 1 : 0); }
+    { ProfScope ps(ctx, K_LEVEL, st); e = launch_kernel(expand_level_kernel, B, LEVEL_THREADS, level_smem, st, true, a, d, scout ? 1 : 0); }
     scouted_prev = scout;
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(level)", e);
@@ -567,7 +264,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   f.pl_hash = a.pl_hash; f.pl_path = a.pl_path; f.root_lseT = a.root_lseT; f.req_nscored = a.req_nscored;
   f.n_nodes = n_nodes; f.tok = tok; f.parent = parent; f.depth = depth; f.sib_rank = sib_rank; f.logS = logS; f.q0 = q0;
   f.logqT = logqT; f.logkey = logkey; f.pop_rank = pop_rank; f.node_hash = node_hash; f.node_lseT = node_lseT;
-  f.mask = mask; f.n_scored = n_scored;
+  f.mask = mask; f.n_scored = n_scored; f.err = a.err; f.status = status;
   { ProfScope ps(ctx, K_FINAL, st); e = launch_kernel(expand_finalize_kernel, B, 256, 0, st, true, f); }
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(finalize)", e);

@@ -59,6 +59,9 @@ size_t thr_bytes(const ts_ctx* ctx, int cap);
 // p_bound: an upper bound of *P_dev the host knows (-1: none).  A list that cannot exceed FEW_MAX parents
 // goes to the few-parents kernel where the context has one.
 // rec: record scratch of score_scratch_bytes(ctx, max parents) bytes with slot capacity cap.
+ScoreArgs make_score_args(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W, float T,
+                          uint64_t seed);
+void set_seed_pointers(const ts_ctx* ctx, ScoreArgs& a);
 // What the expansion adds to a scoring pass: seed bounds that the level kernel already wrote (no seed launch),
 // and scouting of the next level's rows (see ScoreArgs).
 struct ScoreExtras {
@@ -98,7 +101,7 @@ cudaError_t launch_score_few(const ts_ctx* ctx, const ScoreArgs& a, int p_bound,
 // encodes (or finds cached in the context) the tensor map of W for 64-token boxes; false: not available
 bool w_tensor_map(ts_ctx* ctx, const void* W);
 
-enum KernelId { K_INIT, K_SCORE, K_MERGE, K_LEVEL, K_FINAL, K_ZROWS, K_GREEDY, K_WALK, K_CHECK, K_SCORE_FEW, K_ALLOC_SELECT, K_ALLOC_CUT, K_CALIB_ACC, K_CALIB_FIT, K_ATTN_INPUTS, K_SEED, K_COUNT };
+enum KernelId { K_INIT, K_SCORE, K_MERGE, K_LEVEL, K_FINAL, K_ZROWS, K_GREEDY, K_WALK, K_CHECK, K_SCORE_FEW, K_ALLOC_SELECT, K_ALLOC_CUT, K_CALIB_ACC, K_CALIB_FIT, K_ATTN_INPUTS, K_SEED, K_PERSIST, K_COUNT };
 
 struct Prof {
   bool on = false;

@@ -9,6 +9,7 @@
 // merge_kernel then folds the records of each parent.
 #include "ts_internal.h"
 #include "ts_scan.cuh"
+#include "ts_merge.cuh"
 
 namespace ts {
 
@@ -101,220 +102,15 @@ __global__ void __launch_bounds__(SCORE_THREADS, 1) score_tile_kernel(ScoreArgs 
   }
 }
 
-// ------------------------------------------------------------------------------------------------
-// Merge of the per-piece records: one CTA per parent.
-// Every thread folds its share of the pieces into a private (max, sums) pair and private top-K
-// lists; the block then takes K rounds of arg-max over the list heads (value desc, token asc).
-// ------------------------------------------------------------------------------------------------
-constexpr int MERGE_THREADS = 512;
-constexpr int MERGE_WARPS = MERGE_THREADS / 32;
-
-__device__ __forceinline__ bool better(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
-
-// Sorted list (value desc, token asc) with compile-time indices only, so it lives in registers.
-// The head is always entry 0: taking it shifts the rest up.
-template <int KR>
-struct MList {
-  float v[KR]; int i[KR]; float l[KR];
-  __device__ __forceinline__ void init() {
-#pragma unroll
-    for (int j = 0; j < KR; ++j) { v[j] = -INFINITY; i[j] = 0x7FFFFFFF; l[j] = 0.f; }
-  }
-  __device__ __forceinline__ void insert(float val, int idx, float lg) {
-    if (!better(val, idx, v[KR - 1], i[KR - 1])) return;
-#pragma unroll
-    for (int j = KR - 1; j >= 0; --j) {
-      const bool up = (j > 0) && better(val, idx, v[j > 0 ? j - 1 : 0], i[j > 0 ? j - 1 : 0]);
-      if (up) { v[j] = v[j > 0 ? j - 1 : 0]; i[j] = i[j > 0 ? j - 1 : 0]; l[j] = l[j > 0 ? j - 1 : 0]; }
-      else if (j == KR - 1 || better(val, idx, v[j], i[j])) { v[j] = val; i[j] = idx; l[j] = lg; }
-    }
-  }
-  __device__ __forceinline__ void pop() {
-#pragma unroll
-    for (int j = 0; j + 1 < KR; ++j) { v[j] = v[j + 1]; i[j] = i[j + 1]; l[j] = l[j + 1]; }
-    v[KR - 1] = -INFINITY; i[KR - 1] = 0x7FFFFFFF; l[KR - 1] = 0.f;
-  }
-};
-
-// K rounds of block-wide arg-max over the heads of the threads' sorted lists
-template <int KR>
-__device__ void block_select(MList<KR>& mine, int K, int* out_tok, float* out_val, float* s_v, int* s_i, float* s_l) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int j = 0; j < K; ++j) {
-    float wv = mine.v[0]; int wi = mine.i[0]; float wl = mine.l[0];
-    for (int off = 16; off > 0; off >>= 1) {
-      const float ov = __shfl_xor_sync(0xFFFFFFFFu, wv, off);
-      const int oi = __shfl_xor_sync(0xFFFFFFFFu, wi, off);
-      const float ol = __shfl_xor_sync(0xFFFFFFFFu, wl, off);
-      if (better(ov, oi, wv, wi)) { wv = ov; wi = oi; wl = ol; }
-    }
-    if (lane == 0) { s_v[warp] = wv; s_i[warp] = wi; s_l[warp] = wl; }
-    __syncthreads();
-    float gv = s_v[0]; int gi = s_i[0]; float gl = s_l[0];
-#pragma unroll
-    for (int w = 1; w < MERGE_WARPS; ++w)
-      if (better(s_v[w], s_i[w], gv, gi)) { gv = s_v[w]; gi = s_i[w]; gl = s_l[w]; }
-    if (gi != 0x7FFFFFFF && mine.i[0] == gi) mine.pop();  // tokens are unique per list
-    if (tid == 0) { out_tok[j] = gi == 0x7FFFFFFF ? -1 : gi; out_val[j] = gi == 0x7FFFFFFF ? 0.f : gl; }
-    __syncthreads();
-  }
-}
-
-constexpr int MERGE_CAP = 768;   // candidates per list the fast path can hold
-
-// The K best of a candidate array in shared memory (value desc, token asc), by counting: a candidate's
-// place is the number of candidates that beat it (tokens are unique per list, so places are too).  With
-// tight bounds a few dozen candidates arrive here, and the whole selection is one short pass.
-__device__ void rank_select(const float* cv, const int* ci, const float* cl, int n, int K, int t, int nt, int* out_tok, float* out_val) {
-  for (int e = t; e < n; e += nt) {
-    const float v = cv[e]; const int idx = ci[e];
-    int rank = 0;
-    for (int f = 0; f < n; ++f) rank += better(cv[f], ci[f], v, idx) ? 1 : 0;
-    if (rank < K) { out_tok[rank] = idx; out_val[rank] = cl[e]; }
-  }
-  for (int j = n + t; j < K; j += nt) { out_tok[j] = -1; out_val[j] = 0.f; }
-}
-
+// merge_kernel: one CTA of MERGE_THREADS threads per parent (the body lives in ts_merge.cuh; the persistent
+// expansion kernel runs the same body)
 template <int KR>
 __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(MergeArgs a) {
-  __shared__ float s_v[MERGE_WARPS]; __shared__ int s_i[MERGE_WARPS]; __shared__ float s_l[MERGE_WARPS];
-  __shared__ float s_m[MERGE_WARPS], s_s0[MERGE_WARPS], s_sT[MERGE_WARPS];
-  __shared__ float c_v[2][MERGE_CAP]; __shared__ int c_i[2][MERGE_CAP]; __shared__ float c_l[2][MERGE_CAP];
-  __shared__ int c_n[2];
+  __shared__ MergeSmem sm;
   pdl_wait();               // the scoring launch's records and the level's parent count
   pdl_launch_dependents();
   const int P = a.P_dev ? *a.P_dev : a.P;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float invT = a.T > 0.f ? 1.f / a.T : 1.f;
-  const int K = a.K, rw = rec_words(K);
-  const bool few = a.few_ntiles > 0;   // the level was scored by the few-parents kernel
-  const int R = few ? 1 : (a.mma ? mma_replicas(P) : 1);
-  const int npieces = few ? a.few_ntiles : a.ntiles * a.S * R;
-  for (int p = blockIdx.x; p < P; p += gridDim.x) {
-    // final launch-wide lower bounds of this parent's K-th best logit / key: entries below cannot win
-    const SharedThr gl{a.slots + (size_t)p * K * SLOT_STRIDE, 0}, gk{a.slots + ((size_t)a.cap + p) * K * SLOT_STRIDE, 0};
-    float bL = dec_f(slots_min(gl, K)), bK = a.T > 0.f ? dec_f(slots_min(gk, K)) : -INFINITY;
-    if (a.thr0) {   // never below the parent's seed bounds
-      bL = fmaxf(bL, dec_f(__ldcg(a.thr0 + p)));
-      if (a.T > 0.f) bK = fmaxf(bK, dec_f(__ldcg(a.thr0 + (size_t)a.cap + p)));
-    }
-    if (tid < 2) c_n[tid] = 0;
-    __syncthreads();
-    float m = -INFINITY, s0 = 0.f, sT = 0.f;
-    auto rec_of = [&](int q) {
-      if (few) return a.rec + ((size_t)q * FEW_MAX + p) * rw;
-      const int ts_ = q / R, rho = q % R;
-      const int slot = R > 1 ? rho * (128 / R) + p : p;
-      return a.rec + ((size_t)ts_ * a.cap + slot) * rw;
-    };
-    // the header of the next record is requested before this one's entries, so that a thread with
-    // several records pays one memory round trip per record, not two
-    // ... together with the record's best key: a record whose best logit (its maximum, in the header) and
-    // best key are below the final bounds has nothing to offer, and its entries are not read at all
-    float4 hn = make_float4(-INFINITY, 0.f, 0.f, 0.f);
-    float kn = -INFINITY;
-    if (tid < npieces) {
-      hn = __ldcg(reinterpret_cast<const float4*>(rec_of(tid)));
-      if (a.T > 0.f) kn = __ldcg(rec_of(tid) + 4 + 2 * K);
-    }
-    for (int q = tid; q < npieces; q += MERGE_THREADS) {
-      const float* rec = rec_of(q);
-      const float4 h = hn;
-      const float kbest = kn;
-      if (q + MERGE_THREADS < npieces) {
-        hn = __ldcg(reinterpret_cast<const float4*>(rec_of(q + MERGE_THREADS)));
-        if (a.T > 0.f) kn = __ldcg(rec_of(q + MERGE_THREADS) + 4 + 2 * K);
-      }
-      const float* f = rec + 4; const int* ii = reinterpret_cast<const int*>(rec) + 4;
-      // all entries of the record are requested at once (independent loads), then filtered
-      float tv[KR], kv[KR], kl[KR]; int ti[KR], ki[KR];
-      const int cnt = __float_as_int(h.w);
-      const int nt = h.x >= bL ? (cnt & 255) : 0, nk = kbest >= bK ? ((cnt >> 8) & 255) : 0;   // entries worth reading
-#pragma unroll
-      for (int j = 0; j < KR; ++j) {
-        ti[j] = j < nt ? __ldcg(ii + K + j) : -1;
-        tv[j] = j < nt ? __ldcg(f + j) : 0.f;
-        ki[j] = (j < nk && a.T > 0.f) ? __ldcg(ii + 3 * K + j) : -1;
-        kv[j] = (j < nk && a.T > 0.f) ? __ldcg(f + 2 * K + j) : 0.f;
-        kl[j] = (j < nk && a.T > 0.f) ? __ldcg(f + 4 * K + j) : 0.f;
-      }
-      if (h.x == -INFINITY) continue;  // a piece that scanned nothing
-      if (h.x > m) { const float d = m - h.x; s0 *= __expf(d); sT *= __expf(d * invT); m = h.x; }
-      const float d = h.x - m;
-      s0 += h.y * __expf(d); sT += h.z * __expf(d * invT);
-#pragma unroll
-      for (int j = 0; j < KR; ++j) {
-        if (ti[j] >= 0 && tv[j] >= bL) {
-          const int e = atomicAdd(&c_n[0], 1);
-          if (e < MERGE_CAP) { c_v[0][e] = tv[j]; c_i[0][e] = ti[j]; c_l[0][e] = tv[j]; }
-        }
-        if (ki[j] >= 0 && kv[j] >= bK) {
-          const int e = atomicAdd(&c_n[1], 1);
-          if (e < MERGE_CAP) { c_v[1][e] = kv[j]; c_i[1][e] = ki[j]; c_l[1][e] = kl[j]; }
-        }
-      }
-    }
-    // fold the (max, sums) pairs
-    for (int off = 16; off > 0; off >>= 1) {
-      const float om = __shfl_xor_sync(0xFFFFFFFFu, m, off);
-      const float o0 = __shfl_xor_sync(0xFFFFFFFFu, s0, off);
-      const float oT = __shfl_xor_sync(0xFFFFFFFFu, sT, off);
-      const float nm = fmaxf(m, om);
-      if (nm > -INFINITY) {
-        s0 = s0 * __expf(m - nm) + o0 * __expf(om - nm);
-        sT = sT * __expf((m - nm) * invT) + oT * __expf((om - nm) * invT);
-      }
-      m = nm;
-    }
-    if (lane == 0) { s_m[warp] = m; s_s0[warp] = s0; s_sT[warp] = sT; }
-    __syncthreads();
-    if (tid == 0) {
-      float gm = -INFINITY;
-      for (int w = 0; w < MERGE_WARPS; ++w) gm = fmaxf(gm, s_m[w]);
-      float g0 = 0.f, gT = 0.f;
-      for (int w = 0; w < MERGE_WARPS; ++w)
-        if (s_m[w] > -INFINITY) { g0 += s_s0[w] * __expf(s_m[w] - gm); gT += s_sT[w] * __expf((s_m[w] - gm) * invT); }
-      a.lse0[p] = gm + logf(g0);
-      a.lseT[p] = a.T > 0.f ? gm * invT + logf(gT) : gm + logf(g0);
-    }
-    // leave the launch-wide pruning state of this parent clean for the next launch
-    if (tid < 2 * K) a.slots[(((size_t)(tid / K) * a.cap + p) * K + tid % K) * SLOT_STRIDE] = 0u;
-    if (tid < 2) a.thr[(size_t)tid * a.cap + p] = 0u;   // and its condensed copy
-    const bool fits = c_n[0] <= MERGE_CAP && c_n[1] <= MERGE_CAP;   // uniform: read after the barrier above
-    if (fits) {
-      // the usual case: a few dozen candidates survive the bounds; half of the block ranks each list
-      const int half = tid / (MERGE_THREADS / 2), t = tid % (MERGE_THREADS / 2);
-      if (half == 0) rank_select(c_v[0], c_i[0], c_l[0], c_n[0], K, t, MERGE_THREADS / 2, a.top_tok + (size_t)p * K, a.top_logit + (size_t)p * K);
-      else if (a.T > 0.f)
-        rank_select(c_v[1], c_i[1], c_l[1], c_n[1], K, t, MERGE_THREADS / 2, a.draw_tok + (size_t)p * K, a.draw_logit + (size_t)p * K);
-      __syncthreads();
-    } else {
-      // too many candidates for the shared arrays (bounds not formed, e.g. tiny vocabularies): every
-      // thread rebuilds private sorted lists from its pieces and the block selects over their heads
-      MList<KR> top, key;
-      top.init(); key.init();
-      for (int q = tid; q < npieces; q += MERGE_THREADS) {
-        const float* rec = rec_of(q);
-        if (__ldcg(rec) == -INFINITY) continue;
-        const float* f = rec + 4; const int* ii = reinterpret_cast<const int*>(rec) + 4;
-        for (int j = 0; j < K; ++j) {
-          const int t = __ldcg(ii + K + j);
-          if (t >= 0) top.insert(__ldcg(f + j), t, __ldcg(f + j));
-          if (a.T > 0.f) { const int k2 = __ldcg(ii + 3 * K + j); if (k2 >= 0) key.insert(__ldcg(f + 2 * K + j), k2, __ldcg(f + 4 * K + j)); }
-        }
-      }
-      __syncthreads();
-      block_select<KR>(top, K, a.top_tok + (size_t)p * K, a.top_logit + (size_t)p * K, s_v, s_i, s_l);
-      if (a.T > 0.f) block_select<KR>(key, K, a.draw_tok + (size_t)p * K, a.draw_logit + (size_t)p * K, s_v, s_i, s_l);
-    }
-    if (!(a.T > 0.f)) {
-      if (tid < K) {
-        a.draw_tok[(size_t)p * K + tid] = a.top_tok[(size_t)p * K + tid];
-        a.draw_logit[(size_t)p * K + tid] = a.top_logit[(size_t)p * K + tid];
-      }
-    }
-    __syncthreads();
-  }
+  for (int p = blockIdx.x; p < P; p += gridDim.x) merge_parent<KR>(a, p, P, sm, (int)threadIdx.x, [] { __syncthreads(); });
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -337,21 +133,37 @@ unsigned* thr_base(const ts_ctx* ctx, float* rec, int cap) {
 // kernel's candidate scratch follows it and needs no clearing)
 size_t thr_bytes(const ts_ctx* ctx, int cap) { return ((size_t)cap * (4 + 2 * (size_t)ctx->cfg.K * SLOT_STRIDE) + SEED_SPLIT_PARENTS) * sizeof(unsigned); }
 
+// the part of the scoring arguments that does not depend on the parent list
+ScoreArgs make_score_args(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W, float T,
+                          uint64_t seed) {
+  const ts_config& c = ctx->cfg;
+  ScoreArgs a{};
+  a.U = U; a.A = A; a.W = W; a.V = c.V; a.D = c.D; a.r = c.r; a.K = c.K; a.T = T; a.seed = seed;
+  a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.cap = cap; a.S = 1; a.rec = rec; a.err = err;
+  a.wait_limit = ctx->wait_limit;
+  a.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
+  a.thr = thr_base(ctx, rec, cap); a.slots = a.thr + 2 * (size_t)cap;
+  a.thr0 = nullptr;
+  return a;
+}
+
+// where the seed bounds and the seed kernel's scratch sit behind the slots
+void set_seed_pointers(const ts_ctx* ctx, ScoreArgs& a) {
+  a.thr0 = a.slots + 2 * (size_t)a.cap * ctx->cfg.K * SLOT_STRIDE;
+  a.seed_cnt = a.thr0 + 2 * (size_t)a.cap;
+  a.seed_cand = a.seed_cnt + SEED_SPLIT_PARENTS;
+}
+
 cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,
                          const uint64_t* p_hash, float T, uint64_t seed, float* lse0, float* lseT, int* top_tok,
                          float* top_logit, int* draw_tok, float* draw_logit, cudaStream_t st, bool pdl, const int* P_prev_dev,
                          int p_bound, const ScoreExtras* extras) {
   const ts_config& c = ctx->cfg;
-  ScoreArgs a{};
+  ScoreArgs a = make_score_args(ctx, rec, cap, err, U, A, W, T, seed);
   a.pdl = pdl ? 1 : 0; a.P_prev_dev = P_prev_dev;
-  a.U = U; a.A = A; a.W = W; a.V = c.V; a.D = c.D; a.r = c.r; a.K = c.K; a.P = P; a.P_dev = P_dev;
-  a.p_req = p_req; a.p_depth = p_depth; a.p_token = p_token; a.p_hash = p_hash; a.T = T; a.seed = seed;
-  a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.cap = cap; a.S = 1; a.rec = rec; a.err = err;
-  a.wait_limit = ctx->wait_limit;
-  a.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
-  a.thr = thr_base(ctx, rec, cap); a.slots = a.thr + 2 * (size_t)cap;
-  a.thr0 = nullptr;
+  a.P = P; a.P_dev = P_dev;
+  a.p_req = p_req; a.p_depth = p_depth; a.p_token = p_token; a.p_hash = p_hash;
   cudaError_t e = cudaSuccess;
   // Which kernel scores the level: the few-parents kernel when the host knows that the list cannot hold
   // more than FEW_MAX parents (its own P, or a bound of the device-side count), the tile kernel otherwise.
@@ -361,9 +173,7 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
   a.few = run_few ? 1 : 0;
   if (run_tile && ctx->use_mma && !(ctx->test_mode & TS_TEST_NO_SEED)) {
     // seed bounds first: exact values of the tokens with the largest base logits of every parent's row
-    a.thr0 = a.slots + 2 * (size_t)cap * c.K * SLOT_STRIDE;
-    a.seed_cnt = a.thr0 + 2 * (size_t)cap;
-    a.seed_cand = a.seed_cnt + SEED_SPLIT_PARENTS;
+    set_seed_pointers(ctx, a);
     if (!(extras && extras->thr0_ready)) {   // (an expansion's level kernel writes them for the level after it)
       ProfScope ps(ctx, K_SEED, st);
       e = launch_seed(ctx, a, st);

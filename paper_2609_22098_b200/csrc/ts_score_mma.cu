@@ -40,6 +40,8 @@
 #include "ts_tc.cuh"
 #include "ts_internal.h"
 #include "ts_scan.cuh"
+#include "ts_merge.cuh"
+#include "ts_level.cuh"
 
 namespace ts {
 
@@ -57,6 +59,11 @@ constexpr uint32_t TMEM_COLS = NBUF * BLK_N;
 constexpr int MAX_BLK = 32;             // W load barriers (WBLK tokens each) of the largest tile (4096 tokens)
 constexpr int QCAP = 256;               // entries per candidate queue (power of two)
 constexpr uint32_t KIND_TOP = 1u, KIND_KEY = 2u;
+
+template <int ID, int NT>
+struct NamedSync {
+  __device__ __forceinline__ void operator()() const { asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(NT) : "memory"); }
+};
 
 // Shared-memory state of the selection side of one CTA.
 struct SelShared {
@@ -85,7 +92,7 @@ __device__ __forceinline__ float list_insert(float* v, int* t, float* aux, int K
 // One candidate, handled by one selector lane: exact key, insertion, publication.
 __device__ __forceinline__ void select_candidate(const ScoreArgs& a, const SelShared& sh, const uint4 e, const float* ghi,
                                                  float invT, int K, int tile, int R, int g, const volatile unsigned* s_thr,
-                                                 int pbase, bool do_insert) {
+                                                 int pbase, bool do_insert, const int* lp_req, const uint64_t* lp_hash) {
   const int tok = (int)e.x;
   const float lg = __uint_as_float(e.y);
   const int row = (int)(e.z & 0xFFu), s = (int)((e.z >> 8) & 0xFu);
@@ -107,7 +114,7 @@ __device__ __forceinline__ void select_candidate(const ScoreArgs& a, const SelSh
     const float thr = fmaxf(dec_f(s_thr[128 + prow]), sh.lthr[128 + row]);
     const float bnd = lg * invT + ghi[noise_bound_index(c16)];
     if (bnd >= thr && do_insert) {   // the bounds have often risen since the candidate was queued
-      const uint4 fw = stream_words(a.seed, a.p_req[p], a.p_hash[p], STREAM_GUMBEL_FINE, (uint32_t)tok >> 3);
+      const uint4 fw = stream_words(a.seed, __ldcg(lp_req + p), __ldcg(lp_hash + p), STREAM_GUMBEL_FINE, (uint32_t)tok >> 3);
       const uint32_t f16 = (word_of(fw, (tok & 7) >> 1) >> (16 * (tok & 1))) & 0xFFFFu;
       const float key = lg * invT + gumbel_from_bits((c16 << 16) | f16);
       if (key >= thr) {
@@ -119,7 +126,7 @@ __device__ __forceinline__ void select_candidate(const ScoreArgs& a, const SelSh
   }
 }
 
-__global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma) {
+__global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma, const __grid_constant__ PersistArgs pa) {
   extern __shared__ unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // The preamble below (shared-memory carve-up, tensor-memory allocation, barriers, bulk loads of W, noise
@@ -218,8 +225,22 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   const uint32_t tmem_base = *s_tmem;
   pdl_wait();                // parent lists and the level's parent count come from the previous kernel
   pdl_launch_dependents();
-  const int P = a.P_dev ? *a.P_dev : a.P;   // may be 0: an empty level only tears down
-  if (use_tma && !early_w && P > 0 && tid == 0) issue_w();
+  const bool persist = pa.on != 0;
+  int gg = 0;               // groups scanned so far, over all levels (barrier parities and use counts run on)
+  unsigned gen = 0;         // grid barriers passed
+  bool dead = false;        // a bounded wait ran out somewhere
+  bool w_issued = use_tma && early_w;   // bulk loads of the W tile are (or were) in flight
+  for (int lvl = 0; !dead; ++lvl) {
+  // the parent list of this level (in the persistent form written by the level step before it: read around L1)
+  const int cur = lvl & 1;
+  const int* lp_req = persist ? pa.ex.lst_req[cur] : a.p_req;
+  const int* lp_depth = persist ? pa.ex.lst_depth[cur] : a.p_depth;
+  const int* lp_token = persist ? pa.ex.lst_token[cur] : a.p_token;
+  const uint64_t* lp_hash = persist ? pa.ex.lst_hash[cur] : a.p_hash;
+  const int scout_depth = persist ? lvl + 1 : a.scout_depth;
+  const bool scout = a.utop != nullptr && scout_depth < a.D;
+  const int P = persist ? __ldcg(pa.ex.lvl_count + lvl) : (a.P_dev ? *a.P_dev : a.P);   // may be 0: an empty level only tears down
+  if (use_tma && !early_w && P > 0 && lvl == 0) { if (tid == 0) issue_w(); w_issued = true; }
 
   const int R = mma_replicas(P);
   const int per = 128 / R;
@@ -230,9 +251,9 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   const int rw = rec_words(K);
 
   for (int g = 0; g < ngroups; ++g) {
-    const int pbase = (g & 1) * 256;   // rows of group g use the bound buffer of parity g & 1
+    const int pbase = (gg & 1) * 256;   // successive groups alternate between two bound buffers
     // ---- per-group reset of the selection state (every thread) ---------------------------------------
-    if (g > 0) reset_selection();
+    if (gg > 0) reset_selection();
     for (int i = tid; i < 2 * 128; i += MMA_THREADS) {
       // the row's bounds start at its parent's seed bounds (exact values of K tokens, found before the launch)
       const int which = i >> 7, rr = i & 127;
@@ -252,18 +273,18 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
         const int rr = idx / cpr, ck = idx % cpr;
         const int p = R > 1 ? rr % per : g * 128 + rr;
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (p < P && ck * 8 < r) v = __ldg(reinterpret_cast<const uint4*>(Ag + (size_t)a.p_token[p] * r + ck * 8));
+        if (p < P && ck * 8 < r) v = __ldg(reinterpret_cast<const uint4*>(Ag + (size_t)__ldcg(lp_token + p) * r + ck * 8));
         *reinterpret_cast<uint4*>(As + (size_t)(ck >> 3) * a_slab_bytes + rr * 128 + (((ck & 7) ^ (rr & 7)) << 4)) = v;
       }
       fence_async_smem();
       mbar_arrive(a_full);
-      if (a.utop && g == 0) {
+      if (scout && g == 0) {
         // scouting (see ScoreArgs): fills the wait for the first accumulators, and brings the rows the next
         // level will score into L2
         const int nvec = tlen / 8;
         for (int b = warp; b < a.scout_B; b += EPI_WARPS) {
-          if (a.scout_live[b] <= 0) continue;   // warp-uniform
-          const uint4* src = reinterpret_cast<const uint4*>(Ug + ((size_t)b * a.D + a.scout_depth) * V + t0);
+          if (__ldcg(a.scout_live + b) <= 0) continue;   // warp-uniform
+          const uint4* src = reinterpret_cast<const uint4*>(Ug + ((size_t)b * a.D + scout_depth) * V + t0);
           float bv = -INFINITY; int bi = 0x7FFFFFFF;
           for (int c0 = 0; c0 < nvec; c0 += 5 * 32) {
             uint4 x[5];
@@ -286,7 +307,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
             const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, off);
             if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
           }
-          if (lane == 0) a.utop[((size_t)b * a.D + a.scout_depth) * a.ntiles + tile] = make_uint2(__float_as_uint(bv), (unsigned)bi);
+          if (lane == 0) a.utop[((size_t)b * a.D + scout_depth) * a.ntiles + tile] = make_uint2(__float_as_uint(bv), (unsigned)bi);
         }
       }
 
@@ -295,8 +316,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       const bool active = p < P;
       int req = 0; uint64_t hash = 0; const __nv_bfloat16* Urow = Ug;
       if (active) {
-        req = a.p_req[p]; hash = a.p_hash[p];
-        Urow = Ug + ((size_t)req * a.D + a.p_depth[p]) * V;
+        req = __ldcg(lp_req + p); hash = __ldcg(lp_hash + p);
+        Urow = Ug + ((size_t)req * a.D + __ldcg(lp_depth + p)) * V;
       }
       const int prow = pbase + (R > 1 ? row % per : row);
       const int sel = row >> 6;
@@ -317,7 +338,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       prefetch_block(s);
       for (int nb = s; nb < nblk && alive; nb += EPI_S) {
         const int j = nb / EPI_S, h = j & 1;
-        const int tb = s + EPI_S * h, u = g * ((nuse + 1 - h) >> 1) + (j >> 1);   // buffer, and how often it was used before
+        const int tb = s + EPI_S * h, u = gg * ((nuse + 1 - h) >> 1) + (j >> 1);   // buffer, and how often it was used before
         prefetch_block(nb + EPI_S);
         {
           int ok = 1;
@@ -467,7 +488,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       // keeps the shared-memory copies of every row's launch-wide pruning bounds current, so that the
       // other warps never wait on those (contended) global words
       for (uint32_t spin = 0; spin < wait_limit; ++spin) {
-        if (*s_done >= (g + 1) * EPI_WARPS || *s_abort) break;
+        if (*s_done >= (gg + 1) * EPI_WARPS || *s_abort) break;
         // (1) This CTA condenses the slots of the parents it is responsible for (parent p belongs to tile
         // p mod ntiles) into two words per parent; (2) every CTA reads the condensed words of its rows.
         // Only one CTA per parent reads the slot lines, which the whole launch is hitting with
@@ -512,7 +533,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       // ======================= selector warps ==========================================================
       const int sel = warp - W_SEL;
       unsigned head = sh.q_head[sel];
-      const int done_target = (g + 1) * EPI_WARPS;
+      const int done_target = (gg + 1) * EPI_WARPS;
       for (uint32_t spin = 0; spin < wait_limit; ++spin) {
         if (*s_abort) break;
         const bool finished = *s_done >= done_target;   // read before the tail: pushes precede the tick
@@ -547,14 +568,14 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
         const int turn = __popc(peers & ((1u << lane) - 1u));
         const int turns = __reduce_max_sync(0xFFFFFFFFu, have ? turn + 1 : 0);
         for (int t = 0; t < turns; ++t) {
-          if (have && turn == t) select_candidate(a, sh, e, ghi, invT, K, tile, R, g, s_thr, pbase, true);
+          if (have && turn == t) select_candidate(a, sh, e, ghi, invT, K, tile, R, g, s_thr, pbase, true, lp_req, lp_hash);
           __syncwarp();
         }
       }
     } else if (warp == W_MMA && lane == 0) {
       // ======================= MMA issuer ===========================================================
       const uint32_t ws_addr = smem_u32(Ws), as_addr = smem_u32(As);
-      if (mbar_wait(a_full, g & 1, s_abort, a.err, wait_limit)) {
+      if (mbar_wait(a_full, gg & 1, s_abort, a.err, wait_limit)) {
         tc_fence_after();
         // each split's pipeline advances on its own: whichever buffer is drained (and whose W block has landed) is refilled
         int nxt[EPI_S];
@@ -570,9 +591,9 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
             if (nb >= nblk) continue;
             const int nuse = (nblk - sp + EPI_S - 1) / EPI_S;
             const int j = nb / EPI_S, h = j & 1, tb = sp + EPI_S * h;
-            const int u = g * ((nuse + 1 - h) >> 1) + (j >> 1);
+            const int u = gg * ((nuse + 1 - h) >> 1) + (j >> 1);
             if (u >= 1 && !mbar_try_wait(t_empty + tb, (u - 1) & 1)) continue;
-            if (use_tma && g == 0 && !mbar_try_wait(w_full + nb * BLK_N / WBLK, 0)) continue;
+            if (use_tma && gg == 0 && !mbar_try_wait(w_full + nb * BLK_N / WBLK, 0)) continue;
             tc_fence_after();
             const uint32_t idesc = instr_desc(BLK_N);
             const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
@@ -597,7 +618,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (*s_abort) break;
+    if (*s_abort) { dead = true; break; }
     if (tid < 128) {
       const int row = tid;
       const int p = R > 1 ? row % per : g * 128 + row;
@@ -626,9 +647,38 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       }
     }
     __syncthreads();
+    ++gg;
   }
+  if (!persist || dead) break;
+  // ---- persistent form: merge, level step, next level -------------------------------------------------------
+  {
+    unsigned char* ov = reinterpret_cast<unsigned char*>(sh.q);   // queues, lists and partial sums are idle between scans
+    const unsigned nexpect = gridDim.x + (pa.lost_arrival ? 1u : 0u);
+    __threadfence();   // this CTA's records
+    if (!grid_barrier(pa.barrier, nexpect, gen, wait_limit)) { dead = true; break; }
+    if (tid < MERGE_THREADS) {
+      MergeArgs mg = pa.mg;
+      mg.P = P; mg.P_dev = nullptr;
+      for (int p = blockIdx.x; p < P; p += gridDim.x)
+        merge_parent<8>(mg, p, P, *reinterpret_cast<MergeSmem*>(ov), tid, NamedSync<1, MERGE_THREADS>());
+    }
+    __threadfence();   // merged results
+    if (!grid_barrier(pa.barrier, nexpect, gen, wait_limit)) { dead = true; break; }
+    if (tid < LEVEL_THREADS) {
+      for (int b = blockIdx.x; b < pa.ex.B; b += gridDim.x)
+        level_step(pa.ex, lvl, (scout && lvl + 1 < pa.nlevels) ? 1 : 0, b, *reinterpret_cast<LevelSmem*>(ov),
+                   ov + ((sizeof(LevelSmem) + 15) & ~(size_t)15), tid, NamedSync<2, LEVEL_THREADS>());
+    }
+    __syncthreads();
+    for (int i = tid; i < NSEL * QCAP; i += MMA_THREADS) sh.q[i] = make_uint4(0u, 0u, 0u, 0u);   // the queues' tags start clean again
+    __threadfence();   // next level's parent list and seed bounds
+    if (!grid_barrier(pa.barrier, nexpect, gen, wait_limit)) { dead = true; break; }
+    if (lvl + 1 >= pa.nlevels || __ldcg(pa.ex.lvl_count + lvl + 1) <= 0) break;
+  }
+  }
+  if (dead && persist && tid == 0) { atomicExch(pa.barrier + 1, 1u); if (a.err) atomicExch(a.err, 1); }
   // ---- tear-down -----------------------------------------------------------------------------------
-  if (use_tma && tid == 0 && ((*s_abort && (early_w || P > 0)) || (P <= 0 && early_w))) {
+  if (use_tma && tid == 0 && w_issued && (*s_abort || dead || gg == 0)) {
     // gave up somewhere, or nothing to score: do not leave while a bulk load may still be writing this
     // CTA's shared memory
     for (int nb = 0; nb < nblk_w; ++nb) {
@@ -721,7 +771,45 @@ cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t
   const int use_tma = w_tensor_map(c, a.W) ? 1 : 0;
   CUtensorMap tm;
   memcpy(&tm, c->tmapW, sizeof(tm));
-  const cudaError_t e = launch_kernel(score_mma_kernel, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma);
+  PersistArgs pa{};   // pa.on = 0: one scan
+  const cudaError_t e = launch_kernel(score_mma_kernel, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma, pa);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+// Shared memory that is idle between two scans (queues, lists, local thresholds, published bests, partial sums):
+// the merge and the level step of the persistent form work in it.
+static size_t persist_overlay_bytes(const ts_config& c) {
+  return (size_t)NSEL * QCAP * 16 + (size_t)128 * 5 * c.K * 4 + 2 * 128 * 4 + 2 * EPI_S * 128 * 4 + EPI_S * 128 * 16;
+}
+
+bool persistent_supported(const ts_ctx* ctx, int B) {
+  const ts_config& c = ctx->cfg;
+  if (!ctx->use_mma || c.K > 8) return false;                 // (the merge of the persistent form keeps 8-entry lists in registers)
+  if (ctx->few_ok && B <= FEW_MAX) return false;              // single-request decoding: the few-parents kernel serves the first levels
+  if (ctx->tile.ntiles > ctx->num_sms) return false;          // every CTA must be resident: the phases are separated by grid barriers
+  const size_t ov = persist_overlay_bytes(c);
+  return sizeof(MergeSmem) <= ov && ((sizeof(LevelSmem) + 15) & ~(size_t)15) + level_smem_bytes(c) <= ov;
+}
+
+cudaError_t launch_expand_persistent(const ts_ctx* ctx, const ScoreArgs& a, const PersistArgs& pa, cudaStream_t st) {
+  ts_ctx* c = const_cast<ts_ctx*>(ctx);
+  int use_tma = w_tensor_map(c, a.W) ? 1 : 0;
+  CUtensorMap tm;
+  memcpy(&tm, c->tmapW, sizeof(tm));
+  void* kargs[] = {(void*)&a, (void*)&tm, (void*)&use_tma, (void*)&pa};
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.ntiles); cfg.blockDim = dim3(MMA_THREADS); cfg.dynamicSmemBytes = ctx->tile.smem; cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeCooperative; attr[0].val.cooperative = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = c->persist_pdl >= 0 ? 2 : 1;
+  cudaError_t e = cudaLaunchKernelExC(&cfg, (const void*)score_mma_kernel, kargs);
+  if (e != cudaSuccess && cfg.numAttrs == 2) {   // not accepted together: remember, and launch cooperative only
+    (void)cudaGetLastError();
+    c->persist_pdl = -1;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelExC(&cfg, (const void*)score_mma_kernel, kargs);
+  }
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -160,11 +160,12 @@ def test_back_to_back_rounds_reproduce_bitwise():
             assert torch.equal(verdict["acc_tok"].cpu()[b, :L], v0["acc_tok"][b, :L]), (i, b)
 
 
-@pytest.mark.parametrize("mode", ["TEST_FORCE_FMA", "TEST_NO_TMA", "TEST_NO_FEW", "TEST_NO_SEED"])
+@pytest.mark.parametrize("mode", ["TEST_FORCE_FMA", "TEST_NO_TMA", "TEST_NO_FEW", "TEST_NO_SEED", "TEST_NO_PERSIST"])
 def test_alternative_kernel_paths_match_oracle(mode):
     """bf16 inputs on the fp32-FMA kernels; the tensor-core kernels with W staged by plain loads (the path
     taken when no tensor map can be encoded); every level on the tile kernel; the tile kernel without seeded
-    bounds (the path of vocabularies with fewer pieces than bound slots): chosen by the library's test switches."""
+    bounds; one launch per step of every level instead of the persistent expansion kernel: chosen by the library's
+    test switches."""
     from paper_2609_22098_b200 import binding
     wl = small("serve32", V=20000, B=5)
     rnd = Round(wl, seed=77)
@@ -494,3 +495,32 @@ def test_gpu_losslessness_chi_square():
         assert chisquare(h2[x1], p2 * nrow).pvalue > 1e-4
         checked += 1
     assert checked >= 2
+
+
+@pytest.mark.parametrize("T", [0.0, 1.0])
+@pytest.mark.parametrize("persist", [True, False])
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(T, persist):
+    """Bounded device-side waits: with the test switch that makes barriers expect one arrival more than will ever
+    come (and shortens the limit to a few thousand polls) the kernels give up, every call returns, the requests
+    are reported with TS_ERR_TIMEOUT, and the same context then runs an ordinary round correctly."""
+    from paper_2609_22098_b200 import binding
+    wl = small("serve32", V=20000, B=6)
+    rnd = Round(wl, seed=91)
+    base = 0 if persist else binding.TEST_NO_PERSIST
+    ts = make_gpu(wl, rnd.table, max_batch=rnd.B, test_mode=base)
+    orc = make_oracle(wl, rnd.table)
+    good = ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, 5)
+    Z, off = rnd.target_logits(good)
+    torch.cuda.synchronize()
+    ts.set_test_mode(base | binding.TEST_SHORT_WAITS | binding.TEST_LOST_ARRIVAL)
+    bad_tree = ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, 5)
+    torch.cuda.synchronize()
+    assert (bad_tree["status"].cpu() == -5).all(), bad_tree["status"]          # TS_ERR_TIMEOUT, and the call came back
+    if T > 0:
+        bad_verdict = ts.verify_tree(rnd.U, rnd.A, rnd.W, Z, off, rnd.anchor, good, T, 5)
+        torch.cuda.synchronize()
+        assert (bad_verdict["status"].cpu() == -5).all(), bad_verdict["status"]
+    ts.set_test_mode(base)
+    for rs in range(2):
+        st = check_round(ts, orc, rnd, T, round_seed=40 + rs)
+        assert st["nodes"] > 0
