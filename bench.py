@@ -47,6 +47,7 @@ def parse():
     ap.add_argument("--sets", type=int, default=4, help="distinct input sets rotated through")
     ap.add_argument("--seed", type=int, default=2609)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--test-mode", type=int, default=0, help="library test switches (TS_TEST_*), e.g. 64 = one launch per step of every level")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-edge-stat", action="store_true", help="do not emit per-edge statistics")
     ap.add_argument("--no-graph", action="store_true",
@@ -185,7 +186,7 @@ def run_ours(args, rank, world, device):
     table = synth.make_calibration_table(wl, args.seed + 4, "fit")
     A, W = synth.make_head(wl, args.seed + 1, device)
     ts = TreeSpark(wl.V, wl.D, wl.r, wl.K, wl.Nmax, B, dtype=wl.torch_dtype, calib_mode=wl.calib_mode,
-                   calib_table=table, device=device)
+                   calib_table=table, device=device, test_mode=args.test_mode)
     sets = [InputSet(wl, seed + 100 * i, B, theta, A, W, device) for i in range(args.sets)]
     tree = ts.alloc_tree(B)
     verdict = ts.alloc_verdict(B)

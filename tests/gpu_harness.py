@@ -3,6 +3,10 @@ compare under the stated tolerances.  Imported by the GPU tests, the smoke check
 parity check; nothing in the product imports it."""
 from __future__ import annotations
 
+import atexit
+import json
+import os
+
 import numpy as np
 import torch
 
@@ -15,9 +19,31 @@ from paper_2609_22098_b200.binding import TreeSpark
 # magnitude <= 32 (the inputs of every scalar are such logits).
 RTOL = 1e-5
 ATOL = 4e-6
-ACCEPT_MARGIN = 1e-5   # |u - rho| below this exempts an accept test (fp32-accumulated logits feed rho)
+ACCEPT_MARGIN = 1e-6   # |u - rho| below this exempts an accept test (the stated allowance; no walk of the suite sits in [1e-6, 1e-5))
 TREE_FLAGS = oracle.FLAG_NEAR_TOPK | oracle.FLAG_NEAR_THETA | oracle.FLAG_NEAR_CAP
 WALK_FLAGS = oracle.FLAG_NEAR_ACCEPT | oracle.FLAG_NEAR_CDF | oracle.FLAG_ZERO_MASS
+
+
+# Every compared round adds to these counts; when the scratch folder of a GPU run exists they are written there at
+# exit, so that the exemption rates behind the tolerances can be read off a test run (tests still assert ceilings).
+PARITY_TOTALS = dict(trees=0, trees_exempt=0, walks=0, walks_exempt=0, accept_band_walks=0, accept_band_disagree=0)
+_BY_FLAG = {}
+
+
+def _dump_totals():
+    out = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
+    if PARITY_TOTALS["trees"] and os.path.isdir(out):
+        with open(os.path.join(out, f"parity_exemptions_{os.getpid()}.json"), "w") as f:
+            json.dump(dict(totals=PARITY_TOTALS, by_flag=_BY_FLAG), f)
+
+
+atexit.register(_dump_totals)
+
+
+def _count_flags(flags, which):
+    for name in ("NEAR_TOPK", "NEAR_THETA", "NEAR_CAP", "NEAR_ACCEPT", "NEAR_CDF", "ZERO_MASS"):
+        if flags & getattr(oracle, "FLAG_" + name) & which:
+            _BY_FLAG[name] = _BY_FLAG.get(name, 0) + 1
 
 
 def make_oracle(wl, table):
@@ -92,6 +118,7 @@ class Round:
         self.wl = wl
         self.B = wl.B if B is None else B
         gen_device = gen_device or device
+        self.gen_device, self.device = gen_device, device
         self.table = synth.make_calibration_table(wl, seed + 4, table_kind) if wl.calib_mode == 1 else None
         A, W = synth.make_head(wl, seed + 1, gen_device)
         Ufull = synth.make_base_logits(wl, seed + 2, gen_device, B=self.B)
@@ -105,8 +132,13 @@ class Round:
         return dict(A=self.A.cpu(), W=self.W.cpu(), U=self.Ufull.cpu(), anchor=self.anchor.cpu(), theta=self.theta.cpu())
 
     def target_logits(self, tree, sigma=None):
-        """Z for the given (GPU) tree; generated once on the inputs' device."""
+        """Z for the given (GPU) tree; generated once, on the device the inputs were generated on."""
         wl = self.wl
+        if str(self.gen_device) == "cpu" and str(self.device) != "cpu":
+            c = self.cpu()
+            Z, off = synth.make_target_logits(wl, self.seed + 5, c["U"], c["A"], c["W"], c["anchor"], tree["n_nodes"].cpu(),
+                                              tree["tok"].cpu(), tree["depth"].cpu(), tree["node_hash"].cpu(), sigma=sigma)
+            return Z.to(self.device), off.to(self.device)
         return synth.make_target_logits(wl, self.seed + 5, self.Ufull, self.A, self.W, self.anchor, tree["n_nodes"],
                                         tree["tok"], tree["depth"], tree["node_hash"], sigma=sigma)
 
@@ -144,6 +176,7 @@ def check_round(ts, orc, rnd: Round, T, round_seed, reqs=None, want_edge=True, t
         stats["nodes"] += int(otrees[b]["n"])
         if exempt:
             stats["trees_exempt"] += 1
+            _count_flags(otrees[b]["flags"], TREE_FLAGS)
         else:
             ok_reqs.append(b)
     overd, _ = oracle.run_batch(verify_one, ok_reqs, threads)
@@ -154,9 +187,26 @@ def check_round(ts, orc, rnd: Round, T, round_seed, reqs=None, want_edge=True, t
         stats["acc"] += int(ov["acc_len"])
         if exempt:
             stats["walks_exempt"] += 1
+            _count_flags(ov["flags"], WALK_FLAGS)
+            if (ov["flags"] & WALK_FLAGS) == oracle.FLAG_NEAR_ACCEPT:
+                # exempt only by the accept margin: is the walk inside a ten times narrower band too?  If not, it sits
+                # in [1e-7, 1e-6): count it, and count whether the two sides disagree there
+                o6 = orc.verify_tree(c["U"][b].float().numpy(), Af, Wf,
+                                     Zc[int(offc[b]):int(offc[b]) + otrees[b]["n"] + 1].float().numpy(), int(c["anchor"][b]),
+                                     otrees[b], T, round_seed, b, accept_margin=1e-7)
+                if not (o6["flags"] & oracle.FLAG_NEAR_ACCEPT):
+                    stats["accept_band_walks"] = stats.get("accept_band_walks", 0) + 1
+                    same = (int(v["acc_len"][b]) == int(o6["acc_len"]) and int(v["bonus_tok"][b]) == int(o6["bonus"]) and
+                            v["acc_tok"][b, :int(o6["acc_len"])].tolist() == o6["acc_tok"][:int(o6["acc_len"])].tolist())
+                    if not same:
+                        stats["accept_band_disagree"] = stats.get("accept_band_disagree", 0) + 1
         if want_edge:
             n = int(otrees[b]["n"])
             ge = v["edge_stat"][b, :n].numpy()
             for i in range(n):
                 assert close(ge[i], ov["edge_stat"][i], rtol=2e-5, atol=1e-6), (b, i, ge[i], ov["edge_stat"][i])
+    for k in PARITY_TOTALS:
+        PARITY_TOTALS[k] += stats.get(k, 0)
+    print(f"parity: {stats['trees']} trees ({stats['trees_exempt']} exempt), {stats['walks']} walks ({stats['walks_exempt']} exempt), "
+          f"{stats.get('accept_band_walks', 0)} walks with |u - rho| in [1e-7, 1e-6) ({stats.get('accept_band_disagree', 0)} disagree)")
     return stats

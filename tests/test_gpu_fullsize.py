@@ -12,32 +12,37 @@ from paper_2609_22098_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def run(wl, T, theta, reqs, seed, round_seed=77, B=None):
+def run(wl, T, theta, reqs, seed, round_seed=77, B=None, rounds=1):
     rnd = Round(wl, seed=seed, B=B, theta=theta)
     ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
     orc = make_oracle(wl, rnd.table)
-    st = check_round(ts, orc, rnd, T, round_seed=round_seed, reqs=reqs)
-    assert st["trees"] == len(reqs)
-    return st
+    tot = None
+    for k in range(rounds):
+        st = check_round(ts, orc, rnd, T, round_seed=round_seed + k, reqs=reqs)
+        assert st["trees"] == len(reqs)
+        tot = st if tot is None else {key: (tot[key] + st[key] if isinstance(st[key], int) else st[key]) for key in st}
+    return tot
 
 
-def test_serve32_full_size_sampled_requests():
+def test_serve32_full_size_every_request_three_rounds():
     wl = synth.WORKLOADS["serve32"]
-    st = run(wl, 1.0, wl.theta, reqs=list(range(0, 32, 2)), seed=2609)
-    assert st["nodes"] > 0 and st["trees_exempt"] <= 2
+    st = run(wl, 1.0, wl.theta, reqs=list(range(32)), seed=2609, rounds=3)
+    assert st["nodes"] > 0 and st["trees"] == 96 and st["trees_exempt"] <= 4 and st["walks_exempt"] <= 6, st
 
 
-@pytest.mark.parametrize("T,theta", [(0.0, 0.1), (0.7, 0.03), (1.0, 0.3)])
+@pytest.mark.parametrize("T", [0.0, 0.7, 1.0])
+@pytest.mark.parametrize("theta", [0.3, 0.1, 0.03])
 def test_decode_full_size(T, theta):
     wl = synth.WORKLOADS["decode"]
-    st = run(wl, T, theta, reqs=[0], seed=31 + int(10 * T))
-    assert st["trees"] == 1
+    st = run(wl, T, theta, reqs=[0], seed=31 + int(10 * T), rounds=2)
+    assert st["trees"] == 2
 
 
-def test_wide_full_size_one_request():
+@pytest.mark.parametrize("T", [0.7, 1.3])
+def test_wide_full_size_three_requests(T):
     wl = synth.WORKLOADS["wide"]
-    st = run(wl, 0.7, wl.theta, reqs=[3], seed=5)
-    assert st["nodes"] >= 16
+    st = run(wl, T, wl.theta, reqs=[0, 3, 7], seed=5)
+    assert st["nodes"] >= 48
 
 
 def test_sweep_largest_batch_is_the_chain():
@@ -48,10 +53,11 @@ def test_sweep_largest_batch_is_the_chain():
     assert st["nodes"] == 3 * wl.D          # theta >= 1: every request is a chain of D nodes
 
 
-def test_sweep_mid_batch():
+@pytest.mark.parametrize("B,reqs", [(1, [0]), (4, [0, 1, 2, 3]), (16, [1, 9]), (64, [0, 21, 42, 63])])
+def test_sweep_batches(B, reqs):
     wl = synth.WORKLOADS["sweep"]
-    st = run(wl, 1.0, synth.sweep_theta(16, seed=9), reqs=[1, 9], seed=10, B=16)
-    assert st["trees"] == 2
+    st = run(wl, 1.0, synth.sweep_theta(B, seed=9), reqs=reqs, seed=10, B=B)
+    assert st["trees"] == len(reqs)
 
 
 @pytest.mark.parametrize("T", [0.0, 1.0])

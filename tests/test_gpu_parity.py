@@ -87,8 +87,10 @@ def test_round_matches_oracle(name, over, temps, thetas):
                 st = check_round(ts, orc, rnd, T, round_seed=1000 + rs)
                 for k in tot:
                     tot[k] += st[k]
-    assert tot["trees_exempt"] <= 0.15 * tot["trees"] + 2
-    assert tot["walks_exempt"] <= 0.3 * tot["walks"] + 1
+    # measured over the whole suite: 0.9 % of trees and 0.5 % of walks are exempt (none by the accept margin); a
+    # test of a few dozen rounds may see a handful
+    assert tot["trees_exempt"] <= 0.03 * tot["trees"] + 3
+    assert tot["walks_exempt"] <= 0.03 * tot["walks"] + 3
     assert tot["nodes"] > 0
 
 
@@ -118,7 +120,7 @@ def test_tiny_reference_config_100_rounds():
             st = check_round(ts, orc, rnd, T, round_seed=5000 + rs, want_edge=(rs % 10 == 0))
             for k in tot:
                 tot[k] += st[k]
-        assert tot["trees_exempt"] <= 5 and tot["walks_exempt"] <= 10, tot
+        assert tot["trees_exempt"] <= 4 and tot["walks_exempt"] <= 4, tot
         assert tot["nodes"] >= 100
 
 
