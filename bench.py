@@ -161,7 +161,9 @@ def tree_stats(wl, tree, verdict):
     return dict(nodes=int(n.sum()), parents=parents, u_rows=urows, z_rows=int((n + 1).sum()),
                 levels_used=sum(1 for p in per_level if p > 0), parents_per_level=per_level,
                 acc=int(verdict["acc_len"].sum()), walk_rows=int((verdict["acc_len"].long() + 1).sum()),
-                walk_passes=int(((verdict["flags"].long() >> 8) & 0xFFFF).sum()))
+                walk_passes=int(((verdict["flags"].long() >> 8) & 0xFFFF).sum()),
+                # a request's reductions follow one another, one grid step each: the longest chain bounds the walk's steps
+                walk_chain=int(((verdict["flags"].long() >> 8) & 0xFFFF).max()))
 
 
 def snapshot(tree, verdict):
@@ -295,7 +297,7 @@ def run_ours(args, rank, world, device):
     # walk: every residual reduction streams one target row and (recomputing the proposal) one base row;
     # its range of W is staged once per launch
     bytes_walk = mean("walk_passes") * 2 * row_b + w_b
-    alg = {"score_tile": bytes_score, "zrow_stats": bytes_zrows, "verify_walk": bytes_walk}
+    alg = {"score_tile": bytes_score, "expand_persistent": bytes_score, "zrow_stats": bytes_zrows, "verify_walk": bytes_walk}
     # DRAM bytes of the dominant kernel from a committed ncu capture of one round of this workload
     # (per launch: the round's bytes over the round's launches), null where none was captured
     traffic, traffic_src = None, None
@@ -319,7 +321,7 @@ def run_ours(args, rank, world, device):
                     "alg_bytes_per_launch": (a_bytes / max(kern[dom]["launches_per_round"], 1e-9)) if a_bytes else None,
                     "alg_bytes_per_round": a_bytes, "ms_per_launch": per_launch_ms,
                     "launches_per_round": kern[dom]["launches_per_round"], "share_of_kernel_time": kern[dom]["share"]}
-        if dom == "score_tile":
+        if dom in ("score_tile", "expand_persistent"):
             roofline["alg_bytes_per_round_w_every_level"] = bytes_score_w_levels
     sec = ms_per_step * 1e-3
     round_hbm = {"alg_bytes_all_rows": bytes_round_all, "alg_bytes_walk_rows_only": bytes_round_min,
@@ -345,7 +347,8 @@ def run_ours(args, rank, world, device):
         "parents_scored_per_s": world * mean("parents") / sec, "nodes_per_s": world * mean("nodes") / sec,
         "detail": {"mean_nodes_per_tree": mean("nodes") / B, "mean_parents_per_round": mean("parents"),
                    "mean_accepted_len": mean("acc") / B, "mean_z_rows": mean("z_rows"),
-                   "mean_walk_reductions": mean("walk_passes"),
+                   "mean_walk_reductions": mean("walk_passes"), "mean_longest_walk_chain": mean("walk_chain"),
+                   "launches_per_round": launches / max(args.steps, 1),
                    "parents_per_level": used[0]["parents_per_level"], "outputs_reproduced": same},
         "clocks": clocks, "gpu_launches": launches, "kernels": kern,
         # the per-kernel milliseconds come from a separate loop with an event pair around every launch (no chaining

@@ -94,6 +94,8 @@ int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags);
  *   TS_TEST_NO_SEED       the tensor-core scoring kernel runs without seed bounds (no seed kernel ahead of it)
  *   TS_TEST_NO_PERSIST    ts_expand_tree launches one kernel per step of every level instead of the
  *                         persistent kernel that runs all levels (the path of configurations it does not fit)
+ *   TS_TEST_NO_UMMA       the scanning threads of the tensor-core scoring kernel load the base logits themselves
+ *                         instead of receiving them through the MMA (the path of batches above 32 requests)
  *   TS_TEST_SHORT_WAITS   bounded waits give up after 4096 polls instead of 2^22
  *   TS_TEST_LOST_ARRIVAL  the walk's grid barriers and the scoring kernel's operand barrier expect one
  *                         arrival more than will come: the waits run out, the kernels return, and the
@@ -105,6 +107,7 @@ int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags);
 #define TS_TEST_SHORT_WAITS 16u
 #define TS_TEST_LOST_ARRIVAL 32u
 #define TS_TEST_NO_PERSIST 64u
+#define TS_TEST_NO_UMMA 128u
 int32_t ts_set_test_mode(ts_ctx* ctx, uint32_t flags);
 
 /* Bytes of workspace the hot calls need for a batch of `batch` requests (<= max_batch). */

@@ -30,6 +30,7 @@ constexpr int SLOT_STRIDE = 32;
 // the parts of at most SEED_SPLIT_PARENTS parents meet in a scratch of NSEED_MAX candidates per part.
 constexpr int SEED_PARTS_MAX = 16, SEED_SPLIT_PARENTS = 256, NSEED_MAX = 32;
 constexpr size_t SEED_CAND_WORDS = (size_t)SEED_SPLIT_PARENTS * SEED_PARTS_MAX * NSEED_MAX * 2;
+constexpr int UMMA_REQ = 32;         // requests whose base logits can ride through the tensor cores (rows of one extra B-operand slab)
 constexpr int FEW_MAX = 8;           // levels with at most this many parents go to the few-parents scoring kernel
 constexpr int SCORE_THREADS = 128;   // one parent per thread; every thread scans the CTA's whole tile
 constexpr int CHUNK = 16;            // tokens per coarse generator call
@@ -71,6 +72,8 @@ struct ts_ctx {
   // driver's encoder is not available, the kernel stages W with plain loads
   alignas(64) unsigned char tmapW[128];
   const void* tmapW_ptr;
+  alignas(64) unsigned char tmapU[128];   // tensor map of the base logits last expanded with ([request][depth][token] boxes)
+  const void* tmapU_ptr; int tmapU_B;
   int tma_state;   // 0 not tried yet, 1 encoder found, -1 unavailable
   int walk_pdl;    // -1: the driver refused a cooperative launch with programmatic serialization
   int persist_pdl; // the same for the persistent expansion kernel

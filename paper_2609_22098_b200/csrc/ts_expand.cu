@@ -223,6 +223,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
     { ProfScope ps(ctx, K_SEED, st); e = launch_seed(ctx, sa, st); }
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(seed)", e);
     sa.utop = (uint2*)(ws + L.utop); sa.scout_live = a.req_npar; sa.scout_B = B; sa.scout_depth = 1;
+    sa.u_depth = 0; sa.u_B = B;
     PersistArgs pa{};
     pa.on = 1; pa.nlevels = c.D; pa.ex = a; pa.barrier = a.ex_barrier;
     pa.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
@@ -245,6 +246,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
     ScoreExtras ex;
     ex.thr0_ready = scouted_prev;
     const bool scout = seeds_on && on_mma && d + 1 < c.D;
+    ex.u_depth = d; ex.u_B = B;
     if (scout) { ex.utop = (uint2*)(ws + L.utop); ex.scout_live = a.req_npar; ex.scout_B = B; ex.scout_depth = d + 1; }
     e = launch_score(ctx, (float*)(ws + L.rec), L.rec_cap, (int*)(ws + L.err), U, A, W, 0, a.lvl_count + d,
                      a.lst_req[cur], a.lst_depth[cur], a.lst_token[cur],

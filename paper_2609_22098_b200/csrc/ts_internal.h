@@ -33,6 +33,11 @@ struct ScoreArgs {
   // every request b < scout_B that has parents in this launch (scout_live[b] > 0), and leaves (value, token)
   // at utop[(b * D + scout_depth) * ntiles + tile]: the next level's seed bounds are made from those.
   const int* scout_live; int scout_B, scout_depth; uint2* utop;
+  // Base logits through the tensor cores (expansion only, at most UMMA_REQ requests): all parents of the launch
+  // sit at depth u_depth (-1: not so; the persistent form takes the level instead), and the base logits of
+  // requests 0 .. u_B-1 at that depth enter the MMA as extra rows of the B operand against one-hot columns of
+  // the A operand, fetched by bulk-tensor loads: the scanning threads load no base logits at all.
+  int u_depth, u_B;
   unsigned* seed_cnt;    // [SEED_SPLIT_PARENTS] arrival counters of the seed kernel (zero between launches)
   unsigned* seed_cand;   // [SEED_SPLIT_PARENTS][SEED_PARTS_MAX][NSEED_MAX][2] candidates (value, token) of the parts
   unsigned* thr0;   // [2][cap]: seed bounds (logit, key) per parent, written ahead of the launch; nullptr: none
@@ -67,6 +72,7 @@ void set_seed_pointers(const ts_ctx* ctx, ScoreArgs& a);
 struct ScoreExtras {
   bool thr0_ready = false;
   const int* scout_live = nullptr; int scout_B = 0, scout_depth = -1; uint2* utop = nullptr;
+  int u_depth = -1, u_B = 0;
 };
 cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const void* U, const void* A, const void* W,
                          int P, const int* P_dev, const int* p_req, const int* p_depth, const int* p_token,

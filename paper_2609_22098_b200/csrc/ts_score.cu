@@ -144,6 +144,7 @@ ScoreArgs make_score_args(const ts_ctx* ctx, float* rec, int cap, int* err, cons
   a.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
   a.thr = thr_base(ctx, rec, cap); a.slots = a.thr + 2 * (size_t)cap;
   a.thr0 = nullptr;
+  a.u_depth = -1; a.u_B = 0;
   return a;
 }
 
@@ -179,6 +180,7 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
       e = launch_seed(ctx, a, st);
       if (e != cudaSuccess) return e;
     }
+    if (extras) { a.u_depth = extras->u_depth; a.u_B = extras->u_B; }
     if (extras && extras->utop) {
       a.utop = extras->utop; a.scout_live = extras->scout_live; a.scout_B = extras->scout_B; a.scout_depth = extras->scout_depth;
     }

@@ -57,7 +57,8 @@ constexpr int WBLK = 128;               // tokens per bulk-load barrier of W (tw
 constexpr int NBUF = 8;                 // accumulator buffers of BLK_N columns in tensor memory: two per split
 constexpr uint32_t TMEM_COLS = NBUF * BLK_N;
 constexpr int MAX_BLK = 32;             // W load barriers (WBLK tokens each) of the largest tile (4096 tokens)
-constexpr int QCAP = 256;               // entries per candidate queue (power of two)
+constexpr int QCAP = 128;               // entries per candidate queue (power of two)
+constexpr int NUB = 4;                  // ring of base-logit slabs (UMMA_REQ rows x 64 tokens) ahead of the MMAs
 constexpr uint32_t KIND_TOP = 1u, KIND_KEY = 2u;
 
 template <int ID, int NT>
@@ -126,7 +127,9 @@ __device__ __forceinline__ void select_candidate(const ScoreArgs& a, const SelSh
   }
 }
 
-__global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma, const __grid_constant__ PersistArgs pa) {
+template <bool UMMA>
+__global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma, const __grid_constant__ PersistArgs pa,
+                                                                   const __grid_constant__ CUtensorMap tmU) {
   extern __shared__ unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // The preamble below (shared-memory carve-up, tensor-memory allocation, barriers, bulk loads of W, noise
@@ -143,20 +146,24 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   unsigned char* sm = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* Ws = sm;
   unsigned char* As = Ws + (size_t)nslab * slab_bytes;
-  float* ghi = reinterpret_cast<float*>(As + (size_t)(rp / 64) * a_slab_bytes);
+  // (one more slab of the A tile holds the one-hot request columns, and a ring of slabs the base logits they select)
+  unsigned char* Us = As + (size_t)(rp / 64 + 1) * a_slab_bytes;   // [NUB][UMMA_REQ rows][128 B], 128-byte swizzle
+  float* ghi = reinterpret_cast<float*>(Us + (size_t)NUB * UMMA_REQ * 128);
   SelShared sh;
   sh.q = reinterpret_cast<uint4*>(ghi + 512);                                   // 16-byte aligned
   sh.lists = reinterpret_cast<float*>(sh.q + NSEL * QCAP);
   sh.lthr = sh.lists + (size_t)128 * 5 * K;
   sh.best = sh.lthr + 2 * 128;
-  float* s_part = const_cast<float*>(sh.best) + 2 * EPI_S * 128;                // [EPI_S][128][4]: m, s0, sT of every (split, row)
-  volatile unsigned* s_thr = reinterpret_cast<volatile unsigned*>(s_part + EPI_S * 128 * 4);   // [group parity][2][128]
+  float* s_part = const_cast<float*>(sh.best) + 2 * EPI_S * 128;                // [3][EPI_S][128]: m, s0, sT of every (split, row)
+  volatile unsigned* s_thr = reinterpret_cast<volatile unsigned*>(s_part + 3 * EPI_S * 128);   // [group parity][2][128]
   uint64_t* bars = reinterpret_cast<uint64_t*>(const_cast<unsigned*>(s_thr) + 512);
   uint64_t* a_full = bars;            // scanning threads -> MMA: the A tile of this group is in place
   uint64_t* t_full = bars + 1;             // [NBUF] MMA -> scan: accumulator buffer written
   uint64_t* t_empty = bars + 1 + NBUF;     // [NBUF] scan -> MMA: accumulator buffer drained
   uint64_t* w_full = bars + 1 + 2 * NBUF;  // [MAX_BLK] W slabs of block nb landed
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(w_full + MAX_BLK);
+  uint64_t* u_full = w_full + MAX_BLK;     // [NUB] base-logit slab landed
+  uint64_t* u_free = u_full + NUB;         // [NUB] the MMAs that read the slab are done
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(u_free + NUB);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   volatile int* s_done = reinterpret_cast<volatile int*>(s_tmem + 2);             // scanning warps finished (cumulative)
   sh.q_head = reinterpret_cast<volatile unsigned*>(s_tmem + 4);
@@ -188,6 +195,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
     *s_done = 0;
     for (int i = 0; i < NSEL; ++i) { sh.q_head[i] = 0u; sh.q_tail[i] = 0u; }
     if (use_tma) for (int i = 0; i < nblk_w; ++i) mbar_init(w_full + i, 1);
+    for (int i = 0; i < NUB; ++i) { mbar_init(u_full + i, 1); mbar_init(u_free + i, 1); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // W tile by bulk-tensor loads, one barrier per block of 128 tokens so that the first MMAs start while
     // the rest of the tile is still in flight; tokens past V and rows past r arrive as zeros.  Issued here,
@@ -227,6 +235,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   pdl_launch_dependents();
   const bool persist = pa.on != 0;
   int gg = 0;               // groups scanned so far, over all levels (barrier parities and use counts run on)
+  uint32_t ul = 0;          // block pairs of all groups before this one (MMA issuer: slot and use of their base-logit slabs)
   unsigned gen = 0;         // grid barriers passed
   bool dead = false;        // a bounded wait ran out somewhere
   bool w_issued = use_tma && early_w;   // bulk loads of the W tile are (or were) in flight
@@ -239,6 +248,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   const uint64_t* lp_hash = persist ? pa.ex.lst_hash[cur] : a.p_hash;
   const int scout_depth = persist ? lvl + 1 : a.scout_depth;
   const bool scout = a.utop != nullptr && scout_depth < a.D;
+  const int u_depth = persist ? lvl : a.u_depth;   // UMMA: the depth every parent of this level sits at
   const int P = persist ? __ldcg(pa.ex.lvl_count + lvl) : (a.P_dev ? *a.P_dev : a.P);   // may be 0: an empty level only tears down
   if (use_tma && !early_w && P > 0 && lvl == 0) { if (tid == 0) issue_w(); w_issued = true; }
 
@@ -275,6 +285,24 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
         uint4 v = make_uint4(0, 0, 0, 0);
         if (p < P && ck * 8 < r) v = __ldg(reinterpret_cast<const uint4*>(Ag + (size_t)__ldcg(lp_token + p) * r + ck * 8));
         *reinterpret_cast<uint4*>(As + (size_t)(ck >> 3) * a_slab_bytes + rr * 128 + (((ck & 7) ^ (rr & 7)) << 4)) = v;
+      }
+      if (UMMA) {
+        // one more K-slab of the A tile: column b of row rr is 1 when the row's parent belongs to request b, so the
+        // MMA adds that request's base logits (rows of the base-logit slab) to the row's bias
+        for (int idx = e; idx < 128 * 8; idx += EPI_WARPS * 32) {
+          const int rr = idx >> 3, ck = idx & 7;
+          const int p = R > 1 ? rr % per : g * 128 + rr;
+          uint4 v = make_uint4(0, 0, 0, 0);
+          if (p < P) {
+            const int b = __ldcg(lp_req + p);
+            if ((b >> 3) == ck) {
+              const uint32_t one = 0x3F80u << (16 * (b & 1));   // bf16 1.0 in the half-word of column b
+              const int w = (b & 7) >> 1;
+              v.x = w == 0 ? one : 0u; v.y = w == 1 ? one : 0u; v.z = w == 2 ? one : 0u; v.w = w == 3 ? one : 0u;
+            }
+          }
+          *reinterpret_cast<uint4*>(As + (size_t)(rp / 64) * a_slab_bytes + rr * 128 + ((ck ^ (rr & 7)) << 4)) = v;
+        }
       }
       fence_async_smem();
       mbar_arrive(a_full);
@@ -335,11 +363,11 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       auto prefetch_block = [&](int nb) {
         if (active && nb < nblk) asm volatile("prefetch.global.L2 [%0];" ::"l"(Urow + t0 + nb * BLK_N));
       };
-      prefetch_block(s);
+      if (!UMMA) prefetch_block(s);
       for (int nb = s; nb < nblk && alive; nb += EPI_S) {
         const int j = nb / EPI_S, h = j & 1;
         const int tb = s + EPI_S * h, u = gg * ((nuse + 1 - h) >> 1) + (j >> 1);   // buffer, and how often it was used before
-        prefetch_block(nb + EPI_S);
+        if (!UMMA) prefetch_block(nb + EPI_S);
         {
           int ok = 1;
           if (lane == 0) ok = mbar_wait(t_full + tb, u & 1, s_abort, a.err, wait_limit) ? 1 : 0;
@@ -356,24 +384,26 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
           if (!active) continue;
           const int v0 = t0 + cg * 16;
           const int valid = min(16, V - v0);   // 8 or 16: V and v0 are multiples of 8
-          // this chunk's base logits were requested one chunk ago; request the next owned chunk's now
-          const uint4 u0 = have_next ? nx0 : __ldg(reinterpret_cast<const uint4*>(Urow + v0));
-          const uint4 u1 = have_next ? nx1 : (valid > 8 ? __ldg(reinterpret_cast<const uint4*>(Urow + v0 + 8)) : make_uint4(0, 0, 0, 0));
-          {
-            const int cgn = (c + R < BLK_N / 16) ? cg + R : (nb + EPI_S) * (BLK_N / 16) + rho;   // the next chunk this warp owns
-            const int vn = t0 + cgn * 16;
-            have_next = (cgn * 16 < tlen);
-            if (have_next) {
-              nx0 = __ldg(reinterpret_cast<const uint4*>(Urow + vn));
-              nx1 = (V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8)) : make_uint4(0, 0, 0, 0);
+          if (!UMMA) {
+            // this chunk's base logits were requested one chunk ago; request the next owned chunk's now
+            const uint4 u0 = have_next ? nx0 : __ldg(reinterpret_cast<const uint4*>(Urow + v0));
+            const uint4 u1 = have_next ? nx1 : (valid > 8 ? __ldg(reinterpret_cast<const uint4*>(Urow + v0 + 8)) : make_uint4(0, 0, 0, 0));
+            {
+              const int cgn = (c + R < BLK_N / 16) ? cg + R : (nb + EPI_S) * (BLK_N / 16) + rho;   // the next chunk this warp owns
+              const int vn = t0 + cgn * 16;
+              have_next = (cgn * 16 < tlen);
+              if (have_next) {
+                nx0 = __ldg(reinterpret_cast<const uint4*>(Urow + vn));
+                nx1 = (V - vn > 8) ? __ldg(reinterpret_cast<const uint4*>(Urow + vn + 8)) : make_uint4(0, 0, 0, 0);
+              }
             }
-          }
-          {
-            float ub[16];
-            unpack_bf16x8(u0, ub);
-            unpack_bf16x8(u1, ub + 8);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] += ub[i];
+            {
+              float ub[16];
+              unpack_bf16x8(u0, ub);
+              unpack_bf16x8(u1, ub + 8);
+  #pragma unroll
+              for (int i = 0; i < 16; ++i) acc[i] += ub[i];
+            }
           }
           if (valid < 16) {   // warp-uniform and rare (the vocabulary's last chunk): padding that loses every comparison
 #pragma unroll
@@ -479,7 +509,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
         if (lane == 0) mbar_arrive(t_empty + tb);
       }
       // this piece's sums; the row's record is put together when the group is over
-      *reinterpret_cast<float4*>(s_part + ((size_t)s * 128 + row) * 4) = make_float4(m, s0, sT, 0.f);
+      s_part[(0 * EPI_S + s) * 128 + row] = m; s_part[(1 * EPI_S + s) * 128 + row] = s0; s_part[(2 * EPI_S + s) * 128 + row] = sT;
       __threadfence_block();
       __syncwarp();
       if (lane == 0) atomicAdd((int*)s_done, alive ? 1 : (1 << 20));   // one tick per warp per group (a large one releases the others after a failed wait)
@@ -577,6 +607,71 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       const uint32_t ws_addr = smem_u32(Ws), as_addr = smem_u32(As);
       if (mbar_wait(a_full, gg & 1, s_abort, a.err, wait_limit)) {
         tc_fence_after();
+        if (UMMA) {
+          // Blocks go to the tensor cores in pairs (blocks 2x and 2x + 1 belong to neighbouring splits, whose accumulator
+          // buffers are neighbours in tensor memory, so one N = 128 instruction per K step fills both: issuing is what
+          // limits this warp).  A pair needs the base-logit slabs of its 128 tokens: two bulk-tensor loads into one of
+          // NUP ring slots (pair x of the kernel's running count uses slot x % NUP; a slot is free again as soon as the
+          // MMAs that read it are done, long before the blocks are scanned).  Within the window of NUP requested pairs,
+          // whichever pair has its buffers drained and its slabs landed is issued.
+          constexpr int NUP = NUB / 2;
+          constexpr uint32_t SLAB = (uint32_t)UMMA_REQ * 128u;
+          const uint32_t us_addr = smem_u32(Us);
+          const int KU = UMMA_REQ / 16;   // extra K steps: the one-hot columns against the slabs' rows
+          const int npair = (nblk + 1) / 2;
+          int base = 0, unext = 0;        // first pair not yet issued; first pair whose slabs are not yet requested
+          uint32_t done = 0;              // bit w: pair base + w is issued
+          uint32_t spin = 0;
+          while (base < npair) {
+            while (unext < npair && unext < base + NUP) {
+              const uint32_t gx = ul + (uint32_t)unext, slot = gx % NUP, use = gx / NUP;
+              if (use >= 1 && !mbar_test_wait(u_free + slot, (use - 1) & 1)) break;
+              const bool two = 2 * unext + 1 < nblk;
+              mbar_expect_tx(u_full + slot, two ? 2u * SLAB : SLAB);
+              tma_load_box3(Us + (size_t)slot * 2 * SLAB, &tmU, t0 + 2 * unext * BLK_N, u_depth, 0, u_full + slot);
+              if (two) tma_load_box3(Us + (size_t)slot * 2 * SLAB + SLAB, &tmU, t0 + (2 * unext + 1) * BLK_N, u_depth, 0, u_full + slot);
+              ++unext;
+            }
+            bool progressed = false;
+#pragma unroll
+            for (int w = 0; w < NUP; ++w) {
+              const int pr = base + w;
+              if (pr >= unext || ((done >> w) & 1u)) continue;
+              const int nb = 2 * pr;
+              const bool two = nb + 1 < nblk;
+              const int sp = nb % EPI_S;                      // even: the pair's splits are sp and sp + 1
+              const int j = nb / EPI_S, h = j & 1, tb = sp + EPI_S * h;
+              const int nuse0 = (nblk - sp + EPI_S - 1) / EPI_S, nuse1 = (nblk - sp - 1 + EPI_S - 1) / EPI_S;
+              const int u0 = gg * ((nuse0 + 1 - h) >> 1) + (j >> 1), u1 = gg * ((nuse1 + 1 - h) >> 1) + (j >> 1);
+              if (u0 >= 1 && !mbar_test_wait(t_empty + tb, (u0 - 1) & 1)) continue;
+              if (two && u1 >= 1 && !mbar_test_wait(t_empty + tb + 1, (u1 - 1) & 1)) continue;
+              if (use_tma && gg == 0 && !mbar_test_wait(w_full + nb * BLK_N / WBLK, 0)) continue;
+              const uint32_t gx = ul + (uint32_t)pr, slot = gx % NUP;
+              if (!mbar_test_wait(u_full + slot, (gx / NUP) & 1)) continue;
+              tc_fence_after();
+              const uint32_t idesc = instr_desc(two ? 2 * BLK_N : BLK_N);
+              const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
+              const uint32_t wb = ws_addr + (uint32_t)nb * slab_bytes, ub = us_addr + slot * 2u * SLAB;
+              for (int ks = 0; ks < rp / 16; ++ks)
+                mma_bf16(d_tmem, smem_desc(as_addr + (uint32_t)(ks >> 2) * a_slab_bytes + (uint32_t)(ks & 3) * 32u, 16u, 1024u),
+                         smem_desc(wb + (uint32_t)ks * 2048u, slab_bytes, 1024u), idesc, ks > 0 ? 1u : 0u);
+              for (int ks = 0; ks < KU; ++ks)
+                mma_bf16(d_tmem, smem_desc(as_addr + (uint32_t)(rp / 64) * a_slab_bytes + (uint32_t)ks * 32u, 16u, 1024u),
+                         smem_desc(ub + (uint32_t)ks * 2048u, SLAB, 1024u), idesc, 1u);
+              mma_commit(t_full + tb);
+              if (two) mma_commit(t_full + tb + 1);
+              mma_commit(u_free + slot);
+              done |= 1u << w;
+              progressed = true;
+            }
+            while (done & 1u) { done >>= 1; ++base; }
+            if (progressed) { spin = 0; continue; }
+            if (*s_abort) break;
+            if (++spin > wait_limit) { *s_abort = 1; if (a.err) atomicExch(a.err, 1); break; }
+            if (spin > 8) __nanosleep(32);
+          }
+          ul += (uint32_t)npair;
+        } else {
         // each split's pipeline advances on its own: whichever buffer is drained (and whose W block has landed) is refilled
         int nxt[EPI_S];
 #pragma unroll
@@ -592,8 +687,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
             const int nuse = (nblk - sp + EPI_S - 1) / EPI_S;
             const int j = nb / EPI_S, h = j & 1, tb = sp + EPI_S * h;
             const int u = gg * ((nuse + 1 - h) >> 1) + (j >> 1);
-            if (u >= 1 && !mbar_try_wait(t_empty + tb, (u - 1) & 1)) continue;
-            if (use_tma && gg == 0 && !mbar_try_wait(w_full + nb * BLK_N / WBLK, 0)) continue;
+            if (u >= 1 && !mbar_test_wait(t_empty + tb, (u - 1) & 1)) continue;
+            if (use_tma && gg == 0 && !mbar_test_wait(w_full + nb * BLK_N / WBLK, 0)) continue;
             tc_fence_after();
             const uint32_t idesc = instr_desc(BLK_N);
             const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
@@ -612,6 +707,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
           if (++spin > wait_limit) { *s_abort = 1; if (a.err) atomicExch(a.err, 1); break; }
           if (spin > 8) __nanosleep(32);
         }
+        }
       }
     }
     // ---- the group is over: one record per row -----------------------------------------------------------
@@ -627,7 +723,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
         float m = -INFINITY, s0 = 0.f, sT = 0.f;
 #pragma unroll
         for (int s = 0; s < EPI_S; ++s) {
-          const float4 h = *reinterpret_cast<const float4*>(s_part + ((size_t)s * 128 + row) * 4);
+          const float3 h = make_float3(s_part[(0 * EPI_S + s) * 128 + row], s_part[(1 * EPI_S + s) * 128 + row], s_part[(2 * EPI_S + s) * 128 + row]);
           if (h.x == -INFINITY) continue;
           if (h.x > m) { const float d = m - h.x; s0 *= __expf(d); sT *= __expf(d * invT); m = h.x; }
           const float d = h.x - m;
@@ -699,8 +795,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
 static size_t mma_fixed_smem(const ts_config& c) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
   const size_t K = (size_t)c.K;
-  return (rp / 64) * 128 * 128 + 512 * 4 + (size_t)NSEL * QCAP * 16 + 128 * 5 * K * 4 + 2 * 128 * 4 + 2 * EPI_S * 128 * 4 +
-         EPI_S * 128 * 16 + 512 * 4 + (1 + 2 * NBUF + MAX_BLK) * 8 + 64 + 1024;
+  return (rp / 64 + 1) * 128 * 128 + (size_t)NUB * UMMA_REQ * 128 + 512 * 4 + (size_t)NSEL * QCAP * 16 + 128 * 5 * K * 4 + 2 * 128 * 4 +
+         2 * EPI_S * 128 * 4 + 3 * EPI_S * 128 * 4 + 512 * 4 + (1 + 2 * NBUF + MAX_BLK + 2 * NUB) * 8 + 64 + 1024;
 }
 
 // tile size for the tensor-core path: W tile + the rest within the shared-memory limit,
@@ -724,7 +820,9 @@ bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out
 }
 
 cudaError_t score_mma_setup(ts_ctx* ctx) {
-  return cudaFuncSetAttribute(score_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
+  cudaError_t e = cudaFuncSetAttribute(score_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(score_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
 }
 
 // Tensor map of W = [r][V] bf16 for boxes of 64 tokens x rp rows with the 128-byte swizzle the MMA's
@@ -766,20 +864,51 @@ bool w_tensor_map(ts_ctx* ctx, const void* W) {
   return true;
 }
 
+// Tensor map of the base logits U = [B][D][V] bf16 for boxes of 64 tokens x 1 depth x UMMA_REQ requests (requests past
+// B arrive as zeros), in the 128-byte swizzle of a B-operand slab whose K rows are the requests.
+static bool u_tensor_map(ts_ctx* ctx, const void* U, int B) {
+  if (ctx->tma_state != 1 || !g_encode || ((uintptr_t)U & 15u) != 0 || B < 1 || B > UMMA_REQ) return false;
+  if (ctx->tmapU_ptr == U && ctx->tmapU_B == B) return true;
+  const ts_config& c = ctx->cfg;
+  const cuuint64_t gdim[3] = {(cuuint64_t)c.V, (cuuint64_t)c.D, (cuuint64_t)B};
+  const cuuint64_t gstride[2] = {(cuuint64_t)c.V * 2, (cuuint64_t)c.V * 2 * (cuuint64_t)c.D};
+  const cuuint32_t box[3] = {64u, 1u, (cuuint32_t)UMMA_REQ};
+  const cuuint32_t estr[3] = {1u, 1u, 1u};
+  CUtensorMap tm;
+  const CUresult rc = g_encode(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(U), gdim, gstride, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (rc != CUDA_SUCCESS) return false;
+  memcpy(ctx->tmapU, &tm, sizeof(tm));
+  ctx->tmapU_ptr = U; ctx->tmapU_B = B;
+  return true;
+}
+
+// base logits through the tensor cores: every parent at one known depth, few enough requests, bulk-tensor loads available
+static bool use_umma(ts_ctx* c, const ScoreArgs& a, bool persist, int use_tma) {
+  return use_tma && (persist || a.u_depth >= 0) && a.u_B >= 1 && a.u_B <= UMMA_REQ && !(c->test_mode & TS_TEST_NO_UMMA) &&
+         u_tensor_map(c, a.U, a.u_B);
+}
+
 cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st) {
   ts_ctx* c = const_cast<ts_ctx*>(ctx);
   const int use_tma = w_tensor_map(c, a.W) ? 1 : 0;
   CUtensorMap tm;
   memcpy(&tm, c->tmapW, sizeof(tm));
   PersistArgs pa{};   // pa.on = 0: one scan
-  const cudaError_t e = launch_kernel(score_mma_kernel, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma, pa);
+  CUtensorMap tu;
+  memset(&tu, 0, sizeof(tu));
+  const bool umma = use_umma(c, a, false, use_tma);
+  if (umma) memcpy(&tu, c->tmapU, sizeof(tu));
+  const cudaError_t e = umma ? launch_kernel(score_mma_kernel<true>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma, pa, tu)
+                             : launch_kernel(score_mma_kernel<false>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma, pa, tu);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // Shared memory that is idle between two scans (queues, lists, local thresholds, published bests, partial sums):
 // the merge and the level step of the persistent form work in it.
 static size_t persist_overlay_bytes(const ts_config& c) {
-  return (size_t)NSEL * QCAP * 16 + (size_t)128 * 5 * c.K * 4 + 2 * 128 * 4 + 2 * EPI_S * 128 * 4 + EPI_S * 128 * 16;
+  return (size_t)NSEL * QCAP * 16 + (size_t)128 * 5 * c.K * 4 + 2 * 128 * 4 + 2 * EPI_S * 128 * 4 + 3 * EPI_S * 128 * 4;
 }
 
 bool persistent_supported(const ts_ctx* ctx, int B) {
@@ -796,19 +925,24 @@ cudaError_t launch_expand_persistent(const ts_ctx* ctx, const ScoreArgs& a, cons
   int use_tma = w_tensor_map(c, a.W) ? 1 : 0;
   CUtensorMap tm;
   memcpy(&tm, c->tmapW, sizeof(tm));
-  void* kargs[] = {(void*)&a, (void*)&tm, (void*)&use_tma, (void*)&pa};
+  CUtensorMap tu;
+  memset(&tu, 0, sizeof(tu));
+  const bool umma = use_umma(c, a, true, use_tma);
+  if (umma) memcpy(&tu, c->tmapU, sizeof(tu));
+  const void* fn = umma ? (const void*)score_mma_kernel<true> : (const void*)score_mma_kernel<false>;
+  void* kargs[] = {(void*)&a, (void*)&tm, (void*)&use_tma, (void*)&pa, (void*)&tu};
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(a.ntiles); cfg.blockDim = dim3(MMA_THREADS); cfg.dynamicSmemBytes = ctx->tile.smem; cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeCooperative; attr[0].val.cooperative = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization; attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = c->persist_pdl >= 0 ? 2 : 1;
-  cudaError_t e = cudaLaunchKernelExC(&cfg, (const void*)score_mma_kernel, kargs);
+  cudaError_t e = cudaLaunchKernelExC(&cfg, fn, kargs);
   if (e != cudaSuccess && cfg.numAttrs == 2) {   // not accepted together: remember, and launch cooperative only
     (void)cudaGetLastError();
     c->persist_pdl = -1;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelExC(&cfg, (const void*)score_mma_kernel, kargs);
+    e = cudaLaunchKernelExC(&cfg, fn, kargs);
   }
   return e != cudaSuccess ? e : cudaGetLastError();
 }

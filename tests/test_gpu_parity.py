@@ -162,7 +162,7 @@ def test_back_to_back_rounds_reproduce_bitwise():
             assert torch.equal(verdict["acc_tok"].cpu()[b, :L], v0["acc_tok"][b, :L]), (i, b)
 
 
-@pytest.mark.parametrize("mode", ["TEST_FORCE_FMA", "TEST_NO_TMA", "TEST_NO_FEW", "TEST_NO_SEED", "TEST_NO_PERSIST"])
+@pytest.mark.parametrize("mode", ["TEST_FORCE_FMA", "TEST_NO_TMA", "TEST_NO_FEW", "TEST_NO_SEED", "TEST_NO_PERSIST", "TEST_NO_UMMA"])
 def test_alternative_kernel_paths_match_oracle(mode):
     """bf16 inputs on the fp32-FMA kernels; the tensor-core kernels with W staged by plain loads (the path
     taken when no tensor map can be encoded); every level on the tile kernel; the tile kernel without seeded
