@@ -47,7 +47,7 @@ def parse():
     ap.add_argument("--sets", type=int, default=4, help="distinct input sets rotated through")
     ap.add_argument("--seed", type=int, default=2609)
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--test-mode", type=int, default=0, help="library test switches (TS_TEST_*), e.g. 64 = one launch per step of every level")
+    ap.add_argument("--test-mode", type=int, default=0, help="library test switches (TS_TEST_*), e.g. 64 = every level of the expansion inside one cooperative launch")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-edge-stat", action="store_true", help="do not emit per-edge statistics")
     ap.add_argument("--no-graph", action="store_true",

@@ -92,8 +92,9 @@ int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags);
  *   TS_TEST_NO_TMA        the tensor-core kernels stage W with plain loads (no tensor map)
  *   TS_TEST_NO_FEW        levels with few parents run on the tile kernel too
  *   TS_TEST_NO_SEED       the tensor-core scoring kernel runs without seed bounds (no seed kernel ahead of it)
- *   TS_TEST_NO_PERSIST    ts_expand_tree launches one kernel per step of every level instead of the
- *                         persistent kernel that runs all levels (the path of configurations it does not fit)
+ *   TS_TEST_PERSIST       ts_expand_tree runs every level inside one cooperative launch (scan, merge and level
+ *                         step separated by grid barriers; nothing is launched for empty levels) instead of one
+ *                         launch per step of every level, where the configuration fits that kernel
  *   TS_TEST_NO_UMMA       the scanning threads of the tensor-core scoring kernel load the base logits themselves
  *                         instead of receiving them through the MMA (the path of batches above 32 requests)
  *   TS_TEST_SHORT_WAITS   bounded waits give up after 4096 polls instead of 2^22
@@ -106,7 +107,7 @@ int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags);
 #define TS_TEST_NO_SEED 8u
 #define TS_TEST_SHORT_WAITS 16u
 #define TS_TEST_LOST_ARRIVAL 32u
-#define TS_TEST_NO_PERSIST 64u
+#define TS_TEST_PERSIST 64u
 #define TS_TEST_NO_UMMA 128u
 int32_t ts_set_test_mode(ts_ctx* ctx, uint32_t flags);
 

@@ -212,7 +212,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(init)", e);
   const size_t level_smem = level_smem_bytes(c);   // opted into at ts_create when above 48 KB
   const bool seeds_on = ctx->use_mma && !(ctx->test_mode & TS_TEST_NO_SEED);
-  const bool persistent = seeds_on && !(ctx->test_mode & TS_TEST_NO_PERSIST) && persistent_supported(ctx, B);
+  const bool persistent = seeds_on && (ctx->test_mode & TS_TEST_PERSIST) && persistent_supported(ctx, B);
   if (persistent) {
     // One cooperative launch runs every level: scan, merge, level step, separated by grid barriers.  Ahead of it the
     // seed bounds of the root level (deeper levels get theirs from the level step before them).

@@ -605,33 +605,38 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
     } else if (warp == W_MMA && lane == 0) {
       // ======================= MMA issuer ===========================================================
       const uint32_t ws_addr = smem_u32(Ws), as_addr = smem_u32(As);
+      // (UMMA) Blocks go to the tensor cores in pairs (blocks 2x and 2x + 1 belong to neighbouring splits, whose accumulator
+      // buffers are neighbours in tensor memory, so one N = 128 instruction per K step fills both: issuing is what
+      // limits this warp).  A pair needs the base-logit slabs of its 128 tokens: two bulk-tensor loads into one of
+      // NUP ring slots (pair x of the kernel's running count uses slot x % NUP; a slot is free again as soon as the
+      // MMAs that read it are done, long before the blocks are scanned).  Within the window of NUP requested pairs,
+      // whichever pair has its buffers drained and its slabs landed is issued.  The first slabs are requested
+      // before the A tile is complete: they do not depend on it.
+      constexpr int NUP = NUB / 2;
+      constexpr uint32_t SLAB = (uint32_t)UMMA_REQ * 128u;
+      const int npair = (nblk + 1) / 2;
+      int base = 0, unext = 0;        // first pair not yet issued; first pair whose slabs are not yet requested
+      uint32_t done = 0;              // bit w: pair base + w is issued
+      auto request_slabs = [&]() {
+        while (unext < npair && unext < base + NUP) {
+          const uint32_t gx = ul + (uint32_t)unext, slot = gx % NUP, use = gx / NUP;
+          if (use >= 1 && !mbar_test_wait(u_free + slot, (use - 1) & 1)) break;
+          const bool two = 2 * unext + 1 < nblk;
+          mbar_expect_tx(u_full + slot, two ? 2u * SLAB : SLAB);
+          tma_load_box3(Us + (size_t)slot * 2 * SLAB, &tmU, t0 + 2 * unext * BLK_N, u_depth, 0, u_full + slot);
+          if (two) tma_load_box3(Us + (size_t)slot * 2 * SLAB + SLAB, &tmU, t0 + (2 * unext + 1) * BLK_N, u_depth, 0, u_full + slot);
+          ++unext;
+        }
+      };
+      if (UMMA) request_slabs();
       if (mbar_wait(a_full, gg & 1, s_abort, a.err, wait_limit)) {
         tc_fence_after();
         if (UMMA) {
-          // Blocks go to the tensor cores in pairs (blocks 2x and 2x + 1 belong to neighbouring splits, whose accumulator
-          // buffers are neighbours in tensor memory, so one N = 128 instruction per K step fills both: issuing is what
-          // limits this warp).  A pair needs the base-logit slabs of its 128 tokens: two bulk-tensor loads into one of
-          // NUP ring slots (pair x of the kernel's running count uses slot x % NUP; a slot is free again as soon as the
-          // MMAs that read it are done, long before the blocks are scanned).  Within the window of NUP requested pairs,
-          // whichever pair has its buffers drained and its slabs landed is issued.
-          constexpr int NUP = NUB / 2;
-          constexpr uint32_t SLAB = (uint32_t)UMMA_REQ * 128u;
           const uint32_t us_addr = smem_u32(Us);
           const int KU = UMMA_REQ / 16;   // extra K steps: the one-hot columns against the slabs' rows
-          const int npair = (nblk + 1) / 2;
-          int base = 0, unext = 0;        // first pair not yet issued; first pair whose slabs are not yet requested
-          uint32_t done = 0;              // bit w: pair base + w is issued
           uint32_t spin = 0;
           while (base < npair) {
-            while (unext < npair && unext < base + NUP) {
-              const uint32_t gx = ul + (uint32_t)unext, slot = gx % NUP, use = gx / NUP;
-              if (use >= 1 && !mbar_test_wait(u_free + slot, (use - 1) & 1)) break;
-              const bool two = 2 * unext + 1 < nblk;
-              mbar_expect_tx(u_full + slot, two ? 2u * SLAB : SLAB);
-              tma_load_box3(Us + (size_t)slot * 2 * SLAB, &tmU, t0 + 2 * unext * BLK_N, u_depth, 0, u_full + slot);
-              if (two) tma_load_box3(Us + (size_t)slot * 2 * SLAB + SLAB, &tmU, t0 + (2 * unext + 1) * BLK_N, u_depth, 0, u_full + slot);
-              ++unext;
-            }
+            request_slabs();
             bool progressed = false;
 #pragma unroll
             for (int w = 0; w < NUP; ++w) {
@@ -707,6 +712,17 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
           if (++spin > wait_limit) { *s_abort = 1; if (a.err) atomicExch(a.err, 1); break; }
           if (spin > 8) __nanosleep(32);
         }
+        }
+      }
+      if (UMMA && base < npair) {
+        // gave up with slabs on their way: do not go on (to the tear-down) while a bulk load may still be writing
+        // this CTA's shared memory
+        for (int w = 0; w < NUP; ++w) {
+          const int pr = base + w;
+          if (pr >= unext || ((done >> w) & 1u)) continue;
+          const uint32_t gx = ul + (uint32_t)pr, slot = gx % NUP;
+          bool landed = false;
+          for (uint32_t t = 0; t < WAIT_LIMIT && !landed; ++t) { landed = mbar_test_wait(u_full + slot, (gx / NUP) & 1); if (!landed) __nanosleep(100); }
         }
       }
     }

@@ -162,11 +162,11 @@ def test_back_to_back_rounds_reproduce_bitwise():
             assert torch.equal(verdict["acc_tok"].cpu()[b, :L], v0["acc_tok"][b, :L]), (i, b)
 
 
-@pytest.mark.parametrize("mode", ["TEST_FORCE_FMA", "TEST_NO_TMA", "TEST_NO_FEW", "TEST_NO_SEED", "TEST_NO_PERSIST", "TEST_NO_UMMA"])
+@pytest.mark.parametrize("mode", ["TEST_FORCE_FMA", "TEST_NO_TMA", "TEST_NO_FEW", "TEST_NO_SEED", "TEST_PERSIST", "TEST_NO_UMMA"])
 def test_alternative_kernel_paths_match_oracle(mode):
     """bf16 inputs on the fp32-FMA kernels; the tensor-core kernels with W staged by plain loads (the path
     taken when no tensor map can be encoded); every level on the tile kernel; the tile kernel without seeded
-    bounds; one launch per step of every level instead of the persistent expansion kernel: chosen by the library's
+    bounds; every level inside one cooperative launch instead of one launch per step of every level: chosen by the library's
     test switches."""
     from paper_2609_22098_b200 import binding
     wl = small("serve32", V=20000, B=5)
@@ -508,7 +508,7 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(T, persis
     from paper_2609_22098_b200 import binding
     wl = small("serve32", V=20000, B=6)
     rnd = Round(wl, seed=91)
-    base = 0 if persist else binding.TEST_NO_PERSIST
+    base = binding.TEST_PERSIST if persist else 0
     ts = make_gpu(wl, rnd.table, max_batch=rnd.B, test_mode=base)
     orc = make_oracle(wl, rnd.table)
     good = ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, 5)
