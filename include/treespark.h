@@ -193,10 +193,16 @@ int32_t ts_score_parents_static(ts_ctx* ctx, const void* U, const void* A, const
  *   logS = log survival; q0 = q0(token | parent); logqT = log q_T(token | parent) (log q0 at T == 0);
  *   logkey = log of the slot key the node was admitted under; pop_rank = best-first admission order;
  *   node_hash [B][Nmax+1] (slot 0 = root); node_lseT [B][Nmax+1] = log-normaliser of q_T(.|node)
- *   for every node that was scored, NaN otherwise (slot 0 = root);
+ *   (slot 0 = root).  It is defined for the nodes whose conditional was computed: the root and every
+ *   node that has children, plus scored nodes all of whose candidates were refused.  A node that was
+ *   never a parent (depth D, survival below theta, or admitted when the tree was already full) holds
+ *   NaN; ts_verify_tree needs the value only where a node has children;
  *   mask [B][Nmax][ceil(Nmax/64)]: ancestor bitmask, bit i of row i set, root implicit (the tree
  *   attention mask of Section 3.2 item 3; position id = depth);
- *   n_scored [B] = parents scored for the request; status [B].
+ *   n_scored [B] = parent conditionals actually computed for the request (Eq. 1 evaluations): one per
+ *   node on a level's parent list.  That is at least 1 + the number of nodes with children; it also
+ *   counts nodes that were scored and later evicted by the cut to Nmax, and it does not count admitted
+ *   nodes that never became parents.  status [B].
  * logkey, pop_rank, node_lseT, n_scored may be NULL.
  */
 int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, const void* W,

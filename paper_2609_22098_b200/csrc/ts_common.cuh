@@ -51,6 +51,7 @@ struct TileCfg {
   int TV;       // tokens per vocabulary tile (multiple of 64)
   int ntiles;   // tiles covering V
   size_t smem;  // dynamic shared memory of the scoring kernel
+  int umma;     // the tiling leaves room for the one-hot slab and the base-logit slab ring (base logits through the MMA)
 };
 
 }  // namespace ts

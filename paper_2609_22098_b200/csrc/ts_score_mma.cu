@@ -138,17 +138,20 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   if (a.P_prev_dev && *a.P_prev_dev <= 0) { pdl_wait(); return; }
 
   const int r = a.r, rp = (r + 63) / 64 * 64, V = a.V, TV = a.TV, K = a.K;
-  const int tile = blockIdx.x, t0 = tile * TV, tlen = min(TV, V - t0);
+  // This CTA's vocabulary tiles: blockIdx.x, blockIdx.x + gridDim.x, ... (one tile per CTA whenever the tiles fit
+  // the SMs; at large ranks, where the W tile is small, a CTA takes several in turn and pays its set-up once)
+  int tile = blockIdx.x, t0 = tile * TV, tlen = min(TV, V - t0);
+  int tile_it = 0;          // tiles this CTA has finished: the W barriers' phase
   const int nslab = TV / 64;
-  const int nblk_w = (tlen + WBLK - 1) / WBLK;
+  int nblk_w = (tlen + WBLK - 1) / WBLK;
   const uint32_t slab_bytes = (uint32_t)rp * 128u;       // one 64-token slab of W
   const uint32_t a_slab_bytes = 128u * 128u;             // 128 rows x 128 B
   unsigned char* sm = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* Ws = sm;
   unsigned char* As = Ws + (size_t)nslab * slab_bytes;
   // (one more slab of the A tile holds the one-hot request columns, and a ring of slabs the base logits they select)
-  unsigned char* Us = As + (size_t)(rp / 64 + 1) * a_slab_bytes;   // [NUB][UMMA_REQ rows][128 B], 128-byte swizzle
-  float* ghi = reinterpret_cast<float*>(Us + (size_t)NUB * UMMA_REQ * 128);
+  unsigned char* Us = As + (size_t)(rp / 64 + (UMMA ? 1 : 0)) * a_slab_bytes;   // [NUB][UMMA_REQ rows][128 B], 128-byte swizzle
+  float* ghi = reinterpret_cast<float*>(Us + (UMMA ? (size_t)NUB * UMMA_REQ * 128 : 0));
   SelShared sh;
   sh.q = reinterpret_cast<uint4*>(ghi + 512);                                   // 16-byte aligned
   sh.lists = reinterpret_cast<float*>(sh.q + NSEL * QCAP);
@@ -204,7 +207,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
     // fetches nothing).
     if (use_tma && early_w) issue_w();
   }
-  if (!use_tma) {  // W tile: 16-byte chunks (8 tokens of one row), swizzled: chunk j of row k lands at chunk j ^ (k & 7)
+  auto fill_w_plain = [&]() {  // W tile: 16-byte chunks (8 tokens of one row), swizzled: chunk j of row k lands at chunk j ^ (k & 7)
     const int per_slab = rp * 8;
     for (int idx = tid; idx < nslab * per_slab; idx += MMA_THREADS) {
       const int slab = idx / per_slab, rem = idx % per_slab, k = rem >> 3, j = rem & 7;
@@ -213,7 +216,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       if (k < r && tok < V) v = __ldg(reinterpret_cast<const uint4*>(Wg + (size_t)k * V + tok));
       *reinterpret_cast<uint4*>(Ws + (size_t)slab * slab_bytes + k * 128 + ((j ^ (k & 7)) << 4)) = v;
     }
-  }
+  };
+  if (!use_tma) fill_w_plain();
   fill_gumbel_bounds(ghi, tid, MMA_THREADS);
   for (int i = tid; i < 512; i += MMA_THREADS) s_thr[i] = 0u;
   auto reset_selection = [&]() {   // empty lists, no local thresholds, nothing published
@@ -239,6 +243,9 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   unsigned gen = 0;         // grid barriers passed
   bool dead = false;        // a bounded wait ran out somewhere
   bool w_issued = use_tma && early_w;   // bulk loads of the W tile are (or were) in flight
+  int gg_tile = 0;          // value of gg when the current tile began: its first group waits for the tile's W blocks
+  for (;;) {   // this CTA's tiles
+  gg_tile = gg;
   for (int lvl = 0; !dead; ++lvl) {
   // the parent list of this level (in the persistent form written by the level step before it: read around L1)
   const int cur = lvl & 1;
@@ -250,7 +257,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   const bool scout = a.utop != nullptr && scout_depth < a.D;
   const int u_depth = persist ? lvl : a.u_depth;   // UMMA: the depth every parent of this level sits at
   const int P = persist ? __ldcg(pa.ex.lvl_count + lvl) : (a.P_dev ? *a.P_dev : a.P);   // may be 0: an empty level only tears down
-  if (use_tma && !early_w && P > 0 && lvl == 0) { if (tid == 0) issue_w(); w_issued = true; }
+  if (use_tma && !w_issued && P > 0 && lvl == 0) { if (tid == 0) issue_w(); w_issued = true; }
 
   const int R = mma_replicas(P);
   const int per = 128 / R;
@@ -650,7 +657,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
               const int u0 = gg * ((nuse0 + 1 - h) >> 1) + (j >> 1), u1 = gg * ((nuse1 + 1 - h) >> 1) + (j >> 1);
               if (u0 >= 1 && !mbar_test_wait(t_empty + tb, (u0 - 1) & 1)) continue;
               if (two && u1 >= 1 && !mbar_test_wait(t_empty + tb + 1, (u1 - 1) & 1)) continue;
-              if (use_tma && gg == 0 && !mbar_test_wait(w_full + nb * BLK_N / WBLK, 0)) continue;
+              if (use_tma && gg == gg_tile && !mbar_test_wait(w_full + nb * BLK_N / WBLK, tile_it & 1)) continue;
               const uint32_t gx = ul + (uint32_t)pr, slot = gx % NUP;
               if (!mbar_test_wait(u_full + slot, (gx / NUP) & 1)) continue;
               tc_fence_after();
@@ -693,7 +700,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
             const int j = nb / EPI_S, h = j & 1, tb = sp + EPI_S * h;
             const int u = gg * ((nuse + 1 - h) >> 1) + (j >> 1);
             if (u >= 1 && !mbar_test_wait(t_empty + tb, (u - 1) & 1)) continue;
-            if (use_tma && gg == 0 && !mbar_test_wait(w_full + nb * BLK_N / WBLK, 0)) continue;
+            if (use_tma && gg == gg_tile && !mbar_test_wait(w_full + nb * BLK_N / WBLK, tile_it & 1)) continue;
             tc_fence_after();
             const uint32_t idesc = instr_desc(BLK_N);
             const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
@@ -788,14 +795,23 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
     if (lvl + 1 >= pa.nlevels || __ldcg(pa.ex.lvl_count + lvl + 1) <= 0) break;
   }
   }
+  // ---- the next tile of this CTA (never in the persistent form, whose grid covers the tiles) ---------------
+  if (persist || dead || *s_abort || gg == gg_tile || tile + (int)gridDim.x >= a.ntiles) break;
+  // Every block of the finished tile was drained, so the MMAs that read its W are done, and the barrier that ended
+  // the last group has every thread past its scan: the W tile may be overwritten.
+  tile += (int)gridDim.x; ++tile_it;
+  t0 = tile * TV; tlen = min(TV, V - t0); nblk_w = (tlen + WBLK - 1) / WBLK;
+  if (use_tma) { if (tid == 0) issue_w(); }
+  else { fill_w_plain(); fence_async_smem(); __syncthreads(); }
+  }
   if (dead && persist && tid == 0) { atomicExch(pa.barrier + 1, 1u); if (a.err) atomicExch(a.err, 1); }
   // ---- tear-down -----------------------------------------------------------------------------------
-  if (use_tma && tid == 0 && w_issued && (*s_abort || dead || gg == 0)) {
+  if (use_tma && tid == 0 && w_issued && (*s_abort || dead || gg == gg_tile)) {
     // gave up somewhere, or nothing to score: do not leave while a bulk load may still be writing this
     // CTA's shared memory
     for (int nb = 0; nb < nblk_w; ++nb) {
       bool done = false;
-      for (uint32_t i = 0; i < WAIT_LIMIT && !done; ++i) { done = mbar_try_wait(w_full + nb, 0); if (!done) __nanosleep(100); }
+      for (uint32_t i = 0; i < WAIT_LIMIT && !done; ++i) { done = mbar_test_wait(w_full + nb, tile_it & 1); if (!done) __nanosleep(100); }
     }
   }
   tc_fence_before();
@@ -808,18 +824,19 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
 }
 
 // shared memory beside the W tile: A tile, noise tables, queues, lists, bounds, partial sums, barriers
-static size_t mma_fixed_smem(const ts_config& c) {
+static size_t mma_fixed_smem(const ts_config& c, bool umma) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
   const size_t K = (size_t)c.K;
-  return (rp / 64 + 1) * 128 * 128 + (size_t)NUB * UMMA_REQ * 128 + 512 * 4 + (size_t)NSEL * QCAP * 16 + 128 * 5 * K * 4 + 2 * 128 * 4 +
+  return (rp / 64 + (umma ? 1 : 0)) * 128 * 128 + (umma ? (size_t)NUB * UMMA_REQ * 128 : 0) + 512 * 4 + (size_t)NSEL * QCAP * 16 + 128 * 5 * K * 4 + 2 * 128 * 4 +
          2 * EPI_S * 128 * 4 + 3 * EPI_S * 128 * 4 + 512 * 4 + (1 + 2 * NBUF + MAX_BLK + 2 * NUB) * 8 + 64 + 1024;
 }
 
 // tile size for the tensor-core path: W tile + the rest within the shared-memory limit,
 // a whole number of waves over the SMs
-bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
+static bool choose_tile_mma_for(const ts_config& c, int num_sms, int max_smem, bool umma, TileCfg* out) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
-  const size_t fixed = mma_fixed_smem(c);
+  const size_t fixed = mma_fixed_smem(c, umma);
+  out->umma = umma ? 1 : 0;
   if ((size_t)max_smem < fixed + rp * 128) return false;
   int tv_max = (int)(((size_t)max_smem - fixed) / (rp * 2) / 64) * 64;
   if (tv_max < 64) return false;
@@ -833,6 +850,18 @@ bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out
   out->ntiles = (c.V + tv - 1) / tv;
   out->smem = (size_t)(tv / 64) * rp * 128 + fixed;
   return out->ntiles <= 4096;
+}
+
+// With room for the one-hot slab and the base-logit slabs (base logits through the MMA) unless that costs waves: at
+// large ranks the W tile is what shared memory is short of, and every wave pays the kernel's set-up again.
+bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
+  TileCfg with{}, without{};
+  const bool ok_with = choose_tile_mma_for(c, num_sms, max_smem, true, &with);
+  const bool ok_without = choose_tile_mma_for(c, num_sms, max_smem, false, &without);
+  if (!ok_with && !ok_without) return false;
+  auto waves = [&](const TileCfg& t) { return (t.ntiles + num_sms - 1) / num_sms; };
+  *out = (ok_with && (!ok_without || waves(with) <= waves(without))) ? with : without;
+  return true;
 }
 
 cudaError_t score_mma_setup(ts_ctx* ctx) {
@@ -902,7 +931,7 @@ static bool u_tensor_map(ts_ctx* ctx, const void* U, int B) {
 
 // base logits through the tensor cores: every parent at one known depth, few enough requests, bulk-tensor loads available
 static bool use_umma(ts_ctx* c, const ScoreArgs& a, bool persist, int use_tma) {
-  return use_tma && (persist || a.u_depth >= 0) && a.u_B >= 1 && a.u_B <= UMMA_REQ && !(c->test_mode & TS_TEST_NO_UMMA) &&
+  return c->tile.umma && use_tma && (persist || a.u_depth >= 0) && a.u_B >= 1 && a.u_B <= UMMA_REQ && !(c->test_mode & TS_TEST_NO_UMMA) &&
          u_tensor_map(c, a.U, a.u_B);
 }
 
@@ -916,8 +945,9 @@ cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t
   memset(&tu, 0, sizeof(tu));
   const bool umma = use_umma(c, a, false, use_tma);
   if (umma) memcpy(&tu, c->tmapU, sizeof(tu));
-  const cudaError_t e = umma ? launch_kernel(score_mma_kernel<true>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma, pa, tu)
-                             : launch_kernel(score_mma_kernel<false>, a.ntiles, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma, pa, tu);
+  const int grid = a.ntiles < ctx->num_sms ? a.ntiles : ctx->num_sms;   // one CTA per SM at most: a CTA takes its tiles in turn
+  const cudaError_t e = umma ? launch_kernel(score_mma_kernel<true>, grid, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma, pa, tu)
+                             : launch_kernel(score_mma_kernel<false>, grid, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma, pa, tu);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 

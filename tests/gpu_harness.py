@@ -90,6 +90,21 @@ def compare_tree(g, b, o, D):
         for name in ("logS", "q0", "logqT", "logkey"):
             if not close(g[name][b, i], o[name][i]):
                 return False, False, f"req {b} node {i}: {name} {float(g[name][b, i])!r} vs {o[name][i]!r}"
+    # what the header promises about the two outputs whose coverage differs from the oracle's (the oracle scores
+    # every admitted node above depth D; the library only the nodes that reach a level's parent list)
+    has_child = np.zeros(n + 1, dtype=bool)          # slot 0 = root
+    has_child[np.asarray(o["parent"][:n], dtype=np.int64) + 1] = True
+    if n > 0 and "n_scored" in g and int(g["n_scored"][b]) < int(has_child.sum()):
+        return False, False, f"req {b}: n_scored {int(g['n_scored'][b])} < nodes with children {int(has_child.sum())}"
+    if "node_lseT" in g:
+        lse = g["node_lseT"][b, :n + 1].numpy()
+        if not np.isfinite(lse[has_child]).all():
+            return False, False, f"req {b}: node_lseT not finite at a node with children"
+        if "node_lseT" in o:
+            ol = np.asarray(o["node_lseT"][:n + 1], dtype=np.float64)
+            for i in np.nonzero(has_child)[0]:
+                if not close(lse[i], ol[i]):
+                    return False, False, f"req {b} slot {i}: node_lseT {float(lse[i])!r} vs {float(ol[i])!r}"
     return True, False, ""
 
 
@@ -143,12 +158,17 @@ class Round:
                                         tree["tok"], tree["depth"], tree["node_hash"], sigma=sigma)
 
 
-def check_round(ts, orc, rnd: Round, T, round_seed, reqs=None, want_edge=True, threads=None):
+def check_round(ts, orc, rnd: Round, T, round_seed, reqs=None, want_edge=True, threads=None, sigma_by_req=None):
     """Expand + verify on the GPU, then the oracle on the same bytes for `reqs`; returns statistics.
-    Raises AssertionError on any mismatch outside the flagged near-ties."""
+    Raises AssertionError on any mismatch outside the flagged near-ties.  sigma_by_req = {request: sigma}
+    regenerates those requests' target rows with another noise level (0: the target is the drafter)."""
     wl = rnd.wl
     tree = ts.expand_tree(rnd.U, rnd.A, rnd.W, rnd.anchor, rnd.theta, T, round_seed)
     Z, off = rnd.target_logits(tree)
+    for b, sg in (sigma_by_req or {}).items():
+        Z2, _ = rnd.target_logits(tree, sigma=sg)
+        Z[int(off[b]):int(off[b + 1])] = Z2[int(off[b]):int(off[b + 1])]
+        del Z2
     verdict = ts.verify_tree(rnd.U, rnd.A, rnd.W, Z, off, rnd.anchor, tree, T, round_seed)
     torch.cuda.synchronize()
     g, v = to_cpu(tree), to_cpu(verdict)
@@ -159,7 +179,7 @@ def check_round(ts, orc, rnd: Round, T, round_seed, reqs=None, want_edge=True, t
     otrees, used = oracle_trees(orc, c["U"], c["A"], c["W"], c["anchor"], c["theta"], T, round_seed, reqs, threads)
     Zc, offc = Z.cpu(), off.cpu()
     Af, Wf = c["A"].float().numpy(), c["W"].float().numpy()
-    stats = dict(trees=0, trees_exempt=0, walks=0, walks_exempt=0, nodes=0, acc=0, threads=used)
+    stats = dict(trees=0, trees_exempt=0, walks=0, walks_exempt=0, nodes=0, acc=0, threads=used, acc_len={}, n_nodes={})
 
     def verify_one(b):
         o = otrees[b]
@@ -185,6 +205,8 @@ def check_round(ts, orc, rnd: Round, T, round_seed, reqs=None, want_edge=True, t
         assert ok, msg
         stats["walks"] += 1
         stats["acc"] += int(ov["acc_len"])
+        stats["acc_len"][b] = int(v["acc_len"][b])
+        stats["n_nodes"][b] = int(g["n_nodes"][b])
         if exempt:
             stats["walks_exempt"] += 1
             _count_flags(ov["flags"], WALK_FLAGS)
