@@ -46,6 +46,8 @@ __device__ __forceinline__ void request_caps(const ExpandArgs& a, int b, int& K_
 
 struct Entry { double key; uint64_t path; int depth; };
 
+__device__ __forceinline__ int warp_of(int tid) { return tid >> 5; }
+
 __device__ __forceinline__ bool before(double ka, int da, uint64_t pa, double kb, int db, uint64_t pb) {
   if (ka != kb) return ka > kb;
   if (da != db) return da < db;
@@ -206,15 +208,66 @@ __device__ __forceinline__ void level_step(const ExpandArgs& a, const int d, con
       ent[e] = x;
     }
     sync();
+    // The N_eff-th largest key by radix selection over the keys' order-preserving bit patterns (eight passes of
+    // eight bits, a 256-bin histogram each); entries above it stay, entries below it go, and the entries that tie
+    // with it are ranked among themselves by (depth asc, path asc) for the places that are left.
+    auto skey = [](double k) -> uint64_t {
+      if (k == 0.0) k = 0.0;   // -0 and +0 compare equal: one pattern
+      const uint64_t b = (uint64_t)__double_as_longlong(k);
+      return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
+    };
+    int* hist = s_free;          // 256 bins (the free-slot list is built in phase 3)
+    uint64_t prefix = 0;
+    int need = N_eff;            // the entry sought is the need-th largest among those that match the prefix so far
+    for (int sh8 = 56; sh8 >= 0; sh8 -= 8) {
+      hist[tid] = 0;             // LEVEL_THREADS == 256 bins
+      sync();
+      for (int e = tid; e < M; e += LEVEL_THREADS) {
+        if (ent[e].depth < 0) continue;
+        const uint64_t k = skey(ent[e].key);
+        if (sh8 == 56 || (k >> (sh8 + 8)) == (prefix >> (sh8 + 8))) atomicAdd(&hist[(int)((k >> sh8) & 255u)], 1);
+      }
+      sync();
+      if (warp_of(tid) == 0) {
+        // lane l owns bins 255 - 8l .. 248 - 8l (descending); the bin where the running count reaches `need`
+        const int l = tid & 31;
+        int mine = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) mine += hist[255 - 8 * l - j];
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (l >= o) incl += v; }
+        const unsigned reach = __ballot_sync(0xFFFFFFFFu, incl >= need);
+        const int owner = __ffs(reach) - 1;   // reach != 0: at least `need` entries match the prefix
+        if (l == owner) {
+          int cum = incl - mine, bin = 255 - 8 * l;
+          for (int j = 0; j < 8; ++j) {
+            const int h = hist[255 - 8 * l - j];
+            if (cum + h >= need) { bin = 255 - 8 * l - j; break; }
+            cum += h;
+          }
+          s_warp[0] = bin; s_warp[1] = need - cum;
+        }
+      }
+      sync();
+      prefix |= (uint64_t)s_warp[0] << sh8;
+      need = s_warp[1];
+      sync();
+    }
     for (int e = tid; e < M; e += LEVEL_THREADS) {
       const Entry x = ent[e];
       if (x.depth < 0) continue;
-      int rank = 0;
-      for (int f = 0; f < M; ++f) {
-        const Entry y = ent[f];
-        if (y.depth >= 0 && f != e && before(y.key, y.depth, y.path, x.key, x.depth, x.path)) ++rank;
+      const uint64_t k = skey(x.key);
+      bool drop = k < prefix;
+      if (k == prefix) {
+        int rank = 0;
+        for (int f = 0; f < M; ++f) {
+          const Entry y = ent[f];
+          if (y.depth >= 0 && f != e && skey(y.key) == prefix && before(y.key, y.depth, y.path, x.key, x.depth, x.path)) ++rank;
+        }
+        drop = rank >= need;
       }
-      if (rank >= N_eff) {
+      if (drop) {
         if (e < N) a.pl_alive[pb + e] = 0; else a.cd_valid[cb + (e - N)] = 0;
       }
     }
