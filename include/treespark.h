@@ -155,10 +155,10 @@ int32_t ts_score_parents(ts_ctx* ctx, const void* U, const void* A, const void* 
  *
  * Limits and rules:
  *   - The array bounds P: every parent slot needs one record of (4 + 5K) words (rounded up to 16 bytes)
- *     per vocabulary tile and column split, plus its pruning-bound words, and slots come in blocks of
- *     128 on the tensor-core path: 128 parents for a 152k vocabulary with K = 8 in bf16, a few hundred
- *     on the fp32 path.  A larger P is refused with TS_ERR_WORKSPACE and a message that names the
- *     limit; nothing is launched.
+ *     per vocabulary tile, plus its pruning-bound words (2K lines of 128 bytes), the array also holds 1 MiB
+ *     of scratch for the seed-bound kernel, and slots come in blocks of 128 on the tensor-core path: 256
+ *     parents for a 152k vocabulary with K = 8 in bf16 (140 tiles), a few hundred on the fp32 path.  A
+ *     larger P is refused with TS_ERR_WORKSPACE and a message that names the limit; nothing is launched.
  *   - The context's device must be the current device.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
  *     remembers it; make that first call before starting any stream capture.
