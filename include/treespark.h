@@ -95,6 +95,8 @@ int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags);
  *   TS_TEST_PERSIST       ts_expand_tree runs every level inside one cooperative launch (scan, merge and level
  *                         step separated by grid barriers; nothing is launched for empty levels) instead of one
  *                         launch per step of every level, where the configuration fits that kernel
+ *   TS_TEST_NO_TAIL       ts_expand_tree launches every level's kernels one by one up to the last level, instead of
+ *                         handing the levels from the fifth on (mostly empty) to one cooperative launch
  *   TS_TEST_NO_UMMA       the scanning threads of the tensor-core scoring kernel load the base logits themselves
  *                         instead of receiving them through the MMA (the path of batches above 32 requests)
  *   TS_TEST_SHORT_WAITS   bounded waits give up after 4096 polls instead of 2^22
@@ -109,6 +111,7 @@ int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags);
 #define TS_TEST_LOST_ARRIVAL 32u
 #define TS_TEST_PERSIST 64u
 #define TS_TEST_NO_UMMA 128u
+#define TS_TEST_NO_TAIL 256u
 int32_t ts_set_test_mode(ts_ctx* ctx, uint32_t flags);
 
 /* Bytes of workspace the hot calls need for a batch of `batch` requests (<= max_batch). */

@@ -21,7 +21,7 @@ KNOTS = 16
 
 ABLATE_CALIB_QT = 1
 TEST_FORCE_FMA, TEST_NO_TMA, TEST_NO_FEW, TEST_NO_SEED, \
-    TEST_SHORT_WAITS, TEST_LOST_ARRIVAL, TEST_PERSIST, TEST_NO_UMMA = 1, 2, 4, 8, 16, 32, 64, 128
+    TEST_SHORT_WAITS, TEST_LOST_ARRIVAL, TEST_PERSIST, TEST_NO_UMMA, TEST_NO_TAIL = 1, 2, 4, 8, 16, 32, 64, 128, 256
 
 EXPORTS = ("ts_create", "ts_destroy", "ts_set_ablation", "ts_set_test_mode", "ts_workspace_bytes", "ts_last_error_string",
            "ts_score_parents", "ts_score_parents_static", "ts_expand_tree", "ts_verify_tree",

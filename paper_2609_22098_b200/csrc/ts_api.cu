@@ -141,7 +141,7 @@ extern "C" int32_t ts_set_ablation(ts_ctx* ctx, uint32_t flags) {
 
 extern "C" int32_t ts_set_test_mode(ts_ctx* ctx, uint32_t flags) {
   if (!ctx) return set_error(TS_ERR_INVALID, "ts_set_test_mode: null context");
-  const uint32_t known = TS_TEST_FORCE_FMA | TS_TEST_NO_TMA | TS_TEST_NO_FEW | TS_TEST_NO_SEED | TS_TEST_SHORT_WAITS | TS_TEST_LOST_ARRIVAL | TS_TEST_PERSIST | TS_TEST_NO_UMMA;
+  const uint32_t known = TS_TEST_FORCE_FMA | TS_TEST_NO_TMA | TS_TEST_NO_FEW | TS_TEST_NO_SEED | TS_TEST_SHORT_WAITS | TS_TEST_LOST_ARRIVAL | TS_TEST_PERSIST | TS_TEST_NO_UMMA | TS_TEST_NO_TAIL;
   if (flags & ~known) return set_error(TS_ERR_INVALID, "ts_set_test_mode: unknown switch");
   const unsigned before = ctx->test_mode;
   ctx->test_mode = flags;

@@ -212,35 +212,21 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(init)", e);
   const size_t level_smem = level_smem_bytes(c);   // opted into at ts_create when above 48 KB
   const bool seeds_on = ctx->use_mma && !(ctx->test_mode & TS_TEST_NO_SEED);
-  const bool persistent = seeds_on && (ctx->test_mode & TS_TEST_PERSIST) && persistent_supported(ctx, B);
-  if (persistent) {
-    // One cooperative launch runs every level: scan, merge, level step, separated by grid barriers.  Ahead of it the
-    // seed bounds of the root level (deeper levels get theirs from the level step before them).
-    ScoreArgs sa = make_score_args(ctx, (float*)(ws + L.rec), L.rec_cap, (int*)(ws + L.err), U, A, W, T, seed);
-    sa.pdl = 1; sa.P = 0; sa.P_dev = a.lvl_count;
-    sa.p_req = a.lst_req[0]; sa.p_depth = a.lst_depth[0]; sa.p_token = a.lst_token[0]; sa.p_hash = a.lst_hash[0];
-    set_seed_pointers(ctx, sa);
-    { ProfScope ps(ctx, K_SEED, st); e = launch_seed(ctx, sa, st); }
-    if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(seed)", e);
-    sa.utop = (uint2*)(ws + L.utop); sa.scout_live = a.req_npar; sa.scout_B = B; sa.scout_depth = 1;
-    sa.u_depth = 0; sa.u_B = B;
-    PersistArgs pa{};
-    pa.on = 1; pa.nlevels = c.D; pa.ex = a; pa.barrier = a.ex_barrier;
-    pa.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
-    MergeArgs& m = pa.mg;
-    m.pdl = 0; m.few_ntiles = 0; m.P = 0; m.P_dev = nullptr; m.K = c.K; m.ntiles = sa.ntiles; m.cap = L.rec_cap; m.S = 1; m.mma = 1; m.T = T;
-    m.rec = sa.rec; m.thr = sa.thr; m.slots = sa.slots; m.thr0 = sa.thr0;
-    m.lse0 = res_lse0; m.lseT = res_lseT; m.top_tok = res_top_tok; m.top_logit = res_top_logit; m.draw_tok = res_draw_tok;
-    m.draw_logit = res_draw_logit;
-    { ProfScope ps(ctx, K_PERSIST, st); e = launch_expand_persistent(ctx, sa, pa, st); }
-    if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(persistent)", e);
-  }
+  // Three forms.  Default: one launch per step of every level (score, merge, level step), chained, for the first
+  // TAIL_FROM levels, and one cooperative launch for all levels after those: trees usually end before them, and
+  // three launches per empty level (each a hop in the chain of dependent launches) become one that returns at once.
+  // TS_TEST_PERSIST: the cooperative launch runs every level.  TS_TEST_NO_TAIL: no cooperative launch at all.
+  constexpr int TAIL_FROM = 4;
+  const bool coop_ok = seeds_on && persistent_supported(ctx, B);
+  int coop_from = c.D;   // first level of the cooperative launch (D: none)
+  if (coop_ok && (ctx->test_mode & TS_TEST_PERSIST)) coop_from = 0;
+  else if (coop_ok && !(ctx->test_mode & TS_TEST_NO_TAIL) && c.D > TAIL_FROM + 1) coop_from = TAIL_FROM;
   long long level_bound = B;   // parents a level can have at most: B at the root, K times more per level, B * Nmax overall
   // Seed bounds of a level on the tensor-core kernel: made by the level kernel before it when that level's scoring
   // launch scouted the rows (it does whenever it runs on the tensor-core kernel itself); by a seed launch otherwise
   // (the root level, and the first tensor-core level after levels on the few-parents kernel).
   bool scouted_prev = false;
-  for (int d = 0; d < c.D && !persistent; ++d) {
+  for (int d = 0; d < coop_from; ++d) {
     const int cur = d & 1;
     const bool on_mma = ctx->use_mma && !(ctx->few_ok && level_bound <= FEW_MAX);
     ScoreExtras ex;
@@ -258,6 +244,33 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
     scouted_prev = scout;
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(level)", e);
+  }
+  if (coop_from < c.D) {
+    // One cooperative launch runs the remaining levels: scan, merge, level step, separated by grid barriers.  Its
+    // first level's seed bounds come from a seed launch (the root level) or from the level kernel before it.
+    ScoreArgs sa = make_score_args(ctx, (float*)(ws + L.rec), L.rec_cap, (int*)(ws + L.err), U, A, W, T, seed);
+    sa.pdl = 1; sa.P = 0; sa.P_dev = a.lvl_count + coop_from;
+    sa.P_prev_dev = coop_from > 0 ? a.lvl_count + coop_from - 1 : nullptr;
+    const int cur = coop_from & 1;
+    sa.p_req = a.lst_req[cur]; sa.p_depth = a.lst_depth[cur]; sa.p_token = a.lst_token[cur]; sa.p_hash = a.lst_hash[cur];
+    set_seed_pointers(ctx, sa);
+    if (coop_from == 0) {
+      ProfScope ps(ctx, K_SEED, st);
+      e = launch_seed(ctx, sa, st);
+      if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(seed)", e);
+    }
+    sa.utop = (uint2*)(ws + L.utop); sa.scout_live = a.req_npar; sa.scout_B = B; sa.scout_depth = coop_from + 1;
+    sa.u_depth = coop_from; sa.u_B = B;
+    PersistArgs pa{};
+    pa.on = 1; pa.first = coop_from; pa.nlevels = c.D; pa.ex = a; pa.barrier = a.ex_barrier;
+    pa.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
+    MergeArgs& m = pa.mg;
+    m.pdl = 0; m.few_ntiles = 0; m.P = 0; m.P_dev = nullptr; m.K = c.K; m.ntiles = sa.ntiles; m.cap = L.rec_cap; m.S = 1; m.mma = 1; m.T = T;
+    m.rec = sa.rec; m.thr = sa.thr; m.slots = sa.slots; m.thr0 = sa.thr0;
+    m.lse0 = res_lse0; m.lseT = res_lseT; m.top_tok = res_top_tok; m.top_logit = res_top_logit; m.draw_tok = res_draw_tok;
+    m.draw_logit = res_draw_logit;
+    { ProfScope ps(ctx, K_PERSIST, st); e = launch_expand_persistent(ctx, sa, pa, st); }
+    if (e != cudaSuccess) return set_cuda_error("ts_expand_tree(cooperative)", e);
   }
   FinalArgs f{};
   f.B = B; f.N = c.Nmax; f.words = L.words;

@@ -60,6 +60,7 @@ __device__ __forceinline__ bool before(double ka, int da, uint64_t pa, double kb
 // tile, tensor memory and barriers are set up once; grid barriers (bounded) separate the phases.
 struct PersistArgs {
   int on;               // 0: one scan of the parent list in ScoreArgs, nothing else
+  int first;            // first level this launch runs (levels before it were run by launches of their own)
   int nlevels;          // D
   ExpandArgs ex;        // level lists, pools, seeds
   MergeArgs mg;         // merged-result arrays

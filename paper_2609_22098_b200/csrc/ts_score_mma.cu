@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   int gg_tile = 0;          // value of gg when the current tile began: its first group waits for the tile's W blocks
   for (;;) {   // this CTA's tiles
   gg_tile = gg;
-  for (int lvl = 0; !dead; ++lvl) {
+  for (int lvl = persist ? pa.first : 0; !dead; ++lvl) {
   // the parent list of this level (in the persistent form written by the level step before it: read around L1)
   const int cur = lvl & 1;
   const int* lp_req = persist ? pa.ex.lst_req[cur] : a.p_req;
@@ -257,7 +257,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   const bool scout = a.utop != nullptr && scout_depth < a.D;
   const int u_depth = persist ? lvl : a.u_depth;   // UMMA: the depth every parent of this level sits at
   const int P = persist ? __ldcg(pa.ex.lvl_count + lvl) : (a.P_dev ? *a.P_dev : a.P);   // may be 0: an empty level only tears down
-  if (use_tma && !w_issued && P > 0 && lvl == 0) { if (tid == 0) issue_w(); w_issued = true; }
+  if (persist && P <= 0) break;   // (a launch that starts at a later level finds out here that the tree ended before it)
+  if (use_tma && !w_issued && P > 0) { if (tid == 0) issue_w(); w_issued = true; }
 
   const int R = mma_replicas(P);
   const int per = 128 / R;

@@ -187,11 +187,11 @@ def test_a_request_that_accepts_a_full_depth_path_beside_requests_that_reject(dt
     assert full >= 1, "no round accepted the whole chain: the case under test was not reached"
 
 
-@pytest.mark.parametrize("mode", ["TEST_FORCE_FMA", "TEST_NO_TMA", "TEST_NO_FEW", "TEST_NO_SEED", "TEST_PERSIST", "TEST_NO_UMMA"])
+@pytest.mark.parametrize("mode", ["TEST_FORCE_FMA", "TEST_NO_TMA", "TEST_NO_FEW", "TEST_NO_SEED", "TEST_PERSIST", "TEST_NO_UMMA", "TEST_NO_TAIL"])
 def test_alternative_kernel_paths_match_oracle(mode):
     """bf16 inputs on the fp32-FMA kernels; the tensor-core kernels with W staged by plain loads (the path
     taken when no tensor map can be encoded); every level on the tile kernel; the tile kernel without seeded
-    bounds; every level inside one cooperative launch instead of one launch per step of every level: chosen by the library's
+    bounds; every level inside one cooperative launch, or none of them (by default the levels from the fifth on): chosen by the library's
     test switches."""
     from paper_2609_22098_b200 import binding
     wl = small("serve32", V=20000, B=5)
