@@ -177,12 +177,22 @@ def snapshot(tree, verdict):
             verdict["acc_len"].clone(), torch.where(va, verdict["acc_tok"], -1), verdict["bonus_tok"].clone())
 
 
+def workload_theta(args, wl, B):
+    """The stopping threshold of the run: --theta if given; for the load sweep the seeded monotone
+    load -> theta schedule at this batch size (the chain sentinel at the largest); the workload's own otherwise."""
+    if args.theta is not None:
+        return args.theta
+    if wl.name == "sweep" and B in synth.SWEEP_BATCHES:
+        return synth.sweep_theta(B, seed=args.seed)
+    return wl.theta
+
+
 def run_ours(args, rank, world, device):
     from paper_2609_22098_b200.binding import TreeSpark
     wl = synth.WORKLOADS[args.workload]
     B = args.batch or wl.B
     T = wl.temps[-1] if args.T is None else args.T
-    theta = wl.theta if args.theta is None else args.theta
+    theta = workload_theta(args, wl, B)
     es = 2 if wl.dtype == "bf16" else 4
     seed = shard.shard_seed(args.seed, rank)
     table = synth.make_calibration_table(wl, args.seed + 4, "fit")
@@ -560,7 +570,7 @@ def run_reference(args):
     wl = synth.WORKLOADS[args.workload]
     B = args.batch or wl.B
     T = wl.temps[-1] if args.T is None else args.T
-    theta = wl.theta if args.theta is None else args.theta
+    theta = workload_theta(args, wl, B)
     cores = os.cpu_count() or 1
     table = synth.make_calibration_table(wl, args.seed + 4, "fit")
     A, W = synth.make_head(wl, args.seed + 1, "cpu")

@@ -231,6 +231,7 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
     const bool on_mma = ctx->use_mma && !(ctx->few_ok && level_bound <= FEW_MAX);
     ScoreExtras ex;
     ex.thr0_ready = scouted_prev;
+    ex.root_B = d == 0 ? B : 0;
     const bool scout = seeds_on && on_mma && d + 1 < c.D;
     ex.u_depth = d; ex.u_B = B;
     if (scout) { ex.utop = (uint2*)(ws + L.utop); ex.scout_live = a.req_npar; ex.scout_B = B; ex.scout_depth = d + 1; }

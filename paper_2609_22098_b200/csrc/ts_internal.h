@@ -20,6 +20,7 @@ struct ScoreArgs {
   int V, D, r, K;
   int P; const int* P_dev;
   const int* P_prev_dev;   // parent count of the previous level (nullptr: none); 0 there means 0 here
+  int seed_root_B;         // seed kernel: > 0 = the parents are the roots of that many requests (parent p = request p at depth 0)
   int pdl;                 // host side: launch with programmatic stream serialization
   int few;                 // host side: this launch runs on the few-parents kernel
   const int *p_req, *p_depth, *p_token; const uint64_t* p_hash;
@@ -71,6 +72,7 @@ void set_seed_pointers(const ts_ctx* ctx, ScoreArgs& a);
 // and scouting of the next level's rows (see ScoreArgs).
 struct ScoreExtras {
   bool thr0_ready = false;
+  int root_B = 0;   // > 0: the parents are the roots of requests 0 .. root_B-1 (parent p = request p, depth 0)
   const int* scout_live = nullptr; int scout_B = 0, scout_depth = -1; uint2* utop = nullptr;
   int u_depth = -1, u_B = 0;
 };

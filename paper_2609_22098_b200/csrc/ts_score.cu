@@ -177,7 +177,9 @@ cudaError_t launch_score(const ts_ctx* ctx, float* rec, int cap, int* err, const
     set_seed_pointers(ctx, a);
     if (!(extras && extras->thr0_ready)) {   // (an expansion's level kernel writes them for the level after it)
       ProfScope ps(ctx, K_SEED, st);
+      a.seed_root_B = extras ? extras->root_B : 0;
       e = launch_seed(ctx, a, st);
+      a.seed_root_B = 0;
       if (e != cudaSuccess) return e;
     }
     if (extras) { a.u_depth = extras->u_depth; a.u_B = extras->u_B; }

@@ -43,10 +43,15 @@ __global__ void __launch_bounds__(SEED_THREADS, 2) seed_parents_kernel(const Sco
   __shared__ int s_last;
   static_assert((SEED_THREADS / 32) * (NSEED_MAX / (SEED_THREADS / 32)) <= NSEED_MAX, "picks fit the candidate arrays");
   const int tid = threadIdx.x;
-  pdl_wait();                // the parent list and its length come from the kernel before
+  // The parent list and its length come from the kernel before -- except for the root level of an expansion, where
+  // parent p is request p at depth 0: there the sweep of the first row (most of this kernel's time) needs nothing
+  // from that kernel and runs beside it; the wait comes before the first thing that does.
+  const bool root = a.seed_root_B > 0;
+  bool waited = !root;
+  if (!root) pdl_wait();
   pdl_launch_dependents();
-  const int P = a.P_dev ? *a.P_dev : a.P;
-  if (P <= 0) return;
+  const int P = root ? a.seed_root_B : (a.P_dev ? *a.P_dev : a.P);
+  if (P <= 0) { if (!waited) pdl_wait(); return; }
   const int V = a.V, r = a.r, K = a.K;
   const int npick = max(1, min(2 * K, NSEED_MAX) / (SEED_THREADS / 32));   // 2K tokens per parent (at least 8)
   const float T = a.T, invT = T > 0.f ? 1.f / T : 1.f;
@@ -61,7 +66,7 @@ __global__ void __launch_bounds__(SEED_THREADS, 2) seed_parents_kernel(const Sco
   const int nvec = V / 8;
   for (int item = blockIdx.x; item < P * nparts; item += gridDim.x) {
     const int p = item / nparts, part = item % nparts;
-    const int req = a.p_req[p], dep = a.p_depth[p];
+    const int req = root ? p : a.p_req[p], dep = root ? 0 : a.p_depth[p];
     const __nv_bfloat16* Urow = Ug + ((size_t)req * a.D + dep) * V;
     if (tid == 0) s_last = 0;
     // ---- the best base logit of every thread's share of this part of the row ------------------------------
@@ -91,6 +96,7 @@ __global__ void __launch_bounds__(SEED_THREADS, 2) seed_parents_kernel(const Sco
     }
     warp_picks(bv, bi, npick, s_tok, s_log);
     __syncthreads();
+    if (!waited) { pdl_wait(); waited = true; }   // arrival counters, parent tokens and hashes, the bound words
     const int n = (SEED_THREADS / 32) * npick;   // places; an empty one holds token -1
     if (nparts > 1) {
       // leave this part's candidates for whoever finishes the parent; the last part to arrive does
@@ -179,6 +185,7 @@ __global__ void __launch_bounds__(SEED_THREADS, 2) seed_parents_kernel(const Sco
     }
     __syncthreads();
   }
+  if (!waited) pdl_wait();
 }
 
 cudaError_t launch_seed(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st) {
