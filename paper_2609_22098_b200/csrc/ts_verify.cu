@@ -135,6 +135,7 @@ struct VerifyArgs {
   uint32_t wait_limit;   // polls before a bounded wait (grid barrier, mbarrier) gives up
   int lost_arrival;      // test switch: grid barriers expect one arrival more than will come
   int w_smem;   // 1: the kernel keeps its range of W in dynamic shared memory
+  int w_stream; // 1 (tensor-core form only): the range does not fit; blocks of W stream through a ring instead
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -486,7 +487,12 @@ constexpr int WALK_MAX_BLK = 32;
 struct WalkTc {
   unsigned char* Ws; unsigned char* As; uint64_t* t_full; uint64_t* t_empty; volatile int* s_abort;
   uint32_t tmem_base, slab_bytes; int rp; uint32_t it;
+  // Streaming form (ranks at which the range of W does not fit shared memory): Ws is a ring of WALK_RING blocks
+  // of WALK_SBLK tokens, refilled by bulk-tensor loads for every block of every reduction.
+  int stream; const CUtensorMap* tm; uint64_t* w_full; uint64_t* w_free; uint32_t wit;
 };
+constexpr int WALK_SBLK = 128;   // tokens per block of the streaming form (two 64-token slabs of W)
+constexpr int WALK_RING = 2;     // blocks of W in flight or in use
 
 // One reduction step on the tensor cores: sum over this CTA's tokens [t0, t0 + tlen) of
 // max(p(w) - C q(w), 0) for up to 128 requests at once.  The low-rank part of the draft logits,
@@ -494,7 +500,7 @@ struct WalkTc {
 // there are few); worker warp w reads the rows of quarter w % 4 and the 16-token chunks of column split
 // w / 4, adds the base logits, and accumulates the residual with the target row.  Partial sums are
 // combined in a fixed order.  Returns false when a bounded wait ran out.
-template <typename TIn>
+template <typename TIn, int BLK>
 __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int tlen, float invT,
                          const int* sb_req, const int* sb_dep, const int* sb_tok, const long long* sb_row,
                          const float* sb_C, const float* sb_zmax, const float* sb_zlogs, const float* sb_lseT, float* s_part) {
@@ -528,7 +534,7 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const int nblk = (tlen + WALK_BLK - 1) / WALK_BLK;
+  const int nblk = (tlen + BLK - 1) / BLK;
   if (warp < WALK_EPI) {
     const int q = warp & 3, s = warp >> 2;
     const int row = q * 32 + lane;
@@ -585,11 +591,11 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
       ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
       if (!ok) { alive = false; break; }
       tc_fence_after();
-      const int nch = min(WALK_BLK / 16, (tlen - nb * WALK_BLK + 15) / 16);
+      const int nch = min(BLK / 16, (tlen - nb * BLK + 15) / 16);
       for (int ca = c0; ca < nch; ca += 2 * cstep) {
         const int cb = ca + cstep;
         const bool hb = cb < nch;   // warp-uniform
-        const int cga = nb * (WALK_BLK / 16) + ca;
+        const int cga = nb * (BLK / 16) + ca;
         uint32_t ra[16], rb[16];
         const uint32_t tbase = tc.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(tb * WALK_BLK);
         tmem_ld16_issue(tbase + (uint32_t)(ca * 16), ra);
@@ -600,7 +606,7 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
         // next pair: the rest of this block, else the first pair of the next block
         {
           int na = cga + 2 * cstep;
-          if (ca + 2 * cstep >= WALK_BLK / 16) na = (nb + 1) * (WALK_BLK / 16) + c0;
+          if (ca + 2 * cstep >= BLK / 16) na = (nb + 1) * (BLK / 16) + c0;
           request(na, 0);
           request(na + cstep, 1);
         }
@@ -617,23 +623,54 @@ __device__ bool mma_pass(const VerifyArgs& a, WalkTc& tc, int nreq, int t0, int 
     s_part[row * 2 + s] = active ? sum : 0.f;
   } else if (warp == WALK_EPI && lane == 0) {
     const uint32_t ws_addr = smem_u32(tc.Ws), as_addr = smem_u32(tc.As);
-    for (int nb = 0; nb < nblk; ++nb) {
+    // streaming form: block nb of this pass goes to ring slot (wit + nb) % WALK_RING, once the MMAs that read the
+    // slot's previous block are done; the next block is requested before this one is waited for
+    int requested = 0, consumed = 0;   // blocks whose loads were issued / whose loads were waited for
+    auto w_request = [&](int nb) -> bool {
+      const uint32_t wi = tc.wit + (uint32_t)nb, slot = wi % WALK_RING, use = wi / WALK_RING;
+      if (use >= 1 && !mbar_wait(tc.w_free + slot, (use - 1) & 1, tc.s_abort, nullptr, a.wait_limit)) return false;
+      const int ns = (tlen - nb * BLK > 64) ? 2 : 1;
+      mbar_expect_tx(tc.w_full + slot, (uint32_t)ns * tc.slab_bytes);
+      for (int h = 0; h < ns; ++h)
+        tma_load_box(tc.Ws + (size_t)(slot * (BLK / 64) + h) * tc.slab_bytes, tc.tm, t0 + nb * BLK + h * 64, 0, tc.w_full + slot);
+      ++requested;
+      return true;
+    };
+    bool live = true;
+    if (tc.stream) live = w_request(0);
+    for (int nb = 0; nb < nblk && live; ++nb) {
       const uint32_t it = tc.it + (uint32_t)nb, tb = it % WALK_NBUF, u = it / WALK_NBUF;
+      uint32_t wslab = (uint32_t)(BLK / 64 * nb);   // first slab of the block's W (resident form)
+      if (tc.stream) {
+        if (nb + 1 < nblk && !w_request(nb + 1)) break;
+        const uint32_t wi = tc.wit + (uint32_t)nb, slot = wi % WALK_RING;
+        if (!mbar_wait(tc.w_full + slot, (wi / WALK_RING) & 1, tc.s_abort, nullptr, a.wait_limit)) break;
+        ++consumed;
+        wslab = slot * (uint32_t)(BLK / 64);
+      }
       if (u >= 1) {
         if (!mbar_wait(tc.t_empty + tb, (u - 1) & 1, tc.s_abort, nullptr, a.wait_limit)) break;
         tc_fence_after();
       }
-      const int n = min(WALK_BLK, (tlen - nb * WALK_BLK + 63) / 64 * 64);   // whole 64-token slabs
+      const int n = min(BLK, (tlen - nb * BLK + 63) / 64 * 64);   // whole 64-token slabs
       const uint32_t idesc = instr_desc(n);
       const uint32_t d_tmem = tc.tmem_base + tb * (uint32_t)WALK_BLK;
       for (int ks = 0; ks < rp / 16; ++ks) {
         const uint64_t adesc = smem_desc(as_addr + (uint32_t)(ks >> 2) * a_slab_bytes + (uint32_t)(ks & 3) * 32u, 16u, 1024u);
-        const uint64_t bdesc = smem_desc(ws_addr + (uint32_t)(WALK_BLK / 64 * nb) * tc.slab_bytes + (uint32_t)ks * 2048u, tc.slab_bytes, 1024u);
+        const uint64_t bdesc = smem_desc(ws_addr + wslab * tc.slab_bytes + (uint32_t)ks * 2048u, tc.slab_bytes, 1024u);
         mma_bf16(d_tmem, adesc, bdesc, idesc, ks > 0 ? 1u : 0u);
       }
       mma_commit(tc.t_full + tb);
+      if (tc.stream) mma_commit(tc.w_free + ((tc.wit + (uint32_t)nb) % WALK_RING));
+    }
+    if (tc.stream && requested > consumed) {
+      // gave up with a block of W on its way: it writes this CTA's shared memory, so wait for it (bounded)
+      const uint32_t wi = tc.wit + (uint32_t)consumed, slot = wi % WALK_RING;
+      bool landed = false;
+      for (uint32_t i = 0; i < WAIT_LIMIT && !landed; ++i) { landed = mbar_try_wait(tc.w_full + slot, (wi / WALK_RING) & 1); if (!landed) __nanosleep(100); }
     }
   }
+  if (tc.stream) tc.wit += (uint32_t)nblk;
   tc.it += (uint32_t)nblk;
   tc_fence_before();
   __syncthreads();
@@ -776,8 +813,11 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
           sb_lseT[tid] = a.node_lseT[(size_t)b * (N + 1) + v + 1];
         }
         __syncthreads();
-        if (!mma_pass<TIn>(a, tc, nreq, v_lo, v_hi - v_lo, invT, sb_req, sb_dep, sb_tok, sb_row, sb_C, sb_zmax, sb_zlogs,
-                           sb_lseT, sb_part)) {
+        const bool pass_ok = tc.stream ? mma_pass<TIn, WALK_SBLK>(a, tc, nreq, v_lo, v_hi - v_lo, invT, sb_req, sb_dep, sb_tok, sb_row, sb_C,
+                                                                  sb_zmax, sb_zlogs, sb_lseT, sb_part)
+                                       : mma_pass<TIn, WALK_BLK>(a, tc, nreq, v_lo, v_hi - v_lo, invT, sb_req, sb_dep, sb_tok, sb_row, sb_C,
+                                                                 sb_zmax, sb_zlogs, sb_lseT, sb_part);
+        if (!pass_ok) {
           if (tid == 0) atomicExch(a.barrier + 1, 1u);   // the word the follow-up kernel checks
           return false;
         }
@@ -942,7 +982,7 @@ __device__ __forceinline__ bool walk_body(const VerifyArgs& a, WalkTc& tc, unsig
           double q = 0.0;
           if (Cw != 0.0) {
             float acc = Elem<TIn>::to_f(reinterpret_cast<const TIn*>(a.U)[((size_t)b * a.D + dep) * a.V + w]);
-            if (MMA && own) {
+            if (MMA && own && !tc.stream) {
               // the range's W columns sit in the tensor-core operand layout: 64-token slabs of [rp][128 B],
               // 16-byte chunk j of row k at chunk j ^ (k & 7)
               const unsigned char* wsl = tc.Ws + (size_t)(o >> 6) * tc.slab_bytes + (o & 7) * 2;
@@ -1010,14 +1050,17 @@ __global__ void __launch_bounds__(WT, 1) verify_walk_kernel(const VerifyArgs a, 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int r = a.r, rp = (r + 63) / 64 * 64;
   const int t0 = blockIdx.x * a.vt_TV, tlen = min(a.vt_TV, a.V - t0);
-  const int nslab = a.vt_TV / 64, nblk = (tlen + 127) / 128;
+  const bool stream = a.w_stream != 0;   // (needs the tensor map: the host selects it only then)
+  const int nslab = stream ? WALK_RING * (WALK_SBLK / 64) : a.vt_TV / 64, nblk = stream ? 0 : (tlen + 127) / 128;
   unsigned char* sm = w_raw + ((1024u - (smem_u32(w_raw) & 1023u)) & 1023u);
   tc.rp = rp; tc.slab_bytes = (uint32_t)rp * 128u; tc.it = 0;
+  tc.stream = stream ? 1 : 0; tc.tm = &tmW; tc.wit = 0;
   tc.Ws = sm;
   tc.As = tc.Ws + (size_t)nslab * tc.slab_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(tc.As + (size_t)(rp / 64) * 128 * 128);
   tc.t_full = bars; tc.t_empty = bars + WALK_NBUF;
   uint64_t* w_full = bars + 2 * WALK_NBUF;
+  tc.w_full = w_full; tc.w_free = w_full + WALK_RING;   // (streaming form: the first 2 * WALK_RING of these barriers)
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(w_full + WALK_MAX_BLK);
   tc.s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   constexpr uint32_t TMEM_COLS = WALK_NBUF * WALK_BLK;
@@ -1028,7 +1071,7 @@ __global__ void __launch_bounds__(WT, 1) verify_walk_kernel(const VerifyArgs a, 
   if (tid == 0) {
     for (int i = 0; i < WALK_NBUF; ++i) { mbar_init(tc.t_full + i, 1); mbar_init(tc.t_empty + i, WALK_EPI); }
     *tc.s_abort = 0;
-    if (use_tma) for (int i = 0; i < nblk; ++i) mbar_init(w_full + i, 1);
+    if (use_tma) for (int i = 0; i < (stream ? 2 * WALK_RING : nblk); ++i) mbar_init(w_full + i, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (use_tma) {
       for (int nb = 0; nb < nblk; ++nb) {
@@ -1095,7 +1138,7 @@ cudaError_t verify_setup(ts_ctx* ctx) {
   cudaError_t e = cudaFuncSetAttribute(verify_walk_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        ctx->max_smem - 40 * 1024);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(verify_walk_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem - 32 * 1024);
+  e = cudaFuncSetAttribute(verify_walk_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem - 12 * 1024);
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(verify_walk_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem - 40 * 1024);
 }
@@ -1165,18 +1208,25 @@ extern "C" int32_t ts_verify_tree(ts_ctx* ctx, const void* U, const void* A, con
   // tensor-core reductions: bf16 everywhere, the range of W in operand layout plus the A tile within shared memory
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
   const size_t mma_bytes = (size_t)(ctx->vt_TV / 64) * rp * 128 + (rp / 64) * 128 * 128 + (2 * WALK_NBUF + WALK_MAX_BLK) * 8 + 64 + 1024;
-  const bool mma = ctx->use_mma && c.dt_Z == TS_DTYPE_BF16 && c.dt_U == TS_DTYPE_BF16 && c.dt_W == TS_DTYPE_BF16 &&
-                   c.dt_A == TS_DTYPE_BF16 && ctx->vt_TV % 64 == 0 && ctx->vt_TV / 128 < WALK_MAX_BLK &&
-                   mma_bytes + 32 * 1024 <= (size_t)ctx->max_smem;
+  const bool mma_shape = ctx->use_mma && c.dt_Z == TS_DTYPE_BF16 && c.dt_U == TS_DTYPE_BF16 && c.dt_W == TS_DTYPE_BF16 &&
+                         c.dt_A == TS_DTYPE_BF16 && ctx->vt_TV % 64 == 0 && ctx->vt_TV / 128 < WALK_MAX_BLK;
+  const bool resident = mma_shape && mma_bytes + 32 * 1024 <= (size_t)ctx->max_smem;
+  // The range of W does not fit (large ranks): blocks of 128 tokens stream through a ring of two, by bulk-tensor
+  // loads, for every reduction.  Needs the tensor map; the kernel's static shared memory is about 9 KB.
+  const size_t stream_bytes = (size_t)WALK_RING * (WALK_SBLK / 64) * rp * 128 + (rp / 64) * 128 * 128 + (2 * WALK_NBUF + WALK_MAX_BLK) * 8 + 64 + 1024;
   int use_tma = 0;
   CUtensorMap tm;
   memset(&tm, 0, sizeof(tm));
-  if (mma && w_tensor_map(ctx, W)) { memcpy(&tm, ctx->tmapW, sizeof(tm)); use_tma = 1; }
+  if (mma_shape && w_tensor_map(ctx, W)) { memcpy(&tm, ctx->tmapW, sizeof(tm)); use_tma = 1; }
+  const bool streaming = mma_shape && !resident && use_tma && stream_bytes + 12 * 1024 <= (size_t)ctx->max_smem;
+  const bool mma = resident || streaming;
+  a.w_stream = streaming ? 1 : 0;
+  if (!mma) use_tma = 0;
   void* kargs[] = {(void*)&a, (void*)&tm, (void*)&use_tma};
   const void* fn = mma ? (const void*)verify_walk_kernel<__nv_bfloat16, true>
                        : (c.dt_Z == TS_DTYPE_BF16 ? (const void*)verify_walk_kernel<__nv_bfloat16, false>
                                                   : (const void*)verify_walk_kernel<float, false>);
-  if (mma) w_bytes = mma_bytes;
+  if (mma) w_bytes = streaming ? stream_bytes : mma_bytes;
   {
     ProfScope ps(ctx, K_WALK, st);
     // cooperative (the grid barriers need every CTA resident) and, where the driver takes both attributes,

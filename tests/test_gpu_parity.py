@@ -329,10 +329,11 @@ def test_tempered_calibrator_switch_matches_oracle(calib_mode):
         ts.set_ablation(2)
 
 
-@pytest.mark.parametrize("dtype", ["bf16", "f32"])
-def test_round_at_the_papers_own_shape_matches_oracle(dtype):
+@pytest.mark.parametrize("dtype,V,B", [("bf16", 20000 + 8, 6), ("f32", 20000 + 8, 6),
+                                       ("bf16", 60000 + 8, 4)])   # a range of W that no longer fits shared memory: the walk streams it
+def test_round_at_the_papers_own_shape_matches_oracle(dtype, V, B):
     # rank 256, block of 7, 56 nodes, 8 siblings (Section 5.1), on a vocabulary the oracle finishes quickly
-    wl = small("serve32", V=20000 + 8, r=256, D=7, Nmax=56, K=8, B=6, dtype=dtype)
+    wl = small("serve32", V=V, r=256, D=7, Nmax=56, K=8, B=B, dtype=dtype)
     rnd = Round(wl, seed=97)
     ts = make_gpu(wl, rnd.table, max_batch=rnd.B)
     orc = make_oracle(wl, rnd.table)
