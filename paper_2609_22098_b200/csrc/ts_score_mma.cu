@@ -286,8 +286,10 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       const int row = q * 32 + lane;
       const int e = warp * 32 + lane;
       const int cpr = rp / 8;          // 16-byte chunks per A row
-      // gather this group's parent rows A[x_p] into the swizzled A tile
-      for (int idx = e; idx < 128 * cpr; idx += EPI_WARPS * 32) {
+      // gather this group's parent rows A[x_p] into the swizzled A tile (a later tile of a launch with one group
+      // finds them in place)
+      const bool a_in_place = tile_it > 0 && ngroups == 1;
+      for (int idx = e; idx < 128 * cpr && !a_in_place; idx += EPI_WARPS * 32) {
         const int rr = idx / cpr, ck = idx % cpr;
         const int p = R > 1 ? rr % per : g * 128 + rr;
         uint4 v = make_uint4(0, 0, 0, 0);
@@ -297,7 +299,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       if (UMMA) {
         // one more K-slab of the A tile: column b of row rr is 1 when the row's parent belongs to request b, so the
         // MMA adds that request's base logits (rows of the base-logit slab) to the row's bias
-        for (int idx = e; idx < 128 * 8; idx += EPI_WARPS * 32) {
+        for (int idx = e; idx < 128 * 8 && !a_in_place; idx += EPI_WARPS * 32) {
           const int rr = idx >> 3, ck = idx & 7;
           const int p = R > 1 ? rr % per : g * 128 + rr;
           uint4 v = make_uint4(0, 0, 0, 0);
