@@ -217,10 +217,13 @@ extern "C" int32_t ts_expand_tree(ts_ctx* ctx, const void* U, const void* A, con
   // three launches per empty level (each a hop in the chain of dependent launches) become one that returns at once.
   // TS_TEST_PERSIST: the cooperative launch runs every level.  TS_TEST_NO_TAIL: no cooperative launch at all.
   constexpr int TAIL_FROM = 4;
-  const bool coop_ok = seeds_on && persistent_supported(ctx, B);
   int coop_from = c.D;   // first level of the cooperative launch (D: none)
-  if (coop_ok && (ctx->test_mode & TS_TEST_PERSIST)) coop_from = 0;
-  else if (coop_ok && !(ctx->test_mode & TS_TEST_NO_TAIL) && c.D > TAIL_FROM + 1) coop_from = TAIL_FROM;
+  if (seeds_on && (ctx->test_mode & TS_TEST_PERSIST) && persistent_supported(ctx, B, 0)) coop_from = 0;
+  else if (seeds_on && !(ctx->test_mode & TS_TEST_NO_TAIL)) {
+    // (a handful of requests rarely has parents at the fourth level either: one level earlier there)
+    const int from = (ctx->few_ok && B <= FEW_MAX) ? TAIL_FROM - 1 : TAIL_FROM;
+    if (c.D > from + 1 && persistent_supported(ctx, B, from)) coop_from = from;
+  }
   long long level_bound = B;   // parents a level can have at most: B at the root, K times more per level, B * Nmax overall
   // Seed bounds of a level on the tensor-core kernel: made by the level kernel before it when that level's scoring
   // launch scouted the rows (it does whenever it runs on the tensor-core kernel itself); by a seed launch otherwise

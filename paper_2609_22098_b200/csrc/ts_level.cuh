@@ -69,7 +69,7 @@ struct PersistArgs {
 };
 
 // host side of the persistent form (ts_score_mma.cu)
-bool persistent_supported(const ts_ctx* ctx, int B);
+bool persistent_supported(const ts_ctx* ctx, int B, int first_level);
 cudaError_t launch_expand_persistent(const ts_ctx* ctx, const ScoreArgs& a, const PersistArgs& pa, cudaStream_t st);
 
 constexpr int LEVEL_THREADS = 256;

@@ -960,10 +960,17 @@ static size_t persist_overlay_bytes(const ts_config& c) {
   return (size_t)NSEL * QCAP * 16 + (size_t)128 * 5 * c.K * 4 + 2 * 128 * 4 + 2 * EPI_S * 128 * 4 + 3 * EPI_S * 128 * 4;
 }
 
-bool persistent_supported(const ts_ctx* ctx, int B) {
+bool persistent_supported(const ts_ctx* ctx, int B, int first_level) {
   const ts_config& c = ctx->cfg;
   if (!ctx->use_mma || c.K > 8) return false;                 // (the merge of the persistent form keeps 8-entry lists in registers)
-  if (ctx->few_ok && B <= FEW_MAX) return false;              // single-request decoding: the few-parents kernel serves the first levels
+  if (ctx->few_ok) {
+    // Levels that can hold only a few parents run on the few-parents kernel, which neither scouts nor takes seed bounds:
+    // the cooperative launch must start at a level that the tensor-core kernel serves, and (unless it starts at the
+    // root, where a seed launch precedes it) so must the level before, whose scouts feed its first seed bounds.
+    long long bound = B;
+    for (int l = 0; l < (first_level > 0 ? first_level - 1 : 0); ++l) bound = bound * c.K < (long long)B * c.Nmax ? bound * c.K : (long long)B * c.Nmax;
+    if (bound <= FEW_MAX) return false;
+  }
   if (ctx->tile.ntiles > ctx->num_sms) return false;          // every CTA must be resident: the phases are separated by grid barriers
   const size_t ov = persist_overlay_bytes(c);
   return sizeof(MergeSmem) <= ov && ((sizeof(LevelSmem) + 15) & ~(size_t)15) + level_smem_bytes(c) <= ov;
