@@ -50,7 +50,7 @@ static bool select_paths(ts_ctx* ctx) {
   ctx->use_mma = (c.dt_U == TS_DTYPE_BF16 && c.r % 8 == 0 && c.V % 8 == 0 && ctx->cc_major == 10 && !(tm & TS_TEST_FORCE_FMA)) ? 1 : 0;
   ctx->tma_state = (tm & TS_TEST_NO_TMA) ? -1 : 0;
   ctx->tmapW_ptr = nullptr;
-  if (ctx->use_mma && !choose_tile_mma(c, ctx->num_sms, ctx->max_smem, &ctx->tile)) ctx->use_mma = 0;
+  if (ctx->use_mma && !choose_tile_mma(c, ctx->num_sms, ctx->max_smem, !(tm & TS_TEST_NO_TMA), &ctx->tile)) ctx->use_mma = 0;
   if (!ctx->use_mma && !choose_tile(c, ctx->num_sms, ctx->max_smem, &ctx->tile)) return false;
   ctx->few_ok = (few_supported(ctx) && !(tm & TS_TEST_NO_FEW)) ? 1 : 0;
   ctx->wait_limit = (tm & TS_TEST_SHORT_WAITS) ? 4096u : WAIT_LIMIT;

@@ -52,6 +52,7 @@ struct TileCfg {
   int ntiles;   // tiles covering V
   size_t smem;  // dynamic shared memory of the scoring kernel
   int umma;     // the tiling leaves room for the one-hot slab and the base-logit slab ring (base logits through the MMA)
+  int w_ring;   // 0: the W tile is resident; > 0: that many 64-token slabs of W stream through a ring (large ranks)
 };
 
 }  // namespace ts

@@ -20,6 +20,7 @@ struct ScoreArgs {
   int V, D, r, K;
   int P; const int* P_dev;
   const int* P_prev_dev;   // parent count of the previous level (nullptr: none); 0 there means 0 here
+  int w_ring;              // tensor-core kernel: 0 = resident W tile, > 0 = slabs of the W ring (streaming form)
   int seed_root_B;         // seed kernel: > 0 = the parents are the roots of that many requests (parent p = request p at depth 0)
   int pdl;                 // host side: launch with programmatic stream serialization
   int few;                 // host side: this launch runs on the few-parents kernel
@@ -97,7 +98,7 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out);
+bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, bool allow_stream, TileCfg* out);
 cudaError_t score_mma_setup(ts_ctx* ctx);
 cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t st);
 // seed bounds of every parent of the list (ts_seed.cu); runs ahead of the tensor-core scoring kernel

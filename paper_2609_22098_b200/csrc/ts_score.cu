@@ -139,7 +139,7 @@ ScoreArgs make_score_args(const ts_ctx* ctx, float* rec, int cap, int* err, cons
   const ts_config& c = ctx->cfg;
   ScoreArgs a{};
   a.U = U; a.A = A; a.W = W; a.V = c.V; a.D = c.D; a.r = c.r; a.K = c.K; a.T = T; a.seed = seed;
-  a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.cap = cap; a.S = 1; a.rec = rec; a.err = err;
+  a.TV = ctx->tile.TV; a.ntiles = ctx->tile.ntiles; a.w_ring = ctx->use_mma ? ctx->tile.w_ring : 0; a.cap = cap; a.S = 1; a.rec = rec; a.err = err;
   a.wait_limit = ctx->wait_limit;
   a.lost_arrival = (ctx->test_mode & TS_TEST_LOST_ARRIVAL) ? 1 : 0;
   a.thr = thr_base(ctx, rec, cap); a.slots = a.thr + 2 * (size_t)cap;

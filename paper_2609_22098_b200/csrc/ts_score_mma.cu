@@ -142,8 +142,9 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   // the SMs; at large ranks, where the W tile is small, a CTA takes several in turn and pays its set-up once)
   int tile = blockIdx.x, t0 = tile * TV, tlen = min(TV, V - t0);
   int tile_it = 0;          // tiles this CTA has finished: the W barriers' phase
-  const int nslab = TV / 64;
-  int nblk_w = (tlen + WBLK - 1) / WBLK;
+  const int wring = UMMA ? 0 : a.w_ring;   // > 0: W streams through a ring of that many 64-token slabs (one tile per CTA)
+  const int nslab = wring ? wring : TV / 64;
+  int nblk_w = wring ? 0 : (tlen + WBLK - 1) / WBLK;
   const uint32_t slab_bytes = (uint32_t)rp * 128u;       // one 64-token slab of W
   const uint32_t a_slab_bytes = 128u * 128u;             // 128 rows x 128 B
   unsigned char* sm = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -166,7 +167,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   uint64_t* w_full = bars + 1 + 2 * NBUF;  // [MAX_BLK] W slabs of block nb landed
   uint64_t* u_full = w_full + MAX_BLK;     // [NUB] base-logit slab landed
   uint64_t* u_free = u_full + NUB;         // [NUB] the MMAs that read the slab are done
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(u_free + NUB);
+  uint64_t* w_free = u_free + NUB;         // [MAX_BLK] streaming form: the MMAs that read the ring slot are done
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(w_free + MAX_BLK);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   volatile int* s_done = reinterpret_cast<volatile int*>(s_tmem + 2);             // scanning warps finished (cumulative)
   sh.q_head = reinterpret_cast<volatile unsigned*>(s_tmem + 4);
@@ -197,7 +199,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
     *s_abort = 0;
     *s_done = 0;
     for (int i = 0; i < NSEL; ++i) { sh.q_head[i] = 0u; sh.q_tail[i] = 0u; }
-    if (use_tma) for (int i = 0; i < nblk_w; ++i) mbar_init(w_full + i, 1);
+    if (use_tma) for (int i = 0; i < (wring ? wring : nblk_w); ++i) mbar_init(w_full + i, 1);
+    for (int i = 0; i < wring; ++i) mbar_init(w_free + i, 1);
     for (int i = 0; i < NUB; ++i) { mbar_init(u_full + i, 1); mbar_init(u_free + i, 1); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // W tile by bulk-tensor loads, one barrier per block of 128 tokens so that the first MMAs start while
@@ -205,7 +208,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
     // before the kernel may look at its own parent count, when the level before was large enough for this
     // one to be populated almost surely; after the count is known otherwise (a level that turns out empty then
     // fetches nothing).
-    if (use_tma && early_w) issue_w();
+    if (use_tma && early_w && !wring) issue_w();
   }
   auto fill_w_plain = [&]() {  // W tile: 16-byte chunks (8 tokens of one row), swizzled: chunk j of row k lands at chunk j ^ (k & 7)
     const int per_slab = rp * 8;
@@ -217,7 +220,7 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
       *reinterpret_cast<uint4*>(Ws + (size_t)slab * slab_bytes + k * 128 + ((j ^ (k & 7)) << 4)) = v;
     }
   };
-  if (!use_tma) fill_w_plain();
+  if (!use_tma && !wring) fill_w_plain();
   fill_gumbel_bounds(ghi, tid, MMA_THREADS);
   for (int i = tid; i < 512; i += MMA_THREADS) s_thr[i] = 0u;
   auto reset_selection = [&]() {   // empty lists, no local thresholds, nothing published
@@ -242,7 +245,8 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   uint32_t ul = 0;          // block pairs of all groups before this one (MMA issuer: slot and use of their base-logit slabs)
   unsigned gen = 0;         // grid barriers passed
   bool dead = false;        // a bounded wait ran out somewhere
-  bool w_issued = use_tma && early_w;   // bulk loads of the W tile are (or were) in flight
+  bool w_issued = (use_tma && early_w) || wring;   // bulk loads of the W tile are (or were) in flight (streaming form: the issuer's business)
+  uint32_t wl = 0;          // streaming form: slabs of all groups before this one (ring slot and use of a block's slab)
   int gg_tile = 0;          // value of gg when the current tile began: its first group waits for the tile's W blocks
   for (;;) {   // this CTA's tiles
   gg_tile = gg;
@@ -686,6 +690,51 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
             if (spin > 8) __nanosleep(32);
           }
           ul += (uint32_t)npair;
+        } else if (wring) {
+          // Streaming form: the tile's 64-token slabs of W pass through a ring of `wring` slots, block nb of the
+          // kernel's running count in slot nb % wring; a slot is free again when the MMAs that read it are done.
+          // Blocks are issued in order, each as soon as its slab has landed and its accumulator buffer is drained;
+          // slabs are requested as far ahead as the ring allows.
+          int nb = 0, req = 0;
+          uint32_t spin = 0;
+          while (nb < nblk) {
+            while (req < nblk && req < nb + wring) {
+              const uint32_t gx = wl + (uint32_t)req, slot = gx % (uint32_t)wring, use = gx / (uint32_t)wring;
+              if (use >= 1 && !mbar_test_wait(w_free + slot, (use - 1) & 1)) break;
+              mbar_expect_tx(w_full + slot, slab_bytes);
+              tma_load_box(Ws + (size_t)slot * slab_bytes, &tmW, t0 + req * BLK_N, 0, w_full + slot);
+              ++req;
+            }
+            const int sp = nb % EPI_S, nuse = (nblk - sp + EPI_S - 1) / EPI_S;
+            const int j = nb / EPI_S, h = j & 1, tb = sp + EPI_S * h;
+            const int u = gg * ((nuse + 1 - h) >> 1) + (j >> 1);
+            const uint32_t gx = wl + (uint32_t)nb, slot = gx % (uint32_t)wring;
+            if (nb < req && (u < 1 || mbar_test_wait(t_empty + tb, (u - 1) & 1)) && mbar_test_wait(w_full + slot, (gx / (uint32_t)wring) & 1)) {
+              tc_fence_after();
+              const uint32_t idesc = instr_desc(BLK_N);
+              const uint32_t d_tmem = tmem_base + (uint32_t)(tb * BLK_N);
+              for (int ks = 0; ks < rp / 16; ++ks) {
+                const uint64_t adesc = smem_desc(as_addr + (uint32_t)(ks >> 2) * a_slab_bytes + (uint32_t)(ks & 3) * 32u, 16u, 1024u);
+                const uint64_t bdesc = smem_desc(ws_addr + slot * slab_bytes + (uint32_t)ks * 2048u, slab_bytes, 1024u);
+                mma_bf16(d_tmem, adesc, bdesc, idesc, ks > 0 ? 1u : 0u);
+              }
+              mma_commit(t_full + tb);
+              mma_commit(w_free + slot);
+              ++nb;
+              spin = 0;
+              continue;
+            }
+            if (*s_abort) break;
+            if (++spin > wait_limit) { *s_abort = 1; if (a.err) atomicExch(a.err, 1); break; }
+            if (spin > 8) __nanosleep(32);
+          }
+          // gave up with slabs on their way: they write this CTA's shared memory, so wait for them (bounded)
+          for (int x = nb; x < req; ++x) {
+            const uint32_t gx = wl + (uint32_t)x, slot = gx % (uint32_t)wring;
+            bool landed = false;
+            for (uint32_t t = 0; t < WAIT_LIMIT && !landed; ++t) { landed = mbar_test_wait(w_full + slot, (gx / (uint32_t)wring) & 1); if (!landed) __nanosleep(100); }
+          }
+          wl += (uint32_t)nblk;
         } else {
         // each split's pipeline advances on its own: whichever buffer is drained (and whose W block has landed) is refilled
         int nxt[EPI_S];
@@ -831,7 +880,7 @@ static size_t mma_fixed_smem(const ts_config& c, bool umma) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
   const size_t K = (size_t)c.K;
   return (rp / 64 + (umma ? 1 : 0)) * 128 * 128 + (umma ? (size_t)NUB * UMMA_REQ * 128 : 0) + 512 * 4 + (size_t)NSEL * QCAP * 16 + 128 * 5 * K * 4 + 2 * 128 * 4 +
-         2 * EPI_S * 128 * 4 + 3 * EPI_S * 128 * 4 + 512 * 4 + (1 + 2 * NBUF + MAX_BLK + 2 * NUB) * 8 + 64 + 1024;
+         2 * EPI_S * 128 * 4 + 3 * EPI_S * 128 * 4 + 512 * 4 + (1 + 2 * NBUF + 2 * MAX_BLK + 2 * NUB) * 8 + 64 + 1024;
 }
 
 // tile size for the tensor-core path: W tile + the rest within the shared-memory limit,
@@ -852,18 +901,37 @@ static bool choose_tile_mma_for(const ts_config& c, int num_sms, int max_smem, b
   out->TV = tv;
   out->ntiles = (c.V + tv - 1) / tv;
   out->smem = (size_t)(tv / 64) * rp * 128 + fixed;
+  out->w_ring = 0;
   return out->ntiles <= 4096;
+}
+
+// Streaming form for ranks at which a resident W tile would take more than two waves of CTAs: one tile per SM, W
+// in 64-token slabs through a ring that takes what shared memory is left (the scanning threads add the base logits).
+static bool choose_stream_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
+  const size_t rp = (size_t)(c.r + 63) / 64 * 64;
+  const size_t fixed = mma_fixed_smem(c, false);
+  if ((size_t)max_smem < fixed + 3 * rp * 128) return false;
+  int ring = (int)(((size_t)max_smem - fixed) / (rp * 128));
+  if (ring > MAX_BLK) ring = MAX_BLK;
+  const int tv = ((c.V + num_sms - 1) / num_sms + 63) / 64 * 64;
+  if (tv > 4096) return false;
+  out->TV = tv; out->ntiles = (c.V + tv - 1) / tv; out->umma = 0; out->w_ring = ring;
+  out->smem = (size_t)ring * rp * 128 + fixed;
+  return true;
 }
 
 // With room for the one-hot slab and the base-logit slabs (base logits through the MMA) unless that costs waves: at
 // large ranks the W tile is what shared memory is short of, and every wave pays the kernel's set-up again.
-bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
+bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, bool allow_stream, TileCfg* out) {
   TileCfg with{}, without{};
   const bool ok_with = choose_tile_mma_for(c, num_sms, max_smem, true, &with);
   const bool ok_without = choose_tile_mma_for(c, num_sms, max_smem, false, &without);
-  if (!ok_with && !ok_without) return false;
   auto waves = [&](const TileCfg& t) { return (t.ntiles + num_sms - 1) / num_sms; };
-  *out = (ok_with && (!ok_without || waves(with) <= waves(without))) ? with : without;
+  TileCfg stream{};
+  const bool ok_stream = allow_stream && choose_stream_mma(c, num_sms, max_smem, &stream);
+  if (!ok_with && !ok_without && !ok_stream) return false;
+  if (ok_with || ok_without) *out = (ok_with && (!ok_without || waves(with) <= waves(without))) ? with : without;
+  if (ok_stream && ((!ok_with && !ok_without) || waves(*out) > 2)) *out = stream;
   return true;
 }
 
@@ -949,6 +1017,7 @@ cudaError_t launch_score_mma(const ts_ctx* ctx, const ScoreArgs& a, cudaStream_t
   const bool umma = use_umma(c, a, false, use_tma);
   if (umma) memcpy(&tu, c->tmapU, sizeof(tu));
   const int grid = a.ntiles < ctx->num_sms ? a.ntiles : ctx->num_sms;   // one CTA per SM at most: a CTA takes its tiles in turn
+  if (a.w_ring > 0 && !use_tma) return cudaErrorNotSupported;           // the streaming form moves W by bulk-tensor loads only
   const cudaError_t e = umma ? launch_kernel(score_mma_kernel<true>, grid, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma, pa, tu)
                              : launch_kernel(score_mma_kernel<false>, grid, MMA_THREADS, ctx->tile.smem, st, a.pdl != 0, a, tm, use_tma, pa, tu);
   return e != cudaSuccess ? e : cudaGetLastError();
