@@ -905,7 +905,7 @@ static bool choose_tile_mma_for(const ts_config& c, int num_sms, int max_smem, b
   return out->ntiles <= 4096;
 }
 
-// Streaming form for ranks at which a resident W tile would take more than two waves of CTAs: one tile per SM, W
+// Streaming form for ranks at which a resident W tile would take more than one wave of CTAs: one tile per SM, W
 // in 64-token slabs through a ring that takes what shared memory is left (the scanning threads add the base logits).
 static bool choose_stream_mma(const ts_config& c, int num_sms, int max_smem, TileCfg* out) {
   const size_t rp = (size_t)(c.r + 63) / 64 * 64;
@@ -931,7 +931,7 @@ bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, bool allow_s
   const bool ok_stream = allow_stream && choose_stream_mma(c, num_sms, max_smem, &stream);
   if (!ok_with && !ok_without && !ok_stream) return false;
   if (ok_with || ok_without) *out = (ok_with && (!ok_without || waves(with) <= waves(without))) ? with : without;
-  if (ok_stream && ((!ok_with && !ok_without) || waves(*out) > 2)) *out = stream;
+  if (ok_stream && ((!ok_with && !ok_without) || waves(*out) > 1)) *out = stream;
   return true;
 }
 
