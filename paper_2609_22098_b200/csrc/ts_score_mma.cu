@@ -127,7 +127,9 @@ __device__ __forceinline__ void select_candidate(const ScoreArgs& a, const SelSh
   }
 }
 
-template <bool UMMA>
+// BIGK: the instantiation whose cooperative form merges with 16-entry lists (K > 8); it exists beside the other
+// one so that the merge's registers do not weigh on the scan of the launches that never merge.
+template <bool UMMA, bool BIGK = false>
 __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreArgs a, const __grid_constant__ CUtensorMap tmW, const int use_tma, const __grid_constant__ PersistArgs pa,
                                                                    const __grid_constant__ CUtensorMap tmU) {
   extern __shared__ unsigned char smem_raw[];
@@ -823,15 +825,19 @@ __global__ void __launch_bounds__(MMA_THREADS, 1) score_mma_kernel(const ScoreAr
   if (!persist || dead) break;
   // ---- persistent form: merge, level step, next level -------------------------------------------------------
   {
-    unsigned char* ov = reinterpret_cast<unsigned char*>(sh.q);   // queues, lists and partial sums are idle between scans
+    // queues, lists and partial sums are idle between scans; in the streaming form so is the (larger) ring of W slabs:
+    // every slab of the level was consumed before its last group ended, and none is requested ahead of a level
+    unsigned char* ov = wring ? Ws : reinterpret_cast<unsigned char*>(sh.q);
     const unsigned nexpect = gridDim.x + (pa.lost_arrival ? 1u : 0u);
     __threadfence();   // this CTA's records
     if (!grid_barrier(pa.barrier, nexpect, gen, wait_limit)) { dead = true; break; }
     if (tid < MERGE_THREADS) {
       MergeArgs mg = pa.mg;
       mg.P = P; mg.P_dev = nullptr;
-      for (int p = blockIdx.x; p < P; p += gridDim.x)
-        merge_parent<8>(mg, p, P, *reinterpret_cast<MergeSmem*>(ov), tid, NamedSync<1, MERGE_THREADS>());
+      for (int p = blockIdx.x; p < P; p += gridDim.x) {
+        if (BIGK) merge_parent<KMAX>(mg, p, P, *reinterpret_cast<MergeSmem*>(ov), tid, NamedSync<1, MERGE_THREADS>());
+        else merge_parent<8>(mg, p, P, *reinterpret_cast<MergeSmem*>(ov), tid, NamedSync<1, MERGE_THREADS>());
+      }
     }
     __threadfence();   // merged results
     if (!grid_barrier(pa.barrier, nexpect, gen, wait_limit)) { dead = true; break; }
@@ -938,6 +944,8 @@ bool choose_tile_mma(const ts_config& c, int num_sms, int max_smem, bool allow_s
 cudaError_t score_mma_setup(ts_ctx* ctx) {
   cudaError_t e = cudaFuncSetAttribute(score_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(score_mma_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(score_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->tile.smem);
 }
 
@@ -1031,7 +1039,7 @@ static size_t persist_overlay_bytes(const ts_config& c) {
 
 bool persistent_supported(const ts_ctx* ctx, int B, int first_level) {
   const ts_config& c = ctx->cfg;
-  if (!ctx->use_mma || c.K > 8) return false;                 // (the merge of the persistent form keeps 8-entry lists in registers)
+  if (!ctx->use_mma || (c.K > 8 && !ctx->tile.w_ring)) return false;   // (only the streaming form's instantiation carries the merge with 16-entry lists)
   if (ctx->few_ok) {
     // Levels that can hold only a few parents run on the few-parents kernel, which neither scouts nor takes seed bounds:
     // the cooperative launch must start at a level that the tensor-core kernel serves, and (unless it starts at the
@@ -1041,7 +1049,7 @@ bool persistent_supported(const ts_ctx* ctx, int B, int first_level) {
     if (bound <= FEW_MAX) return false;
   }
   if (ctx->tile.ntiles > ctx->num_sms) return false;          // every CTA must be resident: the phases are separated by grid barriers
-  const size_t ov = persist_overlay_bytes(c);
+  const size_t ov = ctx->tile.w_ring ? (size_t)ctx->tile.w_ring * ((size_t)(c.r + 63) / 64 * 64) * 128 : persist_overlay_bytes(c);
   return sizeof(MergeSmem) <= ov && ((sizeof(LevelSmem) + 15) & ~(size_t)15) + level_smem_bytes(c) <= ov;
 }
 
@@ -1054,7 +1062,8 @@ cudaError_t launch_expand_persistent(const ts_ctx* ctx, const ScoreArgs& a, cons
   memset(&tu, 0, sizeof(tu));
   const bool umma = use_umma(c, a, true, use_tma);
   if (umma) memcpy(&tu, c->tmapU, sizeof(tu));
-  const void* fn = umma ? (const void*)score_mma_kernel<true> : (const void*)score_mma_kernel<false>;
+  const void* fn = umma ? (const void*)score_mma_kernel<true>
+                        : (ctx->cfg.K > 8 ? (const void*)score_mma_kernel<false, true> : (const void*)score_mma_kernel<false>);
   void* kargs[] = {(void*)&a, (void*)&tm, (void*)&use_tma, (void*)&pa, (void*)&tu};
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(a.ntiles); cfg.blockDim = dim3(MMA_THREADS); cfg.dynamicSmemBytes = ctx->tile.smem; cfg.stream = st;
