@@ -29,13 +29,13 @@ def small(name, **kw):
                                    (45000 + 8, 256, 8)])                   # more vocabulary tiles than SMs: a CTA takes several in turn
 @pytest.mark.parametrize("T", [0.0, 0.7, 1.0])
 @pytest.mark.parametrize("P", [11, 3])   # 3: the few-parents kernel where the context has one
-def test_score_parents_matches_oracle(dtype, V, r, K, T, P):
+def test_score_parents_matches_oracle(dtype, V, r, K, T, P, test_mode=0):
     if dtype == "f32" and V > 40000 and r == 256:
         pytest.skip("the fp32 kernel keeps r x 128 head values and its W tile in shared memory: at this rank it tiles "
                     "vocabularies up to 32,768 tokens and ts_create answers TS_ERR_UNSUPPORTED beyond")
     wl = small("tiny", V=V, r=r, K=K, D=3, Nmax=16, dtype=dtype, B=3, calib_mode=0)
     rnd = Round(wl, seed=11 + V)
-    ts = make_gpu(wl, None, max_batch=3)
+    ts = make_gpu(wl, None, max_batch=3, test_mode=test_mode)
     orc = make_oracle(wl, None)
     g = torch.Generator().manual_seed(V)
     req = torch.randint(0, 3, (P,), generator=g, dtype=torch.int32)
@@ -61,6 +61,14 @@ def test_score_parents_matches_oracle(dtype, V, r, K, T, P):
         if K > V:
             assert (out["top_tok"][i, V:] == -1).all() and (out["draw_tok"][i, V:] == -1).all()
     assert checked >= P - 2
+
+
+def test_score_parents_more_tiles_than_sms_without_a_tensor_map():
+    """Rank 256 on a vocabulary that needs more resident W tiles than there are SMs: with a tensor map the kernel
+    streams W through a ring (the case in the list above); without one it keeps the tiled form, a CTA taking its
+    tiles in turn and staging W with plain loads."""
+    from paper_2609_22098_b200 import binding
+    test_score_parents_matches_oracle("bf16", 45000 + 8, 256, 8, 1.0, 11, test_mode=binding.TEST_NO_TMA)
 
 
 # ---------------------------------------------------------------------------------------------
