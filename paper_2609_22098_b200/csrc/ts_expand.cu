@@ -133,11 +133,11 @@ __global__ void __launch_bounds__(256) expand_finalize_kernel(FinalArgs a) {
 
 // the level kernel ranks a request's pool and candidates out of dynamic shared memory: opt in once per context
 // dynamic shared memory of the level kernel: the ranking entries of a request's pool and candidates, later
-// reused for the seed bounds' staged W columns [2K][r] and per-pair results [Nmax][2K][2]
+// reused for the seed bounds' staged W columns [2K][r], per-pair results [Nmax][2K][2] and a batch of rows of A
 size_t level_smem_bytes(const ts_config& c) {
   const size_t entries = (size_t)(c.Nmax + c.Nmax * c.K) * sizeof(Entry);
   const size_t ns = (size_t)(2 * c.K > NSEED_MAX ? NSEED_MAX : (2 * c.K < 8 ? 8 : 2 * c.K));
-  const size_t seeds = ns * (size_t)c.r * 4 + (size_t)c.Nmax * ns * 2 * 4;
+  const size_t seeds = ns * (size_t)(c.r + 1) * 4 + (size_t)c.Nmax * ns * 2 * 4 + (size_t)SEED_PBATCH * c.r * 2;
   return entries > seeds ? entries : seeds;
 }
 

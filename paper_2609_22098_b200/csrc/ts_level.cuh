@@ -73,6 +73,7 @@ bool persistent_supported(const ts_ctx* ctx, int B, int first_level);
 cudaError_t launch_expand_persistent(const ts_ctx* ctx, const ScoreArgs& a, const PersistArgs& pa, cudaStream_t st);
 
 constexpr int LEVEL_THREADS = 256;
+constexpr int SEED_PBATCH = 64;    // parents whose rows of A the seed phase stages at a time
 
 // shared-memory state of one level step (beside the dynamic array of level_smem_bytes())
 struct LevelSmem {
@@ -354,8 +355,11 @@ __device__ __forceinline__ void level_step(const ExpandArgs& a, const int d, con
       const int npick = max(1, min(2 * K, NSEED_MAX) / 8), NSn = 8 * npick;
       const float invT = a.T > 0.f ? 1.f / a.T : 1.f;
       sync();   // the Entry array in dynamic shared memory is free now
-      float* Wc = reinterpret_cast<float*>(sm_raw);            // [NSn][r]
-      float* res = Wc + (size_t)NSn * r;                        // [cnt][NSn][2]: logit, key
+      // (rows of r + 1 words: the threads of a warp read the same k of different picks, which an even row length
+      // puts into one bank)
+      const int rs = r + 1;
+      float* Wc = reinterpret_cast<float*>(sm_raw);            // [NSn][r + 1]
+      float* res = Wc + (size_t)NSn * rs;                       // [cnt][NSn][2]: logit, key
       if (par) {
         const int i = off + __popc(bal & ((1u << lane) - 1u));
         s_pli[i] = my_li; s_ptok[i] = a.pl_tok[pb + s_new[tid]]; s_phash[i] = a.pl_hash[pb + s_new[tid]];
@@ -386,36 +390,47 @@ __device__ __forceinline__ void level_step(const ExpandArgs& a, const int d, con
       const __nv_bfloat16* Urow = reinterpret_cast<const __nv_bfloat16*>(a.U) + ((size_t)b * a.D + (d + 1)) * V;
       for (int e = tid; e < NSn * r; e += LEVEL_THREADS) {
         const int j = e / r, k = e % r;
-        Wc[e] = s_stok[j] >= 0 ? __bfloat162float(Wg[(size_t)k * V + s_stok[j]]) : 0.f;
+        Wc[(size_t)j * rs + k] = s_stok[j] >= 0 ? __bfloat162float(Wg[(size_t)k * V + s_stok[j]]) : 0.f;
       }
       if (tid < NSn) s_sval[tid] = s_stok[tid] >= 0 ? __bfloat162float(Urow[s_stok[tid]]) : -INFINITY;
       sync();
-      for (int e = tid; e < cnt * NSn; e += LEVEL_THREADS) {
-        const int i = e / NSn, j = e % NSn;
-        float lg = -INFINITY, key = -INFINITY;
-        const int tok = s_stok[j];
-        if (tok >= 0) {
-          const uint4* arow = reinterpret_cast<const uint4*>(Ag + (size_t)s_ptok[i] * r);   // r is a multiple of 8 on this path
-          float dot = 0.f;
-          for (int k8 = 0; k8 < r / 8; ++k8) {
-            float av[8];
-            unpack_bf16x8(__ldg(arow + k8), av);
+      // The parents' rows of A are staged in shared memory a batch of SEED_PBATCH parents at a time (one coalesced
+      // sweep per batch): read per pair from global memory they were r / 8 dependent round trips per pair, and a
+      // request of the wide configuration has 5,000 pairs.
+      uint4* Ast = reinterpret_cast<uint4*>(res + (size_t)a.N * NSn * 2);   // [SEED_PBATCH][r] bf16
+      const int cpr = r / 8;                                                  // r is a multiple of 8 on this path
+      for (int i0 = 0; i0 < cnt; i0 += SEED_PBATCH) {
+        const int nbat = min(SEED_PBATCH, cnt - i0);
+        for (int e = tid; e < nbat * cpr; e += LEVEL_THREADS)
+          Ast[e] = __ldg(reinterpret_cast<const uint4*>(Ag + (size_t)s_ptok[i0 + e / cpr] * r) + e % cpr);
+        sync();
+        for (int e = tid; e < nbat * NSn; e += LEVEL_THREADS) {
+          const int il = e / NSn, i = i0 + il, j = e % NSn;
+          float lg = -INFINITY, key = -INFINITY;
+          const int tok = s_stok[j];
+          if (tok >= 0) {
+            const uint4* arow = Ast + (size_t)il * cpr;
+            float dot = 0.f;
+            for (int k8 = 0; k8 < cpr; ++k8) {
+              float av[8];
+              unpack_bf16x8(arow[k8], av);
 #pragma unroll
-            for (int u = 0; u < 8; ++u) dot = fmaf(av[u], Wc[(size_t)j * r + k8 * 8 + u], dot);
+              for (int u = 0; u < 8; ++u) dot = fmaf(av[u], Wc[(size_t)j * rs + k8 * 8 + u], dot);
+            }
+            lg = s_sval[j] + dot;
+            key = lg;
+            if (a.T > 0.f) {
+              const uint4 cw = stream_words(a.seed, b, s_phash[i], STREAM_GUMBEL_COARSE, (uint32_t)tok >> 3);
+              const uint4 fw = stream_words(a.seed, b, s_phash[i], STREAM_GUMBEL_FINE, (uint32_t)tok >> 3);
+              const uint32_t c16 = (word_of(cw, (tok & 7) >> 1) >> (16 * (tok & 1))) & 0xFFFFu;
+              const uint32_t f16 = (word_of(fw, (tok & 7) >> 1) >> (16 * (tok & 1))) & 0xFFFFu;
+              key = lg * invT + gumbel_from_bits((c16 << 16) | f16);
+            }
           }
-          lg = s_sval[j] + dot;
-          key = lg;
-          if (a.T > 0.f) {
-            const uint4 cw = stream_words(a.seed, b, s_phash[i], STREAM_GUMBEL_COARSE, (uint32_t)tok >> 3);
-            const uint4 fw = stream_words(a.seed, b, s_phash[i], STREAM_GUMBEL_FINE, (uint32_t)tok >> 3);
-            const uint32_t c16 = (word_of(cw, (tok & 7) >> 1) >> (16 * (tok & 1))) & 0xFFFFu;
-            const uint32_t f16 = (word_of(fw, (tok & 7) >> 1) >> (16 * (tok & 1))) & 0xFFFFu;
-            key = lg * invT + gumbel_from_bits((c16 << 16) | f16);
-          }
+          res[2 * ((size_t)i * NSn + j)] = lg; res[2 * ((size_t)i * NSn + j) + 1] = key;
         }
-        res[2 * e] = lg; res[2 * e + 1] = key;
+        sync();
       }
-      sync();
       for (int e = tid; e < 2 * cnt; e += LEVEL_THREADS) a.thr0[(size_t)(e & 1) * a.cap + s_pli[e >> 1]] = 0u;   // no bound unless K finite values turn up
       sync();
       for (int e = tid; e < 2 * cnt * NSn; e += LEVEL_THREADS) {
