@@ -256,16 +256,37 @@ __device__ __forceinline__ void level_step(const ExpandArgs& a, const int d, con
       need = s_warp[1];
       sync();
     }
+    // the entries that tie with the threshold key (at least the one that defines it), gathered: they are ranked
+    // among themselves only, and only when there are more of them than places left
+    int* tie_list = s_new;   // (the list of placed slots is built in phase 3)
+    if (tid == 0) s_cnt[0] = 0;
+    sync();
+    for (int e = tid; e < M; e += LEVEL_THREADS) {
+      if (ent[e].depth >= 0 && skey(ent[e].key) == prefix) {
+        const int idx = atomicAdd(&s_cnt[0], 1);
+        if (idx < 256) tie_list[idx] = e;
+      }
+    }
+    sync();
+    const int ntie = s_cnt[0];
     for (int e = tid; e < M; e += LEVEL_THREADS) {
       const Entry x = ent[e];
       if (x.depth < 0) continue;
       const uint64_t k = skey(x.key);
       bool drop = k < prefix;
-      if (k == prefix) {
+      if (k == prefix && ntie > need) {
         int rank = 0;
-        for (int f = 0; f < M; ++f) {
-          const Entry y = ent[f];
-          if (y.depth >= 0 && f != e && skey(y.key) == prefix && before(y.key, y.depth, y.path, x.key, x.depth, x.path)) ++rank;
+        if (ntie <= 256) {
+          for (int t = 0; t < ntie; ++t) {
+            const int f = tie_list[t];
+            const Entry y = ent[f];
+            if (f != e && before(y.key, y.depth, y.path, x.key, x.depth, x.path)) ++rank;
+          }
+        } else {
+          for (int f = 0; f < M; ++f) {
+            const Entry y = ent[f];
+            if (y.depth >= 0 && f != e && skey(y.key) == prefix && before(y.key, y.depth, y.path, x.key, x.depth, x.path)) ++rank;
+          }
         }
         drop = rank >= need;
       }
@@ -291,35 +312,50 @@ __device__ __forceinline__ void level_step(const ExpandArgs& a, const int d, con
   }
   int nfree = 0;
   for (int w = 0; w < 8; ++w) nfree += s_warp[w];
-  for (int c0 = 0; c0 < ncand; c0 += LEVEL_THREADS) {
-    const int c = c0 + tid;
-    const size_t ci = cb + c;
-    const bool v = c < ncand && a.cd_valid[ci];
+  // Candidate c = it * LEVEL_THREADS + tid.  Pass 1: every thread notes which of its candidates survive (one bit
+  // per trip) and every warp leaves its count per trip; a prefix over (trip, warp) gives every warp's first
+  // place; pass 2 places.  (One trip at a time with the running total carried through shared memory cost four
+  // block barriers and a chain of loads per trip: 11 trips at the wide configuration, 100 us.)
+  const int ntrip = (ncand + LEVEL_THREADS - 1) / LEVEL_THREADS;   // <= Nmax * K / 256 <= 16
+  int* trip_cnt = s_pli;    // [ntrip][8] (phase 5 fills these arrays later)
+  int* trip_off = s_ptok;
+  unsigned vm = 0;
+  for (int it = 0; it < ntrip; ++it) {
+    const int c = it * LEVEL_THREADS + tid;
+    const bool v = c < ncand && a.cd_valid[cb + c];
     const unsigned bal = __ballot_sync(0xFFFFFFFFu, v);
-    sync();  // s_warp is reused
-    if (lane == 0) s_warp[warp] = __popc(bal);
-    sync();
-    int off = s_run;
-    for (int w = 0; w < warp; ++w) off += s_warp[w];
-    const int t = off + __popc(bal & ((1u << lane) - 1u));
-    if (v) {
-      if (t >= nfree) { a.status[b] = TS_ERR_OVERFLOW; }
-      else {
-        const int sl = s_free[t];
-        const int slot = a.cd_parent[ci];
-        const int x = a.cd_tok[ci];
-        a.pl_alive[pb + sl] = 1; a.pl_depth[pb + sl] = d + 1; a.pl_parent[pb + sl] = slot; a.pl_sib[pb + sl] = a.cd_sib[ci];
-        a.pl_tok[pb + sl] = x; a.pl_logkey[pb + sl] = a.cd_logkey[ci]; a.pl_logS[pb + sl] = a.cd_logS[ci];
-        a.pl_q0[pb + sl] = a.cd_q0[ci]; a.pl_logqT[pb + sl] = a.cd_logqT[ci]; a.pl_lseT[pb + sl] = nanf("");
-        a.pl_hash[pb + sl] = path_hash(slot < 0 ? 0ull : a.pl_hash[pb + slot], x);
-        a.pl_path[pb + sl] = (slot < 0 ? 0ull : a.pl_path[pb + slot]) | ((uint64_t)a.cd_sib[ci] << shift);
-        s_new[t] = sl;
-      }
-    }
-    sync();
-    if (tid == 0) { int tot = 0; for (int w = 0; w < 8; ++w) tot += s_warp[w]; s_run += tot; }
-    sync();
+    vm |= (v ? 1u : 0u) << it;
+    if (lane == 0) trip_cnt[it * 8 + warp] = __popc(bal);
   }
+  sync();
+  if (tid < ntrip * 8) {
+    int off = 0;
+    for (int e = 0; e < tid; ++e) off += trip_cnt[e];
+    trip_off[tid] = off;
+    if (tid == ntrip * 8 - 1) s_run = off + trip_cnt[tid];
+  }
+  if (ntrip == 0 && tid == 0) s_run = 0;
+  sync();
+  for (int it = 0; it < ntrip; ++it) {
+    const bool v = (vm >> it) & 1u;
+    const unsigned bal = __ballot_sync(0xFFFFFFFFu, v);
+    if (!v) continue;
+    const size_t ci = cb + (size_t)it * LEVEL_THREADS + tid;
+    const int t = trip_off[it * 8 + warp] + __popc(bal & ((1u << lane) - 1u));
+    if (t >= nfree) { a.status[b] = TS_ERR_OVERFLOW; }
+    else {
+      const int sl = s_free[t];
+      const int slot = a.cd_parent[ci];
+      const int x = a.cd_tok[ci];
+      a.pl_alive[pb + sl] = 1; a.pl_depth[pb + sl] = d + 1; a.pl_parent[pb + sl] = slot; a.pl_sib[pb + sl] = a.cd_sib[ci];
+      a.pl_tok[pb + sl] = x; a.pl_logkey[pb + sl] = a.cd_logkey[ci]; a.pl_logS[pb + sl] = a.cd_logS[ci];
+      a.pl_q0[pb + sl] = a.cd_q0[ci]; a.pl_logqT[pb + sl] = a.cd_logqT[ci]; a.pl_lseT[pb + sl] = nanf("");
+      a.pl_hash[pb + sl] = path_hash(slot < 0 ? 0ull : a.pl_hash[pb + slot], x);
+      a.pl_path[pb + sl] = (slot < 0 ? 0ull : a.pl_path[pb + slot]) | ((uint64_t)a.cd_sib[ci] << shift);
+      s_new[t] = sl;
+    }
+  }
+  sync();
   const int nnew = min(s_run, nfree);
   // ---- phase 4: next level's parents = new nodes that can still have admissible children -----------
   {
