@@ -18,8 +18,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     deps.append(os.path.join(os.path.dirname(HERE), "include", "treespark.h"))
     if not force and os.path.exists(LIB) and all(os.path.getmtime(LIB) >= os.path.getmtime(d) for d in deps):
         return LIB
-    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC", "-o", LIB] + srcs
+    cmd = ["nvcc", "--threads", "0", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "-shared", "-Xcompiler", "-fPIC", "-o", LIB] + srcs   # (--threads 0: the sources compile side by side)
     extra = os.environ.get("TS_NVCC_FLAGS", "").split()
     cmd[1:1] = extra
     if verbose:
