@@ -24,15 +24,15 @@ TREE_FLAGS = oracle.FLAG_NEAR_TOPK | oracle.FLAG_NEAR_THETA | oracle.FLAG_NEAR_C
 WALK_FLAGS = oracle.FLAG_NEAR_ACCEPT | oracle.FLAG_NEAR_CDF | oracle.FLAG_ZERO_MASS
 
 
-# Every compared round adds to these counts; when the scratch folder of a GPU run exists they are written there at
+# Every compared round adds to these counts; when TS_PARITY_REPORT_DIR names a folder they are written there at
 # exit, so that the exemption rates behind the tolerances can be read off a test run (tests still assert ceilings).
 PARITY_TOTALS = dict(trees=0, trees_exempt=0, walks=0, walks_exempt=0, accept_band_walks=0, accept_band_disagree=0)
 _BY_FLAG = {}
 
 
 def _dump_totals():
-    out = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-    if PARITY_TOTALS["trees"] and os.path.isdir(out):
+    out = os.environ.get("TS_PARITY_REPORT_DIR", "")
+    if PARITY_TOTALS["trees"] and out and os.path.isdir(out):
         with open(os.path.join(out, f"parity_exemptions_{os.getpid()}.json"), "w") as f:
             json.dump(dict(totals=PARITY_TOTALS, by_flag=_BY_FLAG), f)
 
