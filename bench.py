@@ -361,6 +361,8 @@ def run_ours(args, rank, world, device):
                    "launches_per_round": launches / max(args.steps, 1),
                    "parents_per_level": used[0]["parents_per_level"], "outputs_reproduced": same},
         "clocks": clocks, "gpu_launches": launches, "kernels": kern,
+        # the round's time in SM cycles (time x median SM clock under load): comparable across runs whose clocks differ
+        "mcycles_per_step": (ms_per_step * 1e-3 * clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None,
         # the per-kernel milliseconds come from a separate loop with an event pair around every launch (no chaining
         # of launches there): multiply them by this factor to read them as parts of the timed round
         "kernels_chained_scale": ms_per_step / tot_kernel_ms,
